@@ -1,0 +1,212 @@
+/*
+ * treelstm.h - C ABI of the B200 (sm_100a) binary TreeLSTM library.
+ *
+ * The library evaluates a binary TreeLSTM over a forest (a batch of differently shaped binary
+ * trees) by dependency-driven scheduling: every node whose children are finished is evaluated
+ * together with all other ready nodes of the whole forest, forward and backward through the
+ * tree structure.  Reference: "Improving the Expressiveness of Deep Learning Frameworks with
+ * Recursion" (arXiv 1809.00832); the passages each call follows are cited at the call.
+ *
+ * Conventions
+ *   - Every function returns an int: TREELSTM_OK (0) or a negative treelstm_status code.  No
+ *     function throws, aborts or traps.
+ *   - Unless a parameter is marked [host], array pointers are DEVICE pointers owned by the
+ *     caller (e.g. PyTorch tensors); the library never frees them.  Scalars are passed by value.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work
+ *     of a call is enqueued on that stream.
+ *   - Matrices are dense row-major, fp32, int32 indices.
+ *   - A forest of n_nodes nodes is three int32 arrays: left[n], right[n] (both -1 for a leaf,
+ *     both valid distinct node ids otherwise) and token[n] (vocabulary id of a leaf; ignored
+ *     for internal nodes).  Node ids may be in any order (no topological numbering needed,
+ *     Section 2.2); roots are the nodes that are nobody's child.
+ *   - The cell (the paper writes it only as LSTM(...), Figures 1 and 2; this is the standard
+ *     binary TreeLSTM):  in = [x ; h_l ; h_r],  z = W^T in + b  split into (i, f_l, f_r, o, u),
+ *     c = sig(i)*tanh(u) + sig(f_l)*c_l + sig(f_r)*c_r,  h = sig(o)*tanh(c);  x = emb[token] and
+ *     zero child state at a leaf, x = 0 at an internal node.
+ */
+#ifndef TREELSTM_H_
+#define TREELSTM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define TREELSTM_API __attribute__((visibility("default")))
+#else
+#define TREELSTM_API
+#endif
+
+typedef struct treelstm treelstm_t;
+
+typedef enum treelstm_status {
+  TREELSTM_OK = 0,
+  TREELSTM_ERR_INVALID_ARG = -1,        /* null pointer, non-positive size, workspace too small    */
+  TREELSTM_ERR_INVALID_FOREST = -2,     /* child out of range, single child, two parents, cycle     */
+  TREELSTM_ERR_TOKEN_OUT_OF_RANGE = -3, /* a leaf token outside [0, vocab)                          */
+  TREELSTM_ERR_LABEL_OUT_OF_RANGE = -4, /* a label outside [0, C)                                   */
+  TREELSTM_ERR_TIMEOUT = -5,            /* a bounded device-side wait expired                        */
+  TREELSTM_ERR_CUDA = -6,               /* a CUDA runtime call failed; see treelstm_last_cuda_error */
+  TREELSTM_ERR_NO_DEVICE = -7,          /* no sm_100 device is current                               */
+  TREELSTM_ERR_UNSUPPORTED = -8,        /* size outside what the kernels support                     */
+  TREELSTM_ERR_STATE = -9               /* call order violated (e.g. backward without forward)       */
+} treelstm_status;
+
+/* precision of the gate contraction */
+#define TREELSTM_FP32 0 /* fp32 operands, fp32 FMA accumulation, accurate activations            */
+#define TREELSTM_BF16 1 /* x, h_l, h_r, W rounded to bf16; tcgen05 tensor cores, fp32 accumulate; */
+                        /* bias, activations, c and the returned h stay fp32                      */
+
+/* flags of treelstm_forward (or-ed together) */
+#define TREELSTM_PER_LEVEL 0    /* one launch per wavefront; synchronises the stream once to read   */
+                                /* the level table, returns device-detected errors directly          */
+#define TREELSTM_PERSISTENT 1   /* one cooperative launch loops over the wavefronts with a bounded   */
+                                /* grid-wide barrier; fully asynchronous (see treelstm_status_sync)  */
+#define TREELSTM_SAVE_FOR_BACKWARD 2 /* keep every node's gate activations for treelstm_backward   */
+
+/* option keys of treelstm_set_option */
+#define TREELSTM_OPT_SCHED_SINGLE_CTA_MAX 1 /* forests up to this many nodes are scheduled by one  */
+                                            /* CTA in shared memory (0 forces the multi-CTA path)   */
+#define TREELSTM_OPT_WAIT_LIMIT_CYCLES 2    /* upper bound of every device-side wait, in units of   */
+                                            /* 1024 SM clock cycles                                  */
+#define TREELSTM_OPT_MAX_CTAS 3             /* cap on the persistent grid (0 = all co-resident CTAs) */
+
+/*
+ * treelstm_create - build a context for one set of parameters.
+ *   Model: Section 2.2 (TreeLSTM cells composed in the shape of the input tree).
+ *   H, E, vocab  hidden size, embedding size, vocabulary size (> 0).
+ *   emb          [vocab][E]   embedding table.
+ *   W            [E + 2H][5H] gate weights; rows [0,E) multiply x, [E,E+H) h_l, [E+H,E+2H) h_r;
+ *                column blocks of width H in the order i, f_l, f_r, o, u.
+ *   b            [5H]         gate bias, same column order.
+ *   precision    TREELSTM_FP32 or TREELSTM_BF16.
+ * The library copies (and for bf16 repacks, pads and converts) the parameters into device
+ * memory it owns; the caller may free or change its arrays after the call returns (the call
+ * synchronises `stream`).  *out is set to NULL on failure.  Release with treelstm_destroy.
+ */
+TREELSTM_API int treelstm_create(treelstm_t** out, int H, int E, int vocab, const float* emb, const float* W,
+                    const float* b, int precision, void* stream);
+
+/* Re-read emb, W, b (same shapes as at create) after the caller changed them. Synchronises. */
+TREELSTM_API int treelstm_update_weights(treelstm_t* ctx, const float* emb, const float* W, const float* b,
+                            void* stream);
+
+/*
+ * treelstm_set_classifier - per-node softmax classifier used by treelstm_backward
+ *   (Section 6.1: every node of every tree carries a label).
+ *   Wc [H][C], bc [C]; copied; synchronises `stream`.  1 <= C <= 32.
+ */
+TREELSTM_API int treelstm_set_classifier(treelstm_t* ctx, int C, const float* Wc, const float* bc, void* stream);
+
+TREELSTM_API int treelstm_set_option(treelstm_t* ctx, int key, long long value);
+
+/*
+ * treelstm_workspace_bytes - size of the caller-provided device scratch buffer that
+ * treelstm_forward (and, if with_backward != 0, treelstm_backward) needs for forests of up to
+ * max_nodes nodes.  Returns 0 on invalid arguments.  The buffer must be 256-byte aligned.
+ */
+TREELSTM_API size_t treelstm_workspace_bytes(const treelstm_t* ctx, int max_nodes, int with_backward);
+
+/*
+ * treelstm_forward - schedule the forest on the device and evaluate every node.
+ *   Schedule: Section 4.1.1 (an operation is ready once all its inputs are resolved; completed
+ *   operations release their dependants) and Section 4.1.2 (each invocation keeps a pointer to
+ *   its caller).  Evaluation: Figure 2 (Section 3.1), all ready nodes of the forest at once;
+ *   sibling subtrees are independent (Section 2.2).
+ *   n_nodes       number of nodes (>= 0; 0 is a no-op that reports 0 levels).
+ *   left,right,token  [n_nodes] the forest (see Conventions).
+ *   h, c          [n_nodes][H] out: state of every node, indexed by node id.
+ *   level         [n_nodes] out: wavefront of each node: 0 for a leaf, else
+ *                 1 + max(level of its children).
+ *   order         [n_nodes] out: node ids by ascending (level, node id) - the ready order.
+ *   level_offset  [n_nodes + 2] out or NULL: wavefront l is order[level_offset[l] ..
+ *                 level_offset[l+1]); entries past n_levels are unspecified.
+ *   n_levels      [1] out (device): number of wavefronts.
+ *   flags         TREELSTM_PER_LEVEL or TREELSTM_PERSISTENT, optionally | TREELSTM_SAVE_FOR_BACKWARD.
+ *   workspace     device scratch of at least treelstm_workspace_bytes(ctx, n_nodes, save) bytes;
+ *                 with TREELSTM_SAVE_FOR_BACKWARD it must stay untouched until backward is done.
+ * Errors: INVALID_ARG for bad arguments (nothing is launched).  A malformed forest or a token
+ * out of range is detected on the device: no out-of-bounds access happens, the outputs are
+ * unspecified, and the code is returned by this call (TREELSTM_PER_LEVEL) or by
+ * treelstm_status_sync (TREELSTM_PERSISTENT).
+ */
+TREELSTM_API int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const int32_t* right,
+                     const int32_t* token, float* h, float* c, int32_t* level, int32_t* order,
+                     int32_t* level_offset, int32_t* n_levels, int flags, void* workspace,
+                     size_t workspace_bytes, void* stream);
+
+/*
+ * treelstm_status_sync - wait for the stream of the last forward/backward call and return the
+ * status its kernels recorded (TREELSTM_OK, INVALID_FOREST, TOKEN/LABEL_OUT_OF_RANGE, TIMEOUT).
+ */
+TREELSTM_API int treelstm_status_sync(treelstm_t* ctx);
+
+/*
+ * treelstm_roots - after a forward on this context: the roots of the forest in ascending node
+ * id, with their states gathered (Figure 2: root_state = TreeLSTM(root_idx)).
+ *   root_ids [max_roots] out, root_h / root_c [max_roots][H] out (either may be NULL),
+ *   n_roots [1] out (device).  Roots beyond max_roots are dropped.  Enqueued on `stream`.
+ */
+TREELSTM_API int treelstm_roots(treelstm_t* ctx, int max_roots, int32_t* root_ids, float* root_h, float* root_c,
+                   int32_t* n_roots, void* stream);
+
+/*
+ * treelstm_backward - training step after treelstm_forward(... | TREELSTM_SAVE_FOR_BACKWARD) on
+ * the same context: mean softmax cross-entropy of the classifier on every node's h, and
+ * backpropagation through structure.
+ *   Section 4.2.2: the gradient computation recurses at the same positions as the forward
+ *   computation (here: wavefronts in reverse, parents before children); Sections 4.2.1 and 5:
+ *   each node instance uses its own retained forward values (here: dense per-node arrays, the
+ *   node id being the unique key).
+ *   labels       [n_nodes] class of every node, in [0, C).
+ *   loss         [1] out (device): mean over all nodes of -log softmax(Wc^T h_n + bc)[label_n].
+ *   dW [E+2H][5H], db [5H], dWc [H][C], dbc [C]  out: gradients (overwritten, not accumulated).
+ *   touched_ids  [n_leaves] out: sorted unique leaf tokens; dEmb_rows [n_leaves][E] out: one
+ *                summed gradient row per touched id (duplicates accumulate); n_touched [1] out.
+ *                Rows past n_touched are unspecified.
+ * The forest arrays, h, c, order, level and the workspace of the forward call must still be
+ * valid and unchanged.  Synchronises the stream once (to read the level table) unless the
+ * forward ran in TREELSTM_PER_LEVEL mode.  Computes in fp32 from the fp32 parameters whatever
+ * the forward precision.
+ */
+TREELSTM_API int treelstm_backward(treelstm_t* ctx, const int32_t* labels, float* loss, float* dW, float* db,
+                      float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,
+                      int32_t* n_touched, void* stream);
+
+/*
+ * treelstm_forward_host - the same forward for callers whose data lives in HOST memory: copies
+ * the forest to the device, runs treelstm_forward with `flags`, copies the requested results
+ * back and synchronises.  Device staging and workspace buffers are owned by the context and
+ * grown on demand (cudaMalloc on the first call or when n_nodes grows).
+ *   left,right,token [host][n_nodes] in (pinned memory makes the copies asynchronous).
+ *   h, c           [host][n_nodes][H] out, or NULL to skip the all-node states.
+ *   level, order   [host][n_nodes] out, or NULL.
+ *   max_roots, root_ids [host][max_roots], root_h, root_c [host][max_roots][H]: the roots in
+ *                  ascending node id with their states, or NULL; n_roots [host][1] out or NULL.
+ *   n_levels       [host][1] out or NULL.
+ * Returns the device status as well (it has synchronised).
+ */
+TREELSTM_API int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, const int32_t* right,
+                          const int32_t* token, float* h, float* c, int32_t* level, int32_t* order,
+                          int32_t* n_levels, int max_roots, int32_t* root_ids, float* root_h,
+                          float* root_c, int32_t* n_roots, int flags, void* stream);
+
+/* Number of kernels the last forward / backward call on this context launched. */
+TREELSTM_API int treelstm_last_launch_count(const treelstm_t* ctx);
+
+/* cudaError_t of the last failed CUDA call on this context (0 if none). */
+TREELSTM_API int treelstm_last_cuda_error(const treelstm_t* ctx);
+
+/* Frees everything the context owns.  NULL is allowed. */
+TREELSTM_API int treelstm_destroy(treelstm_t* ctx);
+
+/* Static description of a status code. */
+TREELSTM_API const char* treelstm_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TREELSTM_H_ */

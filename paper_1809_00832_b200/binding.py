@@ -1,0 +1,266 @@
+"""ctypes binding of libtreelstm_b200.so: the same calls as include/treelstm.h, with torch tensors
+standing in for the raw device pointers.  Argument marshalling only - every step of the path runs
+inside the library's CUDA kernels.  There is no CPU fallback: without the built library or
+without a CUDA device every call raises."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libtreelstm_b200.so")
+
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_INVALID_FOREST = -2
+ERR_TOKEN_OUT_OF_RANGE = -3
+ERR_LABEL_OUT_OF_RANGE = -4
+ERR_TIMEOUT = -5
+ERR_CUDA = -6
+ERR_NO_DEVICE = -7
+ERR_UNSUPPORTED = -8
+ERR_STATE = -9
+
+FP32 = 0
+BF16 = 1
+PER_LEVEL = 0
+PERSISTENT = 1
+SAVE_FOR_BACKWARD = 2
+OPT_SCHED_SINGLE_CTA_MAX = 1
+OPT_WAIT_LIMIT_CYCLES = 2
+OPT_MAX_CTAS = 3
+
+_vp = ctypes.c_void_p
+_i = ctypes.c_int
+
+# name -> (restype, argtypes); mirrors include/treelstm.h
+SIGNATURES = {
+    "treelstm_create": (_i, [ctypes.POINTER(_vp), _i, _i, _i, _vp, _vp, _vp, _i, _vp]),
+    "treelstm_update_weights": (_i, [_vp, _vp, _vp, _vp, _vp]),
+    "treelstm_set_classifier": (_i, [_vp, _i, _vp, _vp, _vp]),
+    "treelstm_set_option": (_i, [_vp, _i, ctypes.c_longlong]),
+    "treelstm_workspace_bytes": (ctypes.c_size_t, [_vp, _i, _i]),
+    "treelstm_forward": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp,
+                              ctypes.c_size_t, _vp]),
+    "treelstm_status_sync": (_i, [_vp]),
+    "treelstm_roots": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp]),
+    "treelstm_backward": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "treelstm_forward_host": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp,
+                                   _vp, _vp, _i, _vp]),
+    "treelstm_last_launch_count": (_i, [_vp]),
+    "treelstm_last_cuda_error": (_i, [_vp]),
+    "treelstm_destroy": (_i, [_vp]),
+    "treelstm_strerror": (ctypes.c_char_p, [_i]),
+}
+
+_lib = None
+
+
+class TreeLSTMError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = load_library().treelstm_strerror(code).decode()
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen the in-tree shared library and declare every prototype.  Raises if it is not built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_1809_00832_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    for name, (res, args) in SIGNATURES.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor of dtype {dtype}")
+    return t
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class TreeLSTM:
+    """Thin handle around a treelstm_t*.  Tensors are the caller's; the handle only keeps the
+    workspace it allocates through torch (device memory is PyTorch's job here)."""
+
+    def __init__(self, H: int, E: int, vocab: int, emb: torch.Tensor, W: torch.Tensor, b: torch.Tensor,
+                 precision: int = FP32):
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the TreeLSTM library has no CPU path")
+        self.lib = load_library()
+        self.H, self.E, self.vocab, self.precision = H, E, vocab, precision
+        self.C = 0
+        _dev(emb, torch.float32, "emb"); _dev(W, torch.float32, "W"); _dev(b, torch.float32, "b")
+        assert emb.shape == (vocab, E) and W.shape == (E + 2 * H, 5 * H) and b.shape == (5 * H,)
+        handle = ctypes.c_void_p()
+        rc = self.lib.treelstm_create(ctypes.byref(handle), H, E, vocab, _ptr(emb), _ptr(W), _ptr(b),
+                                      precision, _stream())
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_create")
+        self.handle = handle
+        self._ws: Optional[torch.Tensor] = None
+        self._keep = None
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.treelstm_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- parameters ---------------------------------------------------------------------------
+    def update_weights(self, emb, W, b):
+        rc = self.lib.treelstm_update_weights(self.handle, _ptr(emb), _ptr(W), _ptr(b), _stream())
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_update_weights")
+
+    def set_classifier(self, Wc: torch.Tensor, bc: torch.Tensor):
+        _dev(Wc, torch.float32, "Wc"); _dev(bc, torch.float32, "bc")
+        C = int(bc.shape[0])
+        assert Wc.shape == (self.H, C)
+        rc = self.lib.treelstm_set_classifier(self.handle, C, _ptr(Wc), _ptr(bc), _stream())
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_set_classifier")
+        self.C = C
+
+    def set_option(self, key: int, value: int):
+        rc = self.lib.treelstm_set_option(self.handle, key, value)
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_set_option")
+
+    def workspace_bytes(self, max_nodes: int, with_backward: bool) -> int:
+        return int(self.lib.treelstm_workspace_bytes(self.handle, max_nodes, int(with_backward)))
+
+    def _workspace(self, n: int, with_backward: bool) -> torch.Tensor:
+        need = self.workspace_bytes(n, with_backward)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need + 256, dtype=torch.uint8, device="cuda")
+        return self._ws
+
+    # -- forward ------------------------------------------------------------------------------
+    def forward(self, left: torch.Tensor, right: torch.Tensor, token: torch.Tensor, flags: int = PERSISTENT,
+                out: Optional[dict] = None, check: bool = True) -> dict:
+        """treelstm_forward.  Returns a dict of device tensors h, c, level, order, level_offset,
+        n_levels.  `out` lets the caller reuse the output tensors of an earlier call.  With
+        check=False the call stays asynchronous in persistent mode (status is not read)."""
+        n = int(left.shape[0])
+        for name, t in (("left", left), ("right", right), ("token", token)):
+            _dev(t, torch.int32, name)
+        if out is None:
+            out = dict(
+                h=torch.empty((n, self.H), dtype=torch.float32, device="cuda"),
+                c=torch.empty((n, self.H), dtype=torch.float32, device="cuda"),
+                level=torch.empty(n, dtype=torch.int32, device="cuda"),
+                order=torch.empty(n, dtype=torch.int32, device="cuda"),
+                level_offset=torch.empty(n + 2, dtype=torch.int32, device="cuda"),
+                n_levels=torch.zeros(1, dtype=torch.int32, device="cuda"),
+            )
+        ws = self._workspace(n, bool(flags & SAVE_FOR_BACKWARD))
+        base = ws.data_ptr()
+        aligned = (base + 255) // 256 * 256
+        rc = self.lib.treelstm_forward(self.handle, n, _ptr(left), _ptr(right), _ptr(token), _ptr(out["h"]),
+                                       _ptr(out["c"]), _ptr(out["level"]), _ptr(out["order"]),
+                                       _ptr(out["level_offset"]), _ptr(out["n_levels"]), flags,
+                                       ctypes.c_void_p(aligned), ws.numel() - (aligned - base), _stream())
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_forward")
+        self._keep = (left, right, token, out)
+        if check:
+            rc = self.lib.treelstm_status_sync(self.handle)
+            if rc != OK:
+                raise TreeLSTMError(rc, "treelstm_forward (device status)")
+        return out
+
+    def status_sync(self) -> int:
+        return int(self.lib.treelstm_status_sync(self.handle))
+
+    def roots(self, max_roots: int) -> dict:
+        out = dict(
+            root_ids=torch.empty(max_roots, dtype=torch.int32, device="cuda"),
+            root_h=torch.empty((max_roots, self.H), dtype=torch.float32, device="cuda"),
+            root_c=torch.empty((max_roots, self.H), dtype=torch.float32, device="cuda"),
+            n_roots=torch.zeros(1, dtype=torch.int32, device="cuda"),
+        )
+        rc = self.lib.treelstm_roots(self.handle, max_roots, _ptr(out["root_ids"]), _ptr(out["root_h"]),
+                                     _ptr(out["root_c"]), _ptr(out["n_roots"]), _stream())
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_roots")
+        return out
+
+    # -- backward -----------------------------------------------------------------------------
+    def backward(self, labels: torch.Tensor, n_leaves: int) -> dict:
+        """treelstm_backward after forward(..., flags | SAVE_FOR_BACKWARD)."""
+        _dev(labels, torch.int32, "labels")
+        H, E, C = self.H, self.E, self.C
+        f32 = dict(dtype=torch.float32, device="cuda")
+        out = dict(
+            loss=torch.zeros(1, **f32), dW=torch.empty((E + 2 * H, 5 * H), **f32), db=torch.empty(5 * H, **f32),
+            dWc=torch.empty((H, C), **f32), dbc=torch.empty(C, **f32),
+            touched_ids=torch.empty(max(n_leaves, 1), dtype=torch.int32, device="cuda"),
+            dEmb_rows=torch.empty((max(n_leaves, 1), E), **f32),
+            n_touched=torch.zeros(1, dtype=torch.int32, device="cuda"),
+        )
+        rc = self.lib.treelstm_backward(self.handle, _ptr(labels), _ptr(out["loss"]), _ptr(out["dW"]),
+                                        _ptr(out["db"]), _ptr(out["dWc"]), _ptr(out["dbc"]),
+                                        _ptr(out["touched_ids"]), _ptr(out["dEmb_rows"]),
+                                        _ptr(out["n_touched"]), _stream())
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_backward")
+        rc = self.lib.treelstm_status_sync(self.handle)
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_backward (device status)")
+        return out
+
+    # -- host-buffer forward ------------------------------------------------------------------
+    def forward_host(self, left: torch.Tensor, right: torch.Tensor, token: torch.Tensor, *, flags: int = PERSISTENT,
+                     all_states: bool = False, max_roots: int = 0, out: Optional[dict] = None) -> dict:
+        """treelstm_forward_host: host (ideally pinned) int32 tensors in, host tensors out."""
+        n = int(left.shape[0])
+        for t in (left, right, token):
+            if t.is_cuda or t.dtype != torch.int32 or not t.is_contiguous():
+                raise ValueError("forest arrays must be contiguous CPU int32 tensors")
+        if out is None:
+            pin = dict(pin_memory=True)
+            out = dict(n_levels=torch.zeros(1, dtype=torch.int32, **pin),
+                       n_roots=torch.zeros(1, dtype=torch.int32, **pin))
+            if all_states:
+                out["h"] = torch.empty((n, self.H), dtype=torch.float32, **pin)
+                out["c"] = torch.empty((n, self.H), dtype=torch.float32, **pin)
+                out["level"] = torch.empty(n, dtype=torch.int32, **pin)
+                out["order"] = torch.empty(n, dtype=torch.int32, **pin)
+            if max_roots > 0:
+                out["root_ids"] = torch.empty(max_roots, dtype=torch.int32, **pin)
+                out["root_h"] = torch.empty((max_roots, self.H), dtype=torch.float32, **pin)
+                out["root_c"] = torch.empty((max_roots, self.H), dtype=torch.float32, **pin)
+        g = out.get
+        rc = self.lib.treelstm_forward_host(self.handle, n, _ptr(left), _ptr(right), _ptr(token), _ptr(g("h")),
+                                            _ptr(g("c")), _ptr(g("level")), _ptr(g("order")), _ptr(g("n_levels")),
+                                            max_roots, _ptr(g("root_ids")), _ptr(g("root_h")), _ptr(g("root_c")),
+                                            _ptr(g("n_roots")), flags, _stream())
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_forward_host")
+        return out
+
+    def last_launch_count(self) -> int:
+        return int(self.lib.treelstm_last_launch_count(self.handle))

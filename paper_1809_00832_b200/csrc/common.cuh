@@ -1,0 +1,185 @@
+// Internal declarations shared by the translation units of libtreelstm_b200.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/treelstm.h"
+
+namespace tl {
+
+// Device-resident control block at the start of the caller's workspace.  Zeroed at the start
+// of every forward call.
+struct DevStatus {
+  int status;            // 0 or the most negative treelstm_status any kernel reported
+  int n_levels;          // number of wavefronts
+  int n_roots;           // number of trees
+  int max_level;         // scratch of the multi-CTA level assignment
+  unsigned int barrier;  // arrival counter of the persistent kernels' grid barrier
+  int n_touched;         // distinct leaf tokens (backward)
+  int pad[58];
+};
+static_assert(sizeof(DevStatus) == 256, "control block is one 256-byte line group");
+
+// Offsets (bytes) of the regions inside the workspace for a forest of up to n nodes.
+struct WsLayout {
+  size_t status, parent, pending, order_tmp, level_offset, roots, table, hb, gates, dh, dc, dz,
+      tok_slot, total;
+};
+
+struct Options {
+  int sched_single_cta_max = 49152;
+  long long wait_limit_kcycles = 1 << 20;  // ~1e9 cycles, about half a second at 2 GHz
+  int max_ctas = 0;
+};
+
+constexpr int kRadixBins = 256;
+constexpr int kRadixChunk = 1024;        // items per single-warp CTA of the multi-CTA sort
+constexpr int kSchedSingleMaxNodes = 49152;
+
+// Padded sizes of the tensor-core path: hidden units in groups of 8 (one packed weight group =
+// 5 gates x 8 units = 40 rows), K blocks of 64 bf16 (one 128-byte swizzle span).
+constexpr int kUnitGroup = 8;
+constexpr int kKBlock = 64;
+
+inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+inline size_t round_up_sz(size_t x, size_t m) { return (x + m - 1) / m * m; }
+
+}  // namespace tl
+
+// The context behind the opaque handle of the C ABI.
+struct treelstm {
+  int H = 0, E = 0, vocab = 0, precision = 0, C = 0;
+  int Hp = 0, Ep = 0;  // bf16 path: H padded to a multiple of 64, E padded to a multiple of 64
+  int device = 0;
+  int sm_count = 0;
+
+  // fp32 parameters (library-owned device copies)
+  float* emb = nullptr;  // [vocab][E]
+  float* W = nullptr;    // [E+2H][5H]
+  float* b = nullptr;    // [5H]
+  float* Wc = nullptr;   // [H][C]
+  float* bc = nullptr;   // [C]
+
+  // bf16 tensor-core path (library-owned)
+  __nv_bfloat16* emb_bf = nullptr;  // [vocab][Ep]
+  __nv_bfloat16* Wp_h = nullptr;    // [(Hp/8)*40][2*Hp]  packed recurrent weights, K contiguous
+  __nv_bfloat16* Wp_x = nullptr;    // [(Hp/8)*24][Ep]    packed input weights (gates i, o, u)
+  float* bp_h = nullptr;            // [(Hp/8)*40] bias in packed column order
+  float* bp_x = nullptr;            // [(Hp/8)*24]
+  CUtensorMap tmap_wh, tmap_wx;
+  bool have_tmaps = false;
+
+  tl::Options opt;
+
+  // what the last forward call saw (needed by roots / backward / status_sync)
+  struct Last {
+    bool valid = false;
+    int n = 0, flags = 0;
+    const int32_t *left = nullptr, *right = nullptr, *token = nullptr;
+    float *h = nullptr, *c = nullptr;
+    int32_t *level = nullptr, *order = nullptr, *level_offset = nullptr;
+    void* ws = nullptr;
+    tl::WsLayout lay{};
+    cudaStream_t stream = nullptr;
+    bool host_levels_valid = false;
+    int n_levels = 0;
+  } last;
+  int32_t* host_level_offset = nullptr;  // pinned, grows on demand
+  int host_level_cap = 0;
+  int* host_status = nullptr;            // pinned copy of DevStatus
+
+  // buffers of treelstm_forward_host (library-owned, grown on demand)
+  struct HostPath {
+    int cap_nodes = 0;
+    int32_t *left = nullptr, *right = nullptr, *token = nullptr, *level = nullptr, *order = nullptr,
+            *n_levels = nullptr, *root_ids = nullptr, *n_roots = nullptr;
+    float *h = nullptr, *c = nullptr, *root_h = nullptr, *root_c = nullptr;
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+  } hp;
+
+  int launches = 0;
+  int cuda_error = 0;
+};
+
+namespace tl {
+
+WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward);
+
+// schedule.cu: enqueue the on-device ready-set construction.  Returns a treelstm_status.
+int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
+                    const int32_t* token, int32_t* level, int32_t* order, int32_t* level_offset,
+                    void* ws, const WsLayout& lay, cudaStream_t stream);
+
+// cell_fp32.cu
+int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
+                        const int32_t* token, float* h, float* c, const int32_t* order,
+                        const int32_t* level_offset_dev, const int32_t* level_offset_host,
+                        int n_levels_host, int flags, void* ws, const WsLayout& lay,
+                        cudaStream_t stream);
+
+// gemm_tc.cu
+int pack_weights_bf16(treelstm* ctx, cudaStream_t stream);
+int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
+                        const int32_t* token, float* h, float* c, const int32_t* order,
+                        const int32_t* level_offset_dev, const int32_t* level_offset_host,
+                        int n_levels_host, int flags, void* ws, const WsLayout& lay,
+                        cudaStream_t stream);
+
+// backward.cu
+int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW, float* db,
+                    float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,
+                    int32_t* n_touched, cudaStream_t stream);
+
+// roots (schedule.cu)
+int launch_gather_roots(treelstm* ctx, int max_roots, int32_t* root_ids, float* root_h,
+                        float* root_c, int32_t* n_roots, cudaStream_t stream);
+
+#define TL_CUDA(ctx, expr)                                  \
+  do {                                                      \
+    cudaError_t e_ = (expr);                                \
+    if (e_ != cudaSuccess) {                                \
+      (ctx)->cuda_error = (int)e_;                          \
+      return TREELSTM_ERR_CUDA;                             \
+    }                                                       \
+  } while (0)
+
+#ifdef __CUDACC__
+// Record an error in the control block; the most negative code wins.
+__device__ __forceinline__ void report(DevStatus* st, int code) { atomicMin(&st->status, code); }
+
+__device__ __forceinline__ int ld_volatile(const int* p) { return *(const volatile int*)p; }
+
+// Bounded grid-wide barrier for cooperative (co-resident) launches.  `target` is the total
+// number of arrivals expected so far (gridDim.x * number of barriers passed, this one included).
+// Returns false if the wait expired or another CTA reported an error: the caller must then
+// leave its level loop (every CTA sees the same outcome within one more barrier).
+__device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
+                                             long long limit_cycles, int* s_flag) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(&st->barrier, 1u);
+    long long t0 = clock64();
+    int ok = 1;
+    while (*(volatile unsigned int*)&st->barrier < target) {
+      if (*(volatile int*)&st->status != 0) { ok = 0; break; }
+      if (clock64() - t0 > limit_cycles) {
+        report(st, TREELSTM_ERR_TIMEOUT);
+        ok = 0;
+        break;
+      }
+      __nanosleep(32);
+    }
+    __threadfence();
+    *s_flag = ok;
+  }
+  __syncthreads();
+  return *s_flag != 0;
+}
+#endif
+
+}  // namespace tl

@@ -1,0 +1,467 @@
+// On-device ready-set construction for a forest given as child-index arrays.
+//
+// Paper, Section 4.1.1: an operation with no unresolved input is ready; when an operation
+// completes, the operations that waited on it and have all inputs resolved become ready.  For a
+// tree node this gives wavefront ("level") 0 for leaves and 1 + max(level of children) for
+// internal nodes.  Section 4.1.2: every invocation keeps a pointer to its caller -> parent[].
+// The ready order reported to the caller is canonical: ascending (level, node id).
+//
+// Two implementations produce identical arrays:
+//   * k_schedule_single: one CTA, levels in shared memory, for forests up to 49152 nodes;
+//   * a multi-CTA path (dependency counters walked up from the leaves, LSD radix sort with
+//     per-chunk histograms) for anything larger.
+#include "common.cuh"
+
+namespace tl {
+namespace {
+
+constexpr int kSingleThreads = 1024;
+constexpr int kSingleWarps = kSingleThreads / 32;
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ unsigned lanemask_lt() {
+  unsigned m;
+  asm volatile("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+
+// Node check shared by both paths.  Returns 0, or the error code.  is_leaf is set for valid nodes.
+__device__ __forceinline__ int check_node(int n, int k, int l, int r, const int* token, int vocab,
+                                          bool* is_leaf) {
+  if (l < 0 && r < 0) {
+    *is_leaf = true;
+    if (l != -1 || r != -1) return TREELSTM_ERR_INVALID_FOREST;
+    int t = token[k];
+    if (t < 0 || t >= vocab) return TREELSTM_ERR_TOKEN_OUT_OF_RANGE;
+    return 0;
+  }
+  *is_leaf = false;
+  if (l < 0 || r < 0 || l >= n || r >= n || l == r || l == k || r == k)
+    return TREELSTM_ERR_INVALID_FOREST;
+  return 0;
+}
+
+// ------------------------------------------------------------------------------------------ //
+// Stable counting pass executed by one CTA of 32 warps over `n` items.
+// Item r of the source sequence is src ? src[r] : r.  key(item) in [0, 256).  Items are written
+// to dst ordered by key, ties in source order.  hist is shared memory [256][32] ints.
+// After the scan step, *bin1_start (if non-null) receives the number of items with key 0.
+// ------------------------------------------------------------------------------------------ //
+template <class KeyFn>
+__device__ void block_counting_pass(int n, const int* src, int* dst, KeyFn key, int* hist,
+                                    int* scan_tmp, int* bin1_start) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int i = tid; i < kRadixBins * kSingleWarps; i += kSingleThreads) hist[i] = 0;
+  __syncthreads();
+  int per_warp = (n + kSingleWarps - 1) / kSingleWarps;
+  per_warp = (per_warp + 31) & ~31;
+  const int begin = min(n, warp * per_warp), end = min(n, begin + per_warp);
+  for (int r = begin + lane; r < end; r += 32) {
+    int item = src ? src[r] : r;
+    atomicAdd(&hist[key(item) * kSingleWarps + warp], 1);
+  }
+  __syncthreads();
+  // exclusive scan of hist in (bin-major, warp-minor) order: 8 consecutive entries per thread
+  {
+    constexpr int kPer = kRadixBins * kSingleWarps / kSingleThreads;  // 8
+    int v[kPer], sum = 0;
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) { v[j] = hist[tid * kPer + j]; sum += v[j]; }
+    int incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      int t = __shfl_up_sync(kFull, incl, d);
+      if (lane >= d) incl += t;
+    }
+    if (lane == 31) scan_tmp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = scan_tmp[lane], wi = w;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        int t = __shfl_up_sync(kFull, wi, d);
+        if (lane >= d) wi += t;
+      }
+      scan_tmp[lane] = wi - w;
+    }
+    __syncthreads();
+    int run = scan_tmp[warp] + incl - sum;
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) { hist[tid * kPer + j] = run; run += v[j]; }
+  }
+  __syncthreads();
+  if (bin1_start && tid == 0) *bin1_start = hist[1 * kSingleWarps + 0];
+  __syncthreads();
+  for (int r0 = begin; r0 < end; r0 += 32) {
+    const int r = r0 + lane;
+    const bool valid = r < end;
+    const unsigned act = __ballot_sync(kFull, valid);
+    int item = 0, k = 0, base = 0;
+    unsigned peers = 0;
+    if (valid) {
+      item = src ? src[r] : r;
+      k = key(item);
+      peers = __match_any_sync(act, k);
+      base = hist[k * kSingleWarps + warp];
+    }
+    __syncwarp();
+    if (valid && lane == __ffs(peers) - 1) hist[k * kSingleWarps + warp] = base + __popc(peers);
+    __syncwarp();
+    if (valid) dst[base + __popc(peers & lanemask_lt())] = item;
+  }
+  __syncthreads();
+}
+
+// One CTA schedules the whole forest.  Dynamic shared memory: uint16 level[n] | int hist[256*32].
+__global__ void __launch_bounds__(kSingleThreads, 1)
+k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ right,
+                  const int* __restrict__ token, int vocab, int* parent, int* level, int* order,
+                  int* order_tmp, int* level_offset, int* roots, DevStatus* st) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  unsigned short* lv = reinterpret_cast<unsigned short*>(smem);
+  int* hist = reinterpret_cast<int*>(smem + (((size_t)n * 2 + 15) & ~(size_t)15));
+  __shared__ int scan_tmp[32];
+  __shared__ int s_err, s_maxlevel;
+  const int tid = threadIdx.x;
+  constexpr unsigned short kNone = 0xFFFF;
+  if (tid == 0) { s_err = 0; s_maxlevel = 0; }
+  for (int k = tid; k < n; k += kSingleThreads) parent[k] = -1;
+  __syncthreads();
+  // validate, link children to their caller, leaves are ready at once
+  for (int k = tid; k < n; k += kSingleThreads) {
+    const int l = left[k], r = right[k];
+    bool leaf;
+    int err = check_node(n, k, l, r, token, vocab, &leaf);
+    if (err == 0 && !leaf) {
+      if (atomicCAS(&parent[l], -1, k) != -1) err = TREELSTM_ERR_INVALID_FOREST;
+      if (atomicCAS(&parent[r], -1, k) != -1) err = TREELSTM_ERR_INVALID_FOREST;
+    }
+    if (err) atomicMin(&s_err, err);
+    lv[k] = (err == 0 && leaf) ? 0 : kNone;
+  }
+  __syncthreads();
+  if (s_err != 0) {
+    if (tid == 0) { report(st, s_err); st->n_levels = 0; st->n_roots = 0; }
+    return;
+  }
+  // relaxation rounds: a node whose children both have a level takes 1 + max.  A level, once
+  // written, is final, so reading a value written in the same round is harmless.
+  int local_max = 0;
+  for (int round = 0; round <= n; ++round) {
+    int progress = 0, waiting = 0;
+    for (int k = tid; k < n; k += kSingleThreads) {
+      if (lv[k] != kNone) continue;
+      const unsigned short a = lv[left[k]], b = lv[right[k]];
+      if (a != kNone && b != kNone) {
+        const int v = 1 + max((int)a, (int)b);
+        lv[k] = (unsigned short)v;
+        local_max = max(local_max, v);
+        progress = 1;
+      } else {
+        waiting = 1;
+      }
+    }
+    const int any_progress = __syncthreads_or(progress);
+    const int any_waiting = __syncthreads_or(waiting);
+    if (!any_waiting) break;
+    if (!any_progress) {  // nodes on a cycle never become ready
+      if (tid == 0) { report(st, TREELSTM_ERR_INVALID_FOREST); st->n_levels = 0; st->n_roots = 0; }
+      return;
+    }
+  }
+  atomicMax(&s_maxlevel, local_max);
+  for (int k = tid; k < n; k += kSingleThreads) level[k] = lv[k];
+  __syncthreads();
+  const int n_levels = n > 0 ? s_maxlevel + 1 : 0;
+  if (tid == 0) st->n_levels = n_levels;
+  // canonical ready order: LSD radix on the level, 8 bits per pass, ties by node id
+  int passes = 1;
+  while (passes < 4 && (n_levels - 1) >> (8 * passes)) ++passes;
+  for (int p = 0; p < passes; ++p) {
+    int* dst = ((passes - 1 - p) & 1) ? order_tmp : order;
+    const int* src = p == 0 ? nullptr : (dst == order ? order_tmp : order);
+    const int shift = 8 * p;
+    block_counting_pass(n, src, dst, [=](int item) { return ((int)lv[item] >> shift) & 255; },
+                        hist, scan_tmp, nullptr);
+  }
+  // wavefront boundaries
+  for (int r = tid; r < n; r += kSingleThreads) {
+    const int a = lv[order[r]];
+    if (r == 0 || (int)lv[order[r - 1]] != a) level_offset[a] = r;
+  }
+  if (tid == 0) level_offset[n_levels] = n;
+  // roots in ascending node id: stable partition on "has a caller"
+  block_counting_pass(n, nullptr, roots, [=](int item) { return parent[item] >= 0 ? 1 : 0; }, hist,
+                      scan_tmp, &st->n_roots);
+}
+
+// ------------------------------------------------------------------------------------------ //
+// multi-CTA path
+// ------------------------------------------------------------------------------------------ //
+__global__ void k_sched_init(int n, const int* __restrict__ left, const int* __restrict__ right,
+                             const int* __restrict__ token, int vocab, int* parent, int* level,
+                             DevStatus* st) {
+  // parent[] was set to -1 and pending[] to 0 by memsets enqueued before this kernel
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= n) return;
+  const int l = left[k], r = right[k];
+  bool leaf;
+  int err = check_node(n, k, l, r, token, vocab, &leaf);
+  if (err == 0 && !leaf) {
+    if (atomicCAS(&parent[l], -1, k) != -1) err = TREELSTM_ERR_INVALID_FOREST;
+    if (atomicCAS(&parent[r], -1, k) != -1) err = TREELSTM_ERR_INVALID_FOREST;
+  }
+  if (err) report(st, err);
+  level[k] = (err == 0 && leaf) ? 0 : -1;
+}
+
+// Dependency counters: every leaf walks towards its root; at each caller the first child to
+// arrive stops, the second one knows both children are resolved, assigns the level and goes on.
+__global__ void k_sched_walkup(int n, const int* __restrict__ left, const int* __restrict__ right,
+                               const int* parent, int* pending, int* level, DevStatus* st) {
+  if (ld_volatile(&st->status) != 0) return;
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= n || left[k] >= 0) return;
+  int cur = k, lvl = 0;
+  for (int step = 0; step < n; ++step) {  // a path has fewer than n edges
+    const int p = parent[cur];
+    if (p < 0) break;
+    __threadfence();
+    if (atomicAdd(&pending[p], 1) == 0) return;  // sibling subtree still running
+    __threadfence();
+    const int sib = left[p] == cur ? right[p] : left[p];
+    lvl = 1 + max(lvl, ld_volatile(&level[sib]));
+    *(volatile int*)&level[p] = lvl;
+    cur = p;
+  }
+  atomicMax(&st->max_level, lvl);
+}
+
+__global__ void k_sched_check(int n, const int* level, DevStatus* st) {
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k == 0 && st->status == 0) st->n_levels = n > 0 ? st->max_level + 1 : 0;
+  if (k < n && level[k] < 0) report(st, TREELSTM_ERR_INVALID_FOREST);  // cycle
+}
+
+// mode 0: key = digit `pass` of level; mode 1: key = has-a-caller flag.
+__device__ __forceinline__ int sort_key(int mode, int pass, int item, const int* level,
+                                        const int* parent) {
+  return mode == 0 ? ((level[item] >> (8 * pass)) & 255) : (parent[item] >= 0 ? 1 : 0);
+}
+
+__device__ __forceinline__ int passes_needed(int n_levels) {
+  int passes = 1;
+  while (passes < 4 && (n_levels - 1) >> (8 * passes)) ++passes;
+  return passes;
+}
+
+// Which buffer pass p reads and writes, so that the last needed pass lands in `order`.
+__device__ __forceinline__ void pass_buffers(int mode, int pass, int passes, int* order,
+                                             int* order_tmp, int* roots, const int** src,
+                                             int** dst) {
+  if (mode == 1) { *src = nullptr; *dst = roots; return; }
+  *dst = ((passes - 1 - pass) & 1) ? order_tmp : order;
+  *src = pass == 0 ? nullptr : (*dst == order ? order_tmp : order);
+}
+
+// One warp per CTA, chunk of kRadixChunk consecutive source items; table is [256][n_chunks].
+__global__ void __launch_bounds__(32)
+k_radix_hist(int n, int mode, int pass, const int* level, const int* parent, int* order,
+             int* order_tmp, int* roots, int* table, int n_chunks, const DevStatus* st) {
+  if (st->status != 0) return;
+  const int passes = mode == 0 ? passes_needed(st->n_levels) : 1;
+  if (pass >= passes) return;
+  __shared__ int hist[kRadixBins];
+  const int lane = threadIdx.x, chunk = blockIdx.x;
+  for (int i = lane; i < kRadixBins; i += 32) hist[i] = 0;
+  __syncwarp();
+  const int* src; int* dst;
+  pass_buffers(mode, pass, passes, order, order_tmp, roots, &src, &dst);
+  const int begin = chunk * kRadixChunk, end = min(n, begin + kRadixChunk);
+  for (int r = begin + lane; r < end; r += 32) {
+    const int item = src ? src[r] : r;
+    atomicAdd(&hist[sort_key(mode, pass, item, level, parent)], 1);
+  }
+  __syncwarp();
+  for (int i = lane; i < kRadixBins; i += 32) table[(size_t)i * n_chunks + chunk] = hist[i];
+}
+
+// Exclusive scan of the whole table by one CTA.
+__global__ void __launch_bounds__(1024)
+k_radix_scan(int mode, int pass, int* table, int n_chunks, DevStatus* st) {
+  if (st->status != 0) return;
+  const int passes = mode == 0 ? passes_needed(st->n_levels) : 1;
+  if (pass >= passes) return;
+  __shared__ int warp_sum[32];
+  __shared__ int carry;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long total = (long long)kRadixBins * n_chunks;
+  if (tid == 0) carry = 0;
+  __syncthreads();
+  for (long long base = 0; base < total; base += 1024) {
+    const long long i = base + tid;
+    const int v = i < total ? table[i] : 0;
+    int incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      int t = __shfl_up_sync(kFull, incl, d);
+      if (lane >= d) incl += t;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = warp_sum[lane], wi = w;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        int t = __shfl_up_sync(kFull, wi, d);
+        if (lane >= d) wi += t;
+      }
+      warp_sum[lane] = wi - w;
+    }
+    __syncthreads();
+    const int excl = carry + warp_sum[warp] + incl - v;
+    if (i < total) table[i] = excl;
+    if (mode == 1 && i == (long long)n_chunks) st->n_roots = excl;  // start of bin 1
+    __syncthreads();
+    if (tid == 1023) carry = excl + v;
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(32)
+k_radix_scatter(int n, int mode, int pass, const int* level, const int* parent, int* order,
+                int* order_tmp, int* roots, const int* table, int n_chunks, const DevStatus* st) {
+  if (st->status != 0) return;
+  const int passes = mode == 0 ? passes_needed(st->n_levels) : 1;
+  if (pass >= passes) return;
+  __shared__ int base_of[kRadixBins];
+  const int lane = threadIdx.x, chunk = blockIdx.x;
+  for (int i = lane; i < kRadixBins; i += 32) base_of[i] = table[(size_t)i * n_chunks + chunk];
+  __syncwarp();
+  const int* src; int* dst;
+  pass_buffers(mode, pass, passes, order, order_tmp, roots, &src, &dst);
+  const int begin = chunk * kRadixChunk, end = min(n, begin + kRadixChunk);
+  for (int r0 = begin; r0 < end; r0 += 32) {
+    const int r = r0 + lane;
+    const bool valid = r < end;
+    const unsigned act = __ballot_sync(kFull, valid);
+    int item = 0, k = 0, base = 0;
+    unsigned peers = 0;
+    if (valid) {
+      item = src ? src[r] : r;
+      k = sort_key(mode, pass, item, level, parent);
+      peers = __match_any_sync(act, k);
+      base = base_of[k];
+    }
+    __syncwarp();
+    if (valid && lane == __ffs(peers) - 1) base_of[k] = base + __popc(peers);
+    __syncwarp();
+    if (valid) dst[base + __popc(peers & lanemask_lt())] = item;
+  }
+}
+
+__global__ void k_sched_offsets(int n, const int* level, const int* order, int* level_offset,
+                                const DevStatus* st) {
+  if (st->status != 0) return;
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r == 0) level_offset[st->n_levels] = n;
+  if (r >= n) return;
+  const int a = level[order[r]];
+  if (r == 0 || level[order[r - 1]] != a) level_offset[a] = r;
+}
+
+__global__ void k_gather_roots(int max_roots, int H, const int* roots, const float* h,
+                               const float* c, int* root_ids, float* root_h, float* root_c,
+                               int* n_roots_out, const DevStatus* st) {
+  const int n_roots = st->status == 0 ? min(st->n_roots, max_roots) : 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0 && n_roots_out) *n_roots_out = n_roots;
+  for (int t = blockIdx.x; t < n_roots; t += gridDim.x) {
+    const int node = roots[t];
+    if (threadIdx.x == 0 && root_ids) root_ids[t] = node;
+    for (int j = threadIdx.x; j < H; j += blockDim.x) {
+      if (root_h) root_h[(size_t)t * H + j] = h[(size_t)node * H + j];
+      if (root_c) root_c[(size_t)t * H + j] = c[(size_t)node * H + j];
+    }
+  }
+}
+
+}  // namespace
+
+int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
+                    const int32_t* token, int32_t* level, int32_t* order, int32_t* level_offset,
+                    void* ws, const WsLayout& lay, cudaStream_t stream) {
+  char* base = static_cast<char*>(ws);
+  DevStatus* st = reinterpret_cast<DevStatus*>(base + lay.status);
+  int* parent = reinterpret_cast<int*>(base + lay.parent);
+  int* pending = reinterpret_cast<int*>(base + lay.pending);
+  int* order_tmp = reinterpret_cast<int*>(base + lay.order_tmp);
+  int* roots = reinterpret_cast<int*>(base + lay.roots);
+  int* table = reinterpret_cast<int*>(base + lay.table);
+  if (n == 0) return TREELSTM_OK;  // control block already zero: 0 levels, 0 roots
+
+  const int single_max = ctx->opt.sched_single_cta_max < kSchedSingleMaxNodes
+                             ? ctx->opt.sched_single_cta_max : kSchedSingleMaxNodes;
+  if (n <= single_max) {
+    const size_t smem = round_up_sz((size_t)n * 2, 16) + sizeof(int) * kRadixBins * kSingleWarps;
+    static bool attr_set = false;
+    if (!attr_set) {
+      TL_CUDA(ctx, cudaFuncSetAttribute(k_schedule_single,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(round_up_sz((size_t)kSchedSingleMaxNodes * 2, 16) +
+                                              sizeof(int) * kRadixBins * kSingleWarps)));
+      attr_set = true;
+    }
+    k_schedule_single<<<1, kSingleThreads, smem, stream>>>(n, left, right, token, ctx->vocab, parent,
+                                                           level, order, order_tmp, level_offset,
+                                                           roots, st);
+    ctx->launches += 1;
+    TL_CUDA(ctx, cudaGetLastError());
+    return TREELSTM_OK;
+  }
+
+  TL_CUDA(ctx, cudaMemsetAsync(parent, 0xFF, sizeof(int) * (size_t)n, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(pending, 0, sizeof(int) * (size_t)n, stream));
+  const int tpb = 256, blocks = (n + tpb - 1) / tpb;
+  k_sched_init<<<blocks, tpb, 0, stream>>>(n, left, right, token, ctx->vocab, parent, level, st);
+  k_sched_walkup<<<blocks, tpb, 0, stream>>>(n, left, right, parent, pending, level, st);
+  k_sched_check<<<blocks, tpb, 0, stream>>>(n, level, st);
+  ctx->launches += 3;
+  const int n_chunks = (n + kRadixChunk - 1) / kRadixChunk;
+  // a forest of n nodes has at most (n + 1) / 2 levels; later passes switch themselves off on
+  // the device once the actual level count is known
+  int host_passes = 1;
+  while (host_passes < 4 && (((n + 1) / 2 - 1) >> (8 * host_passes))) ++host_passes;
+  for (int p = 0; p < host_passes; ++p) {
+    k_radix_hist<<<n_chunks, 32, 0, stream>>>(n, 0, p, level, parent, order, order_tmp, roots, table,
+                                              n_chunks, st);
+    k_radix_scan<<<1, 1024, 0, stream>>>(0, p, table, n_chunks, st);
+    k_radix_scatter<<<n_chunks, 32, 0, stream>>>(n, 0, p, level, parent, order, order_tmp, roots,
+                                                 table, n_chunks, st);
+    ctx->launches += 3;
+  }
+  k_sched_offsets<<<blocks, tpb, 0, stream>>>(n, level, order, level_offset, st);
+  k_radix_hist<<<n_chunks, 32, 0, stream>>>(n, 1, 0, level, parent, order, order_tmp, roots, table,
+                                            n_chunks, st);
+  k_radix_scan<<<1, 1024, 0, stream>>>(1, 0, table, n_chunks, st);
+  k_radix_scatter<<<n_chunks, 32, 0, stream>>>(n, 1, 0, level, parent, order, order_tmp, roots,
+                                               table, n_chunks, st);
+  ctx->launches += 4;
+  TL_CUDA(ctx, cudaGetLastError());
+  return TREELSTM_OK;
+}
+
+int launch_gather_roots(treelstm* ctx, int max_roots, int32_t* root_ids, float* root_h,
+                        float* root_c, int32_t* n_roots, cudaStream_t stream) {
+  const auto& L = ctx->last;
+  char* base = static_cast<char*>(L.ws);
+  const DevStatus* st = reinterpret_cast<const DevStatus*>(base + L.lay.status);
+  const int* roots = reinterpret_cast<const int*>(base + L.lay.roots);
+  int blocks = max_roots < 1 ? 1 : (max_roots < 1184 ? max_roots : 1184);
+  k_gather_roots<<<blocks, 128, 0, stream>>>(max_roots, ctx->H, roots, L.h, L.c, root_ids, root_h,
+                                             root_c, n_roots, st);
+  ctx->launches += 1;
+  TL_CUDA(ctx, cudaGetLastError());
+  return TREELSTM_OK;
+}
+
+}  // namespace tl
