@@ -1,5 +1,373 @@
+// Training step: per-node softmax classifier + mean cross-entropy, then backpropagation through
+// structure over the wavefronts in reverse (parents before children).
+//
+// Paper, Section 4.2.2: the gradient computation recurses at the same positions as the forward
+// computation; Sections 4.2.1 / 5: a gradient operation needs the previous gradient and the
+// forward values of its own node instance.  Here those values live in dense per-node arrays
+// (gates, c, h) indexed by node id, so no lookup structure is needed and nothing can be routed
+// to the wrong instance.
+//
+//   dh_n  = Wc (p_n - e_y)/N + [dIn from the caller]          dc_n = dc_caller*f + dh_n o (1 - tanh^2 c)
+//   dz_o = dh tanh(c) o(1-o)   dz_i = dc u i(1-i)   dz_u = dc i (1-u^2)   dz_f* = dc c_* f*(1-f*)
+//   dIn  = W dz  (rows [0,E): embedding row of a leaf; rows [E,E+2H): dh of the two children)
+//   dW   = sum_n in_n (x) dz_n,   db = sum_n dz_n
 #include "common.cuh"
+
 namespace tl {
-int launch_backward(treelstm*, const int32_t*, float*, float*, float*, float*, float*, int32_t*, float*,
-                    int32_t*, cudaStream_t) { return TREELSTM_ERR_UNSUPPORTED; }
+
+int ensure_host_levels(treelstm* ctx);  // api.cu
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+struct BwdParams {
+  int n, H, E, C, vocab, n_leaves;
+  const int *left, *right, *token, *order, *labels;
+  const float *emb, *W, *Wc, *bc, *h, *c, *gates;
+  float *dh, *dc, *dz;
+  float *loss, *dW, *db, *dWc, *dbc, *dEmb_rows;
+  int *tok_slot, *touched_ids, *n_touched;
+  DevStatus* st;
+};
+
+// ---- touched embedding rows: flag, scan, compact ------------------------------------------- //
+__global__ void k_bwd_mark_tokens(BwdParams p) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= p.n_leaves) return;
+  p.tok_slot[p.token[p.order[r]]] = 1;  // level 0 occupies order[0 .. n_leaves)
 }
+
+// Exclusive scan of the flags over the vocabulary by one CTA; flagged ids are emitted in
+// ascending order and tok_slot[id] becomes the row index of id in dEmb_rows.
+__global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) {
+  __shared__ int warp_sum[32];
+  __shared__ int carry;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) carry = 0;
+  __syncthreads();
+  for (int base = 0; base < p.vocab; base += 1024) {
+    const int i = base + tid;
+    const int v = i < p.vocab ? p.tok_slot[i] : 0;
+    int incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      int t = __shfl_up_sync(kFull, incl, d);
+      if (lane >= d) incl += t;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = warp_sum[lane], wi = w;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        int t = __shfl_up_sync(kFull, wi, d);
+        if (lane >= d) wi += t;
+      }
+      warp_sum[lane] = wi - w;
+    }
+    __syncthreads();
+    const int excl = carry + warp_sum[warp] + incl - v;
+    if (i < p.vocab) {
+      p.tok_slot[i] = excl;
+      if (v) p.touched_ids[excl] = i;
+    }
+    __syncthreads();
+    if (tid == 1023) carry = excl + v;
+    __syncthreads();
+  }
+  if (tid == 0) { *p.n_touched = carry; p.st->n_touched = carry; }
+}
+
+// ---- classifier: logits, softmax, loss, dlogits, dh (classifier part), dWc, dbc -------------- //
+// One warp per node; lane k owns class k (C <= 32).
+constexpr int kClsWarps = 8;
+constexpr int kClsNodesPerCta = 64;
+
+__global__ void __launch_bounds__(kClsWarps * 32) k_bwd_classifier(BwdParams p) {
+  extern __shared__ float s_dWc[];  // [H][C] + [C], CTA-local partial sums
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int H = p.H, C = p.C;
+  for (int i = tid; i < H * C + C; i += blockDim.x) s_dWc[i] = 0.f;
+  __syncthreads();
+  const int node0 = blockIdx.x * kClsNodesPerCta;
+  const float inv_n = 1.0f / (float)p.n;
+  for (int q = warp; q < kClsNodesPerCta; q += kClsWarps) {
+    const int node = node0 + q;
+    if (node >= p.n) break;
+    const float* hn = p.h + (size_t)node * H;
+    float logit = -INFINITY;
+    if (lane < C) {
+      float acc = p.bc[lane];
+      for (int j = 0; j < H; ++j) acc = fmaf(hn[j], p.Wc[j * C + lane], acc);
+      logit = acc;
+    }
+    float m = logit;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, d));
+    float e = lane < C ? expf(logit - m) : 0.f, sum = e;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(kFull, sum, d);
+    const int y = p.labels[node];
+    const bool y_ok = y >= 0 && y < C;
+    if (!y_ok && lane == 0) report(p.st, TREELSTM_ERR_LABEL_OUT_OF_RANGE);
+    const float lse = m + logf(sum);
+    const float logit_y = __shfl_sync(kFull, logit, y_ok ? y : 0);
+    if (lane == 0 && y_ok) atomicAdd(p.loss, (lse - logit_y) * inv_n);
+    const float dlogit = lane < C ? (e / sum - (lane == y ? 1.f : 0.f)) * inv_n : 0.f;
+    if (lane < C) atomicAdd(&s_dWc[H * C + lane], dlogit);
+    for (int j0 = 0; j0 < H; j0 += 32) {
+      const int j = j0 + lane;
+      const float hj = j < H ? hn[j] : 0.f;
+      float dhj = 0.f;
+      for (int k = 0; k < C; ++k) {
+        const float dk = __shfl_sync(kFull, dlogit, k);
+        if (j < H) {
+          dhj = fmaf(p.Wc[j * C + k], dk, dhj);
+          atomicAdd(&s_dWc[j * C + k], hj * dk);
+        }
+      }
+      if (j < H) p.dh[(size_t)node * H + j] = dhj;
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < H * C; i += blockDim.x) atomicAdd(&p.dWc[i], s_dWc[i]);
+  for (int i = tid; i < C; i += blockDim.x) atomicAdd(&p.dbc[i], s_dWc[H * C + i]);
+}
+
+// ---- gate gradients of one wavefront -------------------------------------------------------- //
+__global__ void k_bwd_gates(BwdParams p, int row_begin, int row_end, int leaf) {
+  const int H = p.H;
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long total = (long long)(row_end - row_begin) * H;
+  if (idx >= total) return;
+  const int row = row_begin + (int)(idx / H), u = (int)(idx % H);
+  const int node = p.order[row];
+  const float* g = p.gates + (size_t)node * 5 * H + u;
+  const float gi = g[0], go = g[3 * H], gu = g[4 * H];
+  const float cn = p.c[(size_t)node * H + u];
+  const float tc = tanhf(cn);
+  const float dhn = p.dh[(size_t)node * H + u];
+  const float dcn = p.dc[(size_t)node * H + u] + dhn * go * (1.f - tc * tc);
+  float* dz = p.dz + (size_t)node * 5 * H + u;
+  dz[0] = dcn * gu * gi * (1.f - gi);
+  dz[3 * H] = dhn * tc * go * (1.f - go);
+  dz[4 * H] = dcn * gi * (1.f - gu * gu);
+  if (leaf) {
+    dz[H] = 0.f;
+    dz[2 * H] = 0.f;
+  } else {
+    const int l = p.left[node], r = p.right[node];
+    const float gfl = g[H], gfr = g[2 * H];
+    dz[H] = dcn * p.c[(size_t)l * H + u] * gfl * (1.f - gfl);
+    dz[2 * H] = dcn * p.c[(size_t)r * H + u] * gfr * (1.f - gfr);
+    p.dc[(size_t)l * H + u] = dcn * gfl;  // every node has exactly one caller: plain stores
+    p.dc[(size_t)r * H + u] = dcn * gfr;
+  }
+}
+
+// ---- dIn = dz W^T for one wavefront --------------------------------------------------------- //
+// out[row][k] = sum_j dz[row][j] * W[koff + k][j]; tile 64 rows x 64 outputs, 16 x 16 threads.
+constexpr int BT = 64, BK = 16;
+
+__global__ void __launch_bounds__(256)
+k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
+  __shared__ float As[BT][BK + 1];
+  __shared__ float Bs[BT][BK + 1];
+  __shared__ int s_node[BT];
+  const int H = p.H, E = p.E, J = 5 * H;
+  const int K = leaf ? E : 2 * H, koff = leaf ? 0 : E;
+  const int tiles_k = (K + BT - 1) / BT;
+  const int row0 = row_begin + (blockIdx.x / tiles_k) * BT, k0 = (blockIdx.x % tiles_k) * BT;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  for (int i = tid; i < BT; i += 256) s_node[i] = row0 + i < row_end ? p.order[row0 + i] : -1;
+  __syncthreads();
+  float acc[4][4] = {};
+  for (int j0 = 0; j0 < J; j0 += BK) {
+    for (int e = tid; e < BT * BK; e += 256) {
+      const int i = e / BK, jj = e % BK, j = j0 + jj;
+      As[i][jj] = (s_node[i] >= 0 && j < J) ? p.dz[(size_t)s_node[i] * J + j] : 0.f;
+      Bs[i][jj] = (k0 + i < K && j < J) ? __ldg(p.W + (size_t)(koff + k0 + i) * J + j) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int jj = 0; jj < BK; ++jj) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = As[ty + 16 * i][jj]; b[i] = Bs[tx + 16 * i][jj]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[i][q] = fmaf(a[i], b[q], acc[i][q]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int node = s_node[ty + 16 * i];
+    if (node < 0) continue;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int k = k0 + tx + 16 * q;
+      if (k >= K) continue;
+      if (leaf) {
+        atomicAdd(&p.dEmb_rows[(size_t)p.tok_slot[p.token[node]] * E + k], acc[i][q]);
+      } else {
+        const int child = k < H ? p.left[node] : p.right[node];
+        p.dh[(size_t)child * H + (k < H ? k : k - H)] += acc[i][q];  // single caller: no race
+      }
+    }
+  }
+}
+
+// ---- dW = In^T dZ (contraction over nodes) and db ------------------------------------------- //
+// part 0: rows [0,E) from the leaves (In = embedding rows); part 1: rows [E,E+2H) from the
+// internal nodes (In = [h_l | h_r]).  Tile 64 (k) x 64 (j); gridDim.y splits the node range.
+__global__ void __launch_bounds__(256)
+k_bwd_dweight(BwdParams p, int part, int row_begin, int row_end, int rows_per_split) {
+  __shared__ float As[BK][BT];
+  __shared__ float Bs[BK][BT];
+  __shared__ int s_a[BK], s_b[BK], s_node[BK];
+  const int H = p.H, E = p.E, J = 5 * H;
+  const int K = part == 0 ? E : 2 * H, koff = part == 0 ? 0 : E;
+  const int tiles_j = (J + BT - 1) / BT;
+  const int k0 = (blockIdx.x / tiles_j) * BT, j0 = (blockIdx.x % tiles_j) * BT;
+  const int r_lo = row_begin + blockIdx.y * rows_per_split;
+  const int r_hi = min(row_end, r_lo + rows_per_split);
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  float acc[4][4] = {};
+  for (int r0 = r_lo; r0 < r_hi; r0 += BK) {
+    if (tid < BK) {
+      const int row = r0 + tid;
+      int node = -1, a = 0, b = 0;
+      if (row < r_hi) {
+        node = p.order[row];
+        a = part == 0 ? p.token[node] : p.left[node];
+        b = part == 0 ? 0 : p.right[node];
+      }
+      s_node[tid] = node; s_a[tid] = a; s_b[tid] = b;
+    }
+    __syncthreads();
+    for (int e = tid; e < BK * BT; e += 256) {
+      const int rr = e / BT, cc = e % BT;
+      float va = 0.f, vb = 0.f;
+      if (s_node[rr] >= 0) {
+        const int k = k0 + cc, j = j0 + cc;
+        if (k < K)
+          va = part == 0 ? __ldg(p.emb + (size_t)s_a[rr] * E + k)
+                         : (k < H ? p.h[(size_t)s_a[rr] * H + k] : p.h[(size_t)s_b[rr] * H + (k - H)]);
+        if (j < J) vb = p.dz[(size_t)s_node[rr] * J + j];
+      }
+      As[rr][cc] = va;
+      Bs[rr][cc] = vb;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int rr = 0; rr < BK; ++rr) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = As[rr][ty + 16 * i]; b[i] = Bs[rr][tx + 16 * i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[i][q] = fmaf(a[i], b[q], acc[i][q]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int k = k0 + ty + 16 * i;
+    if (k >= K) continue;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int j = j0 + tx + 16 * q;
+      if (j < J) atomicAdd(&p.dW[(size_t)(koff + k) * J + j], acc[i][q]);
+    }
+  }
+}
+
+__global__ void k_bwd_dbias(BwdParams p) {
+  const int J = 5 * p.H;
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= J) return;
+  const int r_lo = blockIdx.y * 256, r_hi = min(p.n, r_lo + 256);
+  float acc = 0.f;
+  for (int r = r_lo; r < r_hi; ++r) acc += p.dz[(size_t)r * J + j];
+  atomicAdd(&p.db[j], acc);
+}
+
+}  // namespace
+
+int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW, float* db,
+                    float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,
+                    int32_t* n_touched, cudaStream_t stream) {
+  auto& L = ctx->last;
+  L.stream = stream;
+  int rc = ensure_host_levels(ctx);
+  if (rc != TREELSTM_OK) return rc;
+  const int n = L.n, H = ctx->H, E = ctx->E, C = ctx->C, n_levels = L.n_levels;
+  const int32_t* off = ctx->host_level_offset;
+  char* base = static_cast<char*>(L.ws);
+  BwdParams p;
+  p.n = n; p.H = H; p.E = E; p.C = C; p.vocab = ctx->vocab;
+  p.n_leaves = n_levels > 0 ? off[1] : 0;
+  p.left = L.left; p.right = L.right; p.token = L.token; p.order = L.order; p.labels = labels;
+  p.emb = ctx->emb; p.W = ctx->W; p.Wc = ctx->Wc; p.bc = ctx->bc; p.h = L.h; p.c = L.c;
+  p.gates = reinterpret_cast<const float*>(base + L.lay.gates);
+  p.dh = reinterpret_cast<float*>(base + L.lay.dh);
+  p.dc = reinterpret_cast<float*>(base + L.lay.dc);
+  p.dz = reinterpret_cast<float*>(base + L.lay.dz);
+  p.loss = loss; p.dW = dW; p.db = db; p.dWc = dWc; p.dbc = dbc; p.dEmb_rows = dEmb_rows;
+  p.tok_slot = reinterpret_cast<int*>(base + L.lay.tok_slot);
+  p.touched_ids = touched_ids; p.n_touched = n_touched;
+  p.st = reinterpret_cast<DevStatus*>(base + L.lay.status);
+
+  const size_t J = 5 * (size_t)H;
+  TL_CUDA(ctx, cudaMemsetAsync(loss, 0, sizeof(float), stream));
+  TL_CUDA(ctx, cudaMemsetAsync(dW, 0, sizeof(float) * (E + 2 * (size_t)H) * J, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(db, 0, sizeof(float) * J, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(dWc, 0, sizeof(float) * H * C, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(dbc, 0, sizeof(float) * C, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(n_touched, 0, sizeof(int), stream));
+  if (n == 0) return TREELSTM_OK;
+  TL_CUDA(ctx, cudaMemsetAsync(p.dc, 0, sizeof(float) * (size_t)n * H, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(p.tok_slot, 0, sizeof(int) * ((size_t)ctx->vocab + 1), stream));
+  TL_CUDA(ctx, cudaMemsetAsync(dEmb_rows, 0, sizeof(float) * (size_t)p.n_leaves * E, stream));
+
+  k_bwd_mark_tokens<<<(p.n_leaves + 255) / 256, 256, 0, stream>>>(p);
+  k_bwd_scan_tokens<<<1, 1024, 0, stream>>>(p);
+  const size_t cls_smem = sizeof(float) * ((size_t)H * C + C);
+  if (cls_smem > 200 * 1024) return TREELSTM_ERR_UNSUPPORTED;
+  if (cls_smem > 48 * 1024)
+    TL_CUDA(ctx, cudaFuncSetAttribute(k_bwd_classifier, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)cls_smem));
+  k_bwd_classifier<<<(n + kClsNodesPerCta - 1) / kClsNodesPerCta, kClsWarps * 32, cls_smem, stream>>>(p);
+  ctx->launches += 3;
+  for (int lvl = n_levels - 1; lvl >= 0; --lvl) {
+    const int begin = off[lvl], end = off[lvl + 1], leaf = lvl == 0 ? 1 : 0;
+    const long long elems = (long long)(end - begin) * H;
+    k_bwd_gates<<<(unsigned)((elems + 255) / 256), 256, 0, stream>>>(p, begin, end, leaf);
+    const int K = leaf ? E : 2 * H;
+    const int tiles = ((end - begin + BT - 1) / BT) * ((K + BT - 1) / BT);
+    k_bwd_dinput<<<tiles, 256, 0, stream>>>(p, begin, end, leaf);
+    ctx->launches += 2;
+  }
+  const int tiles_j = (int)((J + BT - 1) / BT);
+  for (int part = 0; part < 2; ++part) {
+    const int begin = part == 0 ? 0 : p.n_leaves, end = part == 0 ? p.n_leaves : n;
+    if (end <= begin) continue;
+    const int K = part == 0 ? E : 2 * H;
+    const int rows_per_split = 256;
+    const int splits = (end - begin + rows_per_split - 1) / rows_per_split;
+    dim3 grid(((K + BT - 1) / BT) * tiles_j, splits);
+    k_bwd_dweight<<<grid, 256, 0, stream>>>(p, part, begin, end, rows_per_split);
+    ctx->launches += 1;
+  }
+  dim3 gb((unsigned)((J + 127) / 128), (n + 255) / 256);
+  k_bwd_dbias<<<gb, 128, 0, stream>>>(p);
+  ctx->launches += 1;
+  TL_CUDA(ctx, cudaGetLastError());
+  return TREELSTM_OK;
+}
+
+}  // namespace tl

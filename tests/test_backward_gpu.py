@@ -1,0 +1,79 @@
+"""Parity of the CUDA training step (forward + backward through structure, via the C ABI) against
+the fp64 oracle: loss and every gradient group within 1e-4 max-abs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import treelstm_oracle as orc
+from paper_1809_00832_b200 import binding, forests as fg
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def _train_step(model, forest, labels, flags):
+    out = model.forward(util.to_dev(forest.left), util.to_dev(forest.right), util.to_dev(forest.token),
+                        flags=flags | binding.SAVE_FOR_BACKWARD)
+    grads = model.backward(util.to_dev(labels), forest.n_leaves)
+    torch.cuda.synchronize()
+    res = {k: v.cpu().numpy() for k, v in grads.items()}
+    res["h"] = out["h"].cpu().numpy()
+    return res
+
+
+def _compare(res, ref, tol):
+    assert abs(float(res["loss"][0]) - ref["loss"]) < tol
+    for k in ("dW", "db", "dWc", "dbc"):
+        assert util.max_abs(res[k], ref[k]) < tol, k
+    nt = int(res["n_touched"][0])
+    assert nt == len(ref["touched_ids"])
+    np.testing.assert_array_equal(res["touched_ids"][:nt], ref["touched_ids"])
+    assert util.max_abs(res["dEmb_rows"][:nt], ref["dEmb_rows"]) < tol
+
+
+@pytest.mark.parametrize("flags", [binding.PER_LEVEL, binding.PERSISTENT])
+def test_training_step_matches_oracle(flags):
+    w = fg.make_workload("train25_fp32", 0)
+    f, p = w.forest, w.params
+    ref = orc.loss_and_gradients(f.left, f.right, f.token, p.emb, p.W, p.b, p.Wc, p.bc, w.labels)
+    model = util.make_model(p, "fp32")
+    res = _train_step(model, f, w.labels, flags)
+    assert util.max_abs(res["h"], ref["h"]) < util.TOL["fp32"]
+    _compare(res, ref, util.TOL["fp32"])
+    # gradients are overwritten, not accumulated: a second step gives the same numbers
+    res2 = _train_step(model, f, w.labels, flags)
+    _compare(res2, ref, util.TOL["fp32"])
+
+
+def test_training_step_small_odd_sizes_and_duplicates():
+    # larger gradients (weights +-0.5), sizes that match no tile, permuted ids, duplicated tokens and
+    # duplicated subtrees: every node must receive its own forward values
+    rng = np.random.default_rng(4)
+    params = fg.draw_params(rng, 7, 5, 6, emb_dist="uniform", emb_scale=0.5, w_scale=0.5, n_classes=3)
+    shape = fg.random_split_shape(rng, 9)
+    forest = fg.forest_from_shapes([shape, shape, None, fg.left_chain_shape(12)], rng, 6)
+    forest, _ = fg.permute_node_ids(forest, rng)
+    labels = rng.integers(0, 3, size=forest.n_nodes).astype(np.int32)
+    ref = orc.loss_and_gradients(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
+                                 params.Wc, params.bc, labels)
+    model = util.make_model(params, "fp32")
+    res = _train_step(model, forest, labels, binding.PERSISTENT)
+    _compare(res, ref, util.TOL["fp32"])
+
+
+def test_backward_errors():
+    rng = np.random.default_rng(6)
+    params = fg.draw_params(rng, 4, 4, 5, emb_dist="uniform", emb_scale=0.5, w_scale=0.5, n_classes=3)
+    model = util.make_model(params, "fp32")
+    forest = fg.forest_from_shapes([fg.random_split_shape(rng, 5)], rng, 5)
+    arrs = [util.to_dev(a) for a in (forest.left, forest.right, forest.token)]
+    labels = torch.zeros(forest.n_nodes, dtype=torch.int32, device="cuda")
+    model.forward(*arrs, flags=binding.PERSISTENT)                  # nothing saved
+    with pytest.raises(binding.TreeLSTMError) as err:
+        model.backward(labels, forest.n_leaves)
+    assert err.value.code == binding.ERR_STATE
+    model.forward(*arrs, flags=binding.PERSISTENT | binding.SAVE_FOR_BACKWARD)
+    labels[2] = 3
+    with pytest.raises(binding.TreeLSTMError) as err:
+        model.backward(labels, forest.n_leaves)
+    assert err.value.code == binding.ERR_LABEL_OUT_OF_RANGE

@@ -42,8 +42,6 @@ def test_schedule_paths_agree_with_oracle_on_permuted_ids(single_cta):
                                           w.params.W, w.params.b)
     assert util.max_abs(res["h"], href) < util.TOL["fp32"]
     assert util.max_abs(res["c"], cref) < util.TOL["fp32"]
-    res0 = util.gpu_forward(model, w.forest, binding.PERSISTENT)
-    np.testing.assert_allclose(res["h"][new_of_old], res0["h"], atol=2e-6)
     roots = model.roots(forest.n_trees + 3)
     torch.cuda.synchronize()
     n_roots = int(roots["n_roots"].item())
@@ -51,6 +49,9 @@ def test_schedule_paths_agree_with_oracle_on_permuted_ids(single_cta):
     ids = roots["root_ids"].cpu().numpy()[:n_roots]
     np.testing.assert_array_equal(ids, np.sort(forest.roots))
     np.testing.assert_array_equal(roots["root_h"].cpu().numpy()[:n_roots], res["h"][ids])
+    np.testing.assert_array_equal(roots["root_c"].cpu().numpy()[:n_roots], res["c"][ids])
+    res0 = util.gpu_forward(model, w.forest, binding.PERSISTENT)
+    np.testing.assert_allclose(res["h"][new_of_old], res0["h"], atol=2e-6)
 
 
 @pytest.mark.parametrize("single_cta", [True, False])
