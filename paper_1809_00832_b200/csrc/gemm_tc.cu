@@ -1,7 +1,546 @@
+// bf16 tensor-core wavefront evaluation (sm_100a: tcgen05.mma with the accumulator in tensor
+// memory, weights fetched by TMA, operand rows gathered by cp.async, cell update fused into the
+// epilogue that drains tensor memory).
+//
+// Paper: Figure 2 (Section 3.1) - a node is LSTM(embed(word)) or LSTM(left_state, right_state);
+// Section 2.2 - sibling subtrees are independent, so every node whose children are done can be
+// evaluated at once.  Batching those nodes into one wide contraction is what Section 6.3 calls
+// folding and charges with regrouping copies per depth; here nothing is regrouped: the operand
+// rows are gathered straight from the node-indexed state array into the swizzled shared-memory
+// tile the tensor core reads.
+//
+// One tile = 128 ready nodes x (8*G hidden units x 5 gates).  W is pre-packed so that the 5 gate
+// pre-activations of a hidden unit sit in the same accumulator row slice and one thread (one
+// tensor-memory lane = one node) can finish the cell without any exchange.
+//
+// Warp roles (320 threads): warps 0-3 epilogue (tensor-memory lane quadrant = warp id), warp 4
+// TMA producer of W tiles, warp 5 MMA issuer + tensor-memory owner, warps 6-9 gather the A rows.
 #include "common.cuh"
+
 namespace tl {
-int pack_weights_bf16(treelstm*, cudaStream_t) { return TREELSTM_ERR_UNSUPPORTED; }
-int launch_forward_bf16(treelstm*, int, const int32_t*, const int32_t*, const int32_t*, float*, float*,
-                        const int32_t*, const int32_t*, const int32_t*, int, int, void*, const WsLayout&,
-                        cudaStream_t) { return TREELSTM_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr int BM = 128;                 // nodes per tile (UMMA M)
+constexpr int kStages = 4;
+constexpr int kThreads = 320;
+constexpr int kABytes = BM * 128;       // one K block (64 bf16) of 128 rows
+constexpr int kAccCols = 256;           // accumulator stage stride in tensor-memory columns
+constexpr unsigned kFull = 0xffffffffu;
+
+template <int G> struct Cfg {
+  static constexpr int kUnits = 8 * G;
+  static constexpr int NI = 40 * G;     // accumulator columns of an internal tile (5 gates)
+  static constexpr int NL = 24 * G;     // accumulator columns of a leaf tile (gates i, o, u)
+  static constexpr int kBBytes = NI * 128;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static_assert(NI % 16 == 0 && NL % 16 == 0 && NI <= 256, "UMMA N must be a multiple of 16, <= 256");
+  static_assert(kBBytes % 1024 == 0, "stage buffers stay 1024-byte aligned");
+};
+
+struct TcParams {
+  int n, H, Hp, Ep;
+  const int *order, *rowA, *rowB, *level_offset;
+  const __nv_bfloat16* emb_bf;
+  __nv_bfloat16* hb;
+  const float *bp_h, *bp_x;
+  float *h, *c, *gates;
+  DevStatus* st;
+  long long wait_limit;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------- //
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+// Bounded wait: gives up when the cycle budget is spent or another thread of the CTA gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort,
+                                          long long limit, DevStatus* st) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*s_abort) return false;
+    if (clock64() - t0 > limit) {
+      *s_abort = 1;
+      report(st, TREELSTM_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* v) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the
+// 128-byte swizzle (8-row groups of 1024 bytes): start address, stride between 8-row groups,
+// descriptor version 1, swizzle mode 2.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset
+  d |= (uint64_t)1 << 46;                 // version
+  d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+__device__ __forceinline__ float sigmoid_fast(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
+__device__ __forceinline__ float tanh_fast(float x) { return 2.0f * sigmoid_fast(2.0f * x) - 1.0f; }
+
+__device__ __forceinline__ void ld_row8(const float* p, bool vec, float* out) {
+  if (vec) {
+    const float4 a = __ldcg(reinterpret_cast<const float4*>(p));
+    const float4 b = __ldcg(reinterpret_cast<const float4*>(p) + 1);
+    out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+    out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) out[j] = __ldcg(p + j);
+  }
+}
+__device__ __forceinline__ void st_row8(float* p, bool vec, int count, const float* v) {
+  if (vec && count == 8) {
+    reinterpret_cast<float4*>(p)[0] = make_float4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<float4*>(p)[1] = make_float4(v[4], v[5], v[6], v[7]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (j < count) p[j] = v[j];
+  }
+}
+
+// ---- the kernel -------------------------------------------------------------------------------- //
+// only_level >= 0: process that wavefront only (one launch per level).  only_level < 0: all
+// wavefronts, separated by the bounded grid barrier (cooperative launch).
+template <int G>
+__global__ void __launch_bounds__(kThreads, 1)
+k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CUtensorMap tmap_wx,
+         TcParams p, int only_level) {
+  using C = Cfg<G>;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
+  unsigned char* tiles_ptr = smem_raw + (tiles_addr - raw_addr);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + kStages * C::kStageBytes);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  int* s_flag = const_cast<int*>(s_abort) + 1;
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (ld_volatile(&p.st->status) != 0) return;      // schedule failed: nothing to evaluate
+  const int n_levels = p.st->n_levels;
+
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 128 + 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+
+  const int Hp = p.Hp, H = p.H;
+  const int ntn = Hp / C::kUnits;                    // column tiles per row tile
+  const int kb_leaf = p.Ep / kKBlock, kb_int = 2 * Hp / kKBlock, kb_half = Hp / kKBlock;
+  const bool vec = (H % 4) == 0;
+
+  // pipeline positions; every role walks the same tile sequence, so they stay in step
+  uint32_t stage = 0, phase = 0;        // smem ring (producers and MMA)
+  uint32_t acc_iter = 0;                // accumulator ring (MMA and epilogue)
+  bool alive = true;
+
+  const int lvl_begin = only_level >= 0 ? only_level : 0;
+  const int lvl_end = only_level >= 0 ? only_level + 1 : n_levels;
+  for (int lvl = lvl_begin; lvl < lvl_end; ++lvl) {   // uniform trip count: barriers inside
+    const int begin = p.level_offset[lvl], end = p.level_offset[lvl + 1];
+    const bool leaf = lvl == 0;
+    const int tiles = ((end - begin + BM - 1) / BM) * ntn;
+    const int kblocks = leaf ? kb_leaf : kb_int;
+    const int ncols = leaf ? C::NL : C::NI;
+
+    for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
+      const int row0 = begin + (t / ntn) * BM, nt = t % ntn;
+
+      if (warp == 4) {
+        // ---------------- W tile producer (TMA) ----------------
+        if (lane == 0) {
+          const CUtensorMap* map = leaf ? &tmap_wx : &tmap_wh;
+          const uint32_t bytes = (uint32_t)ncols * 128u;
+          for (int kb = 0; kb < kblocks; ++kb) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1, s_abort, p.wait_limit, p.st)) { alive = false; break; }
+            mbar_arrive_expect_tx(full_bar(stage), bytes);
+            tma_load_2d(tiles_addr + stage * C::kStageBytes + kABytes, map, kb * kKBlock, nt * ncols,
+                        full_bar(stage));
+            if (++stage == kStages) { stage = 0; phase ^= 1; }
+          }
+        }
+      } else if (warp == 5) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+          const uint32_t acc = acc_iter & 1, acc_phase = (acc_iter >> 1) & 1;
+          if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + acc * kAccCols;
+          const uint32_t idesc = umma_idesc(ncols);
+          for (int kb = 0; kb < kblocks && alive; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, s_abort, p.wait_limit, p.st)) { alive = false; break; }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            tc_fence_after();
+            const uint32_t a_addr = tiles_addr + stage * C::kStageBytes;
+            const uint64_t a_desc = umma_desc(a_addr), b_desc = umma_desc(a_addr + kABytes);
+#pragma unroll
+            for (int k = 0; k < kKBlock / 16; ++k)   // UMMA K = 16 bf16 = 32 bytes = 2 descriptor units
+              umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+            umma_commit(empty_bar(stage));           // frees the smem stage when these MMAs retire
+            if (++stage == kStages) { stage = 0; phase ^= 1; }
+          }
+          if (alive) umma_commit(tfull_bar(acc));    // accumulator complete
+        }
+        ++acc_iter;
+      } else if (warp >= 6) {
+        // ---------------- A row gather (cp.async into the swizzled tile) ----------------
+        const int r = tid - 6 * 32;                  // tile row owned by this thread
+        const int row = row0 + r;
+        const bool valid = row < end;
+        const int ia = valid ? p.rowA[row] : 0, ib = valid ? p.rowB[row] : 0;
+        const uint32_t nbytes = valid ? 16u : 0u;    // rows past the wavefront are zero-filled
+        const uint32_t row_off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1, s_abort, p.wait_limit, p.st)) { alive = false; break; }
+          const __nv_bfloat16* src;
+          if (leaf) src = p.emb_bf + (size_t)ia * p.Ep + kb * kKBlock;
+          else if (kb < kb_half) src = p.hb + (size_t)ia * Hp + kb * kKBlock;
+          else src = p.hb + (size_t)ib * Hp + (kb - kb_half) * kKBlock;
+          const uint32_t dst = tiles_addr + stage * C::kStageBytes + row_off;
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch)
+            cp_async16(dst + (uint32_t)((ch ^ (r & 7)) << 4), src + ch * 8, nbytes);
+          cp_async_arrive_noinc(full_bar(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+      } else {
+        // ---------------- epilogue: drain tensor memory, finish the cell ----------------
+        const int r = warp * 32 + lane;
+        const int row = row0 + r;
+        const bool valid = row < end;
+        const int node = valid ? p.order[row] : 0;
+        const int il = (valid && !leaf) ? p.rowA[row] : 0, ir = (valid && !leaf) ? p.rowB[row] : 0;
+        const uint32_t acc = acc_iter & 1, acc_phase = (acc_iter >> 1) & 1;
+        if (!mbar_wait(tfull_bar(acc), acc_phase, s_abort, p.wait_limit, p.st)) alive = false;
+        alive = __all_sync(kFull, alive);
+        if (alive) {
+          tc_fence_after();
+          const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(warp * 32) << 16);
+          const float* bias = leaf ? p.bp_x + nt * C::NL : p.bp_h + nt * C::NI;
+#pragma unroll 1
+          for (int g = 0; g < G; ++g) {
+            uint32_t v[40];
+            const int gcols = leaf ? 24 : 40;
+            const uint32_t col0 = (uint32_t)(g * gcols);
+            if (leaf) {
+#pragma unroll
+              for (int q = 0; q < 3; ++q) tmem_ld8(taddr + col0 + 8 * q, v + 8 * q);
+            } else {
+#pragma unroll
+              for (int q = 0; q < 5; ++q) tmem_ld8(taddr + col0 + 8 * q, v + 8 * q);
+            }
+            tmem_ld_wait();
+            if (valid) {
+              const int u0 = (nt * G + g) * 8;
+              const int count = min(8, H - u0);     // real (unpadded) units in this group
+              float cl[8] = {}, cr[8] = {}, hv[8], cv[8], gi[8], gfl[8], gfr[8], go[8], gu[8];
+              const float* bg = bias + g * gcols;
+              if (!leaf && count > 0) {
+                if (count == 8) {
+                  ld_row8(p.c + (size_t)il * H + u0, vec, cl);
+                  ld_row8(p.c + (size_t)ir * H + u0, vec, cr);
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) {
+                    cl[j] = j < count ? __ldcg(p.c + (size_t)il * H + u0 + j) : 0.f;
+                    cr[j] = j < count ? __ldcg(p.c + (size_t)ir * H + u0 + j) : 0.f;
+                  }
+                }
+              }
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                if (leaf) {
+                  gi[j] = sigmoid_fast(__uint_as_float(v[j]) + __ldg(bg + j));
+                  go[j] = sigmoid_fast(__uint_as_float(v[8 + j]) + __ldg(bg + 8 + j));
+                  gu[j] = tanh_fast(__uint_as_float(v[16 + j]) + __ldg(bg + 16 + j));
+                  gfl[j] = gfr[j] = 0.f;
+                  cv[j] = gi[j] * gu[j];
+                } else {
+                  gi[j] = sigmoid_fast(__uint_as_float(v[j]) + __ldg(bg + j));
+                  gfl[j] = sigmoid_fast(__uint_as_float(v[8 + j]) + __ldg(bg + 8 + j));
+                  gfr[j] = sigmoid_fast(__uint_as_float(v[16 + j]) + __ldg(bg + 16 + j));
+                  go[j] = sigmoid_fast(__uint_as_float(v[24 + j]) + __ldg(bg + 24 + j));
+                  gu[j] = tanh_fast(__uint_as_float(v[32 + j]) + __ldg(bg + 32 + j));
+                  cv[j] = gi[j] * gu[j] + gfl[j] * cl[j] + gfr[j] * cr[j];
+                }
+                hv[j] = go[j] * tanh_fast(cv[j]);
+              }
+              // bf16 copy of h feeds the next wavefront's gather; padded units are written as 0
+              uint32_t packed[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float lo = 2 * j < count ? hv[2 * j] : 0.f, hi = 2 * j + 1 < count ? hv[2 * j + 1] : 0.f;
+                __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+                packed[j] = *reinterpret_cast<uint32_t*>(&b2);
+              }
+              *reinterpret_cast<uint4*>(p.hb + (size_t)node * Hp + u0) =
+                  make_uint4(packed[0], packed[1], packed[2], packed[3]);
+              if (count > 0) {
+                st_row8(p.h + (size_t)node * H + u0, vec, count, hv);
+                st_row8(p.c + (size_t)node * H + u0, vec, count, cv);
+                if (p.gates) {
+                  float* gp = p.gates + (size_t)node * 5 * H + u0;
+                  st_row8(gp, vec, count, gi);
+                  st_row8(gp + H, vec, count, gfl);
+                  st_row8(gp + 2 * H, vec, count, gfr);
+                  st_row8(gp + 3 * H, vec, count, go);
+                  st_row8(gp + 4 * H, vec, count, gu);
+                }
+              }
+            }
+          }
+          tc_fence_before();
+          mbar_arrive(tempty_bar(acc));              // accumulator stage may be overwritten
+        }
+        ++acc_iter;
+      }
+    }
+    if (only_level < 0 && lvl + 1 < lvl_end) {
+      // every role of every CTA joins the barrier.  A role that gave up has set s_abort before
+      // this point, so the flag read after the CTA barrier is the same for all threads and the
+      // loop is left by all of them together.
+      __syncthreads();
+      if (*s_abort) break;
+      if (!grid_barrier(p.st, (unsigned)(lvl + 1) * gridDim.x, p.wait_limit, s_flag)) break;
+    }
+  }
+
+  // teardown: let in-flight asynchronous copies land before shared/tensor memory is released
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  tc_fence_before();
+  __syncthreads();
+  if (*s_abort) __nanosleep(100000);
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---- weight packing ---------------------------------------------------------------------------- //
+// Packed row of hidden unit u, gate g (internal order i, f_l, f_r, o, u): (u/8)*40 + g*8 + u%8;
+// leaf tiles keep gates i, o, u only: (u/8)*24 + gi*8 + u%8.  Each packed row holds the K vector.
+__global__ void k_pack_weights(int H, int E, int Hp, int Ep, const float* W, const float* b,
+                               __nv_bfloat16* Wp_h, __nv_bfloat16* Wp_x, float* bp_h, float* bp_x) {
+  const int groups = Hp / 8;
+  const size_t J = 5 * (size_t)H;
+  const size_t total_h = (size_t)groups * 40 * 2 * Hp, total_x = (size_t)groups * 24 * Ep;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total_h; i += stride) {
+    const int k = (int)(i % (2 * Hp)), prow = (int)(i / (2 * Hp));
+    const int u = (prow / 40) * 8 + prow % 8, g = (prow % 40) / 8;
+    const int kk = k < Hp ? k : k - Hp;
+    float v = 0.f;
+    if (u < H && kk < H) v = W[(size_t)(E + (k < Hp ? 0 : H) + kk) * J + g * H + u];
+    Wp_h[i] = __float2bfloat16_rn(v);
+    if (k == 0) bp_h[prow] = u < H ? b[g * H + u] : 0.f;
+  }
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total_x; i += stride) {
+    const int k = (int)(i % Ep), prow = (int)(i / Ep);
+    const int u = (prow / 24) * 8 + prow % 8, gi = (prow % 24) / 8;
+    const int g = gi == 0 ? 0 : (gi == 1 ? 3 : 4);
+    float v = 0.f;
+    if (u < H && k < E) v = W[(size_t)k * J + g * H + u];
+    Wp_x[i] = __float2bfloat16_rn(v);
+    if (k == 0) bp_x[prow] = u < H ? b[g * H + u] : 0.f;
+  }
+}
+
+__global__ void k_pack_embedding(int vocab, int E, int Ep, const float* emb, __nv_bfloat16* emb_bf) {
+  const size_t total = (size_t)vocab * Ep, stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int k = (int)(i % Ep);
+    const size_t v = i / Ep;
+    emb_bf[i] = __float2bfloat16_rn(k < E ? emb[v * E + k] : 0.f);
+  }
+}
+
+// Per-row operand indices in ready order: rowA = token (leaf) or left child, rowB = right child.
+__global__ void k_row_operands(int n, const int* order, const int* left, const int* right,
+                               const int* token, int* rowA, int* rowB, const DevStatus* st) {
+  if (st->status != 0) return;
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= n) return;
+  const int node = order[r];
+  const int l = left[node];
+  rowA[r] = l < 0 ? token[node] : l;
+  rowB[r] = l < 0 ? 0 : right[node];
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+int make_tmap(treelstm* ctx, CUtensorMap* map, void* base, uint64_t inner, uint64_t rows, uint32_t box_rows) {
+  static EncodeTiledFn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    TL_CUDA(ctx, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+    if (!fn || q != cudaDriverEntryPointSuccess) return TREELSTM_ERR_CUDA;
+    encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  const cuuint64_t dims[2] = {inner, rows};
+  const cuuint64_t strides[1] = {inner * 2};           // bytes between rows
+  const cuuint32_t box[2] = {kKBlock, box_rows};       // 64 bf16 = one 128-byte swizzle span
+  const cuuint32_t elem[2] = {1, 1};
+  CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, elem,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { ctx->cuda_error = (int)r; return TREELSTM_ERR_CUDA; }
+  return TREELSTM_OK;
+}
+
+constexpr int kG = 4;   // unit groups per tile: 32 hidden units, 160 accumulator columns
+
+}  // namespace
+
+int pack_weights_bf16(treelstm* ctx, cudaStream_t stream) {
+  k_pack_weights<<<512, 256, 0, stream>>>(ctx->H, ctx->E, ctx->Hp, ctx->Ep, ctx->W, ctx->b, ctx->Wp_h,
+                                          ctx->Wp_x, ctx->bp_h, ctx->bp_x);
+  k_pack_embedding<<<1024, 256, 0, stream>>>(ctx->vocab, ctx->E, ctx->Ep, ctx->emb, ctx->emb_bf);
+  TL_CUDA(ctx, cudaGetLastError());
+  const int groups = ctx->Hp / kUnitGroup;
+  int rc = make_tmap(ctx, &ctx->tmap_wh, ctx->Wp_h, 2 * (uint64_t)ctx->Hp, (uint64_t)groups * 40, Cfg<kG>::NI);
+  if (rc != TREELSTM_OK) return rc;
+  rc = make_tmap(ctx, &ctx->tmap_wx, ctx->Wp_x, (uint64_t)ctx->Ep, (uint64_t)groups * 24, Cfg<kG>::NL);
+  if (rc != TREELSTM_OK) return rc;
+  ctx->have_tmaps = true;
+  return TREELSTM_OK;
+}
+
+int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
+                        const int32_t* token, float* h, float* c, const int32_t* order,
+                        const int32_t* level_offset_dev, const int32_t* level_offset_host,
+                        int n_levels_host, int flags, void* ws, const WsLayout& lay,
+                        cudaStream_t stream) {
+  using C = Cfg<kG>;
+  if (!ctx->have_tmaps) return TREELSTM_ERR_STATE;
+  char* base = static_cast<char*>(ws);
+  TcParams p;
+  p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep;
+  p.order = order;
+  p.rowA = reinterpret_cast<int*>(base + lay.pending);     // dependency counters are dead by now
+  p.rowB = reinterpret_cast<int*>(base + lay.order_tmp);
+  p.level_offset = level_offset_dev;
+  p.emb_bf = ctx->emb_bf;
+  p.hb = reinterpret_cast<__nv_bfloat16*>(base + lay.hb);
+  p.bp_h = ctx->bp_h; p.bp_x = ctx->bp_x;
+  p.h = h; p.c = c;
+  p.gates = (flags & TREELSTM_SAVE_FOR_BACKWARD) ? reinterpret_cast<float*>(base + lay.gates) : nullptr;
+  p.st = reinterpret_cast<DevStatus*>(base + lay.status);
+  p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
+
+  k_row_operands<<<(n + 255) / 256, 256, 0, stream>>>(n, order, left, right, token, const_cast<int*>(p.rowA),
+                                                      const_cast<int*>(p.rowB), p.st);
+  ctx->launches += 1;
+  static bool attr_set = false;
+  if (!attr_set) {
+    TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc<kG>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+    attr_set = true;
+  }
+  const int ntn = ctx->Hp / C::kUnits;
+  if (flags & TREELSTM_PERSISTENT) {
+    int grid = ctx->sm_count;                       // one CTA per SM (shared and tensor memory)
+    const int want = ((n + BM - 1) / BM + 1) * ntn;
+    if (grid > want) grid = want;
+    if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
+    int only = -1;
+    void* args[] = {&ctx->tmap_wh, &ctx->tmap_wx, &p, &only};
+    TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc<kG>, dim3(grid), dim3(kThreads), args,
+                                             C::kSmemBytes, stream));
+    ctx->launches += 1;
+    return TREELSTM_OK;
+  }
+  for (int lvl = 0; lvl < n_levels_host; ++lvl) {
+    const int w = level_offset_host[lvl + 1] - level_offset_host[lvl];
+    const int tiles = ((w + BM - 1) / BM) * ntn;
+    if (tiles <= 0) continue;
+    k_fwd_tc<kG><<<tiles, kThreads, C::kSmemBytes, stream>>>(ctx->tmap_wh, ctx->tmap_wx, p, lvl);
+    ctx->launches += 1;
+  }
+  TL_CUDA(ctx, cudaGetLastError());
+  return TREELSTM_OK;
+}
+
+}  // namespace tl

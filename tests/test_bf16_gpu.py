@@ -1,0 +1,95 @@
+"""Parity of the bf16 tensor-core forward (tcgen05 path, through the C ABI) against the fp64 oracle:
+schedule bit-exact, h and c within 3e-2 max-abs; against the oracle with the same operands rounded
+to bf16 the agreement must be much tighter (separates operand rounding from kernel mistakes)."""
+import numpy as np
+import pytest
+
+from oracle import treelstm_oracle as orc
+from paper_1809_00832_b200 import binding, forests as fg
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+MODES = [binding.PER_LEVEL, binding.PERSISTENT]
+TIGHT = 2e-3        # vs. the oracle fed bf16-rounded operands: only accumulation order, fast
+                    # activations and the bf16 rounding of h at slightly different values remain
+
+
+def _check(params, forest, flags, full_ref=None):
+    model = util.make_model(params, "bf16")
+    res = util.gpu_forward(model, forest, flags)
+    status, _, level, order, off = orc.schedule(forest.left, forest.right)
+    util.check_schedule(res, dict(level=level, order=order, level_offset=off), forest.n_nodes)
+    if full_ref is None:
+        h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
+    else:
+        h, c = full_ref["h"], full_ref["c"]
+    assert util.max_abs(res["h"], h) < util.TOL["bf16"]
+    assert util.max_abs(res["c"], c) < util.TOL["bf16"]
+    return res
+
+
+@pytest.mark.parametrize("flags", MODES)
+@pytest.mark.parametrize("H,E", [(64, 64), (32, 20), (150, 300), (72, 130)])
+def test_bf16_small_matches_oracle_and_rounded_oracle(H, E, flags):
+    rng = np.random.default_rng(H + E)
+    params = fg.draw_params(rng, H, E, 500, emb_dist="normal", emb_scale=0.3, w_scale=0.2)
+    forest = fg.random_forest(rng, 9, 1, 40, 500)          # > 128 leaves: several row tiles + ragged tail
+    forest, _ = fg.permute_node_ids(forest, rng)
+    res = _check(params, forest, flags)
+    hr, cr, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
+                                      operand_round=orc.round_to_bf16)
+    assert util.max_abs(res["h"], hr) < TIGHT
+    assert util.max_abs(res["c"], cr) < TIGHT
+
+
+@pytest.mark.parametrize("flags", MODES)
+def test_bf16_batch256_matches_oracle(flags):
+    w = fg.make_workload("batch256_bf16", 0)
+    ref = util.oracle_forward_cached("batch256_bf16", 0)
+    _check(w.params, w.forest, flags, ref)
+
+
+@pytest.mark.parametrize("flags", MODES)
+def test_bf16_chains_match_oracle(flags):
+    """64 left chains of 64 leaves: 64 dependent wavefronts, error growth over depth stays bounded"""
+    w = fg.make_workload("chains64_bf16", 0)
+    ref = util.oracle_forward_cached("chains64_bf16", 0)
+    res = _check(w.params, w.forest, flags, ref)
+    assert res["n_levels"] == 64
+
+
+def test_bf16_balanced_full_size_sampled():
+    """16 balanced trees of 1024 leaves in the benchmark's launch configuration: schedule exact on
+    all nodes; states checked on two whole trees the oracle evaluates on their own."""
+    w = fg.make_workload("balanced1024_bf16", 0)
+    model = util.make_model(w.params, "bf16")
+    res = util.gpu_forward(model, w.forest, binding.PERSISTENT)
+    status, _, level, order, off = orc.schedule(w.forest.left, w.forest.right)
+    util.check_schedule(res, dict(level=level, order=order, level_offset=off), w.forest.n_nodes)
+    assert np.diff(off).tolist() == [16 * 1024 >> k for k in range(11)]
+    sample = [0, 11]
+    sub = fg.select_trees(w.forest, sample)
+    h, c, _ = orc.forward_recursive(sub.left, sub.right, sub.token, w.params.emb, w.params.W, w.params.b)
+    ids = np.nonzero(np.isin(w.forest.tree_of, sample))[0]
+    assert util.max_abs(res["h"][ids], h) < util.TOL["bf16"]
+    assert util.max_abs(res["c"][ids], c) < util.TOL["bf16"]
+    assert np.all(np.isfinite(res["h"])) and np.all(np.abs(res["h"]) < 1.0)
+
+
+def test_bf16_forward_then_fp32_backward():
+    """a bf16 forward keeps the gates; backward (fp32 arithmetic) then matches the oracle's gradients
+    to the accuracy the bf16 forward values allow"""
+    rng = np.random.default_rng(12)
+    params = fg.draw_params(rng, 64, 40, 300, emb_dist="normal", emb_scale=0.3, w_scale=0.1, n_classes=5)
+    forest = fg.random_forest(rng, 6, 2, 30, 300)
+    labels = rng.integers(0, 5, size=forest.n_nodes).astype(np.int32)
+    ref = orc.loss_and_gradients(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
+                                 params.Wc, params.bc, labels)
+    model = util.make_model(params, "bf16")
+    model.forward(util.to_dev(forest.left), util.to_dev(forest.right), util.to_dev(forest.token),
+                  flags=binding.PERSISTENT | binding.SAVE_FOR_BACKWARD)
+    g = model.backward(util.to_dev(labels), forest.n_leaves)
+    assert abs(float(g["loss"].item()) - ref["loss"]) < util.TOL["bf16"]
+    assert util.max_abs(g["dW"].cpu().numpy(), ref["dW"]) < util.TOL["bf16"]
+    assert util.max_abs(g["db"].cpu().numpy(), ref["db"]) < util.TOL["bf16"]
