@@ -73,6 +73,8 @@ typedef enum treelstm_status {
 #define TREELSTM_OPT_WAIT_LIMIT_CYCLES 2    /* upper bound of every device-side wait, in units of   */
                                             /* 1024 SM clock cycles                                  */
 #define TREELSTM_OPT_MAX_CTAS 3             /* cap on the persistent grid (0 = all co-resident CTAs) */
+#define TREELSTM_OPT_TIME_WAVEFRONT_KERNEL 4 /* 1: bracket the wavefront kernel launch(es) of each  */
+                                            /* forward with CUDA events (treelstm_last_kernel_ms)    */
 
 /*
  * treelstm_create - build a context for one set of parameters.
@@ -193,6 +195,14 @@ TREELSTM_API int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32
                           const int32_t* token, float* h, float* c, int32_t* level, int32_t* order,
                           int32_t* n_levels, int max_roots, int32_t* root_ids, float* root_h,
                           float* root_c, int32_t* n_roots, int flags, void* stream);
+
+/*
+ * treelstm_last_kernel_ms - device time of the wavefront kernel launch(es) of the last forward
+ * (the persistent kernel, or the per-level launches together), measured with CUDA events on the
+ * call's stream.  Needs TREELSTM_OPT_TIME_WAVEFRONT_KERNEL = 1 before that forward; waits for the
+ * kernel to finish.  ms [host][1] out.
+ */
+TREELSTM_API int treelstm_last_kernel_ms(treelstm_t* ctx, float* ms);
 
 /* Number of kernels the last forward / backward call on this context launched. */
 TREELSTM_API int treelstm_last_launch_count(const treelstm_t* ctx);

@@ -32,6 +32,7 @@ SAVE_FOR_BACKWARD = 2
 OPT_SCHED_SINGLE_CTA_MAX = 1
 OPT_WAIT_LIMIT_CYCLES = 2
 OPT_MAX_CTAS = 3
+OPT_TIME_WAVEFRONT_KERNEL = 4
 
 _vp = ctypes.c_void_p
 _i = ctypes.c_int
@@ -50,6 +51,7 @@ SIGNATURES = {
     "treelstm_backward": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "treelstm_forward_host": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp,
                                    _vp, _vp, _i, _vp]),
+    "treelstm_last_kernel_ms": (_i, [_vp, ctypes.POINTER(ctypes.c_float)]),
     "treelstm_last_launch_count": (_i, [_vp]),
     "treelstm_last_cuda_error": (_i, [_vp]),
     "treelstm_destroy": (_i, [_vp]),
@@ -261,6 +263,13 @@ class TreeLSTM:
         if rc != OK:
             raise TreeLSTMError(rc, "treelstm_forward_host")
         return out
+
+    def last_kernel_ms(self) -> float:
+        ms = ctypes.c_float()
+        rc = self.lib.treelstm_last_kernel_ms(self.handle, ctypes.byref(ms))
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_last_kernel_ms")
+        return float(ms.value)
 
     def last_launch_count(self) -> int:
         return int(self.lib.treelstm_last_launch_count(self.handle))

@@ -182,6 +182,13 @@ int treelstm_set_option(treelstm_t* ctx, int key, long long value) {
     case TREELSTM_OPT_MAX_CTAS:
       ctx->opt.max_ctas = value > 65535 ? 65535 : (int)value;
       return TREELSTM_OK;
+    case TREELSTM_OPT_TIME_WAVEFRONT_KERNEL:
+      if (value && !ctx->ev_begin) {
+        TL_CUDA(ctx, cudaEventCreate(&ctx->ev_begin));
+        TL_CUDA(ctx, cudaEventCreate(&ctx->ev_end));
+      }
+      ctx->opt.time_kernel = value != 0;
+      return TREELSTM_OK;
     default:
       return TREELSTM_ERR_INVALID_ARG;
   }
@@ -229,14 +236,28 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
     rc = read_levels(ctx);
     if (rc != TREELSTM_OK) { L.valid = false; return rc; }
   }
+  ctx->ev_valid = false;
+  if (ctx->opt.time_kernel) TL_CUDA(ctx, cudaEventRecord(ctx->ev_begin, s));
   if (ctx->precision == TREELSTM_BF16)
     rc = launch_forward_bf16(ctx, n_nodes, left, right, token, h, c, order, lvl_off,
                              ctx->host_level_offset, L.n_levels, flags, workspace, lay, s);
   else
     rc = launch_forward_fp32(ctx, n_nodes, left, right, token, h, c, order, lvl_off,
                              ctx->host_level_offset, L.n_levels, flags, workspace, lay, s);
+  if (ctx->opt.time_kernel && rc == TREELSTM_OK) {
+    TL_CUDA(ctx, cudaEventRecord(ctx->ev_end, s));
+    ctx->ev_valid = true;
+  }
   if (rc != TREELSTM_OK) L.valid = false;
   return rc;
+}
+
+int treelstm_last_kernel_ms(treelstm_t* ctx, float* ms) {
+  if (!ctx || !ms) return TREELSTM_ERR_INVALID_ARG;
+  if (!ctx->ev_valid) return TREELSTM_ERR_STATE;
+  TL_CUDA(ctx, cudaEventSynchronize(ctx->ev_end));
+  TL_CUDA(ctx, cudaEventElapsedTime(ms, ctx->ev_begin, ctx->ev_end));
+  return TREELSTM_OK;
 }
 
 int treelstm_status_sync(treelstm_t* ctx) {
@@ -347,6 +368,8 @@ int treelstm_destroy(treelstm_t* ctx) {
   if (ctx->host_level_offset) cudaFreeHost(ctx->host_level_offset);
   if (ctx->host_status) cudaFreeHost(ctx->host_status);
   free_host_path(ctx);
+  if (ctx->ev_begin) cudaEventDestroy(ctx->ev_begin);
+  if (ctx->ev_end) cudaEventDestroy(ctx->ev_end);
   delete ctx;
   return TREELSTM_OK;
 }

@@ -33,6 +33,7 @@ struct Options {
   int sched_single_cta_max = 49152;
   long long wait_limit_kcycles = 1 << 20;  // ~1e9 cycles, about half a second at 2 GHz
   int max_ctas = 0;
+  int time_kernel = 0;
 };
 
 constexpr int kRadixBins = 256;
@@ -100,6 +101,9 @@ struct treelstm {
     void* ws = nullptr;
     size_t ws_bytes = 0;
   } hp;
+
+  cudaEvent_t ev_begin = nullptr, ev_end = nullptr;  // around the wavefront kernel (optional)
+  bool ev_valid = false;
 
   int launches = 0;
   int cuda_error = 0;

@@ -514,6 +514,7 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   k_row_operands<<<(n + 255) / 256, 256, 0, stream>>>(n, order, left, right, token, const_cast<int*>(p.rowA),
                                                       const_cast<int*>(p.rowB), p.st);
   ctx->launches += 1;
+  if (ctx->opt.time_kernel) TL_CUDA(ctx, cudaEventRecord(ctx->ev_begin, stream));  // wavefront kernel only
   static bool attr_set = false;
   if (!attr_set) {
     TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc<kG>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
