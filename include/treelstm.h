@@ -197,6 +197,43 @@ TREELSTM_API int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32
                           float* root_c, int32_t* n_roots, int flags, void* stream);
 
 /*
+ * treelstm_schedule_static - the ready-set construction of treelstm_forward on its own, for
+ * callers that are not allowed to allocate device memory.  (The paper has no counterpart to this
+ * call; it exists for the sake of such callers only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a framework that owns all
+ * device memory through its own pool and forbids side allocations, in a process whose memory
+ * budget was fixed at start-up, or on a latency-critical path where an allocation (which may
+ * synchronise the whole device) is unacceptable.  Such a caller cannot create a context
+ * (treelstm_create copies the parameters into memory it allocates) and has nowhere to get the
+ * workspace treelstm_forward wants.  This call needs neither: it takes no context, and the
+ * scratch the scheduling kernel needs (caller links, sort buffers, control block - about 193 KB)
+ * lives in a fixed array inside the library's device image, present on every GPU that loads the
+ * library until the process exits.
+ *
+ *   n_nodes       0 .. TREELSTM_STATIC_MAX_NODES (16384); more returns TREELSTM_ERR_UNSUPPORTED
+ *                 and launches nothing.
+ *   left,right,token  [n_nodes] the forest, as for treelstm_forward; vocab bounds the leaf tokens.
+ *   level, order  [n_nodes] out;  level_offset [n_nodes + 2] out;  n_levels [1] out - the same
+ *                 values treelstm_forward reports.
+ *   status        [1] out (device): TREELSTM_OK, TREELSTM_ERR_INVALID_FOREST or
+ *                 TREELSTM_ERR_TOKEN_OUT_OF_RANGE as found by the kernel; read it after the stream
+ *                 has finished.  On an error the other outputs are unspecified.
+ * The call only enqueues work on `stream` (two small memory operations and one kernel); it never
+ * calls cudaMalloc, cudaFree or any routine that allocates.  The first call on each device looks
+ * up the device address of the built-in scratch array (with that device current); make that first
+ * call outside any stream capture.  All calls on a device share the one scratch array, and it keeps
+ * whatever the previous call left there - the call clears the parts that must start from zero
+ * itself - so two calls whose work overlaps on the GPU (different streams without ordering between
+ * them) corrupt each other: order them.
+ */
+#define TREELSTM_STATIC_MAX_NODES 16384
+TREELSTM_API int treelstm_schedule_static(int n_nodes, const int32_t* left, const int32_t* right,
+                                          const int32_t* token, int vocab, int32_t* level, int32_t* order,
+                                          int32_t* level_offset, int32_t* n_levels, int32_t* status,
+                                          void* stream);
+
+/*
  * treelstm_last_kernel_ms - device time of the wavefront kernel launch(es) of the last forward
  * (the persistent kernel, or the per-level launches together), measured with CUDA events on the
  * call's stream.  Needs TREELSTM_OPT_TIME_WAVEFRONT_KERNEL = 1 before that forward; waits for the

@@ -51,6 +51,7 @@ SIGNATURES = {
     "treelstm_backward": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "treelstm_forward_host": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp,
                                    _vp, _vp, _i, _vp]),
+    "treelstm_schedule_static": (_i, [_i, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "treelstm_last_kernel_ms": (_i, [_vp, ctypes.POINTER(ctypes.c_float)]),
     "treelstm_last_launch_count": (_i, [_vp]),
     "treelstm_last_cuda_error": (_i, [_vp]),
@@ -96,6 +97,22 @@ def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
 
 def _stream() -> ctypes.c_void_p:
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+STATIC_MAX_NODES = 16384
+
+
+def schedule_static(left: torch.Tensor, right: torch.Tensor, token: torch.Tensor, vocab: int, out: dict) -> int:
+    """treelstm_schedule_static: ready-set construction for callers that may not allocate device
+    memory.  Everything, outputs included, is passed in: `out` holds the caller's int32 CUDA tensors
+    level [n], order [n], level_offset [n + 2], n_levels [1] and status [1].  Neither this wrapper
+    nor the library allocates; the kernel's scratch is a fixed array inside the library.  Returns
+    the host-side return code (the device-side status lands in out["status"])."""
+    lib = load_library()
+    n = int(left.shape[0])
+    return int(lib.treelstm_schedule_static(n, _ptr(left), _ptr(right), _ptr(token), vocab, _ptr(out["level"]),
+                                            _ptr(out["order"]), _ptr(out["level_offset"]), _ptr(out["n_levels"]),
+                                            _ptr(out["status"]), _stream()))
 
 
 class TreeLSTM:

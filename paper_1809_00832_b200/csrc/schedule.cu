@@ -465,3 +465,60 @@ int launch_gather_roots(treelstm* ctx, int max_roots, int32_t* root_ids, float* 
 }
 
 }  // namespace tl
+
+// ------------------------------------------------------------------------------------------ //
+// Scheduling without any allocation: the scratch of the single-CTA scheduler in a fixed array of
+// the device image.  Layout: control block | parent | order_tmp | roots, each for
+// TREELSTM_STATIC_MAX_NODES nodes.
+// ------------------------------------------------------------------------------------------ //
+namespace {
+constexpr size_t kStaticNodes = TREELSTM_STATIC_MAX_NODES;
+constexpr size_t kStaticBytes = sizeof(tl::DevStatus) + 3 * sizeof(int) * kStaticNodes;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_scratch_addr[kMaxDevices] = {};   // device address per device ordinal
+}  // namespace
+
+extern "C" int treelstm_schedule_static(int n_nodes, const int32_t* left, const int32_t* right,
+                                        const int32_t* token, int vocab, int32_t* level,
+                                        int32_t* order, int32_t* level_offset, int32_t* n_levels,
+                                        int32_t* status, void* stream) {
+  using namespace tl;
+  if (n_nodes < 0 || vocab <= 0 || !level_offset || !n_levels || !status) return TREELSTM_ERR_INVALID_ARG;
+  if (n_nodes > 0 && (!left || !right || !token || !level || !order)) return TREELSTM_ERR_INVALID_ARG;
+  if (n_nodes > TREELSTM_STATIC_MAX_NODES) return TREELSTM_ERR_UNSUPPORTED;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TREELSTM_ERR_NO_DEVICE;
+  if (!g_static_scratch_addr[dev]) {
+    // In host code the array's name is only a handle for the symbol; the address the kernel can
+    // use has to be asked for, once per device, with that device current.
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return TREELSTM_ERR_CUDA;
+    if (cudaFuncSetAttribute(k_schedule_single, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(round_up_sz((size_t)kSchedSingleMaxNodes * 2, 16) +
+                                   sizeof(int) * kRadixBins * kSingleWarps)) != cudaSuccess)
+      return TREELSTM_ERR_CUDA;
+    g_static_scratch_addr[dev] = static_cast<unsigned char*>(addr);
+  }
+  unsigned char* base = g_static_scratch_addr[dev];
+  DevStatus* st = reinterpret_cast<DevStatus*>(base);
+  int* parent = reinterpret_cast<int*>(base + sizeof(DevStatus));
+  int* order_tmp = parent + kStaticNodes;
+  int* roots = order_tmp + kStaticNodes;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // the control block keeps the previous call's status and counts: it must start from zero
+  if (cudaMemsetAsync(st, 0, sizeof(DevStatus), s) != cudaSuccess) return TREELSTM_ERR_CUDA;
+  if (n_nodes > 0) {
+    const size_t smem = round_up_sz((size_t)n_nodes * 2, 16) + sizeof(int) * kRadixBins * kSingleWarps;
+    k_schedule_single<<<1, kSingleThreads, smem, s>>>(n_nodes, left, right, token, vocab, parent, level,
+                                                      order, order_tmp, level_offset, roots, st);
+    if (cudaGetLastError() != cudaSuccess) return TREELSTM_ERR_CUDA;
+  } else {
+    if (cudaMemsetAsync(level_offset, 0, sizeof(int32_t), s) != cudaSuccess) return TREELSTM_ERR_CUDA;
+  }
+  if (cudaMemcpyAsync(n_levels, &st->n_levels, sizeof(int), cudaMemcpyDeviceToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(status, &st->status, sizeof(int), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return TREELSTM_ERR_CUDA;
+  return TREELSTM_OK;
+}
