@@ -165,20 +165,22 @@ __device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
                                              long long limit_cycles, int* s_flag) {
   __syncthreads();
   if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(&st->barrier, 1u);
+    // release: everything this CTA wrote (ordered before by the CTA barrier) is visible to whoever
+    // acquires the counter afterwards
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&st->barrier) : "memory");
     long long t0 = clock64();
     int ok = 1;
-    while (*(volatile unsigned int*)&st->barrier < target) {
+    for (;;) {
+      unsigned int seen;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&st->barrier) : "memory");
+      if (seen >= target) break;
       if (*(volatile int*)&st->status != 0) { ok = 0; break; }
       if (clock64() - t0 > limit_cycles) {
         report(st, TREELSTM_ERR_TIMEOUT);
         ok = 0;
         break;
       }
-      __nanosleep(32);
     }
-    __threadfence();
     *s_flag = ok;
   }
   __syncthreads();

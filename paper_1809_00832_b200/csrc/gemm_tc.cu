@@ -13,8 +13,9 @@
 // pre-activations of a hidden unit sit in the same accumulator row slice and one thread (one
 // tensor-memory lane = one node) can finish the cell without any exchange.
 //
-// Warp roles (320 threads): warps 0-3 epilogue (tensor-memory lane quadrant = warp id), warp 4
-// TMA producer of W tiles, warp 5 MMA issuer + tensor-memory owner, warps 6-9 gather the A rows.
+// Warp roles (448 threads): warps 0-3 and 10-13 epilogue (tensor-memory lane quadrant = warp id
+// mod 4; the two sets split every unit group in halves), warp 4 TMA producer of W tiles, warp 5
+// MMA issuer + tensor-memory owner, warps 6-9 gather the A rows.
 #include "common.cuh"
 
 namespace tl {
@@ -22,24 +23,37 @@ namespace {
 
 constexpr int BM = 128;                 // nodes per tile (UMMA M)
 constexpr int kStages = 4;
-constexpr int kThreads = 320;
+constexpr int kThreads = 448;
 constexpr int kABytes = BM * 128;       // one K block (64 bf16) of 128 rows
 constexpr int kAccCols = 256;           // accumulator stage stride in tensor-memory columns
 constexpr unsigned kFull = 0xffffffffu;
+constexpr int kMaxG = 4;                // unit groups (of 8 hidden units) per tile: 1, 2 or 4
+constexpr int kGColsI = 40;             // packed rows per unit group, internal nodes (5 gates)
+constexpr int kGColsL = 24;             // packed rows per unit group, leaves (gates i, o, u)
+constexpr int kBBytes = kMaxG * kGColsI * 128;
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kCBytes = BM * 2 * kMaxG * 8 * 4;   // staged child cell states: 128 rows x 2 x 32 fp32
+constexpr int kSmemBytes = kStages * kStageBytes + kCBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+static_assert(kBBytes % 1024 == 0 && (kGColsI * 128) % 1024 == 0 && (kGColsL * 128) % 1024 == 0,
+              "every TMA box lands on a 1024-byte boundary of the swizzle pattern");
 
-template <int G> struct Cfg {
-  static constexpr int kUnits = 8 * G;
-  static constexpr int NI = 40 * G;     // accumulator columns of an internal tile (5 gates)
-  static constexpr int NL = 24 * G;     // accumulator columns of a leaf tile (gates i, o, u)
-  static constexpr int kBBytes = NI * 128;
-  static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-  static_assert(NI % 16 == 0 && NL % 16 == 0 && NI <= 256, "UMMA N must be a multiple of 16, <= 256");
-  static_assert(kBBytes % 1024 == 0, "stage buffers stay 1024-byte aligned");
-};
+// How many unit groups a tile of this wavefront covers.  Narrow wavefronts are cut into many thin
+// tiles (all SMs get work, short MMA and epilogue per tile); wide ones into fat tiles (fewer
+// re-reads of the operand rows).  Cost model: rounds x (fixed latency + per-group work).
+__host__ __device__ inline int choose_groups_per_tile(int rows, int groups, int n_ctas) {
+  const int mt = (rows + BM - 1) / BM;
+  int best_g = 1, best_cost = 1 << 30;
+  for (int g = 1; g <= kMaxG; g <<= 1) {
+    const int tiles = mt * (groups / g);
+    const int rounds = (tiles + n_ctas - 1) / n_ctas;
+    const int cost = rounds * (4 + g);
+    if (cost <= best_cost) { best_cost = cost; best_g = g; }
+  }
+  return best_g;
+}
 
 struct TcParams {
-  int n, H, Hp, Ep;
+  int n, H, Hp, Ep, sched_ctas;
   const int *order, *rowA, *rowB, *level_offset;
   const __nv_bfloat16* emb_bf;
   __nv_bfloat16* hb;
@@ -122,6 +136,10 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* v) {
                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
                : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t* v) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the
@@ -141,27 +159,21 @@ __device__ __forceinline__ uint32_t umma_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
-__device__ __forceinline__ float sigmoid_fast(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
-__device__ __forceinline__ float tanh_fast(float x) { return 2.0f * sigmoid_fast(2.0f * x) - 1.0f; }
-
-__device__ __forceinline__ void ld_row8(const float* p, bool vec, float* out) {
-  if (vec) {
-    const float4 a = __ldcg(reinterpret_cast<const float4*>(p));
-    const float4 b = __ldcg(reinterpret_cast<const float4*>(p) + 1);
-    out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
-    out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
-  } else {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) out[j] = __ldcg(p + j);
-  }
+// Activations of the bf16 path.  tanh.approx has an absolute error of about 5e-4, far inside the
+// 3e-2 budget of this path (the operands are already rounded to 8 mantissa bits).
+__device__ __forceinline__ float act_tanh(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
-__device__ __forceinline__ void st_row8(float* p, bool vec, int count, const float* v) {
-  if (vec && count == 8) {
-    reinterpret_cast<float4*>(p)[0] = make_float4(v[0], v[1], v[2], v[3]);
-    reinterpret_cast<float4*>(p)[1] = make_float4(v[4], v[5], v[6], v[7]);
+__device__ __forceinline__ float act_sigmoid(float x) { return fmaf(0.5f, act_tanh(0.5f * x), 0.5f); }
+
+__device__ __forceinline__ void st_row4(float* p, bool vec, int count, const float* v) {
+  if (vec && count == 4) {
+    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
   } else {
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
+    for (int j = 0; j < 4; ++j)
       if (j < count) p[j] = v[j];
   }
 }
@@ -169,16 +181,16 @@ __device__ __forceinline__ void st_row8(float* p, bool vec, int count, const flo
 // ---- the kernel -------------------------------------------------------------------------------- //
 // only_level >= 0: process that wavefront only (one launch per level).  only_level < 0: all
 // wavefronts, separated by the bounded grid barrier (cooperative launch).
-template <int G>
 __global__ void __launch_bounds__(kThreads, 1)
 k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CUtensorMap tmap_wx,
          TcParams p, int only_level) {
-  using C = Cfg<G>;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
   unsigned char* tiles_ptr = smem_raw + (tiles_addr - raw_addr);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + kStages * C::kStageBytes);
+  const uint32_t cstage_addr = tiles_addr + kStages * kStageBytes;
+  const unsigned char* cstage_ptr = tiles_ptr + kStages * kStageBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + kStages * kStageBytes + kCBytes);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
@@ -195,7 +207,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
 
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 128 + 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -206,7 +218,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   const uint32_t tmem_base = *s_tmem;
 
   const int Hp = p.Hp, H = p.H;
-  const int ntn = Hp / C::kUnits;                    // column tiles per row tile
+  const int groups = Hp / kUnitGroup;
   const int kb_leaf = p.Ep / kKBlock, kb_int = 2 * Hp / kKBlock, kb_half = Hp / kKBlock;
   const bool vec = (H % 4) == 0;
 
@@ -220,9 +232,13 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   for (int lvl = lvl_begin; lvl < lvl_end; ++lvl) {   // uniform trip count: barriers inside
     const int begin = p.level_offset[lvl], end = p.level_offset[lvl + 1];
     const bool leaf = lvl == 0;
+    const int G = choose_groups_per_tile(end - begin, groups, p.sched_ctas);
+    const int ntn = groups / G;                      // column tiles per row tile
     const int tiles = ((end - begin + BM - 1) / BM) * ntn;
     const int kblocks = leaf ? kb_leaf : kb_int;
-    const int ncols = leaf ? C::NL : C::NI;
+    const int gcols = leaf ? kGColsL : kGColsI;
+    const int ncols = G * gcols;                     // accumulator columns in use
+    const int ncols_mma = (ncols + 15) & ~15;        // UMMA N (columns past ncols are never read)
 
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
       const int row0 = begin + (t / ntn) * BM, nt = t % ntn;
@@ -235,8 +251,9 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
           for (int kb = 0; kb < kblocks; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1, s_abort, p.wait_limit, p.st)) { alive = false; break; }
             mbar_arrive_expect_tx(full_bar(stage), bytes);
-            tma_load_2d(tiles_addr + stage * C::kStageBytes + kABytes, map, kb * kKBlock, nt * ncols,
-                        full_bar(stage));
+            for (int g = 0; g < G; ++g)              // one box = the packed rows of one unit group
+              tma_load_2d(tiles_addr + stage * kStageBytes + kABytes + (uint32_t)(g * gcols) * 128u, map,
+                          kb * kKBlock, (nt * G + g) * gcols, full_bar(stage));
             if (++stage == kStages) { stage = 0; phase ^= 1; }
           }
         }
@@ -247,12 +264,12 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
           if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + acc * kAccCols;
-          const uint32_t idesc = umma_idesc(ncols);
+          const uint32_t idesc = umma_idesc(ncols_mma);
           for (int kb = 0; kb < kblocks && alive; ++kb) {
             if (!mbar_wait(full_bar(stage), phase, s_abort, p.wait_limit, p.st)) { alive = false; break; }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             tc_fence_after();
-            const uint32_t a_addr = tiles_addr + stage * C::kStageBytes;
+            const uint32_t a_addr = tiles_addr + stage * kStageBytes;
             const uint64_t a_desc = umma_desc(a_addr), b_desc = umma_desc(a_addr + kABytes);
 #pragma unroll
             for (int k = 0; k < kKBlock / 16; ++k)   // UMMA K = 16 bf16 = 32 bytes = 2 descriptor units
@@ -263,109 +280,149 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
           if (alive) umma_commit(tfull_bar(acc));    // accumulator complete
         }
         ++acc_iter;
-      } else if (warp >= 6) {
+      } else if (warp >= 6 && warp < 10) {
         // ---------------- A row gather (cp.async into the swizzled tile) ----------------
-        const int r = tid - 6 * 32;                  // tile row owned by this thread
-        const int row = row0 + r;
-        const bool valid = row < end;
-        const int ia = valid ? p.rowA[row] : 0, ib = valid ? p.rowB[row] : 0;
-        const uint32_t nbytes = valid ? 16u : 0u;    // rows past the wavefront are zero-filled
-        const uint32_t row_off = (uint32_t)(r >> 3) * 1024u + (uint32_t)(r & 7) * 128u;
+        // Eight consecutive lanes copy the eight 16-byte chunks of one row's 128-byte K block, so a
+        // warp instruction touches 4 whole lines instead of 32 partial ones.  Thread (rsel, sub)
+        // serves rows rsel, rsel + 16, ... of the tile.
+        const int gtid = tid - 6 * 32, sub = gtid & 7, rsel = gtid >> 3;
+        int ia[8], ib[8];
+        uint32_t valid_mask = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int row = row0 + j * 16 + rsel;
+          const bool valid = row < end;
+          ia[j] = valid ? p.rowA[row] : 0;
+          ib[j] = (valid && !leaf) ? p.rowB[row] : 0;
+          valid_mask |= (valid ? 1u : 0u) << j;
+        }
+        const uint32_t dst_off = (uint32_t)(rsel >> 3) * 1024u + (uint32_t)(rsel & 7) * 128u +
+                                 (uint32_t)((sub ^ (rsel & 7)) << 4);
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1, s_abort, p.wait_limit, p.st)) { alive = false; break; }
-          const __nv_bfloat16* src;
-          if (leaf) src = p.emb_bf + (size_t)ia * p.Ep + kb * kKBlock;
-          else if (kb < kb_half) src = p.hb + (size_t)ia * Hp + kb * kKBlock;
-          else src = p.hb + (size_t)ib * Hp + (kb - kb_half) * kKBlock;
-          const uint32_t dst = tiles_addr + stage * C::kStageBytes + row_off;
+          const uint32_t dst = tiles_addr + stage * kStageBytes + dst_off;
+          const bool second = !leaf && kb >= kb_half;
+          const size_t col = (size_t)((second ? kb - kb_half : kb) * kKBlock + sub * 8);
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch)
-            cp_async16(dst + (uint32_t)((ch ^ (r & 7)) << 4), src + ch * 8, nbytes);
+          for (int j = 0; j < 8; ++j) {
+            const __nv_bfloat16* src = leaf ? p.emb_bf + (size_t)ia[j] * p.Ep + col
+                                            : p.hb + (size_t)(second ? ib[j] : ia[j]) * Hp + col;
+            cp_async16(dst + (uint32_t)j * 2048u, src, (valid_mask >> j) & 1u ? 16u : 0u);
+          }
           cp_async_arrive_noinc(full_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       } else {
         // ---------------- epilogue: drain tensor memory, finish the cell ----------------
-        const int r = warp * 32 + lane;
+        // Two sets of four warps; set e takes hidden units [4e, 4e + 4) of every unit group.  A
+        // warp may only read the tensor-memory lanes of quadrant (warp id mod 4).
+        const int e = warp < 4 ? 0 : 1;
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;
         const int row = row0 + r;
         const bool valid = row < end;
         const int node = valid ? p.order[row] : 0;
         const int il = (valid && !leaf) ? p.rowA[row] : 0, ir = (valid && !leaf) ? p.rowB[row] : 0;
+        // stage the children's cell states for this thread's row while the MMAs run
+        const bool staged = !leaf && vec && (nt + 1) * G * 8 <= H;
+        const uint32_t my_c = cstage_addr + (uint32_t)r * 256u;
+        if (staged) {
+          const float* sl = p.c + (size_t)il * H + nt * G * 8;
+          const float* sr = p.c + (size_t)ir * H + nt * G * 8;
+          const uint32_t nb = valid ? 16u : 0u;
+          for (int ch = e; ch < 2 * G; ch += 2) {
+            cp_async16(my_c + (uint32_t)((ch ^ (r & 7)) << 4), sl + ch * 4, nb);
+            cp_async16(my_c + (uint32_t)(((8 + ch) ^ (r & 7)) << 4), sr + ch * 4, nb);
+          }
+        }
+        const float* bias = (leaf ? p.bp_x : p.bp_h) + nt * ncols + 4 * e;
+        const int ngates = leaf ? 3 : 5;
+        float4 bnext[5];
+#pragma unroll
+        for (int q = 0; q < 5; ++q)
+          if (q < ngates) bnext[q] = __ldg(reinterpret_cast<const float4*>(bias + 8 * q));
         const uint32_t acc = acc_iter & 1, acc_phase = (acc_iter >> 1) & 1;
         if (!mbar_wait(tfull_bar(acc), acc_phase, s_abort, p.wait_limit, p.st)) alive = false;
         alive = __all_sync(kFull, alive);
+        asm volatile("cp.async.wait_all;" ::: "memory");
         if (alive) {
           tc_fence_after();
-          const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(warp * 32) << 16);
-          const float* bias = leaf ? p.bp_x + nt * C::NL : p.bp_h + nt * C::NI;
+          const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(quad * 32) << 16) + 4u * e;
 #pragma unroll 1
           for (int g = 0; g < G; ++g) {
-            uint32_t v[40];
-            const int gcols = leaf ? 24 : 40;
+            uint32_t v[20];
             const uint32_t col0 = (uint32_t)(g * gcols);
             if (leaf) {
 #pragma unroll
-              for (int q = 0; q < 3; ++q) tmem_ld8(taddr + col0 + 8 * q, v + 8 * q);
+              for (int q = 0; q < 3; ++q) tmem_ld4(taddr + col0 + 8 * q, v + 4 * q);
             } else {
 #pragma unroll
-              for (int q = 0; q < 5; ++q) tmem_ld8(taddr + col0 + 8 * q, v + 8 * q);
+              for (int q = 0; q < 5; ++q) tmem_ld4(taddr + col0 + 8 * q, v + 4 * q);
+            }
+            float4 bcur[5];
+#pragma unroll
+            for (int q = 0; q < 5; ++q) bcur[q] = bnext[q];
+            if (g + 1 < G) {
+#pragma unroll
+              for (int q = 0; q < 5; ++q)
+                if (q < ngates) bnext[q] = __ldg(reinterpret_cast<const float4*>(bias + (g + 1) * gcols + 8 * q));
             }
             tmem_ld_wait();
             if (valid) {
-              const int u0 = (nt * G + g) * 8;
-              const int count = min(8, H - u0);     // real (unpadded) units in this group
-              float cl[8] = {}, cr[8] = {}, hv[8], cv[8], gi[8], gfl[8], gfr[8], go[8], gu[8];
-              const float* bg = bias + g * gcols;
-              if (!leaf && count > 0) {
-                if (count == 8) {
-                  ld_row8(p.c + (size_t)il * H + u0, vec, cl);
-                  ld_row8(p.c + (size_t)ir * H + u0, vec, cr);
-                } else {
+              const int u0 = (nt * G + g) * 8 + 4 * e;
+              const int count = min(4, H - u0);     // real (unpadded) units among these four
+              float cl[4] = {}, cr[4] = {}, hv[4], cv[4], gi[4], gfl[4], gfr[4], go[4], gu[4];
+              if (staged) {
+                const unsigned char* mine = cstage_ptr + r * 256;
+                const float4 a = *reinterpret_cast<const float4*>(mine + (((2 * g + e) ^ (r & 7)) << 4));
+                const float4 b = *reinterpret_cast<const float4*>(mine + (((8 + 2 * g + e) ^ (r & 7)) << 4));
+                cl[0] = a.x; cl[1] = a.y; cl[2] = a.z; cl[3] = a.w;
+                cr[0] = b.x; cr[1] = b.y; cr[2] = b.z; cr[3] = b.w;
+              } else if (!leaf && count > 0) {
 #pragma unroll
-                  for (int j = 0; j < 8; ++j) {
-                    cl[j] = j < count ? __ldcg(p.c + (size_t)il * H + u0 + j) : 0.f;
-                    cr[j] = j < count ? __ldcg(p.c + (size_t)ir * H + u0 + j) : 0.f;
-                  }
+                for (int j = 0; j < 4; ++j) {
+                  cl[j] = j < count ? __ldcg(p.c + (size_t)il * H + u0 + j) : 0.f;
+                  cr[j] = j < count ? __ldcg(p.c + (size_t)ir * H + u0 + j) : 0.f;
                 }
               }
+              const float* bq = reinterpret_cast<const float*>(bcur);
 #pragma unroll
-              for (int j = 0; j < 8; ++j) {
+              for (int j = 0; j < 4; ++j) {
                 if (leaf) {
-                  gi[j] = sigmoid_fast(__uint_as_float(v[j]) + __ldg(bg + j));
-                  go[j] = sigmoid_fast(__uint_as_float(v[8 + j]) + __ldg(bg + 8 + j));
-                  gu[j] = tanh_fast(__uint_as_float(v[16 + j]) + __ldg(bg + 16 + j));
+                  gi[j] = act_sigmoid(__uint_as_float(v[j]) + bq[j]);
+                  go[j] = act_sigmoid(__uint_as_float(v[4 + j]) + bq[4 + j]);
+                  gu[j] = act_tanh(__uint_as_float(v[8 + j]) + bq[8 + j]);
                   gfl[j] = gfr[j] = 0.f;
                   cv[j] = gi[j] * gu[j];
                 } else {
-                  gi[j] = sigmoid_fast(__uint_as_float(v[j]) + __ldg(bg + j));
-                  gfl[j] = sigmoid_fast(__uint_as_float(v[8 + j]) + __ldg(bg + 8 + j));
-                  gfr[j] = sigmoid_fast(__uint_as_float(v[16 + j]) + __ldg(bg + 16 + j));
-                  go[j] = sigmoid_fast(__uint_as_float(v[24 + j]) + __ldg(bg + 24 + j));
-                  gu[j] = tanh_fast(__uint_as_float(v[32 + j]) + __ldg(bg + 32 + j));
+                  gi[j] = act_sigmoid(__uint_as_float(v[j]) + bq[j]);
+                  gfl[j] = act_sigmoid(__uint_as_float(v[4 + j]) + bq[4 + j]);
+                  gfr[j] = act_sigmoid(__uint_as_float(v[8 + j]) + bq[8 + j]);
+                  go[j] = act_sigmoid(__uint_as_float(v[12 + j]) + bq[12 + j]);
+                  gu[j] = act_tanh(__uint_as_float(v[16 + j]) + bq[16 + j]);
                   cv[j] = gi[j] * gu[j] + gfl[j] * cl[j] + gfr[j] * cr[j];
                 }
-                hv[j] = go[j] * tanh_fast(cv[j]);
+                hv[j] = go[j] * act_tanh(cv[j]);
               }
               // bf16 copy of h feeds the next wavefront's gather; padded units are written as 0
-              uint32_t packed[4];
+              uint32_t packed[2];
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
+              for (int j = 0; j < 2; ++j) {
                 const float lo = 2 * j < count ? hv[2 * j] : 0.f, hi = 2 * j + 1 < count ? hv[2 * j + 1] : 0.f;
                 __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
                 packed[j] = *reinterpret_cast<uint32_t*>(&b2);
               }
-              *reinterpret_cast<uint4*>(p.hb + (size_t)node * Hp + u0) =
-                  make_uint4(packed[0], packed[1], packed[2], packed[3]);
+              *reinterpret_cast<uint2*>(p.hb + (size_t)node * Hp + u0) = make_uint2(packed[0], packed[1]);
               if (count > 0) {
-                st_row8(p.h + (size_t)node * H + u0, vec, count, hv);
-                st_row8(p.c + (size_t)node * H + u0, vec, count, cv);
+                st_row4(p.h + (size_t)node * H + u0, vec, count, hv);
+                st_row4(p.c + (size_t)node * H + u0, vec, count, cv);
                 if (p.gates) {
                   float* gp = p.gates + (size_t)node * 5 * H + u0;
-                  st_row8(gp, vec, count, gi);
-                  st_row8(gp + H, vec, count, gfl);
-                  st_row8(gp + 2 * H, vec, count, gfr);
-                  st_row8(gp + 3 * H, vec, count, go);
-                  st_row8(gp + 4 * H, vec, count, gu);
+                  st_row4(gp, vec, count, gi);
+                  st_row4(gp + H, vec, count, gfl);
+                  st_row4(gp + 2 * H, vec, count, gfr);
+                  st_row4(gp + 3 * H, vec, count, go);
+                  st_row4(gp + 4 * H, vec, count, gu);
                 }
               }
             }
@@ -471,7 +528,6 @@ int make_tmap(treelstm* ctx, CUtensorMap* map, void* base, uint64_t inner, uint6
   return TREELSTM_OK;
 }
 
-constexpr int kG = 4;   // unit groups per tile: 32 hidden units, 160 accumulator columns
 
 }  // namespace
 
@@ -481,9 +537,9 @@ int pack_weights_bf16(treelstm* ctx, cudaStream_t stream) {
   k_pack_embedding<<<1024, 256, 0, stream>>>(ctx->vocab, ctx->E, ctx->Ep, ctx->emb, ctx->emb_bf);
   TL_CUDA(ctx, cudaGetLastError());
   const int groups = ctx->Hp / kUnitGroup;
-  int rc = make_tmap(ctx, &ctx->tmap_wh, ctx->Wp_h, 2 * (uint64_t)ctx->Hp, (uint64_t)groups * 40, Cfg<kG>::NI);
+  int rc = make_tmap(ctx, &ctx->tmap_wh, ctx->Wp_h, 2 * (uint64_t)ctx->Hp, (uint64_t)groups * kGColsI, kGColsI);
   if (rc != TREELSTM_OK) return rc;
-  rc = make_tmap(ctx, &ctx->tmap_wx, ctx->Wp_x, (uint64_t)ctx->Ep, (uint64_t)groups * 24, Cfg<kG>::NL);
+  rc = make_tmap(ctx, &ctx->tmap_wx, ctx->Wp_x, (uint64_t)ctx->Ep, (uint64_t)groups * kGColsL, kGColsL);
   if (rc != TREELSTM_OK) return rc;
   ctx->have_tmaps = true;
   return TREELSTM_OK;
@@ -494,11 +550,10 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
                         const int32_t* level_offset_dev, const int32_t* level_offset_host,
                         int n_levels_host, int flags, void* ws, const WsLayout& lay,
                         cudaStream_t stream) {
-  using C = Cfg<kG>;
   if (!ctx->have_tmaps) return TREELSTM_ERR_STATE;
   char* base = static_cast<char*>(ws);
   TcParams p;
-  p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep;
+  p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep; p.sched_ctas = ctx->sm_count;
   p.order = order;
   p.rowA = reinterpret_cast<int*>(base + lay.pending);     // dependency counters are dead by now
   p.rowB = reinterpret_cast<int*>(base + lay.order_tmp);
@@ -517,27 +572,27 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   if (ctx->opt.time_kernel) TL_CUDA(ctx, cudaEventRecord(ctx->ev_begin, stream));  // wavefront kernel only
   static bool attr_set = false;
   if (!attr_set) {
-    TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc<kG>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+    TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     attr_set = true;
   }
-  const int ntn = ctx->Hp / C::kUnits;
+  const int groups = ctx->Hp / kUnitGroup;
   if (flags & TREELSTM_PERSISTENT) {
     int grid = ctx->sm_count;                       // one CTA per SM (shared and tensor memory)
-    const int want = ((n + BM - 1) / BM + 1) * ntn;
+    const int want = ((n + BM - 1) / BM + 1) * groups;   // never more CTAs than the thinnest tiling has tiles
     if (grid > want) grid = want;
     if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
     int only = -1;
     void* args[] = {&ctx->tmap_wh, &ctx->tmap_wx, &p, &only};
-    TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc<kG>, dim3(grid), dim3(kThreads), args,
-                                             C::kSmemBytes, stream));
+    TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc, dim3(grid), dim3(kThreads), args,
+                                             kSmemBytes, stream));
     ctx->launches += 1;
     return TREELSTM_OK;
   }
   for (int lvl = 0; lvl < n_levels_host; ++lvl) {
     const int w = level_offset_host[lvl + 1] - level_offset_host[lvl];
-    const int tiles = ((w + BM - 1) / BM) * ntn;
-    if (tiles <= 0) continue;
-    k_fwd_tc<kG><<<tiles, kThreads, C::kSmemBytes, stream>>>(ctx->tmap_wh, ctx->tmap_wx, p, lvl);
+    if (w <= 0) continue;
+    const int tiles = ((w + BM - 1) / BM) * (groups / choose_groups_per_tile(w, groups, p.sched_ctas));
+    k_fwd_tc<<<tiles, kThreads, kSmemBytes, stream>>>(ctx->tmap_wh, ctx->tmap_wx, p, lvl);
     ctx->launches += 1;
   }
   TL_CUDA(ctx, cudaGetLastError());
