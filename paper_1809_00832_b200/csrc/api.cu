@@ -18,6 +18,8 @@ WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward) {
   L.level_offset = take(4 * (nn + 2));
   L.roots = take(4 * nn);
   L.table = take(4 * (size_t)kRadixBins * ((nn + kRadixChunk - 1) / kRadixChunk));
+  L.rowA = take(4 * nn);
+  L.rowB = take(4 * nn);
   L.hb = off;
   if (ctx->precision == TREELSTM_BF16) L.hb = take(2 * nn * (size_t)ctx->Hp);
   L.gates = L.dh = L.dc = L.dz = L.tok_slot = off;
@@ -223,11 +225,9 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
   L.h = h; L.c = c; L.level = level; L.order = order; L.level_offset = lvl_off;
   L.ws = workspace; L.lay = lay; L.stream = s; L.host_levels_valid = false; L.n_levels = 0;
 
-  TL_CUDA(ctx, cudaMemsetAsync(base + lay.status, 0, sizeof(DevStatus), s));
-  int rc = launch_schedule(ctx, n_nodes, left, right, token, level, order, lvl_off, workspace, lay, s);
+  int rc = launch_schedule(ctx, n_nodes, left, right, token, level, order, lvl_off, n_levels, workspace,
+                           lay, s);
   if (rc != TREELSTM_OK) return rc;
-  DevStatus* st = reinterpret_cast<DevStatus*>(base + lay.status);
-  TL_CUDA(ctx, cudaMemcpyAsync(n_levels, &st->n_levels, sizeof(int), cudaMemcpyDeviceToDevice, s));
   L.valid = true;
   if (n_nodes == 0) return TREELSTM_OK;
 

@@ -25,12 +25,12 @@ static_assert(sizeof(DevStatus) == 256, "control block is one 256-byte line grou
 
 // Offsets (bytes) of the regions inside the workspace for a forest of up to n nodes.
 struct WsLayout {
-  size_t status, parent, pending, order_tmp, level_offset, roots, table, hb, gates, dh, dc, dz,
-      tok_slot, total;
+  size_t status, parent, pending, order_tmp, level_offset, roots, table, rowA, rowB, hb, gates, dh,
+      dc, dz, tok_slot, total;
 };
 
 struct Options {
-  int sched_single_cta_max = 49152;
+  int sched_single_cta_max = 32768;
   long long wait_limit_kcycles = 1 << 20;  // ~1e9 cycles, about half a second at 2 GHz
   int max_ctas = 0;
   int time_kernel = 0;
@@ -38,7 +38,7 @@ struct Options {
 
 constexpr int kRadixBins = 256;
 constexpr int kRadixChunk = 1024;        // items per single-warp CTA of the multi-CTA sort
-constexpr int kSchedSingleMaxNodes = 49152;
+constexpr int kSchedSingleMaxNodes = 32768;
 
 // Padded sizes of the tensor-core path: hidden units in groups of 8 (one packed weight group =
 // 5 gates x 8 units = 40 rows), K blocks of 64 bf16 (one 128-byte swizzle span).
@@ -116,7 +116,7 @@ WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward);
 // schedule.cu: enqueue the on-device ready-set construction.  Returns a treelstm_status.
 int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
                     const int32_t* token, int32_t* level, int32_t* order, int32_t* level_offset,
-                    void* ws, const WsLayout& lay, cudaStream_t stream);
+                    int32_t* n_levels_out, void* ws, const WsLayout& lay, cudaStream_t stream);
 
 // cell_fp32.cu
 int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t* right,

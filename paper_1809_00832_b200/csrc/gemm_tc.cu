@@ -22,7 +22,7 @@ namespace tl {
 namespace {
 
 constexpr int BM = 128;                 // nodes per tile (UMMA M)
-constexpr int kStages = 4;
+constexpr int kMaxStages = 8;
 constexpr int kThreads = 448;
 constexpr int kABytes = BM * 128;       // one K block (64 bf16) of 128 rows
 constexpr int kAccCols = 256;           // accumulator stage stride in tensor-memory columns
@@ -31,9 +31,9 @@ constexpr int kMaxG = 4;                // unit groups (of 8 hidden units) per t
 constexpr int kGColsI = 40;             // packed rows per unit group, internal nodes (5 gates)
 constexpr int kGColsL = 24;             // packed rows per unit group, leaves (gates i, o, u)
 constexpr int kBBytes = kMaxG * kGColsI * 128;
-constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kRingBytes = kMaxStages * (kABytes + kGColsI * 128);   // 8 stages of the thinnest tile
 constexpr int kCBytes = BM * 2 * kMaxG * 8 * 4;   // staged child cell states: 128 rows x 2 x 32 fp32
-constexpr int kSmemBytes = kStages * kStageBytes + kCBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kSmemBytes = kRingBytes + kCBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 static_assert(kBBytes % 1024 == 0 && (kGColsI * 128) % 1024 == 0 && (kGColsL * 128) % 1024 == 0,
               "every TMA box lands on a 1024-byte boundary of the swizzle pattern");
 
@@ -188,25 +188,25 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
   unsigned char* tiles_ptr = smem_raw + (tiles_addr - raw_addr);
-  const uint32_t cstage_addr = tiles_addr + kStages * kStageBytes;
-  const unsigned char* cstage_ptr = tiles_ptr + kStages * kStageBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + kStages * kStageBytes + kCBytes);
+  const uint32_t cstage_addr = tiles_addr + kRingBytes;
+  const unsigned char* cstage_ptr = tiles_ptr + kRingBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + kRingBytes + kCBytes);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 4);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   int* s_flag = const_cast<int*>(s_abort) + 1;
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
-  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
-  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + 2 + a); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (ld_volatile(&p.st->status) != 0) return;      // schedule failed: nothing to evaluate
   const int n_levels = p.st->n_levels;
 
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 128 + 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 128 + 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -223,7 +223,9 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   const bool vec = (H % 4) == 0;
 
   // pipeline positions; every role walks the same tile sequence, so they stay in step
-  uint32_t stage = 0, phase = 0;        // smem ring (producers and MMA)
+  // The ring is re-cut at every wavefront (thin tiles leave room for more stages); each mbarrier
+  // keeps its own phase, tracked per stage in a bit mask.
+  uint32_t stage = 0, phase_bits = 0;   // smem ring (producers and MMA)
   uint32_t acc_iter = 0;                // accumulator ring (MMA and epilogue)
   bool alive = true;
 
@@ -239,6 +241,9 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
     const int gcols = leaf ? kGColsL : kGColsI;
     const int ncols = G * gcols;                     // accumulator columns in use
     const int ncols_mma = (ncols + 15) & ~15;        // UMMA N (columns past ncols are never read)
+    const uint32_t stage_bytes = kABytes + (uint32_t)G * kGColsI * 128u;
+    const uint32_t n_stages = min((uint32_t)kMaxStages, (uint32_t)kRingBytes / stage_bytes);
+    stage = 0;
 
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
       const int row0 = begin + (t / ntn) * BM, nt = t % ntn;
@@ -249,12 +254,16 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
           const CUtensorMap* map = leaf ? &tmap_wx : &tmap_wh;
           const uint32_t bytes = (uint32_t)ncols * 128u;
           for (int kb = 0; kb < kblocks; ++kb) {
-            if (!mbar_wait(empty_bar(stage), phase ^ 1, s_abort, p.wait_limit, p.st)) { alive = false; break; }
+            if (!mbar_wait(empty_bar(stage), ((phase_bits >> stage) & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) {
+              alive = false;
+              break;
+            }
             mbar_arrive_expect_tx(full_bar(stage), bytes);
             for (int g = 0; g < G; ++g)              // one box = the packed rows of one unit group
-              tma_load_2d(tiles_addr + stage * kStageBytes + kABytes + (uint32_t)(g * gcols) * 128u, map,
+              tma_load_2d(tiles_addr + stage * stage_bytes + kABytes + (uint32_t)(g * gcols) * 128u, map,
                           kb * kKBlock, (nt * G + g) * gcols, full_bar(stage));
-            if (++stage == kStages) { stage = 0; phase ^= 1; }
+            phase_bits ^= 1u << stage;
+            if (++stage == n_stages) stage = 0;
           }
         }
       } else if (warp == 5) {
@@ -266,16 +275,20 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
           const uint32_t d_tmem = tmem_base + acc * kAccCols;
           const uint32_t idesc = umma_idesc(ncols_mma);
           for (int kb = 0; kb < kblocks && alive; ++kb) {
-            if (!mbar_wait(full_bar(stage), phase, s_abort, p.wait_limit, p.st)) { alive = false; break; }
+            if (!mbar_wait(full_bar(stage), (phase_bits >> stage) & 1u, s_abort, p.wait_limit, p.st)) {
+              alive = false;
+              break;
+            }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             tc_fence_after();
-            const uint32_t a_addr = tiles_addr + stage * kStageBytes;
+            const uint32_t a_addr = tiles_addr + stage * stage_bytes;
             const uint64_t a_desc = umma_desc(a_addr), b_desc = umma_desc(a_addr + kABytes);
 #pragma unroll
             for (int k = 0; k < kKBlock / 16; ++k)   // UMMA K = 16 bf16 = 32 bytes = 2 descriptor units
               umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
             umma_commit(empty_bar(stage));           // frees the smem stage when these MMAs retire
-            if (++stage == kStages) { stage = 0; phase ^= 1; }
+            phase_bits ^= 1u << stage;
+            if (++stage == n_stages) stage = 0;
           }
           if (alive) umma_commit(tfull_bar(acc));    // accumulator complete
         }
@@ -299,8 +312,11 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
         const uint32_t dst_off = (uint32_t)(rsel >> 3) * 1024u + (uint32_t)(rsel & 7) * 128u +
                                  (uint32_t)((sub ^ (rsel & 7)) << 4);
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1, s_abort, p.wait_limit, p.st)) { alive = false; break; }
-          const uint32_t dst = tiles_addr + stage * kStageBytes + dst_off;
+          if (!mbar_wait(empty_bar(stage), ((phase_bits >> stage) & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) {
+            alive = false;
+            break;
+          }
+          const uint32_t dst = tiles_addr + stage * stage_bytes + dst_off;
           const bool second = !leaf && kb >= kb_half;
           const size_t col = (size_t)((second ? kb - kb_half : kb) * kKBlock + sub * 8);
 #pragma unroll
@@ -310,7 +326,8 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
             cp_async16(dst + (uint32_t)j * 2048u, src, (valid_mask >> j) & 1u ? 16u : 0u);
           }
           cp_async_arrive_noinc(full_bar(stage));
-          if (++stage == kStages) { stage = 0; phase ^= 1; }
+          phase_bits ^= 1u << stage;
+          if (++stage == n_stages) stage = 0;
         }
       } else {
         // ---------------- epilogue: drain tensor memory, finish the cell ----------------
@@ -348,9 +365,9 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
         if (alive) {
           tc_fence_after();
           const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(quad * 32) << 16) + 4u * e;
-#pragma unroll 1
-          for (int g = 0; g < G; ++g) {
-            uint32_t v[20];
+          // the tensor-memory loads of group g + 1 are in flight while group g is computed
+          uint32_t vbuf[2][20];
+          auto load_group = [&](int g, uint32_t* v) {
             const uint32_t col0 = (uint32_t)(g * gcols);
             if (leaf) {
 #pragma unroll
@@ -359,15 +376,22 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
 #pragma unroll
               for (int q = 0; q < 5; ++q) tmem_ld4(taddr + col0 + 8 * q, v + 4 * q);
             }
+          };
+          load_group(0, vbuf[0]);
+#pragma unroll
+          for (int g = 0; g < kMaxG; ++g) {
+            if (g >= G) break;
+            uint32_t* v = vbuf[g & 1];
             float4 bcur[5];
 #pragma unroll
             for (int q = 0; q < 5; ++q) bcur[q] = bnext[q];
+            tmem_ld_wait();
             if (g + 1 < G) {
+              load_group(g + 1, vbuf[(g + 1) & 1]);
 #pragma unroll
               for (int q = 0; q < 5; ++q)
                 if (q < ngates) bnext[q] = __ldg(reinterpret_cast<const float4*>(bias + (g + 1) * gcols + 8 * q));
             }
-            tmem_ld_wait();
             if (valid) {
               const int u0 = (nt * G + g) * 8 + 4 * e;
               const int count = min(4, H - u0);     // real (unpadded) units among these four
@@ -492,18 +516,6 @@ __global__ void k_pack_embedding(int vocab, int E, int Ep, const float* emb, __n
   }
 }
 
-// Per-row operand indices in ready order: rowA = token (leaf) or left child, rowB = right child.
-__global__ void k_row_operands(int n, const int* order, const int* left, const int* right,
-                               const int* token, int* rowA, int* rowB, const DevStatus* st) {
-  if (st->status != 0) return;
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= n) return;
-  const int node = order[r];
-  const int l = left[node];
-  rowA[r] = l < 0 ? token[node] : l;
-  rowB[r] = l < 0 ? 0 : right[node];
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -555,8 +567,8 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   TcParams p;
   p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep; p.sched_ctas = ctx->sm_count;
   p.order = order;
-  p.rowA = reinterpret_cast<int*>(base + lay.pending);     // dependency counters are dead by now
-  p.rowB = reinterpret_cast<int*>(base + lay.order_tmp);
+  p.rowA = reinterpret_cast<int*>(base + lay.rowA);
+  p.rowB = reinterpret_cast<int*>(base + lay.rowB);
   p.level_offset = level_offset_dev;
   p.emb_bf = ctx->emb_bf;
   p.hb = reinterpret_cast<__nv_bfloat16*>(base + lay.hb);
@@ -566,10 +578,6 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.st = reinterpret_cast<DevStatus*>(base + lay.status);
   p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
 
-  k_row_operands<<<(n + 255) / 256, 256, 0, stream>>>(n, order, left, right, token, const_cast<int*>(p.rowA),
-                                                      const_cast<int*>(p.rowB), p.st);
-  ctx->launches += 1;
-  if (ctx->opt.time_kernel) TL_CUDA(ctx, cudaEventRecord(ctx->ev_begin, stream));  // wavefront kernel only
   static bool attr_set = false;
   if (!attr_set) {
     TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));

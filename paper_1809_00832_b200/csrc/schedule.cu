@@ -7,7 +7,7 @@
 // The ready order reported to the caller is canonical: ascending (level, node id).
 //
 // Two implementations produce identical arrays:
-//   * k_schedule_single: one CTA, levels in shared memory, for forests up to 49152 nodes;
+//   * k_schedule_single: one CTA, dependency words in shared memory, forests up to 32768 nodes;
 //   * a multi-CTA path (dependency counters walked up from the leaves, LSD radix sort with
 //     per-chunk histograms) for anything larger.
 #include "common.cuh"
@@ -45,11 +45,12 @@ __device__ __forceinline__ int check_node(int n, int k, int l, int r, const int*
 // Stable counting pass executed by one CTA of 32 warps over `n` items.
 // Item r of the source sequence is src ? src[r] : r.  key(item) in [0, 256).  Items are written
 // to dst ordered by key, ties in source order.  hist is shared memory [256][32] ints.
-// After the scan step, *bin1_start (if non-null) receives the number of items with key 0.
+// After the scan step, bin_starts[b] (b < n_bin_starts) receives the position of the first item
+// with key b.
 // ------------------------------------------------------------------------------------------ //
 template <class KeyFn>
 __device__ void block_counting_pass(int n, const int* src, int* dst, KeyFn key, int* hist,
-                                    int* scan_tmp, int* bin1_start) {
+                                    int* scan_tmp, int* bin_starts, int n_bin_starts) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int i = tid; i < kRadixBins * kSingleWarps; i += kSingleThreads) hist[i] = 0;
   __syncthreads();
@@ -90,7 +91,7 @@ __device__ void block_counting_pass(int n, const int* src, int* dst, KeyFn key, 
     for (int j = 0; j < kPer; ++j) { hist[tid * kPer + j] = run; run += v[j]; }
   }
   __syncthreads();
-  if (bin1_start && tid == 0) *bin1_start = hist[1 * kSingleWarps + 0];
+  for (int b = tid; b < n_bin_starts; b += kSingleThreads) bin_starts[b] = hist[b * kSingleWarps];
   __syncthreads();
   for (int r0 = begin; r0 < end; r0 += 32) {
     const int r = r0 + lane;
@@ -112,68 +113,92 @@ __device__ void block_counting_pass(int n, const int* src, int* dst, KeyFn key, 
   __syncthreads();
 }
 
-// One CTA schedules the whole forest.  Dynamic shared memory: uint16 level[n] | int hist[256*32].
+// One CTA schedules the whole forest in shared memory (forests up to 32768 nodes).
+//
+// Dependency counters, as in Section 4.1.1: every internal node waits for two inputs.  A finished
+// child swaps (its level + 1) into its caller's word; the child that finds the word empty was first
+// and stops, the one that finds its sibling's entry knows both inputs are resolved, gives the caller
+// level 1 + max and goes on upwards.  No global atomics, no grid-wide rounds.
+//
+// Dynamic shared memory: uint32 w[n] (dependency words; later the radix histogram, at least 32 KB)
+// followed by uint16 par[n] (caller of each node; later level | root flag).
 __global__ void __launch_bounds__(kSingleThreads, 1)
 k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ right,
                   const int* __restrict__ token, int vocab, int* parent, int* level, int* order,
-                  int* order_tmp, int* level_offset, int* roots, DevStatus* st) {
+                  int* order_tmp, int* level_offset, int* roots, int* rowA, int* rowB,
+                  int* n_levels_out, DevStatus* st) {
   extern __shared__ __align__(16) unsigned char smem[];
-  unsigned short* lv = reinterpret_cast<unsigned short*>(smem);
-  int* hist = reinterpret_cast<int*>(smem + (((size_t)n * 2 + 15) & ~(size_t)15));
+  const size_t w_bytes = (size_t)n * 4 > sizeof(int) * kRadixBins * kSingleWarps
+                             ? (((size_t)n * 4 + 15) & ~(size_t)15) : sizeof(int) * kRadixBins * kSingleWarps;
+  unsigned int* w = reinterpret_cast<unsigned int*>(smem);
+  int* hist = reinterpret_cast<int*>(smem);
+  unsigned short* par = reinterpret_cast<unsigned short*>(smem + w_bytes);
+  unsigned short* lv16 = par;
   __shared__ int scan_tmp[32];
-  __shared__ int s_err, s_maxlevel;
+  __shared__ int s_err, s_maxlevel, s_bins[2];
   const int tid = threadIdx.x;
-  constexpr unsigned short kNone = 0xFFFF;
+  constexpr unsigned short kNoParent = 0xFFFF;
+  constexpr unsigned int kDone = 0x80000000u;
+  if (tid < (int)(sizeof(DevStatus) / sizeof(int))) reinterpret_cast<int*>(st)[tid] = 0;
   if (tid == 0) { s_err = 0; s_maxlevel = 0; }
-  for (int k = tid; k < n; k += kSingleThreads) parent[k] = -1;
+  for (int k = tid; k < n; k += kSingleThreads) { w[k] = 0; par[k] = kNoParent; }
   __syncthreads();
-  // validate, link children to their caller, leaves are ready at once
+  // validate; children record their caller; leaves are complete at once (level 0)
+#pragma unroll 4
   for (int k = tid; k < n; k += kSingleThreads) {
     const int l = left[k], r = right[k];
     bool leaf;
-    int err = check_node(n, k, l, r, token, vocab, &leaf);
-    if (err == 0 && !leaf) {
-      if (atomicCAS(&parent[l], -1, k) != -1) err = TREELSTM_ERR_INVALID_FOREST;
-      if (atomicCAS(&parent[r], -1, k) != -1) err = TREELSTM_ERR_INVALID_FOREST;
-    }
+    const int err = check_node(n, k, l, r, token, vocab, &leaf);
     if (err) atomicMin(&s_err, err);
-    lv[k] = (err == 0 && leaf) ? 0 : kNone;
+    else if (leaf) w[k] = kDone;
+    else { par[l] = (unsigned short)k; par[r] = (unsigned short)k; }
+  }
+  __syncthreads();
+  if (s_err == 0) {
+    // a child claimed by two callers kept only one of them
+#pragma unroll 4
+    for (int k = tid; k < n; k += kSingleThreads) {
+      const int l = left[k];
+      if (l >= 0 && (par[l] != k || par[right[k]] != k)) atomicMin(&s_err, (int)TREELSTM_ERR_INVALID_FOREST);
+    }
+  }
+  __syncthreads();
+  if (s_err == 0) {
+    for (int k = tid; k < n; k += kSingleThreads) {
+      if (left[k] >= 0) continue;
+      int cur = k, lvl = 0;
+      for (int step = 0; step < n; ++step) {   // a path to the root has fewer than n edges
+        const unsigned short p = par[cur];
+        if (p == kNoParent) break;
+        const unsigned int old = atomicExch(&w[p], (unsigned int)lvl + 1u);
+        if (old == 0) break;                   // sibling subtree still unresolved
+        lvl = 1 + max(lvl, (int)old - 1);
+        w[p] = kDone | (unsigned int)lvl;
+        cur = p;
+      }
+    }
+  }
+  __syncthreads();
+  int local_max = 0;
+  if (s_err == 0) {
+    for (int k = tid; k < n; k += kSingleThreads) {
+      const unsigned int wk = w[k];
+      if (!(wk & kDone)) atomicMin(&s_err, (int)TREELSTM_ERR_INVALID_FOREST);   // on a cycle: never ready
+      const int lvl = (int)(wk & 0x7FFFu);
+      const unsigned short pk = par[k];
+      lv16[k] = (unsigned short)(lvl | (pk == kNoParent ? 0x8000 : 0));
+      level[k] = lvl;
+      parent[k] = pk == kNoParent ? -1 : (int)pk;
+      local_max = max(local_max, lvl);
+    }
+    atomicMax(&s_maxlevel, local_max);
   }
   __syncthreads();
   if (s_err != 0) {
-    if (tid == 0) { report(st, s_err); st->n_levels = 0; st->n_roots = 0; }
+    if (tid == 0) { report(st, s_err); *n_levels_out = 0; }
     return;
   }
-  // relaxation rounds: a node whose children both have a level takes 1 + max.  A level, once
-  // written, is final, so reading a value written in the same round is harmless.
-  int local_max = 0;
-  for (int round = 0; round <= n; ++round) {
-    int progress = 0, waiting = 0;
-    for (int k = tid; k < n; k += kSingleThreads) {
-      if (lv[k] != kNone) continue;
-      const unsigned short a = lv[left[k]], b = lv[right[k]];
-      if (a != kNone && b != kNone) {
-        const int v = 1 + max((int)a, (int)b);
-        lv[k] = (unsigned short)v;
-        local_max = max(local_max, v);
-        progress = 1;
-      } else {
-        waiting = 1;
-      }
-    }
-    const int any_progress = __syncthreads_or(progress);
-    const int any_waiting = __syncthreads_or(waiting);
-    if (!any_waiting) break;
-    if (!any_progress) {  // nodes on a cycle never become ready
-      if (tid == 0) { report(st, TREELSTM_ERR_INVALID_FOREST); st->n_levels = 0; st->n_roots = 0; }
-      return;
-    }
-  }
-  atomicMax(&s_maxlevel, local_max);
-  for (int k = tid; k < n; k += kSingleThreads) level[k] = lv[k];
-  __syncthreads();
   const int n_levels = n > 0 ? s_maxlevel + 1 : 0;
-  if (tid == 0) st->n_levels = n_levels;
   // canonical ready order: LSD radix on the level, 8 bits per pass, ties by node id
   int passes = 1;
   while (passes < 4 && (n_levels - 1) >> (8 * passes)) ++passes;
@@ -181,18 +206,30 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
     int* dst = ((passes - 1 - p) & 1) ? order_tmp : order;
     const int* src = p == 0 ? nullptr : (dst == order ? order_tmp : order);
     const int shift = 8 * p;
-    block_counting_pass(n, src, dst, [=](int item) { return ((int)lv[item] >> shift) & 255; },
-                        hist, scan_tmp, nullptr);
+    block_counting_pass(n, src, dst, [=](int item) { return ((lv16[item] & 0x7FFF) >> shift) & 255; },
+                        hist, scan_tmp, passes == 1 ? level_offset : nullptr, passes == 1 ? n_levels : 0);
   }
-  // wavefront boundaries
-  for (int r = tid; r < n; r += kSingleThreads) {
-    const int a = lv[order[r]];
-    if (r == 0 || (int)lv[order[r - 1]] != a) level_offset[a] = r;
+  if (passes > 1) {   // wavefront boundaries from the sorted order
+    for (int r = tid; r < n; r += kSingleThreads) {
+      const int a = lv16[order[r]] & 0x7FFF;
+      if (r == 0 || (lv16[order[r - 1]] & 0x7FFF) != a) level_offset[a] = r;
+    }
   }
-  if (tid == 0) level_offset[n_levels] = n;
+  if (tid == 0) { level_offset[n_levels] = n; st->n_levels = n_levels; *n_levels_out = n_levels; }
   // roots in ascending node id: stable partition on "has a caller"
-  block_counting_pass(n, nullptr, roots, [=](int item) { return parent[item] >= 0 ? 1 : 0; }, hist,
-                      scan_tmp, &st->n_roots);
+  block_counting_pass(n, nullptr, roots, [=](int item) { return (lv16[item] & 0x8000) ? 0 : 1; }, hist,
+                      scan_tmp, s_bins, 2);
+  if (tid == 0) st->n_roots = s_bins[1];
+  // operand rows of every wavefront position: token (leaf) or left child, and right child
+  if (rowA) {
+#pragma unroll 4
+    for (int r = tid; r < n; r += kSingleThreads) {
+      const int node = order[r];
+      const int l = left[node];
+      rowA[r] = l < 0 ? token[node] : l;
+      rowB[r] = l < 0 ? 0 : right[node];
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------ //
@@ -370,6 +407,18 @@ __global__ void k_sched_offsets(int n, const int* level, const int* order, int* 
   if (r == 0 || level[order[r - 1]] != a) level_offset[a] = r;
 }
 
+// Per-row operand indices in ready order: rowA = token (leaf) or left child, rowB = right child.
+__global__ void k_row_operands(int n, const int* order, const int* left, const int* right,
+                               const int* token, int* rowA, int* rowB, const DevStatus* st) {
+  if (st->status != 0) return;
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= n) return;
+  const int node = order[r];
+  const int l = left[node];
+  rowA[r] = l < 0 ? token[node] : l;
+  rowB[r] = l < 0 ? 0 : right[node];
+}
+
 __global__ void k_gather_roots(int max_roots, int H, const int* roots, const float* h,
                                const float* c, int* root_ids, float* root_h, float* root_c,
                                int* n_roots_out, const DevStatus* st) {
@@ -387,9 +436,16 @@ __global__ void k_gather_roots(int max_roots, int H, const int* roots, const flo
 
 }  // namespace
 
+size_t single_smem_bytes(int n) {
+  size_t w = (size_t)n * 4;
+  const size_t hist = sizeof(int) * kRadixBins * kSingleWarps;
+  w = w > hist ? round_up_sz(w, 16) : hist;
+  return w + round_up_sz((size_t)n * 2, 16);
+}
+
 int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
                     const int32_t* token, int32_t* level, int32_t* order, int32_t* level_offset,
-                    void* ws, const WsLayout& lay, cudaStream_t stream) {
+                    int32_t* n_levels_out, void* ws, const WsLayout& lay, cudaStream_t stream) {
   char* base = static_cast<char*>(ws);
   DevStatus* st = reinterpret_cast<DevStatus*>(base + lay.status);
   int* parent = reinterpret_cast<int*>(base + lay.parent);
@@ -397,28 +453,32 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   int* order_tmp = reinterpret_cast<int*>(base + lay.order_tmp);
   int* roots = reinterpret_cast<int*>(base + lay.roots);
   int* table = reinterpret_cast<int*>(base + lay.table);
-  if (n == 0) return TREELSTM_OK;  // control block already zero: 0 levels, 0 roots
+  int* rowA = reinterpret_cast<int*>(base + lay.rowA);
+  int* rowB = reinterpret_cast<int*>(base + lay.rowB);
 
   const int single_max = ctx->opt.sched_single_cta_max < kSchedSingleMaxNodes
                              ? ctx->opt.sched_single_cta_max : kSchedSingleMaxNodes;
-  if (n <= single_max) {
-    const size_t smem = round_up_sz((size_t)n * 2, 16) + sizeof(int) * kRadixBins * kSingleWarps;
+  if (n > 0 && n <= single_max) {
     static bool attr_set = false;
     if (!attr_set) {
-      TL_CUDA(ctx, cudaFuncSetAttribute(k_schedule_single,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)(round_up_sz((size_t)kSchedSingleMaxNodes * 2, 16) +
-                                              sizeof(int) * kRadixBins * kSingleWarps)));
+      TL_CUDA(ctx, cudaFuncSetAttribute(k_schedule_single, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)single_smem_bytes(kSchedSingleMaxNodes)));
       attr_set = true;
     }
-    k_schedule_single<<<1, kSingleThreads, smem, stream>>>(n, left, right, token, ctx->vocab, parent,
-                                                           level, order, order_tmp, level_offset,
-                                                           roots, st);
+    // the kernel clears the control block itself and writes the level count to the caller
+    k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n), stream>>>(
+        n, left, right, token, ctx->vocab, parent, level, order, order_tmp, level_offset, roots, rowA, rowB,
+        n_levels_out, st);
     ctx->launches += 1;
     TL_CUDA(ctx, cudaGetLastError());
     return TREELSTM_OK;
   }
 
+  TL_CUDA(ctx, cudaMemsetAsync(st, 0, sizeof(DevStatus), stream));
+  if (n == 0) {
+    TL_CUDA(ctx, cudaMemsetAsync(n_levels_out, 0, sizeof(int), stream));
+    return TREELSTM_OK;
+  }
   TL_CUDA(ctx, cudaMemsetAsync(parent, 0xFF, sizeof(int) * (size_t)n, stream));
   TL_CUDA(ctx, cudaMemsetAsync(pending, 0, sizeof(int) * (size_t)n, stream));
   const int tpb = 256, blocks = (n + tpb - 1) / tpb;
@@ -445,8 +505,10 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   k_radix_scan<<<1, 1024, 0, stream>>>(1, 0, table, n_chunks, st);
   k_radix_scatter<<<n_chunks, 32, 0, stream>>>(n, 1, 0, level, parent, order, order_tmp, roots,
                                                table, n_chunks, st);
-  ctx->launches += 4;
+  k_row_operands<<<blocks, tpb, 0, stream>>>(n, order, left, right, token, rowA, rowB, st);
+  ctx->launches += 5;
   TL_CUDA(ctx, cudaGetLastError());
+  TL_CUDA(ctx, cudaMemcpyAsync(n_levels_out, &st->n_levels, sizeof(int), cudaMemcpyDeviceToDevice, stream));
   return TREELSTM_OK;
 }
 
@@ -496,8 +558,7 @@ extern "C" int treelstm_schedule_static(int n_nodes, const int32_t* left, const 
     void* addr = nullptr;
     if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return TREELSTM_ERR_CUDA;
     if (cudaFuncSetAttribute(k_schedule_single, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)(round_up_sz((size_t)kSchedSingleMaxNodes * 2, 16) +
-                                   sizeof(int) * kRadixBins * kSingleWarps)) != cudaSuccess)
+                             (int)single_smem_bytes(kSchedSingleMaxNodes)) != cudaSuccess)
       return TREELSTM_ERR_CUDA;
     g_static_scratch_addr[dev] = static_cast<unsigned char*>(addr);
   }
@@ -507,18 +568,20 @@ extern "C" int treelstm_schedule_static(int n_nodes, const int32_t* left, const 
   int* order_tmp = parent + kStaticNodes;
   int* roots = order_tmp + kStaticNodes;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // the control block keeps the previous call's status and counts: it must start from zero
-  if (cudaMemsetAsync(st, 0, sizeof(DevStatus), s) != cudaSuccess) return TREELSTM_ERR_CUDA;
   if (n_nodes > 0) {
-    const size_t smem = round_up_sz((size_t)n_nodes * 2, 16) + sizeof(int) * kRadixBins * kSingleWarps;
-    k_schedule_single<<<1, kSingleThreads, smem, s>>>(n_nodes, left, right, token, vocab, parent, level,
-                                                      order, order_tmp, level_offset, roots, st);
+    // the control block keeps the previous call's status and counts; the kernel's first step is
+    // to clear it, everything else in the array is rewritten before it is read
+    k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n_nodes), s>>>(
+        n_nodes, left, right, token, vocab, parent, level, order, order_tmp, level_offset, roots, nullptr,
+        nullptr, n_levels, st);
     if (cudaGetLastError() != cudaSuccess) return TREELSTM_ERR_CUDA;
   } else {
-    if (cudaMemsetAsync(level_offset, 0, sizeof(int32_t), s) != cudaSuccess) return TREELSTM_ERR_CUDA;
+    if (cudaMemsetAsync(st, 0, sizeof(DevStatus), s) != cudaSuccess ||
+        cudaMemsetAsync(level_offset, 0, sizeof(int32_t), s) != cudaSuccess ||
+        cudaMemsetAsync(n_levels, 0, sizeof(int32_t), s) != cudaSuccess)
+      return TREELSTM_ERR_CUDA;
   }
-  if (cudaMemcpyAsync(n_levels, &st->n_levels, sizeof(int), cudaMemcpyDeviceToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(status, &st->status, sizeof(int), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+  if (cudaMemcpyAsync(status, &st->status, sizeof(int), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
     return TREELSTM_ERR_CUDA;
   return TREELSTM_OK;
 }

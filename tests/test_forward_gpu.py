@@ -78,12 +78,12 @@ def test_deep_and_wide_schedules(single_cta):
 
 
 def test_large_forest_uses_multi_cta_schedule():
-    """more nodes than the single-CTA scheduler takes (49152): properties that hold at any size plus
+    """more nodes than the single-CTA scheduler takes (32768): properties that hold at any size plus
     sampled trees against the oracle"""
     rng = np.random.default_rng(5)
     params = fg.draw_params(rng, 16, 16, 100, emb_dist="uniform", emb_scale=0.1, w_scale=0.1)
     forest = fg.random_forest(rng, 2200, 2, 56, 100)
-    assert forest.n_nodes > 49152
+    assert forest.n_nodes > 32768
     model = util.make_model(params, "fp32")
     res = util.gpu_forward(model, forest, binding.PERSISTENT)
     status, _, level, order, off = orc.schedule(forest.left, forest.right)
