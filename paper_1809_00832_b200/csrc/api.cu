@@ -20,8 +20,13 @@ WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward) {
   L.table = take(4 * (size_t)kRadixBins * ((nn + kRadixChunk - 1) / kRadixChunk));
   L.rowA = take(4 * nn);
   L.rowB = take(4 * nn);
-  L.hb = off;
-  if (ctx->precision == TREELSTM_BF16) L.hb = take(2 * nn * (size_t)ctx->Hp);
+  L.slot = take(4 * nn);
+  L.xin = L.ain = L.cin = off;
+  if (ctx->precision == TREELSTM_BF16) {
+    L.xin = take(2 * nn * (size_t)ctx->Ep);          // leaf embedding rows in ready order
+    L.ain = take(2 * nn * 2 * (size_t)ctx->Hp);      // [h_l | h_r] of every position, bf16
+    L.cin = take(4 * nn * 2 * (size_t)ctx->H);       // [c_l | c_r] of every position, fp32
+  }
   L.gates = L.dh = L.dc = L.dz = L.tok_slot = off;
   if (with_backward) {
     const size_t H = (size_t)ctx->H;

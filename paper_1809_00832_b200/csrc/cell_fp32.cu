@@ -13,13 +13,15 @@ namespace {
 
 constexpr int TM = 64;       // rows (nodes) per tile
 constexpr int TU = 16;       // hidden units per tile (x 5 gates = 80 columns)
-constexpr int KC = 16;       // contraction chunk
+constexpr int KC = 32;       // contraction chunk
 constexpr int kThreads = 256;
 constexpr int RPT = TM / (kThreads / TU);  // rows per thread = 4
+constexpr int kALoads = TM * KC / kThreads;        // 8 operand elements per thread and chunk
+constexpr int kWLoads = KC * 5 * TU / kThreads;    // 10 weight elements per thread and chunk
 
 struct FwdParams {
   int n, H, E;
-  const int *left, *right, *token, *order, *level_offset;
+  const int *left, *right, *token, *order, *rowA, *rowB, *level_offset;
   const float *emb, *W, *b;
   float *h, *c, *gates;
   DevStatus* st;
@@ -29,26 +31,28 @@ struct FwdParams {
 __device__ __forceinline__ float sigmoidf_acc(float x) { return 1.0f / (1.0f + expf(-x)); }
 
 struct TileSmem {
-  float A[TM][KC + 1];
-  float W[KC][5 * TU];
+  float A[2][TM][KC + 1];
+  float W[2][KC][5 * TU];
   int node[TM], l[TM], r[TM];
 };
 
 // One tile: rows [row0, row0 + TM) of the ready order (clipped to row_end), hidden units
 // [u0, u0 + TU).  `leaf` selects x = emb[token] with W rows [0, E) and gates i, o, u only.
+// The next K chunk is fetched into registers while the current one is multiplied out of shared
+// memory (two buffers, one CTA barrier per chunk).
 __device__ void fp32_tile(const FwdParams& p, int row0, int row_end, int u0, bool leaf,
                           TileSmem& s) {
   const int tid = threadIdx.x, tx = tid % TU, ty = tid / TU;
   const int H = p.H, E = p.E, K = leaf ? E : 2 * H;
   const float* Wk = p.W + (size_t)(leaf ? 0 : E) * 5 * H;
-  __syncthreads();  // previous tile's readers of s.node are done
+  __syncthreads();  // previous tile's readers of s are done
   for (int i = tid; i < TM; i += kThreads) {
     const int row = row0 + i;
     int node = -1, l = 0, r = 0;
     if (row < row_end) {
       node = p.order[row];
-      l = leaf ? p.token[node] : p.left[node];
-      r = leaf ? 0 : p.right[node];
+      l = p.rowA[row];
+      r = p.rowB[row];
     }
     s.node[i] = node; s.l[i] = l; s.r[i] = r;
   }
@@ -59,36 +63,59 @@ __device__ void fp32_tile(const FwdParams& p, int row0, int row_end, int u0, boo
 #pragma unroll
     for (int g = 0; g < 5; ++g) acc[i][g] = 0.f;
 
-  for (int k0 = 0; k0 < K; k0 += KC) {
-    for (int e = tid; e < TM * KC; e += kThreads) {
-      const int i = e / KC, kk = e % KC, k = k0 + kk;
+  float ra[kALoads], rw[kWLoads];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int j = 0; j < kALoads; ++j) {
+      const int e = tid + j * kThreads, i = e / KC, k = k0 + e % KC;
       float v = 0.f;
       if (s.node[i] >= 0 && k < K) {
         if (leaf) v = __ldg(p.emb + (size_t)s.l[i] * E + k);
         else v = k < H ? __ldcg(p.h + (size_t)s.l[i] * H + k) : __ldcg(p.h + (size_t)s.r[i] * H + (k - H));
       }
-      s.A[i][kk] = v;
+      ra[j] = v;
     }
-    for (int e = tid; e < KC * 5 * TU; e += kThreads) {
-      const int kk = e / (5 * TU), g = (e % (5 * TU)) / TU, uu = e % TU, k = k0 + kk;
+#pragma unroll
+    for (int j = 0; j < kWLoads; ++j) {
+      const int e = tid + j * kThreads, kk = e / (5 * TU), g = (e % (5 * TU)) / TU, uu = e % TU, k = k0 + kk;
       float v = 0.f;
       if (k < K && u0 + uu < H && !(leaf && (g == 1 || g == 2)))
         v = __ldg(Wk + (size_t)k * 5 * H + g * H + u0 + uu);
-      s.W[kk][g * TU + uu] = v;
+      rw[j] = v;
     }
-    __syncthreads();
+  };
+  auto stash = [&](int buf) {
+#pragma unroll
+    for (int j = 0; j < kALoads; ++j) {
+      const int e = tid + j * kThreads;
+      s.A[buf][e / KC][e % KC] = ra[j];
+    }
+#pragma unroll
+    for (int j = 0; j < kWLoads; ++j) {
+      const int e = tid + j * kThreads;
+      s.W[buf][e / (5 * TU)][e % (5 * TU)] = rw[j];
+    }
+  };
+  fetch(0);
+  stash(0);
+  __syncthreads();
+  const int chunks = (K + KC - 1) / KC;
+  for (int cidx = 0; cidx < chunks; ++cidx) {
+    const int buf = cidx & 1;
+    if (cidx + 1 < chunks) fetch((cidx + 1) * KC);
 #pragma unroll
     for (int kk = 0; kk < KC; ++kk) {
       float a[RPT], w[5];
 #pragma unroll
-      for (int i = 0; i < RPT; ++i) a[i] = s.A[ty * RPT + i][kk];
+      for (int i = 0; i < RPT; ++i) a[i] = s.A[buf][ty * RPT + i][kk];
 #pragma unroll
-      for (int g = 0; g < 5; ++g) w[g] = s.W[kk][g * TU + tx];
+      for (int g = 0; g < 5; ++g) w[g] = s.W[buf][kk][g * TU + tx];
 #pragma unroll
       for (int i = 0; i < RPT; ++i)
 #pragma unroll
         for (int g = 0; g < 5; ++g) acc[i][g] = fmaf(a[i], w[g], acc[i][g]);
     }
+    if (cidx + 1 < chunks) stash(buf ^ 1);
     __syncthreads();
   }
 
@@ -159,6 +186,8 @@ int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.n = n; p.H = ctx->H; p.E = ctx->E;
   p.left = left; p.right = right; p.token = token; p.order = order;
   p.level_offset = level_offset_dev;
+  p.rowA = reinterpret_cast<const int*>(base + lay.rowA);
+  p.rowB = reinterpret_cast<const int*>(base + lay.rowB);
   p.emb = ctx->emb; p.W = ctx->W; p.b = ctx->b;
   p.h = h; p.c = c;
   p.gates = (flags & TREELSTM_SAVE_FOR_BACKWARD) ? reinterpret_cast<float*>(base + lay.gates) : nullptr;

@@ -25,8 +25,8 @@ static_assert(sizeof(DevStatus) == 256, "control block is one 256-byte line grou
 
 // Offsets (bytes) of the regions inside the workspace for a forest of up to n nodes.
 struct WsLayout {
-  size_t status, parent, pending, order_tmp, level_offset, roots, table, rowA, rowB, hb, gates, dh,
-      dc, dz, tok_slot, total;
+  size_t status, parent, pending, order_tmp, level_offset, roots, table, rowA, rowB, slot, xin, ain,
+      cin, gates, dh, dc, dz, tok_slot, total;
 };
 
 struct Options {
@@ -70,7 +70,9 @@ struct treelstm {
   __nv_bfloat16* Wp_x = nullptr;    // [(Hp/8)*24][Ep]    packed input weights (gates i, o, u)
   float* bp_h = nullptr;            // [(Hp/8)*40] bias in packed column order
   float* bp_x = nullptr;            // [(Hp/8)*24]
-  CUtensorMap tmap_wh, tmap_wx;
+  CUtensorMap tmap_wh, tmap_wx, tmap_x, tmap_a;
+  const void* tmap_ws_base = nullptr;   // tmap_x / tmap_a are rebuilt when the workspace or node count changes
+  int tmap_ws_rows = 0;
   bool have_tmaps = false;
 
   tl::Options opt;

@@ -1,6 +1,6 @@
 // bf16 tensor-core wavefront evaluation (sm_100a: tcgen05.mma with the accumulator in tensor
-// memory, weights fetched by TMA, operand rows gathered by cp.async, cell update fused into the
-// epilogue that drains tensor memory).
+// memory, both operands fetched by tiled TMA, cell update fused into the epilogue that drains
+// tensor memory).
 //
 // Paper: Figure 2 (Section 3.1) - a node is LSTM(embed(word)) or LSTM(left_state, right_state);
 // Section 2.2 - sibling subtrees are independent, so every node whose children are done can be
@@ -13,9 +13,16 @@
 // pre-activations of a hidden unit sit in the same accumulator row slice and one thread (one
 // tensor-memory lane = one node) can finish the cell without any exchange.
 //
-// Warp roles (448 threads): warps 0-3 and 10-13 epilogue (tensor-memory lane quadrant = warp id
-// mod 4; the two sets split every unit group in halves), warp 4 TMA producer of W tiles, warp 5
-// MMA issuer + tensor-memory owner, warps 6-9 gather the A rows.
+// No gather on the operand side: a tree node has exactly one caller, so the epilogue writes a
+// node's state straight into the slot its caller will read - row pos(caller) of the dense operand
+// matrix Ain[pos][h_l | h_r] (bf16) and of Cin[pos][c_l | c_r] (fp32), pos being the caller's
+// position in the ready order.  Every wavefront's operand is then a contiguous block of rows and
+// one tiled TMA load per K block feeds the tensor core.  Leaves: the embedding rows are copied
+// once into ready order (Xin) by all CTAs before the first wavefront.
+//
+// Warp roles (320 threads): warps 0-3 and 6-9 epilogue (tensor-memory lane quadrant = warp id
+// mod 4; the two sets split every unit group in halves), warp 4 TMA producer (A and W tiles),
+// warp 5 MMA issuer + tensor-memory owner.
 #include "common.cuh"
 
 namespace tl {
@@ -23,7 +30,7 @@ namespace {
 
 constexpr int BM = 128;                 // nodes per tile (UMMA M)
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 448;
+constexpr int kThreads = 320;
 constexpr int kABytes = BM * 128;       // one K block (64 bf16) of 128 rows
 constexpr int kAccCols = 256;           // accumulator stage stride in tensor-memory columns
 constexpr unsigned kFull = 0xffffffffu;
@@ -54,9 +61,10 @@ __host__ __device__ inline int choose_groups_per_tile(int rows, int groups, int 
 
 struct TcParams {
   int n, H, Hp, Ep, sched_ctas;
-  const int *order, *rowA, *rowB, *level_offset;
+  const int *order, *rowA, *slot, *level_offset;
   const __nv_bfloat16* emb_bf;
-  __nv_bfloat16* hb;
+  __nv_bfloat16 *xin, *ain;
+  float* cin;
   const float *bp_h, *bp_x;
   float *h, *c, *gates;
   DevStatus* st;
@@ -110,6 +118,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// Four rows (r0..r3, any order) of a 2-D tensor, `x` the first column: lands as four consecutive
+// 128-byte rows of the swizzled tile.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int x, int r0, int r1, int r2,
+                                            int r3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
@@ -179,10 +196,29 @@ __device__ __forceinline__ void st_row4(float* p, bool vec, int count, const flo
 }
 
 // ---- the kernel -------------------------------------------------------------------------------- //
-// only_level >= 0: process that wavefront only (one launch per level).  only_level < 0: all
-// wavefronts, separated by the bounded grid barrier (cooperative launch).
+// Embedding rows of the leaves into ready order: Xin[r] = emb_bf[token of the r-th leaf].
+__device__ void gather_leaf_rows(const TcParams& p, int n_leaves, int gtid, int gthreads) {
+  const int cpr = p.Ep / 8;                              // 16-byte chunks per row
+  const long long total = (long long)n_leaves * cpr;
+  for (long long ch = gtid; ch < total; ch += gthreads) {
+    const int row = (int)(ch / cpr), cc = (int)(ch % cpr);
+    const int tok = p.rowA[row];
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.emb_bf + (size_t)tok * p.Ep) + cc);
+    reinterpret_cast<uint4*>(p.xin + (size_t)row * p.Ep)[cc] = v;
+  }
+}
+
+__global__ void k_gather_leaf_rows(TcParams p) {
+  if (ld_volatile(&p.st->status) != 0) return;
+  gather_leaf_rows(p, p.level_offset[1], blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
+}
+
+// only_level >= 0: process that wavefront only (one launch per level; Xin already filled).
+// only_level < 0: fill Xin, then all wavefronts, separated by the bounded grid barrier (cooperative
+// launch).
 __global__ void __launch_bounds__(kThreads, 1)
 k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CUtensorMap tmap_wx,
+         const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_a,
          TcParams p, int only_level) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -206,7 +242,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   const int n_levels = p.st->n_levels;
 
   if (tid == 0) {
-    for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 128 + 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -219,19 +255,28 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
 
   const int Hp = p.Hp, H = p.H;
   const int groups = Hp / kUnitGroup;
-  const int kb_leaf = p.Ep / kKBlock, kb_int = 2 * Hp / kKBlock, kb_half = Hp / kKBlock;
+  const int kb_leaf = p.Ep / kKBlock, kb_int = 2 * Hp / kKBlock;
   const bool vec = (H % 4) == 0;
 
-  // pipeline positions; every role walks the same tile sequence, so they stay in step
-  // The ring is re-cut at every wavefront (thin tiles leave room for more stages); each mbarrier
-  // keeps its own phase, tracked per stage in a bit mask.
-  uint32_t stage = 0, phase_bits = 0;   // smem ring (producers and MMA)
+  // Pipeline positions; every role walks the same tile sequence, so they stay in step.  The ring
+  // is re-cut at every wavefront (thin tiles leave room for more stages); each mbarrier keeps its
+  // own phase, tracked per stage in a bit mask.
+  uint32_t stage = 0, phase_bits = 0;   // smem ring (producer and MMA)
   uint32_t acc_iter = 0;                // accumulator ring (MMA and epilogue)
+  uint32_t barriers_passed = 0;
   bool alive = true;
+  bool stop = false;                    // uniform over the CTA
+
+  if (only_level < 0 && n_levels > 0) {
+    gather_leaf_rows(p, p.level_offset[1], blockIdx.x * kThreads + tid, gridDim.x * kThreads);
+    asm volatile("fence.proxy.async;" ::: "memory");    // Xin is read through TMA
+    ++barriers_passed;
+    if (!grid_barrier(p.st, barriers_passed * gridDim.x, p.wait_limit, s_flag)) stop = true;
+  }
 
   const int lvl_begin = only_level >= 0 ? only_level : 0;
   const int lvl_end = only_level >= 0 ? only_level + 1 : n_levels;
-  for (int lvl = lvl_begin; lvl < lvl_end; ++lvl) {   // uniform trip count: barriers inside
+  for (int lvl = lvl_begin; lvl < lvl_end && !stop; ++lvl) {   // uniform trip count: barriers inside
     const int begin = p.level_offset[lvl], end = p.level_offset[lvl + 1];
     const bool leaf = lvl == 0;
     const int G = choose_groups_per_tile(end - begin, groups, p.sched_ctas);
@@ -244,24 +289,31 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
     const uint32_t stage_bytes = kABytes + (uint32_t)G * kGColsI * 128u;
     const uint32_t n_stages = min((uint32_t)kMaxStages, (uint32_t)kRingBytes / stage_bytes);
     stage = 0;
+    if (warp == 4) asm volatile("fence.proxy.async;" ::: "memory");   // TMA reads after the barrier's acquire
 
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
       const int row0 = begin + (t / ntn) * BM, nt = t % ntn;
 
       if (warp == 4) {
-        // ---------------- W tile producer (TMA) ----------------
+        // ---------------- operand producer (TMA) ----------------
+        // A: 128 consecutive rows of the dense operand matrix (rows past its end read as zero, rows
+        // past the wavefront belong to later wavefronts and only feed accumulator rows that are
+        // never stored).  W: one box per unit group of the packed weights.
         if (lane == 0) {
-          const CUtensorMap* map = leaf ? &tmap_wx : &tmap_wh;
-          const uint32_t bytes = (uint32_t)ncols * 128u;
+          const CUtensorMap* map_w = leaf ? &tmap_wx : &tmap_wh;
+          const CUtensorMap* map_a = leaf ? &tmap_x : &tmap_a;
+          const uint32_t bytes = (uint32_t)kABytes + (uint32_t)ncols * 128u;
           for (int kb = 0; kb < kblocks; ++kb) {
             if (!mbar_wait(empty_bar(stage), ((phase_bits >> stage) & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) {
               alive = false;
               break;
             }
+            const uint32_t sa = tiles_addr + stage * stage_bytes;
             mbar_arrive_expect_tx(full_bar(stage), bytes);
-            for (int g = 0; g < G; ++g)              // one box = the packed rows of one unit group
-              tma_load_2d(tiles_addr + stage * stage_bytes + kABytes + (uint32_t)(g * gcols) * 128u, map,
-                          kb * kKBlock, (nt * G + g) * gcols, full_bar(stage));
+            tma_load_2d(sa, map_a, kb * kKBlock, row0, full_bar(stage));
+            for (int g = 0; g < G; ++g)
+              tma_load_2d(sa + kABytes + (uint32_t)(g * gcols) * 128u, map_w, kb * kKBlock,
+                          (nt * G + g) * gcols, full_bar(stage));
             phase_bits ^= 1u << stage;
             if (++stage == n_stages) stage = 0;
           }
@@ -279,7 +331,6 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
               alive = false;
               break;
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             tc_fence_after();
             const uint32_t a_addr = tiles_addr + stage * stage_bytes;
             const uint64_t a_desc = umma_desc(a_addr), b_desc = umma_desc(a_addr + kABytes);
@@ -293,59 +344,24 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
           if (alive) umma_commit(tfull_bar(acc));    // accumulator complete
         }
         ++acc_iter;
-      } else if (warp >= 6 && warp < 10) {
-        // ---------------- A row gather (cp.async into the swizzled tile) ----------------
-        // Eight consecutive lanes copy the eight 16-byte chunks of one row's 128-byte K block, so a
-        // warp instruction touches 4 whole lines instead of 32 partial ones.  Thread (rsel, sub)
-        // serves rows rsel, rsel + 16, ... of the tile.
-        const int gtid = tid - 6 * 32, sub = gtid & 7, rsel = gtid >> 3;
-        int ia[8], ib[8];
-        uint32_t valid_mask = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int row = row0 + j * 16 + rsel;
-          const bool valid = row < end;
-          ia[j] = valid ? p.rowA[row] : 0;
-          ib[j] = (valid && !leaf) ? p.rowB[row] : 0;
-          valid_mask |= (valid ? 1u : 0u) << j;
-        }
-        const uint32_t dst_off = (uint32_t)(rsel >> 3) * 1024u + (uint32_t)(rsel & 7) * 128u +
-                                 (uint32_t)((sub ^ (rsel & 7)) << 4);
-        for (int kb = 0; kb < kblocks; ++kb) {
-          if (!mbar_wait(empty_bar(stage), ((phase_bits >> stage) & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) {
-            alive = false;
-            break;
-          }
-          const uint32_t dst = tiles_addr + stage * stage_bytes + dst_off;
-          const bool second = !leaf && kb >= kb_half;
-          const size_t col = (size_t)((second ? kb - kb_half : kb) * kKBlock + sub * 8);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const __nv_bfloat16* src = leaf ? p.emb_bf + (size_t)ia[j] * p.Ep + col
-                                            : p.hb + (size_t)(second ? ib[j] : ia[j]) * Hp + col;
-            cp_async16(dst + (uint32_t)j * 2048u, src, (valid_mask >> j) & 1u ? 16u : 0u);
-          }
-          cp_async_arrive_noinc(full_bar(stage));
-          phase_bits ^= 1u << stage;
-          if (++stage == n_stages) stage = 0;
-        }
       } else {
         // ---------------- epilogue: drain tensor memory, finish the cell ----------------
         // Two sets of four warps; set e takes hidden units [4e, 4e + 4) of every unit group.  A
         // warp may only read the tensor-memory lanes of quadrant (warp id mod 4).
-        const int e = warp < 4 ? 0 : 1;
+        const int e = warp < 4 ? 0 : 1;   // warps 0-3: set 0, warps 6-9: set 1
         const int quad = warp & 3;
         const int r = quad * 32 + lane;
         const int row = row0 + r;
         const bool valid = row < end;
         const int node = valid ? p.order[row] : 0;
-        const int il = (valid && !leaf) ? p.rowA[row] : 0, ir = (valid && !leaf) ? p.rowB[row] : 0;
-        // stage the children's cell states for this thread's row while the MMAs run
+        const int slot = valid ? p.slot[node] : -1;   // 2 * pos(caller) + side, -1 for a root
+        // stage the children's cell states of this thread's row while the MMAs run
+        const float* crow = p.cin + (size_t)row * 2 * H;   // [c_l | c_r] of the node at this position
         const bool staged = !leaf && vec && (nt + 1) * G * 8 <= H;
         const uint32_t my_c = cstage_addr + (uint32_t)r * 256u;
         if (staged) {
-          const float* sl = p.c + (size_t)il * H + nt * G * 8;
-          const float* sr = p.c + (size_t)ir * H + nt * G * 8;
+          const float* sl = crow + nt * G * 8;
+          const float* sr = sl + H;
           const uint32_t nb = valid ? 16u : 0u;
           for (int ch = e; ch < 2 * G; ch += 2) {
             cp_async16(my_c + (uint32_t)((ch ^ (r & 7)) << 4), sl + ch * 4, nb);
@@ -405,8 +421,8 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
               } else if (!leaf && count > 0) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                  cl[j] = j < count ? __ldcg(p.c + (size_t)il * H + u0 + j) : 0.f;
-                  cr[j] = j < count ? __ldcg(p.c + (size_t)ir * H + u0 + j) : 0.f;
+                  cl[j] = j < count ? __ldcg(crow + u0 + j) : 0.f;
+                  cr[j] = j < count ? __ldcg(crow + H + u0 + j) : 0.f;
                 }
               }
               const float* bq = reinterpret_cast<const float*>(bcur);
@@ -428,15 +444,19 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
                 }
                 hv[j] = go[j] * act_tanh(cv[j]);
               }
-              // bf16 copy of h feeds the next wavefront's gather; padded units are written as 0
-              uint32_t packed[2];
+              if (slot >= 0) {
+                // hand the state to the caller: bf16 h into its operand row (padded units as 0),
+                // fp32 c next to it
+                uint32_t packed[2];
 #pragma unroll
-              for (int j = 0; j < 2; ++j) {
-                const float lo = 2 * j < count ? hv[2 * j] : 0.f, hi = 2 * j + 1 < count ? hv[2 * j + 1] : 0.f;
-                __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
-                packed[j] = *reinterpret_cast<uint32_t*>(&b2);
+                for (int j = 0; j < 2; ++j) {
+                  const float lo = 2 * j < count ? hv[2 * j] : 0.f, hi = 2 * j + 1 < count ? hv[2 * j + 1] : 0.f;
+                  __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+                  packed[j] = *reinterpret_cast<uint32_t*>(&b2);
+                }
+                *reinterpret_cast<uint2*>(p.ain + (size_t)slot * Hp + u0) = make_uint2(packed[0], packed[1]);
+                if (count > 0) st_row4(p.cin + (size_t)slot * H + u0, vec, count, cv);
               }
-              *reinterpret_cast<uint2*>(p.hb + (size_t)node * Hp + u0) = make_uint2(packed[0], packed[1]);
               if (count > 0) {
                 st_row4(p.h + (size_t)node * H + u0, vec, count, hv);
                 st_row4(p.c + (size_t)node * H + u0, vec, count, cv);
@@ -451,6 +471,8 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
               }
             }
           }
+          // the operand rows written above are read through TMA (async proxy) by later wavefronts
+          asm volatile("fence.proxy.async;" ::: "memory");
           tc_fence_before();
           mbar_arrive(tempty_bar(acc));              // accumulator stage may be overwritten
         }
@@ -463,7 +485,8 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
       // loop is left by all of them together.
       __syncthreads();
       if (*s_abort) break;
-      if (!grid_barrier(p.st, (unsigned)(lvl + 1) * gridDim.x, p.wait_limit, s_flag)) break;
+      ++barriers_passed;
+      if (!grid_barrier(p.st, barriers_passed * gridDim.x, p.wait_limit, s_flag)) break;
     }
   }
 
@@ -520,7 +543,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-int make_tmap(treelstm* ctx, CUtensorMap* map, void* base, uint64_t inner, uint64_t rows, uint32_t box_rows) {
+int make_tmap(treelstm* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows) {
   static EncodeTiledFn encode = nullptr;
   if (!encode) {
     void* fn = nullptr;
@@ -533,7 +556,7 @@ int make_tmap(treelstm* ctx, CUtensorMap* map, void* base, uint64_t inner, uint6
   const cuuint64_t strides[1] = {inner * 2};           // bytes between rows
   const cuuint32_t box[2] = {kKBlock, box_rows};       // 64 bf16 = one 128-byte swizzle span
   const cuuint32_t elem[2] = {1, 1};
-  CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, elem,
+  CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { ctx->cuda_error = (int)r; return TREELSTM_ERR_CUDA; }
@@ -553,6 +576,7 @@ int pack_weights_bf16(treelstm* ctx, cudaStream_t stream) {
   if (rc != TREELSTM_OK) return rc;
   rc = make_tmap(ctx, &ctx->tmap_wx, ctx->Wp_x, (uint64_t)ctx->Ep, (uint64_t)groups * kGColsL, kGColsL);
   if (rc != TREELSTM_OK) return rc;
+  ctx->tmap_ws_base = nullptr;
   ctx->have_tmaps = true;
   return TREELSTM_OK;
 }
@@ -568,15 +592,25 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep; p.sched_ctas = ctx->sm_count;
   p.order = order;
   p.rowA = reinterpret_cast<int*>(base + lay.rowA);
-  p.rowB = reinterpret_cast<int*>(base + lay.rowB);
   p.level_offset = level_offset_dev;
   p.emb_bf = ctx->emb_bf;
-  p.hb = reinterpret_cast<__nv_bfloat16*>(base + lay.hb);
+  p.slot = reinterpret_cast<int*>(base + lay.slot);
+  p.xin = reinterpret_cast<__nv_bfloat16*>(base + lay.xin);
+  p.ain = reinterpret_cast<__nv_bfloat16*>(base + lay.ain);
+  p.cin = reinterpret_cast<float*>(base + lay.cin);
   p.bp_h = ctx->bp_h; p.bp_x = ctx->bp_x;
   p.h = h; p.c = c;
   p.gates = (flags & TREELSTM_SAVE_FOR_BACKWARD) ? reinterpret_cast<float*>(base + lay.gates) : nullptr;
   p.st = reinterpret_cast<DevStatus*>(base + lay.status);
   p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
+  if (ctx->tmap_ws_base != ws || ctx->tmap_ws_rows != n) {   // the dense operands live in the caller's workspace
+    int rc = make_tmap(ctx, &ctx->tmap_x, p.xin, (uint64_t)ctx->Ep, (uint64_t)n, BM);
+    if (rc != TREELSTM_OK) return rc;
+    rc = make_tmap(ctx, &ctx->tmap_a, p.ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, BM);
+    if (rc != TREELSTM_OK) return rc;
+    ctx->tmap_ws_base = ws;
+    ctx->tmap_ws_rows = n;
+  }
 
   static bool attr_set = false;
   if (!attr_set) {
@@ -590,17 +624,23 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     if (grid > want) grid = want;
     if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
     int only = -1;
-    void* args[] = {&ctx->tmap_wh, &ctx->tmap_wx, &p, &only};
+    void* args[] = {&ctx->tmap_wh, &ctx->tmap_wx, &ctx->tmap_x, &ctx->tmap_a, &p, &only};
     TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc, dim3(grid), dim3(kThreads), args,
                                              kSmemBytes, stream));
     ctx->launches += 1;
     return TREELSTM_OK;
   }
+  if (n_levels_host > 0) {
+    const int n_leaves = level_offset_host[1];
+    const int blocks = (int)(((long long)n_leaves * (ctx->Ep / 8) + 255) / 256);
+    k_gather_leaf_rows<<<blocks < 1 ? 1 : (blocks > 2048 ? 2048 : blocks), 256, 0, stream>>>(p);
+    ctx->launches += 1;
+  }
   for (int lvl = 0; lvl < n_levels_host; ++lvl) {
     const int w = level_offset_host[lvl + 1] - level_offset_host[lvl];
     if (w <= 0) continue;
     const int tiles = ((w + BM - 1) / BM) * (groups / choose_groups_per_tile(w, groups, p.sched_ctas));
-    k_fwd_tc<<<tiles, kThreads, kSmemBytes, stream>>>(ctx->tmap_wh, ctx->tmap_wx, p, lvl);
+    k_fwd_tc<<<tiles, kThreads, kSmemBytes, stream>>>(ctx->tmap_wh, ctx->tmap_wx, ctx->tmap_x, ctx->tmap_a, p, lvl);
     ctx->launches += 1;
   }
   TL_CUDA(ctx, cudaGetLastError());

@@ -48,18 +48,30 @@ __device__ __forceinline__ int check_node(int n, int k, int l, int r, const int*
 // After the scan step, bin_starts[b] (b < n_bin_starts) receives the position of the first item
 // with key b.
 // ------------------------------------------------------------------------------------------ //
-template <class KeyFn>
+struct NoPlace {
+  __device__ void operator()(int, int) const {}
+};
+
+template <class KeyFn, class PlaceFn = NoPlace>
 __device__ void block_counting_pass(int n, const int* src, int* dst, KeyFn key, int* hist,
-                                    int* scan_tmp, int* bin_starts, int n_bin_starts) {
+                                    int* scan_tmp, int* bin_starts, int n_bin_starts,
+                                    PlaceFn place = NoPlace()) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int i = tid; i < kRadixBins * kSingleWarps; i += kSingleThreads) hist[i] = 0;
   __syncthreads();
   int per_warp = (n + kSingleWarps - 1) / kSingleWarps;
   per_warp = (per_warp + 31) & ~31;
   const int begin = min(n, warp * per_warp), end = min(n, begin + per_warp);
-  for (int r = begin + lane; r < end; r += 32) {
-    int item = src ? src[r] : r;
-    atomicAdd(&hist[key(item) * kSingleWarps + warp], 1);
+  for (int r0 = begin; r0 < end; r0 += 32) {   // one add per distinct key of the 32 items
+    const int r = r0 + lane;
+    const bool valid = r < end;
+    const unsigned act = __ballot_sync(kFull, valid);
+    if (valid) {
+      const int k = key(src ? src[r] : r);
+      const unsigned peers = __match_any_sync(act, k);
+      if (lane == __ffs(peers) - 1) hist[k * kSingleWarps + warp] += __popc(peers);
+    }
+    __syncwarp();
   }
   __syncthreads();
   // exclusive scan of hist in (bin-major, warp-minor) order: 8 consecutive entries per thread
@@ -108,9 +120,46 @@ __device__ void block_counting_pass(int n, const int* src, int* dst, KeyFn key, 
     __syncwarp();
     if (valid && lane == __ffs(peers) - 1) hist[k * kSingleWarps + warp] = base + __popc(peers);
     __syncwarp();
-    if (valid) dst[base + __popc(peers & lanemask_lt())] = item;
+    if (valid) {
+      const int pos = base + __popc(peers & lanemask_lt());
+      dst[pos] = item;
+      place(pos, item);
+    }
   }
   __syncthreads();
+}
+
+// Ids of the items with flag(item) set, in ascending order, to dst; returns their number to every
+// thread.  One CTA of 32 warps; warp w owns a contiguous range of ids.
+template <class FlagFn>
+__device__ int block_compact(int n, int* dst, FlagFn flag, int* scan_tmp) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int per_warp = (n + kSingleWarps - 1) / kSingleWarps;
+  per_warp = (per_warp + 31) & ~31;
+  const int begin = min(n, warp * per_warp), end = min(n, begin + per_warp);
+  int count = 0;
+  for (int r0 = begin; r0 < end; r0 += 32) {
+    const int r = r0 + lane;
+    count += __popc(__ballot_sync(kFull, r < end && flag(r)));
+  }
+  __syncthreads();
+  if (lane == 0) scan_tmp[warp] = count;
+  __syncthreads();
+  int total = 0, base = 0;
+  for (int w2 = 0; w2 < kSingleWarps; ++w2) {
+    const int c = scan_tmp[w2];
+    if (w2 < warp) base += c;
+    total += c;
+  }
+  for (int r0 = begin; r0 < end; r0 += 32) {
+    const int r = r0 + lane;
+    const bool f = r < end && flag(r);
+    const unsigned m = __ballot_sync(kFull, f);
+    if (f) dst[base + __popc(m & lanemask_lt())] = r;
+    base += __popc(m);
+  }
+  __syncthreads();
+  return total;
 }
 
 // One CTA schedules the whole forest in shared memory (forests up to 32768 nodes).
@@ -125,7 +174,7 @@ __device__ void block_counting_pass(int n, const int* src, int* dst, KeyFn key, 
 __global__ void __launch_bounds__(kSingleThreads, 1)
 k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ right,
                   const int* __restrict__ token, int vocab, int* parent, int* level, int* order,
-                  int* order_tmp, int* level_offset, int* roots, int* rowA, int* rowB,
+                  int* order_tmp, int* level_offset, int* roots, int* rowA, int* rowB, int* slot,
                   int* n_levels_out, DevStatus* st) {
   extern __shared__ __align__(16) unsigned char smem[];
   const size_t w_bytes = (size_t)n * 4 > sizeof(int) * kRadixBins * kSingleWarps
@@ -135,46 +184,82 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
   unsigned short* par = reinterpret_cast<unsigned short*>(smem + w_bytes);
   unsigned short* lv16 = par;
   __shared__ int scan_tmp[32];
-  __shared__ int s_err, s_maxlevel, s_bins[2];
+  __shared__ int s_err, s_maxlevel;
   const int tid = threadIdx.x;
   constexpr unsigned short kNoParent = 0xFFFF;
   constexpr unsigned int kDone = 0x80000000u;
   if (tid < (int)(sizeof(DevStatus) / sizeof(int))) reinterpret_cast<int*>(st)[tid] = 0;
   if (tid == 0) { s_err = 0; s_maxlevel = 0; }
-  for (int k = tid; k < n; k += kSingleThreads) { w[k] = 0; par[k] = kNoParent; }
-  __syncthreads();
-  // validate; children record their caller; leaves are complete at once (level 0)
-#pragma unroll 4
   for (int k = tid; k < n; k += kSingleThreads) {
-    const int l = left[k], r = right[k];
-    bool leaf;
-    const int err = check_node(n, k, l, r, token, vocab, &leaf);
-    if (err) atomicMin(&s_err, err);
-    else if (leaf) w[k] = kDone;
-    else { par[l] = (unsigned short)k; par[r] = (unsigned short)k; }
+    w[k] = 0;
+    par[k] = kNoParent;
+    if (slot) slot[k] = -1;
   }
   __syncthreads();
-  if (s_err == 0) {
-    // a child claimed by two callers kept only one of them
-#pragma unroll 4
-    for (int k = tid; k < n; k += kSingleThreads) {
-      const int l = left[k];
-      if (l >= 0 && (par[l] != k || par[right[k]] != k)) atomicMin(&s_err, (int)TREELSTM_ERR_INVALID_FOREST);
+  // validate; children record their caller; leaves are complete at once (level 0)
+  for (int k0 = tid; k0 < n; k0 += 4 * kSingleThreads) {   // four nodes per trip: loads first
+    int l[4], r[4], t[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int k = k0 + j * kSingleThreads;
+      l[j] = k < n ? left[k] : -1;
+      r[j] = k < n ? right[k] : -1;
+      t[j] = k < n ? token[k] : 0;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int k = k0 + j * kSingleThreads;
+      if (k >= n) break;
+      int err = 0;
+      if (l[j] < 0 && r[j] < 0) {
+        if (l[j] != -1 || r[j] != -1) err = TREELSTM_ERR_INVALID_FOREST;
+        else if (t[j] < 0 || t[j] >= vocab) err = TREELSTM_ERR_TOKEN_OUT_OF_RANGE;
+        else w[k] = kDone;
+      } else if (l[j] < 0 || r[j] < 0 || l[j] >= n || r[j] >= n || l[j] == r[j] || l[j] == k || r[j] == k) {
+        err = TREELSTM_ERR_INVALID_FOREST;
+      } else {
+        par[l[j]] = (unsigned short)k;
+        par[r[j]] = (unsigned short)k;
+      }
+      if (err) atomicMin(&s_err, err);
     }
   }
   __syncthreads();
   if (s_err == 0) {
+    // Pass 1: a child claimed by two callers kept only one of them (checked at the caller); every
+    // leaf reports to its caller.  A caller whose second child reports here is complete (level 1)
+    // and is remembered by the reporting thread.  Pass 2 then climbs from those callers, so no
+    // climb ever waits for a leaf that its owner has not reached yet.
+    constexpr int kMaxReady = 32;              // at most 32768 / 1024 nodes per thread
+    unsigned short ready[kMaxReady];
+    int n_ready = 0;
+#pragma unroll 4
     for (int k = tid; k < n; k += kSingleThreads) {
-      if (left[k] >= 0) continue;
-      int cur = k, lvl = 0;
-      for (int step = 0; step < n; ++step) {   // a path to the root has fewer than n edges
-        const unsigned short p = par[cur];
-        if (p == kNoParent) break;
-        const unsigned int old = atomicExch(&w[p], (unsigned int)lvl + 1u);
-        if (old == 0) break;                   // sibling subtree still unresolved
-        lvl = 1 + max(lvl, (int)old - 1);
-        w[p] = kDone | (unsigned int)lvl;
-        cur = p;
+      const int l = left[k];
+      if (l >= 0) {
+        if (par[l] != k || par[right[k]] != k) atomicMin(&s_err, (int)TREELSTM_ERR_INVALID_FOREST);
+        continue;
+      }
+      const unsigned short p = par[k];
+      if (p == kNoParent) continue;
+      if (atomicExch(&w[p], 1u) != 0) {         // both children are leaves
+        w[p] = kDone | 1u;
+        if (n_ready < kMaxReady) ready[n_ready++] = p;
+      }
+    }
+    __syncthreads();
+    if (s_err == 0) {
+      for (int q = 0; q < n_ready; ++q) {
+        int cur = ready[q], lvl = 1;
+        for (int step = 0; step < n; ++step) {   // a path to the root has fewer than n edges
+          const unsigned short p = par[cur];
+          if (p == kNoParent) break;
+          const unsigned int old = atomicExch(&w[p], (unsigned int)lvl + 1u);
+          if (old == 0) break;                   // sibling subtree still unresolved
+          lvl = 1 + max(lvl, (int)old - 1);
+          w[p] = kDone | (unsigned int)lvl;
+          cur = p;
+        }
       }
     }
   }
@@ -206,8 +291,28 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
     int* dst = ((passes - 1 - p) & 1) ? order_tmp : order;
     const int* src = p == 0 ? nullptr : (dst == order ? order_tmp : order);
     const int shift = 8 * p;
-    block_counting_pass(n, src, dst, [=](int item) { return ((lv16[item] & 0x7FFF) >> shift) & 255; },
-                        hist, scan_tmp, passes == 1 ? level_offset : nullptr, passes == 1 ? n_levels : 0);
+    auto key = [=](int item) { return ((lv16[item] & 0x7FFF) >> shift) & 255; };
+    if (p + 1 < passes || !rowA) {
+      block_counting_pass(n, src, dst, key, hist, scan_tmp, passes == 1 ? level_offset : nullptr,
+                          passes == 1 ? n_levels : 0);
+    } else {
+      // last pass: the final position of a node is known here, so its operand rows (token or left
+      // child, right child) are written along with it
+      block_counting_pass(n, src, dst, key, hist, scan_tmp, passes == 1 ? level_offset : nullptr,
+                          passes == 1 ? n_levels : 0, [=](int pos, int node) {
+                            const int l = left[node];
+                            if (l < 0) {
+                              rowA[pos] = token[node];
+                              rowB[pos] = 0;
+                            } else {
+                              const int r = right[node];
+                              rowA[pos] = l;
+                              rowB[pos] = r;
+                              slot[l] = 2 * pos;        // where each child delivers its state
+                              slot[r] = 2 * pos + 1;
+                            }
+                          });
+    }
   }
   if (passes > 1) {   // wavefront boundaries from the sorted order
     for (int r = tid; r < n; r += kSingleThreads) {
@@ -216,20 +321,9 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
     }
   }
   if (tid == 0) { level_offset[n_levels] = n; st->n_levels = n_levels; *n_levels_out = n_levels; }
-  // roots in ascending node id: stable partition on "has a caller"
-  block_counting_pass(n, nullptr, roots, [=](int item) { return (lv16[item] & 0x8000) ? 0 : 1; }, hist,
-                      scan_tmp, s_bins, 2);
-  if (tid == 0) st->n_roots = s_bins[1];
-  // operand rows of every wavefront position: token (leaf) or left child, and right child
-  if (rowA) {
-#pragma unroll 4
-    for (int r = tid; r < n; r += kSingleThreads) {
-      const int node = order[r];
-      const int l = left[node];
-      rowA[r] = l < 0 ? token[node] : l;
-      rowB[r] = l < 0 ? 0 : right[node];
-    }
-  }
+  // roots (nodes without a caller) in ascending node id
+  const int n_roots = block_compact(n, roots, [=](int item) { return (lv16[item] & 0x8000) != 0; }, scan_tmp);
+  if (tid == 0) st->n_roots = n_roots;
 }
 
 // ------------------------------------------------------------------------------------------ //
@@ -408,15 +502,24 @@ __global__ void k_sched_offsets(int n, const int* level, const int* order, int* 
 }
 
 // Per-row operand indices in ready order: rowA = token (leaf) or left child, rowB = right child.
+// slot[child] = 2 * position of its caller + side; slot[] was preset to -1 (roots keep it).
 __global__ void k_row_operands(int n, const int* order, const int* left, const int* right,
-                               const int* token, int* rowA, int* rowB, const DevStatus* st) {
+                               const int* token, int* rowA, int* rowB, int* slot, const DevStatus* st) {
   if (st->status != 0) return;
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= n) return;
-  const int node = order[r];
+  const int pos = blockIdx.x * blockDim.x + threadIdx.x;
+  if (pos >= n) return;
+  const int node = order[pos];
   const int l = left[node];
-  rowA[r] = l < 0 ? token[node] : l;
-  rowB[r] = l < 0 ? 0 : right[node];
+  if (l < 0) {
+    rowA[pos] = token[node];
+    rowB[pos] = 0;
+  } else {
+    const int r = right[node];
+    rowA[pos] = l;
+    rowB[pos] = r;
+    slot[l] = 2 * pos;
+    slot[r] = 2 * pos + 1;
+  }
 }
 
 __global__ void k_gather_roots(int max_roots, int H, const int* roots, const float* h,
@@ -455,6 +558,7 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   int* table = reinterpret_cast<int*>(base + lay.table);
   int* rowA = reinterpret_cast<int*>(base + lay.rowA);
   int* rowB = reinterpret_cast<int*>(base + lay.rowB);
+  int* slot = reinterpret_cast<int*>(base + lay.slot);
 
   const int single_max = ctx->opt.sched_single_cta_max < kSchedSingleMaxNodes
                              ? ctx->opt.sched_single_cta_max : kSchedSingleMaxNodes;
@@ -468,7 +572,7 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
     // the kernel clears the control block itself and writes the level count to the caller
     k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n), stream>>>(
         n, left, right, token, ctx->vocab, parent, level, order, order_tmp, level_offset, roots, rowA, rowB,
-        n_levels_out, st);
+        slot, n_levels_out, st);
     ctx->launches += 1;
     TL_CUDA(ctx, cudaGetLastError());
     return TREELSTM_OK;
@@ -481,6 +585,7 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   }
   TL_CUDA(ctx, cudaMemsetAsync(parent, 0xFF, sizeof(int) * (size_t)n, stream));
   TL_CUDA(ctx, cudaMemsetAsync(pending, 0, sizeof(int) * (size_t)n, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(slot, 0xFF, sizeof(int) * (size_t)n, stream));
   const int tpb = 256, blocks = (n + tpb - 1) / tpb;
   k_sched_init<<<blocks, tpb, 0, stream>>>(n, left, right, token, ctx->vocab, parent, level, st);
   k_sched_walkup<<<blocks, tpb, 0, stream>>>(n, left, right, parent, pending, level, st);
@@ -505,7 +610,7 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   k_radix_scan<<<1, 1024, 0, stream>>>(1, 0, table, n_chunks, st);
   k_radix_scatter<<<n_chunks, 32, 0, stream>>>(n, 1, 0, level, parent, order, order_tmp, roots,
                                                table, n_chunks, st);
-  k_row_operands<<<blocks, tpb, 0, stream>>>(n, order, left, right, token, rowA, rowB, st);
+  k_row_operands<<<blocks, tpb, 0, stream>>>(n, order, left, right, token, rowA, rowB, slot, st);
   ctx->launches += 5;
   TL_CUDA(ctx, cudaGetLastError());
   TL_CUDA(ctx, cudaMemcpyAsync(n_levels_out, &st->n_levels, sizeof(int), cudaMemcpyDeviceToDevice, stream));
@@ -573,7 +678,7 @@ extern "C" int treelstm_schedule_static(int n_nodes, const int32_t* left, const 
     // to clear it, everything else in the array is rewritten before it is read
     k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n_nodes), s>>>(
         n_nodes, left, right, token, vocab, parent, level, order, order_tmp, level_offset, roots, nullptr,
-        nullptr, n_levels, st);
+        nullptr, nullptr, n_levels, st);
     if (cudaGetLastError() != cudaSuccess) return TREELSTM_ERR_CUDA;
   } else {
     if (cudaMemsetAsync(st, 0, sizeof(DevStatus), s) != cudaSuccess ||
