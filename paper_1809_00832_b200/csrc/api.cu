@@ -18,8 +18,6 @@ WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward) {
   L.level_offset = take(4 * (nn + 2));
   L.roots = take(4 * nn);
   L.table = take(4 * (size_t)kRadixBins * ((nn + kRadixChunk - 1) / kRadixChunk));
-  L.rowA = take(4 * nn);
-  L.rowB = take(4 * nn);
   L.slot = take(4 * nn);
   L.xin = L.ain = L.cin = off;
   if (ctx->precision == TREELSTM_BF16) {

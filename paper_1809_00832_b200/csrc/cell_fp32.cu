@@ -21,7 +21,7 @@ constexpr int kWLoads = KC * 5 * TU / kThreads;    // 10 weight elements per thr
 
 struct FwdParams {
   int n, H, E;
-  const int *left, *right, *token, *order, *rowA, *rowB, *level_offset;
+  const int *left, *right, *token, *order, *level_offset;
   const float *emb, *W, *b;
   float *h, *c, *gates;
   DevStatus* st;
@@ -51,8 +51,8 @@ __device__ void fp32_tile(const FwdParams& p, int row0, int row_end, int u0, boo
     int node = -1, l = 0, r = 0;
     if (row < row_end) {
       node = p.order[row];
-      l = p.rowA[row];
-      r = p.rowB[row];
+      l = leaf ? p.token[node] : p.left[node];
+      r = leaf ? 0 : p.right[node];
     }
     s.node[i] = node; s.l[i] = l; s.r[i] = r;
   }
@@ -186,8 +186,6 @@ int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.n = n; p.H = ctx->H; p.E = ctx->E;
   p.left = left; p.right = right; p.token = token; p.order = order;
   p.level_offset = level_offset_dev;
-  p.rowA = reinterpret_cast<const int*>(base + lay.rowA);
-  p.rowB = reinterpret_cast<const int*>(base + lay.rowB);
   p.emb = ctx->emb; p.W = ctx->W; p.b = ctx->b;
   p.h = h; p.c = c;
   p.gates = (flags & TREELSTM_SAVE_FOR_BACKWARD) ? reinterpret_cast<float*>(base + lay.gates) : nullptr;

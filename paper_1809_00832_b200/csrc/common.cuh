@@ -25,8 +25,8 @@ static_assert(sizeof(DevStatus) == 256, "control block is one 256-byte line grou
 
 // Offsets (bytes) of the regions inside the workspace for a forest of up to n nodes.
 struct WsLayout {
-  size_t status, parent, pending, order_tmp, level_offset, roots, table, rowA, rowB, slot, xin, ain,
-      cin, gates, dh, dc, dz, tok_slot, total;
+  size_t status, parent, pending, order_tmp, level_offset, roots, table, slot, xin, ain, cin, gates,
+      dh, dc, dz, tok_slot, total;
 };
 
 struct Options {

@@ -20,9 +20,10 @@
 // one tiled TMA load per K block feeds the tensor core.  Leaves: the embedding rows are copied
 // once into ready order (Xin) by all CTAs before the first wavefront.
 //
-// Warp roles (320 threads): warps 0-3 and 6-9 epilogue (tensor-memory lane quadrant = warp id
-// mod 4; the two sets split every unit group in halves), warp 4 TMA producer (A and W tiles),
-// warp 5 MMA issuer + tensor-memory owner.
+// Warp roles (352 threads): warps 0-3 and 6-9 epilogue (tensor-memory lane quadrant = warp id
+// mod 4; the two sets split every unit group in halves), warp 4 TMA producer of the A tiles,
+// warp 10 TMA producer of the W tiles (issuing a TMA load costs its thread about a hundred
+// cycles, so the two streams are issued side by side), warp 5 MMA issuer + tensor-memory owner.
 #include "common.cuh"
 
 namespace tl {
@@ -30,7 +31,7 @@ namespace {
 
 constexpr int BM = 128;                 // nodes per tile (UMMA M)
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 constexpr int kABytes = BM * 128;       // one K block (64 bf16) of 128 rows
 constexpr int kAccCols = 256;           // accumulator stage stride in tensor-memory columns
 constexpr unsigned kFull = 0xffffffffu;
@@ -61,7 +62,8 @@ __host__ __device__ inline int choose_groups_per_tile(int rows, int groups, int 
 
 struct TcParams {
   int n, H, Hp, Ep, sched_ctas;
-  const int *order, *rowA, *slot, *level_offset;
+  const int *left, *right, *token, *order, *roots, *level_offset;
+  int* slot;
   const __nv_bfloat16* emb_bf;
   __nv_bfloat16 *xin, *ain;
   float* cin;
@@ -196,25 +198,36 @@ __device__ __forceinline__ void st_row4(float* p, bool vec, int count, const flo
 }
 
 // ---- the kernel -------------------------------------------------------------------------------- //
-// Embedding rows of the leaves into ready order: Xin[r] = emb_bf[token of the r-th leaf].
-__device__ void gather_leaf_rows(const TcParams& p, int n_leaves, int gtid, int gthreads) {
+// Before the first wavefront, spread over all threads of the grid:
+//   * Xin[r] = emb_bf[token of the r-th leaf]: the embedding rows in ready order;
+//   * slot[child] = 2 * pos + side for the two children of the node at every internal position pos
+//     (where that child will deliver its state), slot[root] = -1.
+__device__ void prepare_operands(const TcParams& p, int gtid, int gthreads) {
+  const int n_leaves = p.level_offset[1];
   const int cpr = p.Ep / 8;                              // 16-byte chunks per row
   const long long total = (long long)n_leaves * cpr;
   for (long long ch = gtid; ch < total; ch += gthreads) {
     const int row = (int)(ch / cpr), cc = (int)(ch % cpr);
-    const int tok = p.rowA[row];
+    const int tok = p.token[p.order[row]];
     const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.emb_bf + (size_t)tok * p.Ep) + cc);
     reinterpret_cast<uint4*>(p.xin + (size_t)row * p.Ep)[cc] = v;
   }
+  for (int pos = n_leaves + gtid; pos < p.n; pos += gthreads) {
+    const int node = p.order[pos];
+    p.slot[p.left[node]] = 2 * pos;
+    p.slot[p.right[node]] = 2 * pos + 1;
+  }
+  const int n_roots = p.st->n_roots;
+  for (int t = gtid; t < n_roots; t += gthreads) p.slot[p.roots[t]] = -1;
 }
 
-__global__ void k_gather_leaf_rows(TcParams p) {
+__global__ void k_prepare_operands(TcParams p) {
   if (ld_volatile(&p.st->status) != 0) return;
-  gather_leaf_rows(p, p.level_offset[1], blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
+  prepare_operands(p, blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
 }
 
-// only_level >= 0: process that wavefront only (one launch per level; Xin already filled).
-// only_level < 0: fill Xin, then all wavefronts, separated by the bounded grid barrier (cooperative
+// only_level >= 0: process that wavefront only (one launch per level; operands prepared before).
+// only_level < 0: prepare the operands, then all wavefronts, separated by the bounded grid barrier (cooperative
 // launch).
 __global__ void __launch_bounds__(kThreads, 1)
 k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CUtensorMap tmap_wx,
@@ -242,7 +255,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   const int n_levels = p.st->n_levels;
 
   if (tid == 0) {
-    for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -268,7 +281,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   bool stop = false;                    // uniform over the CTA
 
   if (only_level < 0 && n_levels > 0) {
-    gather_leaf_rows(p, p.level_offset[1], blockIdx.x * kThreads + tid, gridDim.x * kThreads);
+    prepare_operands(p, blockIdx.x * kThreads + tid, gridDim.x * kThreads);
     asm volatile("fence.proxy.async;" ::: "memory");    // Xin is read through TMA
     ++barriers_passed;
     if (!grid_barrier(p.st, barriers_passed * gridDim.x, p.wait_limit, s_flag)) stop = true;
@@ -289,20 +302,20 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
     const uint32_t stage_bytes = kABytes + (uint32_t)G * kGColsI * 128u;
     const uint32_t n_stages = min((uint32_t)kMaxStages, (uint32_t)kRingBytes / stage_bytes);
     stage = 0;
-    if (warp == 4) asm volatile("fence.proxy.async;" ::: "memory");   // TMA reads after the barrier's acquire
+    if (warp == 4 || warp == 10) asm volatile("fence.proxy.async;" ::: "memory");   // TMA reads after the barrier's acquire
 
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
       const int row0 = begin + (t / ntn) * BM, nt = t % ntn;
 
-      if (warp == 4) {
-        // ---------------- operand producer (TMA) ----------------
-        // A: 128 consecutive rows of the dense operand matrix (rows past its end read as zero, rows
-        // past the wavefront belong to later wavefronts and only feed accumulator rows that are
-        // never stored).  W: one box per unit group of the packed weights.
+      if (warp == 4 || warp == 10) {
+        // ---------------- operand producers (TMA) ----------------
+        // Warp 4, A: 128 consecutive rows of the dense operand matrix (rows past its end read as
+        // zero, rows past the wavefront belong to later wavefronts and only feed accumulator rows
+        // that are never stored).  Warp 10, W: one box per unit group of the packed weights.
         if (lane == 0) {
-          const CUtensorMap* map_w = leaf ? &tmap_wx : &tmap_wh;
-          const CUtensorMap* map_a = leaf ? &tmap_x : &tmap_a;
-          const uint32_t bytes = (uint32_t)kABytes + (uint32_t)ncols * 128u;
+          const bool is_a = warp == 4;
+          const CUtensorMap* map = is_a ? (leaf ? &tmap_x : &tmap_a) : (leaf ? &tmap_wx : &tmap_wh);
+          const uint32_t bytes = is_a ? (uint32_t)kABytes : (uint32_t)ncols * 128u;
           for (int kb = 0; kb < kblocks; ++kb) {
             if (!mbar_wait(empty_bar(stage), ((phase_bits >> stage) & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) {
               alive = false;
@@ -310,10 +323,13 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
             }
             const uint32_t sa = tiles_addr + stage * stage_bytes;
             mbar_arrive_expect_tx(full_bar(stage), bytes);
-            tma_load_2d(sa, map_a, kb * kKBlock, row0, full_bar(stage));
-            for (int g = 0; g < G; ++g)
-              tma_load_2d(sa + kABytes + (uint32_t)(g * gcols) * 128u, map_w, kb * kKBlock,
-                          (nt * G + g) * gcols, full_bar(stage));
+            if (is_a) {
+              tma_load_2d(sa, map, kb * kKBlock, row0, full_bar(stage));
+            } else {
+              for (int g = 0; g < G; ++g)
+                tma_load_2d(sa + kABytes + (uint32_t)(g * gcols) * 128u, map, kb * kKBlock,
+                            (nt * G + g) * gcols, full_bar(stage));
+            }
             phase_bits ^= 1u << stage;
             if (++stage == n_stages) stage = 0;
           }
@@ -590,8 +606,9 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   char* base = static_cast<char*>(ws);
   TcParams p;
   p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep; p.sched_ctas = ctx->sm_count;
+  p.left = left; p.right = right; p.token = token;
   p.order = order;
-  p.rowA = reinterpret_cast<int*>(base + lay.rowA);
+  p.roots = reinterpret_cast<int*>(base + lay.roots);
   p.level_offset = level_offset_dev;
   p.emb_bf = ctx->emb_bf;
   p.slot = reinterpret_cast<int*>(base + lay.slot);
@@ -633,7 +650,7 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   if (n_levels_host > 0) {
     const int n_leaves = level_offset_host[1];
     const int blocks = (int)(((long long)n_leaves * (ctx->Ep / 8) + 255) / 256);
-    k_gather_leaf_rows<<<blocks < 1 ? 1 : (blocks > 2048 ? 2048 : blocks), 256, 0, stream>>>(p);
+    k_prepare_operands<<<blocks < 1 ? 1 : (blocks > 2048 ? 2048 : blocks), 256, 0, stream>>>(p);
     ctx->launches += 1;
   }
   for (int lvl = 0; lvl < n_levels_host; ++lvl) {

@@ -169,13 +169,13 @@ __device__ int block_compact(int n, int* dst, FlagFn flag, int* scan_tmp) {
 // and stops, the one that finds its sibling's entry knows both inputs are resolved, gives the caller
 // level 1 + max and goes on upwards.  No global atomics, no grid-wide rounds.
 //
-// Dynamic shared memory: uint32 w[n] (dependency words; later the radix histogram, at least 32 KB)
-// followed by uint16 par[n] (caller of each node; later level | root flag).
+// Dynamic shared memory: uint32 w[n] (dependency words; later the radix histogram, at least 32 KB),
+// uint16 par[n] (caller of each node, the return location of Section 4.1.2; later level | root
+// flag), uint16 queue[n / 2] (start nodes of the climb).
 __global__ void __launch_bounds__(kSingleThreads, 1)
 k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ right,
                   const int* __restrict__ token, int vocab, int* parent, int* level, int* order,
-                  int* order_tmp, int* level_offset, int* roots, int* rowA, int* rowB, int* slot,
-                  int* n_levels_out, DevStatus* st) {
+                  int* order_tmp, int* level_offset, int* roots, int* n_levels_out, DevStatus* st) {
   extern __shared__ __align__(16) unsigned char smem[];
   const size_t w_bytes = (size_t)n * 4 > sizeof(int) * kRadixBins * kSingleWarps
                              ? (((size_t)n * 4 + 15) & ~(size_t)15) : sizeof(int) * kRadixBins * kSingleWarps;
@@ -183,38 +183,38 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
   int* hist = reinterpret_cast<int*>(smem);
   unsigned short* par = reinterpret_cast<unsigned short*>(smem + w_bytes);
   unsigned short* lv16 = par;
+  unsigned short* queue = par + (((size_t)n + 7) & ~(size_t)7);   // start nodes of the climb, at most n / 2
   __shared__ int scan_tmp[32];
-  __shared__ int s_err, s_maxlevel;
+  __shared__ int s_err, s_maxlevel, s_qhead, s_qtail;
   const int tid = threadIdx.x;
   constexpr unsigned short kNoParent = 0xFFFF;
   constexpr unsigned int kDone = 0x80000000u;
   if (tid < (int)(sizeof(DevStatus) / sizeof(int))) reinterpret_cast<int*>(st)[tid] = 0;
-  if (tid == 0) { s_err = 0; s_maxlevel = 0; }
-  for (int k = tid; k < n; k += kSingleThreads) {
-    w[k] = 0;
-    par[k] = kNoParent;
-    if (slot) slot[k] = -1;
-  }
+  if (tid == 0) { s_err = 0; s_maxlevel = 0; s_qhead = 0; s_qtail = 0; }
+  for (int k = tid; k < n; k += kSingleThreads) { w[k] = 0; par[k] = kNoParent; }
   __syncthreads();
   // validate; children record their caller; leaves are complete at once (level 0)
-  for (int k0 = tid; k0 < n; k0 += 4 * kSingleThreads) {   // four nodes per trip: loads first
-    int l[4], r[4], t[4];
+  // Node j of this thread is tid + j * 1024 (at most 32 per thread); leaf_bits remembers which are
+  // leaves so that later passes need not look at the child arrays again.
+  unsigned int leaf_bits = 0;
+  for (int j0 = 0; j0 * kSingleThreads + tid < n; j0 += 8) {   // eight nodes per trip: loads first
+    int l[8], r[8], t[8];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int k = k0 + j * kSingleThreads;
+    for (int j = 0; j < 8; ++j) {
+      const int k = tid + (j0 + j) * kSingleThreads;
       l[j] = k < n ? left[k] : -1;
       r[j] = k < n ? right[k] : -1;
       t[j] = k < n ? token[k] : 0;
     }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int k = k0 + j * kSingleThreads;
+    for (int j = 0; j < 8; ++j) {
+      const int k = tid + (j0 + j) * kSingleThreads;
       if (k >= n) break;
       int err = 0;
       if (l[j] < 0 && r[j] < 0) {
         if (l[j] != -1 || r[j] != -1) err = TREELSTM_ERR_INVALID_FOREST;
         else if (t[j] < 0 || t[j] >= vocab) err = TREELSTM_ERR_TOKEN_OUT_OF_RANGE;
-        else w[k] = kDone;
+        else { w[k] = kDone; leaf_bits |= 1u << (j0 + j); }
       } else if (l[j] < 0 || r[j] < 0 || l[j] >= n || r[j] >= n || l[j] == r[j] || l[j] == k || r[j] == k) {
         err = TREELSTM_ERR_INVALID_FOREST;
       } else {
@@ -226,40 +226,50 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
   }
   __syncthreads();
   if (s_err == 0) {
-    // Pass 1: a child claimed by two callers kept only one of them (checked at the caller); every
-    // leaf reports to its caller.  A caller whose second child reports here is complete (level 1)
-    // and is remembered by the reporting thread.  Pass 2 then climbs from those callers, so no
-    // climb ever waits for a leaf that its owner has not reached yet.
-    constexpr int kMaxReady = 32;              // at most 32768 / 1024 nodes per thread
-    unsigned short ready[kMaxReady];
-    int n_ready = 0;
-#pragma unroll 4
-    for (int k = tid; k < n; k += kSingleThreads) {
-      const int l = left[k];
-      if (l >= 0) {
-        if (par[l] != k || par[right[k]] != k) atomicMin(&s_err, (int)TREELSTM_ERR_INVALID_FOREST);
-        continue;
+    // a child claimed by two callers kept only one of them: checked at the caller
+    for (int j0 = 0; j0 * kSingleThreads + tid < n; j0 += 8) {
+      int l[8], r[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int k = tid + (j0 + j) * kSingleThreads;
+        const bool internal = k < n && !((leaf_bits >> (j0 + j)) & 1u);
+        l[j] = internal ? left[k] : -1;
+        r[j] = internal ? right[k] : -1;
       }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int k = tid + (j0 + j) * kSingleThreads;
+        if (l[j] >= 0 && (par[l[j]] != k || par[r[j]] != k)) atomicMin(&s_err, (int)TREELSTM_ERR_INVALID_FOREST);
+      }
+    }
+    // Every leaf reports to its caller.  A caller whose second child reports here is complete
+    // (level 1) and goes into the queue of nodes to climb from; climbing starts only after all
+    // leaves have reported, so no climb waits for a leaf its owner has not reached yet.
+    for (unsigned int bits = leaf_bits; bits; bits &= bits - 1) {
+      const int k = tid + (__ffs(bits) - 1) * kSingleThreads;
       const unsigned short p = par[k];
       if (p == kNoParent) continue;
       if (atomicExch(&w[p], 1u) != 0) {         // both children are leaves
         w[p] = kDone | 1u;
-        if (n_ready < kMaxReady) ready[n_ready++] = p;
+        queue[atomicAdd(&s_qtail, 1)] = p;
       }
     }
-    __syncthreads();
-    if (s_err == 0) {
-      for (int q = 0; q < n_ready; ++q) {
-        int cur = ready[q], lvl = 1;
-        for (int step = 0; step < n; ++step) {   // a path to the root has fewer than n edges
-          const unsigned short p = par[cur];
-          if (p == kNoParent) break;
-          const unsigned int old = atomicExch(&w[p], (unsigned int)lvl + 1u);
-          if (old == 0) break;                   // sibling subtree still unresolved
-          lvl = 1 + max(lvl, (int)old - 1);
-          w[p] = kDone | (unsigned int)lvl;
-          cur = p;
-        }
+  }
+  __syncthreads();
+  if (s_err == 0) {
+    // Climb: threads take start nodes from the queue until it is empty.
+    for (;;) {
+      const int q = atomicAdd(&s_qhead, 1);
+      if (q >= s_qtail) break;
+      int cur = queue[q], lvl = 1;
+      for (int step = 0; step < n; ++step) {   // a path to the root has fewer than n edges
+        const unsigned short p = par[cur];
+        if (p == kNoParent) break;
+        const unsigned int old = atomicExch(&w[p], (unsigned int)lvl + 1u);
+        if (old == 0) break;                   // sibling subtree still unresolved
+        lvl = 1 + max(lvl, (int)old - 1);
+        w[p] = kDone | (unsigned int)lvl;
+        cur = p;
       }
     }
   }
@@ -273,7 +283,6 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
       const unsigned short pk = par[k];
       lv16[k] = (unsigned short)(lvl | (pk == kNoParent ? 0x8000 : 0));
       level[k] = lvl;
-      parent[k] = pk == kNoParent ? -1 : (int)pk;
       local_max = max(local_max, lvl);
     }
     atomicMax(&s_maxlevel, local_max);
@@ -291,28 +300,8 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
     int* dst = ((passes - 1 - p) & 1) ? order_tmp : order;
     const int* src = p == 0 ? nullptr : (dst == order ? order_tmp : order);
     const int shift = 8 * p;
-    auto key = [=](int item) { return ((lv16[item] & 0x7FFF) >> shift) & 255; };
-    if (p + 1 < passes || !rowA) {
-      block_counting_pass(n, src, dst, key, hist, scan_tmp, passes == 1 ? level_offset : nullptr,
-                          passes == 1 ? n_levels : 0);
-    } else {
-      // last pass: the final position of a node is known here, so its operand rows (token or left
-      // child, right child) are written along with it
-      block_counting_pass(n, src, dst, key, hist, scan_tmp, passes == 1 ? level_offset : nullptr,
-                          passes == 1 ? n_levels : 0, [=](int pos, int node) {
-                            const int l = left[node];
-                            if (l < 0) {
-                              rowA[pos] = token[node];
-                              rowB[pos] = 0;
-                            } else {
-                              const int r = right[node];
-                              rowA[pos] = l;
-                              rowB[pos] = r;
-                              slot[l] = 2 * pos;        // where each child delivers its state
-                              slot[r] = 2 * pos + 1;
-                            }
-                          });
-    }
+    block_counting_pass(n, src, dst, [=](int item) { return ((lv16[item] & 0x7FFF) >> shift) & 255; },
+                        hist, scan_tmp, passes == 1 ? level_offset : nullptr, passes == 1 ? n_levels : 0);
   }
   if (passes > 1) {   // wavefront boundaries from the sorted order
     for (int r = tid; r < n; r += kSingleThreads) {
@@ -501,27 +490,6 @@ __global__ void k_sched_offsets(int n, const int* level, const int* order, int* 
   if (r == 0 || level[order[r - 1]] != a) level_offset[a] = r;
 }
 
-// Per-row operand indices in ready order: rowA = token (leaf) or left child, rowB = right child.
-// slot[child] = 2 * position of its caller + side; slot[] was preset to -1 (roots keep it).
-__global__ void k_row_operands(int n, const int* order, const int* left, const int* right,
-                               const int* token, int* rowA, int* rowB, int* slot, const DevStatus* st) {
-  if (st->status != 0) return;
-  const int pos = blockIdx.x * blockDim.x + threadIdx.x;
-  if (pos >= n) return;
-  const int node = order[pos];
-  const int l = left[node];
-  if (l < 0) {
-    rowA[pos] = token[node];
-    rowB[pos] = 0;
-  } else {
-    const int r = right[node];
-    rowA[pos] = l;
-    rowB[pos] = r;
-    slot[l] = 2 * pos;
-    slot[r] = 2 * pos + 1;
-  }
-}
-
 __global__ void k_gather_roots(int max_roots, int H, const int* roots, const float* h,
                                const float* c, int* root_ids, float* root_h, float* root_c,
                                int* n_roots_out, const DevStatus* st) {
@@ -543,7 +511,7 @@ size_t single_smem_bytes(int n) {
   size_t w = (size_t)n * 4;
   const size_t hist = sizeof(int) * kRadixBins * kSingleWarps;
   w = w > hist ? round_up_sz(w, 16) : hist;
-  return w + round_up_sz((size_t)n * 2, 16);
+  return w + round_up_sz((size_t)n * 2, 16) + round_up_sz((size_t)n, 16);
 }
 
 int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
@@ -556,9 +524,6 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   int* order_tmp = reinterpret_cast<int*>(base + lay.order_tmp);
   int* roots = reinterpret_cast<int*>(base + lay.roots);
   int* table = reinterpret_cast<int*>(base + lay.table);
-  int* rowA = reinterpret_cast<int*>(base + lay.rowA);
-  int* rowB = reinterpret_cast<int*>(base + lay.rowB);
-  int* slot = reinterpret_cast<int*>(base + lay.slot);
 
   const int single_max = ctx->opt.sched_single_cta_max < kSchedSingleMaxNodes
                              ? ctx->opt.sched_single_cta_max : kSchedSingleMaxNodes;
@@ -571,8 +536,8 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
     }
     // the kernel clears the control block itself and writes the level count to the caller
     k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n), stream>>>(
-        n, left, right, token, ctx->vocab, parent, level, order, order_tmp, level_offset, roots, rowA, rowB,
-        slot, n_levels_out, st);
+        n, left, right, token, ctx->vocab, parent, level, order, order_tmp, level_offset, roots, n_levels_out,
+        st);
     ctx->launches += 1;
     TL_CUDA(ctx, cudaGetLastError());
     return TREELSTM_OK;
@@ -585,7 +550,6 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   }
   TL_CUDA(ctx, cudaMemsetAsync(parent, 0xFF, sizeof(int) * (size_t)n, stream));
   TL_CUDA(ctx, cudaMemsetAsync(pending, 0, sizeof(int) * (size_t)n, stream));
-  TL_CUDA(ctx, cudaMemsetAsync(slot, 0xFF, sizeof(int) * (size_t)n, stream));
   const int tpb = 256, blocks = (n + tpb - 1) / tpb;
   k_sched_init<<<blocks, tpb, 0, stream>>>(n, left, right, token, ctx->vocab, parent, level, st);
   k_sched_walkup<<<blocks, tpb, 0, stream>>>(n, left, right, parent, pending, level, st);
@@ -610,8 +574,7 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   k_radix_scan<<<1, 1024, 0, stream>>>(1, 0, table, n_chunks, st);
   k_radix_scatter<<<n_chunks, 32, 0, stream>>>(n, 1, 0, level, parent, order, order_tmp, roots,
                                                table, n_chunks, st);
-  k_row_operands<<<blocks, tpb, 0, stream>>>(n, order, left, right, token, rowA, rowB, slot, st);
-  ctx->launches += 5;
+  ctx->launches += 4;
   TL_CUDA(ctx, cudaGetLastError());
   TL_CUDA(ctx, cudaMemcpyAsync(n_levels_out, &st->n_levels, sizeof(int), cudaMemcpyDeviceToDevice, stream));
   return TREELSTM_OK;
@@ -677,8 +640,7 @@ extern "C" int treelstm_schedule_static(int n_nodes, const int32_t* left, const 
     // the control block keeps the previous call's status and counts; the kernel's first step is
     // to clear it, everything else in the array is rewritten before it is read
     k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n_nodes), s>>>(
-        n_nodes, left, right, token, vocab, parent, level, order, order_tmp, level_offset, roots, nullptr,
-        nullptr, nullptr, n_levels, st);
+        n_nodes, left, right, token, vocab, parent, level, order, order_tmp, level_offset, roots, n_levels, st);
     if (cudaGetLastError() != cudaSuccess) return TREELSTM_ERR_CUDA;
   } else {
     if (cudaMemsetAsync(st, 0, sizeof(DevStatus), s) != cudaSuccess ||
