@@ -123,11 +123,49 @@ def oracle_sample_time(w: fg.Workload, budget_s: float = 15.0):
     avg_nodes = w.forest.n_nodes / w.forest.n_trees
     want = int(max(8, min(w.forest.n_trees, budget_s / max(per_node * avg_nodes, 1e-9))))
     sample = fg.select_trees(w.forest, list(range(want)))
+    # whole passes over the sample until about budget_s seconds of CPU work are done
+    passes = int(max(1, min(200, round(budget_s / max(per_node * sample.n_nodes, 1e-9)))))
     t0 = time.perf_counter()
-    orc.schedule(sample.left, sample.right)
-    orc.forward_recursive(sample.left, sample.right, sample.token, p.emb, p.W, p.b)
+    for _ in range(passes):
+        orc.schedule(sample.left, sample.right)
+        orc.forward_recursive(sample.left, sample.right, sample.token, p.emb, p.W, p.b)
     dt = time.perf_counter() - t0
-    return sample.n_trees, sample.n_nodes, dt, threads
+    return sample.n_trees * passes, sample.n_nodes * passes, dt, threads
+
+
+def train_step_time(steps: int = 200, warmup: int = 5):
+    """Extra figure: the training step (forward keeping activations + backward through structure) on
+    the 25-tree fp32 workload, timed with CUDA events, L2 flushed between steps."""
+    import torch
+    from paper_1809_00832_b200 import binding
+    w = fg.make_workload("train25_fp32", 0)
+    f, p = w.forest, w.params
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    model = binding.TreeLSTM(p.H, p.E, p.vocab, dev(p.emb), dev(p.W), dev(p.b), binding.FP32)
+    model.set_classifier(dev(p.Wc), dev(p.bc))
+    left, right, token, labels = dev(f.left), dev(f.right), dev(f.token), dev(w.labels)
+    flags = binding.PERSISTENT | binding.SAVE_FOR_BACKWARD
+    out = model.forward(left, right, token, flags=flags)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    launches = 0
+    for i in range(-warmup, steps):
+        flush.fill_(i & 0xFF)
+        if i >= 0:
+            ev[i][0].record()
+        model.forward(left, right, token, flags=flags, out=out, check=False)
+        launches = model.last_launch_count()
+        model.backward(labels, f.n_leaves)
+        launches += model.last_launch_count()
+        if i >= 0:
+            ev[i][1].record()
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in ev]
+    mean = sum(ms) / len(ms)
+    return {"workload": "train25_fp32", "trees": f.n_trees, "nodes": f.n_nodes, "ms_per_step": mean,
+            "trees_per_sec": f.n_trees / (mean * 1e-3), "nodes_per_sec": f.n_nodes / (mean * 1e-3),
+            "steps": steps, "gpu_launches_per_step": launches, "dtype": "f32",
+            "note": "backward reads the level table back once per step (one stream synchronisation)"}
 
 
 def run_reference(args):
@@ -188,6 +226,7 @@ def main() -> int:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="persistent", choices=["persistent", "per_level"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-train", action="store_true", help="skip the extra training-step figure")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -313,10 +352,12 @@ def main() -> int:
                      "tensor_tflops": achieved_tflops,
                      "tensor_frac_of_sustained": achieved_tflops / peaks["bf16_tflops_sustained"]},
     }
+    if world == 1 and not args.no_train:
+        line["train_step"] = train_step_time()
     if world == 1 and not args.no_cpu_baseline:
         trees, nodes, secs, threads = oracle_sample_time(w)
         line["cpu_baseline"] = {"value": trees / secs, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                "sample": f"first {trees} of {f.n_trees} trees ({nodes} nodes), {secs:.1f} s",
+                                "sample": f"{trees} trees ({nodes} nodes) = whole passes over the first trees of the workload, {secs:.1f} s",
                                 "nodes_per_sec": nodes / secs}
     print(json.dumps(line))
     if dist is not None:

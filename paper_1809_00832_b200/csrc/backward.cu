@@ -168,12 +168,15 @@ __global__ void k_bwd_gates(BwdParams p, int row_begin, int row_end, int leaf) {
 
 // ---- dIn = dz W^T for one wavefront --------------------------------------------------------- //
 // out[row][k] = sum_j dz[row][j] * W[koff + k][j]; tile 64 rows x 64 outputs, 16 x 16 threads.
-constexpr int BT = 64, BK = 16;
+// The next chunk of the contraction is fetched into registers while the current one is
+// multiplied out of shared memory (two buffers, one CTA barrier per chunk).
+constexpr int BT = 64, BK = 32;
+constexpr int kLd = BT * BK / 256;   // elements of each operand per thread and chunk
 
 __global__ void __launch_bounds__(256)
 k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
-  __shared__ float As[BT][BK + 1];
-  __shared__ float Bs[BT][BK + 1];
+  __shared__ float As[2][BT][BK + 1];
+  __shared__ float Bs[2][BT][BK + 1];
   __shared__ int s_node[BT];
   const int H = p.H, E = p.E, J = 5 * H;
   const int K = leaf ? E : 2 * H, koff = leaf ? 0 : E;
@@ -183,23 +186,41 @@ k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
   for (int i = tid; i < BT; i += 256) s_node[i] = row0 + i < row_end ? p.order[row0 + i] : -1;
   __syncthreads();
   float acc[4][4] = {};
-  for (int j0 = 0; j0 < J; j0 += BK) {
-    for (int e = tid; e < BT * BK; e += 256) {
-      const int i = e / BK, jj = e % BK, j = j0 + jj;
-      As[i][jj] = (s_node[i] >= 0 && j < J) ? p.dz[(size_t)s_node[i] * J + j] : 0.f;
-      Bs[i][jj] = (k0 + i < K && j < J) ? __ldg(p.W + (size_t)(koff + k0 + i) * J + j) : 0.f;
+  float ra[kLd], rb[kLd];
+  auto fetch = [&](int j0) {
+#pragma unroll
+    for (int q = 0; q < kLd; ++q) {
+      const int e = tid + q * 256, i = e / BK, j = j0 + e % BK;
+      ra[q] = (s_node[i] >= 0 && j < J) ? p.dz[(size_t)s_node[i] * J + j] : 0.f;
+      rb[q] = (k0 + i < K && j < J) ? __ldg(p.W + (size_t)(koff + k0 + i) * J + j) : 0.f;
     }
-    __syncthreads();
+  };
+  auto stash = [&](int buf) {
+#pragma unroll
+    for (int q = 0; q < kLd; ++q) {
+      const int e = tid + q * 256;
+      As[buf][e / BK][e % BK] = ra[q];
+      Bs[buf][e / BK][e % BK] = rb[q];
+    }
+  };
+  fetch(0);
+  stash(0);
+  __syncthreads();
+  const int chunks = (J + BK - 1) / BK;
+  for (int cidx = 0; cidx < chunks; ++cidx) {
+    const int buf = cidx & 1;
+    if (cidx + 1 < chunks) fetch((cidx + 1) * BK);
 #pragma unroll
     for (int jj = 0; jj < BK; ++jj) {
       float a[4], b[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) { a[i] = As[ty + 16 * i][jj]; b[i] = Bs[tx + 16 * i][jj]; }
+      for (int i = 0; i < 4; ++i) { a[i] = As[buf][ty + 16 * i][jj]; b[i] = Bs[buf][tx + 16 * i][jj]; }
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int q = 0; q < 4; ++q) acc[i][q] = fmaf(a[i], b[q], acc[i][q]);
     }
+    if (cidx + 1 < chunks) stash(buf ^ 1);
     __syncthreads();
   }
 #pragma unroll
@@ -223,11 +244,13 @@ k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
 // ---- dW = In^T dZ (contraction over nodes) and db ------------------------------------------- //
 // part 0: rows [0,E) from the leaves (In = embedding rows); part 1: rows [E,E+2H) from the
 // internal nodes (In = [h_l | h_r]).  Tile 64 (k) x 64 (j); gridDim.y splits the node range.
+constexpr int WR = 16;               // nodes per chunk
+constexpr int kLdW = WR * BT / 256;  // 4 elements of each operand per thread and chunk
+
 __global__ void __launch_bounds__(256)
 k_bwd_dweight(BwdParams p, int part, int row_begin, int row_end, int rows_per_split) {
-  __shared__ float As[BK][BT];
-  __shared__ float Bs[BK][BT];
-  __shared__ int s_a[BK], s_b[BK], s_node[BK];
+  __shared__ float As[2][WR][BT];
+  __shared__ float Bs[2][WR][BT];
   const int H = p.H, E = p.E, J = 5 * H;
   const int K = part == 0 ? E : 2 * H, koff = part == 0 ? 0 : E;
   const int tiles_j = (J + BT - 1) / BT;
@@ -236,42 +259,54 @@ k_bwd_dweight(BwdParams p, int part, int row_begin, int row_end, int rows_per_sp
   const int r_hi = min(row_end, r_lo + rows_per_split);
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   float acc[4][4] = {};
-  for (int r0 = r_lo; r0 < r_hi; r0 += BK) {
-    if (tid < BK) {
-      const int row = r0 + tid;
-      int node = -1, a = 0, b = 0;
-      if (row < r_hi) {
-        node = p.order[row];
-        a = part == 0 ? p.token[node] : p.left[node];
-        b = part == 0 ? 0 : p.right[node];
-      }
-      s_node[tid] = node; s_a[tid] = a; s_b[tid] = b;
-    }
-    __syncthreads();
-    for (int e = tid; e < BK * BT; e += 256) {
-      const int rr = e / BT, cc = e % BT;
-      float va = 0.f, vb = 0.f;
-      if (s_node[rr] >= 0) {
-        const int k = k0 + cc, j = j0 + cc;
-        if (k < K)
-          va = part == 0 ? __ldg(p.emb + (size_t)s_a[rr] * E + k)
-                         : (k < H ? p.h[(size_t)s_a[rr] * H + k] : p.h[(size_t)s_b[rr] * H + (k - H)]);
-        if (j < J) vb = p.dz[(size_t)s_node[rr] * J + j];
-      }
-      As[rr][cc] = va;
-      Bs[rr][cc] = vb;
-    }
-    __syncthreads();
+  float ra[kLdW], rb[kLdW];
+  // element e of a chunk: node rr = e / 64 of the chunk, column cc = e % 64 of the tile
+  auto fetch = [&](int r0) {
 #pragma unroll
-    for (int rr = 0; rr < BK; ++rr) {
+    for (int q = 0; q < kLdW; ++q) {
+      const int e = tid + q * 256, rr = e / BT, cc = e % BT;
+      const int row = r0 + rr;
+      float va = 0.f, vb = 0.f;
+      if (row < r_hi) {
+        const int node = p.order[row];
+        const int k = k0 + cc, j = j0 + cc;
+        if (k < K) {
+          if (part == 0) va = __ldg(p.emb + (size_t)p.token[node] * E + k);
+          else va = k < H ? p.h[(size_t)p.left[node] * H + k] : p.h[(size_t)p.right[node] * H + (k - H)];
+        }
+        if (j < J) vb = p.dz[(size_t)node * J + j];
+      }
+      ra[q] = va;
+      rb[q] = vb;
+    }
+  };
+  auto stash = [&](int buf) {
+#pragma unroll
+    for (int q = 0; q < kLdW; ++q) {
+      const int e = tid + q * 256;
+      As[buf][e / BT][e % BT] = ra[q];
+      Bs[buf][e / BT][e % BT] = rb[q];
+    }
+  };
+  if (r_lo < r_hi) {
+    fetch(r_lo);
+    stash(0);
+  }
+  __syncthreads();
+  int buf = 0;
+  for (int r0 = r_lo; r0 < r_hi; r0 += WR, buf ^= 1) {
+    if (r0 + WR < r_hi) fetch(r0 + WR);
+#pragma unroll
+    for (int rr = 0; rr < WR; ++rr) {
       float a[4], b[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) { a[i] = As[rr][ty + 16 * i]; b[i] = Bs[rr][tx + 16 * i]; }
+      for (int i = 0; i < 4; ++i) { a[i] = As[buf][rr][ty + 16 * i]; b[i] = Bs[buf][rr][tx + 16 * i]; }
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int q = 0; q < 4; ++q) acc[i][q] = fmaf(a[i], b[q], acc[i][q]);
     }
+    if (r0 + WR < r_hi) stash(buf ^ 1);
     __syncthreads();
   }
 #pragma unroll
@@ -357,7 +392,7 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
     const int begin = part == 0 ? 0 : p.n_leaves, end = part == 0 ? p.n_leaves : n;
     if (end <= begin) continue;
     const int K = part == 0 ? E : 2 * H;
-    const int rows_per_split = 256;
+    const int rows_per_split = 128;
     const int splits = (end - begin + rows_per_split - 1) / rows_per_split;
     dim3 grid(((K + BT - 1) / BT) * tiles_j, splits);
     k_bwd_dweight<<<grid, 256, 0, stream>>>(p, part, begin, end, rows_per_split);

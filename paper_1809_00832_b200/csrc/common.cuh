@@ -70,7 +70,7 @@ struct treelstm {
   __nv_bfloat16* Wp_x = nullptr;    // [(Hp/8)*24][Ep]    packed input weights (gates i, o, u)
   float* bp_h = nullptr;            // [(Hp/8)*40] bias in packed column order
   float* bp_x = nullptr;            // [(Hp/8)*24]
-  CUtensorMap tmap_wh, tmap_wx, tmap_x, tmap_a;
+  CUtensorMap tmap_wh, tmap_wx, tmap_x, tmap_a, tmap_a64, tmap_a32;
   const void* tmap_ws_base = nullptr;   // tmap_x / tmap_a are rebuilt when the workspace or node count changes
   int tmap_ws_rows = 0;
   bool have_tmaps = false;
@@ -166,24 +166,34 @@ __device__ __forceinline__ int ld_volatile(const int* p) { return *(const volati
 __device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
                                              long long limit_cycles, int* s_flag) {
   __syncthreads();
-  if (threadIdx.x == 0) {
-    // release: everything this CTA wrote (ordered before by the CTA barrier) is visible to whoever
-    // acquires the counter afterwards
-    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&st->barrier) : "memory");
-    long long t0 = clock64();
-    int ok = 1;
-    for (;;) {
-      unsigned int seen;
-      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&st->barrier) : "memory");
-      if (seen >= target) break;
-      if (*(volatile int*)&st->status != 0) { ok = 0; break; }
-      if (clock64() - t0 > limit_cycles) {
-        report(st, TREELSTM_ERR_TIMEOUT);
-        ok = 0;
-        break;
+  if (threadIdx.x < 32) {
+    // Warp 0 polls.  Lane 0 announces the arrival (release: everything this CTA wrote, ordered
+    // before by the CTA barrier, is visible to whoever acquires the counter afterwards); then eight
+    // lanes read the counter a fraction of a round trip apart, so that the last arrival is seen
+    // after an eighth of the memory latency on average instead of half of it.
+    if (threadIdx.x == 0) {
+      *s_flag = -1;
+      asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&st->barrier) : "memory");
+    }
+    __syncwarp();
+    const int lane = threadIdx.x;
+    if (lane < 8) {
+      const long long t0 = clock64();
+      while (clock64() - t0 < 150 * lane) {}
+      for (;;) {
+        if (*(volatile int*)s_flag >= 0) break;          // another lane has the answer
+        unsigned int seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&st->barrier) : "memory");
+        if (seen >= target) { *(volatile int*)s_flag = 1; break; }
+        if (*(volatile int*)&st->status != 0) { *(volatile int*)s_flag = 0; break; }
+        if (clock64() - t0 > limit_cycles) {
+          report(st, TREELSTM_ERR_TIMEOUT);
+          *(volatile int*)s_flag = 0;
+          break;
+        }
       }
     }
-    *s_flag = ok;
+    __syncwarp();
   }
   __syncthreads();
   return *s_flag != 0;

@@ -232,6 +232,7 @@ __global__ void k_prepare_operands(TcParams p) {
 __global__ void __launch_bounds__(kThreads, 1)
 k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CUtensorMap tmap_wx,
          const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_a,
+         const __grid_constant__ CUtensorMap tmap_a64, const __grid_constant__ CUtensorMap tmap_a32,
          TcParams p, int only_level) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -302,6 +303,9 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
     const uint32_t stage_bytes = kABytes + (uint32_t)G * kGColsI * 128u;
     const uint32_t n_stages = min((uint32_t)kMaxStages, (uint32_t)kRingBytes / stage_bytes);
     stage = 0;
+    // a wavefront of at most 64 (32) nodes fetches only that many operand rows per K block; the
+    // MMA still spans 128 rows, the rest of the stage holds stale data for rows that are not stored
+    const int a_rows = leaf || end - begin > 64 ? BM : (end - begin > 32 ? 64 : 32);
     if (warp == 4 || warp == 10) asm volatile("fence.proxy.async;" ::: "memory");   // TMA reads after the barrier's acquire
 
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
@@ -312,28 +316,47 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
         // Warp 4, A: 128 consecutive rows of the dense operand matrix (rows past its end read as
         // zero, rows past the wavefront belong to later wavefronts and only feed accumulator rows
         // that are never stored).  Warp 10, W: one box per unit group of the packed weights.
+        const bool is_a = warp == 4;
+        const CUtensorMap* map = is_a ? (leaf ? &tmap_x : (a_rows == BM ? &tmap_a : (a_rows == 64 ? &tmap_a64 : &tmap_a32)))
+                                      : (leaf ? &tmap_wx : &tmap_wh);
+        const uint32_t bytes = is_a ? (uint32_t)a_rows * 128u : (uint32_t)ncols * 128u;
+        auto issue = [&](int kb, uint32_t st_idx) {
+          const uint32_t sa = tiles_addr + st_idx * stage_bytes;
+          mbar_arrive_expect_tx(full_bar(st_idx), bytes);
+          if (is_a) {
+            tma_load_2d(sa, map, kb * kKBlock, row0, full_bar(st_idx));
+          } else {
+            for (int g = 0; g < G; ++g)
+              tma_load_2d(sa + kABytes + (uint32_t)(g * gcols) * 128u, map, kb * kKBlock,
+                          (nt * G + g) * gcols, full_bar(st_idx));
+          }
+        };
+        int kb_first = 0;
+        if (t == (int)blockIdx.x) {
+          // First tile of a wavefront: the ring was drained before the barrier, so the first
+          // n_stages K blocks need no wait; one lane per K block issues them in a single step.
+          const int burst = min(kblocks, (int)n_stages);
+          if (lane < burst) issue(lane, (uint32_t)lane);
+          __syncwarp();
+          phase_bits ^= (1u << burst) - 1u;
+          stage = (uint32_t)burst == n_stages ? 0u : (uint32_t)burst;
+          kb_first = burst;
+        }
         if (lane == 0) {
-          const bool is_a = warp == 4;
-          const CUtensorMap* map = is_a ? (leaf ? &tmap_x : &tmap_a) : (leaf ? &tmap_wx : &tmap_wh);
-          const uint32_t bytes = is_a ? (uint32_t)kABytes : (uint32_t)ncols * 128u;
-          for (int kb = 0; kb < kblocks; ++kb) {
+          for (int kb = kb_first; kb < kblocks; ++kb) {
             if (!mbar_wait(empty_bar(stage), ((phase_bits >> stage) & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) {
               alive = false;
               break;
             }
-            const uint32_t sa = tiles_addr + stage * stage_bytes;
-            mbar_arrive_expect_tx(full_bar(stage), bytes);
-            if (is_a) {
-              tma_load_2d(sa, map, kb * kKBlock, row0, full_bar(stage));
-            } else {
-              for (int g = 0; g < G; ++g)
-                tma_load_2d(sa + kABytes + (uint32_t)(g * gcols) * 128u, map, kb * kKBlock,
-                            (nt * G + g) * gcols, full_bar(stage));
-            }
+            issue(kb, stage);
             phase_bits ^= 1u << stage;
             if (++stage == n_stages) stage = 0;
           }
         }
+        __syncwarp();
+        stage = __shfl_sync(kFull, stage, 0);
+        phase_bits = __shfl_sync(kFull, phase_bits, 0);
+        alive = __shfl_sync(kFull, (int)alive, 0) != 0;
       } else if (warp == 5) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
@@ -488,7 +511,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
             }
           }
           // the operand rows written above are read through TMA (async proxy) by later wavefronts
-          asm volatile("fence.proxy.async;" ::: "memory");
+          asm volatile("fence.proxy.async.global;" ::: "memory");
           tc_fence_before();
           mbar_arrive(tempty_bar(acc));              // accumulator stage may be overwritten
         }
@@ -625,6 +648,10 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     if (rc != TREELSTM_OK) return rc;
     rc = make_tmap(ctx, &ctx->tmap_a, p.ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, BM);
     if (rc != TREELSTM_OK) return rc;
+    rc = make_tmap(ctx, &ctx->tmap_a64, p.ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, 64);
+    if (rc != TREELSTM_OK) return rc;
+    rc = make_tmap(ctx, &ctx->tmap_a32, p.ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, 32);
+    if (rc != TREELSTM_OK) return rc;
     ctx->tmap_ws_base = ws;
     ctx->tmap_ws_rows = n;
   }
@@ -641,7 +668,7 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     if (grid > want) grid = want;
     if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
     int only = -1;
-    void* args[] = {&ctx->tmap_wh, &ctx->tmap_wx, &ctx->tmap_x, &ctx->tmap_a, &p, &only};
+    void* args[] = {&ctx->tmap_wh, &ctx->tmap_wx, &ctx->tmap_x, &ctx->tmap_a, &ctx->tmap_a64, &ctx->tmap_a32, &p, &only};
     TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc, dim3(grid), dim3(kThreads), args,
                                              kSmemBytes, stream));
     ctx->launches += 1;
@@ -657,7 +684,8 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     const int w = level_offset_host[lvl + 1] - level_offset_host[lvl];
     if (w <= 0) continue;
     const int tiles = ((w + BM - 1) / BM) * (groups / choose_groups_per_tile(w, groups, p.sched_ctas));
-    k_fwd_tc<<<tiles, kThreads, kSmemBytes, stream>>>(ctx->tmap_wh, ctx->tmap_wx, ctx->tmap_x, ctx->tmap_a, p, lvl);
+    k_fwd_tc<<<tiles, kThreads, kSmemBytes, stream>>>(ctx->tmap_wh, ctx->tmap_wx, ctx->tmap_x, ctx->tmap_a, ctx->tmap_a64,
+                                                      ctx->tmap_a32, p, lvl);
     ctx->launches += 1;
   }
   TL_CUDA(ctx, cudaGetLastError());
