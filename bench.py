@@ -28,6 +28,9 @@ from paper_1809_00832_b200 import forests as fg  # noqa: E402
 METRIC = "treelstm_forward_trees_per_sec"
 UNIT = "trees/s"
 L2_FLUSH_BYTES = 256 << 20          # larger than the 126 MB L2
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_fwd_tc launch from the committed ncu capture
+# (profiles/k_fwd_tc_batch256_bf16.md); None for workloads without a capture of the current kernel.
+NCU_TRAFFIC_BYTES = {"batch256_bf16": 12436480}
 
 
 def measured_peaks():
@@ -346,7 +349,7 @@ def main() -> int:
                 "returns": "root ids and root (h, c) of every tree"},
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                     "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload), "peak_source": peaks["source"],
                      "kernel": "k_fwd_tc (persistent wavefront kernel)" if w.precision == "bf16" else "k_fwd_fp32_persistent",
                      "kernel_ms": k_ms, "algorithmic_bytes": abytes, "algorithmic_flops": flops,
                      "tensor_tflops": achieved_tflops,
