@@ -23,7 +23,10 @@
 // Warp roles (352 threads): warps 0-3 and 6-9 epilogue (tensor-memory lane quadrant = warp id
 // mod 4; the two sets split every unit group in halves), warp 4 TMA producer of the A tiles,
 // warp 10 TMA producer of the W tiles (issuing a TMA load costs its thread about a hundred
-// cycles, so the two streams are issued side by side), warp 5 MMA issuer + tensor-memory owner.
+// cycles, so the two streams are issued side by side), warp 5 MMA issuer + tensor-memory owner,
+// warp 11 second MMA issuer: issuing one tcgen05.mma costs its thread about 83 cycles whatever N
+// is, so on thin tiles (N <= 128) the two issuers take alternate K blocks into two partial
+// accumulators that the epilogue adds.
 #include "common.cuh"
 
 namespace tl {
@@ -31,9 +34,10 @@ namespace {
 
 constexpr int BM = 128;                 // nodes per tile (UMMA M)
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 352;
+constexpr int kThreads = 384;
 constexpr int kABytes = BM * 128;       // one K block (64 bf16) of 128 rows
 constexpr int kAccCols = 256;           // accumulator stage stride in tensor-memory columns
+constexpr int kAcc2Off = 128;           // second partial accumulator inside a stage (thin tiles only)
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kMaxG = 4;                // unit groups (of 8 hidden units) per tile: 1, 2 or 4
 constexpr int kGColsI = 40;             // packed rows per unit group, internal nodes (5 gates)
@@ -257,11 +261,11 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
 
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 2); mbar_init(tempty_bar(a), 256); }
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);
+  if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // columns: 2 stages x 256; thin tiles use [0,128) and [128,256)
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -300,6 +304,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
     const int gcols = leaf ? kGColsL : kGColsI;
     const int ncols = G * gcols;                     // accumulator columns in use
     const int ncols_mma = (ncols + 15) & ~15;        // UMMA N (columns past ncols are never read)
+    const bool dual = ncols_mma <= kAcc2Off && kblocks >= 2;   // two issuers, two partial accumulators
     const uint32_t stage_bytes = kABytes + (uint32_t)G * kGColsI * 128u;
     const uint32_t n_stages = min((uint32_t)kMaxStages, (uint32_t)kRingBytes / stage_bytes);
     stage = 0;
@@ -357,30 +362,48 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
         stage = __shfl_sync(kFull, stage, 0);
         phase_bits = __shfl_sync(kFull, phase_bits, 0);
         alive = __shfl_sync(kFull, (int)alive, 0) != 0;
-      } else if (warp == 5) {
-        // ---------------- MMA issuer ----------------
+      } else if (warp == 5 || warp == 11) {
+        // ---------------- MMA issuers ----------------
+        // Issuer w takes the K blocks with kb % 2 == w when the tile is thin (dual), else issuer 0
+        // takes them all.  Both walk the whole ring so that their stage/phase counters agree.
         if (lane == 0) {
+          const int w = warp == 5 ? 0 : 1;
           const uint32_t acc = acc_iter & 1, acc_phase = (acc_iter >> 1) & 1;
-          if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
-          tc_fence_after();
-          const uint32_t d_tmem = tmem_base + acc * kAccCols;
-          const uint32_t idesc = umma_idesc(ncols_mma);
-          for (int kb = 0; kb < kblocks && alive; ++kb) {
-            if (!mbar_wait(full_bar(stage), (phase_bits >> stage) & 1u, s_abort, p.wait_limit, p.st)) {
-              alive = false;
-              break;
+          if (!dual && w == 1) {
+            // nothing to add for this tile; wait for the accumulator stage like issuer 0 does, so that
+            // this arrival cannot run ahead into the stage's next use
+            if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
+            mbar_arrive(tfull_bar(acc));
+            for (int kb = 0; kb < kblocks; ++kb) {
+              phase_bits ^= 1u << stage;
+              if (++stage == n_stages) stage = 0;
             }
+          } else {
+            if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
             tc_fence_after();
-            const uint32_t a_addr = tiles_addr + stage * stage_bytes;
-            const uint64_t a_desc = umma_desc(a_addr), b_desc = umma_desc(a_addr + kABytes);
+            const uint32_t d_tmem = tmem_base + acc * kAccCols + (w == 1 ? (uint32_t)kAcc2Off : 0u);
+            const uint32_t idesc = umma_idesc(ncols_mma);
+            bool first = true;
+            for (int kb = 0; kb < kblocks && alive; ++kb) {
+              if (!dual || (kb & 1) == w) {
+                if (!mbar_wait(full_bar(stage), (phase_bits >> stage) & 1u, s_abort, p.wait_limit, p.st)) {
+                  alive = false;
+                  break;
+                }
+                tc_fence_after();
+                const uint32_t a_addr = tiles_addr + stage * stage_bytes;
+                const uint64_t a_desc = umma_desc(a_addr), b_desc = umma_desc(a_addr + kABytes);
 #pragma unroll
-            for (int k = 0; k < kKBlock / 16; ++k)   // UMMA K = 16 bf16 = 32 bytes = 2 descriptor units
-              umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
-            umma_commit(empty_bar(stage));           // frees the smem stage when these MMAs retire
-            phase_bits ^= 1u << stage;
-            if (++stage == n_stages) stage = 0;
+                for (int k = 0; k < kKBlock / 16; ++k)   // UMMA K = 16 bf16 = 32 bytes = 2 descriptor units
+                  umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, !(first && k == 0));
+                first = false;
+                umma_commit(empty_bar(stage));           // frees the smem stage when these MMAs retire
+              }
+              phase_bits ^= 1u << stage;
+              if (++stage == n_stages) stage = 0;
+            }
+            if (alive) umma_commit(tfull_bar(acc));      // this issuer's partial accumulator is complete
           }
-          if (alive) umma_commit(tfull_bar(acc));    // accumulator complete
         }
         ++acc_iter;
       } else {
@@ -421,7 +444,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
           tc_fence_after();
           const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(quad * 32) << 16) + 4u * e;
           // the tensor-memory loads of group g + 1 are in flight while group g is computed
-          uint32_t vbuf[2][20];
+          uint32_t vbuf[2][20], v2[20];
           auto load_group = [&](int g, uint32_t* v) {
             const uint32_t col0 = (uint32_t)(g * gcols);
             if (leaf) {
@@ -432,6 +455,16 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
               for (int q = 0; q < 5; ++q) tmem_ld4(taddr + col0 + 8 * q, v + 4 * q);
             }
           };
+          auto add_second = [&](int g, uint32_t* v) {   // thin tiles: add the second issuer's partial sums
+            const uint32_t col0 = (uint32_t)kAcc2Off + (uint32_t)(g * gcols);
+#pragma unroll
+            for (int q = 0; q < 5; ++q)
+              if (q < ngates) tmem_ld4(taddr + col0 + 8 * q, v2 + 4 * q);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 20; ++j)
+              if (j < 4 * ngates) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
+          };
           load_group(0, vbuf[0]);
 #pragma unroll
           for (int g = 0; g < kMaxG; ++g) {
@@ -441,6 +474,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
 #pragma unroll
             for (int q = 0; q < 5; ++q) bcur[q] = bnext[q];
             tmem_ld_wait();
+            if (dual) add_second(g, v);
             if (g + 1 < G) {
               load_group(g + 1, vbuf[(g + 1) & 1]);
 #pragma unroll
