@@ -45,7 +45,7 @@ constexpr int kGColsL = 24;             // packed rows per unit group, leaves (g
 constexpr int kBBytes = kMaxG * kGColsI * 128;
 constexpr int kRingBytes = kMaxStages * (kABytes + kGColsI * 128);   // 8 stages of the thinnest tile
 constexpr int kCBytes = BM * 2 * kMaxG * 8 * 4;   // staged child cell states: 128 rows x 2 x 32 fp32
-constexpr int kSmemBytes = kRingBytes + kCBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kSmemBytes = kRingBytes + kCBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*row ids*/;
 static_assert(kBBytes % 1024 == 0 && (kGColsI * 128) % 1024 == 0 && (kGColsL * 128) % 1024 == 0,
               "every TMA box lands on a 1024-byte boundary of the swizzle pattern");
 
@@ -246,9 +246,15 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   const unsigned char* cstage_ptr = tiles_ptr + kRingBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + kRingBytes + kCBytes);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 4);
+  // bars[2S+4]: meeting point of the 256 epilogue threads (output staging)
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 5);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   int* s_flag = const_cast<int*>(s_abort) + 1;
+  int* s_rownode = reinterpret_cast<int*>(tiles_ptr + kRingBytes + kCBytes + 256);   // [128] node id of each tile row
+  int* s_rowslot = s_rownode + BM;                                                   // [128] its delivery slot
+  unsigned char* cstage_w = tiles_ptr + kRingBytes;
+  const uint32_t epi_bar = smem_u32(bars + 2 * kMaxStages + 4);
+  uint32_t epi_phase = 0;
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
@@ -262,6 +268,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 2); mbar_init(tempty_bar(a), 256); }
+    mbar_init(epi_bar, 256);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -420,6 +427,10 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
         // stage the children's cell states of this thread's row while the MMAs run
         const float* crow = p.cin + (size_t)row * 2 * H;   // [c_l | c_r] of the node at this position
         const bool staged = !leaf && vec && (nt + 1) * G * 8 <= H;
+        // Outputs go through the same per-row staging area: each thread parks its 4-unit pieces of
+        // c and h there, then all epilogue threads copy whole row segments out, several lanes per
+        // row, so that a warp store covers a few full lines instead of 32 scattered 16-byte pieces.
+        const bool staged_out = vec && (nt + 1) * G * 8 <= H && p.gates == nullptr;
         const uint32_t my_c = cstage_addr + (uint32_t)r * 256u;
         if (staged) {
           const float* sl = crow + nt * G * 8;
@@ -517,37 +528,75 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
                 }
                 hv[j] = go[j] * act_tanh(cv[j]);
               }
-              if (slot >= 0) {
-                // hand the state to the caller: bf16 h into its operand row (padded units as 0),
-                // fp32 c next to it
-                uint32_t packed[2];
+              if (staged_out) {
+                unsigned char* mine = cstage_w + r * 256;
+                *reinterpret_cast<float4*>(mine + (((2 * g + e) ^ (r & 7)) << 4)) = make_float4(cv[0], cv[1], cv[2], cv[3]);
+                *reinterpret_cast<float4*>(mine + (((8 + 2 * g + e) ^ (r & 7)) << 4)) = make_float4(hv[0], hv[1], hv[2], hv[3]);
+              } else {
+                if (slot >= 0) {
+                  // hand the state to the caller: bf16 h into its operand row (padded units as 0),
+                  // fp32 c next to it
+                  uint32_t packed[2];
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                  const float lo = 2 * j < count ? hv[2 * j] : 0.f, hi = 2 * j + 1 < count ? hv[2 * j + 1] : 0.f;
-                  __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
-                  packed[j] = *reinterpret_cast<uint32_t*>(&b2);
+                  for (int j = 0; j < 2; ++j) {
+                    const float lo = 2 * j < count ? hv[2 * j] : 0.f, hi = 2 * j + 1 < count ? hv[2 * j + 1] : 0.f;
+                    __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+                    packed[j] = *reinterpret_cast<uint32_t*>(&b2);
+                  }
+                  *reinterpret_cast<uint2*>(p.ain + (size_t)slot * Hp + u0) = make_uint2(packed[0], packed[1]);
+                  if (count > 0) st_row4(p.cin + (size_t)slot * H + u0, vec, count, cv);
                 }
-                *reinterpret_cast<uint2*>(p.ain + (size_t)slot * Hp + u0) = make_uint2(packed[0], packed[1]);
-                if (count > 0) st_row4(p.cin + (size_t)slot * H + u0, vec, count, cv);
-              }
-              if (count > 0) {
-                st_row4(p.h + (size_t)node * H + u0, vec, count, hv);
-                st_row4(p.c + (size_t)node * H + u0, vec, count, cv);
-                if (p.gates) {
-                  float* gp = p.gates + (size_t)node * 5 * H + u0;
-                  st_row4(gp, vec, count, gi);
-                  st_row4(gp + H, vec, count, gfl);
-                  st_row4(gp + 2 * H, vec, count, gfr);
-                  st_row4(gp + 3 * H, vec, count, go);
-                  st_row4(gp + 4 * H, vec, count, gu);
+                if (count > 0) {
+                  st_row4(p.h + (size_t)node * H + u0, vec, count, hv);
+                  st_row4(p.c + (size_t)node * H + u0, vec, count, cv);
+                  if (p.gates) {
+                    float* gp = p.gates + (size_t)node * 5 * H + u0;
+                    st_row4(gp, vec, count, gi);
+                    st_row4(gp + H, vec, count, gfl);
+                    st_row4(gp + 2 * H, vec, count, gfr);
+                    st_row4(gp + 3 * H, vec, count, go);
+                    st_row4(gp + 4 * H, vec, count, gu);
+                  }
                 }
               }
             }
           }
-          // the operand rows written above are read through TMA (async proxy) by later wavefronts
-          asm volatile("fence.proxy.async.global;" ::: "memory");
           tc_fence_before();
           mbar_arrive(tempty_bar(acc));              // accumulator stage may be overwritten
+          if (staged_out) {
+            if (e == 0) { s_rownode[r] = valid ? node : -1; s_rowslot[r] = slot; }
+            mbar_arrive(epi_bar);
+            bool ok = mbar_wait(epi_bar, epi_phase, s_abort, p.wait_limit, p.st);
+            epi_phase ^= 1;
+            if (ok) {
+              const int et = e * BM + r, cpr = 2 * G;           // 16-byte chunks (4 units) per row
+              for (int idx = et; idx < BM * cpr; idx += 2 * BM) {
+                const int ro = idx / cpr, ch = idx % cpr;
+                const int node_o = s_rownode[ro];
+                if (node_o < 0) continue;
+                const unsigned char* src = cstage_w + ro * 256;
+                const float4 c4 = *reinterpret_cast<const float4*>(src + ((ch ^ (ro & 7)) << 4));
+                const float4 h4 = *reinterpret_cast<const float4*>(src + (((8 + ch) ^ (ro & 7)) << 4));
+                const int uo = nt * G * 8 + 4 * ch;
+                *reinterpret_cast<float4*>(p.h + (size_t)node_o * H + uo) = h4;
+                *reinterpret_cast<float4*>(p.c + (size_t)node_o * H + uo) = c4;
+                const int slot_o = s_rowslot[ro];
+                if (slot_o >= 0) {
+                  *reinterpret_cast<float4*>(p.cin + (size_t)slot_o * H + uo) = c4;
+                  __nv_bfloat162 lo = __floats2bfloat162_rn(h4.x, h4.y), hi = __floats2bfloat162_rn(h4.z, h4.w);
+                  *reinterpret_cast<uint2*>(p.ain + (size_t)slot_o * Hp + uo) =
+                      make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+                }
+              }
+            }
+            // the staging rows are reused by the next tile's loads of the children's cell states
+            mbar_arrive(epi_bar);
+            ok = mbar_wait(epi_bar, epi_phase, s_abort, p.wait_limit, p.st) && ok;
+            epi_phase ^= 1;
+            if (!ok) alive = false;
+          }
+          // the operand rows written above are read through TMA (async proxy) by later wavefronts
+          asm volatile("fence.proxy.async.global;" ::: "memory");
         }
         ++acc_iter;
       }
