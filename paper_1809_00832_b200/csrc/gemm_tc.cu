@@ -311,7 +311,9 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
     const int gcols = leaf ? kGColsL : kGColsI;
     const int ncols = G * gcols;                     // accumulator columns in use
     const int ncols_mma = (ncols + 15) & ~15;        // UMMA N (columns past ncols are never read)
-    const bool dual = ncols_mma <= kAcc2Off && kblocks >= 2;   // two issuers, two partial accumulators
+    // two issuers and two partial accumulators where the MMA issue chain is the critical path: thin
+    // tiles of a wavefront that takes a single round (the epilogue pays for adding the partial sums)
+    const bool dual = ncols_mma <= kAcc2Off && kblocks >= 2 && tiles <= (int)gridDim.x;
     const uint32_t stage_bytes = kABytes + (uint32_t)G * kGColsI * 128u;
     const uint32_t n_stages = min((uint32_t)kMaxStages, (uint32_t)kRingBytes / stage_bytes);
     stage = 0;
