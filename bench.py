@@ -315,14 +315,9 @@ def main() -> int:
     d2h = f.n_trees * (2 * 4 * p.H + 4) + 8
 
     # ---- max over ranks, aggregate ----
-    agg_trees, agg_nodes = f.n_trees, f.n_nodes
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
-        cnt = torch.tensor([f.n_trees, f.n_nodes], device="cuda", dtype=torch.int64)
-        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
-        agg_trees, agg_nodes = int(cnt[0]), int(cnt[1])
+    from paper_1809_00832_b200 import sharding
+    (total_ms, e2e_ms), (agg_trees, agg_nodes) = sharding.combine([total_ms, e2e_ms], [f.n_trees, f.n_nodes],
+                                                                  device="cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()

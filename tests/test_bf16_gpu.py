@@ -93,3 +93,37 @@ def test_bf16_forward_then_fp32_backward():
     assert abs(float(g["loss"].item()) - ref["loss"]) < util.TOL["bf16"]
     assert util.max_abs(g["dW"].cpu().numpy(), ref["dW"]) < util.TOL["bf16"]
     assert util.max_abs(g["db"].cpu().numpy(), ref["db"]) < util.TOL["bf16"]
+
+
+def test_bf16_large_forest_multi_cta_schedule():
+    """more nodes than the single-CTA scheduler takes: the multi-CTA scheduler feeds the tensor-core
+    kernel; schedule exact on all nodes, states checked on sampled whole trees"""
+    rng = np.random.default_rng(31)
+    params = fg.draw_params(rng, 64, 48, 400, emb_dist="normal", emb_scale=0.3, w_scale=0.15)
+    forest = fg.random_forest(rng, 1500, 2, 56, 400)
+    assert forest.n_nodes > 32768
+    model = util.make_model(params, "bf16")
+    res = util.gpu_forward(model, forest, binding.PERSISTENT)
+    status, _, level, order, off = orc.schedule(forest.left, forest.right)
+    util.check_schedule(res, dict(level=level, order=order, level_offset=off), forest.n_nodes)
+    sample = [3, 700, 1499]
+    sub = fg.select_trees(forest, sample)
+    h, c, _ = orc.forward_recursive(sub.left, sub.right, sub.token, params.emb, params.W, params.b)
+    ids = np.nonzero(np.isin(forest.tree_of, sample))[0]
+    assert util.max_abs(res["h"][ids], h) < util.TOL["bf16"]
+    assert util.max_abs(res["c"][ids], c) < util.TOL["bf16"]
+    assert np.all(np.isfinite(res["h"]))
+
+
+def test_bf16_repeated_calls_and_changing_sizes():
+    """the same context evaluates forests of different sizes back to back (operand maps are rebuilt,
+    stale operand rows of an earlier, larger forest must not leak into a later one)"""
+    rng = np.random.default_rng(32)
+    params = fg.draw_params(rng, 64, 64, 300, emb_dist="normal", emb_scale=0.3, w_scale=0.2)
+    model = util.make_model(params, "bf16")
+    for n_trees in (40, 3, 17, 40):
+        forest = fg.random_forest(rng, n_trees, 1, 30, 300)
+        res = util.gpu_forward(model, forest, binding.PERSISTENT)
+        h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
+        assert util.max_abs(res["h"], h) < util.TOL["bf16"]
+        assert util.max_abs(res["c"], c) < util.TOL["bf16"]
