@@ -5,9 +5,8 @@
 // Paper: Figure 2 (Section 3.1) - a node is LSTM(embed(word)) or LSTM(left_state, right_state);
 // Section 2.2 - sibling subtrees are independent, so every node whose children are done can be
 // evaluated at once.  Batching those nodes into one wide contraction is what Section 6.3 calls
-// folding and charges with regrouping copies per depth; here nothing is regrouped: the operand
-// rows are gathered straight from the node-indexed state array into the swizzled shared-memory
-// tile the tensor core reads.
+// folding and charges with regrouping copies per depth; here nothing is regrouped between depths
+// (see "No gather on the operand side" below).
 //
 // One tile = 128 ready nodes x (8*G hidden units x 5 gates).  W is pre-packed so that the 5 gate
 // pre-activations of a hidden unit sit in the same accumulator row slice and one thread (one
@@ -20,7 +19,7 @@
 // one tiled TMA load per K block feeds the tensor core.  Leaves: the embedding rows are copied
 // once into ready order (Xin) by all CTAs before the first wavefront.
 //
-// Warp roles (352 threads): warps 0-3 and 6-9 epilogue (tensor-memory lane quadrant = warp id
+// Warp roles (384 threads): warps 0-3 and 6-9 epilogue (tensor-memory lane quadrant = warp id
 // mod 4; the two sets split every unit group in halves), warp 4 TMA producer of the A tiles,
 // warp 10 TMA producer of the W tiles (issuing a TMA load costs its thread about a hundred
 // cycles, so the two streams are issued side by side), warp 5 MMA issuer + tensor-memory owner,
