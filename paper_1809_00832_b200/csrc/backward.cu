@@ -203,11 +203,17 @@ k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
       Bs[buf][e / BK][e % BK] = rb[q];
     }
   };
-  fetch(0);
-  stash(0);
+  // gridDim.y CTAs share the contraction: each takes a contiguous run of chunks and adds its
+  // partial sums with atomics (few levels fill the GPU on their own, the chain of dependent
+  // memory round trips per CTA is what costs time)
+  const int chunks_all = (J + BK - 1) / BK;
+  const int per_split = (chunks_all + gridDim.y - 1) / gridDim.y;
+  const int c_lo = blockIdx.y * per_split, chunks = min(chunks_all, c_lo + per_split);
+  if (c_lo >= chunks) return;
+  fetch(c_lo * BK);
+  stash(c_lo & 1);
   __syncthreads();
-  const int chunks = (J + BK - 1) / BK;
-  for (int cidx = 0; cidx < chunks; ++cidx) {
+  for (int cidx = c_lo; cidx < chunks; ++cidx) {
     const int buf = cidx & 1;
     if (cidx + 1 < chunks) fetch((cidx + 1) * BK);
 #pragma unroll
@@ -235,7 +241,7 @@ k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
         atomicAdd(&p.dEmb_rows[(size_t)p.tok_slot[p.token[node]] * E + k], acc[i][q]);
       } else {
         const int child = k < H ? p.left[node] : p.right[node];
-        p.dh[(size_t)child * H + (k < H ? k : k - H)] += acc[i][q];  // single caller: no race
+        atomicAdd(&p.dh[(size_t)child * H + (k < H ? k : k - H)], acc[i][q]);
       }
     }
   }
@@ -384,7 +390,9 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
     k_bwd_gates<<<(unsigned)((elems + 255) / 256), 256, 0, stream>>>(p, begin, end, leaf);
     const int K = leaf ? E : 2 * H;
     const int tiles = ((end - begin + BT - 1) / BT) * ((K + BT - 1) / BT);
-    k_bwd_dinput<<<tiles, 256, 0, stream>>>(p, begin, end, leaf);
+    const int chunks_all = (int)((J + BK - 1) / BK);
+    const int splits = tiles >= 148 ? 1 : (chunks_all < 6 ? chunks_all : 6);
+    k_bwd_dinput<<<dim3(tiles, splits), 256, 0, stream>>>(p, begin, end, leaf);
     ctx->launches += 2;
   }
   const int tiles_j = (int)((J + BT - 1) / BT);
