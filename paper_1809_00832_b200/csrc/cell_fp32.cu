@@ -11,16 +11,15 @@
 namespace tl {
 namespace {
 
-constexpr int TM = 64;       // rows (nodes) per tile
+constexpr int TM = 64;       // rows (nodes) per tile on wide wavefronts
+constexpr int TMS = 16;      // rows per tile where TM-row tiles would leave most SMs idle
 constexpr int TU = 16;       // hidden units per tile (x 5 gates = 80 columns)
 constexpr int KC = 32;       // contraction chunk
 constexpr int kThreads = 256;
-constexpr int RPT = TM / (kThreads / TU);  // rows per thread = 4
-constexpr int kALoads = TM * KC / kThreads;        // 8 operand elements per thread and chunk
 constexpr int kWLoads = KC * 5 * TU / kThreads;    // 10 weight elements per thread and chunk
 
 struct FwdParams {
-  int n, H, E;
+  int n, H, E, n_sms;
   const int *left, *right, *token, *order, *level_offset;
   const float *emb, *W, *b;
   float *h, *c, *gates;
@@ -36,12 +35,20 @@ struct TileSmem {
   int node[TM], l[TM], r[TM];
 };
 
+// Rows per tile of a wavefront of `rows` nodes: a level-uniform choice.
+__host__ __device__ inline int rows_per_tile(int rows, int tiles_u, int n_sms) {
+  return ((rows + TM - 1) / TM) * tiles_u >= n_sms ? TM : TMS;
+}
+
 // One tile: rows [row0, row0 + TM) of the ready order (clipped to row_end), hidden units
 // [u0, u0 + TU).  `leaf` selects x = emb[token] with W rows [0, E) and gates i, o, u only.
 // The next K chunk is fetched into registers while the current one is multiplied out of shared
 // memory (two buffers, one CTA barrier per chunk).
+template <int TM>
 __device__ void fp32_tile(const FwdParams& p, int row0, int row_end, int u0, bool leaf,
                           TileSmem& s) {
+  constexpr int RPT = TM / (kThreads / TU);          // rows per thread: 4 or 1
+  constexpr int kALoads = TM * KC / kThreads;        // operand elements per thread and chunk: 8 or 2
   const int tid = threadIdx.x, tx = tid % TU, ty = tid / TU;
   const int H = p.H, E = p.E, K = leaf ? E : 2 * H;
   const float* Wk = p.W + (size_t)(leaf ? 0 : E) * 5 * H;
@@ -152,7 +159,9 @@ k_fwd_fp32_level(FwdParams p, int row_begin, int row_end, int leaf) {
   __shared__ TileSmem s;
   const int tiles_u = (p.H + TU - 1) / TU;
   const int tm = blockIdx.x / tiles_u, tu = blockIdx.x % tiles_u;
-  fp32_tile(p, row_begin + tm * TM, row_end, tu * TU, leaf != 0, s);
+  const int tmr = rows_per_tile(row_end - row_begin, tiles_u, p.n_sms);
+  if (tmr == TM) fp32_tile<TM>(p, row_begin + tm * TM, row_end, tu * TU, leaf != 0, s);
+  else fp32_tile<TMS>(p, row_begin + tm * TMS, row_end, tu * TU, leaf != 0, s);
 }
 
 // All wavefronts in one cooperative launch; a bounded grid barrier separates the levels.
@@ -165,9 +174,12 @@ k_fwd_fp32_persistent(FwdParams p) {
   const int tiles_u = (p.H + TU - 1) / TU;
   for (int lvl = 0; lvl < n_levels; ++lvl) {
     const int begin = p.level_offset[lvl], end = p.level_offset[lvl + 1];
-    const int tiles = ((end - begin + TM - 1) / TM) * tiles_u;
-    for (int t = blockIdx.x; t < tiles; t += gridDim.x)
-      fp32_tile(p, begin + (t / tiles_u) * TM, end, (t % tiles_u) * TU, lvl == 0, s);
+    const int tmr = rows_per_tile(end - begin, tiles_u, p.n_sms);
+    const int tiles = ((end - begin + tmr - 1) / tmr) * tiles_u;
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
+      if (tmr == TM) fp32_tile<TM>(p, begin + (t / tiles_u) * TM, end, (t % tiles_u) * TU, lvl == 0, s);
+      else fp32_tile<TMS>(p, begin + (t / tiles_u) * TMS, end, (t % tiles_u) * TU, lvl == 0, s);
+    }
     if (lvl + 1 < n_levels &&
         !grid_barrier(p.st, (unsigned)(lvl + 1) * gridDim.x, p.wait_limit, &s_flag))
       return;
@@ -183,7 +195,7 @@ int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t
                         cudaStream_t stream) {
   char* base = static_cast<char*>(ws);
   FwdParams p;
-  p.n = n; p.H = ctx->H; p.E = ctx->E;
+  p.n = n; p.H = ctx->H; p.E = ctx->E; p.n_sms = ctx->sm_count;
   p.left = left; p.right = right; p.token = token; p.order = order;
   p.level_offset = level_offset_dev;
   p.emb = ctx->emb; p.W = ctx->W; p.b = ctx->b;
@@ -197,7 +209,7 @@ int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t
     TL_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_fwd_fp32_persistent,
                                                                kThreads, 0));
     int grid = per_sm * ctx->sm_count;
-    const int want = ((n + TM - 1) / TM + 1) * tiles_u;   // never more CTAs than the widest level
+    const int want = ((n + TMS - 1) / TMS + 1) * tiles_u;   // never more CTAs than the widest level has tiles
     if (grid > want) grid = want;
     if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
     if (grid < 1) grid = 1;
@@ -209,7 +221,8 @@ int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t
   }
   for (int lvl = 0; lvl < n_levels_host; ++lvl) {
     const int begin = level_offset_host[lvl], end = level_offset_host[lvl + 1];
-    const int tiles = ((end - begin + TM - 1) / TM) * tiles_u;
+    const int tmr = rows_per_tile(end - begin, tiles_u, p.n_sms);
+    const int tiles = ((end - begin + tmr - 1) / tmr) * tiles_u;
     if (tiles <= 0) continue;
     k_fwd_fp32_level<<<tiles, kThreads, 0, stream>>>(p, begin, end, lvl == 0 ? 1 : 0);
     ctx->launches += 1;
