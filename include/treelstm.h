@@ -241,6 +241,20 @@ TREELSTM_API int treelstm_schedule_static(int n_nodes, const int32_t* left, cons
  */
 TREELSTM_API int treelstm_last_kernel_ms(treelstm_t* ctx, float* ms);
 
+/*
+ * treelstm_selftest_waits - exercises the bounded device-side waits without any fault: one CTA
+ * waits on a shared-memory barrier nobody arrives at, then on a grid barrier that expects a CTA
+ * that does not exist.  Both must give up after the limit set with TREELSTM_OPT_WAIT_LIMIT_CYCLES
+ * (set a small one first) and record TREELSTM_ERR_TIMEOUT; the context stays usable.  (Robustness
+ * aid; the paper has no counterpart.)
+ *   workspace  device scratch, >= 256 bytes, 256-byte aligned (its first 256 bytes are overwritten).
+ *   result     [4] out (device): {first wait succeeded (must be 0), status after it (must be
+ *              TREELSTM_ERR_TIMEOUT), second wait succeeded (0), status after it (TIMEOUT)}.
+ * Asynchronous on `stream`.
+ */
+TREELSTM_API int treelstm_selftest_waits(treelstm_t* ctx, void* workspace, size_t workspace_bytes,
+                                         int32_t* result, void* stream);
+
 /* Number of kernels the last forward / backward call on this context launched. */
 TREELSTM_API int treelstm_last_launch_count(const treelstm_t* ctx);
 

@@ -52,6 +52,7 @@ SIGNATURES = {
     "treelstm_forward_host": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp,
                                    _vp, _vp, _i, _vp]),
     "treelstm_schedule_static": (_i, [_i, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "treelstm_selftest_waits": (_i, [_vp, _vp, ctypes.c_size_t, _vp, _vp]),
     "treelstm_last_kernel_ms": (_i, [_vp, ctypes.POINTER(ctypes.c_float)]),
     "treelstm_last_launch_count": (_i, [_vp]),
     "treelstm_last_cuda_error": (_i, [_vp]),
@@ -280,6 +281,18 @@ class TreeLSTM:
         if rc != OK:
             raise TreeLSTMError(rc, "treelstm_forward_host")
         return out
+
+    def selftest_waits(self) -> list:
+        """treelstm_selftest_waits; returns the four result words."""
+        ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+        base = ws.data_ptr()
+        aligned = (base + 255) // 256 * 256
+        res = torch.full((4,), 99, dtype=torch.int32, device="cuda")
+        rc = self.lib.treelstm_selftest_waits(self.handle, ctypes.c_void_p(aligned), 256, _ptr(res), _stream())
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_selftest_waits")
+        torch.cuda.synchronize()
+        return res.cpu().tolist()
 
     def last_kernel_ms(self) -> float:
         ms = ctypes.c_float()

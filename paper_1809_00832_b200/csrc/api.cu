@@ -360,6 +360,14 @@ int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, con
   return rc;
 }
 
+int treelstm_selftest_waits(treelstm_t* ctx, void* workspace, size_t workspace_bytes, int32_t* result,
+                            void* stream) {
+  if (!ctx || !workspace || !result || workspace_bytes < sizeof(DevStatus)) return TREELSTM_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return TREELSTM_ERR_INVALID_ARG;
+  ctx->last.valid = false;   // the control block of an earlier forward is overwritten
+  return launch_selftest_waits(ctx, workspace, result, static_cast<cudaStream_t>(stream));
+}
+
 int treelstm_last_launch_count(const treelstm_t* ctx) { return ctx ? ctx->launches : 0; }
 
 int treelstm_last_cuda_error(const treelstm_t* ctx) { return ctx ? ctx->cuda_error : 0; }

@@ -135,6 +135,8 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
                         int n_levels_host, int flags, void* ws, const WsLayout& lay,
                         cudaStream_t stream);
 
+int launch_selftest_waits(treelstm* ctx, void* ws, int* result_dev, cudaStream_t stream);
+
 // backward.cu
 int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW, float* db,
                     float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,

@@ -624,6 +624,35 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   }
 }
 
+// ---- self-test of the bounded waits ---------------------------------------------------------- //
+// One CTA waits on an mbarrier nobody arrives at and on a grid barrier that expects a second CTA
+// that does not exist.  Both waits must end by their cycle limit and record TREELSTM_ERR_TIMEOUT.
+__global__ void k_selftest_waits(DevStatus* st, long long limit, int* result) {
+  __shared__ uint64_t bar;
+  __shared__ int s_abort, s_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  int outcome = 0;
+  if (threadIdx.x == 0) {
+    const bool ok = mbar_wait(smem_u32(&bar), 0, &s_abort, limit, st);
+    outcome = ok ? 1 : 0;                 // 0 = gave up, as it must
+  }
+  const int after_mbar = ld_volatile(&st->status);
+  if (threadIdx.x == 0) st->status = 0;   // second part starts clean
+  __syncthreads();
+  const bool ok2 = grid_barrier(st, 2u * gridDim.x, limit, &s_flag);
+  if (threadIdx.x == 0) {
+    result[0] = outcome;
+    result[1] = after_mbar;
+    result[2] = ok2 ? 1 : 0;
+    result[3] = ld_volatile(&st->status);
+  }
+}
+
 // ---- weight packing ---------------------------------------------------------------------------- //
 // Packed row of hidden unit u, gate g (internal order i, f_l, f_r, o, u): (u/8)*40 + g*8 + u%8;
 // leaf tiles keep gates i, o, u only: (u/8)*24 + gi*8 + u%8.  Each packed row holds the K vector.
@@ -688,6 +717,14 @@ int make_tmap(treelstm* ctx, CUtensorMap* map, const void* base, uint64_t inner,
 
 
 }  // namespace
+
+int launch_selftest_waits(treelstm* ctx, void* ws, int* result_dev, cudaStream_t stream) {
+  DevStatus* st = static_cast<DevStatus*>(ws);
+  TL_CUDA(ctx, cudaMemsetAsync(st, 0, sizeof(DevStatus), stream));
+  k_selftest_waits<<<1, 64, 0, stream>>>(st, ctx->opt.wait_limit_kcycles * 1024, result_dev);
+  TL_CUDA(ctx, cudaGetLastError());
+  return TREELSTM_OK;
+}
 
 int pack_weights_bf16(treelstm* ctx, cudaStream_t stream) {
   k_pack_weights<<<512, 256, 0, stream>>>(ctx->H, ctx->E, ctx->Hp, ctx->Ep, ctx->W, ctx->b, ctx->Wp_h,

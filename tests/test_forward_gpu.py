@@ -184,3 +184,18 @@ def test_host_buffer_forward():
     # roots only, second call reuses the library's staging buffers
     out2 = model.forward_host(*host, max_roots=f.n_trees)
     np.testing.assert_array_equal(out2["root_h"].numpy(), out["root_h"].numpy())
+
+
+def test_bounded_waits_time_out_cleanly():
+    """failure detection without a fault: a wait on a flag that nothing sets ends by its cycle limit,
+    the status word says TIMEOUT, and the context keeps working afterwards"""
+    w = fg.make_workload("tiny8", 0)
+    ref = util.oracle_forward_cached("tiny8", 0)
+    model = util.make_model(w.params, "fp32")
+    model.set_option(binding.OPT_WAIT_LIMIT_CYCLES, 200)          # 200 * 1024 cycles, about 0.1 ms
+    first_ok, status1, second_ok, status2 = model.selftest_waits()
+    assert first_ok == 0 and status1 == binding.ERR_TIMEOUT
+    assert second_ok == 0 and status2 == binding.ERR_TIMEOUT
+    model.set_option(binding.OPT_WAIT_LIMIT_CYCLES, 1 << 20)
+    res = util.gpu_forward(model, w.forest, binding.PERSISTENT)
+    assert util.max_abs(res["h"], ref["h"]) < util.TOL["fp32"]
