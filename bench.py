@@ -171,6 +171,51 @@ def train_step_time(steps: int = 200, warmup: int = 5):
             "note": "backward reads the level table back once per step (one stream synchronisation)"}
 
 
+def run_sweeps(args):
+    """Extra benchmark lines on synthetic trees, after the paper's shape study (Section 6.3, Table 1:
+    balanced / moderate / linear trees at batch 1, 10, 25) and its time-per-instance-vs-length plot
+    (Figure 11, batch 1).  One JSON line per point; not the headline metric."""
+    import torch
+    from paper_1809_00832_b200 import binding, build
+    build.build()
+    rng = np.random.default_rng(0)
+    p = fg.draw_params(rng, 256, 300, 20000, emb_dist="normal", emb_scale=0.1, w_scale=0.05)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    model = binding.TreeLSTM(p.H, p.E, p.vocab, dev(p.emb), dev(p.W), dev(p.b), binding.BF16)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def time_forest(forest, steps=100, warmup=5):
+        left, right, token = dev(forest.left), dev(forest.right), dev(forest.token)
+        out = model.forward(left, right, token)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(-warmup, steps):
+            flush.fill_(i & 0xFF)
+            if i >= 0:
+                ev[i][0].record()
+            model.forward(left, right, token, out=out, check=False)
+            if i >= 0:
+                ev[i][1].record()
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in ev) / steps, int(out["n_levels"].item())
+
+    shapes = {"balanced": lambda: fg.balanced_shape(32), "moderate": lambda: fg.random_split_shape(rng, 32),
+              "linear": lambda: fg.left_chain_shape(32)}
+    if args.sweep in ("shapes", "all"):
+        for name, make in shapes.items():
+            for batch in (1, 10, 25):
+                forest = fg.forest_from_shapes([make() for _ in range(batch)], rng, p.vocab)
+                ms, levels = time_forest(forest)
+                print(json.dumps({"sweep": "shape", "shape": name, "leaves_per_tree": 32, "batch": batch,
+                                  "levels": levels, "ms_per_step": ms, "trees_per_sec": batch / (ms * 1e-3)}))
+    if args.sweep in ("length", "all"):
+        for leaves in (2, 4, 8, 16, 24, 32, 40, 48, 56):
+            forest = fg.forest_from_shapes([fg.random_split_shape(rng, leaves)], rng, p.vocab)
+            ms, levels = time_forest(forest)
+            print(json.dumps({"sweep": "length", "leaves": leaves, "batch": 1, "levels": levels,
+                              "ms_per_instance": ms}))
+    return 0
+
+
 def run_reference(args):
     """The reference arm of this build is the CPU oracle: one step = the oracle on a bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
@@ -230,11 +275,15 @@ def main() -> int:
     ap.add_argument("--mode", default="persistent", choices=["persistent", "per_level"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-train", action="store_true", help="skip the extra training-step figure")
+    ap.add_argument("--sweep", default=None, choices=["shapes", "length", "all"],
+                    help="print the tree-shape / sentence-length sweeps instead of the benchmark line")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
         return run_reference(args)
+    if args.sweep:
+        return run_sweeps(args)
 
     import torch
     from paper_1809_00832_b200 import binding, build
