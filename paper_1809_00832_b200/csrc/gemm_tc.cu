@@ -44,7 +44,9 @@ constexpr int kGColsL = 24;             // packed rows per unit group, leaves (g
 constexpr int kBBytes = kMaxG * kGColsI * 128;
 constexpr int kRingBytes = kMaxStages * (kABytes + kGColsI * 128);   // 8 stages of the thinnest tile
 constexpr int kCBytes = BM * 2 * kMaxG * 8 * 4;   // staged child cell states: 128 rows x 2 x 32 fp32
-constexpr int kSmemBytes = kRingBytes + kCBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*row ids*/;
+constexpr int kLevelCache = 1024;       // wavefront boundaries kept in shared memory
+constexpr int kSmemBytes = kRingBytes + kCBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*row ids*/ +
+                           4 * kLevelCache;
 static_assert(kBBytes % 1024 == 0 && (kGColsI * 128) % 1024 == 0 && (kGColsL * 128) % 1024 == 0,
               "every TMA box lands on a 1024-byte boundary of the swizzle pattern");
 
@@ -251,6 +253,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   int* s_flag = const_cast<int*>(s_abort) + 1;
   int* s_rownode = reinterpret_cast<int*>(tiles_ptr + kRingBytes + kCBytes + 256);   // [128] node id of each tile row
   int* s_rowslot = s_rownode + BM;                                                   // [128] its delivery slot
+  int* s_level_offset = s_rowslot + BM;   // first kLevelCache wavefront boundaries: no global round trip per level
   unsigned char* cstage_w = tiles_ptr + kRingBytes;
   const uint32_t epi_bar = smem_u32(bars + 2 * kMaxStages + 4);
   uint32_t epi_phase = 0;
@@ -271,6 +274,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  for (int i = tid; i < kLevelCache && i <= n_levels; i += kThreads) s_level_offset[i] = p.level_offset[i];
   if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // columns: 2 stages x 256; thin tiles use [0,128) and [128,256)
   tc_fence_before();
   __syncthreads();
@@ -293,7 +297,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
 
   if (only_level < 0 && n_levels > 0) {
     prepare_operands(p, blockIdx.x * kThreads + tid, gridDim.x * kThreads);
-    asm volatile("fence.proxy.async;" ::: "memory");    // Xin is read through TMA
+    asm volatile("fence.proxy.async.global;" ::: "memory");    // Xin is read through TMA
     ++barriers_passed;
     if (!grid_barrier(p.st, barriers_passed * gridDim.x, p.wait_limit, s_flag)) stop = true;
   }
@@ -301,7 +305,8 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   const int lvl_begin = only_level >= 0 ? only_level : 0;
   const int lvl_end = only_level >= 0 ? only_level + 1 : n_levels;
   for (int lvl = lvl_begin; lvl < lvl_end && !stop; ++lvl) {   // uniform trip count: barriers inside
-    const int begin = p.level_offset[lvl], end = p.level_offset[lvl + 1];
+    const int begin = lvl < kLevelCache ? s_level_offset[lvl] : p.level_offset[lvl];
+    const int end = lvl + 1 < kLevelCache ? s_level_offset[lvl + 1] : p.level_offset[lvl + 1];
     const bool leaf = lvl == 0;
     const int G = choose_groups_per_tile(end - begin, groups, p.sched_ctas);
     const int ntn = groups / G;                      // column tiles per row tile
@@ -319,7 +324,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
     // a wavefront of at most 64 (32) nodes fetches only that many operand rows per K block; the
     // MMA still spans 128 rows, the rest of the stage holds stale data for rows that are not stored
     const int a_rows = leaf || end - begin > 64 ? BM : (end - begin > 32 ? 64 : 32);
-    if (warp == 4 || warp == 10) asm volatile("fence.proxy.async;" ::: "memory");   // TMA reads after the barrier's acquire
+    if (warp == 4 || warp == 10) asm volatile("fence.proxy.async.global;" ::: "memory");   // TMA reads after the barrier's acquire
 
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
       const int row0 = begin + (t / ntn) * BM, nt = t % ntn;
