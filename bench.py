@@ -272,7 +272,7 @@ def main() -> int:
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="batch256_bf16", choices=fg.WORKLOADS)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--mode", default="persistent", choices=["persistent", "per_level"])
+    ap.add_argument("--mode", default="persistent", choices=["persistent", "per_level", "subforests"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-train", action="store_true", help="skip the extra training-step figure")
     ap.add_argument("--sweep", default=None, choices=["shapes", "length", "all"],
@@ -310,8 +310,9 @@ def main() -> int:
     model = binding.TreeLSTM(p.H, p.E, p.vocab, dev(p.emb), dev(p.W), dev(p.b), prec)
     model.set_option(binding.OPT_TIME_WAVEFRONT_KERNEL, 1)
     left, right, token = dev(f.left), dev(f.right), dev(f.token)
-    flags = binding.PERSISTENT if args.mode == "persistent" else binding.PER_LEVEL
+    flags = {"persistent": binding.PERSISTENT, "per_level": binding.PER_LEVEL, "subforests": binding.SUBFORESTS}[args.mode]
     out = model.forward(left, right, token, flags=flags)          # allocates outputs, checks status
+    ran = {binding.PERSISTENT: "persistent", binding.PER_LEVEL: "per_level", binding.SUBFORESTS: "subforests"}[model.last_mode()]
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
 
     sampler = ClockSampler(local_rank)
@@ -383,7 +384,7 @@ def main() -> int:
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.precision == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": args.workload, "trees": f.n_trees, "nodes": f.n_nodes, "leaves": f.n_leaves,
-                   "levels": int(out["n_levels"].item()), "H": p.H, "E": p.E, "vocab": p.vocab, "mode": args.mode,
+                   "levels": int(out["n_levels"].item()), "H": p.H, "E": p.E, "vocab": p.vocab, "mode": ran,
                    "l2": "flushed between timed steps (256 MB write, untimed)", "seed": "rank"},
         "nodes_per_sec": agg_nodes * args.steps / (total_ms * 1e-3),
         "step_ms_p10_p50_p90": [float(np.percentile(step_ms, q)) for q in (10, 50, 90)],

@@ -66,6 +66,15 @@ typedef enum treelstm_status {
 #define TREELSTM_PERSISTENT 1   /* one cooperative launch loops over the wavefronts with a bounded   */
                                 /* grid-wide barrier; fully asynchronous (see treelstm_status_sync)  */
 #define TREELSTM_SAVE_FOR_BACKWARD 2 /* keep every node's gate activations for treelstm_backward   */
+#define TREELSTM_SUBFORESTS 4   /* bf16 only: the trees are dealt out to as many sub-forests as      */
+                                /* thread-block clusters fit on the GPU; one cluster evaluates one   */
+                                /* sub-forest wavefront by wavefront with its slice of the recurrent */
+                                /* weights resident in shared memory and only the hardware cluster   */
+                                /* barrier between wavefronts (trees are independent, Section 2.2).  */
+                                /* One launch, asynchronous like TREELSTM_PERSISTENT, same results   */
+                                /* and same reported schedule.  Where it does not apply (fp32, H     */
+                                /* padded beyond 256, more than 24576 nodes) the call runs           */
+                                /* TREELSTM_PERSISTENT instead; treelstm_last_mode tells which.      */
 
 /* option keys of treelstm_set_option */
 #define TREELSTM_OPT_SCHED_SINGLE_CTA_MAX 1 /* forests up to this many nodes are scheduled by one  */
@@ -127,13 +136,14 @@ TREELSTM_API size_t treelstm_workspace_bytes(const treelstm_t* ctx, int max_node
  *   level_offset  [n_nodes + 2] out or NULL: wavefront l is order[level_offset[l] ..
  *                 level_offset[l+1]); entries past n_levels are unspecified.
  *   n_levels      [1] out (device): number of wavefronts.
- *   flags         TREELSTM_PER_LEVEL or TREELSTM_PERSISTENT, optionally | TREELSTM_SAVE_FOR_BACKWARD.
+ *   flags         TREELSTM_PER_LEVEL, TREELSTM_PERSISTENT or TREELSTM_SUBFORESTS, optionally
+ *                 | TREELSTM_SAVE_FOR_BACKWARD.
  *   workspace     device scratch of at least treelstm_workspace_bytes(ctx, n_nodes, save) bytes;
  *                 with TREELSTM_SAVE_FOR_BACKWARD it must stay untouched until backward is done.
  * Errors: INVALID_ARG for bad arguments (nothing is launched).  A malformed forest or a token
  * out of range is detected on the device: no out-of-bounds access happens, the outputs are
  * unspecified, and the code is returned by this call (TREELSTM_PER_LEVEL) or by
- * treelstm_status_sync (TREELSTM_PERSISTENT).
+ * treelstm_status_sync (TREELSTM_PERSISTENT, TREELSTM_SUBFORESTS).
  */
 TREELSTM_API int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const int32_t* right,
                      const int32_t* token, float* h, float* c, int32_t* level, int32_t* order,
@@ -257,6 +267,14 @@ TREELSTM_API int treelstm_selftest_waits(treelstm_t* ctx, void* workspace, size_
 
 /* Number of kernels the last forward / backward call on this context launched. */
 TREELSTM_API int treelstm_last_launch_count(const treelstm_t* ctx);
+
+/* Which evaluation the last successful forward ran: TREELSTM_PER_LEVEL, TREELSTM_PERSISTENT or
+ * TREELSTM_SUBFORESTS; -1 before any forward. */
+TREELSTM_API int treelstm_last_mode(const treelstm_t* ctx);
+
+/* Number of sub-forests TREELSTM_SUBFORESTS splits a forest into on this context's device (the
+ * number of co-resident clusters); 0 if that mode is not available for this context. */
+TREELSTM_API int treelstm_subforest_count(const treelstm_t* ctx);
 
 /* cudaError_t of the last failed CUDA call on this context (0 if none). */
 TREELSTM_API int treelstm_last_cuda_error(const treelstm_t* ctx);

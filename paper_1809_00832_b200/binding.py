@@ -29,6 +29,7 @@ BF16 = 1
 PER_LEVEL = 0
 PERSISTENT = 1
 SAVE_FOR_BACKWARD = 2
+SUBFORESTS = 4
 OPT_SCHED_SINGLE_CTA_MAX = 1
 OPT_WAIT_LIMIT_CYCLES = 2
 OPT_MAX_CTAS = 3
@@ -55,6 +56,8 @@ SIGNATURES = {
     "treelstm_selftest_waits": (_i, [_vp, _vp, ctypes.c_size_t, _vp, _vp]),
     "treelstm_last_kernel_ms": (_i, [_vp, ctypes.POINTER(ctypes.c_float)]),
     "treelstm_last_launch_count": (_i, [_vp]),
+    "treelstm_last_mode": (_i, [_vp]),
+    "treelstm_subforest_count": (_i, [_vp]),
     "treelstm_last_cuda_error": (_i, [_vp]),
     "treelstm_destroy": (_i, [_vp]),
     "treelstm_strerror": (ctypes.c_char_p, [_i]),
@@ -303,3 +306,10 @@ class TreeLSTM:
 
     def last_launch_count(self) -> int:
         return int(self.lib.treelstm_last_launch_count(self.handle))
+
+    def last_mode(self) -> int:
+        """PER_LEVEL, PERSISTENT or SUBFORESTS: the evaluation the last forward actually ran."""
+        return int(self.lib.treelstm_last_mode(self.handle))
+
+    def subforest_count(self) -> int:
+        return int(self.lib.treelstm_subforest_count(self.handle))

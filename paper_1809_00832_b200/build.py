@@ -9,7 +9,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libtreelstm_b200.so")
-SOURCES = ("api.cu", "schedule.cu", "cell_fp32.cu", "gemm_tc.cu", "backward.cu")
+SOURCES = ("api.cu", "schedule.cu", "cell_fp32.cu", "gemm_tc.cu", "subforest_tc.cu", "backward.cu")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

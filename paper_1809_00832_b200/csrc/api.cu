@@ -19,8 +19,11 @@ WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward) {
   L.roots = take(4 * nn);
   L.table = take(4 * (size_t)kRadixBins * ((nn + kRadixChunk - 1) / kRadixChunk));
   L.slot = take(4 * nn);
-  L.xin = L.ain = L.cin = off;
+  L.part_order = L.part_offset = L.part_spill = L.xin = L.ain = L.cin = off;
   if (ctx->precision == TREELSTM_BF16) {
+    L.part_order = take(4 * nn);                     // node ids by (sub-forest, level, id)
+    L.part_offset = take(4 * (kMaxParts + 1));
+    L.part_spill = take(4 * (nn + kMaxParts + 1));   // wavefront boundaries of very deep sub-forests
     L.xin = take(2 * nn * (size_t)ctx->Ep);          // leaf embedding rows in ready order
     L.ain = take(2 * nn * 2 * (size_t)ctx->Hp);      // [h_l | h_r] of every position, bf16
     L.cin = take(4 * nn * 2 * (size_t)ctx->H);       // [c_l | c_r] of every position, fp32
@@ -149,6 +152,7 @@ int treelstm_create(treelstm_t** out, int H, int E, int vocab, const float* emb,
   }
   int rc = copy_params(ctx, emb, W, b, s);
   if (rc != TREELSTM_OK) return fail(rc);
+  ctx->sf = subforest_plan(ctx);
   *out = ctx;
   return TREELSTM_OK;
 }
@@ -214,7 +218,7 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
   if (n_nodes < 0 || !n_levels || !workspace) return TREELSTM_ERR_INVALID_ARG;
   if (n_nodes > 0 && (!left || !right || !token || !h || !c || !level || !order))
     return TREELSTM_ERR_INVALID_ARG;
-  if (flags & ~(TREELSTM_PERSISTENT | TREELSTM_SAVE_FOR_BACKWARD)) return TREELSTM_ERR_INVALID_ARG;
+  if (flags & ~(TREELSTM_PERSISTENT | TREELSTM_SAVE_FOR_BACKWARD | TREELSTM_SUBFORESTS)) return TREELSTM_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return TREELSTM_ERR_INVALID_ARG;
   const bool save = (flags & TREELSTM_SAVE_FOR_BACKWARD) != 0;
   const WsLayout lay = ws_layout(ctx, n_nodes, save);
@@ -228,25 +232,36 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
   L.h = h; L.c = c; L.level = level; L.order = order; L.level_offset = lvl_off;
   L.ws = workspace; L.lay = lay; L.stream = s; L.host_levels_valid = false; L.n_levels = 0;
 
+  // Sub-forest mode needs the cluster plan of this context and a forest the single-CTA scheduler
+  // can deal out; anything else runs the grid-wide persistent kernel instead.
+  const int single_max = ctx->opt.sched_single_cta_max < kSchedPartMaxNodes ? ctx->opt.sched_single_cta_max
+                                                                             : kSchedPartMaxNodes;
+  const bool subforests = (flags & TREELSTM_SUBFORESTS) && ctx->precision == TREELSTM_BF16 && ctx->sf.ok &&
+                          n_nodes > 0 && n_nodes <= single_max;
   int rc = launch_schedule(ctx, n_nodes, left, right, token, level, order, lvl_off, n_levels, workspace,
-                           lay, s);
+                           lay, subforests ? ctx->sf.n_parts : 0, s);
   if (rc != TREELSTM_OK) return rc;
   L.valid = true;
   if (n_nodes == 0) return TREELSTM_OK;
 
-  const bool persistent = (flags & TREELSTM_PERSISTENT) != 0;
+  const bool persistent = (flags & (TREELSTM_PERSISTENT | TREELSTM_SUBFORESTS)) != 0;
+  L.mode = subforests ? TREELSTM_SUBFORESTS : (persistent ? TREELSTM_PERSISTENT : TREELSTM_PER_LEVEL);
   if (!persistent) {
     rc = read_levels(ctx);
     if (rc != TREELSTM_OK) { L.valid = false; return rc; }
   }
   ctx->ev_valid = false;
   if (ctx->opt.time_kernel) TL_CUDA(ctx, cudaEventRecord(ctx->ev_begin, s));
-  if (ctx->precision == TREELSTM_BF16)
+  if (subforests)
+    rc = launch_forward_bf16_subforest(ctx, n_nodes, left, right, token, h, c, level, flags, workspace, lay, s);
+  else if (ctx->precision == TREELSTM_BF16)
     rc = launch_forward_bf16(ctx, n_nodes, left, right, token, h, c, order, lvl_off,
-                             ctx->host_level_offset, L.n_levels, flags, workspace, lay, s);
+                             ctx->host_level_offset, L.n_levels, persistent ? (flags | TREELSTM_PERSISTENT) : flags,
+                             workspace, lay, s);
   else
     rc = launch_forward_fp32(ctx, n_nodes, left, right, token, h, c, order, lvl_off,
-                             ctx->host_level_offset, L.n_levels, flags, workspace, lay, s);
+                             ctx->host_level_offset, L.n_levels, persistent ? (flags | TREELSTM_PERSISTENT) : flags,
+                             workspace, lay, s);
   if (ctx->opt.time_kernel && rc == TREELSTM_OK) {
     TL_CUDA(ctx, cudaEventRecord(ctx->ev_end, s));
     ctx->ev_valid = true;
@@ -369,6 +384,10 @@ int treelstm_selftest_waits(treelstm_t* ctx, void* workspace, size_t workspace_b
 }
 
 int treelstm_last_launch_count(const treelstm_t* ctx) { return ctx ? ctx->launches : 0; }
+
+int treelstm_last_mode(const treelstm_t* ctx) { return ctx && ctx->last.valid ? ctx->last.mode : -1; }
+
+int treelstm_subforest_count(const treelstm_t* ctx) { return ctx && ctx->sf.ok ? ctx->sf.n_parts : 0; }
 
 int treelstm_last_cuda_error(const treelstm_t* ctx) { return ctx ? ctx->cuda_error : 0; }
 

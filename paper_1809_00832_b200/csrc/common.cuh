@@ -25,8 +25,8 @@ static_assert(sizeof(DevStatus) == 256, "control block is one 256-byte line grou
 
 // Offsets (bytes) of the regions inside the workspace for a forest of up to n nodes.
 struct WsLayout {
-  size_t status, parent, pending, order_tmp, level_offset, roots, table, slot, xin, ain, cin, gates,
-      dh, dc, dz, tok_slot, total;
+  size_t status, parent, pending, order_tmp, level_offset, roots, table, slot, part_order, part_offset,
+      part_spill, xin, ain, cin, gates, dh, dc, dz, tok_slot, total;
 };
 
 struct Options {
@@ -39,11 +39,19 @@ struct Options {
 constexpr int kRadixBins = 256;
 constexpr int kRadixChunk = 1024;        // items per single-warp CTA of the multi-CTA sort
 constexpr int kSchedSingleMaxNodes = 32768;
+constexpr int kSchedPartMaxNodes = 24576;   // largest forest the single-CTA scheduler can also deal out to sub-forests
+constexpr int kMaxParts = 32;               // upper bound on the number of sub-forests (co-resident clusters)
 
 // Padded sizes of the tensor-core path: hidden units in groups of 8 (one packed weight group =
 // 5 gates x 8 units = 40 rows), K blocks of 64 bf16 (one 128-byte swizzle span).
 constexpr int kUnitGroup = 8;
 constexpr int kKBlock = 64;
+
+// How the sub-forest (cluster) kernel runs for a context; ok = false: not available for its sizes.
+struct SubforestPlan {
+  bool ok = false;
+  int cluster_size = 0, groups_per_cta = 0, smem_bytes = 0, n_parts = 0;
+};
 
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 inline size_t round_up_sz(size_t x, size_t m) { return (x + m - 1) / m * m; }
@@ -74,13 +82,14 @@ struct treelstm {
   const void* tmap_ws_base = nullptr;   // tmap_x / tmap_a are rebuilt when the workspace or node count changes
   int tmap_ws_rows = 0;
   bool have_tmaps = false;
+  tl::SubforestPlan sf;                 // filled at create (bf16 only)
 
   tl::Options opt;
 
   // what the last forward call saw (needed by roots / backward / status_sync)
   struct Last {
     bool valid = false;
-    int n = 0, flags = 0;
+    int n = 0, flags = 0, mode = 0;   // mode: which wavefront kernel ran (TREELSTM_PER_LEVEL / PERSISTENT / SUBFORESTS)
     const int32_t *left = nullptr, *right = nullptr, *token = nullptr;
     float *h = nullptr, *c = nullptr;
     int32_t *level = nullptr, *order = nullptr, *level_offset = nullptr;
@@ -118,7 +127,7 @@ WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward);
 // schedule.cu: enqueue the on-device ready-set construction.  Returns a treelstm_status.
 int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
                     const int32_t* token, int32_t* level, int32_t* order, int32_t* level_offset,
-                    int32_t* n_levels_out, void* ws, const WsLayout& lay, cudaStream_t stream);
+                    int32_t* n_levels_out, void* ws, const WsLayout& lay, int n_parts, cudaStream_t stream);
 
 // cell_fp32.cu
 int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
@@ -134,6 +143,15 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
                         const int32_t* level_offset_dev, const int32_t* level_offset_host,
                         int n_levels_host, int flags, void* ws, const WsLayout& lay,
                         cudaStream_t stream);
+
+// Rebuilds the tensor maps over the dense operands when the workspace or the node count changed.
+int ensure_operand_tmaps(treelstm* ctx, void* ws, int n, const void* xin, const void* ain);
+
+// subforest_tc.cu
+SubforestPlan subforest_plan(treelstm* ctx);
+int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
+                                  const int32_t* token, float* h, float* c, const int32_t* level, int flags,
+                                  void* ws, const WsLayout& lay, cudaStream_t stream);
 
 int launch_selftest_waits(treelstm* ctx, void* ws, int* result_dev, cudaStream_t stream);
 

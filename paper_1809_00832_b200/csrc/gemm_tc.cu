@@ -26,25 +26,15 @@
 // warp 11 second MMA issuer: issuing one tcgen05.mma costs its thread about 83 cycles whatever N
 // is, so on thin tiles (N <= 128) the two issuers take alternate K blocks into two partial
 // accumulators that the epilogue adds.
-#include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace tl {
 namespace {
 
-constexpr int BM = 128;                 // nodes per tile (UMMA M)
-constexpr int kMaxStages = 8;
-constexpr int kThreads = 384;
-constexpr int kABytes = BM * 128;       // one K block (64 bf16) of 128 rows
-constexpr int kAccCols = 256;           // accumulator stage stride in tensor-memory columns
-constexpr int kAcc2Off = 128;           // second partial accumulator inside a stage (thin tiles only)
-constexpr unsigned kFull = 0xffffffffu;
-constexpr int kMaxG = 4;                // unit groups (of 8 hidden units) per tile: 1, 2 or 4
-constexpr int kGColsI = 40;             // packed rows per unit group, internal nodes (5 gates)
-constexpr int kGColsL = 24;             // packed rows per unit group, leaves (gates i, o, u)
+constexpr int kThreads = kTcThreads;
 constexpr int kBBytes = kMaxG * kGColsI * 128;
 constexpr int kRingBytes = kMaxStages * (kABytes + kGColsI * 128);   // 8 stages of the thinnest tile
 constexpr int kCBytes = BM * 2 * kMaxG * 8 * 4;   // staged child cell states: 128 rows x 2 x 32 fp32
-constexpr int kLevelCache = 1024;       // wavefront boundaries kept in shared memory
 constexpr int kSmemBytes = kRingBytes + kCBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*row ids*/ +
                            4 * kLevelCache;
 static_assert(kBBytes % 1024 == 0 && (kGColsI * 128) % 1024 == 0 && (kGColsL * 128) % 1024 == 0,
@@ -65,125 +55,7 @@ __host__ __device__ inline int choose_groups_per_tile(int rows, int groups, int 
   return best_g;
 }
 
-struct TcParams {
-  int n, H, Hp, Ep, sched_ctas;
-  const int *left, *right, *token, *order, *roots, *level_offset;
-  int* slot;
-  const __nv_bfloat16* emb_bf;
-  __nv_bfloat16 *xin, *ain;
-  float* cin;
-  const float *bp_h, *bp_x;
-  float *h, *c, *gates;
-  DevStatus* st;
-  long long wait_limit;
-};
 
-// ---- PTX wrappers ---------------------------------------------------------------------------- //
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok;
-}
-// Bounded wait: gives up when the cycle budget is spent or another thread of the CTA gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* s_abort,
-                                          long long limit, DevStatus* st) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*s_abort) return false;
-    if (clock64() - t0 > limit) {
-      *s_abort = 1;
-      report(st, TREELSTM_ERR_TIMEOUT);
-      return false;
-    }
-  }
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t* v) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
-               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the
-// 128-byte swizzle (8-row groups of 1024 bytes): start address, stride between 8-row groups,
-// descriptor version 1, swizzle mode 2.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
-  d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset
-  d |= (uint64_t)1 << 46;                 // version
-  d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
-  return d;
-}
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t umma_idesc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-
-// Activations of the bf16 path.  tanh.approx has an absolute error of about 5e-4, far inside the
-// 3e-2 budget of this path (the operands are already rounded to 8 mantissa bits).
-__device__ __forceinline__ float act_tanh(float x) {
-  float y;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float act_sigmoid(float x) { return fmaf(0.5f, act_tanh(0.5f * x), 0.5f); }
-
-__device__ __forceinline__ void st_row4(float* p, bool vec, int count, const float* v) {
-  if (vec && count == 4) {
-    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
-  } else {
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (j < count) p[j] = v[j];
-  }
-}
 
 // ---- the kernel -------------------------------------------------------------------------------- //
 // Before the first wavefront, spread over all threads of the grid:
@@ -355,9 +227,9 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
           }
         }
         __syncwarp();
-        stage = __shfl_sync(kFull, stage, 0);
-        phase_bits = __shfl_sync(kFull, phase_bits, 0);
-        alive = __shfl_sync(kFull, (int)alive, 0) != 0;
+        stage = __shfl_sync(kFullMask, stage, 0);
+        phase_bits = __shfl_sync(kFullMask, phase_bits, 0);
+        alive = __shfl_sync(kFullMask, (int)alive, 0) != 0;
       } else if (warp == 5 || warp == 11) {
         // ---------------- MMA issuers ----------------
         // Issuer w takes the K blocks with kb % 2 == w when the tile is thin (dual), else issuer 0
@@ -438,7 +310,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
           if (q < ngates) bnext[q] = __ldg(reinterpret_cast<const float4*>(bias + 8 * q));
         const uint32_t acc = acc_iter & 1, acc_phase = (acc_iter >> 1) & 1;
         if (!mbar_wait(tfull_bar(acc), acc_phase, s_abort, p.wait_limit, p.st)) alive = false;
-        alive = __all_sync(kFull, alive);
+        alive = __all_sync(kFullMask, alive);
         asm volatile("cp.async.wait_all;" ::: "memory");
         if (alive) {
           tc_fence_after();
@@ -679,6 +551,8 @@ __global__ void k_pack_embedding(int vocab, int E, int Ep, const float* emb, __n
   }
 }
 
+}  // namespace
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -703,8 +577,21 @@ int make_tmap(treelstm* ctx, CUtensorMap* map, const void* base, uint64_t inner,
   return TREELSTM_OK;
 }
 
-
-}  // namespace
+int ensure_operand_tmaps(treelstm* ctx, void* ws, int n, const void* xin, const void* ain) {
+  if (ctx->tmap_ws_base == ws && ctx->tmap_ws_rows == n) return TREELSTM_OK;
+  // the dense operands live in the caller's workspace
+  int rc = make_tmap(ctx, &ctx->tmap_x, xin, (uint64_t)ctx->Ep, (uint64_t)n, BM);
+  if (rc != TREELSTM_OK) return rc;
+  rc = make_tmap(ctx, &ctx->tmap_a, ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, BM);
+  if (rc != TREELSTM_OK) return rc;
+  rc = make_tmap(ctx, &ctx->tmap_a64, ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, 64);
+  if (rc != TREELSTM_OK) return rc;
+  rc = make_tmap(ctx, &ctx->tmap_a32, ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, 32);
+  if (rc != TREELSTM_OK) return rc;
+  ctx->tmap_ws_base = ws;
+  ctx->tmap_ws_rows = n;
+  return TREELSTM_OK;
+}
 
 int launch_selftest_waits(treelstm* ctx, void* ws, int* result_dev, cudaStream_t stream) {
   DevStatus* st = static_cast<DevStatus*>(ws);
@@ -752,17 +639,9 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.gates = (flags & TREELSTM_SAVE_FOR_BACKWARD) ? reinterpret_cast<float*>(base + lay.gates) : nullptr;
   p.st = reinterpret_cast<DevStatus*>(base + lay.status);
   p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
-  if (ctx->tmap_ws_base != ws || ctx->tmap_ws_rows != n) {   // the dense operands live in the caller's workspace
-    int rc = make_tmap(ctx, &ctx->tmap_x, p.xin, (uint64_t)ctx->Ep, (uint64_t)n, BM);
+  {
+    int rc = ensure_operand_tmaps(ctx, ws, n, p.xin, p.ain);
     if (rc != TREELSTM_OK) return rc;
-    rc = make_tmap(ctx, &ctx->tmap_a, p.ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, BM);
-    if (rc != TREELSTM_OK) return rc;
-    rc = make_tmap(ctx, &ctx->tmap_a64, p.ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, 64);
-    if (rc != TREELSTM_OK) return rc;
-    rc = make_tmap(ctx, &ctx->tmap_a32, p.ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, 32);
-    if (rc != TREELSTM_OK) return rc;
-    ctx->tmap_ws_base = ws;
-    ctx->tmap_ws_rows = n;
   }
 
   static bool attr_set = false;

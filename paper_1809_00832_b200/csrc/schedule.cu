@@ -131,8 +131,8 @@ __device__ void block_counting_pass(int n, const int* src, int* dst, KeyFn key, 
 
 // Ids of the items with flag(item) set, in ascending order, to dst; returns their number to every
 // thread.  One CTA of 32 warps; warp w owns a contiguous range of ids.
-template <class FlagFn>
-__device__ int block_compact(int n, int* dst, FlagFn flag, int* scan_tmp) {
+template <class FlagFn, class PlaceFn = NoPlace>
+__device__ int block_compact(int n, int* dst, FlagFn flag, int* scan_tmp, PlaceFn place = NoPlace()) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   int per_warp = (n + kSingleWarps - 1) / kSingleWarps;
   per_warp = (per_warp + 31) & ~31;
@@ -155,7 +155,11 @@ __device__ int block_compact(int n, int* dst, FlagFn flag, int* scan_tmp) {
     const int r = r0 + lane;
     const bool f = r < end && flag(r);
     const unsigned m = __ballot_sync(kFull, f);
-    if (f) dst[base + __popc(m & lanemask_lt())] = r;
+    if (f) {
+      const int idx = base + __popc(m & lanemask_lt());
+      dst[idx] = r;
+      place(idx, r);
+    }
     base += __popc(m);
   }
   __syncthreads();
@@ -171,11 +175,18 @@ __device__ int block_compact(int n, int* dst, FlagFn flag, int* scan_tmp) {
 //
 // Dynamic shared memory: uint32 w[n] (dependency words; later the radix histogram, at least 32 KB),
 // uint16 par[n] (caller of each node, the return location of Section 4.1.2; later level | root
-// flag), uint16 queue[n / 2] (start nodes of the climb).
+// flag), uint16 queue[n / 2] (start nodes of the climb), and with n_parts > 0 uint16 lab[n].
+//
+// n_parts > 0 additionally deals the trees out to n_parts sub-forests (trees are independent,
+// Section 2.2): every node learns the root of its tree by pointer jumping over the caller links,
+// the t-th root (ascending node id) goes to sub-forest t mod n_parts, and part_order receives the
+// node ids by ascending (sub-forest, level, node id) with part_offset[0 .. n_parts] marking where
+// each sub-forest starts.  slot[] (if given) is set to -1 for every node.
 __global__ void __launch_bounds__(kSingleThreads, 1)
 k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ right,
                   const int* __restrict__ token, int vocab, int* parent, int* level, int* order,
-                  int* order_tmp, int* level_offset, int* roots, int* n_levels_out, DevStatus* st) {
+                  int* order_tmp, int* level_offset, int* roots, int* n_levels_out, DevStatus* st,
+                  int n_parts, int* part_order, int* part_offset, int* slot) {
   extern __shared__ __align__(16) unsigned char smem[];
   const size_t w_bytes = (size_t)n * 4 > sizeof(int) * kRadixBins * kSingleWarps
                              ? (((size_t)n * 4 + 15) & ~(size_t)15) : sizeof(int) * kRadixBins * kSingleWarps;
@@ -184,6 +195,8 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
   unsigned short* par = reinterpret_cast<unsigned short*>(smem + w_bytes);
   unsigned short* lv16 = par;
   unsigned short* queue = par + (((size_t)n + 7) & ~(size_t)7);   // start nodes of the climb, at most n / 2
+  unsigned short* lab = reinterpret_cast<unsigned short*>(
+      smem + w_bytes + ((((size_t)n * 2) + 15) & ~(size_t)15) + (((size_t)n + 15) & ~(size_t)15));
   __shared__ int scan_tmp[32];
   __shared__ int s_err, s_maxlevel, s_qhead, s_qtail;
   const int tid = threadIdx.x;
@@ -282,6 +295,10 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
       const int lvl = (int)(wk & 0x7FFFu);
       const unsigned short pk = par[k];
       lv16[k] = (unsigned short)(lvl | (pk == kNoParent ? 0x8000 : 0));
+      if (n_parts > 0) {
+        lab[k] = pk == kNoParent ? (unsigned short)k : pk;   // start of the pointer jumping
+        if (slot) slot[k] = -1;
+      }
       level[k] = lvl;
       local_max = max(local_max, lvl);
     }
@@ -310,9 +327,34 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
     }
   }
   if (tid == 0) { level_offset[n_levels] = n; st->n_levels = n_levels; *n_levels_out = n_levels; }
-  // roots (nodes without a caller) in ascending node id
-  const int n_roots = block_compact(n, roots, [=](int item) { return (lv16[item] & 0x8000) != 0; }, scan_tmp);
+  if (n_parts > 0) {
+    // lab[k] = root of k's tree: every node replaces its link by its link's link until all links
+    // end at a root (a root links to itself); ceil(log2(depth)) + 1 rounds.  Updates are made in
+    // place: a link read while it is being advanced is still an ancestor.
+    for (int round = 0; round < 17; ++round) {
+      int changed = 0;
+      for (int k = tid; k < n; k += kSingleThreads) {
+        const unsigned short a = lab[k], b = lab[a];
+        if (b != a) { lab[k] = b; changed = 1; }
+      }
+      if (!__syncthreads_or(changed)) break;
+    }
+  }
+  // roots (nodes without a caller) in ascending node id; the t-th root takes sub-forest t mod n_parts
+  const int n_roots = block_compact(n, roots, [=](int item) { return (lv16[item] & 0x8000) != 0; }, scan_tmp,
+                                    [=](int idx, int item) { if (n_parts > 0) lab[item] = (unsigned short)(idx % n_parts); });
   if (tid == 0) st->n_roots = n_roots;
+  if (n_parts > 0) {
+    // every other node takes its root's sub-forest (its own entry is read by nobody else: links
+    // end at roots only)
+    for (int k = tid; k < n; k += kSingleThreads)
+      if (!(lv16[k] & 0x8000)) lab[k] = lab[lab[k]];
+    __syncthreads();
+    // stable pass over the ready order by sub-forest: ascending (sub-forest, level, node id)
+    block_counting_pass(n, order, part_order, [=](int item) { return (int)lab[item]; }, hist, scan_tmp,
+                        part_offset, n_parts);
+    if (tid == 0) part_offset[n_parts] = n;
+  }
 }
 
 // ------------------------------------------------------------------------------------------ //
@@ -507,16 +549,17 @@ __global__ void k_gather_roots(int max_roots, int H, const int* roots, const flo
 
 }  // namespace
 
-size_t single_smem_bytes(int n) {
+size_t single_smem_bytes(int n, bool with_parts) {
   size_t w = (size_t)n * 4;
   const size_t hist = sizeof(int) * kRadixBins * kSingleWarps;
   w = w > hist ? round_up_sz(w, 16) : hist;
-  return w + round_up_sz((size_t)n * 2, 16) + round_up_sz((size_t)n, 16);
+  return w + round_up_sz((size_t)n * 2, 16) + round_up_sz((size_t)n, 16) +
+         (with_parts ? round_up_sz((size_t)n * 2, 16) : 0);
 }
 
 int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
                     const int32_t* token, int32_t* level, int32_t* order, int32_t* level_offset,
-                    int32_t* n_levels_out, void* ws, const WsLayout& lay, cudaStream_t stream) {
+                    int32_t* n_levels_out, void* ws, const WsLayout& lay, int n_parts, cudaStream_t stream) {
   char* base = static_cast<char*>(ws);
   DevStatus* st = reinterpret_cast<DevStatus*>(base + lay.status);
   int* parent = reinterpret_cast<int*>(base + lay.parent);
@@ -531,13 +574,15 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
     static bool attr_set = false;
     if (!attr_set) {
       TL_CUDA(ctx, cudaFuncSetAttribute(k_schedule_single, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)single_smem_bytes(kSchedSingleMaxNodes)));
+                                        (int)single_smem_bytes(kSchedSingleMaxNodes, false)));
       attr_set = true;
     }
     // the kernel clears the control block itself and writes the level count to the caller
-    k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n), stream>>>(
+    const bool parts = n_parts > 0 && n <= kSchedPartMaxNodes;
+    k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n, parts), stream>>>(
         n, left, right, token, ctx->vocab, parent, level, order, order_tmp, level_offset, roots, n_levels_out,
-        st);
+        st, parts ? n_parts : 0, reinterpret_cast<int*>(base + lay.part_order),
+        reinterpret_cast<int*>(base + lay.part_offset), reinterpret_cast<int*>(base + lay.slot));
     ctx->launches += 1;
     TL_CUDA(ctx, cudaGetLastError());
     return TREELSTM_OK;
@@ -626,7 +671,7 @@ extern "C" int treelstm_schedule_static(int n_nodes, const int32_t* left, const 
     void* addr = nullptr;
     if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return TREELSTM_ERR_CUDA;
     if (cudaFuncSetAttribute(k_schedule_single, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)single_smem_bytes(kSchedSingleMaxNodes)) != cudaSuccess)
+                             (int)single_smem_bytes(kSchedSingleMaxNodes, false)) != cudaSuccess)
       return TREELSTM_ERR_CUDA;
     g_static_scratch_addr[dev] = static_cast<unsigned char*>(addr);
   }
@@ -639,8 +684,9 @@ extern "C" int treelstm_schedule_static(int n_nodes, const int32_t* left, const 
   if (n_nodes > 0) {
     // the control block keeps the previous call's status and counts; the kernel's first step is
     // to clear it, everything else in the array is rewritten before it is read
-    k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n_nodes), s>>>(
-        n_nodes, left, right, token, vocab, parent, level, order, order_tmp, level_offset, roots, n_levels, st);
+    k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n_nodes, false), s>>>(
+        n_nodes, left, right, token, vocab, parent, level, order, order_tmp, level_offset, roots, n_levels, st,
+        0, nullptr, nullptr, nullptr);
     if (cudaGetLastError() != cudaSuccess) return TREELSTM_ERR_CUDA;
   } else {
     if (cudaMemsetAsync(st, 0, sizeof(DevStatus), s) != cudaSuccess ||

@@ -1,0 +1,582 @@
+// bf16 tensor-core evaluation of sub-forests on thread-block clusters (sm_100a).
+//
+// Paper: Section 2.2 - the trees of a batch, like sibling subtrees, are independent of each other;
+// Section 4.1.1 - a node is ready once its inputs are resolved.  The scheduler deals the trees of
+// the forest out to as many sub-forests as clusters fit on the GPU.  One cluster evaluates one
+// sub-forest wavefront by wavefront, on its own: the wait between two wavefronts is the hardware
+// cluster barrier (a fraction of a microsecond) instead of a grid-wide barrier through global
+// memory, and nothing ever waits for another sub-forest.
+//
+// Inside a cluster the recurrent weights are stationary: CTA r of the cluster owns the gate columns
+// of hidden units [r * 8 * g, (r + 1) * 8 * g) (g unit groups per CTA) and keeps that slice of the
+// packed W_h in shared memory for the whole kernel, so an internal wavefront only streams its
+// operand rows.  Every CTA walks all row tiles of a wavefront of its sub-forest; a tile is 128 ready
+// nodes x (8 * g hidden units x 5 gates), accumulated in tensor memory by tcgen05.mma and finished
+// by the same fused cell epilogue as the grid-wide kernel (gemm_tc.cu): a node's bf16 h and fp32 c
+// go straight into the operand row of its caller, rows being positions in the ready order of the
+// sub-forest, so every wavefront's operand is a contiguous block of rows fetched by tiled TMA.
+//
+// Warp roles as in gemm_tc.cu (384 threads): warps 0-3 and 6-9 epilogue, warp 4 TMA producer of the
+// operand rows, warp 10 TMA producer of the W_x tiles of the leaf wavefront (and of the resident
+// W_h slice), warps 5 and 11 MMA issuers (both on single-tile wavefronts, alternate K blocks into
+// two partial accumulators).
+#include "tc_ptx.cuh"
+
+namespace tl {
+namespace {
+
+constexpr int kThreads = kTcThreads;
+constexpr int kSmemLimit = 232448;       // 227 KB of dynamic shared memory per CTA
+constexpr int kFixedBytes = 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*row ids*/ + 4 * (kLevelCache + 1);
+
+struct SfLayout {
+  uint32_t wres_bytes, ring_bytes, cstage_bytes, crow_shift, total;
+};
+
+// Shared-memory plan of one CTA: resident W_h slice | operand ring | child-cell / output staging.
+__host__ __device__ inline SfLayout sf_layout(int Hp, int gpc) {
+  SfLayout L;
+  L.wres_bytes = (uint32_t)(2 * Hp / kKBlock) * (uint32_t)gpc * kGColsI * 128u;
+  L.crow_shift = gpc <= 2 ? 7u : 8u;                       // staging row: 2 x (8 * gpc) fp32, padded to 128 / 256 B
+  L.cstage_bytes = (uint32_t)BM << L.crow_shift;
+  const int stage_leaf = kABytes + gpc * kGColsL * 128;
+  int avail = kSmemLimit - 1024 /*static shared memory*/ - kFixedBytes - (int)L.wres_bytes - (int)L.cstage_bytes;
+  int ring = kMaxStages * stage_leaf;
+  if (ring > avail) ring = avail;
+  if (ring < 0) ring = 0;
+  L.ring_bytes = (uint32_t)ring & ~1023u;
+  L.total = L.wres_bytes + L.ring_bytes + L.cstage_bytes + kFixedBytes;
+  return L;
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+// Hardware barrier of the cluster; every thread of every CTA of the cluster takes part.  Release /
+// acquire: what the cluster's threads wrote before it (global memory included) is visible after it.
+__device__ __forceinline__ void cluster_sync_all() {
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CUtensorMap tmap_wx,
+                   const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_a,
+                   const __grid_constant__ CUtensorMap tmap_a64, const __grid_constant__ CUtensorMap tmap_a32,
+                   TcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const int G = p.groups_per_cta;
+  const SfLayout L = sf_layout(p.Hp, G);
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t wres_addr = (raw_addr + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_raw + (wres_addr - raw_addr);
+  const uint32_t ring_addr = wres_addr + L.wres_bytes;
+  const uint32_t cstage_addr = ring_addr + L.ring_bytes;
+  unsigned char* cstage_ptr = base_ptr + L.wres_bytes + L.ring_bytes;
+  unsigned char* fixed_ptr = cstage_ptr + L.cstage_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(fixed_ptr);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty,
+  // bars[2S+4]: meeting point of the 256 epilogue threads, bars[2S+5]: resident W_h slice has landed
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 6);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  int* s_nlev = const_cast<int*>(s_abort) + 1;
+  int* s_rownode = reinterpret_cast<int*>(fixed_ptr + 256);   // [128] node id of each tile row
+  int* s_rowslot = s_rownode + BM;                            // [128] its delivery slot
+  int* s_loff = s_rowslot + BM;                               // wavefront boundaries of this sub-forest
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + 2 + a); };
+  const uint32_t epi_bar = bar0 + 8u * (2 * kMaxStages + 4);
+  const uint32_t wres_bar = bar0 + 8u * (2 * kMaxStages + 5);
+  uint32_t epi_phase = 0;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // A failed schedule leaves the level count at 0.  (The status word is not used for this test: a
+  // sibling cluster may record a timeout in it at any moment, and the CTAs of one cluster have to
+  // take the same decision or the ones that stay would wait at the cluster barrier forever.)
+  if (ld_volatile(&p.st->n_levels) <= 0) return;
+  const int cs = (int)cluster_nctarank(), rank = (int)cluster_ctarank();
+  const int part = blockIdx.x / cs;
+  const int pbeg = p.part_offset[part], pend = p.part_offset[part + 1];
+  if (pbeg >= pend) return;                         // empty sub-forest: the whole cluster leaves
+
+  if (tid == 0) {
+    for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 2); mbar_init(tempty_bar(a), 256); }
+    mbar_init(epi_bar, 256);
+    mbar_init(wres_bar, 1);
+    *s_abort = 0;
+    *s_nlev = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // 2 stages x 256 columns; partial sums at +128
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+
+  const int Hp = p.Hp, H = p.H;
+  const int kb_leaf = p.Ep / kKBlock, kb_int = 2 * Hp / kKBlock;
+  const bool vec = (H % 4) == 0;
+  const int nt = rank;                               // this CTA's slice of the hidden units
+
+  // The slice of the packed recurrent weights this CTA keeps: K block kb, unit group g at
+  // wres + (kb * G + g) * 5120 bytes (40 rows of 128 bytes, 128-byte swizzle).
+  if (warp == 10 && lane == 0) {
+    mbar_arrive_expect_tx(wres_bar, L.wres_bytes);
+    for (int kb = 0; kb < kb_int; ++kb)
+      for (int g = 0; g < G; ++g)
+        tma_load_2d(wres_addr + (uint32_t)(kb * G + g) * (kGColsI * 128u), &tmap_wh, kb * kKBlock,
+                    (nt * G + g) * kGColsI, wres_bar);
+  }
+
+  // Wavefront boundaries of the sub-forest: its nodes are sorted by level, the levels are 0 .. top
+  // without gaps.  Every CTA builds the table for itself.
+  int* spill = p.part_level_spill + pbeg + part;     // entries past the shared-memory table
+  for (int q = pbeg + tid; q < pend; q += kThreads) {
+    const int lv = p.level[p.order[q]];
+    const int lvp = q > pbeg ? p.level[p.order[q - 1]] : -1;
+    if (lv != lvp) { if (lv <= kLevelCache) s_loff[lv] = q; else spill[lv] = q; }
+    if (q == pend - 1) {
+      if (lv + 1 <= kLevelCache) s_loff[lv + 1] = pend; else spill[lv + 1] = pend;
+      *s_nlev = lv + 1;
+    }
+  }
+  __syncthreads();
+  const int n_levels = *s_nlev;
+  auto loff = [&](int l) { return l <= kLevelCache ? s_loff[l] : __ldcg(spill + l); };
+
+  // Operands of the sub-forest, spread over the threads of the cluster: embedding rows of its
+  // leaves in ready order (Xin), and for every internal position the slots its two children
+  // deliver their state to (slot[] of a root stays -1, set by the scheduler).
+  {
+    const int gtid = rank * kThreads + tid, gthreads = cs * kThreads;
+    const int lend = loff(1);
+    const int cpr = p.Ep / 8;                              // 16-byte chunks per row
+    const long long total = (long long)(lend - pbeg) * cpr;
+    for (long long ch = gtid; ch < total; ch += gthreads) {
+      const int row = pbeg + (int)(ch / cpr), cc = (int)(ch % cpr);
+      const int tok = p.token[p.order[row]];
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.emb_bf + (size_t)tok * p.Ep) + cc);
+      reinterpret_cast<uint4*>(p.xin + (size_t)row * p.Ep)[cc] = v;
+    }
+    for (int pos = lend + gtid; pos < pend; pos += gthreads) {
+      const int node = p.order[pos];
+      p.slot[p.left[node]] = 2 * pos;
+      p.slot[p.right[node]] = 2 * pos + 1;
+    }
+    asm volatile("fence.proxy.async.global;" ::: "memory");    // Xin is read through TMA
+  }
+  cluster_sync_all();
+
+  uint32_t stage = 0, phase_bits = 0;   // operand ring (producers and MMA issuers)
+  uint32_t acc_iter = 0;                // accumulator ring (MMA issuers and epilogue)
+  bool alive = true;
+  bool stop = false;                    // uniform over the CTA
+  bool wres_ready = false;
+
+  for (int lvl = 0; lvl < n_levels; ++lvl) {   // same trip count in every CTA of the cluster
+    if (!stop) {
+      const int begin = loff(lvl), end = loff(lvl + 1);
+      const bool leaf = lvl == 0;
+      const int tiles = (end - begin + BM - 1) / BM;
+      const int kblocks = leaf ? kb_leaf : kb_int;
+      const int gcols = leaf ? kGColsL : kGColsI;
+      const int ncols = G * gcols;                     // accumulator columns in use
+      const int ncols_mma = (ncols + 15) & ~15;        // UMMA N (columns past ncols are never read)
+      const bool dual = ncols_mma <= kAcc2Off && kblocks >= 2 && tiles == 1;
+      const uint32_t stage_bytes = leaf ? (uint32_t)kABytes + (uint32_t)ncols * 128u : (uint32_t)kABytes;
+      const uint32_t n_stages = min((uint32_t)kMaxStages, L.ring_bytes / stage_bytes);
+      stage = 0;
+      const int a_rows = leaf || end - begin > 64 ? BM : (end - begin > 32 ? 64 : 32);
+      if (warp == 4 || warp == 10) asm volatile("fence.proxy.async.global;" ::: "memory");   // TMA reads after the barrier's acquire
+
+      for (int t = 0; t < tiles && alive; ++t) {
+        const int row0 = begin + t * BM;
+
+        if (warp == 4 || (warp == 10 && leaf)) {
+          // ---------------- operand producers (TMA) ----------------
+          const bool is_a = warp == 4;
+          const CUtensorMap* map = is_a ? (leaf ? &tmap_x : (a_rows == BM ? &tmap_a : (a_rows == 64 ? &tmap_a64 : &tmap_a32)))
+                                        : &tmap_wx;
+          const uint32_t bytes = is_a ? (uint32_t)a_rows * 128u : (uint32_t)ncols * 128u;
+          auto issue = [&](int kb, uint32_t st_idx) {
+            const uint32_t sa = ring_addr + st_idx * stage_bytes;
+            mbar_arrive_expect_tx(full_bar(st_idx), bytes);
+            if (is_a) {
+              tma_load_2d(sa, map, kb * kKBlock, row0, full_bar(st_idx));
+              if (!leaf) mbar_arrive(full_bar(st_idx));   // stands in for the W producer: W_h is resident
+            } else {
+              for (int g = 0; g < G; ++g)
+                tma_load_2d(sa + kABytes + (uint32_t)(g * gcols) * 128u, map, kb * kKBlock,
+                            (nt * G + g) * gcols, full_bar(st_idx));
+            }
+          };
+          int kb_first = 0;
+          if (t == 0) {
+            // first tile of a wavefront: the ring is empty, the first n_stages K blocks need no wait
+            const int burst = min(kblocks, (int)n_stages);
+            if (lane < burst) issue(lane, (uint32_t)lane);
+            __syncwarp();
+            phase_bits ^= (1u << burst) - 1u;
+            stage = (uint32_t)burst == n_stages ? 0u : (uint32_t)burst;
+            kb_first = burst;
+          }
+          if (lane == 0) {
+            for (int kb = kb_first; kb < kblocks; ++kb) {
+              if (!mbar_wait(empty_bar(stage), ((phase_bits >> stage) & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) {
+                alive = false;
+                break;
+              }
+              issue(kb, stage);
+              phase_bits ^= 1u << stage;
+              if (++stage == n_stages) stage = 0;
+            }
+          }
+          __syncwarp();
+          stage = __shfl_sync(kFullMask, stage, 0);
+          phase_bits = __shfl_sync(kFullMask, phase_bits, 0);
+          alive = __shfl_sync(kFullMask, (int)alive, 0) != 0;
+        } else if (warp == 5 || warp == 11) {
+          // ---------------- MMA issuers ----------------
+          if (lane == 0) {
+            const int w = warp == 5 ? 0 : 1;
+            const uint32_t acc = acc_iter & 1, acc_phase = (acc_iter >> 1) & 1;
+            if (!dual && w == 1) {
+              if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
+              mbar_arrive(tfull_bar(acc));
+              for (int kb = 0; kb < kblocks; ++kb) {
+                phase_bits ^= 1u << stage;
+                if (++stage == n_stages) stage = 0;
+              }
+            } else {
+              if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
+              if (!leaf && !wres_ready) {
+                if (!mbar_wait(wres_bar, 0, s_abort, p.wait_limit, p.st)) alive = false;
+                wres_ready = true;
+              }
+              tc_fence_after();
+              const uint32_t d_tmem = tmem_base + acc * kAccCols + (w == 1 ? (uint32_t)kAcc2Off : 0u);
+              const uint32_t idesc = umma_idesc(ncols_mma);
+              bool first = true;
+              for (int kb = 0; kb < kblocks && alive; ++kb) {
+                if (!dual || (kb & 1) == w) {
+                  if (!mbar_wait(full_bar(stage), (phase_bits >> stage) & 1u, s_abort, p.wait_limit, p.st)) {
+                    alive = false;
+                    break;
+                  }
+                  tc_fence_after();
+                  const uint32_t a_addr = ring_addr + stage * stage_bytes;
+                  const uint32_t b_addr = leaf ? a_addr + kABytes : wres_addr + (uint32_t)kb * (uint32_t)ncols * 128u;
+                  const uint64_t a_desc = umma_desc(a_addr), b_desc = umma_desc(b_addr);
+#pragma unroll
+                  for (int k = 0; k < kKBlock / 16; ++k)   // UMMA K = 16 bf16 = 32 bytes = 2 descriptor units
+                    umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, !(first && k == 0));
+                  first = false;
+                  umma_commit(empty_bar(stage));           // frees the ring stage when these MMAs retire
+                }
+                phase_bits ^= 1u << stage;
+                if (++stage == n_stages) stage = 0;
+              }
+              if (alive) umma_commit(tfull_bar(acc));      // this issuer's partial accumulator is complete
+            }
+          }
+          ++acc_iter;
+        } else if (warp != 10) {
+          // ---------------- epilogue: drain tensor memory, finish the cell ----------------
+          const int e = warp < 4 ? 0 : 1;   // warps 0-3: units [0,4) of every group, warps 6-9: [4,8)
+          const int quad = warp & 3;        // tensor-memory lane quadrant this warp may read
+          const int r = quad * 32 + lane;
+          const int row = row0 + r;
+          const bool valid = row < end;
+          const int node = valid ? p.order[row] : 0;
+          const int slot = valid ? p.slot[node] : -1;   // 2 * pos(caller) + side, -1 for a root
+          const float* crow = p.cin + (size_t)row * 2 * H;   // [c_l | c_r] of the node at this position
+          const bool full_slice = vec && (nt + 1) * G * 8 <= H;   // no padded unit in this CTA's slice
+          const bool staged = !leaf && full_slice;
+          const bool staged_out = full_slice && p.gates == nullptr;
+          const int half = 4 << (L.crow_shift - 7);        // chunk index where the second half of a staging row starts
+          const uint32_t my_c = cstage_addr + ((uint32_t)r << L.crow_shift);
+          unsigned char* mine = cstage_ptr + ((size_t)r << L.crow_shift);
+          if (staged) {
+            const float* sl = crow + nt * G * 8;
+            const float* sr = sl + H;
+            const uint32_t nb = valid ? 16u : 0u;
+            for (int ch = e; ch < 2 * G; ch += 2) {
+              cp_async16(my_c + (uint32_t)((ch ^ (r & 7)) << 4), sl + ch * 4, nb);
+              cp_async16(my_c + (uint32_t)(((half + ch) ^ (r & 7)) << 4), sr + ch * 4, nb);
+            }
+          }
+          const float* bias = (leaf ? p.bp_x : p.bp_h) + nt * ncols + 4 * e;
+          const int ngates = leaf ? 3 : 5;
+          float4 bnext[5];
+#pragma unroll
+          for (int q = 0; q < 5; ++q)
+            if (q < ngates) bnext[q] = __ldg(reinterpret_cast<const float4*>(bias + 8 * q));
+          const uint32_t acc = acc_iter & 1, acc_phase = (acc_iter >> 1) & 1;
+          if (!mbar_wait(tfull_bar(acc), acc_phase, s_abort, p.wait_limit, p.st)) alive = false;
+          alive = __all_sync(kFullMask, alive);
+          asm volatile("cp.async.wait_all;" ::: "memory");
+          if (alive) {
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(quad * 32) << 16) + 4u * e;
+            uint32_t vbuf[2][20], v2[20];
+            auto load_group = [&](int g, uint32_t* v) {
+              const uint32_t col0 = (uint32_t)(g * gcols);
+              if (leaf) {
+#pragma unroll
+                for (int q = 0; q < 3; ++q) tmem_ld4(taddr + col0 + 8 * q, v + 4 * q);
+              } else {
+#pragma unroll
+                for (int q = 0; q < 5; ++q) tmem_ld4(taddr + col0 + 8 * q, v + 4 * q);
+              }
+            };
+            auto add_second = [&](int g, uint32_t* v) {   // single-tile wavefronts: add the second issuer's partial sums
+              const uint32_t col0 = (uint32_t)kAcc2Off + (uint32_t)(g * gcols);
+#pragma unroll
+              for (int q = 0; q < 5; ++q)
+                if (q < ngates) tmem_ld4(taddr + col0 + 8 * q, v2 + 4 * q);
+              tmem_ld_wait();
+#pragma unroll
+              for (int j = 0; j < 20; ++j)
+                if (j < 4 * ngates) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
+            };
+            load_group(0, vbuf[0]);
+#pragma unroll
+            for (int g = 0; g < kMaxG; ++g) {
+              if (g >= G) break;
+              uint32_t* v = vbuf[g & 1];
+              float4 bcur[5];
+#pragma unroll
+              for (int q = 0; q < 5; ++q) bcur[q] = bnext[q];
+              tmem_ld_wait();
+              if (dual) add_second(g, v);
+              if (g + 1 < G) {
+                load_group(g + 1, vbuf[(g + 1) & 1]);
+#pragma unroll
+                for (int q = 0; q < 5; ++q)
+                  if (q < ngates) bnext[q] = __ldg(reinterpret_cast<const float4*>(bias + (g + 1) * gcols + 8 * q));
+              }
+              if (valid) {
+                const int u0 = (nt * G + g) * 8 + 4 * e;
+                const int count = min(4, H - u0);     // real (unpadded) units among these four
+                float cl[4] = {}, cr[4] = {}, hv[4], cv[4], gi[4], gfl[4], gfr[4], go[4], gu[4];
+                if (staged) {
+                  const float4 a = *reinterpret_cast<const float4*>(mine + (((2 * g + e) ^ (r & 7)) << 4));
+                  const float4 b = *reinterpret_cast<const float4*>(mine + (((half + 2 * g + e) ^ (r & 7)) << 4));
+                  cl[0] = a.x; cl[1] = a.y; cl[2] = a.z; cl[3] = a.w;
+                  cr[0] = b.x; cr[1] = b.y; cr[2] = b.z; cr[3] = b.w;
+                } else if (!leaf && count > 0) {
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    cl[j] = j < count ? __ldcg(crow + u0 + j) : 0.f;
+                    cr[j] = j < count ? __ldcg(crow + H + u0 + j) : 0.f;
+                  }
+                }
+                const float* bq = reinterpret_cast<const float*>(bcur);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  if (leaf) {
+                    gi[j] = act_sigmoid(__uint_as_float(v[j]) + bq[j]);
+                    go[j] = act_sigmoid(__uint_as_float(v[4 + j]) + bq[4 + j]);
+                    gu[j] = act_tanh(__uint_as_float(v[8 + j]) + bq[8 + j]);
+                    gfl[j] = gfr[j] = 0.f;
+                    cv[j] = gi[j] * gu[j];
+                  } else {
+                    gi[j] = act_sigmoid(__uint_as_float(v[j]) + bq[j]);
+                    gfl[j] = act_sigmoid(__uint_as_float(v[4 + j]) + bq[4 + j]);
+                    gfr[j] = act_sigmoid(__uint_as_float(v[8 + j]) + bq[8 + j]);
+                    go[j] = act_sigmoid(__uint_as_float(v[12 + j]) + bq[12 + j]);
+                    gu[j] = act_tanh(__uint_as_float(v[16 + j]) + bq[16 + j]);
+                    cv[j] = gi[j] * gu[j] + gfl[j] * cl[j] + gfr[j] * cr[j];
+                  }
+                  hv[j] = go[j] * act_tanh(cv[j]);
+                }
+                if (staged_out) {
+                  *reinterpret_cast<float4*>(mine + (((2 * g + e) ^ (r & 7)) << 4)) = make_float4(cv[0], cv[1], cv[2], cv[3]);
+                  *reinterpret_cast<float4*>(mine + (((half + 2 * g + e) ^ (r & 7)) << 4)) = make_float4(hv[0], hv[1], hv[2], hv[3]);
+                } else {
+                  if (slot >= 0) {
+                    // hand the state to the caller: bf16 h into its operand row (padded units as 0),
+                    // fp32 c next to it
+                    uint32_t packed[2];
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                      const float lo = 2 * j < count ? hv[2 * j] : 0.f, hi = 2 * j + 1 < count ? hv[2 * j + 1] : 0.f;
+                      __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+                      packed[j] = *reinterpret_cast<uint32_t*>(&b2);
+                    }
+                    *reinterpret_cast<uint2*>(p.ain + (size_t)slot * Hp + u0) = make_uint2(packed[0], packed[1]);
+                    if (count > 0) st_row4(p.cin + (size_t)slot * H + u0, vec, count, cv);
+                  }
+                  if (count > 0) {
+                    st_row4(p.h + (size_t)node * H + u0, vec, count, hv);
+                    st_row4(p.c + (size_t)node * H + u0, vec, count, cv);
+                    if (p.gates) {
+                      float* gp = p.gates + (size_t)node * 5 * H + u0;
+                      st_row4(gp, vec, count, gi);
+                      st_row4(gp + H, vec, count, gfl);
+                      st_row4(gp + 2 * H, vec, count, gfr);
+                      st_row4(gp + 3 * H, vec, count, go);
+                      st_row4(gp + 4 * H, vec, count, gu);
+                    }
+                  }
+                }
+              }
+            }
+            tc_fence_before();
+            mbar_arrive(tempty_bar(acc));              // accumulator stage may be overwritten
+            if (staged_out) {
+              // all epilogue threads copy whole row segments out, several lanes per row
+              if (e == 0) { s_rownode[r] = valid ? node : -1; s_rowslot[r] = slot; }
+              mbar_arrive(epi_bar);
+              bool ok = mbar_wait(epi_bar, epi_phase, s_abort, p.wait_limit, p.st);
+              epi_phase ^= 1;
+              if (ok) {
+                const int et = e * BM + r, cpr = 2 * G;           // 16-byte chunks (4 units) per row
+                for (int idx = et; idx < BM * cpr; idx += 2 * BM) {
+                  const int ro = idx / cpr, ch = idx % cpr;
+                  const int node_o = s_rownode[ro];
+                  if (node_o < 0) continue;
+                  const unsigned char* src = cstage_ptr + ((size_t)ro << L.crow_shift);
+                  const float4 c4 = *reinterpret_cast<const float4*>(src + ((ch ^ (ro & 7)) << 4));
+                  const float4 h4 = *reinterpret_cast<const float4*>(src + (((half + ch) ^ (ro & 7)) << 4));
+                  const int uo = nt * G * 8 + 4 * ch;
+                  *reinterpret_cast<float4*>(p.h + (size_t)node_o * H + uo) = h4;
+                  *reinterpret_cast<float4*>(p.c + (size_t)node_o * H + uo) = c4;
+                  const int slot_o = s_rowslot[ro];
+                  if (slot_o >= 0) {
+                    *reinterpret_cast<float4*>(p.cin + (size_t)slot_o * H + uo) = c4;
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(h4.x, h4.y), hi = __floats2bfloat162_rn(h4.z, h4.w);
+                    *reinterpret_cast<uint2*>(p.ain + (size_t)slot_o * Hp + uo) =
+                        make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+                  }
+                }
+              }
+              // the staging rows are reused by the next tile's loads of the children's cell states
+              mbar_arrive(epi_bar);
+              ok = mbar_wait(epi_bar, epi_phase, s_abort, p.wait_limit, p.st) && ok;
+              epi_phase ^= 1;
+              if (!ok) alive = false;
+            }
+            // the operand rows written above are read through TMA (async proxy) by later wavefronts
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+          }
+          ++acc_iter;
+        }
+      }
+    }
+    if (lvl + 1 < n_levels) {
+      // Every thread of the cluster meets here.  A CTA in which a wait expired keeps coming to the
+      // barriers (its peers must not wait for it forever) but does no more work.
+      cluster_sync_all();
+      if (*s_abort) stop = true;
+    }
+  }
+
+  // teardown: let in-flight asynchronous copies land before shared/tensor memory is released
+  if (warp == 10 && lane == 0 && !wres_ready) mbar_wait(wres_bar, 0, s_abort, p.wait_limit, p.st);
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  tc_fence_before();
+  __syncthreads();
+  if (*s_abort) __nanosleep(100000);
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+// How the sub-forest kernel would run for this context: cluster size, unit groups per CTA, bytes of
+// dynamic shared memory, and how many clusters are resident at once (= number of sub-forests).
+// ok = false if the hidden size does not fit the weight-stationary plan.
+SubforestPlan subforest_plan(treelstm* ctx) {
+  SubforestPlan pl{};
+  if (ctx->precision != TREELSTM_BF16) return pl;
+  const int groups = ctx->Hp / kUnitGroup;
+  int cs = 0;
+  if (groups % 16 == 0) cs = 16; else if (groups % 8 == 0) cs = 8; else return pl;
+  const int gpc = groups / cs;
+  if (gpc < 1 || gpc > 3) return pl;
+  const SfLayout L = sf_layout(ctx->Hp, gpc);
+  if (L.ring_bytes < 3u * (kABytes + gpc * kGColsL * 128)) return pl;   // fewer than 3 leaf stages: not worth it
+  if (cudaFuncSetAttribute(k_fwd_tc_subforest, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total) != cudaSuccess ||
+      cudaFuncSetAttribute(k_fwd_tc_subforest, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+    cudaGetLastError();
+    return pl;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(cs); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = L.total;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  int n_clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&n_clusters, k_fwd_tc_subforest, &cfg) != cudaSuccess || n_clusters < 1) {
+    cudaGetLastError();
+    return pl;
+  }
+  pl.ok = true;
+  pl.cluster_size = cs;
+  pl.groups_per_cta = gpc;
+  pl.smem_bytes = (int)L.total;
+  pl.n_parts = n_clusters < kMaxParts ? n_clusters : kMaxParts;
+  return pl;
+}
+
+int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
+                                  const int32_t* token, float* h, float* c, const int32_t* level, int flags,
+                                  void* ws, const WsLayout& lay, cudaStream_t stream) {
+  if (!ctx->have_tmaps || !ctx->sf.ok) return TREELSTM_ERR_STATE;
+  char* base = static_cast<char*>(ws);
+  TcParams p{};
+  p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep; p.sched_ctas = ctx->sm_count;
+  p.left = left; p.right = right; p.token = token;
+  p.order = reinterpret_cast<int*>(base + lay.part_order);   // rows are positions in this order
+  p.roots = reinterpret_cast<int*>(base + lay.roots);
+  p.level_offset = nullptr;
+  p.emb_bf = ctx->emb_bf;
+  p.slot = reinterpret_cast<int*>(base + lay.slot);
+  p.xin = reinterpret_cast<__nv_bfloat16*>(base + lay.xin);
+  p.ain = reinterpret_cast<__nv_bfloat16*>(base + lay.ain);
+  p.cin = reinterpret_cast<float*>(base + lay.cin);
+  p.bp_h = ctx->bp_h; p.bp_x = ctx->bp_x;
+  p.h = h; p.c = c;
+  p.gates = (flags & TREELSTM_SAVE_FOR_BACKWARD) ? reinterpret_cast<float*>(base + lay.gates) : nullptr;
+  p.st = reinterpret_cast<DevStatus*>(base + lay.status);
+  p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
+  p.level = level;
+  p.part_offset = reinterpret_cast<int*>(base + lay.part_offset);
+  p.part_level_spill = reinterpret_cast<int*>(base + lay.part_spill);
+  p.n_parts = ctx->sf.n_parts;
+  p.groups_per_cta = ctx->sf.groups_per_cta;
+  int rc = ensure_operand_tmaps(ctx, ws, n, p.xin, p.ain);
+  if (rc != TREELSTM_OK) return rc;
+
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = ctx->sf.cluster_size; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(ctx->sf.n_parts * ctx->sf.cluster_size);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = ctx->sf.smem_bytes;
+  cfg.stream = stream;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  TL_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_fwd_tc_subforest, ctx->tmap_wh, ctx->tmap_wx, ctx->tmap_x, ctx->tmap_a,
+                                  ctx->tmap_a64, ctx->tmap_a32, p));
+  ctx->launches += 1;
+  return TREELSTM_OK;
+}
+
+}  // namespace tl

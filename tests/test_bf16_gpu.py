@@ -10,14 +10,22 @@ from tests import util
 
 pytestmark = pytest.mark.gpu
 
-MODES = [binding.PER_LEVEL, binding.PERSISTENT]
+MODES = [binding.PER_LEVEL, binding.PERSISTENT, binding.SUBFORESTS]
 TIGHT = 2e-3        # vs. the oracle fed bf16-rounded operands: only accumulation order, fast
                     # activations and the bf16 rounding of h at slightly different values remain
+
+
+def _subforests_apply(params, forest):
+    """sub-forest mode exists for hidden sizes whose 64-padded value is 64, 128, 192 or 256 and
+    forests the single-CTA scheduler can partition"""
+    return -(-params.H // 64) * 64 <= 256 and forest.n_nodes <= 24576
 
 
 def _check(params, forest, flags, full_ref=None):
     model = util.make_model(params, "bf16")
     res = util.gpu_forward(model, forest, flags)
+    if flags == binding.SUBFORESTS and _subforests_apply(params, forest):
+        assert model.last_mode() == binding.SUBFORESTS     # the cluster kernel ran, not its stand-in
     status, _, level, order, off = orc.schedule(forest.left, forest.right)
     util.check_schedule(res, dict(level=level, order=order, level_offset=off), forest.n_nodes)
     if full_ref is None:
@@ -124,6 +132,52 @@ def test_bf16_repeated_calls_and_changing_sizes():
     for n_trees in (40, 3, 17, 40):
         forest = fg.random_forest(rng, n_trees, 1, 30, 300)
         res = util.gpu_forward(model, forest, binding.PERSISTENT)
+        h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
+        assert util.max_abs(res["h"], h) < util.TOL["bf16"]
+        assert util.max_abs(res["c"], c) < util.TOL["bf16"]
+
+
+def test_subforest_mode_single_tree_and_fewer_trees_than_clusters():
+    """fewer trees than clusters: the spare clusters get empty sub-forests and leave at once"""
+    rng = np.random.default_rng(41)
+    params = fg.draw_params(rng, 128, 50, 300, emb_dist="normal", emb_scale=0.3, w_scale=0.15)
+    for n_trees in (1, 2, 5):
+        forest = fg.random_forest(rng, n_trees, 1, 56, 300)
+        forest, _ = fg.permute_node_ids(forest, rng)
+        _check(params, forest, binding.SUBFORESTS)
+
+
+def test_subforest_mode_single_leaf_trees():
+    """trees that are a single leaf: sub-forests with one wavefront only"""
+    rng = np.random.default_rng(42)
+    params = fg.draw_params(rng, 64, 64, 100, emb_dist="normal", emb_scale=0.3, w_scale=0.2)
+    forest = fg.random_forest(rng, 20, 1, 1, 100)
+    assert forest.n_nodes == 20
+    _check(params, forest, binding.SUBFORESTS)
+
+
+def test_subforest_mode_falls_back_when_it_does_not_apply():
+    """H padded beyond 256: the call runs the grid-wide persistent kernel and says so"""
+    rng = np.random.default_rng(43)
+    params = fg.draw_params(rng, 264, 32, 100, emb_dist="normal", emb_scale=0.3, w_scale=0.05)
+    forest = fg.random_forest(rng, 4, 2, 12, 100)
+    model = util.make_model(params, "bf16")
+    assert model.subforest_count() == 0
+    res = util.gpu_forward(model, forest, binding.SUBFORESTS)
+    assert model.last_mode() == binding.PERSISTENT
+    h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
+    assert util.max_abs(res["h"], h) < util.TOL["bf16"]
+
+
+def test_subforest_mode_repeated_calls():
+    rng = np.random.default_rng(44)
+    params = fg.draw_params(rng, 256, 64, 300, emb_dist="normal", emb_scale=0.3, w_scale=0.1)
+    model = util.make_model(params, "bf16")
+    assert model.subforest_count() >= 1
+    for n_trees in (40, 3, 17, 40):
+        forest = fg.random_forest(rng, n_trees, 1, 30, 300)
+        res = util.gpu_forward(model, forest, binding.SUBFORESTS)
+        assert model.last_mode() == binding.SUBFORESTS
         h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
         assert util.max_abs(res["h"], h) < util.TOL["bf16"]
         assert util.max_abs(res["c"], c) < util.TOL["bf16"]
