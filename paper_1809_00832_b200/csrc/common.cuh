@@ -47,6 +47,22 @@ constexpr int kMaxParts = 32;               // upper bound on the number of sub-
 constexpr int kUnitGroup = 8;
 constexpr int kKBlock = 64;
 
+// Tiled tensor maps of the operands, all three-dimensional {64 elements (one 128-byte swizzle span),
+// rows, K blocks} so that one request brings several K blocks of a tile.  Index [..][0]: the box
+// spans all K blocks of the operand, [..][1]: two K blocks.
+struct TmapSet {
+  CUtensorMap a[3][2];    // operand rows of internal wavefronts (Ain), box rows 32 / 64 / 128
+  CUtensorMap x[2];       // operand rows of the leaf wavefront (Xin), box rows 128
+  CUtensorMap wh[3][2];   // packed recurrent weights, box rows 40 g for g = 1, 2, 4 unit groups
+  CUtensorMap wx[3][2];   // packed input weights, box rows 24 g
+};
+
+// Maps of the sub-forest (cluster) kernel: its CTAs take g unit groups each, g = 1, 2 or 3.
+struct SfTmapSet {
+  CUtensorMap wres;       // packed recurrent weights, box = the whole slice of a CTA: 40 g rows x all K blocks
+  CUtensorMap wx[2];      // packed input weights, box rows 24 g
+};
+
 // How the sub-forest (cluster) kernel runs for a context; ok = false: not available for its sizes.
 struct SubforestPlan {
   bool ok = false;
@@ -78,8 +94,9 @@ struct treelstm {
   __nv_bfloat16* Wp_x = nullptr;    // [(Hp/8)*24][Ep]    packed input weights (gates i, o, u)
   float* bp_h = nullptr;            // [(Hp/8)*40] bias in packed column order
   float* bp_x = nullptr;            // [(Hp/8)*24]
-  CUtensorMap tmap_wh, tmap_wx, tmap_x, tmap_a, tmap_a64, tmap_a32;
-  const void* tmap_ws_base = nullptr;   // tmap_x / tmap_a are rebuilt when the workspace or node count changes
+  tl::TmapSet maps;                     // passed to the kernels by value
+  tl::SfTmapSet sf_maps;
+  const void* tmap_ws_base = nullptr;   // the operand maps are rebuilt when the workspace or node count changes
   int tmap_ws_rows = 0;
   bool have_tmaps = false;
   tl::SubforestPlan sf;                 // filled at create (bf16 only)
@@ -180,11 +197,13 @@ __device__ __forceinline__ void report(DevStatus* st, int code) { atomicMin(&st-
 __device__ __forceinline__ int ld_volatile(const int* p) { return *(const volatile int*)p; }
 
 // Bounded grid-wide barrier for cooperative (co-resident) launches.  `target` is the total
-// number of arrivals expected so far (gridDim.x * number of barriers passed, this one included).
+// number of arrivals expected so far (this barrier included).  A CTA that wrote nothing since the
+// last barrier may pass arrive = false: it only waits, and the caller counts it out of `target`
+// (arrivals on one counter are served one after the other, so fewer of them end the barrier sooner).
 // Returns false if the wait expired or another CTA reported an error: the caller must then
 // leave its level loop (every CTA sees the same outcome within one more barrier).
 __device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
-                                             long long limit_cycles, int* s_flag) {
+                                             long long limit_cycles, int* s_flag, bool arrive = true) {
   __syncthreads();
   if (threadIdx.x < 32) {
     // Warp 0 polls.  Lane 0 announces the arrival (release: everything this CTA wrote, ordered
@@ -193,7 +212,7 @@ __device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
     // after an eighth of the memory latency on average instead of half of it.
     if (threadIdx.x == 0) {
       *s_flag = -1;
-      asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&st->barrier) : "memory");
+      if (arrive) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&st->barrier) : "memory");
     }
     __syncwarp();
     const int lane = threadIdx.x;

@@ -40,22 +40,51 @@ constexpr int kSmemBytes = kRingBytes + kCBytes + 1024 /*alignment slack*/ + 256
 static_assert(kBBytes % 1024 == 0 && (kGColsI * 128) % 1024 == 0 && (kGColsL * 128) % 1024 == 0,
               "every TMA box lands on a 1024-byte boundary of the swizzle pattern");
 
-// How many unit groups a tile of this wavefront covers.  Narrow wavefronts are cut into many thin
-// tiles (all SMs get work, short MMA and epilogue per tile); wide ones into fat tiles (fewer
-// re-reads of the operand rows).  Cost model: rounds x (fixed latency + per-group work).
-__host__ __device__ inline int choose_groups_per_tile(int rows, int groups, int n_ctas) {
-  const int mt = (rows + BM - 1) / BM;
-  int best_g = 1, best_cost = 1 << 30;
-  for (int g = 1; g <= kMaxG; g <<= 1) {
-    const int tiles = mt * (groups / g);
-    const int rounds = (tiles + n_ctas - 1) / n_ctas;
-    const int cost = rounds * (4 + g);
-    if (cost <= best_cost) { best_cost = cost; best_g = g; }
+// Tile shape of a wavefront: rt ready nodes (32, 64 or 128; the MMA always spans 128 rows, the rest
+// of the accumulator is not stored) x g unit groups (1, 2 or 4).  Narrow wavefronts are cut into many
+// small tiles (every SM gets one, each fetches little), wide ones into fat tiles (fewer re-reads of
+// the operand rows).  Cost model, in units of one operand row: rounds x (fixed + rt + 40 g).
+// The operands of a tile arrive in boxes of kbox K blocks (one TMA request per operand and box); a
+// box is one stage of the shared-memory ring: [kbox x rt operand rows | kbox x 40 g weight rows].
+struct TilePlan {
+  int g, lg, rt, lrt, tiles;
+  int sel, kbox, n_box, n_stages;          // sel 0: one box spans all K blocks, 1: boxes of two K blocks
+  uint32_t a_bytes, w_bytes, stage_bytes;  // operand rows / weight rows of one K block; one stage
+};
+__host__ __device__ inline TilePlan choose_tile_plan(int rows, int groups, int n_ctas, bool leaf, int kblocks) {
+  TilePlan best{1, 0, BM, 7, 0, 0, 0, 0, 0, 0u, 0u, 0u};
+  int best_cost = 1 << 30, best_rounds = 1;
+  for (int lrt = 7; lrt >= (leaf ? 7 : 5); --lrt) {      // leaf rows come through a 128-row box only
+    const int rt = 1 << lrt;
+    const int mt = (rows + rt - 1) >> lrt;
+    for (int lg = 0; lg <= 2; ++lg) {
+      if (groups & ((1 << lg) - 1)) break;                // g must divide the number of unit groups
+      const int tiles = mt * (groups >> lg);
+      int rounds = 1;
+      while (rounds * n_ctas < tiles) ++rounds;
+      const int cost = rounds * (256 + rt + (40 << lg));
+      if (cost < best_cost || (cost == best_cost && lg > best.lg)) {
+        best_cost = cost;
+        best_rounds = rounds;
+        best.g = 1 << lg; best.lg = lg; best.rt = rt; best.lrt = lrt; best.tiles = tiles;
+      }
+    }
   }
-  return best_g;
+  best.a_bytes = (uint32_t)best.rt * 128u;
+  best.w_bytes = (uint32_t)(best.g * (leaf ? kGColsL : kGColsI)) * 128u;
+  const uint32_t kb_bytes = best.a_bytes + best.w_bytes;
+  // A wavefront done in one round takes each tile's operands in one request when they fit; with
+  // several rounds, boxes of two K blocks let loads, MMAs and epilogues of consecutive tiles overlap.
+  if (best_rounds == 1 && (uint32_t)kblocks * kb_bytes <= (uint32_t)kRingBytes) {
+    best.sel = 0; best.kbox = kblocks; best.n_box = 1;
+  } else {
+    best.sel = 1; best.kbox = 2; best.n_box = (kblocks + 1) >> 1;
+  }
+  best.stage_bytes = (uint32_t)best.kbox * kb_bytes;
+  best.n_stages = kMaxStages;
+  while ((uint32_t)best.n_stages * best.stage_bytes > (uint32_t)kRingBytes) --best.n_stages;
+  return best;
 }
-
-
 
 // ---- the kernel -------------------------------------------------------------------------------- //
 // Before the first wavefront, spread over all threads of the grid:
@@ -64,14 +93,7 @@ __host__ __device__ inline int choose_groups_per_tile(int rows, int groups, int 
 //     (where that child will deliver its state), slot[root] = -1.
 __device__ void prepare_operands(const TcParams& p, int gtid, int gthreads) {
   const int n_leaves = p.level_offset[1];
-  const int cpr = p.Ep / 8;                              // 16-byte chunks per row
-  const long long total = (long long)n_leaves * cpr;
-  for (long long ch = gtid; ch < total; ch += gthreads) {
-    const int row = (int)(ch / cpr), cc = (int)(ch % cpr);
-    const int tok = p.token[p.order[row]];
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.emb_bf + (size_t)tok * p.Ep) + cc);
-    reinterpret_cast<uint4*>(p.xin + (size_t)row * p.Ep)[cc] = v;
-  }
+  gather_leaf_rows(p, 0, n_leaves, gtid >> 5, gthreads >> 5, gtid & 31);
   for (int pos = n_leaves + gtid; pos < p.n; pos += gthreads) {
     const int node = p.order[pos];
     p.slot[p.left[node]] = 2 * pos;
@@ -90,10 +112,7 @@ __global__ void k_prepare_operands(TcParams p) {
 // only_level < 0: prepare the operands, then all wavefronts, separated by the bounded grid barrier (cooperative
 // launch).
 __global__ void __launch_bounds__(kThreads, 1)
-k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CUtensorMap tmap_wx,
-         const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_a,
-         const __grid_constant__ CUtensorMap tmap_a64, const __grid_constant__ CUtensorMap tmap_a32,
-         TcParams p, int only_level) {
+k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
@@ -109,6 +128,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   int* s_rownode = reinterpret_cast<int*>(tiles_ptr + kRingBytes + kCBytes + 256);   // [128] node id of each tile row
   int* s_rowslot = s_rownode + BM;                                                   // [128] its delivery slot
   int* s_level_offset = s_rowslot + BM;   // first kLevelCache wavefront boundaries: no global round trip per level
+  __shared__ TilePlan s_plan[2];          // tile plans of this and the next wavefront (written by warp 11)
   unsigned char* cstage_w = tiles_ptr + kRingBytes;
   const uint32_t epi_bar = smem_u32(bars + 2 * kMaxStages + 4);
   uint32_t epi_phase = 0;
@@ -124,13 +144,13 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
 
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 2); mbar_init(tempty_bar(a), 256); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
     mbar_init(epi_bar, 256);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   for (int i = tid; i < kLevelCache && i <= n_levels; i += kThreads) s_level_offset[i] = p.level_offset[i];
-  if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // columns: 2 stages x 256; thin tiles use [0,128) and [128,256)
+  if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // columns: 2 accumulator stages x 256
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -146,82 +166,72 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
   // own phase, tracked per stage in a bit mask.
   uint32_t stage = 0, phase_bits = 0;   // smem ring (producer and MMA)
   uint32_t acc_iter = 0;                // accumulator ring (MMA and epilogue)
-  uint32_t barriers_passed = 0;
+  uint32_t arrivals = 0;                // arrivals at the grid barrier expected so far
   bool alive = true;
   bool stop = false;                    // uniform over the CTA
 
   if (only_level < 0 && n_levels > 0) {
     prepare_operands(p, blockIdx.x * kThreads + tid, gridDim.x * kThreads);
     asm volatile("fence.proxy.async.global;" ::: "memory");    // Xin is read through TMA
-    ++barriers_passed;
-    if (!grid_barrier(p.st, barriers_passed * gridDim.x, p.wait_limit, s_flag)) stop = true;
+    arrivals += gridDim.x;
+    if (!grid_barrier(p.st, arrivals, p.wait_limit, s_flag)) stop = true;
   }
 
   const int lvl_begin = only_level >= 0 ? only_level : 0;
   const int lvl_end = only_level >= 0 ? only_level + 1 : n_levels;
+  auto level_begin = [&](int l) { return l < kLevelCache ? s_level_offset[l] : p.level_offset[l]; };
+  auto make_plan = [&](int l) {
+    return choose_tile_plan(level_begin(l + 1) - level_begin(l), groups, p.sched_ctas, l == 0, l == 0 ? kb_leaf : kb_int);
+  };
+  // Choosing a plan costs a few hundred cycles: one otherwise idle thread (warp 11) does it a
+  // wavefront ahead, everybody else picks the result up after the barrier.
+  if (warp == 11 && lane == 0 && lvl_begin < lvl_end) s_plan[lvl_begin & 1] = make_plan(lvl_begin);
+  __syncthreads();
   for (int lvl = lvl_begin; lvl < lvl_end && !stop; ++lvl) {   // uniform trip count: barriers inside
-    const int begin = lvl < kLevelCache ? s_level_offset[lvl] : p.level_offset[lvl];
-    const int end = lvl + 1 < kLevelCache ? s_level_offset[lvl + 1] : p.level_offset[lvl + 1];
+    const int begin = level_begin(lvl), end = level_begin(lvl + 1);
     const bool leaf = lvl == 0;
-    const int G = choose_groups_per_tile(end - begin, groups, p.sched_ctas);
-    const int ntn = groups / G;                      // column tiles per row tile
-    const int tiles = ((end - begin + BM - 1) / BM) * ntn;
+    const TilePlan plan = s_plan[lvl & 1];
+    if (warp == 11 && lane == 0 && lvl + 1 < lvl_end) s_plan[(lvl + 1) & 1] = make_plan(lvl + 1);
+    const int G = plan.g, rt = plan.rt;
+    const int ntn = groups >> plan.lg;               // column tiles per row tile
+    const int tiles = plan.tiles;
     const int kblocks = leaf ? kb_leaf : kb_int;
     const int gcols = leaf ? kGColsL : kGColsI;
     const int ncols = G * gcols;                     // accumulator columns in use
     const int ncols_mma = (ncols + 15) & ~15;        // UMMA N (columns past ncols are never read)
-    // two issuers and two partial accumulators where the MMA issue chain is the critical path: thin
-    // tiles of a wavefront that takes a single round (the epilogue pays for adding the partial sums)
-    const bool dual = ncols_mma <= kAcc2Off && kblocks >= 2 && tiles <= (int)gridDim.x;
-    const uint32_t stage_bytes = kABytes + (uint32_t)G * kGColsI * 128u;
-    const uint32_t n_stages = min((uint32_t)kMaxStages, (uint32_t)kRingBytes / stage_bytes);
+    // A stage holds one box: kbox x rt operand rows, then kbox x ncols weight rows.  The MMA reads 128
+    // rows from the start of a K block; what lies behind the rt fetched rows feeds accumulator rows
+    // that are not stored.
+    const uint32_t a_bytes = plan.a_bytes, w_bytes = plan.w_bytes, stage_bytes = plan.stage_bytes;
+    const uint32_t n_stages = (uint32_t)plan.n_stages;
+    const int kbox = plan.kbox, n_box = plan.n_box;
     stage = 0;
-    // a wavefront of at most 64 (32) nodes fetches only that many operand rows per K block; the
-    // MMA still spans 128 rows, the rest of the stage holds stale data for rows that are not stored
-    const int a_rows = leaf || end - begin > 64 ? BM : (end - begin > 32 ? 64 : 32);
-    if (warp == 4 || warp == 10) asm volatile("fence.proxy.async.global;" ::: "memory");   // TMA reads after the barrier's acquire
 
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
-      const int row0 = begin + (t / ntn) * BM, nt = t % ntn;
+      const int rtile = t / ntn, nt = t - rtile * ntn;
+      const int row0 = begin + (rtile << plan.lrt);
+      const int row_end = min(end, row0 + rt);        // rows of this tile: [row0, row_end)
 
       if (warp == 4 || warp == 10) {
         // ---------------- operand producers (TMA) ----------------
-        // Warp 4, A: 128 consecutive rows of the dense operand matrix (rows past its end read as
-        // zero, rows past the wavefront belong to later wavefronts and only feed accumulator rows
-        // that are never stored).  Warp 10, W: one box per unit group of the packed weights.
-        const bool is_a = warp == 4;
-        const CUtensorMap* map = is_a ? (leaf ? &tmap_x : (a_rows == BM ? &tmap_a : (a_rows == 64 ? &tmap_a64 : &tmap_a32)))
-                                      : (leaf ? &tmap_wx : &tmap_wh);
-        const uint32_t bytes = is_a ? (uint32_t)a_rows * 128u : (uint32_t)ncols * 128u;
-        auto issue = [&](int kb, uint32_t st_idx) {
-          const uint32_t sa = tiles_addr + st_idx * stage_bytes;
-          mbar_arrive_expect_tx(full_bar(st_idx), bytes);
-          if (is_a) {
-            tma_load_2d(sa, map, kb * kKBlock, row0, full_bar(st_idx));
-          } else {
-            for (int g = 0; g < G; ++g)
-              tma_load_2d(sa + kABytes + (uint32_t)(g * gcols) * 128u, map, kb * kKBlock,
-                          (nt * G + g) * gcols, full_bar(st_idx));
-          }
-        };
-        int kb_first = 0;
-        if (t == (int)blockIdx.x) {
-          // First tile of a wavefront: the ring was drained before the barrier, so the first
-          // n_stages K blocks need no wait; one lane per K block issues them in a single step.
-          const int burst = min(kblocks, (int)n_stages);
-          if (lane < burst) issue(lane, (uint32_t)lane);
-          __syncwarp();
-          phase_bits ^= (1u << burst) - 1u;
-          stage = (uint32_t)burst == n_stages ? 0u : (uint32_t)burst;
-          kb_first = burst;
-        }
+        // Warp 4: the operand rows [row0, row0 + rt) of the dense operand matrix (rows past its end
+        // read as zero; rows past the wavefront belong to later wavefronts and only feed accumulator
+        // rows that are never stored).  Warp 10: the g unit groups of the packed weights.  One request
+        // per box and operand; the two warps issue side by side.
         if (lane == 0) {
-          for (int kb = kb_first; kb < kblocks; ++kb) {
+          const bool is_a = warp == 4;
+          const CUtensorMap* map = is_a ? (leaf ? &maps.x[plan.sel] : &maps.a[plan.lrt - 5][plan.sel])
+                                        : (leaf ? &maps.wx[plan.lg][plan.sel] : &maps.wh[plan.lg][plan.sel]);
+          const uint32_t bytes = (uint32_t)kbox * (is_a ? a_bytes : w_bytes);
+          const uint32_t off = is_a ? 0u : (uint32_t)kbox * a_bytes;
+          const int y = is_a ? row0 : nt * ncols;
+          for (int box = 0; box < n_box; ++box) {
             if (!mbar_wait(empty_bar(stage), ((phase_bits >> stage) & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) {
               alive = false;
               break;
             }
-            issue(kb, stage);
+            mbar_arrive_expect_tx(full_bar(stage), bytes);
+            tma_load_3d(tiles_addr + stage * stage_bytes + off, map, 0, y, box * kbox, full_bar(stage));
             phase_bits ^= 1u << stage;
             if (++stage == n_stages) stage = 0;
           }
@@ -230,51 +240,39 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
         stage = __shfl_sync(kFullMask, stage, 0);
         phase_bits = __shfl_sync(kFullMask, phase_bits, 0);
         alive = __shfl_sync(kFullMask, (int)alive, 0) != 0;
-      } else if (warp == 5 || warp == 11) {
-        // ---------------- MMA issuers ----------------
-        // Issuer w takes the K blocks with kb % 2 == w when the tile is thin (dual), else issuer 0
-        // takes them all.  Both walk the whole ring so that their stage/phase counters agree.
+      } else if (warp == 5) {
+        // ---------------- MMA issuer ----------------
         if (lane == 0) {
-          const int w = warp == 5 ? 0 : 1;
           const uint32_t acc = acc_iter & 1, acc_phase = (acc_iter >> 1) & 1;
-          if (!dual && w == 1) {
-            // nothing to add for this tile; wait for the accumulator stage like issuer 0 does, so that
-            // this arrival cannot run ahead into the stage's next use
-            if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
-            mbar_arrive(tfull_bar(acc));
-            for (int kb = 0; kb < kblocks; ++kb) {
-              phase_bits ^= 1u << stage;
-              if (++stage == n_stages) stage = 0;
+          if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + acc * kAccCols;
+          const uint32_t idesc = umma_idesc(ncols_mma);
+          bool first = true;
+          for (int box = 0; box < n_box && alive; ++box) {
+            if (!mbar_wait(full_bar(stage), (phase_bits >> stage) & 1u, s_abort, p.wait_limit, p.st)) {
+              alive = false;
+              break;
             }
-          } else {
-            if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + acc * kAccCols + (w == 1 ? (uint32_t)kAcc2Off : 0u);
-            const uint32_t idesc = umma_idesc(ncols_mma);
-            bool first = true;
-            for (int kb = 0; kb < kblocks && alive; ++kb) {
-              if (!dual || (kb & 1) == w) {
-                if (!mbar_wait(full_bar(stage), (phase_bits >> stage) & 1u, s_abort, p.wait_limit, p.st)) {
-                  alive = false;
-                  break;
-                }
-                tc_fence_after();
-                const uint32_t a_addr = tiles_addr + stage * stage_bytes;
-                const uint64_t a_desc = umma_desc(a_addr), b_desc = umma_desc(a_addr + kABytes);
+            const uint32_t st_addr = tiles_addr + stage * stage_bytes;
+            const int nkb = min(kbox, kblocks - box * kbox);
+            for (int kbi = 0; kbi < nkb; ++kbi) {
+              const uint64_t a_desc = umma_desc(st_addr + (uint32_t)kbi * a_bytes);
+              const uint64_t b_desc = umma_desc(st_addr + (uint32_t)kbox * a_bytes + (uint32_t)kbi * w_bytes);
 #pragma unroll
-                for (int k = 0; k < kKBlock / 16; ++k)   // UMMA K = 16 bf16 = 32 bytes = 2 descriptor units
-                  umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, !(first && k == 0));
-                first = false;
-                umma_commit(empty_bar(stage));           // frees the smem stage when these MMAs retire
-              }
-              phase_bits ^= 1u << stage;
-              if (++stage == n_stages) stage = 0;
+              for (int k = 0; k < kKBlock / 16; ++k)   // UMMA K = 16 bf16 = 32 bytes = 2 descriptor units
+                umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, !(first && k == 0));
+              first = false;
             }
-            if (alive) umma_commit(tfull_bar(acc));      // this issuer's partial accumulator is complete
+            umma_commit(empty_bar(stage));             // frees the stage when these MMAs retire
+            phase_bits ^= 1u << stage;
+            if (++stage == n_stages) stage = 0;
           }
+          if (alive) umma_commit(tfull_bar(acc));      // the accumulator is complete
         }
         ++acc_iter;
-      } else {
+      } else if (warp != 11) {
         // ---------------- epilogue: drain tensor memory, finish the cell ----------------
         // Two sets of four warps; set e takes hidden units [4e, 4e + 4) of every unit group.  A
         // warp may only read the tensor-memory lanes of quadrant (warp id mod 4).
@@ -282,7 +280,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
         const int quad = warp & 3;
         const int r = quad * 32 + lane;
         const int row = row0 + r;
-        const bool valid = row < end;
+        const bool valid = row < row_end;
         const int node = valid ? p.order[row] : 0;
         const int slot = valid ? p.slot[node] : -1;   // 2 * pos(caller) + side, -1 for a root
         // stage the children's cell states of this thread's row while the MMAs run
@@ -316,7 +314,7 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
           tc_fence_after();
           const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(quad * 32) << 16) + 4u * e;
           // the tensor-memory loads of group g + 1 are in flight while group g is computed
-          uint32_t vbuf[2][20], v2[20];
+          uint32_t vbuf[2][20];
           auto load_group = [&](int g, uint32_t* v) {
             const uint32_t col0 = (uint32_t)(g * gcols);
             if (leaf) {
@@ -327,16 +325,6 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
               for (int q = 0; q < 5; ++q) tmem_ld4(taddr + col0 + 8 * q, v + 4 * q);
             }
           };
-          auto add_second = [&](int g, uint32_t* v) {   // thin tiles: add the second issuer's partial sums
-            const uint32_t col0 = (uint32_t)kAcc2Off + (uint32_t)(g * gcols);
-#pragma unroll
-            for (int q = 0; q < 5; ++q)
-              if (q < ngates) tmem_ld4(taddr + col0 + 8 * q, v2 + 4 * q);
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 20; ++j)
-              if (j < 4 * ngates) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
-          };
           load_group(0, vbuf[0]);
 #pragma unroll
           for (int g = 0; g < kMaxG; ++g) {
@@ -346,7 +334,6 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
 #pragma unroll
             for (int q = 0; q < 5; ++q) bcur[q] = bnext[q];
             tmem_ld_wait();
-            if (dual) add_second(g, v);
             if (g + 1 < G) {
               load_group(g + 1, vbuf[(g + 1) & 1]);
 #pragma unroll
@@ -430,9 +417,9 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
             bool ok = mbar_wait(epi_bar, epi_phase, s_abort, p.wait_limit, p.st);
             epi_phase ^= 1;
             if (ok) {
-              const int et = e * BM + r, cpr = 2 * G;           // 16-byte chunks (4 units) per row
+              const int et = e * BM + r, cpr = 2 * G;           // 16-byte chunks (4 units) per row, a power of two
               for (int idx = et; idx < BM * cpr; idx += 2 * BM) {
-                const int ro = idx / cpr, ch = idx % cpr;
+                const int ro = idx >> (plan.lg + 1), ch = idx & (cpr - 1);
                 const int node_o = s_rownode[ro];
                 if (node_o < 0) continue;
                 const unsigned char* src = cstage_w + ro * 256;
@@ -468,8 +455,9 @@ k_fwd_tc(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CU
       // loop is left by all of them together.
       __syncthreads();
       if (*s_abort) break;
-      ++barriers_passed;
-      if (!grid_barrier(p.st, barriers_passed * gridDim.x, p.wait_limit, s_flag)) break;
+      // only the CTAs that had a tile in this wavefront wrote anything: they arrive, the rest just wait
+      arrivals += (uint32_t)min(tiles, (int)gridDim.x);
+      if (!grid_barrier(p.st, arrivals, p.wait_limit, s_flag, (int)blockIdx.x < tiles)) break;
     }
   }
 
@@ -557,7 +545,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-int make_tmap(treelstm* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows) {
+int make_tmap(treelstm* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows,
+              uint32_t box_kb) {
   static EncodeTiledFn encode = nullptr;
   if (!encode) {
     void* fn = nullptr;
@@ -566,11 +555,12 @@ int make_tmap(treelstm* ctx, CUtensorMap* map, const void* base, uint64_t inner,
     if (!fn || q != cudaDriverEntryPointSuccess) return TREELSTM_ERR_CUDA;
     encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
-  const cuuint64_t dims[2] = {inner, rows};
-  const cuuint64_t strides[1] = {inner * 2};           // bytes between rows
-  const cuuint32_t box[2] = {kKBlock, box_rows};       // 64 bf16 = one 128-byte swizzle span
-  const cuuint32_t elem[2] = {1, 1};
-  CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+  // element (k, row, kb) of the view lives at base + kb * 128 + row * pitch + k * 2 bytes
+  const cuuint64_t dims[3] = {kKBlock, rows, inner / kKBlock};
+  const cuuint64_t strides[2] = {inner * 2, kKBlock * 2};   // bytes between rows, between K blocks
+  const cuuint32_t box[3] = {kKBlock, box_rows, box_kb};    // 64 bf16 = one 128-byte swizzle span
+  const cuuint32_t elem[3] = {1, 1, 1};
+  CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem,
                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { ctx->cuda_error = (int)r; return TREELSTM_ERR_CUDA; }
@@ -580,14 +570,16 @@ int make_tmap(treelstm* ctx, CUtensorMap* map, const void* base, uint64_t inner,
 int ensure_operand_tmaps(treelstm* ctx, void* ws, int n, const void* xin, const void* ain) {
   if (ctx->tmap_ws_base == ws && ctx->tmap_ws_rows == n) return TREELSTM_OK;
   // the dense operands live in the caller's workspace
-  int rc = make_tmap(ctx, &ctx->tmap_x, xin, (uint64_t)ctx->Ep, (uint64_t)n, BM);
-  if (rc != TREELSTM_OK) return rc;
-  rc = make_tmap(ctx, &ctx->tmap_a, ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, BM);
-  if (rc != TREELSTM_OK) return rc;
-  rc = make_tmap(ctx, &ctx->tmap_a64, ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, 64);
-  if (rc != TREELSTM_OK) return rc;
-  rc = make_tmap(ctx, &ctx->tmap_a32, ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, 32);
-  if (rc != TREELSTM_OK) return rc;
+  const uint32_t kb_leaf = ctx->Ep / kKBlock, kb_int = 2 * ctx->Hp / kKBlock;
+  for (int sel = 0; sel < 2; ++sel) {
+    int rc = make_tmap(ctx, &ctx->maps.x[sel], xin, (uint64_t)ctx->Ep, (uint64_t)n, BM, sel == 0 ? kb_leaf : 2u);
+    if (rc != TREELSTM_OK) return rc;
+    for (int i = 0; i < 3; ++i) {
+      rc = make_tmap(ctx, &ctx->maps.a[i][sel], ain, 2 * (uint64_t)ctx->Hp, (uint64_t)n, 32u << i,
+                     sel == 0 ? kb_int : 2u);
+      if (rc != TREELSTM_OK) return rc;
+    }
+  }
   ctx->tmap_ws_base = ws;
   ctx->tmap_ws_rows = n;
   return TREELSTM_OK;
@@ -607,10 +599,18 @@ int pack_weights_bf16(treelstm* ctx, cudaStream_t stream) {
   k_pack_embedding<<<1024, 256, 0, stream>>>(ctx->vocab, ctx->E, ctx->Ep, ctx->emb, ctx->emb_bf);
   TL_CUDA(ctx, cudaGetLastError());
   const int groups = ctx->Hp / kUnitGroup;
-  int rc = make_tmap(ctx, &ctx->tmap_wh, ctx->Wp_h, 2 * (uint64_t)ctx->Hp, (uint64_t)groups * kGColsI, kGColsI);
-  if (rc != TREELSTM_OK) return rc;
-  rc = make_tmap(ctx, &ctx->tmap_wx, ctx->Wp_x, (uint64_t)ctx->Ep, (uint64_t)groups * kGColsL, kGColsL);
-  if (rc != TREELSTM_OK) return rc;
+  const uint32_t kb_leaf = ctx->Ep / kKBlock, kb_int = 2 * ctx->Hp / kKBlock;
+  if (kb_leaf > 256 || kb_int > 256) return TREELSTM_ERR_UNSUPPORTED;   // a box dimension holds at most 256
+  for (int sel = 0; sel < 2; ++sel)
+    for (int lg = 0; lg < 3; ++lg) {
+      // groups the number of unit groups does not divide into are never chosen; their maps stay valid anyway
+      int rc = make_tmap(ctx, &ctx->maps.wh[lg][sel], ctx->Wp_h, 2 * (uint64_t)ctx->Hp, (uint64_t)groups * kGColsI,
+                         (uint32_t)kGColsI << lg, sel == 0 ? kb_int : 2u);
+      if (rc != TREELSTM_OK) return rc;
+      rc = make_tmap(ctx, &ctx->maps.wx[lg][sel], ctx->Wp_x, (uint64_t)ctx->Ep, (uint64_t)groups * kGColsL,
+                     (uint32_t)kGColsL << lg, sel == 0 ? kb_leaf : 2u);
+      if (rc != TREELSTM_OK) return rc;
+    }
   ctx->tmap_ws_base = nullptr;
   ctx->have_tmaps = true;
   return TREELSTM_OK;
@@ -652,11 +652,11 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   const int groups = ctx->Hp / kUnitGroup;
   if (flags & TREELSTM_PERSISTENT) {
     int grid = ctx->sm_count;                       // one CTA per SM (shared and tensor memory)
-    const int want = ((n + BM - 1) / BM + 1) * groups;   // never more CTAs than the thinnest tiling has tiles
+    const int want = ((n + 31) / 32 + 1) * groups;       // never more CTAs than the thinnest tiling has tiles
     if (grid > want) grid = want;
     if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
     int only = -1;
-    void* args[] = {&ctx->tmap_wh, &ctx->tmap_wx, &ctx->tmap_x, &ctx->tmap_a, &ctx->tmap_a64, &ctx->tmap_a32, &p, &only};
+    void* args[] = {&ctx->maps, &p, &only};
     TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc, dim3(grid), dim3(kThreads), args,
                                              kSmemBytes, stream));
     ctx->launches += 1;
@@ -671,9 +671,9 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   for (int lvl = 0; lvl < n_levels_host; ++lvl) {
     const int w = level_offset_host[lvl + 1] - level_offset_host[lvl];
     if (w <= 0) continue;
-    const int tiles = ((w + BM - 1) / BM) * (groups / choose_groups_per_tile(w, groups, p.sched_ctas));
-    k_fwd_tc<<<tiles, kThreads, kSmemBytes, stream>>>(ctx->tmap_wh, ctx->tmap_wx, ctx->tmap_x, ctx->tmap_a, ctx->tmap_a64,
-                                                      ctx->tmap_a32, p, lvl);
+    const int tiles = choose_tile_plan(w, groups, p.sched_ctas, lvl == 0,
+                                       lvl == 0 ? ctx->Ep / kKBlock : 2 * ctx->Hp / kKBlock).tiles;
+    k_fwd_tc<<<tiles, kThreads, kSmemBytes, stream>>>(ctx->maps, p, lvl);
     ctx->launches += 1;
   }
   TL_CUDA(ctx, cudaGetLastError());

@@ -18,8 +18,7 @@
 //
 // Warp roles as in gemm_tc.cu (384 threads): warps 0-3 and 6-9 epilogue, warp 4 TMA producer of the
 // operand rows, warp 10 TMA producer of the W_x tiles of the leaf wavefront (and of the resident
-// W_h slice), warps 5 and 11 MMA issuers (both on single-tile wavefronts, alternate K blocks into
-// two partial accumulators).
+// W_h slice), warp 5 MMA issuer; warp 11 only joins the barriers.
 #include "tc_ptx.cuh"
 
 namespace tl {
@@ -68,10 +67,7 @@ __device__ __forceinline__ void cluster_sync_all() {
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_constant__ CUtensorMap tmap_wx,
-                   const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_a,
-                   const __grid_constant__ CUtensorMap tmap_a64, const __grid_constant__ CUtensorMap tmap_a32,
-                   TcParams p) {
+k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTmapSet sfm, TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   const int G = p.groups_per_cta;
   const SfLayout L = sf_layout(p.Hp, G);
@@ -112,14 +108,14 @@ k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_con
 
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 2); mbar_init(tempty_bar(a), 256); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
     mbar_init(epi_bar, 256);
     mbar_init(wres_bar, 1);
     *s_abort = 0;
     *s_nlev = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // 2 stages x 256 columns; partial sums at +128
+  if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // 2 accumulator stages x 256 columns
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -130,14 +126,11 @@ k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_con
   const bool vec = (H % 4) == 0;
   const int nt = rank;                               // this CTA's slice of the hidden units
 
-  // The slice of the packed recurrent weights this CTA keeps: K block kb, unit group g at
-  // wres + (kb * G + g) * 5120 bytes (40 rows of 128 bytes, 128-byte swizzle).
+  // The slice of the packed recurrent weights this CTA keeps, fetched by one request: K block kb of
+  // its 40 G packed rows at wres + kb * G * 5120 bytes (rows of 128 bytes, 128-byte swizzle).
   if (warp == 10 && lane == 0) {
     mbar_arrive_expect_tx(wres_bar, L.wres_bytes);
-    for (int kb = 0; kb < kb_int; ++kb)
-      for (int g = 0; g < G; ++g)
-        tma_load_2d(wres_addr + (uint32_t)(kb * G + g) * (kGColsI * 128u), &tmap_wh, kb * kKBlock,
-                    (nt * G + g) * kGColsI, wres_bar);
+    tma_load_3d(wres_addr, &sfm.wres, 0, nt * G * kGColsI, 0, wres_bar);
   }
 
   // Wavefront boundaries of the sub-forest: its nodes are sorted by level, the levels are 0 .. top
@@ -162,14 +155,7 @@ k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_con
   {
     const int gtid = rank * kThreads + tid, gthreads = cs * kThreads;
     const int lend = loff(1);
-    const int cpr = p.Ep / 8;                              // 16-byte chunks per row
-    const long long total = (long long)(lend - pbeg) * cpr;
-    for (long long ch = gtid; ch < total; ch += gthreads) {
-      const int row = pbeg + (int)(ch / cpr), cc = (int)(ch % cpr);
-      const int tok = p.token[p.order[row]];
-      const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.emb_bf + (size_t)tok * p.Ep) + cc);
-      reinterpret_cast<uint4*>(p.xin + (size_t)row * p.Ep)[cc] = v;
-    }
+    gather_leaf_rows(p, pbeg, lend, gtid >> 5, gthreads >> 5, lane);
     for (int pos = lend + gtid; pos < pend; pos += gthreads) {
       const int node = p.order[pos];
       p.slot[p.left[node]] = 2 * pos;
@@ -189,56 +175,47 @@ k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_con
     if (!stop) {
       const int begin = loff(lvl), end = loff(lvl + 1);
       const bool leaf = lvl == 0;
-      const int tiles = (end - begin + BM - 1) / BM;
+      const int rows = end - begin;
+      const int tiles = (rows + BM - 1) / BM;
       const int kblocks = leaf ? kb_leaf : kb_int;
       const int gcols = leaf ? kGColsL : kGColsI;
       const int ncols = G * gcols;                     // accumulator columns in use
       const int ncols_mma = (ncols + 15) & ~15;        // UMMA N (columns past ncols are never read)
-      const bool dual = ncols_mma <= kAcc2Off && kblocks >= 2 && tiles == 1;
-      const uint32_t stage_bytes = leaf ? (uint32_t)kABytes + (uint32_t)ncols * 128u : (uint32_t)kABytes;
-      const uint32_t n_stages = min((uint32_t)kMaxStages, L.ring_bytes / stage_bytes);
+      // A wavefront of at most 64 (32) nodes fetches only that many operand rows; the MMA still
+      // spans 128 rows, what lies behind the fetched rows feeds accumulator rows that are not stored.
+      const int lrt = leaf || rows > 64 ? 7 : (rows > 32 ? 6 : 5);
+      const uint32_t a_bytes = 128u << lrt;                         // operand rows of one K block
+      const uint32_t w_bytes = leaf ? (uint32_t)ncols * 128u : 0u;  // leaf: W_x rows ride along; W_h is resident
+      // A stage of the ring holds one box: kbox K blocks of operand rows (+ kbox K blocks of W_x rows).
+      // A single-tile wavefront takes its operands in one request when they fit, anything else in
+      // boxes of two K blocks so that loads, MMAs and epilogues of consecutive tiles overlap.
+      const int sel = tiles == 1 && (uint32_t)kblocks * (a_bytes + w_bytes) <= L.ring_bytes ? 0 : 1;
+      const int kbox = sel == 0 ? kblocks : 2;
+      const int n_box = sel == 0 ? 1 : (kblocks + 1) >> 1;
+      const uint32_t stage_bytes = (uint32_t)kbox * (a_bytes + w_bytes);
+      uint32_t n_stages = kMaxStages;
+      while (n_stages * stage_bytes > L.ring_bytes) --n_stages;
       stage = 0;
-      const int a_rows = leaf || end - begin > 64 ? BM : (end - begin > 32 ? 64 : 32);
-      if (warp == 4 || warp == 10) asm volatile("fence.proxy.async.global;" ::: "memory");   // TMA reads after the barrier's acquire
 
       for (int t = 0; t < tiles && alive; ++t) {
         const int row0 = begin + t * BM;
 
         if (warp == 4 || (warp == 10 && leaf)) {
-          // ---------------- operand producers (TMA) ----------------
-          const bool is_a = warp == 4;
-          const CUtensorMap* map = is_a ? (leaf ? &tmap_x : (a_rows == BM ? &tmap_a : (a_rows == 64 ? &tmap_a64 : &tmap_a32)))
-                                        : &tmap_wx;
-          const uint32_t bytes = is_a ? (uint32_t)a_rows * 128u : (uint32_t)ncols * 128u;
-          auto issue = [&](int kb, uint32_t st_idx) {
-            const uint32_t sa = ring_addr + st_idx * stage_bytes;
-            mbar_arrive_expect_tx(full_bar(st_idx), bytes);
-            if (is_a) {
-              tma_load_2d(sa, map, kb * kKBlock, row0, full_bar(st_idx));
-              if (!leaf) mbar_arrive(full_bar(st_idx));   // stands in for the W producer: W_h is resident
-            } else {
-              for (int g = 0; g < G; ++g)
-                tma_load_2d(sa + kABytes + (uint32_t)(g * gcols) * 128u, map, kb * kKBlock,
-                            (nt * G + g) * gcols, full_bar(st_idx));
-            }
-          };
-          int kb_first = 0;
-          if (t == 0) {
-            // first tile of a wavefront: the ring is empty, the first n_stages K blocks need no wait
-            const int burst = min(kblocks, (int)n_stages);
-            if (lane < burst) issue(lane, (uint32_t)lane);
-            __syncwarp();
-            phase_bits ^= (1u << burst) - 1u;
-            stage = (uint32_t)burst == n_stages ? 0u : (uint32_t)burst;
-            kb_first = burst;
-          }
+          // ---------------- operand producers (TMA): one request per box and operand ----------------
           if (lane == 0) {
-            for (int kb = kb_first; kb < kblocks; ++kb) {
+            const bool is_a = warp == 4;
+            const CUtensorMap* map = is_a ? (leaf ? &maps.x[sel] : &maps.a[lrt - 5][sel]) : &sfm.wx[sel];
+            const uint32_t bytes = (uint32_t)kbox * (is_a ? a_bytes : w_bytes);
+            const uint32_t off = is_a ? 0u : (uint32_t)kbox * a_bytes;
+            const int y = is_a ? row0 : nt * ncols;
+            for (int box = 0; box < n_box; ++box) {
               if (!mbar_wait(empty_bar(stage), ((phase_bits >> stage) & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) {
                 alive = false;
                 break;
               }
-              issue(kb, stage);
+              mbar_arrive_expect_tx(full_bar(stage), bytes);
+              tma_load_3d(ring_addr + stage * stage_bytes + off, map, 0, y, box * kbox, full_bar(stage));
+              if (is_a && !leaf) mbar_arrive(full_bar(stage));   // stands in for the W producer: W_h is resident
               phase_bits ^= 1u << stage;
               if (++stage == n_stages) stage = 0;
             }
@@ -247,52 +224,44 @@ k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_con
           stage = __shfl_sync(kFullMask, stage, 0);
           phase_bits = __shfl_sync(kFullMask, phase_bits, 0);
           alive = __shfl_sync(kFullMask, (int)alive, 0) != 0;
-        } else if (warp == 5 || warp == 11) {
-          // ---------------- MMA issuers ----------------
+        } else if (warp == 5) {
+          // ---------------- MMA issuer ----------------
           if (lane == 0) {
-            const int w = warp == 5 ? 0 : 1;
             const uint32_t acc = acc_iter & 1, acc_phase = (acc_iter >> 1) & 1;
-            if (!dual && w == 1) {
-              if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
-              mbar_arrive(tfull_bar(acc));
-              for (int kb = 0; kb < kblocks; ++kb) {
-                phase_bits ^= 1u << stage;
-                if (++stage == n_stages) stage = 0;
-              }
-            } else {
-              if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
-              if (!leaf && !wres_ready) {
-                if (!mbar_wait(wres_bar, 0, s_abort, p.wait_limit, p.st)) alive = false;
-                wres_ready = true;
+            if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, s_abort, p.wait_limit, p.st)) alive = false;
+            if (!leaf && !wres_ready) {
+              if (!mbar_wait(wres_bar, 0, s_abort, p.wait_limit, p.st)) alive = false;
+              wres_ready = true;
+            }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * kAccCols;
+            const uint32_t idesc = umma_idesc(ncols_mma);
+            bool first = true;
+            for (int box = 0; box < n_box && alive; ++box) {
+              if (!mbar_wait(full_bar(stage), (phase_bits >> stage) & 1u, s_abort, p.wait_limit, p.st)) {
+                alive = false;
+                break;
               }
               tc_fence_after();
-              const uint32_t d_tmem = tmem_base + acc * kAccCols + (w == 1 ? (uint32_t)kAcc2Off : 0u);
-              const uint32_t idesc = umma_idesc(ncols_mma);
-              bool first = true;
-              for (int kb = 0; kb < kblocks && alive; ++kb) {
-                if (!dual || (kb & 1) == w) {
-                  if (!mbar_wait(full_bar(stage), (phase_bits >> stage) & 1u, s_abort, p.wait_limit, p.st)) {
-                    alive = false;
-                    break;
-                  }
-                  tc_fence_after();
-                  const uint32_t a_addr = ring_addr + stage * stage_bytes;
-                  const uint32_t b_addr = leaf ? a_addr + kABytes : wres_addr + (uint32_t)kb * (uint32_t)ncols * 128u;
-                  const uint64_t a_desc = umma_desc(a_addr), b_desc = umma_desc(b_addr);
+              const uint32_t st_addr = ring_addr + stage * stage_bytes;
+              const int nkb = min(kbox, kblocks - box * kbox);
+              for (int kbi = 0; kbi < nkb; ++kbi) {
+                const uint32_t b_addr = leaf ? st_addr + (uint32_t)kbox * a_bytes + (uint32_t)kbi * w_bytes
+                                             : wres_addr + (uint32_t)(box * kbox + kbi) * (uint32_t)ncols * 128u;
+                const uint64_t a_desc = umma_desc(st_addr + (uint32_t)kbi * a_bytes), b_desc = umma_desc(b_addr);
 #pragma unroll
-                  for (int k = 0; k < kKBlock / 16; ++k)   // UMMA K = 16 bf16 = 32 bytes = 2 descriptor units
-                    umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, !(first && k == 0));
-                  first = false;
-                  umma_commit(empty_bar(stage));           // frees the ring stage when these MMAs retire
-                }
-                phase_bits ^= 1u << stage;
-                if (++stage == n_stages) stage = 0;
+                for (int k = 0; k < kKBlock / 16; ++k)   // UMMA K = 16 bf16 = 32 bytes = 2 descriptor units
+                  umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, !(first && k == 0));
+                first = false;
               }
-              if (alive) umma_commit(tfull_bar(acc));      // this issuer's partial accumulator is complete
+              umma_commit(empty_bar(stage));             // frees the ring stage when these MMAs retire
+              phase_bits ^= 1u << stage;
+              if (++stage == n_stages) stage = 0;
             }
+            if (alive) umma_commit(tfull_bar(acc));      // the accumulator is complete
           }
           ++acc_iter;
-        } else if (warp != 10) {
+        } else if (warp != 10 && warp != 11) {
           // ---------------- epilogue: drain tensor memory, finish the cell ----------------
           const int e = warp < 4 ? 0 : 1;   // warps 0-3: units [0,4) of every group, warps 6-9: [4,8)
           const int quad = warp & 3;        // tensor-memory lane quadrant this warp may read
@@ -330,7 +299,7 @@ k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_con
           if (alive) {
             tc_fence_after();
             const uint32_t taddr = tmem_base + acc * kAccCols + ((uint32_t)(quad * 32) << 16) + 4u * e;
-            uint32_t vbuf[2][20], v2[20];
+            uint32_t vbuf[2][20];
             auto load_group = [&](int g, uint32_t* v) {
               const uint32_t col0 = (uint32_t)(g * gcols);
               if (leaf) {
@@ -341,16 +310,6 @@ k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_con
                 for (int q = 0; q < 5; ++q) tmem_ld4(taddr + col0 + 8 * q, v + 4 * q);
               }
             };
-            auto add_second = [&](int g, uint32_t* v) {   // single-tile wavefronts: add the second issuer's partial sums
-              const uint32_t col0 = (uint32_t)kAcc2Off + (uint32_t)(g * gcols);
-#pragma unroll
-              for (int q = 0; q < 5; ++q)
-                if (q < ngates) tmem_ld4(taddr + col0 + 8 * q, v2 + 4 * q);
-              tmem_ld_wait();
-#pragma unroll
-              for (int j = 0; j < 20; ++j)
-                if (j < 4 * ngates) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
-            };
             load_group(0, vbuf[0]);
 #pragma unroll
             for (int g = 0; g < kMaxG; ++g) {
@@ -360,7 +319,6 @@ k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_con
 #pragma unroll
               for (int q = 0; q < 5; ++q) bcur[q] = bnext[q];
               tmem_ld_wait();
-              if (dual) add_second(g, v);
               if (g + 1 < G) {
                 load_group(g + 1, vbuf[(g + 1) & 1]);
 #pragma unroll
@@ -444,8 +402,9 @@ k_fwd_tc_subforest(const __grid_constant__ CUtensorMap tmap_wh, const __grid_con
               epi_phase ^= 1;
               if (ok) {
                 const int et = e * BM + r, cpr = 2 * G;           // 16-byte chunks (4 units) per row
+                const int lcpr = G == 1 ? 1 : (G == 2 ? 2 : -1);   // shift instead of a division where 2 G is a power of two
                 for (int idx = et; idx < BM * cpr; idx += 2 * BM) {
-                  const int ro = idx / cpr, ch = idx % cpr;
+                  const int ro = lcpr > 0 ? idx >> lcpr : idx / cpr, ch = idx - ro * cpr;
                   const int node_o = s_rownode[ro];
                   if (node_o < 0) continue;
                   const unsigned char* src = cstage_ptr + ((size_t)ro << L.crow_shift);
@@ -527,6 +486,14 @@ SubforestPlan subforest_plan(treelstm* ctx) {
     cudaGetLastError();
     return pl;
   }
+  const uint32_t kb_leaf = ctx->Ep / kKBlock, kb_int = 2 * ctx->Hp / kKBlock;
+  if (make_tmap(ctx, &ctx->sf_maps.wres, ctx->Wp_h, 2 * (uint64_t)ctx->Hp, (uint64_t)groups * kGColsI,
+                (uint32_t)(gpc * kGColsI), kb_int) != TREELSTM_OK ||
+      make_tmap(ctx, &ctx->sf_maps.wx[0], ctx->Wp_x, (uint64_t)ctx->Ep, (uint64_t)groups * kGColsL,
+                (uint32_t)(gpc * kGColsL), kb_leaf) != TREELSTM_OK ||
+      make_tmap(ctx, &ctx->sf_maps.wx[1], ctx->Wp_x, (uint64_t)ctx->Ep, (uint64_t)groups * kGColsL,
+                (uint32_t)(gpc * kGColsL), 2u) != TREELSTM_OK)
+    return pl;
   pl.ok = true;
   pl.cluster_size = cs;
   pl.groups_per_cta = gpc;
@@ -573,8 +540,7 @@ int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, con
   cfg.dynamicSmemBytes = ctx->sf.smem_bytes;
   cfg.stream = stream;
   cfg.attrs = at; cfg.numAttrs = 1;
-  TL_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_fwd_tc_subforest, ctx->tmap_wh, ctx->tmap_wx, ctx->tmap_x, ctx->tmap_a,
-                                  ctx->tmap_a64, ctx->tmap_a32, p));
+  TL_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_fwd_tc_subforest, ctx->maps, ctx->sf_maps, p));
   ctx->launches += 1;
   return TREELSTM_OK;
 }

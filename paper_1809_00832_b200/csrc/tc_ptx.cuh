@@ -80,6 +80,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+// One request for a box of {64 elements, rows, K blocks}: a request costs the TMA unit of an SM
+// about 180 cycles whatever its size and requests are served one after the other, so a tile's
+// operands are fetched with as few requests as possible.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -142,10 +150,44 @@ __device__ __forceinline__ void st_row4(float* p, bool vec, int count, const flo
   }
 }
 
-#ifndef TL_TC_PTX_NO_HOST
-// Tiled tensor map over a row-major bf16 matrix [rows][inner], boxes of 64 x box_rows elements with
-// the 128-byte swizzle (gemm_tc.cu).
-int make_tmap(treelstm* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows);
-#endif
+// Xin[row] = emb_bf[token of the leaf at ready position row] for rows [row_begin, row_end), spread over
+// n_warps warps.  A warp takes four rows at a time: their order and token entries are fetched side by
+// side, then every lane copies 16-byte pieces of the four embedding rows with all its loads in
+// flight before the first store - the copy is bound by memory latency, not by bandwidth.
+__device__ __forceinline__ void gather_leaf_rows(const TcParams& p, int row_begin, int row_end, int gwarp, int n_warps,
+                                                 int lane) {
+  const int cpr = p.Ep / 8;                              // 16-byte chunks per row
+  for (int base = row_begin + gwarp; base < row_end; base += 4 * n_warps) {
+    const int my_row = base + (lane & 3) * n_warps;
+    const int my_tok = my_row < row_end ? p.token[p.order[my_row]] : 0;
+    int tok[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) tok[k] = __shfl_sync(kFullMask, my_tok, k);
+    for (int c0 = 0; c0 < cpr; c0 += 64) {
+      uint4 v[4][2];
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int cc = c0 + h * 32 + lane;
+          if (base + k * n_warps < row_end && cc < cpr)
+            v[k][h] = __ldg(reinterpret_cast<const uint4*>(p.emb_bf + (size_t)tok[k] * p.Ep) + cc);
+        }
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int cc = c0 + h * 32 + lane;
+          if (base + k * n_warps < row_end && cc < cpr)
+            reinterpret_cast<uint4*>(p.xin + (size_t)(base + k * n_warps) * p.Ep)[cc] = v[k][h];
+        }
+    }
+  }
+}
+
+// Tiled tensor map over a row-major bf16 matrix [rows][inner] seen as {64, rows, inner / 64}: boxes of
+// 64 elements x box_rows rows x box_kb K blocks with the 128-byte swizzle (gemm_tc.cu).
+int make_tmap(treelstm* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows,
+              uint32_t box_kb);
 
 }  // namespace tl
