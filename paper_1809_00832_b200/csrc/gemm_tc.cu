@@ -206,6 +206,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     const uint32_t n_stages = (uint32_t)plan.n_stages;
     const int kbox = plan.kbox, n_box = plan.n_box;
     stage = 0;
+    int nx_node = 0, nx_slot = -1;                  // epilogue: row data of this CTA's next tile, fetched a tile ahead
+    bool nx_have = false;
 
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
       const int rtile = t / ntn, nt = t - rtile * ntn;
@@ -281,8 +283,22 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
         const int r = quad * 32 + lane;
         const int row = row0 + r;
         const bool valid = row < row_end;
-        const int node = valid ? p.order[row] : 0;
-        const int slot = valid ? p.slot[node] : -1;   // 2 * pos(caller) + side, -1 for a root
+        int node, slot;                               // slot: 2 * pos(caller) + side, -1 for a root
+        if (nx_have) {
+          node = nx_node; slot = nx_slot;
+        } else {
+          node = valid ? p.order[row] : 0;
+          slot = valid ? p.slot[node] : -1;
+        }
+        // the same two dependent loads for this CTA's next tile go out now and land while this tile is computed
+        const int t2 = t + (int)gridDim.x;
+        nx_have = t2 < tiles;
+        bool valid2 = false;
+        if (nx_have) {
+          const int rtile2 = t2 / ntn, row2 = begin + (rtile2 << plan.lrt) + r;
+          valid2 = r < rt && row2 < end;
+          nx_node = valid2 ? p.order[row2] : 0;
+        }
         // stage the children's cell states of this thread's row while the MMAs run
         const float* crow = p.cin + (size_t)row * 2 * H;   // [c_l | c_r] of the node at this position
         const bool staged = !leaf && vec && (nt + 1) * G * 8 <= H;
@@ -409,6 +425,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
               }
             }
           }
+          if (nx_have) nx_slot = valid2 ? p.slot[nx_node] : -1;
           tc_fence_before();
           mbar_arrive(tempty_bar(acc));              // accumulator stage may be overwritten
           if (staged_out) {
@@ -443,12 +460,12 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
             epi_phase ^= 1;
             if (!ok) alive = false;
           }
-          // the operand rows written above are read through TMA (async proxy) by later wavefronts
-          asm volatile("fence.proxy.async.global;" ::: "memory");
         }
         ++acc_iter;
       }
     }
+    // the operand rows the epilogue wrote are read through TMA (async proxy) by later wavefronts
+    if (warp < 4 || (warp >= 6 && warp < 10)) asm volatile("fence.proxy.async.global;" ::: "memory");
     if (only_level < 0 && lvl + 1 < lvl_end) {
       // every role of every CTA joins the barrier.  A role that gave up has set s_abort before
       // this point, so the flag read after the CTA barrier is the same for all threads and the

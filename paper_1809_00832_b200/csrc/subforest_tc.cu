@@ -196,6 +196,8 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
       uint32_t n_stages = kMaxStages;
       while (n_stages * stage_bytes > L.ring_bytes) --n_stages;
       stage = 0;
+      int nx_node = 0, nx_slot = -1;                // epilogue: row data of the next tile, fetched a tile ahead
+      bool nx_have = false;
 
       for (int t = 0; t < tiles && alive; ++t) {
         const int row0 = begin + t * BM;
@@ -268,8 +270,17 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
           const int r = quad * 32 + lane;
           const int row = row0 + r;
           const bool valid = row < end;
-          const int node = valid ? p.order[row] : 0;
-          const int slot = valid ? p.slot[node] : -1;   // 2 * pos(caller) + side, -1 for a root
+          int node, slot;                               // slot: 2 * pos(caller) + side, -1 for a root
+          if (nx_have) {
+            node = nx_node; slot = nx_slot;
+          } else {
+            node = valid ? p.order[row] : 0;
+            slot = valid ? p.slot[node] : -1;
+          }
+          // the same two dependent loads for the next tile go out now and land while this tile is computed
+          nx_have = t + 1 < tiles;
+          const bool valid2 = nx_have && row + BM < end;
+          if (nx_have) nx_node = valid2 ? p.order[row + BM] : 0;
           const float* crow = p.cin + (size_t)row * 2 * H;   // [c_l | c_r] of the node at this position
           const bool full_slice = vec && (nt + 1) * G * 8 <= H;   // no padded unit in this CTA's slice
           const bool staged = !leaf && full_slice;
@@ -392,6 +403,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
                 }
               }
             }
+            if (nx_have) nx_slot = valid2 ? p.slot[nx_node] : -1;
             tc_fence_before();
             mbar_arrive(tempty_bar(acc));              // accumulator stage may be overwritten
             if (staged_out) {
@@ -428,12 +440,12 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
               epi_phase ^= 1;
               if (!ok) alive = false;
             }
-            // the operand rows written above are read through TMA (async proxy) by later wavefronts
-            asm volatile("fence.proxy.async.global;" ::: "memory");
           }
           ++acc_iter;
         }
       }
+      // the operand rows the epilogue wrote are read through TMA (async proxy) by later wavefronts
+      if (warp < 4 || (warp >= 6 && warp < 10)) asm volatile("fence.proxy.async.global;" ::: "memory");
     }
     if (lvl + 1 < n_levels) {
       // Every thread of the cluster meets here.  A CTA in which a wait expired keeps coming to the
