@@ -184,15 +184,17 @@ def run_sweeps(args):
     model = binding.TreeLSTM(p.H, p.E, p.vocab, dev(p.emb), dev(p.W), dev(p.b), binding.BF16)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
 
+    flags = {"persistent": binding.PERSISTENT, "per_level": binding.PER_LEVEL, "subforests": binding.SUBFORESTS}[args.mode]
+
     def time_forest(forest, steps=100, warmup=5):
         left, right, token = dev(forest.left), dev(forest.right), dev(forest.token)
-        out = model.forward(left, right, token)
+        out = model.forward(left, right, token, flags=flags)
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
         for i in range(-warmup, steps):
             flush.fill_(i & 0xFF)
             if i >= 0:
                 ev[i][0].record()
-            model.forward(left, right, token, out=out, check=False)
+            model.forward(left, right, token, flags=flags, out=out, check=False)
             if i >= 0:
                 ev[i][1].record()
         torch.cuda.synchronize()
@@ -205,13 +207,13 @@ def run_sweeps(args):
             for batch in (1, 10, 25):
                 forest = fg.forest_from_shapes([make() for _ in range(batch)], rng, p.vocab)
                 ms, levels = time_forest(forest)
-                print(json.dumps({"sweep": "shape", "shape": name, "leaves_per_tree": 32, "batch": batch,
+                print(json.dumps({"sweep": "shape", "mode": args.mode, "shape": name, "leaves_per_tree": 32, "batch": batch,
                                   "levels": levels, "ms_per_step": ms, "trees_per_sec": batch / (ms * 1e-3)}))
     if args.sweep in ("length", "all"):
         for leaves in (2, 4, 8, 16, 24, 32, 40, 48, 56):
             forest = fg.forest_from_shapes([fg.random_split_shape(rng, leaves)], rng, p.vocab)
             ms, levels = time_forest(forest)
-            print(json.dumps({"sweep": "length", "leaves": leaves, "batch": 1, "levels": levels,
+            print(json.dumps({"sweep": "length", "mode": args.mode, "leaves": leaves, "batch": 1, "levels": levels,
                               "ms_per_instance": ms}))
     return 0
 

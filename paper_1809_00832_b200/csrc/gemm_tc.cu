@@ -43,30 +43,45 @@ static_assert(kBBytes % 1024 == 0 && (kGColsI * 128) % 1024 == 0 && (kGColsL * 1
 // Tile shape of a wavefront: rt ready nodes (32, 64 or 128; the MMA always spans 128 rows, the rest
 // of the accumulator is not stored) x g unit groups (1, 2 or 4).  Narrow wavefronts are cut into many
 // small tiles (every SM gets one, each fetches little), wide ones into fat tiles (fewer re-reads of
-// the operand rows).  Cost model, in units of one operand row: rounds x (fixed + rt + 40 g).
+// the operand rows).  Cost of a tile, fitted to clock64 traces and in units of 8 cycles: a fixed
+// part (operand latency, tensor-memory hand-over, output copy) + rt (operand bytes) + 180 g (the
+// epilogue's cell updates).  A wavefront that needs several rounds over the CTAs and whose last
+// round has few tiles splits those into 2 or 4 column pieces (tail_ls), so that the last round costs
+// a thin tile instead of a fat one.
 // The operands of a tile arrive in boxes of kbox K blocks (one TMA request per operand and box); a
 // box is one stage of the shared-memory ring: [kbox x rt operand rows | kbox x 40 g weight rows].
 struct TilePlan {
   int g, lg, rt, lrt, tiles;
+  int tail_from, tail_ls;                  // tiles from tail_from on are pieces of g >> tail_ls unit groups
   int sel, kbox, n_box, n_stages;          // sel 0: one box spans all K blocks, 1: boxes of two K blocks
-  uint32_t a_bytes, w_bytes, stage_bytes;  // operand rows / weight rows of one K block; one stage
+  uint32_t a_bytes, w_bytes, stage_bytes;  // operand rows / weight rows (of a fat tile) of one K block; one stage
 };
+__host__ __device__ inline int tile_cost(int rt, int lg) { return 350 + rt + (180 << lg); }
 __host__ __device__ inline TilePlan choose_tile_plan(int rows, int groups, int n_ctas, bool leaf, int kblocks) {
-  TilePlan best{1, 0, BM, 7, 0, 0, 0, 0, 0, 0u, 0u, 0u};
+  TilePlan best{1, 0, BM, 7, 0, 0, 0, 0, 0, 0, 0, 0u, 0u, 0u};
   int best_cost = 1 << 30, best_rounds = 1;
   for (int lrt = 7; lrt >= (leaf ? 7 : 5); --lrt) {      // leaf rows come through a 128-row box only
     const int rt = 1 << lrt;
     const int mt = (rows + rt - 1) >> lrt;
     for (int lg = 0; lg <= 2; ++lg) {
       if (groups & ((1 << lg) - 1)) break;                // g must divide the number of unit groups
-      const int tiles = mt * (groups >> lg);
+      const int fat = mt * (groups >> lg);
       int rounds = 1;
-      while (rounds * n_ctas < tiles) ++rounds;
-      const int cost = rounds * (256 + rt + (40 << lg));
+      while (rounds * n_ctas < fat) ++rounds;
+      const int rem = fat - (rounds - 1) * n_ctas;        // tiles of the last round
+      int ls = 0;
+      if (rounds > 1) {
+        ls = lg;
+        while (ls > 0 && (rem << ls) > n_ctas) --ls;
+      }
+      const int cost = (rounds - 1) * tile_cost(rt, lg) + tile_cost(rt, lg - ls);
       if (cost < best_cost || (cost == best_cost && lg > best.lg)) {
         best_cost = cost;
         best_rounds = rounds;
-        best.g = 1 << lg; best.lg = lg; best.rt = rt; best.lrt = lrt; best.tiles = tiles;
+        best.g = 1 << lg; best.lg = lg; best.rt = rt; best.lrt = lrt;
+        best.tail_from = ls > 0 ? fat - rem : fat;
+        best.tail_ls = ls;
+        best.tiles = ls > 0 ? fat - rem + (rem << ls) : fat;
       }
     }
   }
@@ -192,17 +207,15 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     const bool leaf = lvl == 0;
     const TilePlan plan = s_plan[lvl & 1];
     if (warp == 11 && lane == 0 && lvl + 1 < lvl_end) s_plan[(lvl + 1) & 1] = make_plan(lvl + 1);
-    const int G = plan.g, rt = plan.rt;
-    const int ntn = groups >> plan.lg;               // column tiles per row tile
+    const int rt = plan.rt;
+    const int ntn = groups >> plan.lg;               // fat column tiles per row tile
     const int tiles = plan.tiles;
     const int kblocks = leaf ? kb_leaf : kb_int;
     const int gcols = leaf ? kGColsL : kGColsI;
-    const int ncols = G * gcols;                     // accumulator columns in use
-    const int ncols_mma = (ncols + 15) & ~15;        // UMMA N (columns past ncols are never read)
     // A stage holds one box: kbox x rt operand rows, then kbox x ncols weight rows.  The MMA reads 128
     // rows from the start of a K block; what lies behind the rt fetched rows feeds accumulator rows
     // that are not stored.
-    const uint32_t a_bytes = plan.a_bytes, w_bytes = plan.w_bytes, stage_bytes = plan.stage_bytes;
+    const uint32_t a_bytes = plan.a_bytes, stage_bytes = plan.stage_bytes;
     const uint32_t n_stages = (uint32_t)plan.n_stages;
     const int kbox = plan.kbox, n_box = plan.n_box;
     stage = 0;
@@ -210,7 +223,20 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     bool nx_have = false;
 
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
-      const int rtile = t / ntn, nt = t - rtile * ntn;
+      // fat tile t = (row tile, column tile); a piece of the split last round is a column piece of a fat tile
+      int lg = plan.lg, fat = t, piece = 0;
+      if (t >= plan.tail_from) {
+        const int u = t - plan.tail_from;
+        fat = plan.tail_from + (u >> plan.tail_ls);
+        piece = u & ((1 << plan.tail_ls) - 1);
+        lg -= plan.tail_ls;
+      }
+      const int rtile = fat / ntn;
+      const int nt = ((fat - rtile * ntn) << (plan.lg - lg)) + piece;   // column tile in units of G groups
+      const int G = 1 << lg;
+      const int ncols = G * gcols;                     // accumulator columns in use
+      const int ncols_mma = (ncols + 15) & ~15;        // UMMA N (columns past ncols are never read)
+      const uint32_t w_bytes = (uint32_t)ncols * 128u; // weight rows of one K block
       const int row0 = begin + (rtile << plan.lrt);
       const int row_end = min(end, row0 + rt);        // rows of this tile: [row0, row_end)
 
@@ -223,7 +249,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
         if (lane == 0) {
           const bool is_a = warp == 4;
           const CUtensorMap* map = is_a ? (leaf ? &maps.x[plan.sel] : &maps.a[plan.lrt - 5][plan.sel])
-                                        : (leaf ? &maps.wx[plan.lg][plan.sel] : &maps.wh[plan.lg][plan.sel]);
+                                        : (leaf ? &maps.wx[lg][plan.sel] : &maps.wh[lg][plan.sel]);
           const uint32_t bytes = (uint32_t)kbox * (is_a ? a_bytes : w_bytes);
           const uint32_t off = is_a ? 0u : (uint32_t)kbox * a_bytes;
           const int y = is_a ? row0 : nt * ncols;
@@ -295,7 +321,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
         nx_have = t2 < tiles;
         bool valid2 = false;
         if (nx_have) {
-          const int rtile2 = t2 / ntn, row2 = begin + (rtile2 << plan.lrt) + r;
+          const int fat2 = t2 < plan.tail_from ? t2 : plan.tail_from + ((t2 - plan.tail_from) >> plan.tail_ls);
+          const int rtile2 = fat2 / ntn, row2 = begin + (rtile2 << plan.lrt) + r;
           valid2 = r < rt && row2 < end;
           nx_node = valid2 ? p.order[row2] : 0;
         }
@@ -305,7 +332,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
         // Outputs go through the same per-row staging area: each thread parks its 4-unit pieces of
         // c and h there, then all epilogue threads copy whole row segments out, several lanes per
         // row, so that a warp store covers a few full lines instead of 32 scattered 16-byte pieces.
-        const bool staged_out = vec && (nt + 1) * G * 8 <= H && p.gates == nullptr;
+        // (a tile of 32 or 64 rows writes so little that it stores straight from registers instead)
+        const bool staged_out = vec && (nt + 1) * G * 8 <= H && p.gates == nullptr && rt == BM;
         const uint32_t my_c = cstage_addr + (uint32_t)r * 256u;
         if (staged) {
           const float* sl = crow + nt * G * 8;
@@ -436,7 +464,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
             if (ok) {
               const int et = e * BM + r, cpr = 2 * G;           // 16-byte chunks (4 units) per row, a power of two
               for (int idx = et; idx < BM * cpr; idx += 2 * BM) {
-                const int ro = idx >> (plan.lg + 1), ch = idx & (cpr - 1);
+                const int ro = idx >> (lg + 1), ch = idx & (cpr - 1);
                 const int node_o = s_rownode[ro];
                 if (node_o < 0) continue;
                 const unsigned char* src = cstage_w + ro * 256;
