@@ -8,24 +8,22 @@
 // folding and charges with regrouping copies per depth; here nothing is regrouped between depths
 // (see "No gather on the operand side" below).
 //
-// One tile = 128 ready nodes x (8*G hidden units x 5 gates).  W is pre-packed so that the 5 gate
-// pre-activations of a hidden unit sit in the same accumulator row slice and one thread (one
-// tensor-memory lane = one node) can finish the cell without any exchange.
+// One tile = rt ready nodes (32, 64 or 128) x (8*G hidden units x 5 gates).  W is pre-packed so
+// that the 5 gate pre-activations of a hidden unit sit in the same accumulator row slice and one
+// thread (one tensor-memory lane = one node) can finish the cell without any exchange.
 //
 // No gather on the operand side: a tree node has exactly one caller, so the epilogue writes a
 // node's state straight into the slot its caller will read - row pos(caller) of the dense operand
 // matrix Ain[pos][h_l | h_r] (bf16) and of Cin[pos][c_l | c_r] (fp32), pos being the caller's
-// position in the ready order.  Every wavefront's operand is then a contiguous block of rows and
-// one tiled TMA load per K block feeds the tensor core.  Leaves: the embedding rows are copied
-// once into ready order (Xin) by all CTAs before the first wavefront.
+// position in the ready order.  Every wavefront's operand is then a contiguous block of rows, and
+// one TMA request per operand brings a box of several (or all) K blocks of a tile.  Leaves: the
+// embedding rows are copied once into ready order (Xin) by all CTAs before the first wavefront.
 //
 // Warp roles (384 threads): warps 0-3 and 6-9 epilogue (tensor-memory lane quadrant = warp id
-// mod 4; the two sets split every unit group in halves), warp 4 TMA producer of the A tiles,
-// warp 10 TMA producer of the W tiles (issuing a TMA load costs its thread about a hundred
+// mod 4; the two sets split every unit group in halves), warp 4 TMA producer of the operand rows,
+// warp 10 TMA producer of the weight rows (issuing a request costs its thread a few hundred
 // cycles, so the two streams are issued side by side), warp 5 MMA issuer + tensor-memory owner,
-// warp 11 second MMA issuer: issuing one tcgen05.mma costs its thread about 83 cycles whatever N
-// is, so on thin tiles (N <= 128) the two issuers take alternate K blocks into two partial
-// accumulators that the epilogue adds.
+// warp 11 chooses the tile plan of the next wavefront.
 #include "tc_ptx.cuh"
 
 namespace tl {
