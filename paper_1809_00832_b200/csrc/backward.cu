@@ -80,9 +80,10 @@ __global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) {
 }
 
 // ---- classifier: logits, softmax, loss, dlogits, dh (classifier part), dWc, dbc -------------- //
-// One warp per node; lane k owns class k (C <= 32).
+// One warp per node: the lanes share the contraction over h (lane j takes units j, j + 32, ...),
+// a butterfly sum gives every lane all logits, lane k keeps class k (C <= 32).
 constexpr int kClsWarps = 8;
-constexpr int kClsNodesPerCta = 64;
+constexpr int kClsNodesPerCta = 16;
 
 __global__ void __launch_bounds__(kClsWarps * 32) k_bwd_classifier(BwdParams p) {
   extern __shared__ float s_dWc[];  // [H][C] + [C], CTA-local partial sums
@@ -97,10 +98,12 @@ __global__ void __launch_bounds__(kClsWarps * 32) k_bwd_classifier(BwdParams p) 
     if (node >= p.n) break;
     const float* hn = p.h + (size_t)node * H;
     float logit = -INFINITY;
-    if (lane < C) {
-      float acc = p.bc[lane];
-      for (int j = 0; j < H; ++j) acc = fmaf(hn[j], p.Wc[j * C + lane], acc);
-      logit = acc;
+    for (int k = 0; k < C; ++k) {
+      float part = 0.f;
+      for (int j = lane; j < H; j += 32) part = fmaf(hn[j], __ldg(p.Wc + j * C + k), part);
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(kFull, part, d);
+      if (lane == k) logit = part + p.bc[k];
     }
     float m = logit;
 #pragma unroll

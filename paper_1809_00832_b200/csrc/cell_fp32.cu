@@ -25,6 +25,7 @@ struct FwdParams {
   float *h, *c, *gates;
   DevStatus* st;
   long long wait_limit;
+  int w_stationary, a_row, w_row;   // persistent kernel: W_h slice resident in shared memory; row strides (floats)
 };
 
 __device__ __forceinline__ float sigmoidf_acc(float x) { return 1.0f / (1.0f + expf(-x)); }
@@ -36,8 +37,10 @@ struct TileSmem {
 };
 
 // Rows per tile of a wavefront of `rows` nodes: a level-uniform choice.
+// (16-row tiles as long as they take at most two rounds over the SMs: a 64-row tile re-uses every
+// weight it reads four times, but costs about twice a 16-row one.)
 __host__ __device__ inline int rows_per_tile(int rows, int tiles_u, int n_sms) {
-  return ((rows + TM - 1) / TM) * tiles_u >= n_sms ? TM : TMS;
+  return ((rows + TMS - 1) / TMS) * tiles_u > 2 * n_sms ? TM : TMS;
 }
 
 // One tile: rows [row0, row0 + TM) of the ready order (clipped to row_end), hidden units
@@ -154,6 +157,143 @@ __device__ void fp32_tile(const FwdParams& p, int row0, int row_end, int u0, boo
   }
 }
 
+// Internal-node tile of the persistent kernel when the recurrent weights of the CTA's 16 hidden
+// units stay in shared memory for the whole kernel (Ws[5 * TU][w_row], one row per gate column, the
+// contraction index contiguous): only the operand rows [h_l | h_r] of the tile are fetched, all
+// loads of a thread in flight together, and the contraction runs out of shared memory in float4
+// steps, every thread on 4 rows x 5 gates of one hidden unit.  A 16-row tile has only 4 such row
+// groups, so its 16 thread groups also split the contraction in four; the partial sums meet in
+// shared memory (red[4][TMS][5 * TU]).  Same cell update as fp32_tile.
+template <int TM>
+__device__ void fp32_tile_stationary(const FwdParams& p, int row0, int row_end, int u0, float* As,
+                                     const float* Ws, float* red, int* s_node, int* s_l, int* s_r) {
+  constexpr bool kSplit = TM == TMS;
+  constexpr int RPT = 4, NQ = kSplit ? 4 : 1;
+  const int tid = threadIdx.x, tx = tid % TU, ty = tid / TU;
+  const int rg = kSplit ? (ty & 3) : ty, kq = kSplit ? (ty >> 2) : 0;
+  const int H = p.H, K = 2 * H, K4 = (K + 3) & ~3, a_row = p.a_row, w_row = p.w_row;
+  __syncthreads();  // previous tile's readers of As, red and the index arrays are done
+  for (int i = tid; i < TM; i += kThreads) {
+    const int row = row0 + i;
+    int node = -1, l = 0, r = 0;
+    if (row < row_end) { node = p.order[row]; l = p.left[node]; r = p.right[node]; }
+    s_node[i] = node; s_l[i] = l; s_r[i] = r;
+  }
+  __syncthreads();
+  if ((H & 1) == 0) {
+    const int hp = H / 2, pairs = K4 / 2;            // float2 pieces per child row / per operand row
+    const int total = TM * pairs;
+    for (int base = 0; base < total; base += 8 * kThreads) {
+      float2 v[8];
+      int dst[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int e = base + j * kThreads + tid;
+        v[j] = make_float2(0.f, 0.f);
+        dst[j] = -1;
+        if (e < total) {
+          const int i = e / pairs, q = e - i * pairs;
+          dst[j] = i * a_row + 2 * q;
+          if (s_node[i] >= 0 && q < 2 * hp) {
+            const float* src = q < hp ? p.h + (size_t)s_l[i] * H + 2 * q : p.h + (size_t)s_r[i] * H + 2 * (q - hp);
+            v[j] = __ldcg(reinterpret_cast<const float2*>(src));
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (dst[j] >= 0) *reinterpret_cast<float2*>(As + dst[j]) = v[j];
+    }
+  } else {
+    const int total = TM * K4;
+    for (int base = 0; base < total; base += 8 * kThreads) {
+      float v[8];
+      int dst[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int e = base + j * kThreads + tid;
+        v[j] = 0.f;
+        dst[j] = -1;
+        if (e < total) {
+          const int i = e / K4, k = e - i * K4;
+          dst[j] = i * a_row + k;
+          if (s_node[i] >= 0 && k < K)
+            v[j] = k < H ? __ldcg(p.h + (size_t)s_l[i] * H + k) : __ldcg(p.h + (size_t)s_r[i] * H + (k - H));
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (dst[j] >= 0) As[dst[j]] = v[j];
+    }
+  }
+  __syncthreads();
+  float acc[RPT][5];
+#pragma unroll
+  for (int i = 0; i < RPT; ++i)
+#pragma unroll
+    for (int g = 0; g < 5; ++g) acc[i][g] = 0.f;
+  const int steps = K4 / 4, per = (steps + NQ - 1) / NQ;
+  const int k_lo = kq * per * 4, k_hi = min(K4, k_lo + per * 4);
+  for (int k = k_lo; k < k_hi; k += 4) {
+    float4 a[RPT], w[5];
+#pragma unroll
+    for (int i = 0; i < RPT; ++i) a[i] = *reinterpret_cast<const float4*>(As + (rg * RPT + i) * a_row + k);
+#pragma unroll
+    for (int g = 0; g < 5; ++g) w[g] = *reinterpret_cast<const float4*>(Ws + (g * TU + tx) * w_row + k);
+#pragma unroll
+    for (int i = 0; i < RPT; ++i)
+#pragma unroll
+      for (int g = 0; g < 5; ++g) {
+        acc[i][g] = fmaf(a[i].x, w[g].x, acc[i][g]);
+        acc[i][g] = fmaf(a[i].y, w[g].y, acc[i][g]);
+        acc[i][g] = fmaf(a[i].z, w[g].z, acc[i][g]);
+        acc[i][g] = fmaf(a[i].w, w[g].w, acc[i][g]);
+      }
+  }
+  const int u = u0 + tx;
+  float bias[5] = {};
+  if (u < H) {
+#pragma unroll
+    for (int g = 0; g < 5; ++g) bias[g] = __ldg(p.b + g * H + u);
+  }
+  auto finish = [&](int ii, const float* z) {   // cell update of tile row ii, hidden unit u
+    const int node = s_node[ii];
+    if (node < 0 || u >= H) return;
+    const float gi = sigmoidf_acc(z[0] + bias[0]);
+    const float gfl = sigmoidf_acc(z[1] + bias[1]);
+    const float gfr = sigmoidf_acc(z[2] + bias[2]);
+    const float go = sigmoidf_acc(z[3] + bias[3]);
+    const float gu = tanhf(z[4] + bias[4]);
+    const float cn = gi * gu + gfl * __ldcg(p.c + (size_t)s_l[ii] * H + u) + gfr * __ldcg(p.c + (size_t)s_r[ii] * H + u);
+    p.c[(size_t)node * H + u] = cn;
+    p.h[(size_t)node * H + u] = go * tanhf(cn);
+    if (p.gates) {
+      float* g = p.gates + (size_t)node * 5 * H + u;
+      g[0] = gi; g[H] = gfl; g[2 * H] = gfr; g[3 * H] = go; g[4 * H] = gu;
+    }
+  };
+  if (kSplit) {
+    // partial sums of the four quarters of the contraction meet here; thread (tx, ty) then finishes row ty
+#pragma unroll
+    for (int i = 0; i < RPT; ++i)
+#pragma unroll
+      for (int g = 0; g < 5; ++g) red[(kq * TMS + rg * RPT + i) * (5 * TU) + g * TU + tx] = acc[i][g];
+    __syncthreads();
+    float z[5];
+#pragma unroll
+    for (int g = 0; g < 5; ++g) {
+      float sum = 0.f;
+#pragma unroll
+      for (int q = 0; q < NQ; ++q) sum += red[(q * TMS + ty) * (5 * TU) + g * TU + tx];
+      z[g] = sum;
+    }
+    finish(ty, z);
+  } else {
+#pragma unroll
+    for (int i = 0; i < RPT; ++i) finish(rg * RPT + i, acc[i]);
+  }
+}
+
 __global__ void __launch_bounds__(kThreads)
 k_fwd_fp32_level(FwdParams p, int row_begin, int row_end, int leaf) {
   __shared__ TileSmem s;
@@ -165,20 +305,50 @@ k_fwd_fp32_level(FwdParams p, int row_begin, int row_end, int leaf) {
 }
 
 // All wavefronts in one cooperative launch; a bounded grid barrier separates the levels.
+// Dynamic shared memory: [operand rows of a tile, at least a TileSmem][resident W_h slice][partial sums][row ids].
 __global__ void __launch_bounds__(kThreads)
 k_fwd_fp32_persistent(FwdParams p) {
-  __shared__ TileSmem s;
+  extern __shared__ float4 dyn_smem[];
   __shared__ int s_flag;
+  TileSmem& s = *reinterpret_cast<TileSmem*>(dyn_smem);
+  float* As = reinterpret_cast<float*>(dyn_smem);
+  size_t a_floats = (size_t)TM * p.a_row;
+  if (a_floats * 4 < sizeof(TileSmem)) a_floats = (sizeof(TileSmem) + 3) / 4;
+  a_floats = (a_floats + 3) & ~(size_t)3;
+  float* Ws = As + a_floats;
+  float* red = Ws + (p.w_stationary ? (size_t)5 * TU * p.w_row : 0);          // [4][TMS][5 * TU] partial sums
+  int* s_node = reinterpret_cast<int*>(red + (p.w_stationary ? 4 * TMS * 5 * TU : 0));
+  int* s_l = s_node + TM;
+  int* s_r = s_l + TM;
   if (ld_volatile(&p.st->status) != 0) return;
   const int n_levels = p.st->n_levels;
   const int tiles_u = (p.H + TU - 1) / TU;
+  const int H = p.H;
+  if (p.w_stationary && n_levels > 1) {
+    // The grid is a multiple of tiles_u, so tile t of any level, t = blockIdx.x + i * gridDim.x, has
+    // the same hidden-unit slice: its rows of W_h are fetched once, transposed to [column][k].
+    const int u0 = (blockIdx.x % tiles_u) * TU, K = 2 * H, w_row = p.w_row;
+    const float* Wk = p.W + (size_t)p.E * 5 * H;
+    for (int e = threadIdx.x; e < 5 * TU * w_row; e += kThreads) {
+      const int k = e / (5 * TU), col = e - k * 5 * TU, g = col / TU, uu = col - g * TU;
+      float v = 0.f;
+      if (k < K && u0 + uu < H) v = __ldg(Wk + (size_t)k * 5 * H + g * H + u0 + uu);
+      Ws[col * w_row + k] = v;
+    }
+  }
   for (int lvl = 0; lvl < n_levels; ++lvl) {
     const int begin = p.level_offset[lvl], end = p.level_offset[lvl + 1];
     const int tmr = rows_per_tile(end - begin, tiles_u, p.n_sms);
     const int tiles = ((end - begin + tmr - 1) / tmr) * tiles_u;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
-      if (tmr == TM) fp32_tile<TM>(p, begin + (t / tiles_u) * TM, end, (t % tiles_u) * TU, lvl == 0, s);
-      else fp32_tile<TMS>(p, begin + (t / tiles_u) * TMS, end, (t % tiles_u) * TU, lvl == 0, s);
+      const int tm = t / tiles_u, u0 = (t - tm * tiles_u) * TU;
+      if (lvl > 0 && p.w_stationary) {
+        if (tmr == TM) fp32_tile_stationary<TM>(p, begin + tm * TM, end, u0, As, Ws, red, s_node, s_l, s_r);
+        else fp32_tile_stationary<TMS>(p, begin + tm * TMS, end, u0, As, Ws, red, s_node, s_l, s_r);
+      } else {
+        if (tmr == TM) fp32_tile<TM>(p, begin + tm * TM, end, u0, lvl == 0, s);
+        else fp32_tile<TMS>(p, begin + tm * TMS, end, u0, lvl == 0, s);
+      }
     }
     if (lvl + 1 < n_levels &&
         !grid_barrier(p.st, (unsigned)(lvl + 1) * gridDim.x, p.wait_limit, &s_flag))
@@ -203,19 +373,41 @@ int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.gates = (flags & TREELSTM_SAVE_FOR_BACKWARD) ? reinterpret_cast<float*>(base + lay.gates) : nullptr;
   p.st = reinterpret_cast<DevStatus*>(base + lay.status);
   p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
+  p.w_stationary = 0; p.a_row = 0; p.w_row = 0;
   const int tiles_u = (ctx->H + TU - 1) / TU;
   if (flags & TREELSTM_PERSISTENT) {
+    // Resident W_h slice: 80 rows of w_row floats (w_row = 4 mod 32, so that the float4 reads of the
+    // sixteen columns of a gate spread over all banks) next to the operand rows of one tile.
+    const int K4 = (2 * ctx->H + 3) & ~3;
+    p.a_row = K4 + 4;
+    p.w_row = K4 + ((4 - K4 % 32) + 32) % 32;
+    size_t a_bytes = sizeof(float) * TM * (size_t)p.a_row;
+    if (a_bytes < sizeof(TileSmem)) a_bytes = sizeof(TileSmem);
+    a_bytes = (a_bytes + 15) & ~(size_t)15;
+    const size_t ids_bytes = 3 * TM * sizeof(int);
+    const size_t smem_stat = a_bytes + sizeof(float) * 5 * TU * (size_t)p.w_row + sizeof(float) * 4 * TMS * 5 * TU + ids_bytes;
+    size_t smem = sizeof(TileSmem) + ids_bytes;
+    p.w_stationary = 0;
+    int cap = ctx->opt.max_ctas > 0 ? ctx->opt.max_ctas : (1 << 30);
+    if (smem_stat <= 216 * 1024 && ctx->sm_count >= tiles_u && cap >= tiles_u) {
+      p.w_stationary = 1;
+      smem = smem_stat;
+    } else {
+      p.a_row = p.w_row = 0;
+    }
+    TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_fp32_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
     TL_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_fwd_fp32_persistent,
-                                                               kThreads, 0));
+                                                               kThreads, smem));
     int grid = per_sm * ctx->sm_count;
     const int want = ((n + TMS - 1) / TMS + 1) * tiles_u;   // never more CTAs than the widest level has tiles
     if (grid > want) grid = want;
-    if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
+    if (grid > cap) grid = cap;
+    if (p.w_stationary) grid = grid / tiles_u * tiles_u;    // every CTA keeps one hidden-unit slice
     if (grid < 1) grid = 1;
     void* args[] = {&p};
     TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_fp32_persistent, dim3(grid), dim3(kThreads),
-                                             args, 0, stream));
+                                             args, smem, stream));
     ctx->launches += 1;
     return TREELSTM_OK;
   }
