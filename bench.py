@@ -168,7 +168,7 @@ def train_step_time(steps: int = 200, warmup: int = 5):
     return {"workload": "train25_fp32", "trees": f.n_trees, "nodes": f.n_nodes, "ms_per_step": mean,
             "trees_per_sec": f.n_trees / (mean * 1e-3), "nodes_per_sec": f.n_nodes / (mean * 1e-3),
             "steps": steps, "gpu_launches_per_step": launches, "dtype": "f32",
-            "note": "backward reads the level table back once per step (one stream synchronisation)"}
+            "note": "persistent forward + one-launch backward; the binding reads the status word back after each"}
 
 
 def run_sweeps(args):

@@ -40,16 +40,19 @@ __global__ void k_bwd_mark_tokens(BwdParams p) {
 
 // Exclusive scan of the flags over the vocabulary by one CTA; flagged ids are emitted in
 // ascending order and tok_slot[id] becomes the row index of id in dEmb_rows.
-__global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) {
+__device__ void scan_tokens(const BwdParams& p) {   // one CTA of any size that is a multiple of 32
   __shared__ int warp_sum[32];
   __shared__ int carry;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int kPer = 8;                            // consecutive ids per thread and trip: fewer CTA barriers
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nw = nt >> 5;
   if (tid == 0) carry = 0;
   __syncthreads();
-  for (int base = 0; base < p.vocab; base += 1024) {
-    const int i = base + tid;
-    const int v = i < p.vocab ? p.tok_slot[i] : 0;
-    int incl = v;
+  for (int base = 0; base < p.vocab; base += nt * kPer) {
+    const int i0 = base + tid * kPer;
+    int v[kPer], sum = 0;
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) { v[j] = i0 + j < p.vocab ? p.tok_slot[i0 + j] : 0; sum += v[j]; }
+    int incl = sum;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
       int t = __shfl_up_sync(kFull, incl, d);
@@ -58,7 +61,7 @@ __global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) {
     if (lane == 31) warp_sum[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-      int w = warp_sum[lane], wi = w;
+      int w = lane < nw ? warp_sum[lane] : 0, wi = w;
 #pragma unroll
       for (int d = 1; d < 32; d <<= 1) {
         int t = __shfl_up_sync(kFull, wi, d);
@@ -67,17 +70,22 @@ __global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) {
       warp_sum[lane] = wi - w;
     }
     __syncthreads();
-    const int excl = carry + warp_sum[warp] + incl - v;
-    if (i < p.vocab) {
-      p.tok_slot[i] = excl;
-      if (v) p.touched_ids[excl] = i;
+    int excl = carry + warp_sum[warp] + incl - sum;
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) {
+      if (i0 + j < p.vocab) {
+        p.tok_slot[i0 + j] = excl;
+        if (v[j]) p.touched_ids[excl] = i0 + j;
+      }
+      excl += v[j];
     }
     __syncthreads();
-    if (tid == 1023) carry = excl + v;
+    if (tid == nt - 1) carry = excl;
     __syncthreads();
   }
   if (tid == 0) { *p.n_touched = carry; p.st->n_touched = carry; }
 }
+__global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) { scan_tokens(p); }
 
 // ---- classifier: logits, softmax, loss, dlogits, dh (classifier part), dWc, dbc -------------- //
 // One warp per node: the lanes share the contraction over h (lane j takes units j, j + 32, ...),
@@ -85,15 +93,17 @@ __global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) {
 constexpr int kClsWarps = 8;
 constexpr int kClsNodesPerCta = 16;
 
-__global__ void __launch_bounds__(kClsWarps * 32) k_bwd_classifier(BwdParams p) {
-  extern __shared__ float s_dWc[];  // [H][C] + [C], CTA-local partial sums
+// The CTA takes the node groups vb_first, vb_first + vb_step, ...; s_dWc [H][C] + [C] collects its partial sums.
+__device__ void classifier_groups(const BwdParams& p, int vb_first, int vb_step, float* s_dWc) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = p.H, C = p.C;
   for (int i = tid; i < H * C + C; i += blockDim.x) s_dWc[i] = 0.f;
   __syncthreads();
-  const int node0 = blockIdx.x * kClsNodesPerCta;
   const float inv_n = 1.0f / (float)p.n;
+  const int n_groups = (p.n + kClsNodesPerCta - 1) / kClsNodesPerCta;
+  for (int vb = vb_first; vb < n_groups; vb += vb_step)
   for (int q = warp; q < kClsNodesPerCta; q += kClsWarps) {
+    const int node0 = vb * kClsNodesPerCta;
     const int node = node0 + q;
     if (node >= p.n) break;
     const float* hn = p.h + (size_t)node * H;
@@ -137,13 +147,14 @@ __global__ void __launch_bounds__(kClsWarps * 32) k_bwd_classifier(BwdParams p) 
   for (int i = tid; i < H * C; i += blockDim.x) atomicAdd(&p.dWc[i], s_dWc[i]);
   for (int i = tid; i < C; i += blockDim.x) atomicAdd(&p.dbc[i], s_dWc[H * C + i]);
 }
+__global__ void __launch_bounds__(kClsWarps * 32) k_bwd_classifier(BwdParams p) {
+  extern __shared__ float s_dyn[];
+  classifier_groups(p, blockIdx.x, gridDim.x, s_dyn);
+}
 
 // ---- gate gradients of one wavefront -------------------------------------------------------- //
-__global__ void k_bwd_gates(BwdParams p, int row_begin, int row_end, int leaf) {
+__device__ __forceinline__ void gates_element(const BwdParams& p, int row_begin, long long idx, int leaf) {
   const int H = p.H;
-  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long total = (long long)(row_end - row_begin) * H;
-  if (idx >= total) return;
   const int row = row_begin + (int)(idx / H), u = (int)(idx % H);
   const int node = p.order[row];
   const float* g = p.gates + (size_t)node * 5 * H + u;
@@ -168,6 +179,10 @@ __global__ void k_bwd_gates(BwdParams p, int row_begin, int row_end, int leaf) {
     p.dc[(size_t)r * H + u] = dcn * gfr;
   }
 }
+__global__ void k_bwd_gates(BwdParams p, int row_begin, int row_end, int leaf) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < (long long)(row_end - row_begin) * p.H) gates_element(p, row_begin, idx, leaf);
+}
 
 // ---- dIn = dz W^T for one wavefront --------------------------------------------------------- //
 // out[row][k] = sum_j dz[row][j] * W[koff + k][j]; tile 64 rows x 64 outputs, 16 x 16 threads.
@@ -176,17 +191,34 @@ __global__ void k_bwd_gates(BwdParams p, int row_begin, int row_end, int leaf) {
 constexpr int BT = 64, BK = 32;
 constexpr int kLd = BT * BK / 256;   // elements of each operand per thread and chunk
 
-__global__ void __launch_bounds__(256)
-k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
-  __shared__ float As[2][BT][BK + 1];
-  __shared__ float Bs[2][BT][BK + 1];
-  __shared__ int s_node[BT];
+constexpr int kDiRow = BK + 4;       // row stride: float4 reads along the contraction, 16 rows spread over all banks
+struct DinputSmem {
+  __align__(16) float As[2][BT][kDiRow];
+  __align__(16) float Bs[2][BT][kDiRow];
+  int node[BT];
+  int dst_a[BT], dst_b[BT];   // where a row's dIn goes: left / right child, or (leaves) its row of dEmb_rows
+};
+__device__ void dinput_block(const BwdParams& p, int row_begin, int row_end, int leaf, int bx, int by, int nby,
+                             DinputSmem& sm) {
+  float (*As)[BT][kDiRow] = sm.As;
+  float (*Bs)[BT][kDiRow] = sm.Bs;
+  int* s_node = sm.node;
   const int H = p.H, E = p.E, J = 5 * H;
   const int K = leaf ? E : 2 * H, koff = leaf ? 0 : E;
   const int tiles_k = (K + BT - 1) / BT;
-  const int row0 = row_begin + (blockIdx.x / tiles_k) * BT, k0 = (blockIdx.x % tiles_k) * BT;
+  const int row0 = row_begin + (bx / tiles_k) * BT, k0 = (bx % tiles_k) * BT;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  for (int i = tid; i < BT; i += 256) s_node[i] = row0 + i < row_end ? p.order[row0 + i] : -1;
+  __syncthreads();   // a previous block of this CTA may still be reading the shared arrays
+  // the index chains (order -> children, or order -> token -> touched row) are resolved once per block
+  for (int i = tid; i < BT; i += 256) {
+    int node = -1, da = 0, db = 0;
+    if (row0 + i < row_end) {
+      node = p.order[row0 + i];
+      if (leaf) da = p.tok_slot[p.token[node]];
+      else { da = p.left[node]; db = p.right[node]; }
+    }
+    s_node[i] = node; sm.dst_a[i] = da; sm.dst_b[i] = db;
+  }
   __syncthreads();
   float acc[4][4] = {};
   float ra[kLd], rb[kLd];
@@ -210,8 +242,8 @@ k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
   // partial sums with atomics (few levels fill the GPU on their own, the chain of dependent
   // memory round trips per CTA is what costs time)
   const int chunks_all = (J + BK - 1) / BK;
-  const int per_split = (chunks_all + gridDim.y - 1) / gridDim.y;
-  const int c_lo = blockIdx.y * per_split, chunks = min(chunks_all, c_lo + per_split);
+  const int per_split = (chunks_all + nby - 1) / nby;
+  const int c_lo = by * per_split, chunks = min(chunks_all, c_lo + per_split);
   if (c_lo >= chunks) return;
   fetch(c_lo * BK);
   stash(c_lo & 1);
@@ -220,14 +252,22 @@ k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
     const int buf = cidx & 1;
     if (cidx + 1 < chunks) fetch((cidx + 1) * BK);
 #pragma unroll
-    for (int jj = 0; jj < BK; ++jj) {
-      float a[4], b[4];
+    for (int jj = 0; jj < BK; jj += 4) {
+      float4 a[4], b[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) { a[i] = As[buf][ty + 16 * i][jj]; b[i] = Bs[buf][tx + 16 * i][jj]; }
+      for (int i = 0; i < 4; ++i) {
+        a[i] = *reinterpret_cast<const float4*>(&As[buf][ty + 16 * i][jj]);
+        b[i] = *reinterpret_cast<const float4*>(&Bs[buf][tx + 16 * i][jj]);
+      }
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc[i][q] = fmaf(a[i], b[q], acc[i][q]);
+        for (int q = 0; q < 4; ++q) {
+          acc[i][q] = fmaf(a[i].x, b[q].x, acc[i][q]);
+          acc[i][q] = fmaf(a[i].y, b[q].y, acc[i][q]);
+          acc[i][q] = fmaf(a[i].z, b[q].z, acc[i][q]);
+          acc[i][q] = fmaf(a[i].w, b[q].w, acc[i][q]);
+        }
     }
     if (cidx + 1 < chunks) stash(buf ^ 1);
     __syncthreads();
@@ -241,13 +281,24 @@ k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
       const int k = k0 + tx + 16 * q;
       if (k >= K) continue;
       if (leaf) {
-        atomicAdd(&p.dEmb_rows[(size_t)p.tok_slot[p.token[node]] * E + k], acc[i][q]);
+        atomicAdd(&p.dEmb_rows[(size_t)sm.dst_a[ty + 16 * i] * E + k], acc[i][q]);
       } else {
-        const int child = k < H ? p.left[node] : p.right[node];
+        const int child = k < H ? sm.dst_a[ty + 16 * i] : sm.dst_b[ty + 16 * i];
         atomicAdd(&p.dh[(size_t)child * H + (k < H ? k : k - H)], acc[i][q]);
       }
     }
   }
+}
+// how many CTAs share the contraction of one dIn tile
+__host__ __device__ inline int dinput_splits(int tiles, int J) {
+  const int chunks_all = (J + BK - 1) / BK;
+  return tiles >= 148 ? 1 : (chunks_all < 6 ? chunks_all : 6);
+}
+__host__ __device__ inline int dinput_tiles(int rows, int K) { return ((rows + BT - 1) / BT) * ((K + BT - 1) / BT); }
+__global__ void __launch_bounds__(256)
+k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
+  __shared__ DinputSmem sm;
+  dinput_block(p, row_begin, row_end, leaf, blockIdx.x, blockIdx.y, gridDim.y, sm);
 }
 
 // ---- dW = In^T dZ (contraction over nodes) and db ------------------------------------------- //
@@ -256,17 +307,35 @@ k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
 constexpr int WR = 16;               // nodes per chunk
 constexpr int kLdW = WR * BT / 256;  // 4 elements of each operand per thread and chunk
 
-__global__ void __launch_bounds__(256)
-k_bwd_dweight(BwdParams p, int part, int row_begin, int row_end, int rows_per_split) {
-  __shared__ float As[2][WR][BT];
-  __shared__ float Bs[2][WR][BT];
+constexpr int kDwRows = 128;         // nodes per block of the dW contraction
+struct DweightSmem {
+  __align__(16) float As[2][WR][BT];
+  __align__(16) float Bs[2][WR][BT];
+  int node[kDwRows], ia[kDwRows], ib[kDwRows];   // node id and where its operand row comes from
+};
+__device__ void dweight_block(const BwdParams& p, int part, int row_begin, int row_end, int rows_per_split,
+                              int bx, int by, DweightSmem& sm) {
+  float (*As)[WR][BT] = sm.As;
+  float (*Bs)[WR][BT] = sm.Bs;
   const int H = p.H, E = p.E, J = 5 * H;
   const int K = part == 0 ? E : 2 * H, koff = part == 0 ? 0 : E;
   const int tiles_j = (J + BT - 1) / BT;
-  const int k0 = (blockIdx.x / tiles_j) * BT, j0 = (blockIdx.x % tiles_j) * BT;
-  const int r_lo = row_begin + blockIdx.y * rows_per_split;
-  const int r_hi = min(row_end, r_lo + rows_per_split);
+  const int k0 = (bx / tiles_j) * BT, j0 = (bx % tiles_j) * BT;
+  const int r_lo = row_begin + by * rows_per_split;
+  __syncthreads();   // a previous block of this CTA may still be reading the shared arrays
+  const int r_hi = min(row_end, r_lo + min(rows_per_split, kDwRows));
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  // the index chain order -> token / children is resolved once per block, not once per fetched element
+  for (int i = tid; i < kDwRows; i += 256) {
+    int node = 0, ia = 0, ib = 0;
+    if (r_lo + i < r_hi) {
+      node = p.order[r_lo + i];
+      if (part == 0) ia = p.token[node];
+      else { ia = p.left[node]; ib = p.right[node]; }
+    }
+    sm.node[i] = node; sm.ia[i] = ia; sm.ib[i] = ib;
+  }
+  __syncthreads();
   float acc[4][4] = {};
   float ra[kLdW], rb[kLdW];
   // element e of a chunk: node rr = e / 64 of the chunk, column cc = e % 64 of the tile
@@ -277,13 +346,13 @@ k_bwd_dweight(BwdParams p, int part, int row_begin, int row_end, int rows_per_sp
       const int row = r0 + rr;
       float va = 0.f, vb = 0.f;
       if (row < r_hi) {
-        const int node = p.order[row];
+        const int li = row - r_lo;
         const int k = k0 + cc, j = j0 + cc;
         if (k < K) {
-          if (part == 0) va = __ldg(p.emb + (size_t)p.token[node] * E + k);
-          else va = k < H ? p.h[(size_t)p.left[node] * H + k] : p.h[(size_t)p.right[node] * H + (k - H)];
+          if (part == 0) va = __ldg(p.emb + (size_t)sm.ia[li] * E + k);
+          else va = k < H ? p.h[(size_t)sm.ia[li] * H + k] : p.h[(size_t)sm.ib[li] * H + (k - H)];
         }
-        if (j < J) vb = p.dz[(size_t)node * J + j];
+        if (j < J) vb = p.dz[(size_t)sm.node[li] * J + j];
       }
       ra[q] = va;
       rb[q] = vb;
@@ -306,10 +375,10 @@ k_bwd_dweight(BwdParams p, int part, int row_begin, int row_end, int rows_per_sp
   for (int r0 = r_lo; r0 < r_hi; r0 += WR, buf ^= 1) {
     if (r0 + WR < r_hi) fetch(r0 + WR);
 #pragma unroll
-    for (int rr = 0; rr < WR; ++rr) {
-      float a[4], b[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) { a[i] = As[buf][rr][ty + 16 * i]; b[i] = Bs[buf][rr][tx + 16 * i]; }
+    for (int rr = 0; rr < WR; ++rr) {   // thread (tx, ty): outputs k0 + 4 ty .. + 3  x  j0 + 4 tx .. + 3
+      const float4 a4 = *reinterpret_cast<const float4*>(&As[buf][rr][4 * ty]);
+      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[buf][rr][4 * tx]);
+      const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -320,24 +389,106 @@ k_bwd_dweight(BwdParams p, int part, int row_begin, int row_end, int rows_per_sp
   }
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const int k = k0 + ty + 16 * i;
+    const int k = k0 + 4 * ty + i;
     if (k >= K) continue;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const int j = j0 + tx + 16 * q;
+      const int j = j0 + 4 * tx + q;
       if (j < J) atomicAdd(&p.dW[(size_t)(koff + k) * J + j], acc[i][q]);
     }
   }
 }
+__global__ void __launch_bounds__(256)
+k_bwd_dweight(BwdParams p, int part, int row_begin, int row_end, int rows_per_split) {
+  __shared__ DweightSmem sm;
+  dweight_block(p, part, row_begin, row_end, rows_per_split, blockIdx.x, blockIdx.y, sm);
+}
 
-__global__ void k_bwd_dbias(BwdParams p) {
+// column j of db over the nodes [256 by, 256 by + 256)
+__device__ __forceinline__ void dbias_piece(const BwdParams& p, int j, int by) {
   const int J = 5 * p.H;
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= J) return;
-  const int r_lo = blockIdx.y * 256, r_hi = min(p.n, r_lo + 256);
+  const int r_lo = by * 256, r_hi = min(p.n, r_lo + 256);
   float acc = 0.f;
   for (int r = r_lo; r < r_hi; ++r) acc += p.dz[(size_t)r * J + j];
   atomicAdd(&p.db[j], acc);
+}
+__global__ void k_bwd_dbias(BwdParams p) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < 5 * p.H) dbias_piece(p, j, blockIdx.y);
+}
+
+// ---- the whole backward pass in one cooperative launch --------------------------------------- //
+// Used after a forward that left the level table on the device only (persistent / sub-forest
+// modes): no host round trip, no launch per wavefront.  Phases, separated by the bounded grid
+// barrier: clear the outputs | mark leaf tokens | token scan (CTA 0) next to the classifier (all
+// other CTAs) | per wavefront from the top: gate gradients, then dIn = dz W^T into the children |
+// dW, db (they only need every dz).
+union BwdSmem {
+  DinputSmem di;
+  DweightSmem dw;
+};
+template <class T>
+__device__ __forceinline__ void zero_range(T* ptr, size_t count, size_t gtid, size_t gthreads) {
+  for (size_t i = gtid; i < count; i += gthreads) ptr[i] = T(0);
+}
+__global__ void __launch_bounds__(256)
+k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
+  extern __shared__ float4 s_dyn4[];
+  BwdSmem& sm = *reinterpret_cast<BwdSmem*>(s_dyn4);
+  float* s_cls = reinterpret_cast<float*>(s_dyn4) + (sizeof(BwdSmem) + 3) / 4;
+  __shared__ int s_flag;
+  if (ld_volatile(&p.st->status) != 0) return;
+  const int n_levels = p.st->n_levels;
+  const int n = p.n, H = p.H, E = p.E, C = p.C, J = 5 * H;
+  p.n_leaves = n_levels > 0 ? level_offset[1] : 0;
+  const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, gthreads = (size_t)gridDim.x * blockDim.x;
+  unsigned int arrivals = 0;
+  auto barrier = [&]() {
+    arrivals += gridDim.x;
+    return grid_barrier(p.st, arrivals, wait_limit, &s_flag, true, &p.st->barrier_bwd);
+  };
+  if (gtid == 0) { *p.loss = 0.f; *p.n_touched = 0; }
+  zero_range(p.dW, (size_t)(E + 2 * H) * J, gtid, gthreads);
+  zero_range(p.db, (size_t)J, gtid, gthreads);
+  zero_range(p.dWc, (size_t)H * C, gtid, gthreads);
+  zero_range(p.dbc, (size_t)C, gtid, gthreads);
+  zero_range(p.dc, (size_t)n * H, gtid, gthreads);
+  zero_range(p.tok_slot, (size_t)p.vocab + 1, gtid, gthreads);
+  zero_range(p.dEmb_rows, (size_t)p.n_leaves * E, gtid, gthreads);
+  if (!barrier()) return;
+  for (size_t r = gtid; r < (size_t)p.n_leaves; r += gthreads) p.tok_slot[p.token[p.order[r]]] = 1;
+  if (!barrier()) return;
+  if (gridDim.x == 1) {
+    scan_tokens(p);
+    classifier_groups(p, 0, 1, s_cls);
+  } else if (blockIdx.x == 0) {
+    scan_tokens(p);
+  } else {
+    classifier_groups(p, blockIdx.x - 1, gridDim.x - 1, s_cls);
+  }
+  if (!barrier()) return;
+  for (int lvl = n_levels - 1; lvl >= 0; --lvl) {
+    const int begin = level_offset[lvl], end = level_offset[lvl + 1], leaf = lvl == 0 ? 1 : 0;
+    const long long elems = (long long)(end - begin) * H;
+    for (long long idx = (long long)gtid; idx < elems; idx += (long long)gthreads) gates_element(p, begin, idx, leaf);
+    if (!barrier()) return;
+    const int tiles = dinput_tiles(end - begin, leaf ? E : 2 * H), splits = dinput_splits(tiles, J);
+    for (int vb = blockIdx.x; vb < tiles * splits; vb += gridDim.x)
+      dinput_block(p, begin, end, leaf, vb % tiles, vb / tiles, splits, sm.di);
+    if (lvl > 0 && !barrier()) return;   // the leaves' dIn goes to the embedding rows only
+  }
+  const int tiles_j = (J + BT - 1) / BT, rows_per_split = kDwRows;
+  for (int part = 0; part < 2; ++part) {
+    const int begin = part == 0 ? 0 : p.n_leaves, end = part == 0 ? p.n_leaves : n;
+    if (end <= begin) continue;
+    const int K = part == 0 ? E : 2 * H;
+    const int nbx = ((K + BT - 1) / BT) * tiles_j, nby = (end - begin + rows_per_split - 1) / rows_per_split;
+    for (int vb = blockIdx.x; vb < nbx * nby; vb += gridDim.x)
+      dweight_block(p, part, begin, end, rows_per_split, vb % nbx, vb / nbx, sm.dw);
+  }
+  const int nby = (n + 255) / 256;
+  for (long long idx = (long long)gtid; idx < (long long)J * nby; idx += (long long)gthreads)
+    dbias_piece(p, (int)(idx % J), (int)(idx / J));
 }
 
 }  // namespace
@@ -347,9 +498,12 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
                     int32_t* n_touched, cudaStream_t stream) {
   auto& L = ctx->last;
   L.stream = stream;
-  int rc = ensure_host_levels(ctx);
-  if (rc != TREELSTM_OK) return rc;
-  const int n = L.n, H = ctx->H, E = ctx->E, C = ctx->C, n_levels = L.n_levels;
+  const bool one_launch = !L.host_levels_valid;   // the forward kept the level table on the device
+  if (!one_launch) {
+    int rc = ensure_host_levels(ctx);
+    if (rc != TREELSTM_OK) return rc;
+  }
+  const int n = L.n, H = ctx->H, E = ctx->E, C = ctx->C, n_levels = one_launch ? 0 : L.n_levels;
   const int32_t* off = ctx->host_level_offset;
   char* base = static_cast<char*>(L.ws);
   BwdParams p;
@@ -367,6 +521,34 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
   p.st = reinterpret_cast<DevStatus*>(base + L.lay.status);
 
   const size_t J = 5 * (size_t)H;
+  const size_t cls_smem = sizeof(float) * ((size_t)H * C + C);
+  if (cls_smem > 160 * 1024) return TREELSTM_ERR_UNSUPPORTED;
+  if (one_launch) {
+    if (n == 0) {
+      TL_CUDA(ctx, cudaMemsetAsync(loss, 0, sizeof(float), stream));
+      TL_CUDA(ctx, cudaMemsetAsync(dW, 0, sizeof(float) * (E + 2 * (size_t)H) * J, stream));
+      TL_CUDA(ctx, cudaMemsetAsync(db, 0, sizeof(float) * J, stream));
+      TL_CUDA(ctx, cudaMemsetAsync(dWc, 0, sizeof(float) * H * C, stream));
+      TL_CUDA(ctx, cudaMemsetAsync(dbc, 0, sizeof(float) * C, stream));
+      TL_CUDA(ctx, cudaMemsetAsync(n_touched, 0, sizeof(int), stream));
+      return TREELSTM_OK;
+    }
+    const size_t smem = ((sizeof(BwdSmem) + 3) / 4) * 4 + cls_smem;
+    TL_CUDA(ctx, cudaFuncSetAttribute(k_bwd_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    TL_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_bwd_persistent, 256, smem));
+    if (per_sm < 1) return TREELSTM_ERR_UNSUPPORTED;
+    int grid = ctx->sm_count * (per_sm < 2 ? per_sm : 2);
+    if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
+    DevStatus* st = p.st;
+    TL_CUDA(ctx, cudaMemsetAsync(&st->barrier_bwd, 0, sizeof(unsigned int), stream));
+    const int* lvl_off = L.level_offset;
+    long long wait_limit = ctx->opt.wait_limit_kcycles * 1024;
+    void* args[] = {&p, &lvl_off, &wait_limit};
+    TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_bwd_persistent, dim3(grid), dim3(256), args, smem, stream));
+    ctx->launches += 1;
+    return TREELSTM_OK;
+  }
   TL_CUDA(ctx, cudaMemsetAsync(loss, 0, sizeof(float), stream));
   TL_CUDA(ctx, cudaMemsetAsync(dW, 0, sizeof(float) * (E + 2 * (size_t)H) * J, stream));
   TL_CUDA(ctx, cudaMemsetAsync(db, 0, sizeof(float) * J, stream));
@@ -380,8 +562,6 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
 
   k_bwd_mark_tokens<<<(p.n_leaves + 255) / 256, 256, 0, stream>>>(p);
   k_bwd_scan_tokens<<<1, 1024, 0, stream>>>(p);
-  const size_t cls_smem = sizeof(float) * ((size_t)H * C + C);
-  if (cls_smem > 200 * 1024) return TREELSTM_ERR_UNSUPPORTED;
   if (cls_smem > 48 * 1024)
     TL_CUDA(ctx, cudaFuncSetAttribute(k_bwd_classifier, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)cls_smem));
@@ -391,10 +571,7 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
     const int begin = off[lvl], end = off[lvl + 1], leaf = lvl == 0 ? 1 : 0;
     const long long elems = (long long)(end - begin) * H;
     k_bwd_gates<<<(unsigned)((elems + 255) / 256), 256, 0, stream>>>(p, begin, end, leaf);
-    const int K = leaf ? E : 2 * H;
-    const int tiles = ((end - begin + BT - 1) / BT) * ((K + BT - 1) / BT);
-    const int chunks_all = (int)((J + BK - 1) / BK);
-    const int splits = tiles >= 148 ? 1 : (chunks_all < 6 ? chunks_all : 6);
+    const int tiles = dinput_tiles(end - begin, leaf ? E : 2 * H), splits = dinput_splits(tiles, (int)J);
     k_bwd_dinput<<<dim3(tiles, splits), 256, 0, stream>>>(p, begin, end, leaf);
     ctx->launches += 2;
   }
@@ -403,7 +580,7 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
     const int begin = part == 0 ? 0 : p.n_leaves, end = part == 0 ? p.n_leaves : n;
     if (end <= begin) continue;
     const int K = part == 0 ? E : 2 * H;
-    const int rows_per_split = 128;
+    const int rows_per_split = kDwRows;
     const int splits = (end - begin + rows_per_split - 1) / rows_per_split;
     dim3 grid(((K + BT - 1) / BT) * tiles_j, splits);
     k_bwd_dweight<<<grid, 256, 0, stream>>>(p, part, begin, end, rows_per_split);

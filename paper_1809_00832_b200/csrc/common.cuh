@@ -19,7 +19,8 @@ struct DevStatus {
   int max_level;         // scratch of the multi-CTA level assignment
   unsigned int barrier;  // arrival counter of the persistent kernels' grid barrier
   int n_touched;         // distinct leaf tokens (backward)
-  int pad[58];
+  unsigned int barrier_bwd;  // arrival counter of the one-launch backward pass (cleared by its launch)
+  int pad[57];
 };
 static_assert(sizeof(DevStatus) == 256, "control block is one 256-byte line group");
 
@@ -203,7 +204,9 @@ __device__ __forceinline__ int ld_volatile(const int* p) { return *(const volati
 // Returns false if the wait expired or another CTA reported an error: the caller must then
 // leave its level loop (every CTA sees the same outcome within one more barrier).
 __device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
-                                             long long limit_cycles, int* s_flag, bool arrive = true) {
+                                             long long limit_cycles, int* s_flag, bool arrive = true,
+                                             unsigned int* counter = nullptr) {
+  if (!counter) counter = &st->barrier;
   __syncthreads();
   if (threadIdx.x < 32) {
     // Warp 0 polls.  Lane 0 announces the arrival (release: everything this CTA wrote, ordered
@@ -212,7 +215,7 @@ __device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
     // after an eighth of the memory latency on average instead of half of it.
     if (threadIdx.x == 0) {
       *s_flag = -1;
-      if (arrive) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&st->barrier) : "memory");
+      if (arrive) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
     }
     __syncwarp();
     const int lane = threadIdx.x;
@@ -222,7 +225,7 @@ __device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
       for (;;) {
         if (*(volatile int*)s_flag >= 0) break;          // another lane has the answer
         unsigned int seen;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&st->barrier) : "memory");
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
         if (seen >= target) { *(volatile int*)s_flag = 1; break; }
         if (*(volatile int*)&st->status != 0) { *(volatile int*)s_flag = 0; break; }
         if (clock64() - t0 > limit_cycles) {
