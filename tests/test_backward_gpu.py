@@ -77,3 +77,17 @@ def test_backward_errors():
     with pytest.raises(binding.TreeLSTMError) as err:
         model.backward(labels, forest.n_leaves)
     assert err.value.code == binding.ERR_LABEL_OUT_OF_RANGE
+
+
+def test_data_parallel_step_single_rank():
+    """the data-parallel wrapper on one rank: same gradients, touched rows trimmed to their count"""
+    from paper_1809_00832_b200 import data_parallel
+    w = fg.make_workload("train25_fp32", 0, n_trees=6)
+    f, p = w.forest, w.params
+    ref = orc.loss_and_gradients(f.left, f.right, f.token, p.emb, p.W, p.b, p.Wc, p.bc, w.labels)
+    model = util.make_model(p, "fp32")
+    out = data_parallel.training_step(model, util.to_dev(f.left), util.to_dev(f.right), util.to_dev(f.token),
+                                      util.to_dev(w.labels), f.n_leaves, binding.PERSISTENT)
+    res = {k: v.cpu().numpy() for k, v in out.items()}
+    assert res["touched_ids"].shape[0] == len(ref["touched_ids"])
+    _compare(res, ref, util.TOL["fp32"])
