@@ -289,10 +289,15 @@ __device__ void dinput_block(const BwdParams& p, int row_begin, int row_end, int
     }
   }
 }
-// how many CTAs share the contraction of one dIn tile
+// How many CTAs share the contraction of one dIn tile.  A 64 x 64 tile costs about 4 k cycles per
+// 32-wide chunk of the contraction whatever the number of valid rows, so a wavefront with few tiles
+// spreads the chunks over as many CTAs as there are (about two per SM), down to one chunk each.
 __host__ __device__ inline int dinput_splits(int tiles, int J) {
   const int chunks_all = (J + BK - 1) / BK;
-  return tiles >= 148 ? 1 : (chunks_all < 6 ? chunks_all : 6);
+  if (tiles >= 148) return 1;
+  int s = 296 / (tiles > 0 ? tiles : 1);
+  if (s < 6) s = 6;
+  return s < chunks_all ? s : chunks_all;
 }
 __host__ __device__ inline int dinput_tiles(int rows, int K) { return ((rows + BT - 1) / BT) * ((K + BT - 1) / BT); }
 __global__ void __launch_bounds__(256)
@@ -304,8 +309,8 @@ k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
 // ---- dW = In^T dZ (contraction over nodes) and db ------------------------------------------- //
 // part 0: rows [0,E) from the leaves (In = embedding rows); part 1: rows [E,E+2H) from the
 // internal nodes (In = [h_l | h_r]).  Tile 64 (k) x 64 (j); gridDim.y splits the node range.
-constexpr int WR = 16;               // nodes per chunk
-constexpr int kLdW = WR * BT / 256;  // 4 elements of each operand per thread and chunk
+constexpr int WR = 32;               // nodes per chunk: enough multiply-adds per chunk to cover the fetch of the next one
+constexpr int kLdW = WR * BT / 256;  // elements of each operand per thread and chunk
 
 constexpr int kDwRows = 128;         // nodes per block of the dW contraction
 struct DweightSmem {
