@@ -181,3 +181,61 @@ def test_subforest_mode_repeated_calls():
         h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
         assert util.max_abs(res["h"], h) < util.TOL["bf16"]
         assert util.max_abs(res["c"], c) < util.TOL["bf16"]
+
+
+def test_subforest_forward_then_backward():
+    """the sub-forest kernel keeps the gate activations too; the one-launch backward then matches the
+    oracle's gradients to the accuracy the bf16 forward values allow"""
+    rng = np.random.default_rng(45)
+    params = fg.draw_params(rng, 64, 40, 300, emb_dist="normal", emb_scale=0.3, w_scale=0.1, n_classes=5)
+    forest = fg.random_forest(rng, 11, 2, 30, 300)
+    forest, _ = fg.permute_node_ids(forest, rng)
+    labels = rng.integers(0, 5, size=forest.n_nodes).astype(np.int32)
+    ref = orc.loss_and_gradients(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
+                                 params.Wc, params.bc, labels)
+    model = util.make_model(params, "bf16")
+    out = model.forward(util.to_dev(forest.left), util.to_dev(forest.right), util.to_dev(forest.token),
+                        flags=binding.SUBFORESTS | binding.SAVE_FOR_BACKWARD)
+    assert model.last_mode() == binding.SUBFORESTS
+    assert util.max_abs(out["h"].cpu().numpy(), ref["h"]) < util.TOL["bf16"]
+    g = model.backward(util.to_dev(labels), forest.n_leaves)
+    assert abs(float(g["loss"].item()) - ref["loss"]) < util.TOL["bf16"]
+    for k in ("dW", "db", "dWc", "dbc"):
+        assert util.max_abs(g[k].cpu().numpy(), ref[k]) < util.TOL["bf16"], k
+    nt = int(g["n_touched"].item())
+    np.testing.assert_array_equal(g["touched_ids"][:nt].cpu().numpy(), ref["touched_ids"])
+    assert util.max_abs(g["dEmb_rows"][:nt].cpu().numpy(), ref["dEmb_rows"]) < util.TOL["bf16"]
+
+
+def test_subforest_mode_through_the_host_entry_point():
+    """treelstm_forward_host with the sub-forest flag: roots and their states come back in node order"""
+    import torch
+    rng = np.random.default_rng(46)
+    params = fg.draw_params(rng, 128, 64, 300, emb_dist="normal", emb_scale=0.3, w_scale=0.1)
+    forest = fg.random_forest(rng, 9, 1, 40, 300)
+    model = util.make_model(params, "bf16")
+    host = [torch.from_numpy(a).pin_memory() for a in (forest.left, forest.right, forest.token)]
+    out = model.forward_host(*host, flags=binding.SUBFORESTS, all_states=True, max_roots=forest.n_trees)
+    assert model.last_mode() == binding.SUBFORESTS
+    h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
+    assert util.max_abs(out["h"].numpy(), h) < util.TOL["bf16"]
+    assert int(out["n_roots"][0]) == forest.n_trees
+    roots = np.sort(forest.roots)
+    np.testing.assert_array_equal(out["root_ids"].numpy(), roots)
+    assert util.max_abs(out["root_h"].numpy(), h[roots]) < util.TOL["bf16"]
+
+
+def test_subforest_mode_large_forest_falls_back():
+    """more nodes than the scheduler deals out to sub-forests: the persistent kernel runs instead"""
+    rng = np.random.default_rng(47)
+    params = fg.draw_params(rng, 64, 48, 400, emb_dist="normal", emb_scale=0.3, w_scale=0.15)
+    forest = fg.random_forest(rng, 900, 10, 56, 400)
+    assert 24576 < forest.n_nodes <= 32768 or forest.n_nodes > 32768
+    model = util.make_model(params, "bf16")
+    res = util.gpu_forward(model, forest, binding.SUBFORESTS)
+    assert model.last_mode() == binding.PERSISTENT
+    sample = [0, 450, 899]
+    sub = fg.select_trees(forest, sample)
+    h, c, _ = orc.forward_recursive(sub.left, sub.right, sub.token, params.emb, params.W, params.b)
+    ids = np.nonzero(np.isin(forest.tree_of, sample))[0]
+    assert util.max_abs(res["h"][ids], h) < util.TOL["bf16"]
