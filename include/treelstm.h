@@ -278,6 +278,18 @@ TREELSTM_API int treelstm_last_mode(const treelstm_t* ctx);
  * number of co-resident clusters); 0 if that mode is not available for this context. */
 TREELSTM_API int treelstm_subforest_count(const treelstm_t* ctx);
 
+/*
+ * treelstm_tile_plan - how the bf16 wavefront kernel would cut a wavefront of `rows` ready nodes into
+ * tiles on a grid of n_ctas CTAs (the kernel takes the same decision on the device for every
+ * wavefront; this host-side view exists for tests and tuning; the paper has no counterpart).
+ *   out [host][10]: rows per tile (32 / 64 / 128), unit groups of 8 hidden units per tile (1 / 2 /
+ *   4), number of tiles, first tile of the split last round (= number of fat tiles if it is not
+ *   split), log2 of the number of pieces a fat tile of that round is cut into, K blocks per operand
+ *   box, boxes per tile, ring stages, bytes per stage, bytes of the ring.
+ * No CUDA call is made.
+ */
+TREELSTM_API int treelstm_tile_plan(int rows, int H, int E, int n_ctas, int leaf, int32_t* out);
+
 /* cudaError_t of the last failed CUDA call on this context (0 if none). */
 TREELSTM_API int treelstm_last_cuda_error(const treelstm_t* ctx);
 

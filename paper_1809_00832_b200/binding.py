@@ -58,6 +58,7 @@ SIGNATURES = {
     "treelstm_last_launch_count": (_i, [_vp]),
     "treelstm_last_mode": (_i, [_vp]),
     "treelstm_subforest_count": (_i, [_vp]),
+    "treelstm_tile_plan": (_i, [_i, _i, _i, _i, _i, _vp]),
     "treelstm_last_cuda_error": (_i, [_vp]),
     "treelstm_destroy": (_i, [_vp]),
     "treelstm_strerror": (ctypes.c_char_p, [_i]),
@@ -117,6 +118,19 @@ def schedule_static(left: torch.Tensor, right: torch.Tensor, token: torch.Tensor
     return int(lib.treelstm_schedule_static(n, _ptr(left), _ptr(right), _ptr(token), vocab, _ptr(out["level"]),
                                             _ptr(out["order"]), _ptr(out["level_offset"]), _ptr(out["n_levels"]),
                                             _ptr(out["status"]), _stream()))
+
+
+TILE_PLAN_FIELDS = ("rows_per_tile", "groups_per_tile", "tiles", "tail_from", "tail_log2_pieces", "kblocks_per_box",
+                    "boxes_per_tile", "stages", "stage_bytes", "ring_bytes")
+
+
+def tile_plan(rows: int, H: int, E: int, n_ctas: int, leaf: bool) -> dict:
+    """treelstm_tile_plan: the tile shape the bf16 kernel picks for a wavefront (host-side, no CUDA)."""
+    out = (ctypes.c_int32 * 10)()
+    rc = load_library().treelstm_tile_plan(rows, H, E, n_ctas, int(leaf), ctypes.cast(out, ctypes.c_void_p))
+    if rc != OK:
+        raise TreeLSTMError(rc, "treelstm_tile_plan")
+    return dict(zip(TILE_PLAN_FIELDS, [int(v) for v in out]))
 
 
 class TreeLSTM:

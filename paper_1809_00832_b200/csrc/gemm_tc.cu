@@ -573,3 +573,15 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
 }
 
 }  // namespace tl
+
+// Host-side view of the tile plan the bf16 wavefront kernel chooses on the device (same function).
+extern "C" int treelstm_tile_plan(int rows, int H, int E, int n_ctas, int leaf, int32_t* out) {
+  using namespace tl;
+  if (rows < 1 || H < 1 || E < 1 || n_ctas < 1 || !out) return TREELSTM_ERR_INVALID_ARG;
+  const int Hp = round_up(H, kKBlock), Ep = round_up(E, kKBlock);
+  const TilePlan pl = choose_tile_plan(rows, Hp / kUnitGroup, n_ctas, leaf != 0, leaf ? Ep / kKBlock : 2 * Hp / kKBlock);
+  out[0] = pl.rt; out[1] = pl.g; out[2] = pl.tiles; out[3] = pl.tail_from; out[4] = pl.tail_ls;
+  out[5] = pl.kbox; out[6] = pl.n_box; out[7] = pl.n_stages; out[8] = (int32_t)pl.stage_bytes; out[9] = kRingBytes;
+  return TREELSTM_OK;
+}
+
