@@ -348,7 +348,7 @@ def main() -> int:
     clocks = sampler.stop()
 
     # ---- end to end through the host-buffer entry point (pinned host arrays in, root states out) ----
-    hl, hr, ht = (torch.from_numpy(a).pin_memory() for a in (f.left, f.right, f.token))
+    hl, hr, ht = binding.pack_forest_host(f.left, f.right, f.token)   # one pinned buffer: one host-to-device copy
     host_out = model.forward_host(hl, hr, ht, flags=flags, max_roots=f.n_trees)
     e2e_steps = max(20, min(args.steps, 200))
     for _ in range(3):

@@ -201,6 +201,9 @@ TREELSTM_API int treelstm_backward(treelstm_t* ctx, const int32_t* labels, float
  *   max_roots, root_ids [host][max_roots], root_h, root_c [host][max_roots][H]: the roots in
  *                  ascending node id with their states, or NULL; n_roots [host][1] out or NULL.
  *   n_levels       [host][1] out or NULL.
+ * Copies are few and small, so their number matters: if right == left + n_nodes and token == right +
+ * n_nodes the forest goes up in one copy, and if root_h == (float*)(root_ids + max_roots) and
+ * root_c == root_h + max_roots * H (with max_roots <= n_nodes) the roots come back in one.
  * Returns the device status as well (it has synchronised).
  */
 TREELSTM_API int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, const int32_t* right,

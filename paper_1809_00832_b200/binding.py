@@ -133,6 +133,16 @@ def tile_plan(rows: int, H: int, E: int, n_ctas: int, leaf: bool) -> dict:
     return dict(zip(TILE_PLAN_FIELDS, [int(v) for v in out]))
 
 
+def pack_forest_host(left, right, token):
+    """The three forest arrays (numpy or CPU tensors) as rows of one pinned int32 tensor; returns the
+    three row views.  treelstm_forward_host copies arrays that are adjacent like this in one piece."""
+    rows = [torch.as_tensor(a, dtype=torch.int32) for a in (left, right, token)]
+    pack = torch.empty((3, rows[0].shape[0]), dtype=torch.int32, pin_memory=torch.cuda.is_available())
+    for i, r in enumerate(rows):
+        pack[i].copy_(r)
+    return pack[0], pack[1], pack[2]
+
+
 class TreeLSTM:
     """Thin handle around a treelstm_t*.  Tensors are the caller's; the handle only keeps the
     workspace it allocates through torch (device memory is PyTorch's job here)."""
@@ -287,9 +297,13 @@ class TreeLSTM:
                 out["level"] = torch.empty(n, dtype=torch.int32, **pin)
                 out["order"] = torch.empty(n, dtype=torch.int32, **pin)
             if max_roots > 0:
-                out["root_ids"] = torch.empty(max_roots, dtype=torch.int32, **pin)
-                out["root_h"] = torch.empty((max_roots, self.H), dtype=torch.float32, **pin)
-                out["root_c"] = torch.empty((max_roots, self.H), dtype=torch.float32, **pin)
+                # one pinned buffer [ids | h | c]: the library then brings the roots back in one copy
+                m, H = max_roots, self.H
+                pack = torch.empty(4 * m * (1 + 2 * H), dtype=torch.uint8, **pin)
+                out["root_ids"] = pack[:4 * m].view(torch.int32)
+                out["root_h"] = pack[4 * m:4 * m * (1 + H)].view(torch.float32).view(m, H)
+                out["root_c"] = pack[4 * m * (1 + H):].view(torch.float32).view(m, H)
+                out["_roots_pack"] = pack
         g = out.get
         rc = self.lib.treelstm_forward_host(self.handle, n, _ptr(left), _ptr(right), _ptr(token), _ptr(g("h")),
                                             _ptr(g("c")), _ptr(g("level")), _ptr(g("order")), _ptr(g("n_levels")),

@@ -58,9 +58,9 @@ int copy_params(treelstm* ctx, const float* emb, const float* W, const float* b,
 
 void free_host_path(treelstm* ctx) {
   auto& p = ctx->hp;
-  cudaFree(p.left); cudaFree(p.right); cudaFree(p.token); cudaFree(p.level); cudaFree(p.order);
-  cudaFree(p.n_levels); cudaFree(p.root_ids); cudaFree(p.n_roots); cudaFree(p.h); cudaFree(p.c);
-  cudaFree(p.root_h); cudaFree(p.root_c); cudaFree(p.ws);
+  cudaFree(p.forest); cudaFree(p.level); cudaFree(p.order);
+  cudaFree(p.n_levels); cudaFree(p.roots_pack); cudaFree(p.n_roots); cudaFree(p.h); cudaFree(p.c);
+  cudaFree(p.ws);
   p = treelstm::HostPath{};
 }
 
@@ -326,12 +326,12 @@ int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, con
     free_host_path(ctx);
     const size_t cap = n_nodes < 1024 ? 1024 : (size_t)n_nodes + n_nodes / 4;
     p.ws_bytes = ws_layout(ctx, (int)cap, false).total;
-    if (cudaMalloc((void**)&p.left, 4 * cap) != cudaSuccess || cudaMalloc((void**)&p.right, 4 * cap) != cudaSuccess ||
-        cudaMalloc((void**)&p.token, 4 * cap) != cudaSuccess || cudaMalloc((void**)&p.level, 4 * cap) != cudaSuccess ||
+    // the three forest arrays share one buffer, the root outputs another: when the caller's host
+    // arrays are adjacent in the same way, each group moves in a single copy
+    if (cudaMalloc((void**)&p.forest, 12 * cap) != cudaSuccess || cudaMalloc((void**)&p.level, 4 * cap) != cudaSuccess ||
         cudaMalloc((void**)&p.order, 4 * cap) != cudaSuccess || cudaMalloc((void**)&p.n_levels, 256) != cudaSuccess ||
-        cudaMalloc((void**)&p.root_ids, 4 * cap) != cudaSuccess || cudaMalloc((void**)&p.n_roots, 256) != cudaSuccess ||
+        cudaMalloc((void**)&p.roots_pack, (4 + 8 * H) * cap) != cudaSuccess || cudaMalloc((void**)&p.n_roots, 256) != cudaSuccess ||
         cudaMalloc((void**)&p.h, 4 * cap * H) != cudaSuccess || cudaMalloc((void**)&p.c, 4 * cap * H) != cudaSuccess ||
-        cudaMalloc((void**)&p.root_h, 4 * cap * H) != cudaSuccess || cudaMalloc((void**)&p.root_c, 4 * cap * H) != cudaSuccess ||
         cudaMalloc(&p.ws, p.ws_bytes) != cudaSuccess) {
       ctx->cuda_error = (int)cudaGetLastError();
       free_host_path(ctx);
@@ -340,10 +340,15 @@ int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, con
     p.cap_nodes = (int)cap;
   }
   const size_t nb = 4 * (size_t)n_nodes;
+  p.left = p.forest; p.right = p.forest + n_nodes; p.token = p.forest + 2 * (size_t)n_nodes;
   if (n_nodes > 0) {
-    TL_CUDA(ctx, cudaMemcpyAsync(p.left, left, nb, cudaMemcpyHostToDevice, s));
-    TL_CUDA(ctx, cudaMemcpyAsync(p.right, right, nb, cudaMemcpyHostToDevice, s));
-    TL_CUDA(ctx, cudaMemcpyAsync(p.token, token, nb, cudaMemcpyHostToDevice, s));
+    if (right == left + n_nodes && token == right + n_nodes) {
+      TL_CUDA(ctx, cudaMemcpyAsync(p.left, left, 3 * nb, cudaMemcpyHostToDevice, s));
+    } else {
+      TL_CUDA(ctx, cudaMemcpyAsync(p.left, left, nb, cudaMemcpyHostToDevice, s));
+      TL_CUDA(ctx, cudaMemcpyAsync(p.right, right, nb, cudaMemcpyHostToDevice, s));
+      TL_CUDA(ctx, cudaMemcpyAsync(p.token, token, nb, cudaMemcpyHostToDevice, s));
+    }
   }
   int rc = treelstm_forward(ctx, n_nodes, p.left, p.right, p.token, p.h, p.c, p.level, p.order, nullptr,
                             p.n_levels, flags, p.ws, p.ws_bytes, s);
@@ -351,6 +356,9 @@ int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, con
   const int launches_fwd = ctx->launches;
   const bool want_roots = root_ids || root_h || root_c || n_roots;
   int max_r = max_roots < n_nodes ? max_roots : n_nodes;
+  p.root_ids = reinterpret_cast<int32_t*>(p.roots_pack);
+  p.root_h = reinterpret_cast<float*>(p.root_ids + max_r);
+  p.root_c = p.root_h + (size_t)max_r * H;
   if (want_roots) {
     rc = launch_gather_roots(ctx, max_r, p.root_ids, p.root_h, p.root_c, p.n_roots, s);
     if (rc != TREELSTM_OK) return rc;
@@ -361,16 +369,24 @@ int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, con
     if (level) TL_CUDA(ctx, cudaMemcpyAsync(level, p.level, nb, cudaMemcpyDeviceToHost, s));
     if (order) TL_CUDA(ctx, cudaMemcpyAsync(order, p.order, nb, cudaMemcpyDeviceToHost, s));
   }
-  if (n_levels) TL_CUDA(ctx, cudaMemcpyAsync(n_levels, p.n_levels, 4, cudaMemcpyDeviceToHost, s));
   if (want_roots && max_r > 0) {
     // the number of roots is not known on the host yet: copy max_r rows (rows past n_roots are
     // unspecified) - callers pass the number of trees they submitted
-    if (root_ids) TL_CUDA(ctx, cudaMemcpyAsync(root_ids, p.root_ids, 4 * (size_t)max_r, cudaMemcpyDeviceToHost, s));
-    if (root_h) TL_CUDA(ctx, cudaMemcpyAsync(root_h, p.root_h, 4 * (size_t)max_r * H, cudaMemcpyDeviceToHost, s));
-    if (root_c) TL_CUDA(ctx, cudaMemcpyAsync(root_c, p.root_c, 4 * (size_t)max_r * H, cudaMemcpyDeviceToHost, s));
+    if (root_ids && root_h && root_c && max_r == max_roots &&
+        root_h == reinterpret_cast<float*>(root_ids + max_r) && root_c == root_h + (size_t)max_r * H) {
+      TL_CUDA(ctx, cudaMemcpyAsync(root_ids, p.root_ids, (4 + 8 * H) * (size_t)max_r, cudaMemcpyDeviceToHost, s));
+    } else {
+      if (root_ids) TL_CUDA(ctx, cudaMemcpyAsync(root_ids, p.root_ids, 4 * (size_t)max_r, cudaMemcpyDeviceToHost, s));
+      if (root_h) TL_CUDA(ctx, cudaMemcpyAsync(root_h, p.root_h, 4 * (size_t)max_r * H, cudaMemcpyDeviceToHost, s));
+      if (root_c) TL_CUDA(ctx, cudaMemcpyAsync(root_c, p.root_c, 4 * (size_t)max_r * H, cudaMemcpyDeviceToHost, s));
+    }
   }
-  if (n_roots) TL_CUDA(ctx, cudaMemcpyAsync(n_roots, p.n_roots, 4, cudaMemcpyDeviceToHost, s));
+  // the level and root counts come back with the control block that the status read copies anyway
   rc = treelstm_status_sync(ctx);
+  const DevStatus* hs = reinterpret_cast<const DevStatus*>(ctx->host_status);
+  const bool ok = rc == TREELSTM_OK;
+  if (n_levels) *n_levels = ok ? hs->n_levels : 0;
+  if (n_roots) *n_roots = ok ? (hs->n_roots < max_r ? hs->n_roots : max_r) : 0;
   ctx->launches = launches_fwd + (want_roots ? 1 : 0);
   return rc;
 }

@@ -124,8 +124,10 @@ struct treelstm {
   // buffers of treelstm_forward_host (library-owned, grown on demand)
   struct HostPath {
     int cap_nodes = 0;
+    int32_t *forest = nullptr;       // [left | right | token] of the current call, packed
+    unsigned char* roots_pack = nullptr;   // [root ids | root h | root c] of the current call, packed
     int32_t *left = nullptr, *right = nullptr, *token = nullptr, *level = nullptr, *order = nullptr,
-            *n_levels = nullptr, *root_ids = nullptr, *n_roots = nullptr;
+            *n_levels = nullptr, *root_ids = nullptr, *n_roots = nullptr;   // left .. token, root_* point into the packs
     float *h = nullptr, *c = nullptr, *root_h = nullptr, *root_c = nullptr;
     void* ws = nullptr;
     size_t ws_bytes = 0;

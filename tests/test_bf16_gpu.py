@@ -214,7 +214,7 @@ def test_subforest_mode_through_the_host_entry_point():
     params = fg.draw_params(rng, 128, 64, 300, emb_dist="normal", emb_scale=0.3, w_scale=0.1)
     forest = fg.random_forest(rng, 9, 1, 40, 300)
     model = util.make_model(params, "bf16")
-    host = [torch.from_numpy(a).pin_memory() for a in (forest.left, forest.right, forest.token)]
+    host = binding.pack_forest_host(forest.left, forest.right, forest.token)   # adjacent arrays: single-copy path
     out = model.forward_host(*host, flags=binding.SUBFORESTS, all_states=True, max_roots=forest.n_trees)
     assert model.last_mode() == binding.SUBFORESTS
     h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
