@@ -239,3 +239,22 @@ def test_subforest_mode_large_forest_falls_back():
     h, c, _ = orc.forward_recursive(sub.left, sub.right, sub.token, params.emb, params.W, params.b)
     ids = np.nonzero(np.isin(forest.tree_of, sample))[0]
     assert util.max_abs(res["h"][ids], h) < util.TOL["bf16"]
+
+
+def test_all_modes_give_identical_states():
+    """how the ready nodes are grouped into launches, tiles or sub-forests must not change a single
+    bit of the result (the paper's recursive and iterative executions are numerically identical,
+    Section 6.2): every node's contraction runs over the same K blocks in the same order"""
+    rng = np.random.default_rng(48)
+    for H, E, n_trees, hi in ((256, 50, 120, 12), (150, 64, 300, 56), (64, 300, 30, 130), (192, 16, 2, 40)):
+        params = fg.draw_params(rng, H, E, 500, emb_dist="normal", emb_scale=0.3, w_scale=0.1)
+        forest = fg.random_forest(rng, n_trees, 1, hi, 500)
+        forest, _ = fg.permute_node_ids(forest, rng)
+        model = util.make_model(params, "bf16")
+        ref = util.gpu_forward(model, forest, binding.PERSISTENT)
+        for flags in (binding.PER_LEVEL, binding.SUBFORESTS, binding.PERSISTENT):
+            res = util.gpu_forward(model, forest, flags)
+            np.testing.assert_array_equal(res["h"], ref["h"])
+            np.testing.assert_array_equal(res["c"], ref["c"])
+            np.testing.assert_array_equal(res["order"], ref["order"])
+        model.close()
