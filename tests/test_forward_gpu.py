@@ -199,3 +199,20 @@ def test_bounded_waits_time_out_cleanly():
     model.set_option(binding.OPT_WAIT_LIMIT_CYCLES, 1 << 20)
     res = util.gpu_forward(model, w.forest, binding.PERSISTENT)
     assert util.max_abs(res["h"], ref["h"]) < util.TOL["fp32"]
+
+
+@pytest.mark.parametrize("H,E", [(33, 7), (170, 20), (200, 12), (96, 300)])
+def test_fp32_persistent_odd_and_large_hidden_sizes(H, E):
+    """hidden sizes that end in a partial 16-unit slice (33), odd sizes (scalar operand fetch), sizes
+    whose weight slice still fits in shared memory (170) and sizes where it does not (200: the kernel
+    streams the weights as in per-level mode); both modes against the oracle, and against each other"""
+    rng = np.random.default_rng(H * 1000 + E)
+    params = fg.draw_params(rng, H, E, 60, emb_dist="uniform", emb_scale=0.5, w_scale=0.3 / np.sqrt(H / 16))
+    forest = fg.random_forest(rng, 40, 1, 30, 60)      # wide leaf wavefront (64-row tiles) and narrow ones
+    forest, _ = fg.permute_node_ids(forest, rng)
+    model = util.make_model(params, "fp32")
+    h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
+    for flags in (binding.PER_LEVEL, binding.PERSISTENT):
+        res = util.gpu_forward(model, forest, flags)
+        assert util.max_abs(res["h"], h) < util.TOL["fp32"]
+        assert util.max_abs(res["c"], c) < util.TOL["fp32"]
