@@ -117,24 +117,32 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, const EpiTile& 
         }
       }
       const float* bq = reinterpret_cast<const float*>(bcur);
+      // every step over all four units before the next one: twenty independent activations in flight
+      if (leaf) {
+        float z[12];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        if (leaf) {
-          gi[j] = act_sigmoid(__uint_as_float(v[j]) + bq[j]);
-          go[j] = act_sigmoid(__uint_as_float(v[4 + j]) + bq[4 + j]);
-          gu[j] = act_tanh(__uint_as_float(v[8 + j]) + bq[8 + j]);
-          gfl[j] = gfr[j] = 0.f;
-          cv[j] = gi[j] * gu[j];
-        } else {
-          gi[j] = act_sigmoid(__uint_as_float(v[j]) + bq[j]);
-          gfl[j] = act_sigmoid(__uint_as_float(v[4 + j]) + bq[4 + j]);
-          gfr[j] = act_sigmoid(__uint_as_float(v[8 + j]) + bq[8 + j]);
-          go[j] = act_sigmoid(__uint_as_float(v[12 + j]) + bq[12 + j]);
-          gu[j] = act_tanh(__uint_as_float(v[16 + j]) + bq[16 + j]);
-          cv[j] = gi[j] * gu[j] + gfl[j] * cl[j] + gfr[j] * cr[j];
+        for (int j = 0; j < 12; ++j) z[j] = __uint_as_float(v[j]) + bq[j];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { gi[j] = act_sigmoid(z[j]); go[j] = act_sigmoid(z[4 + j]); gu[j] = act_tanh(z[8 + j]); }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { gfl[j] = gfr[j] = 0.f; cv[j] = gi[j] * gu[j]; }
+      } else {
+        float z[20];
+#pragma unroll
+        for (int j = 0; j < 20; ++j) z[j] = __uint_as_float(v[j]) + bq[j];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          gi[j] = act_sigmoid(z[j]); gfl[j] = act_sigmoid(z[4 + j]); gfr[j] = act_sigmoid(z[8 + j]);
+          go[j] = act_sigmoid(z[12 + j]); gu[j] = act_tanh(z[16 + j]);
         }
-        hv[j] = go[j] * act_tanh(cv[j]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) cv[j] = gi[j] * gu[j] + gfl[j] * cl[j] + gfr[j] * cr[j];
       }
+      float tcv[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) tcv[j] = act_tanh(cv[j]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) hv[j] = go[j] * tcv[j];
       if (staged_out) {
         *reinterpret_cast<float4*>(mine + (((2 * g + e) ^ (r & 7)) << 4)) = make_float4(cv[0], cv[1], cv[2], cv[3]);
         *reinterpret_cast<float4*>(mine + (((half + 2 * g + e) ^ (r & 7)) << 4)) = make_float4(hv[0], hv[1], hv[2], hv[3]);
