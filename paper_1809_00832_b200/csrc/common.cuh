@@ -205,11 +205,18 @@ __device__ __forceinline__ int ld_volatile(const int* p) { return *(const volati
 // (arrivals on one counter are served one after the other, so fewer of them end the barrier sooner).
 // Returns false if the wait expired or another CTA reported an error: the caller must then
 // leave its level loop (every CTA sees the same outcome within one more barrier).
-__device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
-                                             long long limit_cycles, int* s_flag, bool arrive = true,
-                                             unsigned int* counter = nullptr) {
+// The threads outside warp 0 run `while_waiting` between the arrival and the release.  A thread that
+// wants to act the moment the barrier is complete, ahead of the CTA-wide wake-up, watches *s_early
+// there: the polling lane that sees the last arrival stores `target` (unique per barrier) into it,
+// 0xFFFFFFFF if the barrier failed.
+template <class WaitFn>
+__device__ __forceinline__ bool grid_barrier_with(DevStatus* st, unsigned int target,
+                                                  long long limit_cycles, int* s_flag, bool arrive,
+                                                  unsigned int* counter, unsigned int* s_early,
+                                                  WaitFn while_waiting) {
   if (!counter) counter = &st->barrier;
   __syncthreads();
+  if (threadIdx.x >= 32) while_waiting();
   if (threadIdx.x < 32) {
     // Warp 0 polls.  Lane 0 announces the arrival (release: everything this CTA wrote, ordered
     // before by the CTA barrier, is visible to whoever acquires the counter afterwards); then eight
@@ -228,10 +235,19 @@ __device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
         if (*(volatile int*)s_flag >= 0) break;          // another lane has the answer
         unsigned int seen;
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
-        if (seen >= target) { *(volatile int*)s_flag = 1; break; }
-        if (*(volatile int*)&st->status != 0) { *(volatile int*)s_flag = 0; break; }
+        if (seen >= target) {
+          if (s_early) { __threadfence_block(); *(volatile unsigned int*)s_early = target; }
+          *(volatile int*)s_flag = 1;
+          break;
+        }
+        if (*(volatile int*)&st->status != 0) {
+          if (s_early) *(volatile unsigned int*)s_early = 0xFFFFFFFFu;
+          *(volatile int*)s_flag = 0;
+          break;
+        }
         if (clock64() - t0 > limit_cycles) {
           report(st, TREELSTM_ERR_TIMEOUT);
+          if (s_early) *(volatile unsigned int*)s_early = 0xFFFFFFFFu;
           *(volatile int*)s_flag = 0;
           break;
         }
@@ -241,6 +257,12 @@ __device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
   }
   __syncthreads();
   return *s_flag != 0;
+}
+
+__device__ __forceinline__ bool grid_barrier(DevStatus* st, unsigned int target,
+                                             long long limit_cycles, int* s_flag, bool arrive = true,
+                                             unsigned int* counter = nullptr) {
+  return grid_barrier_with(st, target, limit_cycles, s_flag, arrive, counter, nullptr, []() {});
 }
 #endif
 

@@ -142,6 +142,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   int* s_rowslot = s_rownode + BM;                                                   // [128] its delivery slot
   int* s_level_offset = s_rowslot + BM;   // first kLevelCache wavefront boundaries: no global round trip per level
   __shared__ TilePlan s_plan[2];          // tile plans of this and the next wavefront (written by warp 11)
+  __shared__ unsigned int s_early;        // grid barrier: completion seen by the polling lane (see grid_barrier_with)
+  __shared__ unsigned int s_pre;          // bit 0 / 1: first weight / operand box of the next wavefront requested ahead
   unsigned char* cstage_w = tiles_ptr + kRingBytes;
   const uint32_t epi_bar = smem_u32(bars + 2 * kMaxStages + 4);
   uint32_t epi_phase = 0;
@@ -160,6 +162,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
     mbar_init(epi_bar, 256);
     *s_abort = 0;
+    s_early = 0u;
+    s_pre = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   for (int i = tid; i < kLevelCache && i <= n_levels; i += kThreads) s_level_offset[i] = p.level_offset[i];
@@ -182,6 +186,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   uint32_t arrivals = 0;                // arrivals at the grid barrier expected so far
   bool alive = true;
   bool stop = false;                    // uniform over the CTA
+  bool pre = false;                     // producers: this warp's first box of the wavefront was requested at the barrier
 
   if (only_level < 0 && n_levels > 0) {
     prepare_operands(p, blockIdx.x * kThreads + tid, gridDim.x * kThreads);
@@ -252,6 +257,13 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
           const uint32_t off = is_a ? 0u : (uint32_t)kbox * a_bytes;
           const int y = is_a ? row0 : nt * ncols;
           for (int box = 0; box < n_box; ++box) {
+            if (pre) {   // requested at the grid barrier
+              pre = false;
+              atomicAnd(&s_pre, is_a ? ~2u : ~1u);
+              phase_bits ^= 1u << stage;
+              if (++stage == n_stages) stage = 0;
+              continue;
+            }
             if (!mbar_wait(empty_bar(stage), ((phase_bits >> stage) & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) {
               alive = false;
               break;
@@ -349,13 +361,63 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
       if (*s_abort) break;
       // only the CTAs that had a tile in this wavefront wrote anything: they arrive, the rest just wait
       arrivals += (uint32_t)min(tiles, (int)gridDim.x);
-      if (!grid_barrier(p.st, arrivals, p.wait_limit, s_flag, (int)blockIdx.x < tiles)) break;
+      // The first box of this CTA's first tile of the next wavefront is requested at the barrier, into
+      // stage 0 of the re-cut ring (every MMA of this wavefront has retired: the epilogue waited for
+      // them).  The weights do not depend on the wavefront before, so their producer asks at once;
+      // the operand producer prepares its request and sends it the moment the polling lane reports
+      // the barrier complete, ahead of the CTA-wide wake-up and the tile set-up.
+      const uint32_t target = arrivals;
+      const bool passed = grid_barrier_with(p.st, target, p.wait_limit, s_flag, (int)blockIdx.x < tiles, nullptr, &s_early, [&]() {
+        if (lane != 0 || (warp != 4 && warp != 10)) return;
+        const TilePlan np = s_plan[(lvl + 1) & 1];
+        const int t = blockIdx.x;
+        if (t >= np.tiles) return;
+        int lg = np.lg, fat = t, piece = 0;
+        if (t >= np.tail_from) {
+          const int u = t - np.tail_from;
+          fat = np.tail_from + (u >> np.tail_ls);
+          piece = u & ((1 << np.tail_ls) - 1);
+          lg -= np.tail_ls;
+        }
+        const int ntn2 = groups >> np.lg;
+        const int rtile = fat / ntn2;
+        if (!mbar_wait(empty_bar(0), (phase_bits & 1u) ^ 1u, s_abort, p.wait_limit, p.st)) return;
+        if (warp == 10) {
+          const int nt = ((fat - rtile * ntn2) << (np.lg - lg)) + piece;
+          const int ncols = (1 << lg) * kGColsI;
+          mbar_arrive_expect_tx(full_bar(0), (uint32_t)np.kbox * (uint32_t)ncols * 128u);
+          tma_load_3d(tiles_addr + (uint32_t)np.kbox * np.a_bytes, &maps.wh[lg][np.sel], 0, nt * ncols, 0, full_bar(0));
+          atomicOr(&s_pre, 1u);
+          pre = true;
+        } else {
+          const int row0 = level_begin(lvl + 1) + (rtile << np.lrt);
+          const CUtensorMap* map = &maps.a[np.lrt - 5][np.sel];
+          const long long t0 = clock64();
+          unsigned int seen;
+          while ((seen = *(volatile unsigned int*)&s_early) != target) {
+            if (seen == 0xFFFFFFFFu || clock64() - t0 > p.wait_limit) return;
+          }
+          __threadfence_block();
+          mbar_arrive_expect_tx(full_bar(0), (uint32_t)np.kbox * np.a_bytes);
+          tma_load_3d(tiles_addr, map, 0, row0, 0, full_bar(0));
+          atomicOr(&s_pre, 2u);
+          pre = true;
+        }
+      });
+      if (!passed) break;
     }
   }
 
   // teardown: let in-flight asynchronous copies land before shared/tensor memory is released
   asm volatile("cp.async.wait_all;" ::: "memory");
   tc_fence_before();
+  __syncthreads();
+  if (warp == 10 && lane == 0 && s_pre != 0u) {
+    // the loop was left with a box requested ahead still in flight: stand in for the arrival of the
+    // producer that did not ask, and let the data land
+    if (s_pre != 3u) mbar_arrive(full_bar(0));
+    mbar_wait(full_bar(0), phase_bits & 1u, s_abort, p.wait_limit, p.st);
+  }
   __syncthreads();
   if (*s_abort) __nanosleep(100000);
   if (warp == 5) {
