@@ -258,3 +258,23 @@ def test_all_modes_give_identical_states():
             np.testing.assert_array_equal(res["c"], ref["c"])
             np.testing.assert_array_equal(res["order"], ref["order"])
         model.close()
+
+
+def test_bf16_deeper_than_the_level_cache():
+    """a left chain of 1100 leaves next to a few small trees: 1100 wavefronts, more than the kernels
+    keep wavefront boundaries for in shared memory (the rest is read from global memory, and the
+    sub-forest kernel spills its per-sub-forest table); all modes still agree bit for bit and stay
+    within the bf16 tolerance of the oracle over that depth"""
+    rng = np.random.default_rng(1100)
+    params = fg.draw_params(rng, 64, 32, 200, emb_dist="normal", emb_scale=0.3, w_scale=0.1)
+    shapes = [fg.left_chain_shape(1100), fg.balanced_shape(16), None, fg.left_chain_shape(7)]
+    forest = fg.forest_from_shapes(shapes, rng, 200)
+    forest, _ = fg.permute_node_ids(forest, rng)
+    ref = None
+    for flags in (binding.PERSISTENT, binding.SUBFORESTS, binding.PER_LEVEL):
+        res = _check(params, forest, flags)
+        assert res["n_levels"] == 1100
+        if ref is None:
+            ref = res
+        np.testing.assert_array_equal(res["h"], ref["h"])
+        np.testing.assert_array_equal(res["c"], ref["c"])
