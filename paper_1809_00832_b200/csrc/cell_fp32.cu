@@ -166,14 +166,15 @@ __device__ void fp32_tile(const FwdParams& p, int row0, int row_end, int u0, boo
 // shared memory (red[4][TMS][5 * TU]).  Same cell update as fp32_tile.
 template <int TM>
 __device__ void fp32_tile_stationary(const FwdParams& p, int row0, int row_end, int u0, float* As,
-                                     const float* Ws, float* red, int* s_node, int* s_l, int* s_r) {
+                                     const float* Ws, float* red, int* s_node, int* s_l, int* s_r,
+                                     bool ids_ready = false) {
   constexpr bool kSplit = TM == TMS;
   constexpr int RPT = 4, NQ = kSplit ? 4 : 1;
   const int tid = threadIdx.x, tx = tid % TU, ty = tid / TU;
   const int rg = kSplit ? (ty & 3) : ty, kq = kSplit ? (ty >> 2) : 0;
   const int H = p.H, K = 2 * H, K4 = (K + 3) & ~3, a_row = p.a_row, w_row = p.w_row;
   __syncthreads();  // previous tile's readers of As, red and the index arrays are done
-  for (int i = tid; i < TM; i += kThreads) {
+  for (int i = tid; i < TM && !ids_ready; i += kThreads) {   // ids_ready: fetched while the grid barrier was pending
     const int row = row0 + i;
     int node = -1, l = 0, r = 0;
     if (row < row_end) { node = p.order[row]; l = p.left[node]; r = p.right[node]; }
@@ -336,6 +337,7 @@ k_fwd_fp32_persistent(FwdParams p) {
       Ws[col * w_row + k] = v;
     }
   }
+  bool ids_ahead = false;   // uniform: the row ids of this CTA's first tile of the wavefront are in shared memory
   for (int lvl = 0; lvl < n_levels; ++lvl) {
     const int begin = p.level_offset[lvl], end = p.level_offset[lvl + 1];
     const int tmr = rows_per_tile(end - begin, tiles_u, p.n_sms);
@@ -343,16 +345,36 @@ k_fwd_fp32_persistent(FwdParams p) {
     for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
       const int tm = t / tiles_u, u0 = (t - tm * tiles_u) * TU;
       if (lvl > 0 && p.w_stationary) {
-        if (tmr == TM) fp32_tile_stationary<TM>(p, begin + tm * TM, end, u0, As, Ws, red, s_node, s_l, s_r);
-        else fp32_tile_stationary<TMS>(p, begin + tm * TMS, end, u0, As, Ws, red, s_node, s_l, s_r);
+        const bool ready = ids_ahead && t == (int)blockIdx.x;
+        if (tmr == TM) fp32_tile_stationary<TM>(p, begin + tm * TM, end, u0, As, Ws, red, s_node, s_l, s_r, ready);
+        else fp32_tile_stationary<TMS>(p, begin + tm * TMS, end, u0, As, Ws, red, s_node, s_l, s_r, ready);
       } else {
         if (tmr == TM) fp32_tile<TM>(p, begin + tm * TM, end, u0, lvl == 0, s);
         else fp32_tile<TMS>(p, begin + tm * TMS, end, u0, lvl == 0, s);
       }
     }
-    if (lvl + 1 < n_levels &&
-        !grid_barrier(p.st, (unsigned)(lvl + 1) * gridDim.x, p.wait_limit, &s_flag))
-      return;
+    if (lvl + 1 < n_levels) {
+      // Which rows the next wavefront holds and who their children are is the scheduler's output and
+      // does not depend on the wavefront just finished: threads outside the polling warp fetch the
+      // ids of this CTA's first tile of the next wavefront while the barrier is pending (three
+      // dependent loads off the path that follows the barrier).
+      const bool passed = grid_barrier_with(
+          p.st, (unsigned)(lvl + 1) * gridDim.x, p.wait_limit, &s_flag, true, nullptr, nullptr, [&]() {
+            if (!p.w_stationary) return;
+            const int i = (int)threadIdx.x - 32;
+            if (i >= TM) return;
+            const int nb = p.level_offset[lvl + 1], ne = p.level_offset[lvl + 2];
+            const int tmr2 = rows_per_tile(ne - nb, tiles_u, p.n_sms);
+            const int tiles2 = ((ne - nb + tmr2 - 1) / tmr2) * tiles_u;
+            if ((int)blockIdx.x >= tiles2 || i >= tmr2) return;
+            const int row = nb + ((int)blockIdx.x / tiles_u) * tmr2 + i;
+            int node = -1, l = 0, r = 0;
+            if (row < ne) { node = p.order[row]; l = p.left[node]; r = p.right[node]; }
+            s_node[i] = node; s_l[i] = l; s_r[i] = r;
+          });
+      if (!passed) return;
+      ids_ahead = p.w_stationary != 0;
+    }
   }
 }
 
