@@ -472,8 +472,15 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
     classifier_groups(p, blockIdx.x - 1, gridDim.x - 1, s_cls);
   }
   if (!barrier()) return;
+  // the first wavefront boundaries in shared memory: no dependent global load after every barrier
+  // (filled here, ordered before its first use by the CTA barriers inside the grid barrier above)
+  constexpr int kOffCache = 256;
+  __shared__ int s_off[kOffCache];
+  for (int i = threadIdx.x; i < kOffCache && i <= n_levels; i += blockDim.x) s_off[i] = level_offset[i];
+  __syncthreads();
+  auto level_begin = [&](int l) { return l < kOffCache ? s_off[l] : level_offset[l]; };
   for (int lvl = n_levels - 1; lvl >= 0; --lvl) {
-    const int begin = level_offset[lvl], end = level_offset[lvl + 1], leaf = lvl == 0 ? 1 : 0;
+    const int begin = level_begin(lvl), end = level_begin(lvl + 1), leaf = lvl == 0 ? 1 : 0;
     const long long elems = (long long)(end - begin) * H;
     for (long long idx = (long long)gtid; idx < elems; idx += (long long)gthreads) gates_element(p, begin, idx, leaf);
     if (!barrier()) return;

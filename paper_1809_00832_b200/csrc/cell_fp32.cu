@@ -337,9 +337,15 @@ k_fwd_fp32_persistent(FwdParams p) {
       Ws[col * w_row + k] = v;
     }
   }
+  // the first wavefront boundaries in shared memory: no dependent global load after every barrier
+  constexpr int kOffCache = 256;
+  __shared__ int s_off[kOffCache];
+  for (int i = threadIdx.x; i < kOffCache && i <= n_levels; i += kThreads) s_off[i] = p.level_offset[i];
+  __syncthreads();
+  auto level_begin = [&](int l) { return l < kOffCache ? s_off[l] : p.level_offset[l]; };
   bool ids_ahead = false;   // uniform: the row ids of this CTA's first tile of the wavefront are in shared memory
   for (int lvl = 0; lvl < n_levels; ++lvl) {
-    const int begin = p.level_offset[lvl], end = p.level_offset[lvl + 1];
+    const int begin = level_begin(lvl), end = level_begin(lvl + 1);
     const int tmr = rows_per_tile(end - begin, tiles_u, p.n_sms);
     const int tiles = ((end - begin + tmr - 1) / tmr) * tiles_u;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
@@ -363,7 +369,7 @@ k_fwd_fp32_persistent(FwdParams p) {
             if (!p.w_stationary) return;
             const int i = (int)threadIdx.x - 32;
             if (i >= TM) return;
-            const int nb = p.level_offset[lvl + 1], ne = p.level_offset[lvl + 2];
+            const int nb = level_begin(lvl + 1), ne = level_begin(lvl + 2);
             const int tmr2 = rows_per_tile(ne - nb, tiles_u, p.n_sms);
             const int tiles2 = ((ne - nb + tmr2 - 1) / tmr2) * tiles_u;
             if ((int)blockIdx.x >= tiles2 || i >= tmr2) return;
