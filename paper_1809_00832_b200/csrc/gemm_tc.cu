@@ -106,14 +106,29 @@ __host__ __device__ inline TilePlan choose_tile_plan(int rows, int groups, int n
 //     (where that child will deliver its state), slot[root] = -1.
 __device__ void prepare_operands(const TcParams& p, int gtid, int gthreads) {
   const int n_leaves = p.level_offset[1];
+  // the dependent loads of this thread's first slot entries and root go out before the gather, so
+  // that the two chains of round trips run side by side
+  const int pos0 = n_leaves + gtid;
+  int l0 = -1, r0 = -1, root0 = -1;
+  if (pos0 < p.n) {
+    const int node = p.order[pos0];
+    l0 = p.left[node];
+    r0 = p.right[node];
+  }
+  const int n_roots = p.st->n_roots;
+  if (gtid < n_roots) root0 = p.roots[gtid];
   gather_leaf_rows(p, 0, n_leaves, gtid >> 5, gthreads >> 5, gtid & 31);
-  for (int pos = n_leaves + gtid; pos < p.n; pos += gthreads) {
+  if (l0 >= 0) {
+    p.slot[l0] = 2 * pos0;
+    p.slot[r0] = 2 * pos0 + 1;
+  }
+  for (int pos = pos0 + gthreads; pos < p.n; pos += gthreads) {
     const int node = p.order[pos];
     p.slot[p.left[node]] = 2 * pos;
     p.slot[p.right[node]] = 2 * pos + 1;
   }
-  const int n_roots = p.st->n_roots;
-  for (int t = gtid; t < n_roots; t += gthreads) p.slot[p.roots[t]] = -1;
+  if (root0 >= 0) p.slot[root0] = -1;
+  for (int t = gtid + gthreads; t < n_roots; t += gthreads) p.slot[p.roots[t]] = -1;
 }
 
 __global__ void k_prepare_operands(TcParams p) {
