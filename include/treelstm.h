@@ -52,7 +52,8 @@ typedef enum treelstm_status {
   TREELSTM_ERR_CUDA = -6,               /* a CUDA runtime call failed; see treelstm_last_cuda_error */
   TREELSTM_ERR_NO_DEVICE = -7,          /* no sm_100 device is current                               */
   TREELSTM_ERR_UNSUPPORTED = -8,        /* size outside what the kernels support                     */
-  TREELSTM_ERR_STATE = -9               /* call order violated (e.g. backward without forward)       */
+  TREELSTM_ERR_STATE = -9               /* call order violated (e.g. backward without forward), or   */
+                                        /* the current device is not the one the context was made on */
 } treelstm_status;
 
 /* precision of the gate contraction */
@@ -193,8 +194,9 @@ TREELSTM_API int treelstm_backward(treelstm_t* ctx, const int32_t* labels, float
 /*
  * treelstm_forward_host - the same forward for callers whose data lives in HOST memory: copies
  * the forest to the device, runs treelstm_forward with `flags`, copies the requested results
- * back and synchronises.  Device staging and workspace buffers are owned by the context and
- * grown on demand (cudaMalloc on the first call or when n_nodes grows).
+ * back and synchronises.  Device staging and workspace come from the buffer given with
+ * treelstm_set_host_staging; without one they are owned by the context and grown on demand
+ * (cudaMalloc on the first call or when n_nodes grows).
  *   left,right,token [host][n_nodes] in (pinned memory makes the copies asynchronous).
  *   h, c           [host][n_nodes][H] out, or NULL to skip the all-node states.
  *   level, order   [host][n_nodes] out, or NULL.
@@ -210,6 +212,22 @@ TREELSTM_API int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32
                           const int32_t* token, float* h, float* c, int32_t* level, int32_t* order,
                           int32_t* n_levels, int max_roots, int32_t* root_ids, float* root_h,
                           float* root_c, int32_t* n_roots, int flags, void* stream);
+
+/*
+ * treelstm_host_staging_bytes / treelstm_set_host_staging - let the caller own the device memory
+ * treelstm_forward_host stages through (forest arrays, schedule, all-node states, root pack,
+ * workspace), so that the library allocates nothing on that path either.  (Plumbing; the paper has
+ * no counterpart.)
+ *   treelstm_host_staging_bytes: bytes needed for forests of up to max_nodes nodes (0 on invalid
+ *   arguments).
+ *   treelstm_set_host_staging: device_buffer is 256-byte aligned device memory of `bytes` bytes that
+ *   stays valid until it is replaced, withdrawn (device_buffer = NULL: the library goes back to its
+ *   own buffers) or the context is destroyed; the library never frees it.  A later
+ *   treelstm_forward_host whose forest needs more than `bytes` returns TREELSTM_ERR_INVALID_ARG and
+ *   launches nothing.
+ */
+TREELSTM_API size_t treelstm_host_staging_bytes(const treelstm_t* ctx, int max_nodes);
+TREELSTM_API int treelstm_set_host_staging(treelstm_t* ctx, void* device_buffer, size_t bytes);
 
 /*
  * treelstm_schedule_static - the ready-set construction of treelstm_forward on its own, for
@@ -234,8 +252,9 @@ TREELSTM_API int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32
  *   status        [1] out (device): TREELSTM_OK, TREELSTM_ERR_INVALID_FOREST or
  *                 TREELSTM_ERR_TOKEN_OUT_OF_RANGE as found by the kernel; read it after the stream
  *                 has finished.  On an error the other outputs are unspecified.
- * The call only enqueues work on `stream` (two small memory operations and one kernel); it never
- * calls cudaMalloc, cudaFree or any routine that allocates.  The first call on each device looks
+ * The call only enqueues work on `stream` (one kernel and one 4-byte copy of the status word; for
+ * the empty forest three small memory sets and that copy); it never calls cudaMalloc, cudaFree or
+ * any routine that allocates.  The first call on each device looks
  * up the device address of the built-in scratch array (with that device current); make that first
  * call outside any stream capture.  All calls on a device share the one scratch array, and it keeps
  * whatever the previous call left there - the call clears the parts that must start from zero

@@ -52,6 +52,8 @@ SIGNATURES = {
     "treelstm_backward": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "treelstm_forward_host": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp,
                                    _vp, _vp, _i, _vp]),
+    "treelstm_host_staging_bytes": (ctypes.c_size_t, [_vp, _i]),
+    "treelstm_set_host_staging": (_i, [_vp, _vp, ctypes.c_size_t]),
     "treelstm_schedule_static": (_i, [_i, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "treelstm_selftest_waits": (_i, [_vp, _vp, ctypes.c_size_t, _vp, _vp]),
     "treelstm_last_kernel_ms": (_i, [_vp, ctypes.POINTER(ctypes.c_float)]),
@@ -163,6 +165,7 @@ class TreeLSTM:
             raise TreeLSTMError(rc, "treelstm_create")
         self.handle = handle
         self._ws: Optional[torch.Tensor] = None
+        self._host_staging: Optional[torch.Tensor] = None
         self._keep = None
 
     def close(self):
@@ -287,6 +290,17 @@ class TreeLSTM:
         for t in (left, right, token):
             if t.is_cuda or t.dtype != torch.int32 or not t.is_contiguous():
                 raise ValueError("forest arrays must be contiguous CPU int32 tensors")
+        # device staging is torch's memory too: hand the library a buffer large enough for this forest
+        need = int(self.lib.treelstm_host_staging_bytes(self.handle, n))
+        if self._host_staging is None or self._host_staging.numel() < need + 256:
+            grown = torch.empty(need + need // 4 + 256, dtype=torch.uint8, device="cuda")
+            base = grown.data_ptr()
+            aligned = (base + 255) // 256 * 256
+            rc = self.lib.treelstm_set_host_staging(self.handle, ctypes.c_void_p(aligned),
+                                                    grown.numel() - (aligned - base))
+            if rc != OK:
+                raise TreeLSTMError(rc, "treelstm_set_host_staging")
+            self._host_staging = grown
         if out is None:
             pin = dict(pin_memory=True)
             out = dict(n_levels=torch.zeros(1, dtype=torch.int32, **pin),

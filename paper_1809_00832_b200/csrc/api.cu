@@ -58,10 +58,45 @@ int copy_params(treelstm* ctx, const float* emb, const float* W, const float* b,
 
 void free_host_path(treelstm* ctx) {
   auto& p = ctx->hp;
-  cudaFree(p.forest); cudaFree(p.level); cudaFree(p.order);
-  cudaFree(p.n_levels); cudaFree(p.roots_pack); cudaFree(p.n_roots); cudaFree(p.h); cudaFree(p.c);
-  cudaFree(p.ws);
+  if (p.owned) {
+    cudaFree(p.forest); cudaFree(p.level); cudaFree(p.order);
+    cudaFree(p.n_levels); cudaFree(p.roots_pack); cudaFree(p.n_roots); cudaFree(p.h); cudaFree(p.c);
+    cudaFree(p.ws);
+  }
+  unsigned char* ext = p.ext;
+  const size_t ext_bytes = p.ext_bytes;
   p = treelstm::HostPath{};
+  p.ext = ext; p.ext_bytes = ext_bytes;
+}
+
+// Device staging of treelstm_forward_host for forests of up to `cap` nodes: offsets of its parts in
+// one buffer (every part 256-byte aligned) and the total.
+struct HostStaging {
+  size_t forest, level, order, n_levels, roots_pack, n_roots, h, c, ws, ws_bytes, total;
+};
+HostStaging host_staging_layout(const treelstm* ctx, size_t cap) {
+  HostStaging L{};
+  const size_t H = ctx->H;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += round_up_sz(bytes, 256); return o; };
+  L.forest = take(12 * cap);
+  L.level = take(4 * cap);
+  L.order = take(4 * cap);
+  L.n_levels = take(256);
+  L.roots_pack = take((4 + 8 * H) * cap);
+  L.n_roots = take(256);
+  L.h = take(4 * cap * H);
+  L.c = take(4 * cap * H);
+  L.ws_bytes = ws_layout(ctx, (int)cap, false).total;
+  L.ws = take(L.ws_bytes);
+  L.total = off;
+  return L;
+}
+
+// True if the calling thread's current device is the one the context was created on.
+bool on_own_device(const treelstm* ctx) {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess && dev == ctx->device;
 }
 
 // Read the control block and the level table back (one synchronisation).
@@ -150,7 +185,10 @@ int treelstm_create(treelstm_t** out, int H, int E, int vocab, const float* emb,
         cudaMalloc((void**)&ctx->bp_x, 4 * groups * 24) != cudaSuccess)
       return fail(TREELSTM_ERR_CUDA);
   }
-  int rc = copy_params(ctx, emb, W, b, s);
+  int rc = init_schedule_attributes(ctx);
+  if (rc == TREELSTM_OK && precision == TREELSTM_BF16) rc = init_tc_attributes(ctx);
+  if (rc != TREELSTM_OK) return fail(rc);
+  rc = copy_params(ctx, emb, W, b, s);
   if (rc != TREELSTM_OK) return fail(rc);
   ctx->sf = subforest_plan(ctx);
   *out = ctx;
@@ -215,6 +253,7 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
   if (!ctx) return TREELSTM_ERR_INVALID_ARG;
   ctx->last.valid = false;
   ctx->launches = 0;
+  if (!on_own_device(ctx)) return TREELSTM_ERR_STATE;
   if (n_nodes < 0 || !n_levels || !workspace) return TREELSTM_ERR_INVALID_ARG;
   if (n_nodes > 0 && (!left || !right || !token || !h || !c || !level || !order))
     return TREELSTM_ERR_INVALID_ARG;
@@ -241,11 +280,11 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
   int rc = launch_schedule(ctx, n_nodes, left, right, token, level, order, lvl_off, n_levels, workspace,
                            lay, subforests ? ctx->sf.n_parts : 0, s);
   if (rc != TREELSTM_OK) return rc;
+  const bool persistent = (flags & (TREELSTM_PERSISTENT | TREELSTM_SUBFORESTS)) != 0;
+  L.mode = subforests ? TREELSTM_SUBFORESTS : (persistent ? TREELSTM_PERSISTENT : TREELSTM_PER_LEVEL);
   L.valid = true;
   if (n_nodes == 0) return TREELSTM_OK;
 
-  const bool persistent = (flags & (TREELSTM_PERSISTENT | TREELSTM_SUBFORESTS)) != 0;
-  L.mode = subforests ? TREELSTM_SUBFORESTS : (persistent ? TREELSTM_PERSISTENT : TREELSTM_PER_LEVEL);
   if (!persistent) {
     rc = read_levels(ctx);
     if (rc != TREELSTM_OK) { L.valid = false; return rc; }
@@ -307,6 +346,7 @@ int treelstm_backward(treelstm_t* ctx, const int32_t* labels, float* loss, float
     return TREELSTM_ERR_INVALID_ARG;
   if (!ctx->last.valid || !(ctx->last.flags & TREELSTM_SAVE_FOR_BACKWARD) || ctx->C < 1)
     return TREELSTM_ERR_STATE;
+  if (!on_own_device(ctx)) return TREELSTM_ERR_STATE;
   ctx->launches = 0;
   return launch_backward(ctx, labels, loss, dW, db, dWc, dbc, touched_ids, dEmb_rows, n_touched,
                          static_cast<cudaStream_t>(stream));
@@ -320,12 +360,35 @@ int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, con
   if (n_nodes > 0 && (!left || !right || !token)) return TREELSTM_ERR_INVALID_ARG;
   if (flags & TREELSTM_SAVE_FOR_BACKWARD) return TREELSTM_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (!on_own_device(ctx)) return TREELSTM_ERR_STATE;
   auto& p = ctx->hp;
   const size_t H = ctx->H;
-  if (n_nodes > p.cap_nodes || !p.ws) {
+  if (p.ext) {
+    // the caller's staging memory: carved up anew whenever the forest outgrows the last carving
+    if (n_nodes > p.cap_nodes || !p.ws || p.owned) {
+      const size_t cap = n_nodes < 1 ? 1 : (size_t)n_nodes;
+      const HostStaging L = host_staging_layout(ctx, cap);
+      if (L.total > p.ext_bytes) return TREELSTM_ERR_INVALID_ARG;
+      free_host_path(ctx);
+      unsigned char* b = p.ext;
+      p.forest = reinterpret_cast<int32_t*>(b + L.forest);
+      p.level = reinterpret_cast<int32_t*>(b + L.level);
+      p.order = reinterpret_cast<int32_t*>(b + L.order);
+      p.n_levels = reinterpret_cast<int32_t*>(b + L.n_levels);
+      p.roots_pack = b + L.roots_pack;
+      p.n_roots = reinterpret_cast<int32_t*>(b + L.n_roots);
+      p.h = reinterpret_cast<float*>(b + L.h);
+      p.c = reinterpret_cast<float*>(b + L.c);
+      p.ws = b + L.ws;
+      p.ws_bytes = L.ws_bytes;
+      p.cap_nodes = (int)cap;
+      p.owned = false;
+    }
+  } else if (n_nodes > p.cap_nodes || !p.ws) {
     free_host_path(ctx);
     const size_t cap = n_nodes < 1024 ? 1024 : (size_t)n_nodes + n_nodes / 4;
     p.ws_bytes = ws_layout(ctx, (int)cap, false).total;
+    p.owned = true;
     // the three forest arrays share one buffer, the root outputs another: when the caller's host
     // arrays are adjacent in the same way, each group moves in a single copy
     if (cudaMalloc((void**)&p.forest, 12 * cap) != cudaSuccess || cudaMalloc((void**)&p.level, 4 * cap) != cudaSuccess ||
@@ -391,11 +454,27 @@ int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, con
   return rc;
 }
 
+size_t treelstm_host_staging_bytes(const treelstm_t* ctx, int max_nodes) {
+  if (!ctx || max_nodes < 0) return 0;
+  return host_staging_layout(ctx, max_nodes < 1 ? 1 : (size_t)max_nodes).total;
+}
+
+int treelstm_set_host_staging(treelstm_t* ctx, void* device_buffer, size_t bytes) {
+  if (!ctx) return TREELSTM_ERR_INVALID_ARG;
+  if (device_buffer && reinterpret_cast<uintptr_t>(device_buffer) % 256 != 0) return TREELSTM_ERR_INVALID_ARG;
+  free_host_path(ctx);
+  ctx->hp.ext = static_cast<unsigned char*>(device_buffer);
+  ctx->hp.ext_bytes = device_buffer ? bytes : 0;
+  ctx->last.valid = false;
+  return TREELSTM_OK;
+}
+
 int treelstm_selftest_waits(treelstm_t* ctx, void* workspace, size_t workspace_bytes, int32_t* result,
                             void* stream) {
   if (!ctx || !workspace || !result || workspace_bytes < sizeof(DevStatus)) return TREELSTM_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return TREELSTM_ERR_INVALID_ARG;
-  ctx->last.valid = false;   // the control block of an earlier forward is overwritten
+  ctx->last.valid = false;   // the control block of an earlier forward may be the one overwritten
+  ctx->last.ws = nullptr;    // and its workspace is no longer this context's to read
   return launch_selftest_waits(ctx, workspace, result, static_cast<cudaStream_t>(stream));
 }
 

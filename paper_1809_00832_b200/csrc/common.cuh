@@ -131,6 +131,9 @@ struct treelstm {
     float *h = nullptr, *c = nullptr, *root_h = nullptr, *root_c = nullptr;
     void* ws = nullptr;
     size_t ws_bytes = 0;
+    bool owned = false;              // the buffers above were allocated by the library (else carved from `ext`)
+    unsigned char* ext = nullptr;    // caller-provided device staging memory (treelstm_set_host_staging)
+    size_t ext_bytes = 0;
   } hp;
 
   cudaEvent_t ev_begin = nullptr, ev_end = nullptr;  // around the wavefront kernel (optional)
@@ -143,6 +146,11 @@ struct treelstm {
 namespace tl {
 
 WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward);
+
+// Per-device kernel attributes (the opt-in to more than 48 KB of dynamic shared memory belongs to the
+// device that is current when it is set): called by treelstm_create with the context's device current.
+int init_schedule_attributes(treelstm* ctx);   // schedule.cu
+int init_tc_attributes(treelstm* ctx);         // gemm_tc.cu
 
 // schedule.cu: enqueue the on-device ready-set construction.  Returns a treelstm_status.
 int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* right,

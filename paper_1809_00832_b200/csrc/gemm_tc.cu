@@ -150,7 +150,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + kRingBytes + kCBytes);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
   // bars[2S+4]: meeting point of the 256 epilogue threads (output staging)
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 5);
+  // bars[2S+5]: teardown after a failed wait - the MMA issuer's last commit
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 6);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   int* s_flag = const_cast<int*>(s_abort) + 1;
   int* s_rownode = reinterpret_cast<int*>(tiles_ptr + kRingBytes + kCBytes + 256);   // [128] node id of each tile row
@@ -161,6 +162,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   __shared__ unsigned int s_pre;          // bit 0 / 1: first weight / operand box of the next wavefront requested ahead
   unsigned char* cstage_w = tiles_ptr + kRingBytes;
   const uint32_t epi_bar = smem_u32(bars + 2 * kMaxStages + 4);
+  const uint32_t drain_bar = smem_u32(bars + 2 * kMaxStages + 5);
   uint32_t epi_phase = 0;
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -176,6 +178,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
     mbar_init(epi_bar, 256);
+    mbar_init(drain_bar, 1);
     *s_abort = 0;
     s_early = 0u;
     s_pre = 0u;
@@ -202,6 +205,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   bool alive = true;
   bool stop = false;                    // uniform over the CTA
   bool pre = false;                     // producers: this warp's first box of the wavefront was requested at the barrier
+  uint32_t armed = 0;                   // producers (lane 0): ring stages this thread has requested a box into
 
   if (only_level < 0 && n_levels > 0) {
     prepare_operands(p, blockIdx.x * kThreads + tid, gridDim.x * kThreads);
@@ -285,6 +289,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
             }
             mbar_arrive_expect_tx(full_bar(stage), bytes);
             tma_load_3d(tiles_addr + stage * stage_bytes + off, map, 0, y, box * kbox, full_bar(stage));
+            armed |= 1u << stage;
             phase_bits ^= 1u << stage;
             if (++stage == n_stages) stage = 0;
           }
@@ -431,10 +436,23 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     // the loop was left with a box requested ahead still in flight: stand in for the arrival of the
     // producer that did not ask, and let the data land
     if (s_pre != 3u) mbar_arrive(full_bar(0));
-    mbar_wait(full_bar(0), phase_bits & 1u, s_abort, p.wait_limit, p.st);
+    mbar_drain(full_bar(0), phase_bits & 1u);
   }
   __syncthreads();
-  if (*s_abort) __nanosleep(100000);
+  if (*s_abort) {
+    // A wait expired somewhere.  Before shared and tensor memory go back: every box a producer asked
+    // for gets a bounded time to land (its barrier phase completes once both producers have arrived
+    // and the bytes are in), and the MMAs issued so far a bounded time to retire.
+    if ((warp == 4 || warp == 10) && lane == 0) {
+      for (uint32_t s = 0; s < (uint32_t)kMaxStages; ++s)
+        if (armed & (1u << s)) mbar_drain(full_bar(s), ((phase_bits >> s) & 1u) ^ 1u);
+    }
+    if (warp == 5 && lane == 0) {
+      umma_commit(drain_bar);
+      mbar_drain(drain_bar, 0);
+    }
+    __syncthreads();
+  }
   if (warp == 5) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
@@ -554,6 +572,11 @@ int ensure_operand_tmaps(treelstm* ctx, void* ws, int n, const void* xin, const 
   return TREELSTM_OK;
 }
 
+int init_tc_attributes(treelstm* ctx) {
+  TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  return TREELSTM_OK;
+}
+
 int launch_selftest_waits(treelstm* ctx, void* ws, int* result_dev, cudaStream_t stream) {
   DevStatus* st = static_cast<DevStatus*>(ws);
   TL_CUDA(ctx, cudaMemsetAsync(st, 0, sizeof(DevStatus), stream));
@@ -613,11 +636,6 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     if (rc != TREELSTM_OK) return rc;
   }
 
-  static bool attr_set = false;
-  if (!attr_set) {
-    TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    attr_set = true;
-  }
   const int groups = ctx->Hp / kUnitGroup;
   if (flags & TREELSTM_PERSISTENT) {
     int grid = ctx->sm_count;                       // one CTA per SM (shared and tensor memory)

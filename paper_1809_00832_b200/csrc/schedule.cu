@@ -557,6 +557,12 @@ size_t single_smem_bytes(int n, bool with_parts) {
          (with_parts ? round_up_sz((size_t)n * 2, 16) : 0);
 }
 
+int init_schedule_attributes(treelstm* ctx) {
+  TL_CUDA(ctx, cudaFuncSetAttribute(k_schedule_single, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)single_smem_bytes(kSchedSingleMaxNodes, false)));
+  return TREELSTM_OK;
+}
+
 int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
                     const int32_t* token, int32_t* level, int32_t* order, int32_t* level_offset,
                     int32_t* n_levels_out, void* ws, const WsLayout& lay, int n_parts, cudaStream_t stream) {
@@ -571,12 +577,6 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   const int single_max = ctx->opt.sched_single_cta_max < kSchedSingleMaxNodes
                              ? ctx->opt.sched_single_cta_max : kSchedSingleMaxNodes;
   if (n > 0 && n <= single_max) {
-    static bool attr_set = false;
-    if (!attr_set) {
-      TL_CUDA(ctx, cudaFuncSetAttribute(k_schedule_single, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)single_smem_bytes(kSchedSingleMaxNodes, false)));
-      attr_set = true;
-    }
     // the kernel clears the control block itself and writes the level count to the caller
     const bool parts = n_parts > 0 && n <= kSchedPartMaxNodes;
     k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n, parts), stream>>>(

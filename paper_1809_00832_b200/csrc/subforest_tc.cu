@@ -80,8 +80,9 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
   unsigned char* fixed_ptr = cstage_ptr + L.cstage_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(fixed_ptr);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty,
-  // bars[2S+4]: meeting point of the 256 epilogue threads, bars[2S+5]: resident W_h slice has landed
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 6);
+  // bars[2S+4]: meeting point of the 256 epilogue threads, bars[2S+5]: resident W_h slice has landed,
+  // bars[2S+6]: teardown after a failed wait - the MMA issuer's last commit
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 7);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   int* s_nlev = const_cast<int*>(s_abort) + 1;
   int* s_rownode = reinterpret_cast<int*>(fixed_ptr + 256);   // [128] node id of each tile row
@@ -94,6 +95,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + 2 + a); };
   const uint32_t epi_bar = bar0 + 8u * (2 * kMaxStages + 4);
   const uint32_t wres_bar = bar0 + 8u * (2 * kMaxStages + 5);
+  const uint32_t drain_bar = bar0 + 8u * (2 * kMaxStages + 6);
   uint32_t epi_phase = 0;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -111,6 +113,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
     mbar_init(epi_bar, 256);
     mbar_init(wres_bar, 1);
+    mbar_init(drain_bar, 1);
     *s_abort = 0;
     *s_nlev = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -170,6 +173,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
   bool alive = true;
   bool stop = false;                    // uniform over the CTA
   bool wres_ready = false;
+  uint32_t armed = 0;                   // producers (lane 0): ring stages this thread has requested a box into
 
   for (int lvl = 0; lvl < n_levels; ++lvl) {   // same trip count in every CTA of the cluster
     if (!stop) {
@@ -217,6 +221,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
               }
               mbar_arrive_expect_tx(full_bar(stage), bytes);
               tma_load_3d(ring_addr + stage * stage_bytes + off, map, 0, y, box * kbox, full_bar(stage));
+              armed |= 1u << stage;
               if (is_a && !leaf) mbar_arrive(full_bar(stage));   // stands in for the W producer: W_h is resident
               phase_bits ^= 1u << stage;
               if (++stage == n_stages) stage = 0;
@@ -309,11 +314,24 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
   }
 
   // teardown: let in-flight asynchronous copies land before shared/tensor memory is released
-  if (warp == 10 && lane == 0 && !wres_ready) mbar_wait(wres_bar, 0, s_abort, p.wait_limit, p.st);
+  if (warp == 10 && lane == 0 && !wres_ready) {
+    if (*s_abort) mbar_drain(wres_bar, 0); else mbar_wait(wres_bar, 0, s_abort, p.wait_limit, p.st);
+  }
   asm volatile("cp.async.wait_all;" ::: "memory");
   tc_fence_before();
   __syncthreads();
-  if (*s_abort) __nanosleep(100000);
+  if (*s_abort) {
+    // as in the grid-wide kernel: requested boxes get a bounded time to land, issued MMAs to retire
+    if ((warp == 4 || warp == 10) && lane == 0) {
+      for (uint32_t s = 0; s < (uint32_t)kMaxStages; ++s)
+        if (armed & (1u << s)) mbar_drain(full_bar(s), ((phase_bits >> s) & 1u) ^ 1u);
+    }
+    if (warp == 5 && lane == 0) {
+      umma_commit(drain_bar);
+      mbar_drain(drain_bar, 0);
+    }
+    __syncthreads();
+  }
   if (warp == 5) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);

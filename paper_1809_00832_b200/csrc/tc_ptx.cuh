@@ -72,6 +72,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+// Teardown after a failed wait: give a barrier whose phase may still complete (bytes of a bulk copy
+// in flight, tensor-core work not yet retired) a bounded time to do so, whatever the abort flag says.
+constexpr long long kDrainCycles = 400000;   // about 0.2 ms
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > kDrainCycles) return false;
+  }
+  return true;
+}
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }

@@ -1,5 +1,6 @@
 """Parity of the CUDA training step (forward + backward through structure, via the C ABI) against
-the fp64 oracle: loss and every gradient group within 1e-4 max-abs."""
+the fp64 oracle: loss and every gradient group within 1e-4 max-abs and within 2e-5 of the group's
+own largest entry (several groups of the full-size workload lie below 1e-4 altogether)."""
 import numpy as np
 import pytest
 import torch
@@ -22,13 +23,7 @@ def _train_step(model, forest, labels, flags):
 
 
 def _compare(res, ref, tol):
-    assert abs(float(res["loss"][0]) - ref["loss"]) < tol
-    for k in ("dW", "db", "dWc", "dbc"):
-        assert util.max_abs(res[k], ref[k]) < tol, k
-    nt = int(res["n_touched"][0])
-    assert nt == len(ref["touched_ids"])
-    np.testing.assert_array_equal(res["touched_ids"][:nt], ref["touched_ids"])
-    assert util.max_abs(res["dEmb_rows"][:nt], ref["dEmb_rows"]) < tol
+    util.compare_training_step(res, ref, tol, util.REL["fp32"], loss_rel=1e-5)
 
 
 @pytest.mark.parametrize("flags", [binding.PER_LEVEL, binding.PERSISTENT])
@@ -43,6 +38,25 @@ def test_training_step_matches_oracle(flags):
     # gradients are overwritten, not accumulated: a second step gives the same numbers
     res2 = _train_step(model, f, w.labels, flags)
     _compare(res2, ref, util.TOL["fp32"])
+
+
+@pytest.mark.parametrize("flags", [binding.PER_LEVEL, binding.PERSISTENT])
+def test_training_step_full_size_with_large_gradients(flags):
+    """the sizes of the training workload (H=150, E=300: 64 x 64 dW tiles, dIn chunks split over
+    CTAs) with weights six times larger, so that every gradient group is far above the tolerance"""
+    rng = np.random.default_rng(150)
+    params = fg.draw_params(rng, 150, 300, 2000, emb_dist="normal", emb_scale=0.1, w_scale=0.3, n_classes=5)
+    forest = fg.random_forest(rng, 25, 2, 56, 2000)
+    forest, _ = fg.permute_node_ids(forest, rng)
+    labels = rng.integers(0, 5, size=forest.n_nodes).astype(np.int32)
+    ref = orc.loss_and_gradients(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
+                                 params.Wc, params.bc, labels)
+    for k in util.GRAD_KEYS + ("dEmb_rows",):
+        assert np.max(np.abs(ref[k])) > 5 * util.TOL["fp32"], k      # the case has signal in every group
+    model = util.make_model(params, "fp32")
+    res = _train_step(model, forest, labels, flags)
+    assert util.max_abs(res["h"], ref["h"]) < util.TOL["fp32"]
+    _compare(res, ref, util.TOL["fp32"])
 
 
 def test_training_step_small_odd_sizes_and_duplicates():

@@ -47,7 +47,7 @@ def _worker(rank, world, port, out_dir):
     os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
     params, forest, labels = _problem()
-    mine = sharding.shard_trees(forest.n_trees, rank, world)
+    mine = sharding.shard_trees_by_nodes(np.bincount(forest.tree_of, minlength=forest.n_trees), rank, world)
     shard = fg.select_trees(forest, mine)
     shard_labels = labels[np.isin(forest.tree_of, mine)]
     local = _local_gradients(params, shard, shard_labels, pad=rank + 1)

@@ -49,6 +49,26 @@ def test_shards_partition_the_trees():
         assert max(len(p) for p in parts) - min(len(p) for p in parts) <= 1
 
 
+def test_shards_balanced_by_node_count():
+    """trees dealt out by work: a partition, the same on every rank, and no shard above the mean by
+    a whole largest tree (contiguous blocks of equal tree count can be far off on ragged batches)"""
+    rng = np.random.default_rng(8)
+    for world in (2, 3, 8):
+        forest = fg.random_forest(rng, 57, 2, 56, 100)
+        sizes = np.bincount(forest.tree_of, minlength=forest.n_trees)
+        parts = [sharding.shard_trees_by_nodes(sizes, r, world) for r in range(world)]
+        assert sorted(sum(parts, [])) == list(range(forest.n_trees))
+        loads = [int(sizes[p].sum()) for p in parts]
+        assert max(loads) - sum(loads) / world < sizes.max()
+        assert max(loads) - min(loads) <= sizes.max()
+    assert sharding.shard_trees_by_nodes([], 0, 2) == []
+    assert sharding.shard_trees_by_nodes([5], 1, 2) == []
+    # a skewed batch: one huge tree and many small ones
+    sizes = [1000] + [10] * 100
+    parts = [sharding.shard_trees_by_nodes(sizes, r, 2) for r in range(2)]
+    assert parts[0] == [0] and len(parts[1]) == 100
+
+
 def test_single_process_combine_is_identity():
     times, counts = sharding.combine([3.5], [7, 9])
     assert times == [3.5] and counts == [7, 9]

@@ -9,6 +9,17 @@ from oracle import treelstm_oracle as orc
 from paper_1809_00832_b200 import binding, build, forests as fg
 
 TOL = {"fp32": 1e-4, "bf16": 3e-2}     # max-abs tolerance on h, c and gradients
+# The absolute tolerances above are the stated ones; on the full-size training workload most
+# gradient groups are smaller than 1e-4 altogether, so every group is also held to an error of at
+# most REL x its own largest reference entry (the fp32 kernels measure 4e-7 of that on the training
+# workload, the fp32 loss 9e-7 relative; the bf16 forward feeding an fp32 backward stays below
+# 1e-2).  TIGHT is the bf16 forward against the oracle fed the same bf16-rounded operands: what
+# remains is accumulation order, fast activations and the re-rounding of h (measured on the three
+# full-size bf16 workloads: at most 9.3e-5; the small test shapes use larger weights).
+REL = {"fp32": 2e-5, "bf16": 5e-2}
+TIGHT = 2e-3
+TIGHT_FULL_SIZE = 5e-4
+GRAD_KEYS = ("dW", "db", "dWc", "dbc")
 
 
 def lib_ready():
@@ -42,12 +53,14 @@ def gpu_forward(model, forest: fg.Forest, flags: int):
 
 
 @functools.lru_cache(maxsize=None)
-def oracle_forward_cached(name: str, seed: int, n_trees=None):
+def oracle_forward_cached(name: str, seed: int, n_trees=None, rounded: bool = False):
+    """Oracle schedule and states of a named workload; rounded=True feeds it bf16-rounded operands."""
     w = fg.make_workload(name, seed, n_trees)
     f, p = w.forest, w.params
     status, parent, level, order, off = orc.schedule(f.left, f.right, f.token, p.vocab)
     assert status == orc.OK
-    h, c, _ = orc.forward_recursive(f.left, f.right, f.token, p.emb, p.W, p.b)
+    h, c, _ = orc.forward_recursive(f.left, f.right, f.token, p.emb, p.W, p.b,
+                                    operand_round=orc.round_to_bf16 if rounded else None)
     return dict(parent=parent, level=level, order=order, level_offset=off, h=h, c=c)
 
 
@@ -62,3 +75,23 @@ def check_schedule(res, ref, n):
 
 def max_abs(a, b):
     return float(np.max(np.abs(np.asarray(a, dtype=np.float64) - b))) if a.size else 0.0
+
+
+def compare_training_step(res, ref, tol, rel, loss_rel=None):
+    """Loss and every gradient group of a training step (numpy arrays) against the oracle's: within
+    the absolute tolerance AND within rel x the group's own largest reference entry, so that a
+    group whose entries are all below the absolute tolerance cannot pass by being zero."""
+    loss = float(np.asarray(res["loss"]).reshape(-1)[0])
+    assert abs(loss - ref["loss"]) < tol, ("loss", loss, ref["loss"])
+    if loss_rel is not None:
+        assert abs(loss - ref["loss"]) <= loss_rel * abs(ref["loss"]), ("loss", loss, ref["loss"])
+    nt = int(np.asarray(res["n_touched"]).reshape(-1)[0])
+    assert nt == len(ref["touched_ids"])
+    np.testing.assert_array_equal(np.asarray(res["touched_ids"])[:nt], ref["touched_ids"])
+    groups = [(k, np.asarray(res[k]), ref[k]) for k in GRAD_KEYS]
+    groups.append(("dEmb_rows", np.asarray(res["dEmb_rows"])[:nt], ref["dEmb_rows"]))
+    for k, got, want in groups:
+        err = max_abs(got, want)
+        scale = float(np.max(np.abs(want))) if want.size else 0.0
+        assert err < tol, (k, err)
+        assert err <= rel * scale, (k, err, scale)
