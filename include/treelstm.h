@@ -52,8 +52,11 @@ typedef enum treelstm_status {
   TREELSTM_ERR_CUDA = -6,               /* a CUDA runtime call failed; see treelstm_last_cuda_error */
   TREELSTM_ERR_NO_DEVICE = -7,          /* no sm_100 device is current                               */
   TREELSTM_ERR_UNSUPPORTED = -8,        /* size outside what the kernels support                     */
-  TREELSTM_ERR_STATE = -9               /* call order violated (e.g. backward without forward), or   */
+  TREELSTM_ERR_STATE = -9,              /* call order violated (e.g. backward without forward), or   */
                                         /* the current device is not the one the context was made on */
+  TREELSTM_ERR_CHECK = -10              /* checked build only (-DTREELSTM_CHECKED): a kernel read an */
+                                        /* index out of range from the schedule, or a state row was  */
+                                        /* not written exactly as often as it must be                */
 } treelstm_status;
 
 /* precision of the gate contraction */
@@ -85,6 +88,19 @@ typedef enum treelstm_status {
 #define TREELSTM_OPT_MAX_CTAS 3             /* cap on the persistent grid (0 = all co-resident CTAs) */
 #define TREELSTM_OPT_TIME_WAVEFRONT_KERNEL 4 /* 1: bracket the wavefront kernel launch(es) of each  */
                                             /* forward with CUDA events (treelstm_last_kernel_ms)    */
+#define TREELSTM_OPT_TAIL_WIDTH 5           /* TREELSTM_PERSISTENT, bf16, H padded to <= 256: a forest  */
+                                            /* of at most this many nodes (default and largest value  */
+                                            /* 128) has no wider wavefront and is evaluated by ONE     */
+                                            /* thread-block cluster (recurrent weights resident in     */
+                                            /* shared memory, hardware cluster barrier between          */
+                                            /* wavefronts) instead of the grid-wide kernel - chosen by  */
+                                            /* the library, same results; 0 switches this off          */
+#define TREELSTM_OPT_TAIL_MIN_LEVELS 6      /* > 0: a larger forest whose last wavefronts are all at    */
+                                            /* most TAIL_WIDTH nodes wide hands those over to the       */
+                                            /* cluster (a second launch) if at least this many remain;  */
+                                            /* the hand-over level is found on the device.  Default 0:  */
+                                            /* never (measured: the second launch and the cluster's     */
+                                            /* set-up cost what the narrow wavefronts save)             */
 
 /*
  * treelstm_create - build a context for one set of parameters.
@@ -101,6 +117,27 @@ typedef enum treelstm_status {
  */
 TREELSTM_API int treelstm_create(treelstm_t** out, int H, int E, int vocab, const float* emb, const float* W,
                     const float* b, int precision, void* stream);
+
+/*
+ * treelstm_create_recursive - a context for one of the paper's other two recursive models (Section
+ * 6.1; Table 1 of Section 6.3 is measured on TreeRNN), evaluated by the same dependency-driven
+ * schedule.  The paper prints neither cell; these are the published ones:
+ *   TREELSTM_CELL_TREERNN   p   = tanh(W^T [h_l ; h_r] + b)
+ *   TREELSTM_CELL_RNTN      p_j = tanh([h_l ; h_r]^T V_j [h_l ; h_r] + (W^T [h_l ; h_r])_j + b_j)
+ * A leaf's state is its word vector, h = emb[token] (so the embedding width is H); there is no
+ * cell state.
+ *   emb [vocab][H], W [2H][H] (rows [0,H) multiply h_l, [H,2H) h_r), b [H],
+ *   V [H][2H][2H] (one 2H x 2H slice per output unit; TREELSTM_CELL_RNTN only, else NULL).
+ * fp32 arithmetic.  H <= 4096 (TreeRNN), H <= 128 (RNTN).  Parameters are copied (the tensor is
+ * re-packed); the call synchronises `stream`.  Such a context takes treelstm_forward (flags
+ * TREELSTM_PER_LEVEL or TREELSTM_PERSISTENT; c may be NULL and is not written), treelstm_roots
+ * (root_c is not written), treelstm_forward_host (c, root_c not written), treelstm_status_sync and
+ * treelstm_destroy; the training calls return TREELSTM_ERR_UNSUPPORTED.
+ */
+#define TREELSTM_CELL_TREERNN 1
+#define TREELSTM_CELL_RNTN 2
+TREELSTM_API int treelstm_create_recursive(treelstm_t** out, int cell, int H, int vocab, const float* emb,
+                                           const float* W, const float* b, const float* V, void* stream);
 
 /* Re-read emb, W, b (same shapes as at create) after the caller changed them. Synchronises. */
 TREELSTM_API int treelstm_update_weights(treelstm_t* ctx, const float* emb, const float* W, const float* b,

@@ -23,6 +23,7 @@ ERR_CUDA = -6
 ERR_NO_DEVICE = -7
 ERR_UNSUPPORTED = -8
 ERR_STATE = -9
+ERR_CHECK = -10
 
 FP32 = 0
 BF16 = 1
@@ -30,10 +31,14 @@ PER_LEVEL = 0
 PERSISTENT = 1
 SAVE_FOR_BACKWARD = 2
 SUBFORESTS = 4
+CELL_TREERNN = 1
+CELL_RNTN = 2
 OPT_SCHED_SINGLE_CTA_MAX = 1
 OPT_WAIT_LIMIT_CYCLES = 2
 OPT_MAX_CTAS = 3
 OPT_TIME_WAVEFRONT_KERNEL = 4
+OPT_TAIL_WIDTH = 5
+OPT_TAIL_MIN_LEVELS = 6
 
 _vp = ctypes.c_void_p
 _i = ctypes.c_int
@@ -41,6 +46,7 @@ _i = ctypes.c_int
 # name -> (restype, argtypes); mirrors include/treelstm.h
 SIGNATURES = {
     "treelstm_create": (_i, [ctypes.POINTER(_vp), _i, _i, _i, _vp, _vp, _vp, _i, _vp]),
+    "treelstm_create_recursive": (_i, [ctypes.POINTER(_vp), _i, _i, _i, _vp, _vp, _vp, _vp, _vp]),
     "treelstm_update_weights": (_i, [_vp, _vp, _vp, _vp, _vp]),
     "treelstm_set_classifier": (_i, [_vp, _i, _vp, _vp, _vp]),
     "treelstm_set_option": (_i, [_vp, _i, ctypes.c_longlong]),
@@ -66,7 +72,10 @@ SIGNATURES = {
     "treelstm_strerror": (ctypes.c_char_p, [_i]),
 }
 
-_lib = None
+_libs = {}
+# which build of the library the handles use unless told otherwise: "" (the library itself),
+# "checked" or "trace" (see build.py); the environment variable switches a whole run over
+DEFAULT_VARIANT = os.environ.get("TREELSTM_LIB_VARIANT", "")
 
 
 class TreeLSTMError(RuntimeError):
@@ -76,19 +85,20 @@ class TreeLSTMError(RuntimeError):
         super().__init__(f"{where}: {msg} ({code})")
 
 
-def load_library() -> ctypes.CDLL:
+def load_library(variant: Optional[str] = None) -> ctypes.CDLL:
     """dlopen the in-tree shared library and declare every prototype.  Raises if it is not built."""
-    global _lib
-    if _lib is not None:
-        return _lib
-    if not os.path.exists(LIB_PATH):
-        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_1809_00832_b200.build`")
-    lib = ctypes.CDLL(LIB_PATH)
+    variant = DEFAULT_VARIANT if variant is None else variant
+    if variant in _libs:
+        return _libs[variant]
+    path = LIB_PATH if not variant else os.path.join(_PKG_DIR, f"libtreelstm_b200_{variant}.so")
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_1809_00832_b200.build`")
+    lib = ctypes.CDLL(path)
     for name, (res, args) in SIGNATURES.items():
         fn = getattr(lib, name)
         fn.restype = res
         fn.argtypes = args
-    _lib = lib
+    _libs[variant] = lib
     return lib
 
 
@@ -150,12 +160,13 @@ class TreeLSTM:
     workspace it allocates through torch (device memory is PyTorch's job here)."""
 
     def __init__(self, H: int, E: int, vocab: int, emb: torch.Tensor, W: torch.Tensor, b: torch.Tensor,
-                 precision: int = FP32):
+                 precision: int = FP32, variant: Optional[str] = None):
         if not torch.cuda.is_available():
             raise RuntimeError("no CUDA device: the TreeLSTM library has no CPU path")
-        self.lib = load_library()
+        self.lib = load_library(variant)
         self.H, self.E, self.vocab, self.precision = H, E, vocab, precision
         self.C = 0
+        self.cell = 0
         _dev(emb, torch.float32, "emb"); _dev(W, torch.float32, "W"); _dev(b, torch.float32, "b")
         assert emb.shape == (vocab, E) and W.shape == (E + 2 * H, 5 * H) and b.shape == (5 * H,)
         handle = ctypes.c_void_p()
@@ -167,6 +178,31 @@ class TreeLSTM:
         self._ws: Optional[torch.Tensor] = None
         self._host_staging: Optional[torch.Tensor] = None
         self._keep = None
+
+    @classmethod
+    def recursive(cls, cell: int, H: int, vocab: int, emb: torch.Tensor, W: torch.Tensor, b: torch.Tensor,
+                  V: Optional[torch.Tensor] = None, variant: Optional[str] = None) -> "TreeLSTM":
+        """treelstm_create_recursive: a TreeRNN (CELL_TREERNN) or RNTN (CELL_RNTN) context.  forward()
+        then returns h only (no cell state)."""
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the library has no CPU path")
+        self = cls.__new__(cls)
+        self.lib = load_library(variant)
+        self.H, self.E, self.vocab, self.precision, self.C, self.cell = H, H, vocab, FP32, 0, cell
+        for name, t in (("emb", emb), ("W", W), ("b", b)) + ((("V", V),) if V is not None else ()):
+            _dev(t, torch.float32, name)
+        assert emb.shape == (vocab, H) and W.shape == (2 * H, H) and b.shape == (H,)
+        assert V is None or V.shape == (H, 2 * H, 2 * H)
+        handle = ctypes.c_void_p()
+        rc = self.lib.treelstm_create_recursive(ctypes.byref(handle), cell, H, vocab, _ptr(emb), _ptr(W), _ptr(b),
+                                                _ptr(V), _stream())
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_create_recursive")
+        self.handle = handle
+        self._ws = None
+        self._host_staging = None
+        self._keep = None
+        return self
 
     def close(self):
         if getattr(self, "handle", None):
@@ -220,7 +256,7 @@ class TreeLSTM:
         if out is None:
             out = dict(
                 h=torch.empty((n, self.H), dtype=torch.float32, device="cuda"),
-                c=torch.empty((n, self.H), dtype=torch.float32, device="cuda"),
+                c=torch.empty((n, self.H), dtype=torch.float32, device="cuda") if self.cell == 0 else None,
                 level=torch.empty(n, dtype=torch.int32, device="cuda"),
                 order=torch.empty(n, dtype=torch.int32, device="cuda"),
                 level_offset=torch.empty(n + 2, dtype=torch.int32, device="cuda"),
@@ -230,7 +266,7 @@ class TreeLSTM:
         base = ws.data_ptr()
         aligned = (base + 255) // 256 * 256
         rc = self.lib.treelstm_forward(self.handle, n, _ptr(left), _ptr(right), _ptr(token), _ptr(out["h"]),
-                                       _ptr(out["c"]), _ptr(out["level"]), _ptr(out["order"]),
+                                       _ptr(out.get("c")), _ptr(out["level"]), _ptr(out["order"]),
                                        _ptr(out["level_offset"]), _ptr(out["n_levels"]), flags,
                                        ctypes.c_void_p(aligned), ws.numel() - (aligned - base), _stream())
         if rc != OK:

@@ -37,6 +37,14 @@ WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward) {
     L.dz = take(4 * nn * 5 * H);
     L.tok_slot = take(4 * ((size_t)ctx->vocab + 1));
   }
+  L.trace = off;
+#ifdef TREELSTM_TRACE
+  L.trace = take(2 * sizeof(long long) * kTraceSlots * kTraceLevels);   // grid kernel | cluster kernel
+#endif
+  L.check = off;
+#ifdef TREELSTM_CHECKED
+  L.check = take(3 * 4 * nn);
+#endif
   L.total = off;
   return L;
 }
@@ -195,15 +203,54 @@ int treelstm_create(treelstm_t** out, int H, int E, int vocab, const float* emb,
   return TREELSTM_OK;
 }
 
+int treelstm_create_recursive(treelstm_t** out, int cell, int H, int vocab, const float* emb, const float* W,
+                              const float* b, const float* V, void* stream) {
+  if (!out) return TREELSTM_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cell != TREELSTM_CELL_TREERNN && cell != TREELSTM_CELL_RNTN) return TREELSTM_ERR_INVALID_ARG;
+  if (H <= 0 || vocab <= 0 || !emb || !W || !b || (cell == TREELSTM_CELL_RNTN && !V)) return TREELSTM_ERR_INVALID_ARG;
+  if (H > 4096 || (cell == TREELSTM_CELL_RNTN && H > 128)) return TREELSTM_ERR_UNSUPPORTED;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TREELSTM_ERR_NO_DEVICE;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return TREELSTM_ERR_NO_DEVICE;
+  if (prop.major != 10) return TREELSTM_ERR_NO_DEVICE;
+  treelstm* ctx = new (std::nothrow) treelstm();
+  if (!ctx) return TREELSTM_ERR_INVALID_ARG;
+  ctx->H = H; ctx->E = H; ctx->vocab = vocab; ctx->precision = TREELSTM_FP32; ctx->cell = cell;
+  ctx->Hp = round_up(H, kKBlock); ctx->Ep = ctx->Hp;
+  ctx->device = dev;
+  ctx->sm_count = prop.multiProcessorCount;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t Hs = H, V_ = vocab, K2 = 2 * Hs, KQ = cell == TREELSTM_CELL_RNTN ? K2 * K2 : 0;
+  auto fail = [&](int rc) { treelstm_destroy(ctx); return rc; };
+  if (cudaMalloc((void**)&ctx->emb, sizeof(float) * V_ * Hs) != cudaSuccess ||
+      cudaMalloc((void**)&ctx->Wcat, sizeof(float) * (KQ + K2) * Hs) != cudaSuccess ||
+      cudaMalloc((void**)&ctx->b, sizeof(float) * Hs) != cudaSuccess ||
+      cudaMallocHost((void**)&ctx->host_status, sizeof(DevStatus)) != cudaSuccess)
+    return fail(TREELSTM_ERR_CUDA);
+  int rc = init_schedule_attributes(ctx);
+  if (rc != TREELSTM_OK) return fail(rc);
+  if (cudaMemcpyAsync(ctx->emb, emb, sizeof(float) * V_ * Hs, cudaMemcpyDeviceToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(ctx->b, b, sizeof(float) * Hs, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return fail(TREELSTM_ERR_CUDA);
+  rc = pack_weights_rec(ctx, W, V, s);
+  if (rc != TREELSTM_OK) return fail(rc);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return fail(TREELSTM_ERR_CUDA);
+  *out = ctx;
+  return TREELSTM_OK;
+}
+
 int treelstm_update_weights(treelstm_t* ctx, const float* emb, const float* W, const float* b,
                             void* stream) {
   if (!ctx || !emb || !W || !b) return TREELSTM_ERR_INVALID_ARG;
+  if (ctx->cell != 0) return TREELSTM_ERR_UNSUPPORTED;   // TreeRNN / RNTN contexts are created anew
   return copy_params(ctx, emb, W, b, static_cast<cudaStream_t>(stream));
 }
 
 int treelstm_set_classifier(treelstm_t* ctx, int C, const float* Wc, const float* bc, void* stream) {
   if (!ctx || !Wc || !bc || C < 1) return TREELSTM_ERR_INVALID_ARG;
-  if (C > 32) return TREELSTM_ERR_UNSUPPORTED;
+  if (C > 32 || ctx->cell != 0) return TREELSTM_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaFree(ctx->Wc); cudaFree(ctx->bc);
   ctx->Wc = ctx->bc = nullptr; ctx->C = 0;
@@ -228,6 +275,15 @@ int treelstm_set_option(treelstm_t* ctx, int key, long long value) {
       return TREELSTM_OK;
     case TREELSTM_OPT_MAX_CTAS:
       ctx->opt.max_ctas = value > 65535 ? 65535 : (int)value;
+      return TREELSTM_OK;
+    case 100:
+      ctx->opt.knob = (int)value;
+      return TREELSTM_OK;
+    case TREELSTM_OPT_TAIL_WIDTH:
+      ctx->opt.tail_width = value > 128 ? 128 : (int)value;
+      return TREELSTM_OK;
+    case TREELSTM_OPT_TAIL_MIN_LEVELS:
+      ctx->opt.tail_min_levels = value > (1 << 20) ? (1 << 20) : (int)value;
       return TREELSTM_OK;
     case TREELSTM_OPT_TIME_WAVEFRONT_KERNEL:
       if (value && !ctx->ev_begin) {
@@ -255,9 +311,10 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
   ctx->launches = 0;
   if (!on_own_device(ctx)) return TREELSTM_ERR_STATE;
   if (n_nodes < 0 || !n_levels || !workspace) return TREELSTM_ERR_INVALID_ARG;
-  if (n_nodes > 0 && (!left || !right || !token || !h || !c || !level || !order))
+  if (n_nodes > 0 && (!left || !right || !token || !h || (!c && ctx->cell == 0) || !level || !order))
     return TREELSTM_ERR_INVALID_ARG;
   if (flags & ~(TREELSTM_PERSISTENT | TREELSTM_SAVE_FOR_BACKWARD | TREELSTM_SUBFORESTS)) return TREELSTM_ERR_INVALID_ARG;
+  if (ctx->cell != 0 && (flags & TREELSTM_SAVE_FOR_BACKWARD)) return TREELSTM_ERR_UNSUPPORTED;
   if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return TREELSTM_ERR_INVALID_ARG;
   const bool save = (flags & TREELSTM_SAVE_FOR_BACKWARD) != 0;
   const WsLayout lay = ws_layout(ctx, n_nodes, save);
@@ -289,10 +346,16 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
     rc = read_levels(ctx);
     if (rc != TREELSTM_OK) { L.valid = false; return rc; }
   }
+  rc = launch_check_clear(ctx, n_nodes, workspace, lay, s);
+  if (rc != TREELSTM_OK) { L.valid = false; return rc; }
   ctx->ev_valid = false;
   if (ctx->opt.time_kernel) TL_CUDA(ctx, cudaEventRecord(ctx->ev_begin, s));
-  if (subforests)
-    rc = launch_forward_bf16_subforest(ctx, n_nodes, left, right, token, h, c, level, flags, workspace, lay, s);
+  if (ctx->cell != 0)
+    rc = launch_forward_rec(ctx, n_nodes, left, right, token, h, order, lvl_off, ctx->host_level_offset, L.n_levels,
+                            persistent ? (flags | TREELSTM_PERSISTENT) : flags, workspace, lay, s);
+  else if (subforests)
+    rc = launch_forward_bf16_subforest(ctx, n_nodes, left, right, token, h, c, level, order, lvl_off, false, flags,
+                                       workspace, lay, s);
   else if (ctx->precision == TREELSTM_BF16)
     rc = launch_forward_bf16(ctx, n_nodes, left, right, token, h, c, order, lvl_off,
                              ctx->host_level_offset, L.n_levels, persistent ? (flags | TREELSTM_PERSISTENT) : flags,
@@ -305,6 +368,7 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
     TL_CUDA(ctx, cudaEventRecord(ctx->ev_end, s));
     ctx->ev_valid = true;
   }
+  if (rc == TREELSTM_OK) rc = launch_check_counts(ctx, n_nodes, lvl_off, workspace, lay, s);
   if (rc != TREELSTM_OK) L.valid = false;
   return rc;
 }
@@ -428,7 +492,7 @@ int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, con
   }
   if (n_nodes > 0) {
     if (h) TL_CUDA(ctx, cudaMemcpyAsync(h, p.h, nb * H, cudaMemcpyDeviceToHost, s));
-    if (c) TL_CUDA(ctx, cudaMemcpyAsync(c, p.c, nb * H, cudaMemcpyDeviceToHost, s));
+    if (c && ctx->cell == 0) TL_CUDA(ctx, cudaMemcpyAsync(c, p.c, nb * H, cudaMemcpyDeviceToHost, s));
     if (level) TL_CUDA(ctx, cudaMemcpyAsync(level, p.level, nb, cudaMemcpyDeviceToHost, s));
     if (order) TL_CUDA(ctx, cudaMemcpyAsync(order, p.order, nb, cudaMemcpyDeviceToHost, s));
   }
@@ -478,6 +542,20 @@ int treelstm_selftest_waits(treelstm_t* ctx, void* workspace, size_t workspace_b
   return launch_selftest_waits(ctx, workspace, result, static_cast<cudaStream_t>(stream));
 }
 
+#ifdef TREELSTM_TRACE
+// Trace builds only (not part of the public header): copies the cycle stamps of the last forward to
+// the host, kTraceSlots per wavefront; which = 0 grid-wide kernel, 1 cluster kernel.  Synchronises.
+TREELSTM_API int treelstm_trace_read(treelstm_t* ctx, int which, long long* out, int max_entries) {
+  if (!ctx || !out || which < 0 || which > 1 || !ctx->last.ws) return TREELSTM_ERR_INVALID_ARG;
+  const int total = kTraceSlots * kTraceLevels;
+  const int cnt = max_entries < total ? max_entries : total;
+  const char* src = static_cast<const char*>(ctx->last.ws) + ctx->last.lay.trace + (size_t)which * total * sizeof(long long);
+  TL_CUDA(ctx, cudaStreamSynchronize(ctx->last.stream));
+  TL_CUDA(ctx, cudaMemcpy(out, src, sizeof(long long) * cnt, cudaMemcpyDeviceToHost));
+  return cnt;
+}
+#endif
+
 int treelstm_last_launch_count(const treelstm_t* ctx) { return ctx ? ctx->launches : 0; }
 
 int treelstm_last_mode(const treelstm_t* ctx) { return ctx && ctx->last.valid ? ctx->last.mode : -1; }
@@ -488,7 +566,7 @@ int treelstm_last_cuda_error(const treelstm_t* ctx) { return ctx ? ctx->cuda_err
 
 int treelstm_destroy(treelstm_t* ctx) {
   if (!ctx) return TREELSTM_OK;
-  cudaFree(ctx->emb); cudaFree(ctx->W); cudaFree(ctx->b); cudaFree(ctx->Wc); cudaFree(ctx->bc);
+  cudaFree(ctx->emb); cudaFree(ctx->W); cudaFree(ctx->b); cudaFree(ctx->Wc); cudaFree(ctx->bc); cudaFree(ctx->Wcat);
   cudaFree(ctx->emb_bf); cudaFree(ctx->Wp_h); cudaFree(ctx->Wp_x); cudaFree(ctx->bp_h); cudaFree(ctx->bp_x);
   if (ctx->host_level_offset) cudaFreeHost(ctx->host_level_offset);
   if (ctx->host_status) cudaFreeHost(ctx->host_status);
@@ -511,6 +589,7 @@ const char* treelstm_strerror(int status) {
     case TREELSTM_ERR_NO_DEVICE: return "no sm_100 CUDA device";
     case TREELSTM_ERR_UNSUPPORTED: return "size not supported";
     case TREELSTM_ERR_STATE: return "call order violated";
+    case TREELSTM_ERR_CHECK: return "checked build: index out of range or state row written a wrong number of times";
     default: return "unknown status";
   }
 }

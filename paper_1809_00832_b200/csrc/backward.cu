@@ -35,7 +35,7 @@ struct BwdParams {
 __global__ void k_bwd_mark_tokens(BwdParams p) {
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= p.n_leaves) return;
-  p.tok_slot[p.token[p.order[r]]] = 1;  // level 0 occupies order[0 .. n_leaves)
+  p.tok_slot[chk(p.st, p.token[chk(p.st, p.order[r], p.n)], p.vocab)] = 1;  // level 0 occupies order[0 .. n_leaves)
 }
 
 // Exclusive scan of the flags over the vocabulary by one CTA; flagged ids are emitted in
@@ -156,7 +156,7 @@ __global__ void __launch_bounds__(kClsWarps * 32) k_bwd_classifier(BwdParams p) 
 __device__ __forceinline__ void gates_element(const BwdParams& p, int row_begin, long long idx, int leaf) {
   const int H = p.H;
   const int row = row_begin + (int)(idx / H), u = (int)(idx % H);
-  const int node = p.order[row];
+  const int node = chk(p.st, p.order[row], p.n);
   const float* g = p.gates + (size_t)node * 5 * H + u;
   const float gi = g[0], go = g[3 * H], gu = g[4 * H];
   const float cn = p.c[(size_t)node * H + u];
@@ -171,7 +171,7 @@ __device__ __forceinline__ void gates_element(const BwdParams& p, int row_begin,
     dz[H] = 0.f;
     dz[2 * H] = 0.f;
   } else {
-    const int l = p.left[node], r = p.right[node];
+    const int l = chk(p.st, p.left[node], p.n), r = chk(p.st, p.right[node], p.n);
     const float gfl = g[H], gfr = g[2 * H];
     dz[H] = dcn * p.c[(size_t)l * H + u] * gfl * (1.f - gfl);
     dz[2 * H] = dcn * p.c[(size_t)r * H + u] * gfr * (1.f - gfr);
@@ -213,9 +213,9 @@ __device__ void dinput_block(const BwdParams& p, int row_begin, int row_end, int
   for (int i = tid; i < BT; i += 256) {
     int node = -1, da = 0, db = 0;
     if (row0 + i < row_end) {
-      node = p.order[row0 + i];
-      if (leaf) da = p.tok_slot[p.token[node]];
-      else { da = p.left[node]; db = p.right[node]; }
+      node = chk(p.st, p.order[row0 + i], p.n);
+      if (leaf) da = chk(p.st, p.tok_slot[chk(p.st, p.token[node], p.vocab)], p.n_leaves);
+      else { da = chk(p.st, p.left[node], p.n); db = chk(p.st, p.right[node], p.n); }
     }
     s_node[i] = node; sm.dst_a[i] = da; sm.dst_b[i] = db;
   }
@@ -334,9 +334,9 @@ __device__ void dweight_block(const BwdParams& p, int part, int row_begin, int r
   for (int i = tid; i < kDwRows; i += 256) {
     int node = 0, ia = 0, ib = 0;
     if (r_lo + i < r_hi) {
-      node = p.order[r_lo + i];
-      if (part == 0) ia = p.token[node];
-      else { ia = p.left[node]; ib = p.right[node]; }
+      node = chk(p.st, p.order[r_lo + i], p.n);
+      if (part == 0) ia = chk(p.st, p.token[node], p.vocab);
+      else { ia = chk(p.st, p.left[node], p.n); ib = chk(p.st, p.right[node], p.n); }
     }
     sm.node[i] = node; sm.ia[i] = ia; sm.ib[i] = ib;
   }
@@ -461,7 +461,8 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
   zero_range(p.tok_slot, (size_t)p.vocab + 1, gtid, gthreads);
   zero_range(p.dEmb_rows, (size_t)p.n_leaves * E, gtid, gthreads);
   if (!barrier()) return;
-  for (size_t r = gtid; r < (size_t)p.n_leaves; r += gthreads) p.tok_slot[p.token[p.order[r]]] = 1;
+  for (size_t r = gtid; r < (size_t)p.n_leaves; r += gthreads)
+    p.tok_slot[chk(p.st, p.token[chk(p.st, p.order[r], p.n)], p.vocab)] = 1;
   if (!barrier()) return;
   if (gridDim.x == 1) {
     scan_tokens(p);

@@ -19,7 +19,8 @@ constexpr int kThreads = 256;
 constexpr int kWLoads = KC * 5 * TU / kThreads;    // 10 weight elements per thread and chunk
 
 struct FwdParams {
-  int n, H, E, n_sms;
+  int n, H, E, n_sms, vocab;
+  int* chk_counts;   // checked build: writes of h per node
   const int *left, *right, *token, *order, *level_offset;
   const float *emb, *W, *b;
   float *h, *c, *gates;
@@ -60,9 +61,9 @@ __device__ void fp32_tile(const FwdParams& p, int row0, int row_end, int u0, boo
     const int row = row0 + i;
     int node = -1, l = 0, r = 0;
     if (row < row_end) {
-      node = p.order[row];
-      l = leaf ? p.token[node] : p.left[node];
-      r = leaf ? 0 : p.right[node];
+      node = chk(p.st, p.order[row], p.n);
+      l = leaf ? chk(p.st, p.token[node], p.vocab) : chk(p.st, p.left[node], p.n);
+      r = leaf ? 0 : chk(p.st, p.right[node], p.n);
     }
     s.node[i] = node; s.l[i] = l; s.r[i] = r;
   }
@@ -150,6 +151,7 @@ __device__ void fp32_tile(const FwdParams& p, int row0, int row_end, int u0, boo
     }
     p.c[(size_t)node * H + u] = cn;
     p.h[(size_t)node * H + u] = go * tanhf(cn);
+    count_write(p.chk_counts, node, 1);
     if (p.gates) {
       float* g = p.gates + (size_t)node * 5 * H + u;
       g[0] = gi; g[H] = gfl; g[2 * H] = gfr; g[3 * H] = go; g[4 * H] = gu;
@@ -177,7 +179,11 @@ __device__ void fp32_tile_stationary(const FwdParams& p, int row0, int row_end, 
   for (int i = tid; i < TM && !ids_ready; i += kThreads) {   // ids_ready: fetched while the grid barrier was pending
     const int row = row0 + i;
     int node = -1, l = 0, r = 0;
-    if (row < row_end) { node = p.order[row]; l = p.left[node]; r = p.right[node]; }
+    if (row < row_end) {
+      node = chk(p.st, p.order[row], p.n);
+      l = chk(p.st, p.left[node], p.n);
+      r = chk(p.st, p.right[node], p.n);
+    }
     s_node[i] = node; s_l[i] = l; s_r[i] = r;
   }
   __syncthreads();
@@ -268,6 +274,7 @@ __device__ void fp32_tile_stationary(const FwdParams& p, int row0, int row_end, 
     const float cn = gi * gu + gfl * __ldcg(p.c + (size_t)s_l[ii] * H + u) + gfr * __ldcg(p.c + (size_t)s_r[ii] * H + u);
     p.c[(size_t)node * H + u] = cn;
     p.h[(size_t)node * H + u] = go * tanhf(cn);
+    count_write(p.chk_counts, node, 1);
     if (p.gates) {
       float* g = p.gates + (size_t)node * 5 * H + u;
       g[0] = gi; g[H] = gfl; g[2 * H] = gfr; g[3 * H] = go; g[4 * H] = gu;
@@ -375,7 +382,11 @@ k_fwd_fp32_persistent(FwdParams p) {
             if ((int)blockIdx.x >= tiles2 || i >= tmr2) return;
             const int row = nb + ((int)blockIdx.x / tiles_u) * tmr2 + i;
             int node = -1, l = 0, r = 0;
-            if (row < ne) { node = p.order[row]; l = p.left[node]; r = p.right[node]; }
+            if (row < ne) {
+              node = chk(p.st, p.order[row], p.n);
+              l = chk(p.st, p.left[node], p.n);
+              r = chk(p.st, p.right[node], p.n);
+            }
             s_node[i] = node; s_l[i] = l; s_r[i] = r;
           });
       if (!passed) return;
@@ -393,7 +404,8 @@ int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t
                         cudaStream_t stream) {
   char* base = static_cast<char*>(ws);
   FwdParams p;
-  p.n = n; p.H = ctx->H; p.E = ctx->E; p.n_sms = ctx->sm_count;
+  p.n = n; p.H = ctx->H; p.E = ctx->E; p.n_sms = ctx->sm_count; p.vocab = ctx->vocab;
+  p.chk_counts = check_counters(ws, lay);
   p.left = left; p.right = right; p.token = token; p.order = order;
   p.level_offset = level_offset_dev;
   p.emb = ctx->emb; p.W = ctx->W; p.b = ctx->b;

@@ -27,14 +27,30 @@ static_assert(sizeof(DevStatus) == 256, "control block is one 256-byte line grou
 // Offsets (bytes) of the regions inside the workspace for a forest of up to n nodes.
 struct WsLayout {
   size_t status, parent, pending, order_tmp, level_offset, roots, table, slot, part_order, part_offset,
-      part_spill, xin, ain, cin, gates, dh, dc, dz, tok_slot, total;
+      part_spill, xin, ain, cin, gates, dh, dc, dz, tok_slot, trace, check, total;
 };
+
+// Cycle stamps of the wavefront kernels (builds with -DTREELSTM_TRACE only): kTraceSlots stamps per
+// wavefront for the first kTraceLevels wavefronts, written by the first CTA of each kernel.
+constexpr int kTraceSlots = 8;
+constexpr int kTraceLevels = 256;
+#ifdef TREELSTM_TRACE
+#define TL_STAMP(buf, level, slot)                                                            \
+  do {                                                                                        \
+    if ((buf) != nullptr && (level) < tl::kTraceLevels) (buf)[(level) * tl::kTraceSlots + (slot)] = clock64(); \
+  } while (0)
+#else
+#define TL_STAMP(buf, level, slot) do { } while (0)
+#endif
 
 struct Options {
   int sched_single_cta_max = 32768;
   long long wait_limit_kcycles = 1 << 20;  // ~1e9 cycles, about half a second at 2 GHz
   int max_ctas = 0;
   int time_kernel = 0;
+  int knob = 0;           // development switches of the tensor-core kernels (0 in normal use)
+  int tail_width = 128;   // persistent bf16 forward: forests / trailing wavefronts this narrow run on one cluster (0: never)
+  int tail_min_levels = 0; // hand a larger forest's narrow tail over if at least this many wavefronts remain (0: never)
 };
 
 constexpr int kRadixBins = 256;
@@ -78,6 +94,7 @@ inline size_t round_up_sz(size_t x, size_t m) { return (x + m - 1) / m * m; }
 // The context behind the opaque handle of the C ABI.
 struct treelstm {
   int H = 0, E = 0, vocab = 0, precision = 0, C = 0;
+  int cell = 0;        // 0: TreeLSTM, else TREELSTM_CELL_TREERNN / TREELSTM_CELL_RNTN (no cell state, E == H)
   int Hp = 0, Ep = 0;  // bf16 path: H padded to a multiple of 64, E padded to a multiple of 64
   int device = 0;
   int sm_count = 0;
@@ -86,6 +103,7 @@ struct treelstm {
   float* emb = nullptr;  // [vocab][E]
   float* W = nullptr;    // [E+2H][5H]
   float* b = nullptr;    // [5H]
+  float* Wcat = nullptr; // TreeRNN / RNTN: [4H^2 + 2H][H] (tensor slices transposed, then W) or [2H][H]
   float* Wc = nullptr;   // [H][C]
   float* bc = nullptr;   // [C]
 
@@ -164,6 +182,13 @@ int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t
                         int n_levels_host, int flags, void* ws, const WsLayout& lay,
                         cudaStream_t stream);
 
+// cell_rec.cu (TreeRNN / RNTN)
+int pack_weights_rec(treelstm* ctx, const float* W, const float* V, cudaStream_t stream);
+int launch_forward_rec(treelstm* ctx, int n, const int32_t* left, const int32_t* right, const int32_t* token,
+                       float* h, const int32_t* order, const int32_t* level_offset_dev,
+                       const int32_t* level_offset_host, int n_levels_host, int flags, void* ws,
+                       const WsLayout& lay, cudaStream_t stream);
+
 // gemm_tc.cu
 int pack_weights_bf16(treelstm* ctx, cudaStream_t stream);
 int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
@@ -178,7 +203,8 @@ int ensure_operand_tmaps(treelstm* ctx, void* ws, int n, const void* xin, const 
 // subforest_tc.cu
 SubforestPlan subforest_plan(treelstm* ctx);
 int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
-                                  const int32_t* token, float* h, float* c, const int32_t* level, int flags,
+                                  const int32_t* token, float* h, float* c, const int32_t* level,
+                                  const int32_t* order, const int32_t* level_offset_dev, bool tail, int flags,
                                   void* ws, const WsLayout& lay, cudaStream_t stream);
 
 int launch_selftest_waits(treelstm* ctx, void* ws, int* result_dev, cudaStream_t stream);
@@ -187,6 +213,20 @@ int launch_selftest_waits(treelstm* ctx, void* ws, int* result_dev, cudaStream_t
 int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW, float* db,
                     float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,
                     int32_t* n_touched, cudaStream_t stream);
+
+// Checked build: clears the per-row write counters before a forward / compares them after it
+// (schedule.cu); both do nothing in the normal build.  Counters: [h per node | Ain per position | Cin per position].
+int launch_check_clear(treelstm* ctx, int n, void* ws, const WsLayout& lay, cudaStream_t stream);
+int launch_check_counts(treelstm* ctx, int n, const int32_t* level_offset_dev, void* ws, const WsLayout& lay,
+                        cudaStream_t stream);
+inline int* check_counters(void* ws, const WsLayout& lay) {
+#ifdef TREELSTM_CHECKED
+  return reinterpret_cast<int*>(static_cast<char*>(ws) + lay.check);
+#else
+  (void)ws; (void)lay;
+  return nullptr;
+#endif
+}
 
 // roots (schedule.cu)
 int launch_gather_roots(treelstm* ctx, int max_roots, int32_t* root_ids, float* root_h,
@@ -206,6 +246,34 @@ int launch_gather_roots(treelstm* ctx, int max_roots, int32_t* root_ids, float* 
 __device__ __forceinline__ void report(DevStatus* st, int code) { atomicMin(&st->status, code); }
 
 __device__ __forceinline__ int ld_volatile(const int* p) { return *(const volatile int*)p; }
+
+// Checked build (-DTREELSTM_CHECKED; compute-sanitizer's stand-in where that tool is not available):
+// every index that a kernel reads from the caller's arrays or from the schedule passes through
+// chk() before it addresses anything - out of range: TREELSTM_ERR_CHECK is recorded and index 0 is
+// used instead, so nothing is accessed out of bounds and nothing traps - and every store of state
+// units is counted per row with count_write(); a kernel at the end of the forward compares the
+// counts with what a correct evaluation writes (every node's h once, every internal position's
+// operand row twice - one half per child).  In the normal build both compile to nothing.
+#ifdef TREELSTM_CHECKED
+__device__ __forceinline__ int chk(DevStatus* st, int idx, int limit) {
+  if ((unsigned)idx < (unsigned)limit) return idx;
+  report(st, TREELSTM_ERR_CHECK);
+  return 0;
+}
+// delivery slots are 2 * position + side, or -1 for a root
+__device__ __forceinline__ int chk_slot(DevStatus* st, int slot, int n) {
+  if (slot == -1 || (unsigned)slot < 2u * (unsigned)n) return slot;
+  report(st, TREELSTM_ERR_CHECK);
+  return -1;
+}
+__device__ __forceinline__ void count_write(int* counter, int row, int units) {
+  if (counter && units > 0) atomicAdd(counter + row, units);
+}
+#else
+__device__ __forceinline__ int chk(DevStatus*, int idx, int) { return idx; }
+__device__ __forceinline__ int chk_slot(DevStatus*, int slot, int) { return slot; }
+__device__ __forceinline__ void count_write(int*, int, int) {}
+#endif
 
 // Bounded grid-wide barrier for cooperative (co-resident) launches.  `target` is the total
 // number of arrivals expected so far (this barrier included).  A CTA that wrote nothing since the

@@ -111,24 +111,24 @@ __device__ void prepare_operands(const TcParams& p, int gtid, int gthreads) {
   const int pos0 = n_leaves + gtid;
   int l0 = -1, r0 = -1, root0 = -1;
   if (pos0 < p.n) {
-    const int node = p.order[pos0];
-    l0 = p.left[node];
-    r0 = p.right[node];
+    const int node = chk(p.st, p.order[pos0], p.n);
+    l0 = chk(p.st, p.left[node], p.n);
+    r0 = chk(p.st, p.right[node], p.n);
   }
   const int n_roots = p.st->n_roots;
-  if (gtid < n_roots) root0 = p.roots[gtid];
+  if (gtid < n_roots) root0 = chk(p.st, p.roots[gtid], p.n);
   gather_leaf_rows(p, 0, n_leaves, gtid >> 5, gthreads >> 5, gtid & 31);
   if (l0 >= 0) {
     p.slot[l0] = 2 * pos0;
     p.slot[r0] = 2 * pos0 + 1;
   }
   for (int pos = pos0 + gthreads; pos < p.n; pos += gthreads) {
-    const int node = p.order[pos];
-    p.slot[p.left[node]] = 2 * pos;
-    p.slot[p.right[node]] = 2 * pos + 1;
+    const int node = chk(p.st, p.order[pos], p.n);
+    p.slot[chk(p.st, p.left[node], p.n)] = 2 * pos;
+    p.slot[chk(p.st, p.right[node], p.n)] = 2 * pos + 1;
   }
   if (root0 >= 0) p.slot[root0] = -1;
-  for (int t = gtid + gthreads; t < n_roots; t += gthreads) p.slot[p.roots[t]] = -1;
+  for (int t = gtid + gthreads; t < n_roots; t += gthreads) p.slot[chk(p.st, p.roots[t], p.n)] = -1;
 }
 
 __global__ void k_prepare_operands(TcParams p) {
@@ -173,6 +173,15 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (ld_volatile(&p.st->status) != 0) return;      // schedule failed: nothing to evaluate
   const int n_levels = p.st->n_levels;
+  // Persistent mode: the narrow wavefronts at the end of the forest are left to one cluster (launched
+  // next on the same stream), which keeps the recurrent weights in shared memory and meets at the
+  // hardware cluster barrier instead of the grid-wide one.
+  __shared__ int s_stop;
+  const int lvl_stop = only_level < 0 ? tail_first_level(p.level_offset, n_levels, p.tail_width, p.tail_min_levels, &s_stop) : n_levels;
+  if (only_level < 0 && lvl_stop == 0) return;      // the whole forest is narrow: all of it runs on the cluster
+#ifdef TREELSTM_TRACE
+  long long* const trace = blockIdx.x == 0 && tid == 0 ? p.trace : nullptr;
+#endif
 
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
@@ -215,7 +224,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   }
 
   const int lvl_begin = only_level >= 0 ? only_level : 0;
-  const int lvl_end = only_level >= 0 ? only_level + 1 : n_levels;
+  const int lvl_end = only_level >= 0 ? only_level + 1 : lvl_stop;
   auto level_begin = [&](int l) { return l < kLevelCache ? s_level_offset[l] : p.level_offset[l]; };
   auto make_plan = [&](int l) {
     return choose_tile_plan(level_begin(l + 1) - level_begin(l), groups, p.sched_ctas, l == 0, l == 0 ? kb_leaf : kb_int);
@@ -228,6 +237,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     const int begin = level_begin(lvl), end = level_begin(lvl + 1);
     const bool leaf = lvl == 0;
     const TilePlan plan = s_plan[lvl & 1];
+    TL_STAMP(trace, lvl, 0);
     if (warp == 11 && lane == 0 && lvl + 1 < lvl_end) s_plan[(lvl + 1) & 1] = make_plan(lvl + 1);
     const int rt = plan.rt;
     const int ntn = groups >> plan.lg;               // fat column tiles per row tile
@@ -343,8 +353,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
         if (nx_have) {
           node = nx_node; slot = nx_slot;
         } else {
-          node = valid ? p.order[row] : 0;
-          slot = valid ? p.slot[node] : -1;
+          node = valid ? chk(p.st, p.order[row], p.n) : 0;
+          slot = valid ? chk_slot(p.st, p.slot[node], p.n) : -1;
         }
         // the same two dependent loads for this CTA's next tile go out now and land while this tile is computed
         const int t2 = t + (int)gridDim.x;
@@ -354,7 +364,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
           const int fat2 = t2 < plan.tail_from ? t2 : plan.tail_from + ((t2 - plan.tail_from) >> plan.tail_ls);
           const int rtile2 = fat2 / ntn, row2 = begin + (rtile2 << plan.lrt) + r;
           valid2 = r < rt && row2 < end;
-          nx_node = valid2 ? p.order[row2] : 0;
+          nx_node = valid2 ? chk(p.st, p.order[row2], p.n) : 0;
         }
         EpiTile et;
         et.leaf = leaf; et.G = G; et.gcols = gcols; et.ncols = ncols; et.nt = nt;
@@ -367,12 +377,13 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
         et.tmem_acc = tmem_base + acc * kAccCols;
         et.tfull = tfull_bar(acc); et.tempty = tempty_bar(acc); et.epi_bar = epi_bar; et.acc_phase = (acc_iter >> 1) & 1;
         et.bias = (leaf ? p.bp_x : p.bp_h) + nt * ncols + 4 * e;
-        epilogue_tile(p, et, epi_phase, alive, s_abort, [&]() { if (nx_have) nx_slot = valid2 ? p.slot[nx_node] : -1; });
+        epilogue_tile(p, et, epi_phase, alive, s_abort, [&]() { if (nx_have) nx_slot = valid2 ? chk_slot(p.st, p.slot[nx_node], p.n) : -1; });
         ++acc_iter;
       }
     }
     // the operand rows the epilogue wrote are read through TMA (async proxy) by later wavefronts
     if (warp < 4 || (warp >= 6 && warp < 10)) asm volatile("fence.proxy.async.global;" ::: "memory");
+    TL_STAMP(trace, lvl, 6);
     if (only_level < 0 && lvl + 1 < lvl_end) {
       // every role of every CTA joins the barrier.  A role that gave up has set s_abort before
       // this point, so the flag read after the CTA barrier is the same for all threads and the
@@ -425,6 +436,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
         }
       });
       if (!passed) break;
+      TL_STAMP(trace, lvl, 7);
     }
   }
 
@@ -616,7 +628,8 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   if (!ctx->have_tmaps) return TREELSTM_ERR_STATE;
   char* base = static_cast<char*>(ws);
   TcParams p;
-  p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep; p.sched_ctas = ctx->sm_count;
+  p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep; p.sched_ctas = ctx->sm_count; p.vocab = ctx->vocab;
+  p.chk_counts = check_counters(ws, lay);
   p.left = left; p.right = right; p.token = token;
   p.order = order;
   p.roots = reinterpret_cast<int*>(base + lay.roots);
@@ -631,6 +644,21 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.gates = (flags & TREELSTM_SAVE_FOR_BACKWARD) ? reinterpret_cast<float*>(base + lay.gates) : nullptr;
   p.st = reinterpret_cast<DevStatus*>(base + lay.status);
   p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
+  p.level = nullptr; p.part_offset = nullptr; p.part_level_spill = nullptr; p.n_parts = 0; p.groups_per_cta = 0;
+  // Narrow forests and (if asked for) the narrow wavefronts at the end of a forest go to one cluster,
+  // where the cluster kernel exists for these sizes: a forest of at most tail_width nodes has no wider
+  // wavefront and runs there as a whole; a larger one is handed over only with tail_min_levels > 0.
+  const bool tail_ok = (flags & TREELSTM_PERSISTENT) && ctx->sf.ok && ctx->opt.tail_width > 0 && ctx->opt.max_ctas == 0;
+  const bool cluster_only = tail_ok && n <= ctx->opt.tail_width;
+  const bool with_tail = cluster_only || (tail_ok && ctx->opt.tail_min_levels > 0);
+  p.tail_width = with_tail ? ctx->opt.tail_width : 0;
+  p.tail_min_levels = ctx->opt.tail_min_levels;
+  p.trace = nullptr;
+  p.knob = ctx->opt.knob;
+#ifdef TREELSTM_TRACE
+  p.trace = reinterpret_cast<long long*>(base + lay.trace);
+  TL_CUDA(ctx, cudaMemsetAsync(p.trace, 0, sizeof(long long) * kTraceSlots * kTraceLevels, stream));
+#endif
   {
     int rc = ensure_operand_tmaps(ctx, ws, n, p.xin, p.ain);
     if (rc != TREELSTM_OK) return rc;
@@ -644,9 +672,14 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
     int only = -1;
     void* args[] = {&ctx->maps, &p, &only};
-    TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc, dim3(grid), dim3(kThreads), args,
-                                             kSmemBytes, stream));
-    ctx->launches += 1;
+    if (!cluster_only) {
+      TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc, dim3(grid), dim3(kThreads), args,
+                                               kSmemBytes, stream));
+      ctx->launches += 1;
+    }
+    if (with_tail)
+      return launch_forward_bf16_subforest(ctx, n, left, right, token, h, c, nullptr, order, level_offset_dev, true,
+                                           flags, ws, lay, stream);
     return TREELSTM_OK;
   }
   if (n_levels_host > 0) {

@@ -538,7 +538,7 @@ __global__ void k_gather_roots(int max_roots, int H, const int* roots, const flo
   const int n_roots = st->status == 0 ? min(st->n_roots, max_roots) : 0;
   if (blockIdx.x == 0 && threadIdx.x == 0 && n_roots_out) *n_roots_out = n_roots;
   for (int t = blockIdx.x; t < n_roots; t += gridDim.x) {
-    const int node = roots[t];
+    const int node = roots[t];   // written by the scheduler from ids below n
     if (threadIdx.x == 0 && root_ids) root_ids[t] = node;
     for (int j = threadIdx.x; j < H; j += blockDim.x) {
       if (root_h) root_h[(size_t)t * H + j] = h[(size_t)node * H + j];
@@ -625,6 +625,49 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   return TREELSTM_OK;
 }
 
+#ifdef TREELSTM_CHECKED
+namespace {
+// After a forward: every node's h row written once (H units), every internal position's operand rows
+// (bf16 path) twice - one half per child -, no leaf position's operand row at all.
+__global__ void k_check_counts(int n, int H, int bf16, const int* level_offset, const int* counts, DevStatus* st) {
+  if (st->status != 0) return;
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= n) return;
+  const int n_leaves = level_offset[1];
+  bool ok = counts[k] == H;
+  if (bf16) {
+    const int want = k < n_leaves ? 0 : 2 * H;
+    ok = ok && counts[n + k] == want && counts[2 * n + k] == want;
+  }
+  if (!ok) report(st, TREELSTM_ERR_CHECK);
+}
+}  // namespace
+#endif
+
+int launch_check_clear(treelstm* ctx, int n, void* ws, const WsLayout& lay, cudaStream_t stream) {
+#ifdef TREELSTM_CHECKED
+  if (n > 0) TL_CUDA(ctx, cudaMemsetAsync(check_counters(ws, lay), 0, sizeof(int) * 3 * (size_t)n, stream));
+#else
+  (void)ctx; (void)n; (void)ws; (void)lay; (void)stream;
+#endif
+  return TREELSTM_OK;
+}
+
+int launch_check_counts(treelstm* ctx, int n, const int32_t* level_offset_dev, void* ws, const WsLayout& lay,
+                        cudaStream_t stream) {
+#ifdef TREELSTM_CHECKED
+  if (n > 0) {
+    DevStatus* st = reinterpret_cast<DevStatus*>(static_cast<char*>(ws) + lay.status);
+    k_check_counts<<<(n + 255) / 256, 256, 0, stream>>>(n, ctx->H, ctx->precision == TREELSTM_BF16 ? 1 : 0,
+                                                        level_offset_dev, check_counters(ws, lay), st);
+    TL_CUDA(ctx, cudaGetLastError());
+  }
+#else
+  (void)ctx; (void)n; (void)level_offset_dev; (void)ws; (void)lay; (void)stream;
+#endif
+  return TREELSTM_OK;
+}
+
 int launch_gather_roots(treelstm* ctx, int max_roots, int32_t* root_ids, float* root_h,
                         float* root_c, int32_t* n_roots, cudaStream_t stream) {
   const auto& L = ctx->last;
@@ -633,7 +676,7 @@ int launch_gather_roots(treelstm* ctx, int max_roots, int32_t* root_ids, float* 
   const int* roots = reinterpret_cast<const int*>(base + L.lay.roots);
   int blocks = max_roots < 1 ? 1 : (max_roots < 1184 ? max_roots : 1184);
   k_gather_roots<<<blocks, 128, 0, stream>>>(max_roots, ctx->H, roots, L.h, L.c, root_ids, root_h,
-                                             root_c, n_roots, st);
+                                             L.c ? root_c : nullptr, n_roots, st);
   ctx->launches += 1;
   TL_CUDA(ctx, cudaGetLastError());
   return TREELSTM_OK;

@@ -102,11 +102,23 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
   // A failed schedule leaves the level count at 0.  (The status word is not used for this test: a
   // sibling cluster may record a timeout in it at any moment, and the CTAs of one cluster have to
   // take the same decision or the ones that stay would wait at the cluster barrier forever.)
-  if (ld_volatile(&p.st->n_levels) <= 0) return;
+  const int n_levels_all = ld_volatile(&p.st->n_levels);
+  if (n_levels_all <= 0) return;
   const int cs = (int)cluster_nctarank(), rank = (int)cluster_ctarank();
-  const int part = blockIdx.x / cs;
-  const int pbeg = p.part_offset[part], pend = p.part_offset[part + 1];
+  const bool tail = p.n_parts == 0;                 // one cluster finishes what the grid-wide kernel left
+  const int part = tail ? 0 : blockIdx.x / cs;
+  __shared__ int s_first;
+  int first_level = 0;                              // tail: absolute index of the first wavefront done here
+  if (tail) {
+    first_level = tail_first_level(p.level_offset, n_levels_all, p.tail_width, p.tail_min_levels, &s_first);
+    if (first_level >= n_levels_all) return;        // nothing left (the same answer in every CTA)
+  }
+  const int pbeg = tail ? p.level_offset[first_level] : p.part_offset[part];
+  const int pend = tail ? p.n : p.part_offset[part + 1];
   if (pbeg >= pend) return;                         // empty sub-forest: the whole cluster leaves
+#ifdef TREELSTM_TRACE
+  long long* const trace = blockIdx.x == 0 ? p.trace : nullptr;
+#endif
 
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
@@ -136,33 +148,46 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
     tma_load_3d(wres_addr, &sfm.wres, 0, nt * G * kGColsI, 0, wres_bar);
   }
 
-  // Wavefront boundaries of the sub-forest: its nodes are sorted by level, the levels are 0 .. top
-  // without gaps.  Every CTA builds the table for itself.
-  int* spill = p.part_level_spill + pbeg + part;     // entries past the shared-memory table
-  for (int q = pbeg + tid; q < pend; q += kThreads) {
-    const int lv = p.level[p.order[q]];
-    const int lvp = q > pbeg ? p.level[p.order[q - 1]] : -1;
-    if (lv != lvp) { if (lv <= kLevelCache) s_loff[lv] = q; else spill[lv] = q; }
-    if (q == pend - 1) {
-      if (lv + 1 <= kLevelCache) s_loff[lv + 1] = pend; else spill[lv + 1] = pend;
-      *s_nlev = lv + 1;
+  // Wavefront boundaries.  Sub-forest: its nodes are sorted by level, the levels are 0 .. top without
+  // gaps, every CTA builds the table for itself.  Tail: the forest's own level table from first_level on.
+  int* spill = tail ? nullptr : p.part_level_spill + pbeg + part;     // entries past the shared-memory table
+  if (tail) {
+    const int cnt = n_levels_all - first_level;
+    for (int i = tid; i <= cnt && i <= kLevelCache; i += kThreads) s_loff[i] = p.level_offset[first_level + i];
+    if (tid == 0) *s_nlev = cnt;
+  } else {
+    for (int q = pbeg + tid; q < pend; q += kThreads) {
+      const int lv = p.level[chk(p.st, p.order[q], p.n)];
+      const int lvp = q > pbeg ? p.level[chk(p.st, p.order[q - 1], p.n)] : -1;
+      if (lv != lvp) { if (lv <= kLevelCache) s_loff[lv] = q; else spill[lv] = q; }
+      if (q == pend - 1) {
+        if (lv + 1 <= kLevelCache) s_loff[lv + 1] = pend; else spill[lv + 1] = pend;
+        *s_nlev = lv + 1;
+      }
     }
   }
   __syncthreads();
   const int n_levels = *s_nlev;
-  auto loff = [&](int l) { return l <= kLevelCache ? s_loff[l] : __ldcg(spill + l); };
+  auto loff = [&](int l) {
+    return l <= kLevelCache ? s_loff[l] : (tail ? __ldcg(p.level_offset + first_level + l) : __ldcg(spill + l));
+  };
 
-  // Operands of the sub-forest, spread over the threads of the cluster: embedding rows of its
-  // leaves in ready order (Xin), and for every internal position the slots its two children
-  // deliver their state to (slot[] of a root stays -1, set by the scheduler).
-  {
+  // Operands, spread over the threads of the cluster: embedding rows of the leaves in ready order
+  // (Xin), and for every internal position the slots its two children deliver their state to
+  // (slot[] of a root is -1: set by the scheduler for sub-forests, here for a tail that starts at the
+  // leaves; a tail that starts later finds all of this done by the grid-wide kernel).
+  if (first_level == 0) {
     const int gtid = rank * kThreads + tid, gthreads = cs * kThreads;
     const int lend = loff(1);
     gather_leaf_rows(p, pbeg, lend, gtid >> 5, gthreads >> 5, lane);
     for (int pos = lend + gtid; pos < pend; pos += gthreads) {
-      const int node = p.order[pos];
-      p.slot[p.left[node]] = 2 * pos;
-      p.slot[p.right[node]] = 2 * pos + 1;
+      const int node = chk(p.st, p.order[pos], p.n);
+      p.slot[chk(p.st, p.left[node], p.n)] = 2 * pos;
+      p.slot[chk(p.st, p.right[node], p.n)] = 2 * pos + 1;
+    }
+    if (tail) {
+      const int n_roots = p.st->n_roots;
+      for (int t = gtid; t < n_roots; t += gthreads) p.slot[chk(p.st, p.roots[t], p.n)] = -1;
     }
     asm volatile("fence.proxy.async.global;" ::: "memory");    // Xin is read through TMA
   }
@@ -175,30 +200,55 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
   bool wres_ready = false;
   uint32_t armed = 0;                   // producers (lane 0): ring stages this thread has requested a box into
 
+  // How a wavefront is cut up.  Worked out a wavefront ahead (before the cluster barrier, while the
+  // stores of the current one drain), so that the first operand request goes out the moment the
+  // barrier opens.
+  struct LevelCfg {
+    int begin, end, tiles, lrt, sel, kbox, n_box;
+    uint32_t a_bytes, w_bytes, stage_bytes, n_stages;
+    bool leaf;
+  };
+  auto make_cfg = [&](int lvl) {
+    LevelCfg c;
+    c.begin = loff(lvl); c.end = loff(lvl + 1);
+    c.leaf = first_level + lvl == 0;
+    const int rows = c.end - c.begin;
+    c.tiles = (rows + BM - 1) / BM;
+    const int kblocks = c.leaf ? kb_leaf : kb_int;
+    // A wavefront of at most 64 (32) nodes fetches only that many operand rows; the MMA still
+    // spans 128 rows, what lies behind the fetched rows feeds accumulator rows that are not stored.
+    c.lrt = c.leaf || rows > 64 ? 7 : (rows > 32 ? 6 : 5);
+    c.a_bytes = 128u << c.lrt;                                                // operand rows of one K block
+    c.w_bytes = c.leaf ? (uint32_t)(G * kGColsL) * 128u : 0u;                 // leaf: W_x rows ride along; W_h is resident
+    // A stage of the ring holds one box: kbox K blocks of operand rows (+ kbox K blocks of W_x rows).
+    // A single-tile wavefront takes its operands in one request when they fit, anything else in
+    // boxes of two K blocks so that loads, MMAs and epilogues of consecutive tiles overlap.
+    c.sel = c.tiles == 1 && !(p.knob & 1) && (uint32_t)kblocks * (c.a_bytes + c.w_bytes) <= L.ring_bytes ? 0 : 1;
+    c.kbox = c.sel == 0 ? kblocks : 2;
+    c.n_box = c.sel == 0 ? 1 : (kblocks + 1) >> 1;
+    c.stage_bytes = (uint32_t)c.kbox * (c.a_bytes + c.w_bytes);
+    c.n_stages = kMaxStages;
+    while (c.n_stages * c.stage_bytes > L.ring_bytes) --c.n_stages;
+    return c;
+  };
+  LevelCfg next_cfg = make_cfg(0);
+
   for (int lvl = 0; lvl < n_levels; ++lvl) {   // same trip count in every CTA of the cluster
     if (!stop) {
-      const int begin = loff(lvl), end = loff(lvl + 1);
-      const bool leaf = lvl == 0;
+      const LevelCfg cfg = next_cfg;
+      const int begin = cfg.begin, end = cfg.end;
+      const bool leaf = cfg.leaf;
       const int rows = end - begin;
-      const int tiles = (rows + BM - 1) / BM;
+#ifdef TREELSTM_TRACE
+      if (tid == 0) TL_STAMP(trace, first_level + lvl, 0);
+#endif
+      const int tiles = cfg.tiles;
       const int kblocks = leaf ? kb_leaf : kb_int;
       const int gcols = leaf ? kGColsL : kGColsI;
       const int ncols = G * gcols;                     // accumulator columns in use
       const int ncols_mma = (ncols + 15) & ~15;        // UMMA N (columns past ncols are never read)
-      // A wavefront of at most 64 (32) nodes fetches only that many operand rows; the MMA still
-      // spans 128 rows, what lies behind the fetched rows feeds accumulator rows that are not stored.
-      const int lrt = leaf || rows > 64 ? 7 : (rows > 32 ? 6 : 5);
-      const uint32_t a_bytes = 128u << lrt;                         // operand rows of one K block
-      const uint32_t w_bytes = leaf ? (uint32_t)ncols * 128u : 0u;  // leaf: W_x rows ride along; W_h is resident
-      // A stage of the ring holds one box: kbox K blocks of operand rows (+ kbox K blocks of W_x rows).
-      // A single-tile wavefront takes its operands in one request when they fit, anything else in
-      // boxes of two K blocks so that loads, MMAs and epilogues of consecutive tiles overlap.
-      const int sel = tiles == 1 && (uint32_t)kblocks * (a_bytes + w_bytes) <= L.ring_bytes ? 0 : 1;
-      const int kbox = sel == 0 ? kblocks : 2;
-      const int n_box = sel == 0 ? 1 : (kblocks + 1) >> 1;
-      const uint32_t stage_bytes = (uint32_t)kbox * (a_bytes + w_bytes);
-      uint32_t n_stages = kMaxStages;
-      while (n_stages * stage_bytes > L.ring_bytes) --n_stages;
+      const int lrt = cfg.lrt, sel = cfg.sel, kbox = cfg.kbox, n_box = cfg.n_box;
+      const uint32_t a_bytes = cfg.a_bytes, w_bytes = cfg.w_bytes, stage_bytes = cfg.stage_bytes, n_stages = cfg.n_stages;
       stage = 0;
       int nx_node = 0, nx_slot = -1;                // epilogue: row data of the next tile, fetched a tile ahead
       bool nx_have = false;
@@ -221,6 +271,9 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
               }
               mbar_arrive_expect_tx(full_bar(stage), bytes);
               tma_load_3d(ring_addr + stage * stage_bytes + off, map, 0, y, box * kbox, full_bar(stage));
+#ifdef TREELSTM_TRACE
+              if (is_a && t == 0 && box == 0) TL_STAMP(trace, first_level + lvl, 1);
+#endif
               armed |= 1u << stage;
               if (is_a && !leaf) mbar_arrive(full_bar(stage));   // stands in for the W producer: W_h is resident
               phase_bits ^= 1u << stage;
@@ -250,6 +303,9 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
                 break;
               }
               tc_fence_after();
+#ifdef TREELSTM_TRACE
+              if (t == 0 && box == 0) TL_STAMP(trace, first_level + lvl, 2);
+#endif
               const uint32_t st_addr = ring_addr + stage * stage_bytes;
               const int nkb = min(kbox, kblocks - box * kbox);
               for (int kbi = 0; kbi < nkb; ++kbi) {
@@ -266,6 +322,9 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
               if (++stage == n_stages) stage = 0;
             }
             if (alive) umma_commit(tfull_bar(acc));      // the accumulator is complete
+#ifdef TREELSTM_TRACE
+            if (t == tiles - 1) TL_STAMP(trace, first_level + lvl, 3);
+#endif
           }
           ++acc_iter;
         } else if (warp != 10 && warp != 11) {
@@ -279,17 +338,17 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
           if (nx_have) {
             node = nx_node; slot = nx_slot;
           } else {
-            node = valid ? p.order[row] : 0;
-            slot = valid ? p.slot[node] : -1;
+            node = valid ? chk(p.st, p.order[row], p.n) : 0;
+            slot = valid ? chk_slot(p.st, p.slot[node], p.n) : -1;
           }
           // the same two dependent loads for the next tile go out now and land while this tile is computed
           nx_have = t + 1 < tiles;
           const bool valid2 = nx_have && row + BM < end;
-          if (nx_have) nx_node = valid2 ? p.order[row + BM] : 0;
+          if (nx_have) nx_node = valid2 ? chk(p.st, p.order[row + BM], p.n) : 0;
           EpiTile et;
           et.leaf = leaf; et.G = G; et.gcols = gcols; et.ncols = ncols; et.nt = nt;
           et.row = row; et.node = node; et.slot = slot; et.valid = valid;
-          et.allow_staged_out = true;
+          et.allow_staged_out = rows > 64 || (p.knob & 2);   // a narrow tile writes so little that it stores straight from registers
           et.r = r; et.e = e; et.quad = quad;
           et.cstage_addr = cstage_addr; et.cstage_ptr = cstage_ptr; et.crow_shift = L.crow_shift;
           et.half = 4 << (L.crow_shift - 7);
@@ -298,18 +357,31 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
           et.tmem_acc = tmem_base + acc * kAccCols;
           et.tfull = tfull_bar(acc); et.tempty = tempty_bar(acc); et.epi_bar = epi_bar; et.acc_phase = (acc_iter >> 1) & 1;
           et.bias = (leaf ? p.bp_x : p.bp_h) + nt * ncols + 4 * e;
-          epilogue_tile(p, et, epi_phase, alive, s_abort, [&]() { if (nx_have) nx_slot = valid2 ? p.slot[nx_node] : -1; });
+#ifdef TREELSTM_TRACE
+          if (tid == 0 && t == 0) TL_STAMP(trace, first_level + lvl, 4);
+#endif
+          epilogue_tile(p, et, epi_phase, alive, s_abort, [&]() { if (nx_have) nx_slot = valid2 ? chk_slot(p.st, p.slot[nx_node], p.n) : -1; });
+#ifdef TREELSTM_TRACE
+          if (tid == 0 && t == tiles - 1) TL_STAMP(trace, first_level + lvl, 5);
+#endif
           ++acc_iter;
         }
       }
       // the operand rows the epilogue wrote are read through TMA (async proxy) by later wavefronts
       if (warp < 4 || (warp >= 6 && warp < 10)) asm volatile("fence.proxy.async.global;" ::: "memory");
+#ifdef TREELSTM_TRACE
+      if (tid == 0) TL_STAMP(trace, first_level + lvl, 6);
+#endif
     }
     if (lvl + 1 < n_levels) {
+      next_cfg = make_cfg(lvl + 1);
       // Every thread of the cluster meets here.  A CTA in which a wait expired keeps coming to the
       // barriers (its peers must not wait for it forever) but does no more work.
       cluster_sync_all();
       if (*s_abort) stop = true;
+#ifdef TREELSTM_TRACE
+      if (tid == 0) TL_STAMP(trace, first_level + lvl, 7);
+#endif
     }
   }
 
@@ -385,17 +457,31 @@ SubforestPlan subforest_plan(treelstm* ctx) {
   return pl;
 }
 
+// tail = false: the forest was dealt out to sub-forests by the scheduler, one cluster each.
+// tail = true: one cluster finishes the narrow wavefronts at the end of the forest that the grid-wide
+// kernel (launched before on the same stream with the same tail width) left; rows are positions in the
+// forest's own ready order.
 int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
-                                  const int32_t* token, float* h, float* c, const int32_t* level, int flags,
+                                  const int32_t* token, float* h, float* c, const int32_t* level,
+                                  const int32_t* order, const int32_t* level_offset_dev, bool tail, int flags,
                                   void* ws, const WsLayout& lay, cudaStream_t stream) {
   if (!ctx->have_tmaps || !ctx->sf.ok) return TREELSTM_ERR_STATE;
   char* base = static_cast<char*>(ws);
   TcParams p{};
-  p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep; p.sched_ctas = ctx->sm_count;
+  p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep; p.sched_ctas = ctx->sm_count; p.vocab = ctx->vocab;
+  p.chk_counts = check_counters(ws, lay);
   p.left = left; p.right = right; p.token = token;
-  p.order = reinterpret_cast<int*>(base + lay.part_order);   // rows are positions in this order
+  p.order = tail ? order : reinterpret_cast<int*>(base + lay.part_order);   // rows are positions in this order
   p.roots = reinterpret_cast<int*>(base + lay.roots);
-  p.level_offset = nullptr;
+  p.level_offset = tail ? level_offset_dev : nullptr;
+  p.tail_width = tail ? ctx->opt.tail_width : 0;
+  p.tail_min_levels = ctx->opt.tail_min_levels;
+  p.trace = nullptr;
+  p.knob = ctx->opt.knob;
+#ifdef TREELSTM_TRACE
+  p.trace = reinterpret_cast<long long*>(base + lay.trace) + kTraceSlots * kTraceLevels;
+  TL_CUDA(ctx, cudaMemsetAsync(p.trace, 0, sizeof(long long) * kTraceSlots * kTraceLevels, stream));
+#endif
   p.emb_bf = ctx->emb_bf;
   p.slot = reinterpret_cast<int*>(base + lay.slot);
   p.xin = reinterpret_cast<__nv_bfloat16*>(base + lay.xin);
@@ -409,7 +495,7 @@ int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, con
   p.level = level;
   p.part_offset = reinterpret_cast<int*>(base + lay.part_offset);
   p.part_level_spill = reinterpret_cast<int*>(base + lay.part_spill);
-  p.n_parts = ctx->sf.n_parts;
+  p.n_parts = tail ? 0 : ctx->sf.n_parts;
   p.groups_per_cta = ctx->sf.groups_per_cta;
   int rc = ensure_operand_tmaps(ctx, ws, n, p.xin, p.ain);
   if (rc != TREELSTM_OK) return rc;
@@ -418,7 +504,7 @@ int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, con
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = ctx->sf.cluster_size; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-  cfg.gridDim = dim3(ctx->sf.n_parts * ctx->sf.cluster_size);
+  cfg.gridDim = dim3((tail ? 1 : ctx->sf.n_parts) * ctx->sf.cluster_size);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = ctx->sf.smem_bytes;
   cfg.stream = stream;

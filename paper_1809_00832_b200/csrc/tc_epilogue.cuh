@@ -159,8 +159,11 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, const EpiTile& 
           }
           *reinterpret_cast<uint2*>(p.ain + (size_t)slot * Hp + u0) = make_uint2(packed[0], packed[1]);
           if (count > 0) st_row4(p.cin + (size_t)slot * H + u0, vec, count, cv);
+          count_write(p.chk_counts ? p.chk_counts + p.n : nullptr, slot >> 1, count);
+          count_write(p.chk_counts ? p.chk_counts + 2 * p.n : nullptr, slot >> 1, count);
         }
         if (count > 0) {
+          count_write(p.chk_counts, node, count);
           st_row4(p.h + (size_t)node * H + u0, vec, count, hv);
           st_row4(p.c + (size_t)node * H + u0, vec, count, cv);
           if (p.gates) {
@@ -196,8 +199,11 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, const EpiTile& 
         const int uo = nt * G * 8 + 4 * ch;
         *reinterpret_cast<float4*>(p.h + (size_t)node_o * H + uo) = h4;
         *reinterpret_cast<float4*>(p.c + (size_t)node_o * H + uo) = c4;
+        count_write(p.chk_counts, node_o, 4);
         const int slot_o = t.s_rowslot[ro];
         if (slot_o >= 0) {
+          count_write(p.chk_counts ? p.chk_counts + p.n : nullptr, slot_o >> 1, 4);
+          count_write(p.chk_counts ? p.chk_counts + 2 * p.n : nullptr, slot_o >> 1, 4);
           *reinterpret_cast<float4*>(p.cin + (size_t)slot_o * H + uo) = c4;
           __nv_bfloat162 lo = __floats2bfloat162_rn(h4.x, h4.y), hi = __floats2bfloat162_rn(h4.z, h4.w);
           *reinterpret_cast<uint2*>(p.ain + (size_t)slot_o * Hp + uo) =

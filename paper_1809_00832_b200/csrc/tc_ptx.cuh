@@ -19,7 +19,8 @@ constexpr int kGColsL = 24;             // packed rows per unit group, leaves (g
 constexpr int kLevelCache = 1024;       // wavefront boundaries kept in shared memory
 
 struct TcParams {
-  int n, H, Hp, Ep, sched_ctas;
+  int n, H, Hp, Ep, sched_ctas, vocab;
+  int* chk_counts;               // checked build: write counters [h per node | Ain per position | Cin per position]
   const int *left, *right, *token, *order, *roots, *level_offset;
   int* slot;
   const __nv_bfloat16* emb_bf;
@@ -32,8 +33,34 @@ struct TcParams {
   // sub-forest (cluster) kernel only
   const int *level, *part_offset;
   int* part_level_spill;
-  int n_parts, groups_per_cta;
+  int n_parts, groups_per_cta;   // n_parts == 0: the cluster kernel runs as the tail of the grid-wide kernel
+  // hand-over from the grid-wide kernel to one cluster (persistent mode): see tail_first_level
+  int tail_width, tail_min_levels;
+  int knob;                      // development switches (0 in normal use)
+  long long* trace;              // cycle stamps (trace builds), else nullptr
 };
+
+// Where the grid-wide kernel stops and one cluster takes over: the first wavefront from which on
+// every wavefront has at most tail_width nodes, provided at least tail_min_levels wavefronts remain
+// (a hand-over costs a launch and the cluster's set-up); 0 if no wavefront is wider (the cluster then
+// evaluates the whole forest); n_levels if there is no such tail, tail_width is 0, or tail_min_levels
+// is 0 and some wavefront is wider.  Both kernels call this with the same arguments and take the
+// same decision.  Cooperative over the CTA: every thread calls it; s_tmp is one shared int.
+__device__ __forceinline__ int tail_first_level(const int* level_offset, int n_levels, int tail_width,
+                                                int tail_min_levels, int* s_tmp) {
+  if (threadIdx.x == 0) *s_tmp = 0;
+  __syncthreads();
+  int wide_end = 0;                        // 1 + the last wavefront wider than tail_width
+  for (int l = threadIdx.x; l < n_levels; l += blockDim.x)
+    if (level_offset[l + 1] - level_offset[l] > tail_width) wide_end = l + 1;
+  if (wide_end > 0) atomicMax(s_tmp, wide_end);
+  __syncthreads();
+  const int first = *s_tmp;
+  __syncthreads();                         // s_tmp may be reused by the caller
+  if (tail_width <= 0) return n_levels;
+  if (first == 0) return 0;                // no wide wavefront at all: the cluster takes the whole forest
+  return (tail_min_levels <= 0 || n_levels - first < tail_min_levels) ? n_levels : first;
+}
 
 // ---- PTX wrappers ---------------------------------------------------------------------------- //
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -169,7 +196,7 @@ __device__ __forceinline__ void gather_leaf_rows(const TcParams& p, int row_begi
   const int cpr = p.Ep / 8;                              // 16-byte chunks per row
   for (int base = row_begin + gwarp; base < row_end; base += 4 * n_warps) {
     const int my_row = base + (lane & 3) * n_warps;
-    const int my_tok = my_row < row_end ? p.token[p.order[my_row]] : 0;
+    const int my_tok = my_row < row_end ? chk(p.st, p.token[chk(p.st, p.order[my_row], p.n)], p.vocab) : 0;
     int tok[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) tok[k] = __shfl_sync(kFullMask, my_tok, k);

@@ -248,6 +248,29 @@ def draw_params(rng: np.random.Generator, H: int, E: int, vocab: int, *, emb_dis
     return p
 
 
+@dataclass
+class RecursiveParams:
+    """Parameters of a TreeRNN / RNTN model (float32): word vectors double as leaf states."""
+
+    H: int
+    vocab: int
+    emb: np.ndarray           # [vocab][H]
+    W: np.ndarray             # [2H][H]
+    b: np.ndarray             # [H]
+    V: Optional[np.ndarray] = None    # [H][2H][2H], RNTN only
+
+
+def draw_recursive_params(rng: np.random.Generator, H: int, vocab: int, *, tensor: bool, emb_scale: float,
+                          w_scale: float, v_scale: float = 0.0) -> RecursiveParams:
+    """Word vectors uniform in +-emb_scale, W and b uniform in +-w_scale, the tensor slices (RNTN,
+    tensor=True) uniform in +-v_scale."""
+    emb = rng.uniform(-emb_scale, emb_scale, size=(vocab, H)).astype(np.float32)
+    W = rng.uniform(-w_scale, w_scale, size=(2 * H, H)).astype(np.float32)
+    b = rng.uniform(-w_scale, w_scale, size=(H,)).astype(np.float32)
+    V = rng.uniform(-v_scale, v_scale, size=(H, 2 * H, 2 * H)).astype(np.float32) if tensor else None
+    return RecursiveParams(H=H, vocab=vocab, emb=emb, W=W, b=b, V=V)
+
+
 # --------------------------------------------------------------------------- #
 # named workloads
 # --------------------------------------------------------------------------- #

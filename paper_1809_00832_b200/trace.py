@@ -1,0 +1,91 @@
+"""Per-wavefront cycle tables of the bf16 wavefront kernels, from the trace build of the library.
+
+    python -m paper_1809_00832_b200.trace --workload chains64_bf16 [--mode persistent|subforests]
+                                          [--tail-width N] [--tail-min-levels M] [--trees T] [--levels A:B]
+
+The trace build (-DTREELSTM_TRACE, libtreelstm_b200_trace.so) makes the first CTA of each kernel write
+clock64 stamps for the first 256 wavefronts: the grid-wide kernel at the start of a wavefront (0),
+when its tiles are done (6) and after the grid barrier (7); the cluster kernel at the start of a
+wavefront (0), when its first operand request is out (1), when the MMA issuer sees the first box (2),
+when the last MMAs are committed (3), when the epilogue starts waiting (4), when it has stored its
+last tile (5), when the CTA arrives at the cluster barrier (6) and when it leaves it (7).  The stamps
+cost a few cycles each; the timings of the normal build are a little lower.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+
+import numpy as np
+import torch
+
+from . import binding, build, forests as fg
+
+SLOTS, LEVELS = 8, 256
+
+
+def read_trace(model: binding.TreeLSTM, which: int) -> np.ndarray:
+    buf = (ctypes.c_longlong * (SLOTS * LEVELS))()
+    fn = model.lib.treelstm_trace_read
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int]
+    got = fn(model.handle, which, ctypes.cast(buf, ctypes.c_void_p), SLOTS * LEVELS)
+    if got < 0:
+        raise binding.TreeLSTMError(got, "treelstm_trace_read")
+    return np.frombuffer(buf, dtype=np.int64).reshape(LEVELS, SLOTS).copy()
+
+
+def main() -> int:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="batch256_bf16", choices=[w for w in fg.WORKLOADS if w.endswith("bf16")])
+    ap.add_argument("--mode", default="persistent", choices=["persistent", "subforests"])
+    ap.add_argument("--tail-width", type=int, default=None)
+    ap.add_argument("--tail-min-levels", type=int, default=None)
+    ap.add_argument("--trees", type=int, default=None)
+    ap.add_argument("--levels", default=None, help="A:B - print only wavefronts A..B-1")
+    ap.add_argument("--knob", type=int, default=0, help="development switches of the kernels")
+    args = ap.parse_args()
+    build.build(variant="trace")
+    w = fg.make_workload(args.workload, 0, args.trees)
+    f, p = w.forest, w.params
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    model = binding.TreeLSTM(p.H, p.E, p.vocab, dev(p.emb), dev(p.W), dev(p.b), binding.BF16, variant="trace")
+    if args.tail_width is not None:
+        model.set_option(binding.OPT_TAIL_WIDTH, args.tail_width)
+    if args.tail_min_levels is not None:
+        model.set_option(binding.OPT_TAIL_MIN_LEVELS, args.tail_min_levels)
+    if args.knob:
+        model.set_option(100, args.knob)
+    flags = binding.PERSISTENT if args.mode == "persistent" else binding.SUBFORESTS
+    left, right, token = dev(f.left), dev(f.right), dev(f.token)
+    out = model.forward(left, right, token, flags=flags)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for i in range(4):                                   # the last call is the one read back, caches as in the bench
+        flush.fill_(i)
+        model.forward(left, right, token, flags=flags, out=out, check=False)
+    torch.cuda.synchronize()
+    widths = np.diff(out["level_offset"].cpu().numpy()[:int(out["n_levels"].item()) + 1])
+    lo, hi = 0, len(widths)
+    if args.levels:
+        a, b = args.levels.split(":")
+        lo, hi = int(a or 0), int(b or hi)
+    for which, name in ((0, "grid-wide kernel"), (1, "cluster kernel")):
+        t = read_trace(model, which)
+        rows = [l for l in range(min(len(widths), LEVELS)) if t[l, 0] != 0]
+        if not rows:
+            continue
+        print(f"# {name}: wavefronts {rows[0]}..{rows[-1]}; cycles since the wavefront's start")
+        print("level width " + " ".join(f"s{k:<6d}" for k in range(1, SLOTS)) + " total(to next start)")
+        for l in rows:
+            if not lo <= l < hi:
+                continue
+            base = t[l, 0]
+            cells = " ".join(f"{(t[l, k] - base) if t[l, k] else 0:<7d}" for k in range(1, SLOTS))
+            nxt = t[l + 1, 0] - base if l + 1 < LEVELS and t[l + 1, 0] else 0
+            print(f"{l:<5d} {int(widths[l]):<5d} {cells} {nxt}")
+        print(f"# first stamp to last stamp: {int(t[rows].max() - t[rows[0], 0])} cycles")
+    return 0
+
+
+if __name__ == "__main__":
+    raise SystemExit(main())

@@ -271,3 +271,53 @@ def test_bf16_deeper_than_the_level_cache():
             ref = res
         np.testing.assert_array_equal(res["h"], ref["h"])
         np.testing.assert_array_equal(res["c"], ref["c"])
+
+
+def test_narrow_forests_run_on_one_cluster_and_tails_can_be_handed_over():
+    """the library's own choice in persistent mode: a forest of at most 128 nodes is evaluated by one
+    cluster alone (two launches: scheduler + cluster kernel); with TAIL_MIN_LEVELS set, a larger
+    forest hands its narrow last wavefronts to the cluster.  Neither changes a bit of the result
+    (every node's contraction runs over the same K blocks in the same order)."""
+    rng = np.random.default_rng(77)
+    params = fg.draw_params(rng, 256, 300, 500, emb_dist="normal", emb_scale=0.3, w_scale=0.08)
+    model = util.make_model(params, "bf16")
+    plain = util.make_model(params, "bf16")
+    plain.set_option(binding.OPT_TAIL_WIDTH, 0)            # every wavefront on the grid-wide kernel
+    # (a) small forests: a single tree, a few trees, single leaves, one left chain
+    for shapes in ([fg.random_split_shape(rng, 56)], [fg.random_split_shape(rng, 9) for _ in range(6)], [None] * 5,
+                   [fg.left_chain_shape(60)]):
+        forest = fg.forest_from_shapes(shapes, rng, 500)
+        forest, _ = fg.permute_node_ids(forest, rng)
+        assert forest.n_nodes <= 128
+        res = util.gpu_forward(model, forest, binding.PERSISTENT)
+        assert model.last_launch_count() == 2 and model.last_mode() == binding.PERSISTENT
+        ref = util.gpu_forward(plain, forest, binding.PERSISTENT)
+        np.testing.assert_array_equal(res["h"], ref["h"])
+        np.testing.assert_array_equal(res["c"], ref["c"])
+        np.testing.assert_array_equal(res["order"], ref["order"])
+        h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
+                                        operand_round=orc.round_to_bf16)
+        assert util.max_abs(res["h"], h) < TIGHT and util.max_abs(res["c"], c) < TIGHT
+    # (b) hand-over in the middle of a forest: wide wavefronts first, then a long narrow tail
+    forest = fg.forest_from_shapes([fg.random_split_shape(rng, 40) for _ in range(30)] + [fg.left_chain_shape(50)] * 3,
+                                   rng, 500)
+    forest, _ = fg.permute_node_ids(forest, rng)
+    ref = util.gpu_forward(plain, forest, binding.PERSISTENT)
+    widths = np.diff(ref["level_offset"][:ref["n_levels"] + 1])
+    assert widths[0] > 128 and (widths[-10:] <= 128).all()
+    model.set_option(binding.OPT_TAIL_MIN_LEVELS, 3)
+    res = util.gpu_forward(model, forest, binding.PERSISTENT)
+    assert model.last_launch_count() == 3                  # scheduler, grid-wide kernel, cluster kernel
+    np.testing.assert_array_equal(res["h"], ref["h"])
+    np.testing.assert_array_equal(res["c"], ref["c"])
+    # a forest without a narrow tail long enough stays on the grid-wide kernel (the cluster kernel finds nothing to do)
+    model.set_option(binding.OPT_TAIL_MIN_LEVELS, 1000)
+    res = util.gpu_forward(model, forest, binding.PERSISTENT)
+    np.testing.assert_array_equal(res["h"], ref["h"])
+    # saved gates for backward come out of the cluster kernel too
+    small = fg.forest_from_shapes([fg.random_split_shape(rng, 30)], rng, 500)
+    a = model.forward(*(util.to_dev(x) for x in (small.left, small.right, small.token)),
+                      flags=binding.PERSISTENT | binding.SAVE_FOR_BACKWARD)
+    b = plain.forward(*(util.to_dev(x) for x in (small.left, small.right, small.token)),
+                      flags=binding.PERSISTENT | binding.SAVE_FOR_BACKWARD)
+    np.testing.assert_array_equal(a["h"].cpu().numpy(), b["h"].cpu().numpy())

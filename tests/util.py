@@ -23,7 +23,7 @@ GRAD_KEYS = ("dW", "db", "dWc", "dbc")
 
 
 def lib_ready():
-    build.build()
+    build.build(variant=binding.DEFAULT_VARIANT)
     binding.load_library()
 
 
@@ -34,11 +34,13 @@ def to_dev(a, dtype=None):
     return t.cuda()
 
 
-def make_model(params: fg.Params, precision: str) -> binding.TreeLSTM:
+def make_model(params: fg.Params, precision: str, variant=None) -> binding.TreeLSTM:
     lib_ready()
+    if variant:
+        build.build(variant=variant)
     prec = binding.FP32 if precision == "fp32" else binding.BF16
     model = binding.TreeLSTM(params.H, params.E, params.vocab, to_dev(params.emb), to_dev(params.W),
-                             to_dev(params.b), prec)
+                             to_dev(params.b), prec, variant=variant)
     if params.C:
         model.set_classifier(to_dev(params.Wc), to_dev(params.bc))
     return model
@@ -47,7 +49,7 @@ def make_model(params: fg.Params, precision: str) -> binding.TreeLSTM:
 def gpu_forward(model, forest: fg.Forest, flags: int):
     out = model.forward(to_dev(forest.left), to_dev(forest.right), to_dev(forest.token), flags=flags)
     torch.cuda.synchronize()
-    res = {k: v.cpu().numpy() for k, v in out.items()}
+    res = {k: v.cpu().numpy() for k, v in out.items() if v is not None}
     res["n_levels"] = int(res["n_levels"][0])
     return res
 
