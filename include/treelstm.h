@@ -88,19 +88,16 @@ typedef enum treelstm_status {
 #define TREELSTM_OPT_MAX_CTAS 3             /* cap on the persistent grid (0 = all co-resident CTAs) */
 #define TREELSTM_OPT_TIME_WAVEFRONT_KERNEL 4 /* 1: bracket the wavefront kernel launch(es) of each  */
                                             /* forward with CUDA events (treelstm_last_kernel_ms)    */
-#define TREELSTM_OPT_TAIL_WIDTH 5           /* TREELSTM_PERSISTENT, bf16, H padded to <= 256: a forest  */
-                                            /* of at most this many nodes (default and largest value  */
-                                            /* 128) has no wider wavefront and is evaluated by ONE     */
-                                            /* thread-block cluster (recurrent weights resident in     */
-                                            /* shared memory, hardware cluster barrier between          */
-                                            /* wavefronts) instead of the grid-wide kernel - chosen by  */
-                                            /* the library, same results; 0 switches this off          */
-#define TREELSTM_OPT_TAIL_MIN_LEVELS 6      /* > 0: a larger forest whose last wavefronts are all at    */
-                                            /* most TAIL_WIDTH nodes wide hands those over to the       */
-                                            /* cluster (a second launch) if at least this many remain;  */
-                                            /* the hand-over level is found on the device.  Default 0:  */
-                                            /* never (measured: the second launch and the cluster's     */
-                                            /* set-up cost what the narrow wavefronts save)             */
+#define TREELSTM_OPT_TAIL_WIDTH 5           /* TREELSTM_PERSISTENT, bf16, H padded to <= 256: once every */
+                                            /* remaining wavefront has at most this many nodes (default  */
+                                            /* and largest value 64) the grid-wide kernel stops and ONE   */
+                                            /* thread-block cluster finishes the forest (a second launch): */
+                                            /* recurrent weights resident in shared memory, states passed  */
+                                            /* from child to caller through distributed shared memory.     */
+                                            /* Chosen by the library on the device, same results bit for   */
+                                            /* bit; 0 keeps every wavefront on the grid-wide kernel        */
+#define TREELSTM_OPT_TAIL_MIN_LEVELS 6      /* ... provided at least this many wavefronts remain (default  */
+                                            /* 4: the hand-over costs a launch and the cluster's set-up)   */
 
 /*
  * treelstm_create - build a context for one set of parameters.

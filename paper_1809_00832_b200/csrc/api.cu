@@ -199,6 +199,7 @@ int treelstm_create(treelstm_t** out, int H, int E, int vocab, const float* emb,
   rc = copy_params(ctx, emb, W, b, s);
   if (rc != TREELSTM_OK) return fail(rc);
   ctx->sf = subforest_plan(ctx);
+  ctx->tail_ok = ctx->sf.ok && init_tail_attributes(ctx) == TREELSTM_OK;
   *out = ctx;
   return TREELSTM_OK;
 }
@@ -280,7 +281,7 @@ int treelstm_set_option(treelstm_t* ctx, int key, long long value) {
       ctx->opt.knob = (int)value;
       return TREELSTM_OK;
     case TREELSTM_OPT_TAIL_WIDTH:
-      ctx->opt.tail_width = value > 128 ? 128 : (int)value;
+      ctx->opt.tail_width = value > 64 ? 64 : (int)value;
       return TREELSTM_OK;
     case TREELSTM_OPT_TAIL_MIN_LEVELS:
       ctx->opt.tail_min_levels = value > (1 << 20) ? (1 << 20) : (int)value;
@@ -354,8 +355,7 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
     rc = launch_forward_rec(ctx, n_nodes, left, right, token, h, order, lvl_off, ctx->host_level_offset, L.n_levels,
                             persistent ? (flags | TREELSTM_PERSISTENT) : flags, workspace, lay, s);
   else if (subforests)
-    rc = launch_forward_bf16_subforest(ctx, n_nodes, left, right, token, h, c, level, order, lvl_off, false, flags,
-                                       workspace, lay, s);
+    rc = launch_forward_bf16_subforest(ctx, n_nodes, left, right, token, h, c, level, flags, workspace, lay, s);
   else if (ctx->precision == TREELSTM_BF16)
     rc = launch_forward_bf16(ctx, n_nodes, left, right, token, h, c, order, lvl_off,
                              ctx->host_level_offset, L.n_levels, persistent ? (flags | TREELSTM_PERSISTENT) : flags,
@@ -368,7 +368,9 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
     TL_CUDA(ctx, cudaEventRecord(ctx->ev_end, s));
     ctx->ev_valid = true;
   }
-  if (rc == TREELSTM_OK) rc = launch_check_counts(ctx, n_nodes, lvl_off, workspace, lay, s);
+  if (rc == TREELSTM_OK)
+    rc = launch_check_counts(ctx, n_nodes, subforests ? reinterpret_cast<const int32_t*>(base + lay.part_order) : order,
+                             left, workspace, lay, s);
   if (rc != TREELSTM_OK) L.valid = false;
   return rc;
 }

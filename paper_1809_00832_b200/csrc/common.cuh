@@ -32,7 +32,7 @@ struct WsLayout {
 
 // Cycle stamps of the wavefront kernels (builds with -DTREELSTM_TRACE only): kTraceSlots stamps per
 // wavefront for the first kTraceLevels wavefronts, written by the first CTA of each kernel.
-constexpr int kTraceSlots = 8;
+constexpr int kTraceSlots = 16;
 constexpr int kTraceLevels = 256;
 #ifdef TREELSTM_TRACE
 #define TL_STAMP(buf, level, slot)                                                            \
@@ -49,8 +49,8 @@ struct Options {
   int max_ctas = 0;
   int time_kernel = 0;
   int knob = 0;           // development switches of the tensor-core kernels (0 in normal use)
-  int tail_width = 128;   // persistent bf16 forward: forests / trailing wavefronts this narrow run on one cluster (0: never)
-  int tail_min_levels = 0; // hand a larger forest's narrow tail over if at least this many wavefronts remain (0: never)
+  int tail_width = 64;    // persistent bf16 forward: trailing wavefronts this narrow run on one cluster (0: never)
+  int tail_min_levels = 4; // ... if at least this many of them remain (a hand-over costs a launch and the cluster's set-up)
 };
 
 constexpr int kRadixBins = 256;
@@ -119,6 +119,7 @@ struct treelstm {
   int tmap_ws_rows = 0;
   bool have_tmaps = false;
   tl::SubforestPlan sf;                 // filled at create (bf16 only)
+  bool tail_ok = false;                 // the tail kernel exists for this context's sizes
 
   tl::Options opt;
 
@@ -203,9 +204,14 @@ int ensure_operand_tmaps(treelstm* ctx, void* ws, int n, const void* xin, const 
 // subforest_tc.cu
 SubforestPlan subforest_plan(treelstm* ctx);
 int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
-                                  const int32_t* token, float* h, float* c, const int32_t* level,
-                                  const int32_t* order, const int32_t* level_offset_dev, bool tail, int flags,
+                                  const int32_t* token, float* h, float* c, const int32_t* level, int flags,
                                   void* ws, const WsLayout& lay, cudaStream_t stream);
+
+// tail_tc.cu: one cluster for the narrow wavefronts at the end of a forest
+int init_tail_attributes(treelstm* ctx);
+int launch_forward_bf16_tail(treelstm* ctx, int n, const int32_t* left, const int32_t* right, const int32_t* token,
+                             float* h, float* c, const int32_t* order, const int32_t* level_offset_dev, int flags,
+                             void* ws, const WsLayout& lay, cudaStream_t stream);
 
 int launch_selftest_waits(treelstm* ctx, void* ws, int* result_dev, cudaStream_t stream);
 
@@ -217,7 +223,7 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
 // Checked build: clears the per-row write counters before a forward / compares them after it
 // (schedule.cu); both do nothing in the normal build.  Counters: [h per node | Ain per position | Cin per position].
 int launch_check_clear(treelstm* ctx, int n, void* ws, const WsLayout& lay, cudaStream_t stream);
-int launch_check_counts(treelstm* ctx, int n, const int32_t* level_offset_dev, void* ws, const WsLayout& lay,
+int launch_check_counts(treelstm* ctx, int n, const int32_t* rows, const int32_t* left, void* ws, const WsLayout& lay,
                         cudaStream_t stream);
 inline int* check_counters(void* ws, const WsLayout& lay) {
 #ifdef TREELSTM_CHECKED

@@ -178,7 +178,6 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   // hardware cluster barrier instead of the grid-wide one.
   __shared__ int s_stop;
   const int lvl_stop = only_level < 0 ? tail_first_level(p.level_offset, n_levels, p.tail_width, p.tail_min_levels, &s_stop) : n_levels;
-  if (only_level < 0 && lvl_stop == 0) return;      // the whole forest is narrow: all of it runs on the cluster
 #ifdef TREELSTM_TRACE
   long long* const trace = blockIdx.x == 0 && tid == 0 ? p.trace : nullptr;
 #endif
@@ -645,12 +644,10 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.st = reinterpret_cast<DevStatus*>(base + lay.status);
   p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
   p.level = nullptr; p.part_offset = nullptr; p.part_level_spill = nullptr; p.n_parts = 0; p.groups_per_cta = 0;
-  // Narrow forests and (if asked for) the narrow wavefronts at the end of a forest go to one cluster,
-  // where the cluster kernel exists for these sizes: a forest of at most tail_width nodes has no wider
-  // wavefront and runs there as a whole; a larger one is handed over only with tail_min_levels > 0.
-  const bool tail_ok = (flags & TREELSTM_PERSISTENT) && ctx->sf.ok && ctx->opt.tail_width > 0 && ctx->opt.max_ctas == 0;
-  const bool cluster_only = tail_ok && n <= ctx->opt.tail_width;
-  const bool with_tail = cluster_only || (tail_ok && ctx->opt.tail_min_levels > 0);
+  // The narrow wavefronts at the end of a forest go to one cluster (tail_tc.cu) where that kernel
+  // exists for these sizes; where the hand-over happens is decided on the device from the level table.
+  const bool with_tail = (flags & TREELSTM_PERSISTENT) && ctx->tail_ok && ctx->opt.tail_width > 0 &&
+                         ctx->opt.tail_min_levels > 0 && ctx->opt.max_ctas == 0;
   p.tail_width = with_tail ? ctx->opt.tail_width : 0;
   p.tail_min_levels = ctx->opt.tail_min_levels;
   p.trace = nullptr;
@@ -672,14 +669,12 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
     int only = -1;
     void* args[] = {&ctx->maps, &p, &only};
-    if (!cluster_only) {
-      TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc, dim3(grid), dim3(kThreads), args,
-                                               kSmemBytes, stream));
-      ctx->launches += 1;
-    }
-    if (with_tail)
-      return launch_forward_bf16_subforest(ctx, n, left, right, token, h, c, nullptr, order, level_offset_dev, true,
-                                           flags, ws, lay, stream);
+    TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc, dim3(grid), dim3(kThreads), args,
+                                             kSmemBytes, stream));
+    ctx->launches += 1;
+    // a forest of n nodes has fewer than n / 2 wavefronts above the leaves: too few for a hand-over
+    if (with_tail && n / 2 >= ctx->opt.tail_min_levels)
+      return launch_forward_bf16_tail(ctx, n, left, right, token, h, c, order, level_offset_dev, flags, ws, lay, stream);
     return TREELSTM_OK;
   }
   if (n_levels_host > 0) {

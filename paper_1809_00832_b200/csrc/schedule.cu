@@ -629,14 +629,15 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
 namespace {
 // After a forward: every node's h row written once (H units), every internal position's operand rows
 // (bf16 path) twice - one half per child -, no leaf position's operand row at all.
-__global__ void k_check_counts(int n, int H, int bf16, const int* level_offset, const int* counts, DevStatus* st) {
+__global__ void k_check_counts(int n, int H, int bf16, const int* rows, const int* left, const int* counts,
+                               DevStatus* st) {
   if (st->status != 0) return;
   const int k = blockIdx.x * blockDim.x + threadIdx.x;
   if (k >= n) return;
-  const int n_leaves = level_offset[1];
   bool ok = counts[k] == H;
   if (bf16) {
-    const int want = k < n_leaves ? 0 : 2 * H;
+    // rows[k]: the node whose operand row sits at position k (ready order, or the order by sub-forest)
+    const int want = left[chk(st, rows[k], n)] < 0 ? 0 : 2 * H;
     ok = ok && counts[n + k] == want && counts[2 * n + k] == want;
   }
   if (!ok) report(st, TREELSTM_ERR_CHECK);
@@ -653,17 +654,17 @@ int launch_check_clear(treelstm* ctx, int n, void* ws, const WsLayout& lay, cuda
   return TREELSTM_OK;
 }
 
-int launch_check_counts(treelstm* ctx, int n, const int32_t* level_offset_dev, void* ws, const WsLayout& lay,
+int launch_check_counts(treelstm* ctx, int n, const int32_t* rows, const int32_t* left, void* ws, const WsLayout& lay,
                         cudaStream_t stream) {
 #ifdef TREELSTM_CHECKED
   if (n > 0) {
     DevStatus* st = reinterpret_cast<DevStatus*>(static_cast<char*>(ws) + lay.status);
     k_check_counts<<<(n + 255) / 256, 256, 0, stream>>>(n, ctx->H, ctx->precision == TREELSTM_BF16 ? 1 : 0,
-                                                        level_offset_dev, check_counters(ws, lay), st);
+                                                        rows, left, check_counters(ws, lay), st);
     TL_CUDA(ctx, cudaGetLastError());
   }
 #else
-  (void)ctx; (void)n; (void)level_offset_dev; (void)ws; (void)lay; (void)stream;
+  (void)ctx; (void)n; (void)rows; (void)left; (void)ws; (void)lay; (void)stream;
 #endif
   return TREELSTM_OK;
 }

@@ -105,16 +105,9 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
   const int n_levels_all = ld_volatile(&p.st->n_levels);
   if (n_levels_all <= 0) return;
   const int cs = (int)cluster_nctarank(), rank = (int)cluster_ctarank();
-  const bool tail = p.n_parts == 0;                 // one cluster finishes what the grid-wide kernel left
-  const int part = tail ? 0 : blockIdx.x / cs;
-  __shared__ int s_first;
-  int first_level = 0;                              // tail: absolute index of the first wavefront done here
-  if (tail) {
-    first_level = tail_first_level(p.level_offset, n_levels_all, p.tail_width, p.tail_min_levels, &s_first);
-    if (first_level >= n_levels_all) return;        // nothing left (the same answer in every CTA)
-  }
-  const int pbeg = tail ? p.level_offset[first_level] : p.part_offset[part];
-  const int pend = tail ? p.n : p.part_offset[part + 1];
+  const int part = blockIdx.x / cs;
+  const int pbeg = p.part_offset[part];
+  const int pend = p.part_offset[part + 1];
   if (pbeg >= pend) return;                         // empty sub-forest: the whole cluster leaves
 #ifdef TREELSTM_TRACE
   long long* const trace = blockIdx.x == 0 ? p.trace : nullptr;
@@ -148,35 +141,26 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
     tma_load_3d(wres_addr, &sfm.wres, 0, nt * G * kGColsI, 0, wres_bar);
   }
 
-  // Wavefront boundaries.  Sub-forest: its nodes are sorted by level, the levels are 0 .. top without
-  // gaps, every CTA builds the table for itself.  Tail: the forest's own level table from first_level on.
-  int* spill = tail ? nullptr : p.part_level_spill + pbeg + part;     // entries past the shared-memory table
-  if (tail) {
-    const int cnt = n_levels_all - first_level;
-    for (int i = tid; i <= cnt && i <= kLevelCache; i += kThreads) s_loff[i] = p.level_offset[first_level + i];
-    if (tid == 0) *s_nlev = cnt;
-  } else {
-    for (int q = pbeg + tid; q < pend; q += kThreads) {
-      const int lv = p.level[chk(p.st, p.order[q], p.n)];
-      const int lvp = q > pbeg ? p.level[chk(p.st, p.order[q - 1], p.n)] : -1;
-      if (lv != lvp) { if (lv <= kLevelCache) s_loff[lv] = q; else spill[lv] = q; }
-      if (q == pend - 1) {
-        if (lv + 1 <= kLevelCache) s_loff[lv + 1] = pend; else spill[lv + 1] = pend;
-        *s_nlev = lv + 1;
-      }
+  // Wavefront boundaries of the sub-forest: its nodes are sorted by level, the levels are 0 .. top
+  // without gaps.  Every CTA builds the table for itself.
+  int* spill = p.part_level_spill + pbeg + part;     // entries past the shared-memory table
+  for (int q = pbeg + tid; q < pend; q += kThreads) {
+    const int lv = p.level[chk(p.st, p.order[q], p.n)];
+    const int lvp = q > pbeg ? p.level[chk(p.st, p.order[q - 1], p.n)] : -1;
+    if (lv != lvp) { if (lv <= kLevelCache) s_loff[lv] = q; else spill[lv] = q; }
+    if (q == pend - 1) {
+      if (lv + 1 <= kLevelCache) s_loff[lv + 1] = pend; else spill[lv + 1] = pend;
+      *s_nlev = lv + 1;
     }
   }
   __syncthreads();
   const int n_levels = *s_nlev;
-  auto loff = [&](int l) {
-    return l <= kLevelCache ? s_loff[l] : (tail ? __ldcg(p.level_offset + first_level + l) : __ldcg(spill + l));
-  };
+  auto loff = [&](int l) { return l <= kLevelCache ? s_loff[l] : __ldcg(spill + l); };
 
-  // Operands, spread over the threads of the cluster: embedding rows of the leaves in ready order
-  // (Xin), and for every internal position the slots its two children deliver their state to
-  // (slot[] of a root is -1: set by the scheduler for sub-forests, here for a tail that starts at the
-  // leaves; a tail that starts later finds all of this done by the grid-wide kernel).
-  if (first_level == 0) {
+  // Operands of the sub-forest, spread over the threads of the cluster: embedding rows of its
+  // leaves in ready order (Xin), and for every internal position the slots its two children
+  // deliver their state to (slot[] of a root stays -1, set by the scheduler).
+  {
     const int gtid = rank * kThreads + tid, gthreads = cs * kThreads;
     const int lend = loff(1);
     gather_leaf_rows(p, pbeg, lend, gtid >> 5, gthreads >> 5, lane);
@@ -184,10 +168,6 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
       const int node = chk(p.st, p.order[pos], p.n);
       p.slot[chk(p.st, p.left[node], p.n)] = 2 * pos;
       p.slot[chk(p.st, p.right[node], p.n)] = 2 * pos + 1;
-    }
-    if (tail) {
-      const int n_roots = p.st->n_roots;
-      for (int t = gtid; t < n_roots; t += gthreads) p.slot[chk(p.st, p.roots[t], p.n)] = -1;
     }
     asm volatile("fence.proxy.async.global;" ::: "memory");    // Xin is read through TMA
   }
@@ -211,7 +191,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
   auto make_cfg = [&](int lvl) {
     LevelCfg c;
     c.begin = loff(lvl); c.end = loff(lvl + 1);
-    c.leaf = first_level + lvl == 0;
+    c.leaf = lvl == 0;
     const int rows = c.end - c.begin;
     c.tiles = (rows + BM - 1) / BM;
     const int kblocks = c.leaf ? kb_leaf : kb_int;
@@ -240,7 +220,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
       const bool leaf = cfg.leaf;
       const int rows = end - begin;
 #ifdef TREELSTM_TRACE
-      if (tid == 0) TL_STAMP(trace, first_level + lvl, 0);
+      if (tid == 0) TL_STAMP(trace, lvl, 0);
 #endif
       const int tiles = cfg.tiles;
       const int kblocks = leaf ? kb_leaf : kb_int;
@@ -272,7 +252,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
               mbar_arrive_expect_tx(full_bar(stage), bytes);
               tma_load_3d(ring_addr + stage * stage_bytes + off, map, 0, y, box * kbox, full_bar(stage));
 #ifdef TREELSTM_TRACE
-              if (is_a && t == 0 && box == 0) TL_STAMP(trace, first_level + lvl, 1);
+              if (is_a && t == 0 && box == 0) TL_STAMP(trace, lvl, 1);
 #endif
               armed |= 1u << stage;
               if (is_a && !leaf) mbar_arrive(full_bar(stage));   // stands in for the W producer: W_h is resident
@@ -304,7 +284,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
               }
               tc_fence_after();
 #ifdef TREELSTM_TRACE
-              if (t == 0 && box == 0) TL_STAMP(trace, first_level + lvl, 2);
+              if (t == 0 && box == 0) TL_STAMP(trace, lvl, 2);
 #endif
               const uint32_t st_addr = ring_addr + stage * stage_bytes;
               const int nkb = min(kbox, kblocks - box * kbox);
@@ -323,7 +303,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
             }
             if (alive) umma_commit(tfull_bar(acc));      // the accumulator is complete
 #ifdef TREELSTM_TRACE
-            if (t == tiles - 1) TL_STAMP(trace, first_level + lvl, 3);
+            if (t == tiles - 1) TL_STAMP(trace, lvl, 3);
 #endif
           }
           ++acc_iter;
@@ -358,11 +338,11 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
           et.tfull = tfull_bar(acc); et.tempty = tempty_bar(acc); et.epi_bar = epi_bar; et.acc_phase = (acc_iter >> 1) & 1;
           et.bias = (leaf ? p.bp_x : p.bp_h) + nt * ncols + 4 * e;
 #ifdef TREELSTM_TRACE
-          if (tid == 0 && t == 0) TL_STAMP(trace, first_level + lvl, 4);
+          if (tid == 0 && t == 0) TL_STAMP(trace, lvl, 4);
 #endif
           epilogue_tile(p, et, epi_phase, alive, s_abort, [&]() { if (nx_have) nx_slot = valid2 ? chk_slot(p.st, p.slot[nx_node], p.n) : -1; });
 #ifdef TREELSTM_TRACE
-          if (tid == 0 && t == tiles - 1) TL_STAMP(trace, first_level + lvl, 5);
+          if (tid == 0 && t == tiles - 1) TL_STAMP(trace, lvl, 5);
 #endif
           ++acc_iter;
         }
@@ -370,7 +350,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
       // the operand rows the epilogue wrote are read through TMA (async proxy) by later wavefronts
       if (warp < 4 || (warp >= 6 && warp < 10)) asm volatile("fence.proxy.async.global;" ::: "memory");
 #ifdef TREELSTM_TRACE
-      if (tid == 0) TL_STAMP(trace, first_level + lvl, 6);
+      if (tid == 0) TL_STAMP(trace, lvl, 6);
 #endif
     }
     if (lvl + 1 < n_levels) {
@@ -380,7 +360,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
       cluster_sync_all();
       if (*s_abort) stop = true;
 #ifdef TREELSTM_TRACE
-      if (tid == 0) TL_STAMP(trace, first_level + lvl, 7);
+      if (tid == 0) TL_STAMP(trace, lvl, 7);
 #endif
     }
   }
@@ -457,13 +437,8 @@ SubforestPlan subforest_plan(treelstm* ctx) {
   return pl;
 }
 
-// tail = false: the forest was dealt out to sub-forests by the scheduler, one cluster each.
-// tail = true: one cluster finishes the narrow wavefronts at the end of the forest that the grid-wide
-// kernel (launched before on the same stream with the same tail width) left; rows are positions in the
-// forest's own ready order.
 int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, const int32_t* right,
-                                  const int32_t* token, float* h, float* c, const int32_t* level,
-                                  const int32_t* order, const int32_t* level_offset_dev, bool tail, int flags,
+                                  const int32_t* token, float* h, float* c, const int32_t* level, int flags,
                                   void* ws, const WsLayout& lay, cudaStream_t stream) {
   if (!ctx->have_tmaps || !ctx->sf.ok) return TREELSTM_ERR_STATE;
   char* base = static_cast<char*>(ws);
@@ -471,11 +446,11 @@ int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, con
   p.n = n; p.H = ctx->H; p.Hp = ctx->Hp; p.Ep = ctx->Ep; p.sched_ctas = ctx->sm_count; p.vocab = ctx->vocab;
   p.chk_counts = check_counters(ws, lay);
   p.left = left; p.right = right; p.token = token;
-  p.order = tail ? order : reinterpret_cast<int*>(base + lay.part_order);   // rows are positions in this order
+  p.order = reinterpret_cast<int*>(base + lay.part_order);   // rows are positions in this order
   p.roots = reinterpret_cast<int*>(base + lay.roots);
-  p.level_offset = tail ? level_offset_dev : nullptr;
-  p.tail_width = tail ? ctx->opt.tail_width : 0;
-  p.tail_min_levels = ctx->opt.tail_min_levels;
+  p.level_offset = nullptr;
+  p.tail_width = 0;
+  p.tail_min_levels = 0;
   p.trace = nullptr;
   p.knob = ctx->opt.knob;
 #ifdef TREELSTM_TRACE
@@ -495,7 +470,7 @@ int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, con
   p.level = level;
   p.part_offset = reinterpret_cast<int*>(base + lay.part_offset);
   p.part_level_spill = reinterpret_cast<int*>(base + lay.part_spill);
-  p.n_parts = tail ? 0 : ctx->sf.n_parts;
+  p.n_parts = ctx->sf.n_parts;
   p.groups_per_cta = ctx->sf.groups_per_cta;
   int rc = ensure_operand_tmaps(ctx, ws, n, p.xin, p.ain);
   if (rc != TREELSTM_OK) return rc;
@@ -504,7 +479,7 @@ int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, con
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = ctx->sf.cluster_size; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-  cfg.gridDim = dim3((tail ? 1 : ctx->sf.n_parts) * ctx->sf.cluster_size);
+  cfg.gridDim = dim3(ctx->sf.n_parts * ctx->sf.cluster_size);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = ctx->sf.smem_bytes;
   cfg.stream = stream;

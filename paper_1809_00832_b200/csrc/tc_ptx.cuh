@@ -40,26 +40,24 @@ struct TcParams {
   long long* trace;              // cycle stamps (trace builds), else nullptr
 };
 
-// Where the grid-wide kernel stops and one cluster takes over: the first wavefront from which on
-// every wavefront has at most tail_width nodes, provided at least tail_min_levels wavefronts remain
-// (a hand-over costs a launch and the cluster's set-up); 0 if no wavefront is wider (the cluster then
-// evaluates the whole forest); n_levels if there is no such tail, tail_width is 0, or tail_min_levels
-// is 0 and some wavefront is wider.  Both kernels call this with the same arguments and take the
-// same decision.  Cooperative over the CTA: every thread calls it; s_tmp is one shared int.
+// Where the grid-wide kernel stops and one cluster takes over (persistent mode): the first wavefront
+// - never the leaves - from which on every wavefront has at most tail_width nodes, provided at least
+// tail_min_levels wavefronts remain (a hand-over costs a launch and the cluster's set-up); n_levels if
+// there is no such tail or tail_width is 0.  Both kernels call this with the same arguments and take
+// the same decision.  Cooperative over the CTA: every thread calls it; s_tmp is one shared int.
 __device__ __forceinline__ int tail_first_level(const int* level_offset, int n_levels, int tail_width,
                                                 int tail_min_levels, int* s_tmp) {
-  if (threadIdx.x == 0) *s_tmp = 0;
+  if (threadIdx.x == 0) *s_tmp = 1;        // the leaf wavefront always stays with the grid-wide kernel
   __syncthreads();
   int wide_end = 0;                        // 1 + the last wavefront wider than tail_width
   for (int l = threadIdx.x; l < n_levels; l += blockDim.x)
     if (level_offset[l + 1] - level_offset[l] > tail_width) wide_end = l + 1;
-  if (wide_end > 0) atomicMax(s_tmp, wide_end);
+  if (wide_end > 1) atomicMax(s_tmp, wide_end);
   __syncthreads();
   const int first = *s_tmp;
   __syncthreads();                         // s_tmp may be reused by the caller
-  if (tail_width <= 0) return n_levels;
-  if (first == 0) return 0;                // no wide wavefront at all: the cluster takes the whole forest
-  return (tail_min_levels <= 0 || n_levels - first < tail_min_levels) ? n_levels : first;
+  if (tail_width <= 0 || n_levels - first < (tail_min_levels > 1 ? tail_min_levels : 1)) return n_levels;
+  return first;
 }
 
 // ---- PTX wrappers ---------------------------------------------------------------------------- //

@@ -21,7 +21,7 @@ import torch
 
 from . import binding, build, forests as fg
 
-SLOTS, LEVELS = 8, 256
+SLOTS, LEVELS = 16, 256
 
 
 def read_trace(model: binding.TreeLSTM, which: int) -> np.ndarray:

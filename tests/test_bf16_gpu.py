@@ -273,51 +273,59 @@ def test_bf16_deeper_than_the_level_cache():
         np.testing.assert_array_equal(res["c"], ref["c"])
 
 
-def test_narrow_forests_run_on_one_cluster_and_tails_can_be_handed_over():
-    """the library's own choice in persistent mode: a forest of at most 128 nodes is evaluated by one
-    cluster alone (two launches: scheduler + cluster kernel); with TAIL_MIN_LEVELS set, a larger
-    forest hands its narrow last wavefronts to the cluster.  Neither changes a bit of the result
-    (every node's contraction runs over the same K blocks in the same order)."""
+def test_narrow_tails_are_handed_to_one_cluster():
+    """the library's own choice in persistent mode: once every remaining wavefront has at most 64 nodes
+    (and at least four remain) the grid-wide kernel stops and one cluster finishes the forest, passing
+    states from child to caller through distributed shared memory.  Where the hand-over happens is
+    decided on the device; it changes no bit of the result (every node's contraction runs over the
+    same products in the same order), whatever the shape of the tail."""
     rng = np.random.default_rng(77)
-    params = fg.draw_params(rng, 256, 300, 500, emb_dist="normal", emb_scale=0.3, w_scale=0.08)
-    model = util.make_model(params, "bf16")
-    plain = util.make_model(params, "bf16")
-    plain.set_option(binding.OPT_TAIL_WIDTH, 0)            # every wavefront on the grid-wide kernel
-    # (a) small forests: a single tree, a few trees, single leaves, one left chain
-    for shapes in ([fg.random_split_shape(rng, 56)], [fg.random_split_shape(rng, 9) for _ in range(6)], [None] * 5,
-                   [fg.left_chain_shape(60)]):
-        forest = fg.forest_from_shapes(shapes, rng, 500)
-        forest, _ = fg.permute_node_ids(forest, rng)
-        assert forest.n_nodes <= 128
+    for H, E in ((256, 300), (150, 64), (128, 40), (64, 64)):
+        params = fg.draw_params(rng, H, E, 500, emb_dist="normal", emb_scale=0.3, w_scale=0.08)
+        model = util.make_model(params, "bf16")
+        plain = util.make_model(params, "bf16")
+        plain.set_option(binding.OPT_TAIL_WIDTH, 0)            # every wavefront on the grid-wide kernel
+        cases = [
+            [fg.random_split_shape(rng, 56)],                                        # one tree
+            [fg.random_split_shape(rng, 9) for _ in range(6)] + [None] * 3,          # a few small trees, single leaves
+            [fg.left_chain_shape(60), fg.left_chain_shape(33)],                      # callers one wavefront up, leaves far below
+            [fg.balanced_shape(64)],                                                 # both children always one wavefront below
+            [fg.random_split_shape(rng, 40) for _ in range(30)] + [fg.left_chain_shape(50)] * 3,   # wide first, long narrow tail
+            [fg.left_chain_shape(70)] * 64,                                          # exactly 64 nodes per wavefront
+        ]
+        for shapes in cases:
+            forest = fg.forest_from_shapes(shapes, rng, 500)
+            forest, _ = fg.permute_node_ids(forest, rng)
+            ref = util.gpu_forward(plain, forest, binding.PERSISTENT)
+            assert plain.last_launch_count() == 2
+            res = util.gpu_forward(model, forest, binding.PERSISTENT)
+            widths = np.diff(ref["level_offset"][:ref["n_levels"] + 1])
+            narrow_tail = int(np.argmax(np.append(widths[::-1] > 64, True)))        # wavefronts at the end with <= 64 nodes
+            narrow_tail = min(narrow_tail, len(widths) - 1)                          # the leaves never count
+            assert model.last_launch_count() == 3 and model.last_mode() == binding.PERSISTENT
+            assert narrow_tail >= 4                                                  # every case has a tail to hand over
+            np.testing.assert_array_equal(res["order"], ref["order"])
+            np.testing.assert_array_equal(res["h"], ref["h"])
+            np.testing.assert_array_equal(res["c"], ref["c"])
+            h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
+                                            operand_round=orc.round_to_bf16)
+            assert util.max_abs(res["h"], h) < TIGHT and util.max_abs(res["c"], c) < TIGHT
+        # a forest without a narrow tail long enough stays on the grid-wide kernel (the cluster finds nothing to do)
+        model.set_option(binding.OPT_TAIL_MIN_LEVELS, 1000)
         res = util.gpu_forward(model, forest, binding.PERSISTENT)
-        assert model.last_launch_count() == 2 and model.last_mode() == binding.PERSISTENT
-        ref = util.gpu_forward(plain, forest, binding.PERSISTENT)
         np.testing.assert_array_equal(res["h"], ref["h"])
-        np.testing.assert_array_equal(res["c"], ref["c"])
-        np.testing.assert_array_equal(res["order"], ref["order"])
-        h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
-                                        operand_round=orc.round_to_bf16)
-        assert util.max_abs(res["h"], h) < TIGHT and util.max_abs(res["c"], c) < TIGHT
-    # (b) hand-over in the middle of a forest: wide wavefronts first, then a long narrow tail
-    forest = fg.forest_from_shapes([fg.random_split_shape(rng, 40) for _ in range(30)] + [fg.left_chain_shape(50)] * 3,
-                                   rng, 500)
-    forest, _ = fg.permute_node_ids(forest, rng)
-    ref = util.gpu_forward(plain, forest, binding.PERSISTENT)
-    widths = np.diff(ref["level_offset"][:ref["n_levels"] + 1])
-    assert widths[0] > 128 and (widths[-10:] <= 128).all()
-    model.set_option(binding.OPT_TAIL_MIN_LEVELS, 3)
-    res = util.gpu_forward(model, forest, binding.PERSISTENT)
-    assert model.last_launch_count() == 3                  # scheduler, grid-wide kernel, cluster kernel
-    np.testing.assert_array_equal(res["h"], ref["h"])
-    np.testing.assert_array_equal(res["c"], ref["c"])
-    # a forest without a narrow tail long enough stays on the grid-wide kernel (the cluster kernel finds nothing to do)
-    model.set_option(binding.OPT_TAIL_MIN_LEVELS, 1000)
-    res = util.gpu_forward(model, forest, binding.PERSISTENT)
-    np.testing.assert_array_equal(res["h"], ref["h"])
-    # saved gates for backward come out of the cluster kernel too
-    small = fg.forest_from_shapes([fg.random_split_shape(rng, 30)], rng, 500)
-    a = model.forward(*(util.to_dev(x) for x in (small.left, small.right, small.token)),
-                      flags=binding.PERSISTENT | binding.SAVE_FOR_BACKWARD)
-    b = plain.forward(*(util.to_dev(x) for x in (small.left, small.right, small.token)),
-                      flags=binding.PERSISTENT | binding.SAVE_FOR_BACKWARD)
-    np.testing.assert_array_equal(a["h"].cpu().numpy(), b["h"].cpu().numpy())
+        model.set_option(binding.OPT_TAIL_MIN_LEVELS, 4)
+        # saved gates for backward come out of the cluster kernel too
+        small = fg.forest_from_shapes([fg.random_split_shape(rng, 30)], rng, 500)
+        arrs = [util.to_dev(x) for x in (small.left, small.right, small.token)]
+        labels = util.to_dev(rng.integers(0, 3, size=small.n_nodes).astype(np.int32))
+        Wc, bc = util.to_dev(rng.uniform(-0.1, 0.1, (H, 3)).astype(np.float32)), util.to_dev(np.zeros(3, np.float32))
+        grads = []
+        for m in (model, plain):
+            m.set_classifier(Wc, bc)
+            m.forward(*arrs, flags=binding.PERSISTENT | binding.SAVE_FOR_BACKWARD)
+            g = m.backward(labels, small.n_leaves)
+            grads.append({k: v.cpu().numpy() for k, v in g.items()})
+        np.testing.assert_allclose(grads[0]["dW"], grads[1]["dW"], rtol=0, atol=1e-7)
+        np.testing.assert_allclose(grads[0]["loss"], grads[1]["loss"], rtol=0, atol=1e-6)
+        model.close(); plain.close()
