@@ -350,8 +350,17 @@ def run_sweeps(args):
     from paper_1809_00832_b200 import binding, build
     build.build()
     rng = np.random.default_rng(0)
-    p = fg.draw_params(rng, 256, 300, 20000, emb_dist="normal", emb_scale=0.1, w_scale=0.05)
-    model = binding.TreeLSTM(p.H, p.E, p.vocab, _dev(p.emb), _dev(p.W), _dev(p.b), binding.BF16)
+    if args.cell == "treelstm":
+        p = fg.draw_params(rng, 256, 300, 20000, emb_dist="normal", emb_scale=0.1, w_scale=0.05)
+        model = binding.TreeLSTM(p.H, p.E, p.vocab, _dev(p.emb), _dev(p.W), _dev(p.b), binding.BF16)
+    else:
+        # the paper's Table 1 is measured on TreeRNN; the other cells run fp32 kernels on the same scheduler
+        tensor = args.cell == "rntn"
+        H = 32 if tensor else 128
+        p = fg.draw_recursive_params(rng, H, 20000, tensor=tensor, emb_scale=0.5, w_scale=1.0 / np.sqrt(2 * H),
+                                     v_scale=1.0 / (2 * H))
+        model = binding.TreeLSTM.recursive(binding.CELL_RNTN if tensor else binding.CELL_TREERNN, H, p.vocab,
+                                           _dev(p.emb), _dev(p.W), _dev(p.b), _dev(p.V) if tensor else None)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
 
     flags = {"persistent": binding.PERSISTENT, "per_level": binding.PER_LEVEL, "subforests": binding.SUBFORESTS}[args.mode]
@@ -377,13 +386,13 @@ def run_sweeps(args):
             for batch in (1, 10, 25):
                 forest = fg.forest_from_shapes([make() for _ in range(batch)], rng, p.vocab)
                 ms, levels = time_forest(forest)
-                print(json.dumps({"sweep": "shape", "mode": args.mode, "shape": name, "leaves_per_tree": 32, "batch": batch,
+                print(json.dumps({"sweep": "shape", "cell": args.cell, "mode": args.mode, "shape": name, "leaves_per_tree": 32, "batch": batch,
                                   "levels": levels, "ms_per_step": ms, "trees_per_sec": batch / (ms * 1e-3)}))
     if args.sweep in ("length", "all"):
         for leaves in (2, 4, 8, 16, 24, 32, 40, 48, 56):
             forest = fg.forest_from_shapes([fg.random_split_shape(rng, leaves)], rng, p.vocab)
             ms, levels = time_forest(forest)
-            print(json.dumps({"sweep": "length", "mode": args.mode, "leaves": leaves, "batch": 1, "levels": levels,
+            print(json.dumps({"sweep": "length", "cell": args.cell, "mode": args.mode, "leaves": leaves, "batch": 1, "levels": levels,
                               "ms_per_instance": ms}))
     return 0
 
@@ -449,6 +458,8 @@ def main() -> int:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-train", action="store_true", help="skip the extra training-step figure")
     ap.add_argument("--no-extra", action="store_true", help="skip the extra workloads and the latency-floor probe")
+    ap.add_argument("--cell", default="treelstm", choices=["treelstm", "treernn", "rntn"],
+                    help="cell of the sweeps (the benchmark line itself is always TreeLSTM)")
     ap.add_argument("--sweep", default=None, choices=["shapes", "length", "all"],
                     help="print the tree-shape / sentence-length sweeps instead of the benchmark line")
     args = ap.parse_args()

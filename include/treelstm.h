@@ -88,16 +88,24 @@ typedef enum treelstm_status {
 #define TREELSTM_OPT_MAX_CTAS 3             /* cap on the persistent grid (0 = all co-resident CTAs) */
 #define TREELSTM_OPT_TIME_WAVEFRONT_KERNEL 4 /* 1: bracket the wavefront kernel launch(es) of each  */
                                             /* forward with CUDA events (treelstm_last_kernel_ms)    */
-#define TREELSTM_OPT_TAIL_WIDTH 5           /* TREELSTM_PERSISTENT, bf16, H padded to <= 256: once every */
-                                            /* remaining wavefront has at most this many nodes (default  */
-                                            /* and largest value 64) the grid-wide kernel stops and ONE   */
-                                            /* thread-block cluster finishes the forest (a second launch): */
+#define TREELSTM_OPT_TAIL_WIDTH 5           /* TREELSTM_PERSISTENT, bf16, H padded to <= 256: the last    */
+                                            /* wavefronts of a forest, once every remaining one has at    */
+                                            /* most this many nodes (default 48, largest value 64), may   */
+                                            /* be finished by ONE thread-block cluster (a second launch): */
                                             /* recurrent weights resident in shared memory, states passed  */
                                             /* from child to caller through distributed shared memory.     */
-                                            /* Chosen by the library on the device, same results bit for   */
-                                            /* bit; 0 keeps every wavefront on the grid-wide kernel        */
-#define TREELSTM_OPT_TAIL_MIN_LEVELS 6      /* ... provided at least this many wavefronts remain (default  */
-                                            /* 4: the hand-over costs a launch and the cluster's set-up)   */
+                                            /* Decided by the library on the device (see below), same      */
+                                            /* results bit for bit; 0 keeps every wavefront on the         */
+                                            /* grid-wide kernel                                            */
+#define TREELSTM_OPT_TAIL_MIN_LEVELS 6      /* 0 (default): the hand-over happens if a cost model fitted   */
+                                            /* to cycle traces says that the narrow wavefronts save more   */
+                                            /* than the second launch costs (deep, narrow forests: yes; a  */
+                                            /* few narrow wavefronts on top of a wide forest: no).         */
+                                            /* > 0: it happens whenever at least this many wavefronts      */
+                                            /* remain                                                      */
+#define TREELSTM_OPT_TAIL_MAX_NODES 7       /* forests with more nodes than this (default 4096) never      */
+                                            /* launch the cluster kernel: the host knows the node count    */
+                                            /* only, and a large forest has nothing to gain                */
 
 /*
  * treelstm_create - build a context for one set of parameters.

@@ -286,6 +286,9 @@ int treelstm_set_option(treelstm_t* ctx, int key, long long value) {
     case TREELSTM_OPT_TAIL_MIN_LEVELS:
       ctx->opt.tail_min_levels = value > (1 << 20) ? (1 << 20) : (int)value;
       return TREELSTM_OK;
+    case TREELSTM_OPT_TAIL_MAX_NODES:
+      ctx->opt.tail_max_nodes = value > (1 << 30) ? (1 << 30) : (int)value;
+      return TREELSTM_OK;
     case TREELSTM_OPT_TIME_WAVEFRONT_KERNEL:
       if (value && !ctx->ev_begin) {
         TL_CUDA(ctx, cudaEventCreate(&ctx->ev_begin));

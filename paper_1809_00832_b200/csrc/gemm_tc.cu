@@ -176,8 +176,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   // Persistent mode: the narrow wavefronts at the end of the forest are left to one cluster (launched
   // next on the same stream), which keeps the recurrent weights in shared memory and meets at the
   // hardware cluster barrier instead of the grid-wide one.
-  __shared__ int s_stop;
-  const int lvl_stop = only_level < 0 ? tail_first_level(p.level_offset, n_levels, p.tail_width, p.tail_min_levels, &s_stop) : n_levels;
+  __shared__ int s_stop[2];
+  const int lvl_stop = only_level < 0 ? tail_first_level(p.level_offset, n_levels, p.tail_width, p.tail_min_levels, s_stop) : n_levels;
 #ifdef TREELSTM_TRACE
   long long* const trace = blockIdx.x == 0 && tid == 0 ? p.trace : nullptr;
 #endif
@@ -646,8 +646,9 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.level = nullptr; p.part_offset = nullptr; p.part_level_spill = nullptr; p.n_parts = 0; p.groups_per_cta = 0;
   // The narrow wavefronts at the end of a forest go to one cluster (tail_tc.cu) where that kernel
   // exists for these sizes; where the hand-over happens is decided on the device from the level table.
+  // (the host only knows the node count: forests too large for a narrow tail to matter skip the second launch)
   const bool with_tail = (flags & TREELSTM_PERSISTENT) && ctx->tail_ok && ctx->opt.tail_width > 0 &&
-                         ctx->opt.tail_min_levels > 0 && ctx->opt.max_ctas == 0;
+                         ctx->opt.max_ctas == 0 && n <= ctx->opt.tail_max_nodes && n >= 8;
   p.tail_width = with_tail ? ctx->opt.tail_width : 0;
   p.tail_min_levels = ctx->opt.tail_min_levels;
   p.trace = nullptr;
@@ -672,8 +673,7 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc, dim3(grid), dim3(kThreads), args,
                                              kSmemBytes, stream));
     ctx->launches += 1;
-    // a forest of n nodes has fewer than n / 2 wavefronts above the leaves: too few for a hand-over
-    if (with_tail && n / 2 >= ctx->opt.tail_min_levels)
+    if (with_tail)
       return launch_forward_bf16_tail(ctx, n, left, right, token, h, c, order, level_offset_dev, flags, ws, lay, stream);
     return TREELSTM_OK;
   }

@@ -74,6 +74,10 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 __device__ __forceinline__ void mbar_arrive_remote_release(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// arrival on an mbarrier of another CTA that carries no data of this thread with it (a pure "go ahead")
+__device__ __forceinline__ void mbar_arrive_remote_relaxed(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -128,7 +132,7 @@ __host__ __device__ inline TailLayout tail_layout(int Hp, int gpc) {
   // wavefront after next: it then holds the gate values [node][40 gpc] fp32 and, behind them, the new
   // bf16 h of this CTA's units [node][U] (source of the pushes).
   L.gate_bytes = (uint32_t)kTailRows * (uint32_t)gpc * kGColsI * 4u;
-  L.rows = off; off += 2u * 2u * (uint32_t)kTailRows * 4u;   // [buffer][node ids | slots]
+  L.rows = off; off += 2u * 3u * (uint32_t)kTailRows * 4u;   // [buffer][node ids | slots | which children are recent]
   L.bars = off; off += 256u;
   L.total = off + 1024u;                                  // alignment slack
   return L;
@@ -144,26 +148,27 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
   unsigned char* base_ptr = smem_raw + (base - raw_addr);
   const uint32_t wres_addr = base + L.wres;
   float* cbuf = reinterpret_cast<float*>(base_ptr + L.cbuf);
-  int* s_rows = reinterpret_cast<int*>(base_ptr + L.rows);      // [buf][0: node ids, 1: slots][64]
+  int* s_rows = reinterpret_cast<int*>(base_ptr + L.rows);      // [buf][0: node ids, 1: slots, 2: recent children][64]
   uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + L.bars);
   // bars: 0,1 TL (prefetch landed)  2,3 XF (pushes landed)  4 G  5,6 P  7 TF  8 TE  9 W (weights)  10 drain
-  //       11 E1 (meeting point of the epilogue threads)  12 CB (child cell states of the next wavefront fetched)
+  //       11 E1 (meeting point of the epilogue threads)  12, 14 CB (older child cell states of a wavefront fetched)
   const uint32_t bar0 = smem_u32(bars);
   auto TLb = [&](int b) { return bar0 + 8u * b; };
   auto XFb = [&](int b) { return bar0 + 8u * (2 + b); };
   const uint32_t Gb = bar0 + 8u * 4;
   auto Pb = [&](int b) { return bar0 + 8u * (5 + b); };
   const uint32_t TFb = bar0 + 8u * 7, TEb = bar0 + 8u * 8, Wb = bar0 + 8u * 9, drainb = bar0 + 8u * 10;
-  const uint32_t E1b = bar0 + 8u * 11, CBb = bar0 + 8u * 12;
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 14);
+  const uint32_t E1b = bar0 + 8u * 11;
+  auto CBb = [&](int j) { return bar0 + 8u * (j & 1 ? 14 : 12); };   // by wavefront: a phase every other wavefront
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 16);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   int* s_cnt = const_cast<int*>(s_abort) + 1;                   // [2][2] nodes that push into each buffer, per fetching warp
-  __shared__ int s_first;
+  __shared__ int s_first[2];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_levels_all = ld_volatile(&p.st->n_levels);
   if (n_levels_all <= 0) return;
-  const int first_level = tail_first_level(p.level_offset, n_levels_all, p.tail_width, p.tail_min_levels, &s_first);
+  const int first_level = tail_first_level(p.level_offset, n_levels_all, p.tail_width, p.tail_min_levels, s_first);
   if (first_level >= n_levels_all) return;          // nothing left for the cluster (the same answer in every CTA)
   const int n_lv = n_levels_all - first_level;
   const uint32_t cs = cluster_size(), rank = cluster_rank();
@@ -182,7 +187,8 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
     mbar_init(Wb, 1);
     mbar_init(drainb, 1);
     mbar_init(E1b, kEpiThreads);
-    mbar_init(CBb, 64);
+    mbar_init(CBb(0), 64);
+    mbar_init(CBb(1), 64);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -210,66 +216,82 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
   // nobody pushes into buffer 0 for its first use either: its "peers may push" phase is completed here,
   // so that the k-th use of either buffer waits for phase k of its barriers
   if (warp == 8 && lane < (int)cs) mbar_arrive_remote_release(map_to_cta(Pb(0), (uint32_t)lane));
-  // row tables and child cell states of a wavefront (node ids, delivery slots; [row][side][U] fp32 from
-  // the global operand rows): fetched by warps 10-11, one wavefront ahead
+  // Tables of a wavefront, fetched by warps 10-11 one wavefront ahead: node ids, delivery slots, and
+  // per row which of its two children finished one or two wavefronts before it inside this kernel
+  // (bit 0 left, bit 1 right) - the cell states of those children are put into the caller's shared-memory
+  // row by this CTA's own epilogue, all older ones are read from the global operand rows.
   auto fetch_rows = [&](int i, int b) {             // called by the 64 threads of warps 10-11
     const int t = tid - 320;
     const int begin = loff(i), end = loff(i + 1), nbeg = i + 1 < n_lv ? end : 0, nend = i + 1 < n_lv ? loff(i + 2) : 0;
-    int node = -1, slot = -1;
+    int node = -1, slot = -1, fresh = 0;
     if (begin + t < end) {
       node = chk(p.st, p.order[begin + t], p.n);
       slot = chk_slot(p.st, p.slot[node], p.n);
+      const int l = chk(p.st, p.left[node], p.n), r = chk(p.st, p.right[node], p.n);
+      const int newest = first_level + i - 2 > first_level ? first_level + i - 2 : first_level;
+      fresh = (p.level[l] >= newest ? 1 : 0) | (p.level[r] >= newest ? 2 : 0);
     }
-    s_rows[(b * 2 + 0) * kTailRows + t] = node;
-    s_rows[(b * 2 + 1) * kTailRows + t] = slot;
+    s_rows[(b * 3 + 0) * kTailRows + t] = node;
+    s_rows[(b * 3 + 1) * kTailRows + t] = slot;
+    s_rows[(b * 3 + 2) * kTailRows + t] = fresh;
     // how many of these nodes deliver into the next wavefront (their caller is one of its rows)
     const bool pushes = slot >= 0 && (slot >> 1) >= nbeg && (slot >> 1) < nend;
     const unsigned m = __ballot_sync(kFullMask, pushes);
     if (lane == 0) s_cnt[b * 2 + (warp - 10)] = __popc(m);
   };
-  // Only this CTA ever writes its own units of a caller's cell-state row (here or, below the tail, the
-  // grid-wide kernel), so reading them back needs no more than the CTA's own ordering.
-  auto fetch_cells = [&](int i, int b) {            // child cell states of wavefront i into cbuf[b]
+  // Child cell states of wavefront i that are older than two wavefronts: from the global operand rows
+  // into cbuf[b].  Only this CTA ever writes its own units of such a row (here or, below the tail, the
+  // grid-wide kernel), and what it wrote for children that old was written before the last CTA barrier.
+  auto fetch_cells = [&](int i, int b) {
     const int t = tid - 320;
     const int begin = loff(i), rows = loff(i + 1) - begin;
     float* dst = cbuf + (size_t)b * kTailRows * 2 * U;
+    const int* fresh = s_rows + (b * 3 + 2) * kTailRows;
+    __syncwarp();
+    asm volatile("bar.sync 2, 64;" ::: "memory");   // the flags written by both fetching warps are in
     if ((H & 3) == 0) {                             // 16-byte pieces: (row, side) runs of U floats are aligned
       const int c4 = U / 4, total = rows * 2 * c4;
       for (int e0 = 0; e0 < total; e0 += 64 * 8) {
         float4 v[8];
+        bool take[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int e = e0 + j * 64 + t;
           v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          take[j] = false;
           if (e < total) {
             const int pair = e / c4, q = e - pair * c4;         // pair = row * 2 + side
-            if (U0 + 4 * q < H)
+            take[j] = !((fresh[pair >> 1] >> (pair & 1)) & 1);
+            if (take[j] && U0 + 4 * q < H)
               v[j] = __ldcg(reinterpret_cast<const float4*>(p.cin + (size_t)(2 * begin + pair) * H + U0 + 4 * q));
           }
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int e = e0 + j * 64 + t;
-          if (e < total) reinterpret_cast<float4*>(dst)[e] = v[j];
+          if (take[j]) reinterpret_cast<float4*>(dst)[e] = v[j];
         }
       }
     } else {
       const int total = rows * 2 * U;
       for (int e0 = 0; e0 < total; e0 += 64 * 8) {
         float v[8];
+        bool take[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int e = e0 + j * 64 + t;
           v[j] = 0.f;
+          take[j] = false;
           if (e < total) {
             const int pair = e / U, u = e - pair * U;
-            if (U0 + u < H) v[j] = __ldcg(p.cin + (size_t)(2 * begin + pair) * H + U0 + u);
+            take[j] = !((fresh[pair >> 1] >> (pair & 1)) & 1);
+            if (take[j] && U0 + u < H) v[j] = __ldcg(p.cin + (size_t)(2 * begin + pair) * H + U0 + u);
           }
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int e = e0 + j * 64 + t;
-          if (e < total) dst[e] = v[j];
+          if (take[j]) dst[e] = v[j];
         }
       }
     }
@@ -277,9 +299,55 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
   if (warp >= 10) {
     fetch_rows(0, 0);
     fetch_cells(0, 0);
+    mbar_arrive(CBb(0));                            // the fetched cell states of wavefront 0 are in
   }
 
+  // what an epilogue thread keeps of its (node, unit) pairs until their copies to global memory are made
+  constexpr int kMaxItems = kTailRows * 24 / kEpiThreads;    // pairs per thread at most (U <= 24)
+  float keep_h[kMaxItems], keep_c[kMaxItems];
+  int keep_node[kMaxItems], keep_slot[kMaxItems];
+  unsigned keep_near = 0;                                    // per pair: bit 2 it: caller in the next wavefront; bit 2 it + 1: or the one after
+  int kept = 0;                                              // pairs of the previous wavefront (all threads together)
+  // Copies to global memory, for callers further up than the shared-memory hand-over reaches and for
+  // whoever reads the states later.  The bf16 h in the caller's operand row is what a later prefetch
+  // reads (not needed if the caller sits in the next wavefront: it got the push): it goes out right
+  // after the pushes, before the CTA's per-wavefront barrier, so that the "copies are out" signal can
+  // follow that barrier at once.  The rest (h and c at the node id; c in the caller's row unless the
+  // caller is one or two wavefronts up and got it in shared memory) waits until the next wavefront's
+  // MMAs run.
+  auto copy_operand_rows = [&]() {
+#pragma unroll
+    for (int it = 0; it < kMaxItems; ++it) {
+      const int q = tid + it * kEpiThreads;
+      if (q >= kept) break;
+      const int unit = U0 + q % U, slot = keep_slot[it];
+      if (slot >= 0 && !((keep_near >> (2 * it)) & 1u))
+        p.ain[(size_t)slot * Hp + unit] = __float2bfloat16_rn(unit < H ? keep_h[it] : 0.f);
+    }
+    asm volatile("fence.proxy.async.global;" ::: "memory");    // the operand rows are read through TMA later
+  };
+  auto copy_states = [&]() {
+#pragma unroll
+    for (int it = 0; it < kMaxItems; ++it) {
+      const int q = tid + it * kEpiThreads;
+      if (q >= kept) break;
+      const int unit = U0 + q % U;
+      if (unit >= H) continue;
+      const int node = keep_node[it], slot = keep_slot[it];
+      const float hn = keep_h[it], cn = keep_c[it];
+      p.h[(size_t)node * H + unit] = hn;
+      p.c[(size_t)node * H + unit] = cn;
+      count_write(p.chk_counts, node, 1);
+      if (slot >= 0) {
+        if (!((keep_near >> (2 * it)) & 3u)) p.cin[(size_t)slot * H + unit] = cn;
+        count_write(p.chk_counts ? p.chk_counts + p.n : nullptr, slot >> 1, 1);   // handed over, in shared or global memory
+        count_write(p.chk_counts ? p.chk_counts + 2 * p.n : nullptr, slot >> 1, 1);
+      }
+    }
+  };
+
   bool alive = true;
+  uint32_t e1_phase = 0;                                        // parity of the epilogue's meeting point
   for (int i = 0; i < n_lv; ++i) {
     const int cur = i & 1, nxt = cur ^ 1;
     const uint32_t use = (uint32_t)(i >> 1) & 1u;                 // parity of this use of buffer `cur`
@@ -288,12 +356,12 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
     const int rows = end - begin;
     const int n_pad = (rows + 15) & ~15;                          // UMMA N
     const bool more = i + 1 < n_lv;
-    const int nbeg = end, nend = more ? loff(i + 2) : end;
-    // S0: the tables of this wavefront are in shared memory, the previous wavefront is finished in this
-    // CTA.  The MMA warp does not take part: its operands and its accumulator have barriers of their own,
-    // and it must not wait for the copies to global memory the epilogue still makes for the wavefront before.
-    // The other warps decide together (an OR over the barrier) whether to go on, so that none of them
-    // is left waiting at this barrier by one that saw the flag a moment later.
+    const int nbeg = end, nend = more ? loff(i + 2) : end;        // rows of the next wavefront
+    const int nend2 = i + 2 < n_lv ? loff(i + 3) : nend;          // and of the one after: [nend, nend2)
+    // S0: the tables of this wavefront are in shared memory, the previous wavefront has left this CTA's
+    // shared memory.  The MMA warp does not take part: its operands and its accumulator have barriers of
+    // their own.  The other warps decide together (an OR over the barrier) whether to go on, so that none
+    // of them is left waiting at this barrier by one that saw the flag a moment later.
     if (warp != 9) {
       uint32_t stop_all;
       asm volatile(
@@ -309,18 +377,14 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
 #ifdef TREELSTM_TRACE
     if (tid == 0) TL_STAMP(trace, first_level + i, 0);
 #endif
-    if (warp == 0) {
-      // the global stores of the previous wavefront (all epilogue threads, ordered before by S0) are out:
-      // tell every CTA of the cluster
-      if (lane < (int)cs) mbar_arrive_remote_release(map_to_cta(Gb, (uint32_t)lane));
-    }
 
     if (warp == 8) {
       // ---------------- prefetch of the next wavefront's operand rows, peer signalling ----------------
       if (more) {
         bool ok = true;
         if (lane == 0) {
-          ok = mbar_wait_cluster(Gb, (uint32_t)i & 1u, s_abort, p.wait_limit, p.st);   // stores of wavefront i - 1 visible
+          // the copies every CTA made of wavefront i - 1 are visible (those of older wavefronts were before)
+          ok = mbar_wait_cluster(Gb, (uint32_t)i & 1u, s_abort, p.wait_limit, p.st);
           if (ok) {
             asm volatile("fence.proxy.async;" ::: "memory");   // global rows written, shared buffer last touched, by ordinary stores
             mbar_arrive_expect_tx(XFb(nxt), (uint32_t)(s_cnt[cur * 2] + s_cnt[cur * 2 + 1]) * (uint32_t)(gpc * 16) * cs);
@@ -336,8 +400,9 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
           }
         }
         ok = __shfl_sync(kFullMask, (int)ok, 0) != 0;
-        // the prefetch is in: peers may now overwrite the halves their wavefront produces
-        if (ok && lane < (int)cs) mbar_arrive_remote_release(map_to_cta(Pb(nxt), (uint32_t)lane));
+        // the prefetch is in (lane 0 has seen its barrier flip): peers may now overwrite the halves their
+        // wavefront produces
+        if (ok && lane < (int)cs) mbar_arrive_remote_relaxed(map_to_cta(Pb(nxt), (uint32_t)lane));
       }
     } else if (warp == 9) {
       // ---------------- MMA issuer ----------------
@@ -368,20 +433,53 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
         }
       }
     } else if (warp >= 10) {
-      // ---------------- tables and child cell states of the next wavefront ----------------
+      // ---------------- tables and older child cell states of the next wavefront ----------------
       if (more) {
         fetch_rows(i + 1, nxt);
 #ifdef TREELSTM_TRACE
         if (tid == 320) TL_STAMP(trace, first_level + i, 12);
 #endif
-        fetch_cells(i + 1, nxt);   // what this CTA wrote of them before S0 (or the grid-wide kernel wrote) is there
+        fetch_cells(i + 1, nxt);
 #ifdef TREELSTM_TRACE
         if (tid == 320) TL_STAMP(trace, first_level + i, 13);
 #endif
       }
-      mbar_arrive(CBb);   // the epilogue may now put this wavefront's cell states on top
+      mbar_arrive(CBb(i + 1));                      // (two barriers in turn: the epilogue may still have to look at this wavefront's)
     } else {
       // ---------------- epilogue ----------------
+      // (a) the operand rows of the previous wavefront went to global memory before S0: every CTA of the
+      //     cluster is told (warp 7 has nothing to do with the gate rows); then the rest of that
+      //     wavefront's copies, while this wavefront's MMAs run
+      if (warp == 7 && lane < (int)cs) mbar_arrive_remote_release(map_to_cta(Gb, (uint32_t)lane));
+      if (alive && kept > 0) copy_states();
+#ifdef TREELSTM_TRACE
+      if (tid == 0) TL_STAMP(trace, first_level + i, 14);
+#endif
+      // (b) this thread's (node, unit) pairs of the wavefront: where their gates, child cell states and
+      //     results live
+      const int* s_node = s_rows + (cur * 3 + 0) * kTailRows;
+      const int* s_slot = s_rows + (cur * 3 + 1) * kTailRows;
+      const int n_items = rows * U;
+      int it_g[kMaxItems], it_c[kMaxItems], dep1[kMaxItems], dep2[kMaxItems];
+      unsigned near_now = 0;
+#pragma unroll
+      for (int it = 0; it < kMaxItems; ++it) {
+        const int q = tid + it * kEpiThreads;
+        it_g[it] = -1; dep1[it] = -1; dep2[it] = -1; it_c[it] = 0;
+        if (q < n_items) {
+          const int r = q / U, u = q - r * U;
+          it_g[it] = r * m_rows + (u >> 3) * kGColsI + (u & 7);
+          it_c[it] = r * 2 * U + u;
+          const int slot = s_slot[r];
+          keep_node[it] = s_node[r];
+          keep_slot[it] = slot;
+          if (slot >= 0) {
+            const int pos = slot >> 1, off = (slot & 1) * U + u;
+            if (pos >= nbeg && pos < nend) { dep1[it] = (pos - nbeg) * 2 * U + off; near_now |= 1u << (2 * it); }          // caller in the next wavefront
+            else if (pos >= nend && pos < nend2) { dep2[it] = (pos - nend) * 2 * U + off; near_now |= 2u << (2 * it); }    // caller in the one after
+          }
+        }
+      }
       const int e = warp >> 2, quad = warp & 3;
       const int m = quad * 32 + lane;                              // gate row of this thread
       const int half_cols = n_pad >> 1;                            // columns per half: 8, 16, 24 or 32
@@ -392,13 +490,14 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
       const float a_in = is_tanh ? 1.f : 0.5f, a_mul = is_tanh ? 1.f : 0.5f, a_add = is_tanh ? 0.f : 0.5f;
       if (!mbar_wait(TFb, (uint32_t)i & 1u, s_abort, p.wait_limit, p.st)) alive = false;
       alive = __all_sync(kFullMask, alive);
+      kept = 0;
       if (alive) {
         tc_fence_after();
 #ifdef TREELSTM_TRACE
         if (tid == 0) TL_STAMP(trace, first_level + i, 4);
 #endif
-        // gate values of this row for the nodes of this half -> shared memory, node-major (the operand
-        // buffer of this wavefront is free: its MMAs have retired)
+        // (c) gate values of this row for the nodes of this half -> shared memory, node-major (the operand
+        //     buffer of this wavefront is free: its MMAs have retired)
         float* gsm = reinterpret_cast<float*>(base_ptr + L.xop + (size_t)cur * L.xop_bytes);
         __nv_bfloat16* hs = reinterpret_cast<__nv_bfloat16*>(base_ptr + L.xop + (size_t)cur * L.xop_bytes + L.gate_bytes);
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)col0;
@@ -421,55 +520,61 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
         tc_fence_before();
         mbar_arrive(TEb);                                          // the accumulator may be overwritten
         mbar_arrive(E1b);                                          // every gate row is in shared memory
-        bool ok = mbar_wait(E1b, 0, s_abort, p.wait_limit, p.st);
+        bool ok = mbar_wait(E1b, e1_phase, s_abort, p.wait_limit, p.st);
+        e1_phase ^= 1u;
 #ifdef TREELSTM_TRACE
         if (tid == 0) TL_STAMP(trace, first_level + i, 8);
 #endif
-        ok = mbar_wait(CBb, (uint32_t)i & 1u, s_abort, p.wait_limit, p.st) && ok;   // fetched cell states of the next wavefront are in
+        ok = mbar_wait(CBb(i), use, s_abort, p.wait_limit, p.st) && ok;   // this wavefront's older cell states are in
 #ifdef TREELSTM_TRACE
         if (tid == 0) TL_STAMP(trace, first_level + i, 9);
 #endif
-        // (node, unit) pairs: five gates from shared memory, child cell states, new c and h.  What the
-        // next wavefront needs (bf16 h for the pushes, c of callers in the next wavefront) goes to shared
-        // memory at once; the copies to global memory wait until the pushes are out.
-        const int* s_node = s_rows + (cur * 2 + 0) * kTailRows;
-        const int* s_slot = s_rows + (cur * 2 + 1) * kTailRows;
+        // (d) five gates from shared memory, child cell states, new c and h.  What the next wavefront needs
+        //     goes to shared memory at once: bf16 h for the pushes, c into the caller's row.
         const float* ccur = cbuf + (size_t)cur * kTailRows * 2 * U;
         float* cnext = cbuf + (size_t)nxt * kTailRows * 2 * U;
-        constexpr int kMaxItems = kTailRows * 24 / kEpiThreads;    // (node, unit) pairs per thread at most (U <= 24)
-        float keep_h[kMaxItems], keep_c[kMaxItems], keep_g[kMaxItems][5];
-        const int n_items = rows * U;
+        float* cafter = cbuf + (size_t)cur * kTailRows * 2 * U;    // the buffer of the wavefront after next, once this one has been read
+        if (ok) {
 #pragma unroll
-        for (int it = 0; it < kMaxItems; ++it) {
-          const int q = tid + it * kEpiThreads;
-          if (!ok || q >= n_items) break;
-          const int r = q / U, u = q - r * U, g = u >> 3, u8 = u & 7;
-          const float* gr = gsm + (size_t)r * m_rows + g * kGColsI + u8;
-          const float gi = gr[0], gfl = gr[8], gfr = gr[16], go = gr[24], gu = gr[32];
-          const float cl = ccur[(r * 2 + 0) * U + u], cr = ccur[(r * 2 + 1) * U + u];
-          const float cn = gi * gu + gfl * cl + gfr * cr;
-          const float hn = go * act_tanh(cn);
-          const bool real = U0 + u < H;
-          keep_h[it] = hn; keep_c[it] = cn;
-          if (p.gates) { keep_g[it][0] = gi; keep_g[it][1] = gfl; keep_g[it][2] = gfr; keep_g[it][3] = go; keep_g[it][4] = gu; }
-          hs[r * U + u] = __float2bfloat16_rn(real ? hn : 0.f);
-          const int slot = s_slot[r];
-          if (slot >= 0) {
-            const int pos = slot >> 1;
-            if (pos >= nbeg && pos < nend) cnext[((pos - nbeg) * 2 + (slot & 1)) * U + u] = real ? cn : 0.f;
+          for (int it = 0; it < kMaxItems; ++it) {
+            if (it_g[it] < 0) break;
+            const int q = tid + it * kEpiThreads;
+            const float* gr = gsm + it_g[it];
+            const float gi = gr[0], gfl = gr[8], gfr = gr[16], go = gr[24], gu = gr[32];
+            const float cl = ccur[it_c[it]], cr = ccur[it_c[it] + U];
+            const float cn = gi * gu + gfl * cl + gfr * cr;
+            const float hn = go * act_tanh(cn);
+            const bool real = U0 + (q % U) < H;
+            keep_h[it] = hn; keep_c[it] = cn;
+            hs[q] = __float2bfloat16_rn(real ? hn : 0.f);
+            if (dep1[it] >= 0) cnext[dep1[it]] = real ? cn : 0.f;
+            if (p.gates && real) {
+              float* gp = p.gates + (size_t)keep_node[it] * 5 * H + U0 + (q % U);
+              gp[0] = gi; gp[H] = gfl; gp[2 * H] = gfr; gp[3 * H] = go; gp[4 * H] = gu;
+            }
           }
+          kept = n_items;
+          keep_near = near_now;
         }
 #ifdef TREELSTM_TRACE
         if (tid == 0) TL_STAMP(trace, first_level + i, 5);
 #endif
-        mbar_arrive(E1b);                                          // hs is complete
-        ok = mbar_wait(E1b, 1, s_abort, p.wait_limit, p.st) && ok;
+        mbar_arrive(E1b);                                          // hs is complete, cbuf[cur] has been read
+        ok = mbar_wait(E1b, e1_phase, s_abort, p.wait_limit, p.st) && ok;
+        e1_phase ^= 1u;
         if (!ok) alive = false;
 #ifdef TREELSTM_TRACE
         if (tid == 0) TL_STAMP(trace, first_level + i, 10);
 #endif
+        if (ok) {
+#pragma unroll
+          for (int it = 0; it < kMaxItems; ++it) {
+            if (it_g[it] < 0) break;
+            if (dep2[it] >= 0) cafter[dep2[it]] = U0 + ((tid + it * kEpiThreads) % U) < H ? keep_c[it] : 0.f;
+          }
+        }
         if (more) {
-          // push: 16-byte pieces (8 units) of the new h into the caller's row of every CTA's next buffer
+          // (e) push: 16-byte pieces (8 units) of the new h into the caller's row of every CTA's next buffer
           ok = mbar_wait_cluster(Pb(nxt), use_nxt, s_abort, p.wait_limit, p.st) && ok;
           ok = __all_sync(kFullMask, ok);
 #ifdef TREELSTM_TRACE
@@ -501,41 +606,12 @@ k_fwd_tc_tail(const __grid_constant__ TmapSet maps, const __grid_constant__ SfTm
           if (tid == 0) TL_STAMP(trace, first_level + i, 6);
 #endif
         }
-        // copies to global memory: h and c of every node at its id, bf16 h and fp32 c into the operand
-        // row of its caller (for callers further up than the next wavefront, and for whoever reads the
-        // states later)
-#pragma unroll
-        for (int it = 0; it < kMaxItems; ++it) {
-          const int q = tid + it * kEpiThreads;
-          if (!alive || q >= n_items) break;
-          const int r = q / U, u = q - r * U;
-          const int node = s_node[r], slot = s_slot[r];
-          const int unit = U0 + u;
-          const bool real = unit < H;
-          const float hn = keep_h[it], cn = keep_c[it];
-          if (real) {
-            p.h[(size_t)node * H + unit] = hn;
-            p.c[(size_t)node * H + unit] = cn;
-            count_write(p.chk_counts, node, 1);
-            if (p.gates) {
-              float* gp = p.gates + (size_t)node * 5 * H + unit;
-              gp[0] = keep_g[it][0]; gp[H] = keep_g[it][1]; gp[2 * H] = keep_g[it][2]; gp[3 * H] = keep_g[it][3];
-              gp[4 * H] = keep_g[it][4];
-            }
-          }
-          if (slot >= 0) {
-            p.ain[(size_t)slot * Hp + unit] = __float2bfloat16_rn(real ? hn : 0.f);
-            if (real) {
-              p.cin[(size_t)slot * H + unit] = cn;
-              count_write(p.chk_counts ? p.chk_counts + p.n : nullptr, slot >> 1, 1);
-              count_write(p.chk_counts ? p.chk_counts + 2 * p.n : nullptr, slot >> 1, 1);
-            }
-          }
-        }
-        asm volatile("fence.proxy.async.global;" ::: "memory");    // the operand rows are read through TMA later
+        if (alive && kept > 0) copy_operand_rows();
       }
     }
   }
+  // the last wavefront's copies
+  if (warp < 8 && alive && kept > 0 && !*s_abort) copy_states();
 
   // teardown
   tc_fence_before();
@@ -598,6 +674,7 @@ int launch_forward_bf16_tail(treelstm* ctx, int n, const int32_t* left, const in
   p.gates = (flags & TREELSTM_SAVE_FOR_BACKWARD) ? reinterpret_cast<float*>(base + lay.gates) : nullptr;
   p.st = reinterpret_cast<DevStatus*>(base + lay.status);
   p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
+  p.level = ctx->last.level;
   p.n_parts = 0;
   p.groups_per_cta = ctx->sf.groups_per_cta;
   p.tail_width = ctx->opt.tail_width;

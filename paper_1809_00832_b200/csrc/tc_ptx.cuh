@@ -41,23 +41,38 @@ struct TcParams {
 };
 
 // Where the grid-wide kernel stops and one cluster takes over (persistent mode): the first wavefront
-// - never the leaves - from which on every wavefront has at most tail_width nodes, provided at least
-// tail_min_levels wavefronts remain (a hand-over costs a launch and the cluster's set-up); n_levels if
-// there is no such tail or tail_width is 0.  Both kernels call this with the same arguments and take
-// the same decision.  Cooperative over the CTA: every thread calls it; s_tmp is one shared int.
+// - never the leaves - from which on every wavefront has at most tail_width nodes, if handing those
+// over pays.  With tail_min_levels > 0 it pays when at least that many wavefronts remain.  With
+// tail_min_levels == 0 a cost model fitted to cycle traces decides: a wavefront of w nodes takes the
+// grid-wide kernel about 9.5 k cycles whatever w, the cluster about 5.3 k + 75 w (it passes states
+// through shared memory, at a price per node: every CTA of the cluster gets a copy), and the hand-over
+// itself - a launch and the cluster's set-up - about 24 k; the tail goes to the cluster if the
+// wavefronts it takes save more than that.  Returns n_levels if there is no such tail or tail_width
+// is 0.  Both kernels call this with the same arguments and take the same decision.  Cooperative over
+// the CTA: every thread calls it; s_tmp is two shared ints.
+constexpr int kTailGainBase = 4200, kTailGainPerRow = 75, kTailHandOver = 24000;
 __device__ __forceinline__ int tail_first_level(const int* level_offset, int n_levels, int tail_width,
                                                 int tail_min_levels, int* s_tmp) {
-  if (threadIdx.x == 0) *s_tmp = 1;        // the leaf wavefront always stays with the grid-wide kernel
+  if (threadIdx.x == 0) { s_tmp[0] = 1; s_tmp[1] = 0; }   // the leaf wavefront always stays with the grid-wide kernel
   __syncthreads();
   int wide_end = 0;                        // 1 + the last wavefront wider than tail_width
   for (int l = threadIdx.x; l < n_levels; l += blockDim.x)
     if (level_offset[l + 1] - level_offset[l] > tail_width) wide_end = l + 1;
-  if (wide_end > 1) atomicMax(s_tmp, wide_end);
+  if (wide_end > 1) atomicMax(&s_tmp[0], wide_end);
   __syncthreads();
-  const int first = *s_tmp;
+  const int first = s_tmp[0];
+  if (tail_width > 0 && tail_min_levels <= 0) {
+    int gain = 0;                          // cycles the cluster saves on the wavefronts from `first` on
+    for (int l = first + threadIdx.x; l < n_levels; l += blockDim.x)
+      gain += kTailGainBase - kTailGainPerRow * (level_offset[l + 1] - level_offset[l]);
+    if (gain != 0) atomicAdd(&s_tmp[1], gain);
+  }
+  __syncthreads();
+  const int gain_all = s_tmp[1];
   __syncthreads();                         // s_tmp may be reused by the caller
-  if (tail_width <= 0 || n_levels - first < (tail_min_levels > 1 ? tail_min_levels : 1)) return n_levels;
-  return first;
+  if (tail_width <= 0 || first >= n_levels) return n_levels;
+  if (tail_min_levels > 0) return n_levels - first >= tail_min_levels ? first : n_levels;
+  return gain_all > kTailHandOver ? first : n_levels;
 }
 
 // ---- PTX wrappers ---------------------------------------------------------------------------- //

@@ -4,12 +4,26 @@
                                           [--tail-width N] [--tail-min-levels M] [--trees T] [--levels A:B]
 
 The trace build (-DTREELSTM_TRACE, libtreelstm_b200_trace.so) makes the first CTA of each kernel write
-clock64 stamps for the first 256 wavefronts: the grid-wide kernel at the start of a wavefront (0),
-when its tiles are done (6) and after the grid barrier (7); the cluster kernel at the start of a
-wavefront (0), when its first operand request is out (1), when the MMA issuer sees the first box (2),
-when the last MMAs are committed (3), when the epilogue starts waiting (4), when it has stored its
-last tile (5), when the CTA arrives at the cluster barrier (6) and when it leaves it (7).  The stamps
-cost a few cycles each; the timings of the normal build are a little lower.
+clock64 stamps for the first 256 wavefronts; the table prints them in cycles since the wavefront's
+first stamp (s0), 0 where a stamp was not taken.
+
+Grid-wide kernel (k_fwd_tc): s0 start of the wavefront, s6 its tiles are done in this CTA, s7 the grid
+barrier has opened.
+
+Cluster kernel of the narrow tail (k_fwd_tc_tail), stamps of different warps of one CTA:
+  s0  the CTA's per-wavefront barrier has opened (all warps but the MMA issuer)
+  s14 epilogue: copies of the previous wavefront to global memory are out
+  s12 / s13 fetching warps: tables of the next wavefront read / its older child cell states read
+  s1 / s7 producer: prefetch of the next wavefront's operand rows requested / landed
+  s2 / s3 MMA issuer: operands complete (prefetch and pushes) / last MMA committed
+  s4  epilogue: accumulator complete      s8  gate values in shared memory
+  s9  older child cell states are in      s5  cell updates done
+  s10 new h complete in shared memory     s11 every peer's prefetch has landed (pushes may go)
+  s6  pushes issued
+The sub-forest kernel (--mode subforests) uses s0 start, s1 first operand request, s2 first box seen by
+the MMA issuer, s3 last MMAs committed, s4 epilogue starts waiting, s5 last tile stored, s6 arrival at
+the cluster barrier, s7 barrier left.  The stamps cost a few cycles each; the normal build is a little
+faster.
 """
 from __future__ import annotations
 

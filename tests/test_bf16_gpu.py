@@ -274,15 +274,18 @@ def test_bf16_deeper_than_the_level_cache():
 
 
 def test_narrow_tails_are_handed_to_one_cluster():
-    """the library's own choice in persistent mode: once every remaining wavefront has at most 64 nodes
-    (and at least four remain) the grid-wide kernel stops and one cluster finishes the forest, passing
-    states from child to caller through distributed shared memory.  Where the hand-over happens is
-    decided on the device; it changes no bit of the result (every node's contraction runs over the
-    same products in the same order), whatever the shape of the tail."""
+    """persistent mode: the last wavefronts of a forest, once they are all narrow, can be finished by one
+    cluster that passes states from child to caller through distributed shared memory.  Whether that
+    pays is decided on the device by a cost model (or forced with TAIL_MIN_LEVELS); either way it changes
+    no bit of the result (every node's contraction runs over the same products in the same order),
+    whatever the shape of the tail."""
     rng = np.random.default_rng(77)
     for H, E in ((256, 300), (150, 64), (128, 40), (64, 64)):
         params = fg.draw_params(rng, H, E, 500, emb_dist="normal", emb_scale=0.3, w_scale=0.08)
         model = util.make_model(params, "bf16")
+        forced = util.make_model(params, "bf16")
+        forced.set_option(binding.OPT_TAIL_WIDTH, 64)
+        forced.set_option(binding.OPT_TAIL_MIN_LEVELS, 2)      # hand over whenever two narrow wavefronts remain
         plain = util.make_model(params, "bf16")
         plain.set_option(binding.OPT_TAIL_WIDTH, 0)            # every wavefront on the grid-wide kernel
         cases = [
@@ -292,29 +295,38 @@ def test_narrow_tails_are_handed_to_one_cluster():
             [fg.balanced_shape(64)],                                                 # both children always one wavefront below
             [fg.random_split_shape(rng, 40) for _ in range(30)] + [fg.left_chain_shape(50)] * 3,   # wide first, long narrow tail
             [fg.left_chain_shape(70)] * 64,                                          # exactly 64 nodes per wavefront
+            [fg.random_split_shape(rng, 30) for _ in range(5)] + [fg.left_chain_shape(45)],   # callers one, two and more wavefronts up
         ]
         for shapes in cases:
             forest = fg.forest_from_shapes(shapes, rng, 500)
             forest, _ = fg.permute_node_ids(forest, rng)
             ref = util.gpu_forward(plain, forest, binding.PERSISTENT)
             assert plain.last_launch_count() == 2
-            res = util.gpu_forward(model, forest, binding.PERSISTENT)
-            widths = np.diff(ref["level_offset"][:ref["n_levels"] + 1])
-            narrow_tail = int(np.argmax(np.append(widths[::-1] > 64, True)))        # wavefronts at the end with <= 64 nodes
-            narrow_tail = min(narrow_tail, len(widths) - 1)                          # the leaves never count
-            assert model.last_launch_count() == 3 and model.last_mode() == binding.PERSISTENT
-            assert narrow_tail >= 4                                                  # every case has a tail to hand over
-            np.testing.assert_array_equal(res["order"], ref["order"])
-            np.testing.assert_array_equal(res["h"], ref["h"])
-            np.testing.assert_array_equal(res["c"], ref["c"])
+            for m in (forced, model):
+                res = util.gpu_forward(m, forest, binding.PERSISTENT)
+                assert m.last_launch_count() == (3 if forest.n_nodes <= 4096 else 2) and m.last_mode() == binding.PERSISTENT
+                np.testing.assert_array_equal(res["order"], ref["order"])
+                np.testing.assert_array_equal(res["h"], ref["h"])
+                np.testing.assert_array_equal(res["c"], ref["c"])
             h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
                                             operand_round=orc.round_to_bf16)
             assert util.max_abs(res["h"], h) < TIGHT and util.max_abs(res["c"], c) < TIGHT
+        # a forest above the node limit only reaches the cluster kernel when the limit is raised
+        forced.set_option(binding.OPT_TAIL_MAX_NODES, 1 << 20)
+        wide = fg.forest_from_shapes(cases[5], rng, 500)            # 64 chains: 64 nodes in every wavefront above the leaves
+        ref = util.gpu_forward(plain, wide, binding.PERSISTENT)
+        res = util.gpu_forward(forced, wide, binding.PERSISTENT)
+        assert forced.last_launch_count() == 3
+        np.testing.assert_array_equal(res["h"], ref["h"])
+        np.testing.assert_array_equal(res["c"], ref["c"])
+        model = forced
+        forest = fg.forest_from_shapes(cases[4], rng, 500)
+        ref = util.gpu_forward(plain, forest, binding.PERSISTENT)
         # a forest without a narrow tail long enough stays on the grid-wide kernel (the cluster finds nothing to do)
         model.set_option(binding.OPT_TAIL_MIN_LEVELS, 1000)
         res = util.gpu_forward(model, forest, binding.PERSISTENT)
         np.testing.assert_array_equal(res["h"], ref["h"])
-        model.set_option(binding.OPT_TAIL_MIN_LEVELS, 4)
+        model.set_option(binding.OPT_TAIL_MIN_LEVELS, 2)
         # saved gates for backward come out of the cluster kernel too
         small = fg.forest_from_shapes([fg.random_split_shape(rng, 30)], rng, 500)
         arrs = [util.to_dev(x) for x in (small.left, small.right, small.token)]
