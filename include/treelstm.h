@@ -90,7 +90,7 @@ typedef enum treelstm_status {
                                             /* forward with CUDA events (treelstm_last_kernel_ms)    */
 #define TREELSTM_OPT_TAIL_WIDTH 5           /* TREELSTM_PERSISTENT, bf16, H padded to <= 256: the last    */
                                             /* wavefronts of a forest, once every remaining one has at    */
-                                            /* most this many nodes (default 48, largest value 64), may   */
+                                            /* most this many nodes (default 32, largest value 64), may   */
                                             /* be finished by ONE thread-block cluster (a second launch): */
                                             /* recurrent weights resident in shared memory, states passed  */
                                             /* from child to caller through distributed shared memory.     */

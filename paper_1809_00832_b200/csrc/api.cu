@@ -551,7 +551,15 @@ int treelstm_selftest_waits(treelstm_t* ctx, void* workspace, size_t workspace_b
 // Trace builds only (not part of the public header): copies the cycle stamps of the last forward to
 // the host, kTraceSlots per wavefront; which = 0 grid-wide kernel, 1 cluster kernel.  Synchronises.
 TREELSTM_API int treelstm_trace_read(treelstm_t* ctx, int which, long long* out, int max_entries) {
-  if (!ctx || !out || which < 0 || which > 1 || !ctx->last.ws) return TREELSTM_ERR_INVALID_ARG;
+  if (!ctx || !out || which < 0 || which > 2 || !ctx->last.ws) return TREELSTM_ERR_INVALID_ARG;
+  if (which == 2) {   // the scheduler's phase stamps: the unused words of the control block
+    DevStatus hs;
+    TL_CUDA(ctx, cudaStreamSynchronize(ctx->last.stream));
+    TL_CUDA(ctx, cudaMemcpy(&hs, static_cast<const char*>(ctx->last.ws) + ctx->last.lay.status, sizeof(hs), cudaMemcpyDeviceToHost));
+    int cnt = 0;
+    for (; cnt < 16 && cnt < max_entries; ++cnt) out[cnt] = hs.pad[cnt];
+    return cnt;
+  }
   const int total = kTraceSlots * kTraceLevels;
   const int cnt = max_entries < total ? max_entries : total;
   const char* src = static_cast<const char*>(ctx->last.ws) + ctx->last.lay.trace + (size_t)which * total * sizeof(long long);

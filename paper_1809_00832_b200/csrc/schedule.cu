@@ -17,6 +17,9 @@ namespace {
 
 constexpr int kSingleThreads = 1024;
 constexpr int kSingleWarps = kSingleThreads / 32;
+// the dependency words share their shared memory with what comes after them: the radix histogram
+// (256 x 32 ints) or the per-thread level counts of the few-levels placement (32 x 1024 uint16)
+constexpr size_t kSingleScratch = 65536;
 constexpr unsigned kFull = 0xffffffffu;
 
 __device__ __forceinline__ unsigned lanemask_lt() {
@@ -166,6 +169,128 @@ __device__ int block_compact(int n, int* dst, FlagFn flag, int* scan_tmp, PlaceF
   return total;
 }
 
+// Ready order, wavefront boundaries and roots in one go for forests of at most 32 wavefronts (the
+// usual case: depth grows with the logarithm of the sentence length).  One CTA of 1024 threads;
+// thread t owns the contiguous ids [t * npt, (t + 1) * npt).  tab[L][t] (uint16, 32 x 1024 = 64 KB of
+// shared memory) first counts the thread's nodes of level L, then warp L turns row L into its
+// exclusive prefix over the threads, and finally thread t hands out positions level_start[L] +
+// tab[L][t]++ to its nodes in ascending id - ascending (level, id) overall, with no key matching at
+// all.  The positions are scattered into a shared-memory copy of the order (uint16 ids, `staged`) and
+// go out to global memory as whole lines afterwards: one SM cannot afford 4-byte stores to n
+// different sectors.  Output as the general path: order[], level_offset[0 .. n_levels), roots[] by
+// ascending id; returns the number of roots to every thread.  scan_tmp: shared int[32].
+__device__ int place_few_levels(int n, int n_levels, const unsigned short* lv16, int* order, int* level_offset,
+                                int* roots, unsigned short* tab, unsigned short* staged, int* scan_tmp,
+                                int* stamps) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+#ifdef TREELSTM_TRACE
+  const long long t_in = clock64();
+#define TL_PLACE_STAMP(i) do { if (tid == 0 && stamps) stamps[i] = (int)(clock64() - t_in); } while (0)
+#else
+  (void)stamps;
+#define TL_PLACE_STAMP(i) do { } while (0)
+#endif
+  __shared__ int s_level_start[32];
+  __shared__ int s_root_total;
+  const int npt = ((n + kSingleThreads - 1) / kSingleThreads) | 1;   // odd: the threads' ranges start in different banks
+  const int k0 = min(n, tid * npt), k1 = min(n, k0 + npt);
+  {
+    uint4* z = reinterpret_cast<uint4*>(tab);                   // 64 KB = 4096 pieces of 16 bytes
+    for (int i = tid; i < 32 * kSingleThreads * 2 / 16; i += kSingleThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  __syncthreads();
+  TL_PLACE_STAMP(0);
+  int my_roots = 0;
+  for (int k = k0; k < k1; ++k) {
+    const unsigned short v = lv16[k];
+    tab[(v & 0x7FFF) * kSingleThreads + tid] += 1;
+    my_roots += v >> 15;
+  }
+  __syncthreads();
+  TL_PLACE_STAMP(1);
+  // row L -> exclusive prefix over the threads (warp L; lane j takes the 32 threads 32 j .. 32 j + 31)
+  if (warp < n_levels) {
+    unsigned short* row = tab + warp * kSingleThreads + lane * 32;
+    unsigned short v[32];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint4 x = reinterpret_cast<const uint4*>(row)[q];
+      const unsigned int w4[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { v[q * 8 + 2 * j] = (unsigned short)(w4[j] & 0xFFFFu); v[q * 8 + 2 * j + 1] = (unsigned short)(w4[j] >> 16); }
+    }
+    int sum = 0;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) { const int c = v[j]; v[j] = (unsigned short)sum; sum += c; }
+    int incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int t = __shfl_up_sync(kFull, incl, d);
+      if (lane >= d) incl += t;
+    }
+    const int base = incl - sum;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      unsigned int w4[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        w4[j] = (unsigned int)(unsigned short)(v[q * 8 + 2 * j] + base) | ((unsigned int)(unsigned short)(v[q * 8 + 2 * j + 1] + base) << 16);
+      reinterpret_cast<uint4*>(row)[q] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+    }
+    if (lane == 31) scan_tmp[warp] = incl;                      // nodes of level `warp`
+  }
+  __syncthreads();
+  TL_PLACE_STAMP(2);
+  // level starts (warp 0) and the roots' prefix over the threads (all warps, one value per thread)
+  if (warp == 0) {
+    const int c = lane < n_levels ? scan_tmp[lane] : 0;
+    int incl = c;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int t = __shfl_up_sync(kFull, incl, d);
+      if (lane >= d) incl += t;
+    }
+    s_level_start[lane] = incl - c;
+    if (lane < n_levels) level_offset[lane] = incl - c;
+  }
+  __syncthreads();
+  int rincl = my_roots;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int t = __shfl_up_sync(kFull, rincl, d);
+    if (lane >= d) rincl += t;
+  }
+  if (lane == 31) scan_tmp[warp] = rincl;
+  __syncthreads();
+  if (warp == 0) {
+    const int c = scan_tmp[lane];
+    int incl = c;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int t = __shfl_up_sync(kFull, incl, d);
+      if (lane >= d) incl += t;
+    }
+    scan_tmp[lane] = incl - c;
+    if (lane == 31) s_root_total = incl;
+  }
+  __syncthreads();
+  TL_PLACE_STAMP(3);
+  int rpos = scan_tmp[warp] + rincl - my_roots;
+  for (int k = k0; k < k1; ++k) {
+    const unsigned short v = lv16[k];
+    const int lv = v & 0x7FFF;
+    unsigned short* cell = tab + lv * kSingleThreads + tid;
+    const int pos = s_level_start[lv] + *cell;
+    *cell += 1;
+    staged[pos] = (unsigned short)k;
+    if (v >> 15) roots[rpos++] = k;
+  }
+  __syncthreads();
+  TL_PLACE_STAMP(4);
+  for (int i = tid; i < n; i += kSingleThreads) order[i] = staged[i];
+  return s_root_total;
+}
+
 // One CTA schedules the whole forest in shared memory (forests up to 32768 nodes).
 //
 // Dependency counters, as in Section 4.1.1: every internal node waits for two inputs.  A finished
@@ -173,7 +298,7 @@ __device__ int block_compact(int n, int* dst, FlagFn flag, int* scan_tmp, PlaceF
 // and stops, the one that finds its sibling's entry knows both inputs are resolved, gives the caller
 // level 1 + max and goes on upwards.  No global atomics, no grid-wide rounds.
 //
-// Dynamic shared memory: uint32 w[n] (dependency words; later the radix histogram, at least 32 KB),
+// Dynamic shared memory: uint32 w[n] (dependency words; later the sort's scratch, at least 64 KB),
 // uint16 par[n] (caller of each node, the return location of Section 4.1.2; later level | root
 // flag), uint16 queue[n / 2] (start nodes of the climb), and with n_parts > 0 uint16 lab[n].
 //
@@ -186,10 +311,9 @@ __global__ void __launch_bounds__(kSingleThreads, 1)
 k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ right,
                   const int* __restrict__ token, int vocab, int* parent, int* level, int* order,
                   int* order_tmp, int* level_offset, int* roots, int* n_levels_out, DevStatus* st,
-                  int n_parts, int* part_order, int* part_offset, int* slot) {
+                  int n_parts, int* part_order, int* part_offset, int* slot, int cache_children) {
   extern __shared__ __align__(16) unsigned char smem[];
-  const size_t w_bytes = (size_t)n * 4 > sizeof(int) * kRadixBins * kSingleWarps
-                             ? (((size_t)n * 4 + 15) & ~(size_t)15) : sizeof(int) * kRadixBins * kSingleWarps;
+  const size_t w_bytes = (size_t)n * 4 > kSingleScratch ? (((size_t)n * 4 + 15) & ~(size_t)15) : kSingleScratch;
   unsigned int* w = reinterpret_cast<unsigned int*>(smem);
   int* hist = reinterpret_cast<int*>(smem);
   unsigned short* par = reinterpret_cast<unsigned short*>(smem + w_bytes);
@@ -197,15 +321,26 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
   unsigned short* queue = par + (((size_t)n + 7) & ~(size_t)7);   // start nodes of the climb, at most n / 2
   unsigned short* lab = reinterpret_cast<unsigned short*>(
       smem + w_bytes + ((((size_t)n * 2) + 15) & ~(size_t)15) + (((size_t)n + 15) & ~(size_t)15));
+  // where shared memory allows (no sub-forest labels, forest small enough): both children of every node,
+  // packed, so that the second look at them does not go back to global memory
+  unsigned int* lr = cache_children ? reinterpret_cast<unsigned int*>(lab) : nullptr;
   __shared__ int scan_tmp[32];
   __shared__ int s_err, s_maxlevel, s_qhead, s_qtail;
   const int tid = threadIdx.x;
   constexpr unsigned short kNoParent = 0xFFFF;
   constexpr unsigned int kDone = 0x80000000u;
   if (tid < (int)(sizeof(DevStatus) / sizeof(int))) reinterpret_cast<int*>(st)[tid] = 0;
+#ifdef TREELSTM_TRACE
+  // phase stamps of thread 0 (cycles since the start) in the unused words of the control block
+  const long long t_start = clock64();
+#define TL_SCHED_STAMP(i) do { if (tid == 0) st->pad[i] = (int)(clock64() - t_start); } while (0)
+#else
+#define TL_SCHED_STAMP(i) do { } while (0)
+#endif
   if (tid == 0) { s_err = 0; s_maxlevel = 0; s_qhead = 0; s_qtail = 0; }
   for (int k = tid; k < n; k += kSingleThreads) { w[k] = 0; par[k] = kNoParent; }
   __syncthreads();
+  TL_SCHED_STAMP(0);   // cleared
   // validate; children record their caller; leaves are complete at once (level 0)
   // Node j of this thread is tid + j * 1024 (at most 32 per thread); leaf_bits remembers which are
   // leaves so that later passes need not look at the child arrays again.
@@ -233,11 +368,13 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
       } else {
         par[l[j]] = (unsigned short)k;
         par[r[j]] = (unsigned short)k;
+        if (lr) lr[k] = (unsigned int)l[j] | ((unsigned int)r[j] << 16);
       }
       if (err) atomicMin(&s_err, err);
     }
   }
   __syncthreads();
+  TL_SCHED_STAMP(1);   // validated and linked
   if (s_err == 0) {
     // a child claimed by two callers kept only one of them: checked at the caller
     for (int j0 = 0; j0 * kSingleThreads + tid < n; j0 += 8) {
@@ -246,8 +383,14 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
       for (int j = 0; j < 8; ++j) {
         const int k = tid + (j0 + j) * kSingleThreads;
         const bool internal = k < n && !((leaf_bits >> (j0 + j)) & 1u);
-        l[j] = internal ? left[k] : -1;
-        r[j] = internal ? right[k] : -1;
+        if (lr) {
+          const unsigned int both = internal ? lr[k] : 0xFFFFFFFFu;
+          l[j] = internal ? (int)(both & 0xFFFFu) : -1;
+          r[j] = internal ? (int)(both >> 16) : -1;
+        } else {
+          l[j] = internal ? left[k] : -1;
+          r[j] = internal ? right[k] : -1;
+        }
       }
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -269,6 +412,7 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
     }
   }
   __syncthreads();
+  TL_SCHED_STAMP(2);   // links checked, leaves reported
   if (s_err == 0) {
     // Climb: threads take start nodes from the queue until it is empty.
     for (;;) {
@@ -287,6 +431,7 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
     }
   }
   __syncthreads();
+  TL_SCHED_STAMP(3);   // climbed
   int local_max = 0;
   if (s_err == 0) {
     for (int k = tid; k < n; k += kSingleThreads) {
@@ -310,6 +455,19 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
     return;
   }
   const int n_levels = n > 0 ? s_maxlevel + 1 : 0;
+  TL_SCHED_STAMP(4);   // levels written
+  if (n_levels <= 32 && lr != nullptr) {
+    // (the packed children are no longer needed: their shared memory takes the staged order)
+    const int n_roots = place_few_levels(n, n_levels, lv16, order, level_offset, roots,
+                                         reinterpret_cast<unsigned short*>(smem), reinterpret_cast<unsigned short*>(lr),
+                                         scan_tmp, st->pad + 8);
+    if (tid == 0) {
+      level_offset[n_levels] = n; st->n_levels = n_levels; *n_levels_out = n_levels;
+      st->n_roots = n_roots;
+    }
+    TL_SCHED_STAMP(5);   // ordered
+    return;
+  }
   // canonical ready order: LSD radix on the level, 8 bits per pass, ties by node id
   int passes = 1;
   while (passes < 4 && (n_levels - 1) >> (8 * passes)) ++passes;
@@ -551,10 +709,13 @@ __global__ void k_gather_roots(int max_roots, int H, const int* roots, const flo
 
 size_t single_smem_bytes(int n, bool with_parts) {
   size_t w = (size_t)n * 4;
-  const size_t hist = sizeof(int) * kRadixBins * kSingleWarps;
-  w = w > hist ? round_up_sz(w, 16) : hist;
+  w = w > kSingleScratch ? round_up_sz(w, 16) : kSingleScratch;
   return w + round_up_sz((size_t)n * 2, 16) + round_up_sz((size_t)n, 16) +
          (with_parts ? round_up_sz((size_t)n * 2, 16) : 0);
+}
+// The packed children of every node next to the rest, if that still fits one CTA's shared memory.
+bool single_caches_children(int n, bool with_parts) {
+  return !with_parts && single_smem_bytes(n, false) + (size_t)n * 4 + 16 <= single_smem_bytes(kSchedSingleMaxNodes, false);
 }
 
 int init_schedule_attributes(treelstm* ctx) {
@@ -579,10 +740,11 @@ int launch_schedule(treelstm* ctx, int n, const int32_t* left, const int32_t* ri
   if (n > 0 && n <= single_max) {
     // the kernel clears the control block itself and writes the level count to the caller
     const bool parts = n_parts > 0 && n <= kSchedPartMaxNodes;
-    k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n, parts), stream>>>(
+    const bool cache = single_caches_children(n, parts);
+    k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n, parts) + (cache ? (size_t)n * 4 + 16 : 0), stream>>>(
         n, left, right, token, ctx->vocab, parent, level, order, order_tmp, level_offset, roots, n_levels_out,
         st, parts ? n_parts : 0, reinterpret_cast<int*>(base + lay.part_order),
-        reinterpret_cast<int*>(base + lay.part_offset), reinterpret_cast<int*>(base + lay.slot));
+        reinterpret_cast<int*>(base + lay.part_offset), reinterpret_cast<int*>(base + lay.slot), cache ? 1 : 0);
     ctx->launches += 1;
     TL_CUDA(ctx, cudaGetLastError());
     return TREELSTM_OK;
@@ -728,9 +890,10 @@ extern "C" int treelstm_schedule_static(int n_nodes, const int32_t* left, const 
   if (n_nodes > 0) {
     // the control block keeps the previous call's status and counts; the kernel's first step is
     // to clear it, everything else in the array is rewritten before it is read
-    k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n_nodes, false), s>>>(
+    const bool cache = single_caches_children(n_nodes, false);
+    k_schedule_single<<<1, kSingleThreads, single_smem_bytes(n_nodes, false) + (cache ? (size_t)n_nodes * 4 + 16 : 0), s>>>(
         n_nodes, left, right, token, vocab, parent, level, order, order_tmp, level_offset, roots, n_levels, st,
-        0, nullptr, nullptr, nullptr);
+        0, nullptr, nullptr, nullptr, cache ? 1 : 0);
     if (cudaGetLastError() != cudaSuccess) return TREELSTM_ERR_CUDA;
   } else {
     if (cudaMemsetAsync(st, 0, sizeof(DevStatus), s) != cudaSuccess ||

@@ -43,14 +43,14 @@ struct TcParams {
 // Where the grid-wide kernel stops and one cluster takes over (persistent mode): the first wavefront
 // - never the leaves - from which on every wavefront has at most tail_width nodes, if handing those
 // over pays.  With tail_min_levels > 0 it pays when at least that many wavefronts remain.  With
-// tail_min_levels == 0 a cost model fitted to cycle traces decides: a wavefront of w nodes takes the
-// grid-wide kernel about 9.5 k cycles whatever w, the cluster about 5.3 k + 75 w (it passes states
-// through shared memory, at a price per node: every CTA of the cluster gets a copy), and the hand-over
-// itself - a launch and the cluster's set-up - about 24 k; the tail goes to the cluster if the
-// wavefronts it takes save more than that.  Returns n_levels if there is no such tail or tail_width
+// tail_min_levels == 0 a cost model fitted to cycle traces and step times decides: a wavefront of w
+// nodes takes the grid-wide kernel about 9.5 k cycles whatever w, the cluster about 5.5 k + 100 w (it
+// passes states through shared memory, at a price per node: every CTA of the cluster gets a copy), and
+// the hand-over itself - a launch, the cluster's set-up and its first wavefront waiting for the
+// weights - about 30 k; the tail goes to the cluster if the wavefronts it takes save more than that.  Returns n_levels if there is no such tail or tail_width
 // is 0.  Both kernels call this with the same arguments and take the same decision.  Cooperative over
 // the CTA: every thread calls it; s_tmp is two shared ints.
-constexpr int kTailGainBase = 4200, kTailGainPerRow = 75, kTailHandOver = 24000;
+constexpr int kTailGainBase = 4000, kTailGainPerRow = 100, kTailHandOver = 30000;
 __device__ __forceinline__ int tail_first_level(const int* level_offset, int n_levels, int tail_width,
                                                 int tail_min_levels, int* s_tmp) {
   if (threadIdx.x == 0) { s_tmp[0] = 1; s_tmp[1] = 0; }   // the leaf wavefront always stays with the grid-wide kernel

@@ -83,6 +83,16 @@ def main() -> int:
     if args.levels:
         a, b = args.levels.split(":")
         lo, hi = int(a or 0), int(b or hi)
+    buf = (ctypes.c_longlong * 16)()
+    fn = model.lib.treelstm_trace_read
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int]
+    if fn(model.handle, 2, ctypes.cast(buf, ctypes.c_void_p), 16) > 0:
+        names = ("cleared", "validated+linked", "links checked, leaves reported", "climbed", "levels written", "ordered")
+        print("# single-CTA scheduler, thread 0, cycles since its start: " +
+              ", ".join(f"{nm} {int(buf[i])}" for i, nm in enumerate(names)))
+        print("#   inside the few-levels placement (cycles since its start): counts cleared, counted, rows scanned, "
+              "starts known, placed = " + ", ".join(str(int(buf[8 + i])) for i in range(5)))
     for which, name in ((0, "grid-wide kernel"), (1, "cluster kernel")):
         t = read_trace(model, which)
         rows = [l for l in range(min(len(widths), LEVELS)) if t[l, 0] != 0]
