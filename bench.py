@@ -403,7 +403,7 @@ def run_reference(args):
     if rank != 0:
         return 0
     from oracle import treelstm_oracle as orc
-    w = fg.make_workload(args.workload, 0)
+    w = fg.make_workload(args.workload, 0, args.trees)
     p = w.params
     steps, warmup = args.steps, args.warmup
     # bound the sample so that steps + warmup oracle passes finish in a couple of minutes
@@ -453,6 +453,7 @@ def main() -> int:
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="batch256_bf16", choices=fg.WORKLOADS)
+    ap.add_argument("--trees", type=int, default=None, help="number of trees of the workload (default: its own batch size)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="persistent", choices=MODES)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -479,7 +480,7 @@ def main() -> int:
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the TreeLSTM library has no CPU path")
 
-    w = fg.make_workload(args.workload, seed=rank)
+    w = fg.make_workload(args.workload, seed=rank, n_trees=args.trees)
     f, p = w.forest, w.params
     cpu_one = cpu_many = None
     if world == 1 and not args.no_cpu_baseline:

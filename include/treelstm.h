@@ -105,7 +105,14 @@ typedef enum treelstm_status {
                                             /* remain                                                      */
 #define TREELSTM_OPT_TAIL_MAX_NODES 7       /* forests with more nodes than this (default 4096) never      */
                                             /* launch the cluster kernel: the host knows the node count    */
-                                            /* only, and a large forest has nothing to gain                */
+                                            /* only, and a large forest has nothing to gain.  The second   */
+                                            /* launch costs a few microseconds even when the cluster finds */
+                                            /* nothing to do, so the library also leaves it out while the  */
+                                            /* control block of the last forward it read back              */
+                                            /* (treelstm_status_sync, treelstm_forward_host) said that the */
+                                            /* forest had no tail worth handing over; the grid-wide kernel */
+                                            /* keeps recording what the decision would have been, and the  */
+                                            /* launch comes back with the first forest that has one        */
 
 /*
  * treelstm_create - build a context for one set of parameters.

@@ -145,6 +145,15 @@ int read_levels(treelstm* ctx) {
 
 }  // namespace
 
+// What a control block that has just been read back says about the hand-over to the cluster kernel.
+void learn_tail_hint(treelstm* ctx) {
+  const DevStatus* hs = reinterpret_cast<const DevStatus*>(ctx->host_status);
+  const auto& L = ctx->last;
+  if (!ctx->tail_ok || ctx->precision != TREELSTM_BF16 || L.mode != TREELSTM_PERSISTENT || hs->status != 0 || hs->n_levels <= 0)
+    return;
+  ctx->tail_skip = hs->tail_from >= hs->n_levels;
+}
+
 // used by backward.cu
 int ensure_host_levels(treelstm* ctx) {
   if (ctx->last.host_levels_valid) return TREELSTM_OK;
@@ -282,9 +291,11 @@ int treelstm_set_option(treelstm_t* ctx, int key, long long value) {
       return TREELSTM_OK;
     case TREELSTM_OPT_TAIL_WIDTH:
       ctx->opt.tail_width = value > 64 ? 64 : (int)value;
+      ctx->tail_skip = false;
       return TREELSTM_OK;
     case TREELSTM_OPT_TAIL_MIN_LEVELS:
       ctx->opt.tail_min_levels = value > (1 << 20) ? (1 << 20) : (int)value;
+      ctx->tail_skip = false;
       return TREELSTM_OK;
     case TREELSTM_OPT_TAIL_MAX_NODES:
       ctx->opt.tail_max_nodes = value > (1 << 30) ? (1 << 30) : (int)value;
@@ -396,6 +407,7 @@ int treelstm_status_sync(treelstm_t* ctx) {
   TL_CUDA(ctx, cudaStreamSynchronize(L.stream));
   const int st = reinterpret_cast<const DevStatus*>(ctx->host_status)->status;
   if (st != 0) L.valid = false;
+  else learn_tail_hint(ctx);
   return st;
 }
 

@@ -20,7 +20,8 @@ struct DevStatus {
   unsigned int barrier;  // arrival counter of the persistent kernels' grid barrier
   int n_touched;         // distinct leaf tokens (backward)
   unsigned int barrier_bwd;  // arrival counter of the one-launch backward pass (cleared by its launch)
-  int pad[57];
+  int tail_from;         // persistent bf16 forward: first wavefront the cluster kernel takes (or would take), n_levels if none
+  int pad[56];
 };
 static_assert(sizeof(DevStatus) == 256, "control block is one 256-byte line group");
 
@@ -121,6 +122,7 @@ struct treelstm {
   bool have_tmaps = false;
   tl::SubforestPlan sf;                 // filled at create (bf16 only)
   bool tail_ok = false;                 // the tail kernel exists for this context's sizes
+  bool tail_skip = false;               // the last forward whose control block was read back had no tail worth a hand-over
 
   tl::Options opt;
 

@@ -177,7 +177,11 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   // next on the same stream), which keeps the recurrent weights in shared memory and meets at the
   // hardware cluster barrier instead of the grid-wide one.
   __shared__ int s_stop[2];
-  const int lvl_stop = only_level < 0 ? tail_first_level(p.level_offset, n_levels, p.tail_width, p.tail_min_levels, s_stop) : n_levels;
+  // (Without the cluster kernel on the stream the decision is still worked out and left in the control
+  // block: the host learns from it whether launching that kernel is worth its while for forests like this.)
+  const int tail_from = only_level < 0 ? tail_first_level(p.level_offset, n_levels, p.tail_width, p.tail_min_levels, s_stop) : n_levels;
+  const int lvl_stop = p.tail_launched ? tail_from : n_levels;
+  if (only_level < 0 && blockIdx.x == 0 && tid == 0) p.st->tail_from = tail_from;
 #ifdef TREELSTM_TRACE
   long long* const trace = blockIdx.x == 0 && tid == 0 ? p.trace : nullptr;
 #endif
@@ -647,10 +651,14 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   // The narrow wavefronts at the end of a forest go to one cluster (tail_tc.cu) where that kernel
   // exists for these sizes; where the hand-over happens is decided on the device from the level table.
   // (the host only knows the node count: forests too large for a narrow tail to matter skip the second launch)
-  const bool with_tail = (flags & TREELSTM_PERSISTENT) && ctx->tail_ok && ctx->opt.tail_width > 0 &&
-                         ctx->opt.max_ctas == 0 && n <= ctx->opt.tail_max_nodes && n >= 8;
-  p.tail_width = with_tail ? ctx->opt.tail_width : 0;
+  const bool tail_possible = (flags & TREELSTM_PERSISTENT) && ctx->tail_ok && ctx->opt.tail_width > 0 &&
+                             ctx->opt.max_ctas == 0 && n <= ctx->opt.tail_max_nodes && n >= 8;
+  // the second launch costs a few microseconds even when the cluster finds nothing to do: it is left out
+  // while the control block of the last forward that was read back says that there was no such tail
+  const bool with_tail = tail_possible && !(ctx->tail_skip && ctx->opt.tail_min_levels == 0);
+  p.tail_width = tail_possible ? ctx->opt.tail_width : 0;
   p.tail_min_levels = ctx->opt.tail_min_levels;
+  p.tail_launched = with_tail ? 1 : 0;
   p.trace = nullptr;
   p.knob = ctx->opt.knob;
 #ifdef TREELSTM_TRACE

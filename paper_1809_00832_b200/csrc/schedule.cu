@@ -171,8 +171,8 @@ __device__ int block_compact(int n, int* dst, FlagFn flag, int* scan_tmp, PlaceF
 
 // Ready order, wavefront boundaries and roots in one go for forests of at most 32 wavefronts (the
 // usual case: depth grows with the logarithm of the sentence length).  One CTA of 1024 threads;
-// thread t owns the contiguous ids [t * npt, (t + 1) * npt).  tab[L][t] (uint16, 32 x 1024 = 64 KB of
-// shared memory) first counts the thread's nodes of level L, then warp L turns row L into its
+// thread t owns the contiguous ids [t * npt, (t + 1) * npt).  tab[L][t] (uint16, n_levels x 1024: 2 KB of
+// shared memory per wavefront) first counts the thread's nodes of level L, then warp L turns row L into its
 // exclusive prefix over the threads, and finally thread t hands out positions level_start[L] +
 // tab[L][t]++ to its nodes in ascending id - ascending (level, id) overall, with no key matching at
 // all.  The positions are scattered into a shared-memory copy of the order (uint16 ids, `staged`) and
@@ -195,8 +195,8 @@ __device__ int place_few_levels(int n, int n_levels, const unsigned short* lv16,
   const int npt = ((n + kSingleThreads - 1) / kSingleThreads) | 1;   // odd: the threads' ranges start in different banks
   const int k0 = min(n, tid * npt), k1 = min(n, k0 + npt);
   {
-    uint4* z = reinterpret_cast<uint4*>(tab);                   // 64 KB = 4096 pieces of 16 bytes
-    for (int i = tid; i < 32 * kSingleThreads * 2 / 16; i += kSingleThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    uint4* z = reinterpret_cast<uint4*>(tab);                   // 2 KB = 128 pieces of 16 bytes per wavefront
+    for (int i = tid; i < n_levels * kSingleThreads * 2 / 16; i += kSingleThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   __syncthreads();
   TL_PLACE_STAMP(0);
@@ -456,11 +456,15 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
   }
   const int n_levels = n > 0 ? s_maxlevel + 1 : 0;
   TL_SCHED_STAMP(4);   // levels written
-  if (n_levels <= 32 && lr != nullptr) {
-    // (the packed children are no longer needed: their shared memory takes the staged order)
+  // The few-levels placement needs 2 KB per wavefront for its counts and 2 n bytes for the staged
+  // order: the packed children's shared memory (no longer needed) takes the latter, or what the
+  // dependency words leave free behind the counts.
+  const size_t tab_bytes = (size_t)n_levels * kSingleThreads * 2;
+  unsigned short* staged = lr != nullptr ? reinterpret_cast<unsigned short*>(lr)
+                           : (tab_bytes + (size_t)n * 2 <= w_bytes ? reinterpret_cast<unsigned short*>(smem + tab_bytes) : nullptr);
+  if (n_levels <= 32 && n_parts == 0 && staged != nullptr) {
     const int n_roots = place_few_levels(n, n_levels, lv16, order, level_offset, roots,
-                                         reinterpret_cast<unsigned short*>(smem), reinterpret_cast<unsigned short*>(lr),
-                                         scan_tmp, st->pad + 8);
+                                         reinterpret_cast<unsigned short*>(smem), staged, scan_tmp, st->pad + 8);
     if (tid == 0) {
       level_offset[n_levels] = n; st->n_levels = n_levels; *n_levels_out = n_levels;
       st->n_roots = n_roots;

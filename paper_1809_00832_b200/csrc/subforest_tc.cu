@@ -451,6 +451,7 @@ int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, con
   p.level_offset = nullptr;
   p.tail_width = 0;
   p.tail_min_levels = 0;
+  p.tail_launched = 0;
   p.trace = nullptr;
   p.knob = ctx->opt.knob;
 #ifdef TREELSTM_TRACE

@@ -679,6 +679,7 @@ int launch_forward_bf16_tail(treelstm* ctx, int n, const int32_t* left, const in
   p.groups_per_cta = ctx->sf.groups_per_cta;
   p.tail_width = ctx->opt.tail_width;
   p.tail_min_levels = ctx->opt.tail_min_levels;
+  p.tail_launched = 1;
   p.knob = ctx->opt.knob;
   p.trace = nullptr;
 #ifdef TREELSTM_TRACE

@@ -36,6 +36,7 @@ struct TcParams {
   int n_parts, groups_per_cta;   // n_parts == 0: the cluster kernel runs as the tail of the grid-wide kernel
   // hand-over from the grid-wide kernel to one cluster (persistent mode): see tail_first_level
   int tail_width, tail_min_levels;
+  int tail_launched;             // the cluster kernel follows on the stream (else the decision is only recorded)
   int knob;                      // development switches (0 in normal use)
   long long* trace;              // cycle stamps (trace builds), else nullptr
 };

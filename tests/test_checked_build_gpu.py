@@ -50,6 +50,8 @@ def test_checked_cluster_paths_chains_training_and_other_cells():
     # the narrow tail of a small forest and of a mixed one goes to the cluster kernel
     params = fg.draw_params(rng, 256, 300, 500, emb_dist="normal", emb_scale=0.3, w_scale=0.08)
     model = util.make_model(params, "bf16", variant=CHECKED)
+    model.set_option(binding.OPT_TAIL_WIDTH, 64)
+    model.set_option(binding.OPT_TAIL_MIN_LEVELS, 2)          # hand over whenever two narrow wavefronts remain
     small = fg.forest_from_shapes([fg.random_split_shape(rng, 40), None, fg.left_chain_shape(9)], rng, 500)
     util.gpu_forward(model, small, binding.PERSISTENT)
     assert model.status_sync() == binding.OK and model.last_launch_count() == 3
