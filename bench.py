@@ -361,6 +361,8 @@ def run_sweeps(args):
                                      v_scale=1.0 / (2 * H))
         model = binding.TreeLSTM.recursive(binding.CELL_RNTN if tensor else binding.CELL_TREERNN, H, p.vocab,
                                            _dev(p.emb), _dev(p.W), _dev(p.b), _dev(p.V) if tensor else None)
+    if args.tail_width is not None and args.cell == "treelstm":
+        model.set_option(binding.OPT_TAIL_WIDTH, args.tail_width)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
 
     flags = {"persistent": binding.PERSISTENT, "per_level": binding.PER_LEVEL, "subforests": binding.SUBFORESTS}[args.mode]
@@ -386,13 +388,13 @@ def run_sweeps(args):
             for batch in (1, 10, 25):
                 forest = fg.forest_from_shapes([make() for _ in range(batch)], rng, p.vocab)
                 ms, levels = time_forest(forest)
-                print(json.dumps({"sweep": "shape", "cell": args.cell, "mode": args.mode, "shape": name, "leaves_per_tree": 32, "batch": batch,
+                print(json.dumps({"sweep": "shape", "cell": args.cell, "mode": args.mode, "tail_width": args.tail_width, "shape": name, "leaves_per_tree": 32, "batch": batch,
                                   "levels": levels, "ms_per_step": ms, "trees_per_sec": batch / (ms * 1e-3)}))
     if args.sweep in ("length", "all"):
         for leaves in (2, 4, 8, 16, 24, 32, 40, 48, 56):
             forest = fg.forest_from_shapes([fg.random_split_shape(rng, leaves)], rng, p.vocab)
             ms, levels = time_forest(forest)
-            print(json.dumps({"sweep": "length", "cell": args.cell, "mode": args.mode, "leaves": leaves, "batch": 1, "levels": levels,
+            print(json.dumps({"sweep": "length", "cell": args.cell, "mode": args.mode, "tail_width": args.tail_width, "leaves": leaves, "batch": 1, "levels": levels,
                               "ms_per_instance": ms}))
     return 0
 
@@ -461,6 +463,8 @@ def main() -> int:
     ap.add_argument("--no-extra", action="store_true", help="skip the extra workloads and the latency-floor probe")
     ap.add_argument("--cell", default="treelstm", choices=["treelstm", "treernn", "rntn"],
                     help="cell of the sweeps (the benchmark line itself is always TreeLSTM)")
+    ap.add_argument("--tail-width", type=int, default=None,
+                    help="sweeps only: widest wavefront handed to the one-cluster kernel (0 = never hand over)")
     ap.add_argument("--sweep", default=None, choices=["shapes", "length", "all"],
                     help="print the tree-shape / sentence-length sweeps instead of the benchmark line")
     args = ap.parse_args()

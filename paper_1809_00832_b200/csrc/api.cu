@@ -286,9 +286,6 @@ int treelstm_set_option(treelstm_t* ctx, int key, long long value) {
     case TREELSTM_OPT_MAX_CTAS:
       ctx->opt.max_ctas = value > 65535 ? 65535 : (int)value;
       return TREELSTM_OK;
-    case 100:
-      ctx->opt.knob = (int)value;
-      return TREELSTM_OK;
     case TREELSTM_OPT_TAIL_WIDTH:
       ctx->opt.tail_width = value > 64 ? 64 : (int)value;
       ctx->tail_skip = false;

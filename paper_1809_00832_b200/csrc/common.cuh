@@ -49,7 +49,6 @@ struct Options {
   long long wait_limit_kcycles = 1 << 20;  // ~1e9 cycles, about half a second at 2 GHz
   int max_ctas = 0;
   int time_kernel = 0;
-  int knob = 0;           // development switches of the tensor-core kernels (0 in normal use)
   int tail_width = 32;    // persistent bf16 forward: trailing wavefronts this narrow may run on one cluster (0: never)
   int tail_min_levels = 0; // > 0: hand them over if at least this many remain; 0: the device decides by its cost model
   int tail_max_nodes = 4096;   // forests with more nodes never launch the cluster kernel

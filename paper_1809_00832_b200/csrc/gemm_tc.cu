@@ -660,7 +660,6 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.tail_min_levels = ctx->opt.tail_min_levels;
   p.tail_launched = with_tail ? 1 : 0;
   p.trace = nullptr;
-  p.knob = ctx->opt.knob;
 #ifdef TREELSTM_TRACE
   p.trace = reinterpret_cast<long long*>(base + lay.trace);
   TL_CUDA(ctx, cudaMemsetAsync(p.trace, 0, sizeof(long long) * kTraceSlots * kTraceLevels, stream));

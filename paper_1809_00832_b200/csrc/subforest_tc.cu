@@ -203,7 +203,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
     // A stage of the ring holds one box: kbox K blocks of operand rows (+ kbox K blocks of W_x rows).
     // A single-tile wavefront takes its operands in one request when they fit, anything else in
     // boxes of two K blocks so that loads, MMAs and epilogues of consecutive tiles overlap.
-    c.sel = c.tiles == 1 && !(p.knob & 1) && (uint32_t)kblocks * (c.a_bytes + c.w_bytes) <= L.ring_bytes ? 0 : 1;
+    c.sel = c.tiles == 1 && (uint32_t)kblocks * (c.a_bytes + c.w_bytes) <= L.ring_bytes ? 0 : 1;
     c.kbox = c.sel == 0 ? kblocks : 2;
     c.n_box = c.sel == 0 ? 1 : (kblocks + 1) >> 1;
     c.stage_bytes = (uint32_t)c.kbox * (c.a_bytes + c.w_bytes);
@@ -328,7 +328,7 @@ k_fwd_tc_subforest(const __grid_constant__ TmapSet maps, const __grid_constant__
           EpiTile et;
           et.leaf = leaf; et.G = G; et.gcols = gcols; et.ncols = ncols; et.nt = nt;
           et.row = row; et.node = node; et.slot = slot; et.valid = valid;
-          et.allow_staged_out = rows > 64 || (p.knob & 2);   // a narrow tile writes so little that it stores straight from registers
+          et.allow_staged_out = rows > 64;   // a narrow tile writes so little that it stores straight from registers
           et.r = r; et.e = e; et.quad = quad;
           et.cstage_addr = cstage_addr; et.cstage_ptr = cstage_ptr; et.crow_shift = L.crow_shift;
           et.half = 4 << (L.crow_shift - 7);
@@ -453,7 +453,6 @@ int launch_forward_bf16_subforest(treelstm* ctx, int n, const int32_t* left, con
   p.tail_min_levels = 0;
   p.tail_launched = 0;
   p.trace = nullptr;
-  p.knob = ctx->opt.knob;
 #ifdef TREELSTM_TRACE
   p.trace = reinterpret_cast<long long*>(base + lay.trace) + kTraceSlots * kTraceLevels;
   TL_CUDA(ctx, cudaMemsetAsync(p.trace, 0, sizeof(long long) * kTraceSlots * kTraceLevels, stream));

@@ -680,7 +680,6 @@ int launch_forward_bf16_tail(treelstm* ctx, int n, const int32_t* left, const in
   p.tail_width = ctx->opt.tail_width;
   p.tail_min_levels = ctx->opt.tail_min_levels;
   p.tail_launched = 1;
-  p.knob = ctx->opt.knob;
   p.trace = nullptr;
 #ifdef TREELSTM_TRACE
   p.trace = reinterpret_cast<long long*>(base + lay.trace) + kTraceSlots * kTraceLevels;

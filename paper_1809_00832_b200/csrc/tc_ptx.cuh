@@ -37,7 +37,6 @@ struct TcParams {
   // hand-over from the grid-wide kernel to one cluster (persistent mode): see tail_first_level
   int tail_width, tail_min_levels;
   int tail_launched;             // the cluster kernel follows on the stream (else the decision is only recorded)
-  int knob;                      // development switches (0 in normal use)
   long long* trace;              // cycle stamps (trace builds), else nullptr
 };
 

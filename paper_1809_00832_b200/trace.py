@@ -57,7 +57,6 @@ def main() -> int:
     ap.add_argument("--tail-min-levels", type=int, default=None)
     ap.add_argument("--trees", type=int, default=None)
     ap.add_argument("--levels", default=None, help="A:B - print only wavefronts A..B-1")
-    ap.add_argument("--knob", type=int, default=0, help="development switches of the kernels")
     args = ap.parse_args()
     build.build(variant="trace")
     w = fg.make_workload(args.workload, 0, args.trees)
@@ -68,8 +67,6 @@ def main() -> int:
         model.set_option(binding.OPT_TAIL_WIDTH, args.tail_width)
     if args.tail_min_levels is not None:
         model.set_option(binding.OPT_TAIL_MIN_LEVELS, args.tail_min_levels)
-    if args.knob:
-        model.set_option(100, args.knob)
     flags = binding.PERSISTENT if args.mode == "persistent" else binding.SUBFORESTS
     left, right, token = dev(f.left), dev(f.right), dev(f.token)
     out = model.forward(left, right, token, flags=flags)
