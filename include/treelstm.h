@@ -113,6 +113,17 @@ typedef enum treelstm_status {
                                             /* forest had no tail worth handing over; the grid-wide kernel */
                                             /* keeps recording what the decision would have been, and the  */
                                             /* launch comes back with the first forest that has one        */
+#define TREELSTM_OPT_OVERLAP_LAUNCH 8       /* 1 (default): the persistent bf16 wavefront kernel is        */
+                                            /* launched as a programmatic dependent of the ready-set       */
+                                            /* construction, so that its set-up (barriers, tensor memory,  */
+                                            /* weights and biases asked into L2) runs while that kernel    */
+                                            /* still works; it waits on the device for the schedule.  Such */
+                                            /* a launch cannot be a cooperative one: that every CTA is     */
+                                            /* resident then rests on the grid fitting the device (the     */
+                                            /* library checks) and on the stream having the device to      */
+                                            /* itself; otherwise the bounded grid barrier ends the call    */
+                                            /* with TREELSTM_ERR_TIMEOUT.  0: cooperative launch in plain  */
+                                            /* stream order (residency guaranteed by the runtime)          */
 
 /*
  * treelstm_create - build a context for one set of parameters.

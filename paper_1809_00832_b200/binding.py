@@ -40,6 +40,7 @@ OPT_TIME_WAVEFRONT_KERNEL = 4
 OPT_TAIL_WIDTH = 5
 OPT_TAIL_MIN_LEVELS = 6
 OPT_TAIL_MAX_NODES = 7
+OPT_OVERLAP_LAUNCH = 8
 
 _vp = ctypes.c_void_p
 _i = ctypes.c_int

@@ -294,6 +294,9 @@ int treelstm_set_option(treelstm_t* ctx, int key, long long value) {
       ctx->opt.tail_min_levels = value > (1 << 20) ? (1 << 20) : (int)value;
       ctx->tail_skip = false;
       return TREELSTM_OK;
+    case TREELSTM_OPT_OVERLAP_LAUNCH:
+      ctx->opt.overlap_launch = value != 0;
+      return TREELSTM_OK;
     case TREELSTM_OPT_TAIL_MAX_NODES:
       ctx->opt.tail_max_nodes = value > (1 << 30) ? (1 << 30) : (int)value;
       return TREELSTM_OK;

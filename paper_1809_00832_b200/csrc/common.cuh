@@ -52,6 +52,7 @@ struct Options {
   int tail_width = 32;    // persistent bf16 forward: trailing wavefronts this narrow may run on one cluster (0: never)
   int tail_min_levels = 0; // > 0: hand them over if at least this many remain; 0: the device decides by its cost model
   int tail_max_nodes = 4096;   // forests with more nodes never launch the cluster kernel
+  int overlap_launch = 1;      // persistent bf16 forward: the wavefront kernel starts under the scheduler (programmatic dependent launch)
 };
 
 constexpr int kRadixBins = 256;
@@ -121,6 +122,7 @@ struct treelstm {
   bool have_tmaps = false;
   tl::SubforestPlan sf;                 // filled at create (bf16 only)
   bool tail_ok = false;                 // the tail kernel exists for this context's sizes
+  int tc_resident_ctas = 0;             // CTAs of the grid-wide bf16 kernel the device holds at once
   bool tail_skip = false;               // the last forward whose control block was read back had no tail worth a hand-over
 
   tl::Options opt;

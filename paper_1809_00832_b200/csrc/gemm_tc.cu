@@ -171,21 +171,11 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + 2 + a); };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (ld_volatile(&p.st->status) != 0) return;      // schedule failed: nothing to evaluate
-  const int n_levels = p.st->n_levels;
-  // Persistent mode: the narrow wavefronts at the end of the forest are left to one cluster (launched
-  // next on the same stream), which keeps the recurrent weights in shared memory and meets at the
-  // hardware cluster barrier instead of the grid-wide one.
-  __shared__ int s_stop[2];
-  // (Without the cluster kernel on the stream the decision is still worked out and left in the control
-  // block: the host learns from it whether launching that kernel is worth its while for forests like this.)
-  const int tail_from = only_level < 0 ? tail_first_level(p.level_offset, n_levels, p.tail_width, p.tail_min_levels, s_stop) : n_levels;
-  const int lvl_stop = p.tail_launched ? tail_from : n_levels;
-  if (only_level < 0 && blockIdx.x == 0 && tid == 0) p.st->tail_from = tail_from;
-#ifdef TREELSTM_TRACE
-  long long* const trace = blockIdx.x == 0 && tid == 0 ? p.trace : nullptr;
-#endif
-
+  const int Hp = p.Hp, H = p.H;
+  const int groups = Hp / kUnitGroup;
+  // What needs nothing from the kernel before (the ready-set construction): barriers, tensor memory,
+  // and warming L2.  In persistent mode this kernel is launched as a programmatic dependent of the
+  // scheduler and gets here while that one still runs; the wait below ends when it has finished.
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
@@ -196,15 +186,47 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     s_pre = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  for (int i = tid; i < kLevelCache && i <= n_levels; i += kThreads) s_level_offset[i] = p.level_offset[i];
   if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // columns: 2 accumulator stages x 256
+  if (only_level < 0) {
+    // Every CTA reads the packed weights and biases in every wavefront, but they may have left L2 since
+    // the last call: all CTAs ask for a share of them now, and for the tensor maps, so that the first
+    // tiles do not wait for memory.
+    const int gtid = blockIdx.x * kThreads + tid, gthreads = gridDim.x * kThreads;
+    warm_l2(p.wp_x, (size_t)groups * kGColsL * p.Ep * 2, gtid, gthreads);
+    warm_l2(p.wp_h, (size_t)groups * kGColsI * 2 * Hp * 2, gtid, gthreads);
+    warm_l2(p.bp_x, (size_t)groups * kGColsL * 4, gtid, gthreads);
+    warm_l2(p.bp_h, (size_t)groups * kGColsI * 4, gtid, gthreads);
+    if (tid < (int)(sizeof(TmapSet) / sizeof(CUtensorMap))) prefetch_tmap(reinterpret_cast<const CUtensorMap*>(&maps) + tid);
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const bool failed = ld_volatile(&p.st->status) != 0;      // schedule failed: nothing to evaluate
+  const int n_levels = failed ? 0 : p.st->n_levels;
+  // Persistent mode: the narrow wavefronts at the end of the forest are left to one cluster (launched
+  // next on the same stream), which keeps the recurrent weights in shared memory and meets at the
+  // hardware cluster barrier instead of the grid-wide one.
+  __shared__ int s_stop[2];
+  // (Without the cluster kernel on the stream the decision is still worked out and left in the control
+  // block: the host learns from it whether launching that kernel is worth its while for forests like this.)
+  const int tail_from = only_level < 0 ? tail_first_level(p.level_offset, n_levels, p.tail_width, p.tail_min_levels, s_stop) : n_levels;
+  const int lvl_stop = p.tail_launched ? tail_from : n_levels;
+  if (only_level < 0 && !failed && blockIdx.x == 0 && tid == 0) p.st->tail_from = tail_from;
+#ifdef TREELSTM_TRACE
+  long long* const trace = blockIdx.x == 0 && tid == 0 ? p.trace : nullptr;
+  long long* const trace_cta = blockIdx.x == 0 ? p.trace : nullptr;   // stamps of the producers and the MMA issuer
+#define TL_ROLE_STAMP(slot_first, slot_second)                                                        \
+  do {                                                                                                \
+    if (t < 2 * (int)gridDim.x) TL_STAMP(trace_cta, lvl, t < (int)gridDim.x ? (slot_first) : (slot_second)); \
+  } while (0)
+#else
+#define TL_ROLE_STAMP(slot_first, slot_second) do { } while (0)
+#endif
+
+  for (int i = tid; i < kLevelCache && i <= n_levels; i += kThreads) s_level_offset[i] = p.level_offset[i];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
 
-  const int Hp = p.Hp, H = p.H;
-  const int groups = Hp / kUnitGroup;
   const int kb_leaf = p.Ep / kKBlock, kb_int = 2 * Hp / kKBlock;
   const bool vec = (H % 4) == 0;
 
@@ -302,6 +324,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
             }
             mbar_arrive_expect_tx(full_bar(stage), bytes);
             tma_load_3d(tiles_addr + stage * stage_bytes + off, map, 0, y, box * kbox, full_bar(stage));
+            if (box == 0 && is_a) TL_ROLE_STAMP(14, 11);
+            if (box == n_box - 1 && is_a) TL_ROLE_STAMP(15, 12);
             armed |= 1u << stage;
             phase_bits ^= 1u << stage;
             if (++stage == n_stages) stage = 0;
@@ -326,6 +350,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
               break;
             }
             tc_fence_after();
+            if (box == 0) TL_ROLE_STAMP(4, 13);
             const uint32_t st_addr = tiles_addr + stage * stage_bytes;
             const int nkb = min(kbox, kblocks - box * kbox);
             for (int kbi = 0; kbi < nkb; ++kbi) {
@@ -341,6 +366,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
             if (++stage == n_stages) stage = 0;
           }
           if (alive) umma_commit(tfull_bar(acc));      // the accumulator is complete
+          TL_ROLE_STAMP(5, 5);
         }
         ++acc_iter;
       } else if (warp != 11) {
@@ -380,6 +406,10 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
         et.tmem_acc = tmem_base + acc * kAccCols;
         et.tfull = tfull_bar(acc); et.tempty = tempty_bar(acc); et.epi_bar = epi_bar; et.acc_phase = (acc_iter >> 1) & 1;
         et.bias = (leaf ? p.bp_x : p.bp_h) + nt * ncols + 4 * e;
+#ifdef TREELSTM_TRACE
+        // the CTA's first tile of the wavefront stamps slots 1-3, its second one slots 8-10
+        if (trace != nullptr && lvl < kTraceLevels && t < 2 * (int)gridDim.x) et.stamp = trace + lvl * kTraceSlots + (t < (int)gridDim.x ? 1 : 8);
+#endif
         epilogue_tile(p, et, epi_phase, alive, s_abort, [&]() { if (nx_have) nx_slot = valid2 ? chk_slot(p.st, p.slot[nx_node], p.n) : -1; });
         ++acc_iter;
       }
@@ -589,6 +619,9 @@ int ensure_operand_tmaps(treelstm* ctx, void* ws, int n, const void* xin, const 
 
 int init_tc_attributes(treelstm* ctx) {
   TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  int per_sm = 0;
+  TL_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_fwd_tc, kThreads, kSmemBytes));
+  ctx->tc_resident_ctas = per_sm * ctx->sm_count;
   return TREELSTM_OK;
 }
 
@@ -643,6 +676,7 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.ain = reinterpret_cast<__nv_bfloat16*>(base + lay.ain);
   p.cin = reinterpret_cast<float*>(base + lay.cin);
   p.bp_h = ctx->bp_h; p.bp_x = ctx->bp_x;
+  p.wp_h = ctx->Wp_h; p.wp_x = ctx->Wp_x;
   p.h = h; p.c = c;
   p.gates = (flags & TREELSTM_SAVE_FOR_BACKWARD) ? reinterpret_cast<float*>(base + lay.gates) : nullptr;
   p.st = reinterpret_cast<DevStatus*>(base + lay.status);
@@ -676,9 +710,26 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     if (grid > want) grid = want;
     if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
     int only = -1;
-    void* args[] = {&ctx->maps, &p, &only};
-    TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_tc, dim3(grid), dim3(kThreads), args,
-                                             kSmemBytes, stream));
+    // The grid barrier needs every CTA resident.  Two ways to launch:
+    //  * as a programmatic dependent of the kernel before it on the stream - the ready-set construction:
+    //    the CTAs come up and do their set-up while that kernel still runs (it gives the go-ahead at its
+    //    start) and wait for its results at griddepcontrol.wait.  The runtime takes this attribute on a
+    //    plain launch only (measured: together with the cooperative attribute it has no effect), so
+    //    residency rests on the grid being no larger than what the device holds at once (checked
+    //    here) and on the device not being shared with other work; if CTAs cannot come up, the bounded
+    //    barrier ends the kernel with TREELSTM_ERR_TIMEOUT.
+    //  * as a cooperative launch (TREELSTM_OPT_OVERLAP_LAUNCH = 0): the runtime guarantees residency,
+    //    and the kernel starts when the one before it has ended.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    if (ctx->opt.overlap_launch && grid <= ctx->tc_resident_ctas) {
+      attr.id = cudaLaunchAttributeProgrammaticStreamSerialization; attr.val.programmaticStreamSerializationAllowed = 1;
+    } else {
+      attr.id = cudaLaunchAttributeCooperative; attr.val.cooperative = 1;
+    }
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    TL_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_fwd_tc, ctx->maps, p, only));
     ctx->launches += 1;
     if (with_tail)
       return launch_forward_bf16_tail(ctx, n, left, right, token, h, c, order, level_offset_dev, flags, ws, lay, stream);

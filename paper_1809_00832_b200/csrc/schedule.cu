@@ -329,6 +329,9 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
   const int tid = threadIdx.x;
   constexpr unsigned short kNoParent = 0xFFFF;
   constexpr unsigned int kDone = 0x80000000u;
+  // A kernel launched behind this one as its programmatic dependent may start now: the part of it
+  // that comes before its own wait for this grid needs nothing from here.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid < (int)(sizeof(DevStatus) / sizeof(int))) reinterpret_cast<int*>(st)[tid] = 0;
 #ifdef TREELSTM_TRACE
   // phase stamps of thread 0 (cycles since the start) in the unused words of the control block

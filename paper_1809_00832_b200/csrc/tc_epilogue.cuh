@@ -34,7 +34,13 @@ struct EpiTile {
   uint32_t tmem_acc;            // tensor-memory address of the accumulator stage
   uint32_t tfull, tempty, epi_bar, acc_phase;
   const float* bias;            // packed bias of the tile's first column, this thread's half
+  long long* stamp = nullptr;   // trace builds: three cycle stamps of this tile (accumulator ready, cells done, tile left)
 };
+#ifdef TREELSTM_TRACE
+#define TL_TILE_STAMP(t, k) do { if ((t).stamp) (t).stamp[k] = clock64(); } while (0)
+#else
+#define TL_TILE_STAMP(t, k) do { } while (0)
+#endif
 
 // between_fn runs after the cell updates and before the accumulator is handed back (the callers
 // fetch row data of their next tile there).
@@ -71,6 +77,7 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, const EpiTile& 
   alive = __all_sync(kFullMask, alive);
   asm volatile("cp.async.wait_all;" ::: "memory");
   if (!alive) return;
+  TL_TILE_STAMP(t, 0);
   tc_fence_after();
   const uint32_t taddr = t.tmem_acc + ((uint32_t)(t.quad * 32) << 16) + 4u * e;
   // the tensor-memory loads of group g + 1 are in flight while group g is computed
@@ -178,6 +185,7 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, const EpiTile& 
       }
     }
   }
+  TL_TILE_STAMP(t, 1);
   between_fn();
   tc_fence_before();
   mbar_arrive(t.tempty);                       // accumulator stage may be overwritten
@@ -217,6 +225,7 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, const EpiTile& 
     epi_phase ^= 1;
     if (!ok) alive = false;
   }
+  TL_TILE_STAMP(t, 2);
 }
 
 }  // namespace tl

@@ -24,6 +24,7 @@ struct TcParams {
   const int *left, *right, *token, *order, *roots, *level_offset;
   int* slot;
   const __nv_bfloat16* emb_bf;
+  const __nv_bfloat16 *wp_h = nullptr, *wp_x = nullptr;   // packed weights (grid-wide kernel: warmed into L2 at its start)
   __nv_bfloat16 *xin, *ain;
   float* cin;
   const float *bp_h, *bp_x;
@@ -137,6 +138,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+// Ask for the 128-byte lines of [ptr, ptr + bytes) to be brought into L2, spread over n_threads threads.
+__device__ __forceinline__ void warm_l2(const void* ptr, size_t bytes, int thread, int n_threads) {
+  const char* b = static_cast<const char*>(ptr);
+  for (size_t off = (size_t)thread * 128; off < bytes; off += (size_t)n_threads * 128)
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(b + off));
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");

@@ -8,7 +8,11 @@ clock64 stamps for the first 256 wavefronts; the table prints them in cycles sin
 first stamp (s0), 0 where a stamp was not taken.
 
 Grid-wide kernel (k_fwd_tc): s0 start of the wavefront, s6 its tiles are done in this CTA, s7 the grid
-barrier has opened.
+barrier has opened; first epilogue thread, the CTA's first tile of the wavefront: s1 accumulator
+complete, s2 cell updates done, s3 tile left (outputs copied); s8, s9, s10 the same for the CTA's
+second tile; operand producer: s14 / s15 first / last box of the first tile requested, s11 / s12 the
+same for the second tile; MMA issuer: s4 first box of the first tile has landed, s13 first box of the
+second tile has landed, s5 last MMAs of the (second, if any) tile issued.
 
 Cluster kernel of the narrow tail (k_fwd_tc_tail), stamps of different warps of one CTA:
   s0  the CTA's per-wavefront barrier has opened (all warps but the MMA issuer)

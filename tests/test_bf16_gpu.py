@@ -1,6 +1,8 @@
 """Parity of the bf16 tensor-core forward (tcgen05 path, through the C ABI) against the fp64 oracle:
 schedule bit-exact, h and c within 3e-2 max-abs; against the oracle with the same operands rounded
 to bf16 the agreement must be much tighter (separates operand rounding from kernel mistakes)."""
+import dataclasses
+
 import numpy as np
 import pytest
 
@@ -251,6 +253,36 @@ def test_all_modes_give_identical_states():
             np.testing.assert_array_equal(res["c"], ref["c"])
             np.testing.assert_array_equal(res["order"], ref["order"])
         model.close()
+
+
+def test_both_launch_forms_give_identical_states():
+    """the persistent kernel launched as a programmatic dependent of the scheduler (it starts while
+    the scheduler runs and waits for it on the device) and launched cooperatively in plain stream
+    order: same bits, also when a malformed forest makes the scheduler report an error"""
+    rng = np.random.default_rng(49)
+    w = fg.make_workload("batch256_bf16", 0)
+    model = util.make_model(w.params, "bf16")
+    res = {}
+    for form in (1, 0, 1):
+        model.set_option(binding.OPT_OVERLAP_LAUNCH, form)
+        for _ in range(3):                            # back to back: the next scheduler follows the kernel at once
+            out = util.gpu_forward(model, w.forest, binding.PERSISTENT)
+        res.setdefault(form, out)
+        np.testing.assert_array_equal(out["h"], res[form]["h"])
+    np.testing.assert_array_equal(res[0]["h"], res[1]["h"])
+    np.testing.assert_array_equal(res[0]["c"], res[1]["c"])
+    np.testing.assert_array_equal(res[0]["order"], res[1]["order"])
+    bad = fg.random_forest(rng, 5, 2, 20, w.params.vocab)
+    left = bad.left.copy()
+    left[int(np.flatnonzero(bad.left >= 0)[0])] = bad.n_nodes + 7      # a child index out of range
+    broken = dataclasses.replace(bad, left=left)
+    for form in (1, 0):
+        model.set_option(binding.OPT_OVERLAP_LAUNCH, form)
+        with pytest.raises(binding.TreeLSTMError):
+            util.gpu_forward(model, broken, binding.PERSISTENT)
+        out = util.gpu_forward(model, w.forest, binding.PERSISTENT)     # the context keeps working
+        np.testing.assert_array_equal(out["h"], res[0]["h"])
+    model.close()
 
 
 def test_bf16_deeper_than_the_level_cache():
