@@ -228,12 +228,13 @@ def _dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def time_forward(model, forest, flags, steps, warmup, flush, kernel_every=16):
+def time_forward(model, forest, flags, steps, warmup, flush, kernel_every=16, overlap_launch=None):
     """`steps` forward calls on a device-resident forest, L2 flushed before each (untimed), CUDA events
     on the launching stream around every call.  The wavefront kernel's own device time is taken in a
-    second, shorter pass (steps / kernel_every calls, same flushing): the library's event pair around
+    second pass (same flushing, read on every kernel_every-th call): the library's event pair around
     that kernel sits between the scheduler and the wavefront kernel on the stream and keeps the
-    latter from starting under the former, so it stays out of the timed steps.
+    latter from starting under the former, so it stays out of the timed steps; in that pass the
+    kernel is launched in plain stream order (behind an event a dependent launch only adds latency).
     Returns (per-step ms list, mean kernel ms, launches, outputs)."""
     import torch
     from paper_1809_00832_b200 import binding
@@ -257,12 +258,16 @@ def time_forward(model, forest, flags, steps, warmup, flush, kernel_every=16):
     if status != 0:
         raise RuntimeError(f"device status {status} after the timed region")
     model.set_option(binding.OPT_TIME_WAVEFRONT_KERNEL, 1)
+    if overlap_launch is None or overlap_launch:
+        model.set_option(binding.OPT_OVERLAP_LAUNCH, 0)   # the kernel alone: launched in plain stream order behind the event
     kernel_ms = []
-    for i in range(max(8, steps // kernel_every)):  # live device time of the wavefront kernel
+    for i in range(max(8 * kernel_every, min(steps, 512))):  # live device time of the wavefront kernel
         flush.fill_(i & 0xFF)
         model.forward(left, right, token, flags=flags, out=out, check=False)
-        kernel_ms.append(model.last_kernel_ms())
+        if i % kernel_every == kernel_every - 1:    # reading it waits for the device: not after every call
+            kernel_ms.append(model.last_kernel_ms())
     model.set_option(binding.OPT_TIME_WAVEFRONT_KERNEL, 0)
+    model.set_option(binding.OPT_OVERLAP_LAUNCH, 1 if overlap_launch is None else overlap_launch)
     return [a.elapsed_time(b) for a, b in ev], statistics.mean(kernel_ms), launches, out
 
 
@@ -522,7 +527,7 @@ def main() -> int:
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    step_ms, k_ms, launches, out = time_forward(model, f, flags, args.steps, args.warmup, flush)
+    step_ms, k_ms, launches, out = time_forward(model, f, flags, args.steps, args.warmup, flush, overlap_launch=args.overlap_launch)
     if dist is not None:
         dist.barrier()
     ran = {binding.PERSISTENT: "persistent", binding.PER_LEVEL: "per_level", binding.SUBFORESTS: "subforests"}[model.last_mode()]

@@ -173,20 +173,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int Hp = p.Hp, H = p.H;
   const int groups = Hp / kUnitGroup;
-  // What needs nothing from the kernel before (the ready-set construction): barriers, tensor memory,
-  // and warming L2.  In persistent mode this kernel is launched as a programmatic dependent of the
+  // What needs nothing from the kernel before (the ready-set construction): warming L2.  In persistent mode this kernel is launched as a programmatic dependent of the
   // scheduler and gets here while that one still runs; the wait below ends when it has finished.
-  if (tid == 0) {
-    for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
-    mbar_init(epi_bar, 256);
-    mbar_init(drain_bar, 1);
-    *s_abort = 0;
-    s_early = 0u;
-    s_pre = 0u;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // columns: 2 accumulator stages x 256
   if (only_level < 0) {
     // Every CTA reads the packed weights and biases in every wavefront, but they may have left L2 since
     // the last call: all CTAs ask for a share of them now, and for the tensor maps, so that the first
@@ -221,6 +209,17 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
 #define TL_ROLE_STAMP(slot_first, slot_second) do { } while (0)
 #endif
 
+  if (tid == 0) {
+    for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 256); }
+    mbar_init(epi_bar, 256);
+    mbar_init(drain_bar, 1);
+    *s_abort = 0;
+    s_early = 0u;
+    s_pre = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // columns: 2 accumulator stages x 256
   for (int i = tid; i < kLevelCache && i <= n_levels; i += kThreads) s_level_offset[i] = p.level_offset[i];
   tc_fence_before();
   __syncthreads();
