@@ -27,6 +27,7 @@ WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward) {
     L.xin = take(2 * nn * (size_t)ctx->Ep);          // leaf embedding rows in ready order
     L.ain = take(2 * nn * 2 * (size_t)ctx->Hp);      // [h_l | h_r] of every position, bf16
     L.cin = take(4 * nn * 2 * (size_t)ctx->H);       // [c_l | c_r] of every position, fp32
+    L.pre = take(4 * 1024);                          // leaves per CTA (wavefront kernel started under the scheduler)
   }
   L.gates = L.dh = L.dc = L.dz = L.tok_slot = off;
   if (with_backward) {

@@ -28,7 +28,7 @@ static_assert(sizeof(DevStatus) == 256, "control block is one 256-byte line grou
 // Offsets (bytes) of the regions inside the workspace for a forest of up to n nodes.
 struct WsLayout {
   size_t status, parent, pending, order_tmp, level_offset, roots, table, slot, part_order, part_offset,
-      part_spill, xin, ain, cin, gates, dh, dc, dz, tok_slot, trace, check, total;
+      part_spill, xin, ain, cin, gates, dh, dc, dz, tok_slot, trace, check, pre, total;
 };
 
 // Cycle stamps of the wavefront kernels (builds with -DTREELSTM_TRACE only): kTraceSlots stamps per

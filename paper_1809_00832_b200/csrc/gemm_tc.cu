@@ -131,6 +131,124 @@ __device__ void prepare_operands(const TcParams& p, int gtid, int gthreads) {
   for (int t = gtid + gthreads; t < n_roots; t += gthreads) p.slot[chk(p.st, p.roots[t], p.n)] = -1;
 }
 
+// Leaves evaluated ahead of the schedule.  Their embedding rows: the same copy as gather_leaf_rows,
+// for the rows [row_begin, row_end) of the kernel's own leaf order, with the token ids clamped into
+// the vocabulary (nothing has been validated at that point).
+__device__ __forceinline__ void gather_leaf_rows_unchecked(const TcParams& p, int row_begin, int row_end, int warp, int n_warps, int lane) {
+  const int cpr = p.Ep / 8;                              // 16-byte chunks per row
+  // a warp takes four rows at a time, all their loads in flight before the first store
+  for (int base = row_begin + warp * 4; base < row_end; base += n_warps * 4) {
+    const int my_row = base + (lane & 3);
+    const int my_tok = my_row < row_end ? min(max(p.token[p.pre_order[my_row]], 0), p.vocab - 1) : 0;
+    int tok[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) tok[k] = __shfl_sync(kFullMask, my_tok, k);
+    for (int c0 = 0; c0 < cpr; c0 += 64) {
+      uint4 v[4][2];
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int cc = c0 + h * 32 + lane;
+          if (base + k < row_end && cc < cpr)
+            v[k][h] = __ldg(reinterpret_cast<const uint4*>(p.emb_bf + (size_t)tok[k] * p.Ep) + cc);
+        }
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int cc = c0 + h * 32 + lane;
+          if (base + k < row_end && cc < cpr)
+            reinterpret_cast<uint4*>(p.xin + (size_t)(base + k) * p.Ep)[cc] = v[k][h];
+        }
+    }
+  }
+}
+
+// Once the schedule is known: every internal position pos (one warp each) gets the slots of its two
+// children written - slot[child] = 2 * pos + side -, and a child that is a leaf has its state handed
+// over right here: bf16 h (padded units as 0) and fp32 c into half `side` of the operand rows of pos.
+// Roots get slot -1.
+__device__ __forceinline__ void deliver_leaves(const TcParams& p, int gwarp, int n_warps, int lane) {
+  const int H = p.H, Hp = p.Hp;
+  const int n_leaves = p.level_offset[1];
+  const bool vec = (H % 4) == 0;
+  // A warp takes four positions at a time.  The chain of dependent loads (position -> node -> children
+  // -> are they leaves) runs once for the four, every lane following position base + (lane & 3); then
+  // the rows of a position's leaf children are loaded together before they are stored.
+  for (int base = n_leaves + gwarp * 4; base < p.n; base += n_warps * 4) {
+    const int pos = base + (lane & 3);
+    int c0 = 0, c1 = 0, bits = 0;
+    if (pos < p.n) {
+      const int node = chk(p.st, p.order[pos], p.n);
+      c0 = chk(p.st, p.left[node], p.n);
+      c1 = chk(p.st, p.right[node], p.n);
+      bits = (p.left[c0] < 0 ? 1 : 0) | (p.left[c1] < 0 ? 2 : 0);
+      if (lane < 4) { p.slot[c0] = 2 * pos; p.slot[c1] = 2 * pos + 1; }
+    }
+    for (int k = 0; k < 4; ++k) {
+      // the two children of position base + k; lane k holds their ids and whether they are leaves
+      const int child0 = __shfl_sync(kFullMask, c0, k), child1 = __shfl_sync(kFullMask, c1, k);
+      const int bb = __shfl_sync(kFullMask, bits, k);
+      if (bb == 0) continue;
+      const bool on0 = (bb & 1) != 0, on1 = (bb & 2) != 0;
+      const float* hrow0 = p.h + (size_t)child0 * H;
+      const float* crow0 = p.c + (size_t)child0 * H;
+      const float* hrow1 = p.h + (size_t)child1 * H;
+      const float* crow1 = p.c + (size_t)child1 * H;
+      const size_t row = (size_t)(base + k) * 2;
+      // two chunks of four units per lane and pass, all eight loads in flight before the stores
+      for (int u0 = lane * 4; u0 < Hp; u0 += 256) {
+        float hv[2][2][4], cv[2][2][4];   // [chunk][side][unit]
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int u = u0 + 128 * q;
+#pragma unroll
+          for (int sd = 0; sd < 2; ++sd) {
+            const float* hrow = sd ? hrow1 : hrow0;
+            const float* crow = sd ? crow1 : crow0;
+            const bool on = sd ? on1 : on0;
+            if (on && vec && u + 3 < H) {
+              const float4 a = __ldcg(reinterpret_cast<const float4*>(hrow + u));
+              const float4 b = __ldcg(reinterpret_cast<const float4*>(crow + u));
+              hv[q][sd][0] = a.x; hv[q][sd][1] = a.y; hv[q][sd][2] = a.z; hv[q][sd][3] = a.w;
+              cv[q][sd][0] = b.x; cv[q][sd][1] = b.y; cv[q][sd][2] = b.z; cv[q][sd][3] = b.w;
+            } else {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const bool in = on && u + j < H;
+                hv[q][sd][j] = in ? __ldcg(hrow + u + j) : 0.f;
+                cv[q][sd][j] = in ? __ldcg(crow + u + j) : 0.f;
+              }
+            }
+          }
+        }
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int u = u0 + 128 * q;
+          if (u >= Hp) continue;
+          const int count = min(4, H - u);
+#pragma unroll
+          for (int sd = 0; sd < 2; ++sd) {
+            if (!(sd ? on1 : on0)) continue;
+            __nv_bfloat162 lo = __floats2bfloat162_rn(hv[q][sd][0], hv[q][sd][1]), hi = __floats2bfloat162_rn(hv[q][sd][2], hv[q][sd][3]);
+            *reinterpret_cast<uint2*>(p.ain + (row + sd) * Hp + u) =
+                make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+            if (count > 0) st_row4(p.cin + (row + sd) * H + u, vec, count, cv[q][sd]);
+          }
+        }
+      }
+      if (lane == 0) {
+        const int n_on = (on0 ? 1 : 0) + (on1 ? 1 : 0);
+        count_write(p.chk_counts ? p.chk_counts + p.n : nullptr, base + k, n_on * H);
+        count_write(p.chk_counts ? p.chk_counts + 2 * p.n : nullptr, base + k, n_on * H);
+      }
+    }
+  }
+  const int n_roots = p.st->n_roots;
+  for (int t = gwarp * 32 + lane; t < n_roots; t += n_warps * 32) p.slot[chk(p.st, p.roots[t], p.n)] = -1;
+}
+
 __global__ void k_prepare_operands(TcParams p) {
   if (ld_volatile(&p.st->status) != 0) return;
   prepare_operands(p, blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
@@ -173,8 +291,30 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int Hp = p.Hp, H = p.H;
   const int groups = Hp / kUnitGroup;
-  // What needs nothing from the kernel before (the ready-set construction): warming L2.  In persistent mode this kernel is launched as a programmatic dependent of the
-  // scheduler and gets here while that one still runs; the wait below ends when it has finished.
+  const int kb_leaf = p.Ep / kKBlock, kb_int = 2 * Hp / kKBlock;
+  const bool vec = (H % 4) == 0;
+  // Persistent mode with the leaves taken first (p.leaves_first): this kernel is launched as a
+  // programmatic dependent of the ready-set construction and starts while that kernel still runs.
+  // Leaves have no inputs to wait for (Section 4.1.1: an operation runs as soon as its inputs are
+  // resolved), and their place in the ready order needs no dependency analysis - they are wavefront 0
+  // in ascending node id.  So the CTAs rank the leaves themselves, fetch their embedding rows and
+  // evaluate the whole leaf wavefront beside the scheduler; only then do they wait for it
+  // (griddepcontrol.wait), and the leaves' states are handed to the callers' operand rows together
+  // with the slot table, once the order of the internal nodes is known.
+  const bool leaves_first = only_level < 0 && p.leaves_first != 0;
+#ifdef TREELSTM_TRACE
+  long long* const trace = blockIdx.x == 0 && tid == 0 ? p.trace : nullptr;
+  long long* const trace_cta = blockIdx.x == 0 ? p.trace : nullptr;   // stamps of the producers and the MMA issuer
+#define TL_ROLE_STAMP(slot_first, slot_second)                                                        \
+  do {                                                                                                \
+    if (t < 2 * (int)gridDim.x) TL_STAMP(trace_cta, lvl, t < (int)gridDim.x ? (slot_first) : (slot_second)); \
+  } while (0)
+#else
+#define TL_ROLE_STAMP(slot_first, slot_second) do { } while (0)
+#endif
+  // phases of a leaves-first run: the last row of the stamp table (slot 0: the kernel has started)
+#define TL_PHASE_STAMP(slot) TL_STAMP(trace, kTraceLevels - 1, slot)
+  TL_PHASE_STAMP(0);
   if (only_level < 0) {
     // Every CTA reads the packed weights and biases in every wavefront, but they may have left L2 since
     // the last call: all CTAs ask for a share of them now, and for the tensor maps, so that the first
@@ -186,28 +326,24 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     warm_l2(p.bp_h, (size_t)groups * kGColsI * 4, gtid, gthreads);
     if (tid < (int)(sizeof(TmapSet) / sizeof(CUtensorMap))) prefetch_tmap(reinterpret_cast<const CUtensorMap*>(&maps) + tid);
   }
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  const bool failed = ld_volatile(&p.st->status) != 0;      // schedule failed: nothing to evaluate
-  const int n_levels = failed ? 0 : p.st->n_levels;
-  // Persistent mode: the narrow wavefronts at the end of the forest are left to one cluster (launched
-  // next on the same stream), which keeps the recurrent weights in shared memory and meets at the
-  // hardware cluster barrier instead of the grid-wide one.
   __shared__ int s_stop[2];
-  // (Without the cluster kernel on the stream the decision is still worked out and left in the control
-  // block: the host learns from it whether launching that kernel is worth its while for forests like this.)
-  const int tail_from = only_level < 0 ? tail_first_level(p.level_offset, n_levels, p.tail_width, p.tail_min_levels, s_stop) : n_levels;
-  const int lvl_stop = p.tail_launched ? tail_from : n_levels;
-  if (only_level < 0 && !failed && blockIdx.x == 0 && tid == 0) p.st->tail_from = tail_from;
-#ifdef TREELSTM_TRACE
-  long long* const trace = blockIdx.x == 0 && tid == 0 ? p.trace : nullptr;
-  long long* const trace_cta = blockIdx.x == 0 ? p.trace : nullptr;   // stamps of the producers and the MMA issuer
-#define TL_ROLE_STAMP(slot_first, slot_second)                                                        \
-  do {                                                                                                \
-    if (t < 2 * (int)gridDim.x) TL_STAMP(trace_cta, lvl, t < (int)gridDim.x ? (slot_first) : (slot_second)); \
-  } while (0)
-#else
-#define TL_ROLE_STAMP(slot_first, slot_second) do { } while (0)
-#endif
+  __shared__ int s_scan[16];
+  bool failed = false;
+  int n_levels = 0, lvl_end = 0;
+  // What the scheduler leaves behind is read here and nowhere before: its status, the number of
+  // wavefronts, their boundaries, and where the grid-wide kernel stops (the narrow wavefronts at the end
+  // of a forest may go to one cluster, launched next on the stream; without that launch the decision
+  // is still worked out and left in the control block for the host to learn from).
+  auto take_schedule = [&]() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    failed = ld_volatile(&p.st->status) != 0;      // schedule failed: nothing to evaluate
+    n_levels = failed ? 0 : p.st->n_levels;
+    const int tail_from = only_level < 0 ? tail_first_level(p.level_offset, n_levels, p.tail_width, p.tail_min_levels, s_stop) : n_levels;
+    if (only_level < 0 && !failed && blockIdx.x == 0 && tid == 0) p.st->tail_from = tail_from;
+    lvl_end = only_level >= 0 ? only_level + 1 : (p.tail_launched ? tail_from : n_levels);
+    for (int i = tid; i < kLevelCache && i <= n_levels; i += kThreads) s_level_offset[i] = p.level_offset[i];
+  };
+  if (!leaves_first) take_schedule();
 
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
@@ -220,14 +356,10 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 5) tmem_alloc(smem_u32(s_tmem), 512);   // columns: 2 accumulator stages x 256
-  for (int i = tid; i < kLevelCache && i <= n_levels; i += kThreads) s_level_offset[i] = p.level_offset[i];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-
-  const int kb_leaf = p.Ep / kKBlock, kb_int = 2 * Hp / kKBlock;
-  const bool vec = (H % 4) == 0;
 
   // Pipeline positions; every role walks the same tile sequence, so they stay in step.  The ring
   // is re-cut at every wavefront (thin tiles leave room for more stages); each mbarrier keeps its
@@ -240,15 +372,87 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   bool pre = false;                     // producers: this warp's first box of the wavefront was requested at the barrier
   uint32_t armed = 0;                   // producers (lane 0): ring stages this thread has requested a box into
 
-  if (only_level < 0 && n_levels > 0) {
+  if (leaves_first) {
+    // ---- the leaves' ranks: CTA b looks at the node ids [b * chunk, (b + 1) * chunk) ----
+    // (the control block was cleared by the scheduler before it let this kernel start; its barrier
+    // counter is this kernel's alone)
+    const int chunk = (p.n + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int lo = min(p.n, (int)blockIdx.x * chunk), hi = min(p.n, lo + chunk);
+    const int per = (hi - lo + kThreads - 1) / kThreads;
+    const int my_lo = min(hi, lo + tid * per), my_hi = min(hi, my_lo + per);
+    int mine = 0;
+    for (int k = my_lo; k < my_hi; ++k)
+      if (p.left[k] < 0) {
+        ++mine;
+        // the leaf's embedding row is wanted in L2 by the time the rows are copied into ready order
+        const int tok = min(max(p.token[k], 0), p.vocab - 1);
+        warm_l2(p.emb_bf + (size_t)tok * p.Ep, (size_t)p.Ep * 2, 0, 1);
+      }
+    // exclusive prefix over the threads of the CTA (and the total) of one int per thread
+    auto cta_scan = [&](int v, int& total) {
+      int inc = v;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(kFullMask, inc, d);
+        if (lane >= d) inc += o;
+      }
+      __syncthreads();
+      if (lane == 31) s_scan[warp] = inc;
+      __syncthreads();
+      int before = 0, all = 0;
+#pragma unroll
+      for (int w2 = 0; w2 < kThreads / 32; ++w2) {
+        const int c2 = s_scan[w2];
+        if (w2 < warp) before += c2;
+        all += c2;
+      }
+      total = all;
+      return before + inc - v;
+    };
+    int cta_leaves = 0;
+    TL_PHASE_STAMP(1);   // tensor memory and barriers set up, own share of the child array read
+    const int my_first = cta_scan(mine, cta_leaves);
+    if (tid == 0) p.pre_counts[blockIdx.x] = cta_leaves;
+    arrivals += gridDim.x;
+    if (!grid_barrier(p.st, arrivals, p.wait_limit, s_flag)) stop = true;
+    TL_PHASE_STAMP(2);   // every CTA's leaf count is known
+    int n_leaves = 0, base = 0;
+    {
+      // leaves in front of this CTA's node ids, and all of them (the grid has at most kThreads CTAs)
+      const int v = tid < (int)gridDim.x ? __ldcg(p.pre_counts + tid) : 0;
+      const int before = cta_scan(v, n_leaves);
+      if (tid == (int)blockIdx.x) s_stop[0] = before;
+      __syncthreads();
+      base = s_stop[0];
+    }
+    if (!stop) {
+      int rank = base + my_first;
+      for (int k = my_lo; k < my_hi; ++k)
+        if (p.left[k] < 0) p.pre_order[rank++] = k;
+      __syncthreads();
+      // the embedding rows of this CTA's leaves, in ready order (token ids are clamped: nothing has
+      // been validated yet, and a forest the scheduler rejects must not make this kernel read astray)
+      gather_leaf_rows_unchecked(p, base, base + cta_leaves, warp, kThreads / 32, lane);
+      TL_PHASE_STAMP(3);   // own leaves ranked, their embedding rows copied
+      asm volatile("fence.proxy.async.global;" ::: "memory");    // Xin is read through TMA
+      arrivals += gridDim.x;
+      if (!grid_barrier(p.st, arrivals, p.wait_limit, s_flag)) stop = true;
+    }
+    TL_PHASE_STAMP(4);   // all embedding rows are in place: the leaf wavefront starts
+    if (tid == 0) { s_level_offset[0] = 0; s_level_offset[1] = n_leaves; }
+    n_levels = n_leaves > 0 ? 1 : 0;
+    lvl_end = n_levels;
+    __syncthreads();
+  } else if (only_level < 0 && n_levels > 0) {
+    __syncthreads();                                            // the cached wavefront boundaries
     prepare_operands(p, blockIdx.x * kThreads + tid, gridDim.x * kThreads);
     asm volatile("fence.proxy.async.global;" ::: "memory");    // Xin is read through TMA
     arrivals += gridDim.x;
     if (!grid_barrier(p.st, arrivals, p.wait_limit, s_flag)) stop = true;
   }
+  __syncthreads();
 
   const int lvl_begin = only_level >= 0 ? only_level : 0;
-  const int lvl_end = only_level >= 0 ? only_level + 1 : lvl_stop;
   auto level_begin = [&](int l) { return l < kLevelCache ? s_level_offset[l] : p.level_offset[l]; };
   auto make_plan = [&](int l) {
     return choose_tile_plan(level_begin(l + 1) - level_begin(l), groups, p.sched_ctas, l == 0, l == 0 ? kb_leaf : kb_int);
@@ -257,6 +461,31 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   // wavefront ahead, everybody else picks the result up after the barrier.
   if (warp == 11 && lane == 0 && lvl_begin < lvl_end) s_plan[lvl_begin & 1] = make_plan(lvl_begin);
   __syncthreads();
+  // After the leaf wavefront of a leaves-first run: wait for the schedule, then every internal position
+  // gets its slots written and the states of those of its children that are leaves.
+  auto hand_leaves_over = [&]() {
+    TL_PHASE_STAMP(5);   // all leaf states are in memory
+    take_schedule();
+    __syncthreads();
+    TL_PHASE_STAMP(6);   // the scheduler has ended, its results are read
+    if (n_levels > 0) {
+      deliver_leaves(p, blockIdx.x * (kThreads / 32) + warp, gridDim.x * (kThreads / 32), lane);
+      asm volatile("fence.proxy.async.global;" ::: "memory");    // the operand rows are read through TMA
+    }
+    if (warp == 11 && lane == 0 && 1 < lvl_end) s_plan[1] = make_plan(1);
+    TL_PHASE_STAMP(7);   // slots written, leaf states handed to their callers
+    arrivals += gridDim.x;
+    if (!grid_barrier(p.st, arrivals, p.wait_limit, s_flag)) stop = true;
+    TL_PHASE_STAMP(8);   // the first internal wavefront may start
+  };
+  if (leaves_first && (lvl_end == 0 || stop)) {
+    // Nothing was evaluated: no leaf at all (the scheduler rejects such a forest) or a barrier gave
+    // up.  The scheduler's status word is final once the wait has ended.
+    take_schedule();
+    if (!stop && !failed && tid == 0) report(p.st, TREELSTM_ERR_CHECK);   // a valid forest has leaves
+    stop = true;
+    lvl_end = 0;
+  }
   for (int lvl = lvl_begin; lvl < lvl_end && !stop; ++lvl) {   // uniform trip count: barriers inside
     const int begin = level_begin(lvl), end = level_begin(lvl + 1);
     const bool leaf = lvl == 0;
@@ -277,6 +506,10 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
     stage = 0;
     int nx_node = 0, nx_slot = -1;                  // epilogue: row data of this CTA's next tile, fetched a tile ahead
     bool nx_have = false;
+    // leaves evaluated ahead of the schedule: their order is this kernel's own, and their states are
+    // handed to the callers later (hand_leaves_over)
+    const bool ahead = leaves_first && leaf;
+    const int* const order_cur = ahead ? p.pre_order : p.order;
 
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x) {
       // fat tile t = (row tile, column tile); a piece of the split last round is a column piece of a fat tile
@@ -381,8 +614,8 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
         if (nx_have) {
           node = nx_node; slot = nx_slot;
         } else {
-          node = valid ? chk(p.st, p.order[row], p.n) : 0;
-          slot = valid ? chk_slot(p.st, p.slot[node], p.n) : -1;
+          node = valid ? chk(p.st, order_cur[row], p.n) : 0;
+          slot = valid && !ahead ? chk_slot(p.st, p.slot[node], p.n) : -1;
         }
         // the same two dependent loads for this CTA's next tile go out now and land while this tile is computed
         const int t2 = t + (int)gridDim.x;
@@ -392,7 +625,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
           const int fat2 = t2 < plan.tail_from ? t2 : plan.tail_from + ((t2 - plan.tail_from) >> plan.tail_ls);
           const int rtile2 = fat2 / ntn, row2 = begin + (rtile2 << plan.lrt) + r;
           valid2 = r < rt && row2 < end;
-          nx_node = valid2 ? chk(p.st, p.order[row2], p.n) : 0;
+          nx_node = valid2 ? chk(p.st, order_cur[row2], p.n) : 0;
         }
         EpiTile et;
         et.leaf = leaf; et.G = G; et.gcols = gcols; et.ncols = ncols; et.nt = nt;
@@ -409,13 +642,23 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
         // the CTA's first tile of the wavefront stamps slots 1-3, its second one slots 8-10
         if (trace != nullptr && lvl < kTraceLevels && t < 2 * (int)gridDim.x) et.stamp = trace + lvl * kTraceSlots + (t < (int)gridDim.x ? 1 : 8);
 #endif
-        epilogue_tile(p, et, epi_phase, alive, s_abort, [&]() { if (nx_have) nx_slot = valid2 ? chk_slot(p.st, p.slot[nx_node], p.n) : -1; });
+        epilogue_tile(p, et, epi_phase, alive, s_abort, [&]() { if (nx_have) nx_slot = valid2 && !ahead ? chk_slot(p.st, p.slot[nx_node], p.n) : -1; });
         ++acc_iter;
       }
     }
     // the operand rows the epilogue wrote are read through TMA (async proxy) by later wavefronts
     if (warp < 4 || (warp >= 6 && warp < 10)) asm volatile("fence.proxy.async.global;" ::: "memory");
     TL_STAMP(trace, lvl, 6);
+    if (ahead) {
+      // every CTA's leaf states must be in memory before anyone hands them on
+      __syncthreads();
+      if (*s_abort) break;
+      arrivals += (uint32_t)min(tiles, (int)gridDim.x);
+      if (!grid_barrier(p.st, arrivals, p.wait_limit, s_flag, (int)blockIdx.x < tiles)) break;
+      hand_leaves_over();
+      TL_STAMP(trace, lvl, 7);
+      continue;
+    }
     if (only_level < 0 && lvl + 1 < lvl_end) {
       // every role of every CTA joins the barrier.  A role that gave up has set s_abort before
       // this point, so the flag read after the CTA barrier is the same for all threads and the
@@ -692,10 +935,24 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.tail_width = tail_possible ? ctx->opt.tail_width : 0;
   p.tail_min_levels = ctx->opt.tail_min_levels;
   p.tail_launched = with_tail ? 1 : 0;
+  // Started under the single-CTA scheduler, the kernel takes the leaves first (the scratch of the
+  // multi-CTA scheduler, unused then, holds its leaf order).
+  const int single_max = ctx->opt.sched_single_cta_max < kSchedSingleMaxNodes ? ctx->opt.sched_single_cta_max : kSchedSingleMaxNodes;
+  int grid_persistent = ctx->sm_count;                 // one CTA per SM (shared and tensor memory)
+  if (ctx->opt.max_ctas > 0 && grid_persistent > ctx->opt.max_ctas) grid_persistent = ctx->opt.max_ctas;
+  const bool overlap = (flags & TREELSTM_PERSISTENT) && ctx->opt.overlap_launch && n <= single_max &&
+                       ctx->tc_resident_ctas >= ctx->sm_count && ctx->sm_count > 1 && ctx->sm_count <= kThreads;
+  if (overlap && grid_persistent > ctx->sm_count - 1) grid_persistent = ctx->sm_count - 1;   // the scheduler keeps its SM
+  p.leaves_first = overlap ? 1 : 0;
+  p.pre_counts = reinterpret_cast<int*>(base + lay.pre);
+  p.pre_order = reinterpret_cast<int*>(base + lay.pending);
+  if (overlap) p.sched_ctas = ctx->sm_count - 1;   // the tile plans count on the CTAs that run
   p.trace = nullptr;
 #ifdef TREELSTM_TRACE
   p.trace = reinterpret_cast<long long*>(base + lay.trace);
-  TL_CUDA(ctx, cudaMemsetAsync(p.trace, 0, sizeof(long long) * kTraceSlots * kTraceLevels, stream));
+  // (a run started under the scheduler keeps the stamps of the run before: a clearing operation between
+  // the two kernels would hold this one back until the scheduler has ended)
+  if (!overlap) TL_CUDA(ctx, cudaMemsetAsync(p.trace, 0, sizeof(long long) * kTraceSlots * kTraceLevels, stream));
 #endif
   {
     int rc = ensure_operand_tmaps(ctx, ws, n, p.xin, p.ain);
@@ -704,10 +961,9 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
 
   const int groups = ctx->Hp / kUnitGroup;
   if (flags & TREELSTM_PERSISTENT) {
-    int grid = ctx->sm_count;                       // one CTA per SM (shared and tensor memory)
+    int grid = grid_persistent;
     const int want = ((n + 31) / 32 + 1) * groups;       // never more CTAs than the thinnest tiling has tiles
     if (grid > want) grid = want;
-    if (ctx->opt.max_ctas > 0 && grid > ctx->opt.max_ctas) grid = ctx->opt.max_ctas;
     int only = -1;
     // The grid barrier needs every CTA resident.  Two ways to launch:
     //  * as a programmatic dependent of the kernel before it on the stream - the ready-set construction:
@@ -722,7 +978,7 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = stream;
     cudaLaunchAttribute attr;
-    if (ctx->opt.overlap_launch && grid <= ctx->tc_resident_ctas) {
+    if (overlap) {
       attr.id = cudaLaunchAttributeProgrammaticStreamSerialization; attr.val.programmaticStreamSerializationAllowed = 1;
     } else {
       attr.id = cudaLaunchAttributeCooperative; attr.val.cooperative = 1;

@@ -329,9 +329,6 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
   const int tid = threadIdx.x;
   constexpr unsigned short kNoParent = 0xFFFF;
   constexpr unsigned int kDone = 0x80000000u;
-  // A kernel launched behind this one as its programmatic dependent may start now: the part of it
-  // that comes before its own wait for this grid needs nothing from here.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid < (int)(sizeof(DevStatus) / sizeof(int))) reinterpret_cast<int*>(st)[tid] = 0;
 #ifdef TREELSTM_TRACE
   // phase stamps of thread 0 (cycles since the start) in the unused words of the control block
@@ -343,6 +340,14 @@ k_schedule_single(int n, const int* __restrict__ left, const int* __restrict__ r
   if (tid == 0) { s_err = 0; s_maxlevel = 0; s_qhead = 0; s_qtail = 0; }
   for (int k = tid; k < n; k += kSingleThreads) { w[k] = 0; par[k] = kNoParent; }
   __syncthreads();
+  // A kernel launched behind this one as its programmatic dependent may start now.  The part of it
+  // that comes before its own wait for this grid reads nothing this grid writes, except that it
+  // uses the (now cleared) control block: its barrier counter, and the status word this grid may
+  // still set.
+  if (tid == 0) {
+    __threadfence();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
   TL_SCHED_STAMP(0);   // cleared
   // validate; children record their caller; leaves are complete at once (level 0)
   // Node j of this thread is tid + j * 1024 (at most 32 per thread); leaf_bits remembers which are

@@ -38,6 +38,12 @@ struct TcParams {
   // hand-over from the grid-wide kernel to one cluster (persistent mode): see tail_first_level
   int tail_width, tail_min_levels;
   int tail_launched;             // the cluster kernel follows on the stream (else the decision is only recorded)
+  // grid-wide kernel started under the scheduler: the leaf wavefront is ranked and evaluated before
+  // the schedule is read.  pre_counts [grid]: leaves per CTA's share of the node ids; pre_order [n]: the
+  // leaves in ascending node id
+  int leaves_first = 0;
+  int* pre_counts = nullptr;
+  int* pre_order = nullptr;
   long long* trace;              // cycle stamps (trace builds), else nullptr
 };
 

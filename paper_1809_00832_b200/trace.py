@@ -61,6 +61,8 @@ def main() -> int:
     ap.add_argument("--tail-min-levels", type=int, default=None)
     ap.add_argument("--trees", type=int, default=None)
     ap.add_argument("--levels", default=None, help="A:B - print only wavefronts A..B-1")
+    ap.add_argument("--plain-order", action="store_true",
+                    help="launch the grid-wide kernel cooperatively behind the scheduler instead of under it")
     args = ap.parse_args()
     build.build(variant="trace")
     w = fg.make_workload(args.workload, 0, args.trees)
@@ -73,7 +75,11 @@ def main() -> int:
         model.set_option(binding.OPT_TAIL_MIN_LEVELS, args.tail_min_levels)
     flags = binding.PERSISTENT if args.mode == "persistent" else binding.SUBFORESTS
     left, right, token = dev(f.left), dev(f.right), dev(f.token)
+    # the first call in plain stream order: it clears the stamp table (a call started under the scheduler
+    # keeps the stamps of the call before)
+    model.set_option(binding.OPT_OVERLAP_LAUNCH, 0)
     out = model.forward(left, right, token, flags=flags)
+    model.set_option(binding.OPT_OVERLAP_LAUNCH, 0 if args.plain_order else 1)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     for i in range(4):                                   # the last call is the one read back, caches as in the bench
         flush.fill_(i)
@@ -96,6 +102,14 @@ def main() -> int:
               "starts known, placed = " + ", ".join(str(int(buf[8 + i])) for i in range(5)))
     for which, name in ((0, "grid-wide kernel"), (1, "cluster kernel")):
         t = read_trace(model, which)
+        if which == 0 and t[LEVELS - 1, 4] != 0:
+            ph = t[LEVELS - 1]
+            names = ("set up, own node ids read", "leaf counts of all CTAs known", "own leaves ranked, embedding rows copied",
+                     "all rows in place (leaf wavefront starts)", "leaf wavefront done everywhere", "scheduler ended, schedule read",
+                     "slots written, leaf states handed over", "first internal wavefront may start")
+            print("# grid-wide kernel started under the scheduler, first CTA, cycles since its start: " +
+                  ", ".join(f"{nm} {int(ph[i + 1] - ph[0])}" for i, nm in enumerate(names)))
+            t[LEVELS - 1] = 0
         rows = [l for l in range(min(len(widths), LEVELS)) if t[l, 0] != 0]
         if not rows:
             continue

@@ -285,6 +285,32 @@ def test_both_launch_forms_give_identical_states():
     model.close()
 
 
+def test_leaves_taken_first_on_small_grids_and_leaf_only_forests():
+    """the kernel started under the scheduler ranks the leaves itself (every CTA a share of the node
+    ids): same bits as the run in plain stream order on grids of 1, 5 and 40 CTAs (several node ids
+    per thread), on a forest of single-leaf trees only (one wavefront) and on a mixed one"""
+    rng = np.random.default_rng(50)
+    params = fg.draw_params(rng, 128, 72, 400, emb_dist="normal", emb_scale=0.3, w_scale=0.15)
+    forests = [fg.random_forest(rng, 37, 1, 1, 400),        # leaves only
+               fg.random_forest(rng, 60, 1, 24, 400)]
+    forests[1], _ = fg.permute_node_ids(forests[1], rng)
+    model = util.make_model(params, "bf16")
+    for forest in forests:
+        model.set_option(binding.OPT_MAX_CTAS, 0)
+        model.set_option(binding.OPT_OVERLAP_LAUNCH, 0)
+        ref = util.gpu_forward(model, forest, binding.PERSISTENT)
+        h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
+        assert util.max_abs(ref["h"], h) < util.TOL["bf16"]
+        model.set_option(binding.OPT_OVERLAP_LAUNCH, 1)
+        for ctas in (0, 1, 5, 40):
+            model.set_option(binding.OPT_MAX_CTAS, ctas)
+            res = util.gpu_forward(model, forest, binding.PERSISTENT)
+            np.testing.assert_array_equal(res["h"], ref["h"])
+            np.testing.assert_array_equal(res["c"], ref["c"])
+            np.testing.assert_array_equal(res["order"], ref["order"])
+    model.close()
+
+
 def test_bf16_deeper_than_the_level_cache():
     """a left chain of 1100 leaves next to a few small trees: 1100 wavefronts, more than the kernels
     keep wavefront boundaries for in shared memory (the rest is read from global memory, and the
