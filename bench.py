@@ -31,7 +31,10 @@ L2_FLUSH_BYTES = 256 << 20          # larger than the 126 MB L2
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the wavefront kernel, from the
 # committed ncu capture named beside it (a constant copied from that capture, not measured by this
 # run); None for workloads without a capture of the current kernel.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    "batch256_bf16": (6309632 + 5627392, "profiles/k_fwd_tc_batch256_bf16.md (static: ncu capture of one launch, not measured by this run)"),
+    "balanced1024_bf16": (10463488 + 74443776, "profiles/k_fwd_tc_balanced1024_bf16.md (static: ncu capture of one launch, not measured by this run)"),
+}
 MODES = ("persistent", "per_level", "subforests")
 
 
@@ -478,6 +481,8 @@ def main() -> int:
                     help="cell of the sweeps (the benchmark line itself is always TreeLSTM)")
     ap.add_argument("--tail-width", type=int, default=None,
                     help="sweeps only: widest wavefront handed to the one-cluster kernel (0 = never hand over)")
+    ap.add_argument("--leaves-first-min-nodes", type=int, default=None,
+                    help="headline run only: smallest forest whose leaf wavefront runs before the wait for the schedule")
     ap.add_argument("--overlap-launch", type=int, default=None, choices=[0, 1],
                     help="headline run only: 0 = plain stream order between the scheduler and the wavefront kernel")
     ap.add_argument("--sweep", default=None, choices=["shapes", "length", "all"],
@@ -519,6 +524,8 @@ def main() -> int:
     model = binding.TreeLSTM(p.H, p.E, p.vocab, _dev(p.emb), _dev(p.W), _dev(p.b), prec)
     if args.overlap_launch is not None:
         model.set_option(binding.OPT_OVERLAP_LAUNCH, args.overlap_launch)
+    if args.leaves_first_min_nodes is not None:
+        model.set_option(binding.OPT_LEAVES_FIRST_MIN_NODES, args.leaves_first_min_nodes)
     flags = {"persistent": binding.PERSISTENT, "per_level": binding.PER_LEVEL, "subforests": binding.SUBFORESTS}[args.mode]
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
 

@@ -124,6 +124,11 @@ typedef enum treelstm_status {
                                             /* itself; otherwise the bounded grid barrier ends the call    */
                                             /* with TREELSTM_ERR_TIMEOUT.  0: cooperative launch in plain  */
                                             /* stream order (residency guaranteed by the runtime)          */
+#define TREELSTM_OPT_LEAVES_FIRST_MIN_NODES 9 /* a kernel started that way evaluates the leaf wavefront    */
+                                            /* before it waits for the schedule if the forest has at least */
+                                            /* this many nodes (default 4096); smaller forests keep the    */
+                                            /* order of work of the cooperative launch: their scheduler    */
+                                            /* is too short to hide the two extra grid barriers            */
 
 /*
  * treelstm_create - build a context for one set of parameters.

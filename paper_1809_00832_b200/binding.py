@@ -41,6 +41,7 @@ OPT_TAIL_WIDTH = 5
 OPT_TAIL_MIN_LEVELS = 6
 OPT_TAIL_MAX_NODES = 7
 OPT_OVERLAP_LAUNCH = 8
+OPT_LEAVES_FIRST_MIN_NODES = 9
 
 _vp = ctypes.c_void_p
 _i = ctypes.c_int

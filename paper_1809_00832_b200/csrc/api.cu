@@ -295,6 +295,9 @@ int treelstm_set_option(treelstm_t* ctx, int key, long long value) {
       ctx->opt.tail_min_levels = value > (1 << 20) ? (1 << 20) : (int)value;
       ctx->tail_skip = false;
       return TREELSTM_OK;
+    case TREELSTM_OPT_LEAVES_FIRST_MIN_NODES:
+      ctx->opt.leaves_first_min_nodes = value > (1 << 30) ? (1 << 30) : (int)value;
+      return TREELSTM_OK;
     case TREELSTM_OPT_OVERLAP_LAUNCH:
       ctx->opt.overlap_launch = value != 0;
       return TREELSTM_OK;

@@ -52,6 +52,7 @@ struct Options {
   int tail_width = 32;    // persistent bf16 forward: trailing wavefronts this narrow may run on one cluster (0: never)
   int tail_min_levels = 0; // > 0: hand them over if at least this many remain; 0: the device decides by its cost model
   int tail_max_nodes = 4096;   // forests with more nodes never launch the cluster kernel
+  int leaves_first_min_nodes = 4096;   // forests at least this large: leaf wavefront before the wait for the schedule
   int overlap_launch = 1;      // persistent bf16 forward: the wavefront kernel starts under the scheduler (programmatic dependent launch)
 };
 

@@ -943,7 +943,7 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
   const bool overlap = (flags & TREELSTM_PERSISTENT) && ctx->opt.overlap_launch && n <= single_max &&
                        ctx->tc_resident_ctas >= ctx->sm_count && ctx->sm_count > 1 && ctx->sm_count <= kThreads;
   if (overlap && grid_persistent > ctx->sm_count - 1) grid_persistent = ctx->sm_count - 1;   // the scheduler keeps its SM
-  p.leaves_first = overlap ? 1 : 0;
+  p.leaves_first = overlap && n >= ctx->opt.leaves_first_min_nodes ? 1 : 0;
   p.pre_counts = reinterpret_cast<int*>(base + lay.pre);
   p.pre_order = reinterpret_cast<int*>(base + lay.pending);
   if (overlap) p.sched_ctas = ctx->sm_count - 1;   // the tile plans count on the CTAs that run

@@ -302,6 +302,7 @@ def test_leaves_taken_first_on_small_grids_and_leaf_only_forests():
         h, c, _ = orc.forward_recursive(forest.left, forest.right, forest.token, params.emb, params.W, params.b)
         assert util.max_abs(ref["h"], h) < util.TOL["bf16"]
         model.set_option(binding.OPT_OVERLAP_LAUNCH, 1)
+        model.set_option(binding.OPT_LEAVES_FIRST_MIN_NODES, 0)     # these forests are below the default threshold
         for ctas in (0, 1, 5, 40):
             model.set_option(binding.OPT_MAX_CTAS, ctas)
             res = util.gpu_forward(model, forest, binding.PERSISTENT)
