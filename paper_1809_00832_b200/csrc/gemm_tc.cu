@@ -257,8 +257,11 @@ __global__ void k_prepare_operands(TcParams p) {
 // only_level >= 0: process that wavefront only (one launch per level; operands prepared before).
 // only_level < 0: prepare the operands, then all wavefronts, separated by the bounded grid barrier (cooperative
 // launch).
+template <bool kLeavesFirst>
 __global__ void __launch_bounds__(kThreads, 1)
 k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
+  // kLeavesFirst = false: the instantiation for launches that never take the leaves ahead of the schedule (one
+  // launch per wavefront, cooperative launches); its code is the smaller one
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
@@ -301,7 +304,7 @@ k_fwd_tc(const __grid_constant__ TmapSet maps, TcParams p, int only_level) {
   // evaluate the whole leaf wavefront beside the scheduler; only then do they wait for it
   // (griddepcontrol.wait), and the leaves' states are handed to the callers' operand rows together
   // with the slot table, once the order of the internal nodes is known.
-  const bool leaves_first = only_level < 0 && p.leaves_first != 0;
+  constexpr bool leaves_first = kLeavesFirst;   // (the host launches that instantiation in persistent mode only, with p.leaves_first set)
 #ifdef TREELSTM_TRACE
   long long* const trace = blockIdx.x == 0 && tid == 0 ? p.trace : nullptr;
   long long* const trace_cta = blockIdx.x == 0 ? p.trace : nullptr;   // stamps of the producers and the MMA issuer
@@ -860,9 +863,10 @@ int ensure_operand_tmaps(treelstm* ctx, void* ws, int n, const void* xin, const 
 }
 
 int init_tc_attributes(treelstm* ctx) {
-  TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  TL_CUDA(ctx, cudaFuncSetAttribute(k_fwd_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
   int per_sm = 0;
-  TL_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_fwd_tc, kThreads, kSmemBytes));
+  TL_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_fwd_tc<true>, kThreads, kSmemBytes));
   ctx->tc_resident_ctas = per_sm * ctx->sm_count;
   return TREELSTM_OK;
 }
@@ -984,7 +988,8 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
       attr.id = cudaLaunchAttributeCooperative; attr.val.cooperative = 1;
     }
     cfg.attrs = &attr; cfg.numAttrs = 1;
-    TL_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_fwd_tc, ctx->maps, p, only));
+    if (p.leaves_first) TL_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_fwd_tc<true>, ctx->maps, p, only));
+    else TL_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_fwd_tc<false>, ctx->maps, p, only));
     ctx->launches += 1;
     if (with_tail)
       return launch_forward_bf16_tail(ctx, n, left, right, token, h, c, order, level_offset_dev, flags, ws, lay, stream);
@@ -1001,7 +1006,7 @@ int launch_forward_bf16(treelstm* ctx, int n, const int32_t* left, const int32_t
     if (w <= 0) continue;
     const int tiles = choose_tile_plan(w, groups, p.sched_ctas, lvl == 0,
                                        lvl == 0 ? ctx->Ep / kKBlock : 2 * ctx->Hp / kKBlock).tiles;
-    k_fwd_tc<<<tiles, kThreads, kSmemBytes, stream>>>(ctx->maps, p, lvl);
+    k_fwd_tc<false><<<tiles, kThreads, kSmemBytes, stream>>>(ctx->maps, p, lvl);
     ctx->launches += 1;
   }
   TL_CUDA(ctx, cudaGetLastError());
