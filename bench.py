@@ -79,6 +79,8 @@ def roofline_block(forest, p, precision: str, kernel_ms: float, step_ms: float, 
     head.update({
         "traffic": traffic, "traffic_source": source, "peak_source": peaks["source"],
         "kernel": "k_fwd_tc (persistent wavefront kernel)" if precision == "bf16" else "k_fwd_fp32_persistent",
+        "kernel_timing": "alone, between the library's event pair, launched in plain stream order behind the scheduler "
+                         "(in the timed steps the bf16 kernel starts under the scheduler and takes the leaves first)",
         "kernel_ms": kernel_ms, "algorithmic_bytes": abytes, "algorithmic_flops": flops,
         "frac_of_step": head["frac"] * kernel_ms / step_ms,
         "hbm_gbs": gbs, "hbm_frac": gbs / peaks["hbm_gbs"],
