@@ -159,8 +159,9 @@ TREELSTM_API int treelstm_create(treelstm_t** out, int H, int E, int vocab, cons
  * fp32 arithmetic.  H <= 4096 (TreeRNN), H <= 128 (RNTN).  Parameters are copied (the tensor is
  * re-packed); the call synchronises `stream`.  Such a context takes treelstm_forward (flags
  * TREELSTM_PER_LEVEL or TREELSTM_PERSISTENT; c may be NULL and is not written), treelstm_roots
- * (root_c is not written), treelstm_forward_host (c, root_c not written), treelstm_status_sync and
- * treelstm_destroy; the training calls return TREELSTM_ERR_UNSUPPORTED.
+ * (root_c is not written), treelstm_forward_host (c, root_c not written), treelstm_status_sync,
+ * treelstm_set_classifier, treelstm_backward_recursive (after a forward with
+ * TREELSTM_SAVE_FOR_BACKWARD, which for these cells keeps nothing beyond h) and treelstm_destroy.
  */
 #define TREELSTM_CELL_TREERNN 1
 #define TREELSTM_CELL_RNTN 2
@@ -255,6 +256,26 @@ TREELSTM_API int treelstm_roots(treelstm_t* ctx, int max_roots, int32_t* root_id
 TREELSTM_API int treelstm_backward(treelstm_t* ctx, const int32_t* labels, float* loss, float* dW, float* db,
                       float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,
                       int32_t* n_touched, void* stream);
+
+/*
+ * treelstm_backward_recursive - the same training step for a context made by
+ * treelstm_create_recursive (TreeRNN or RNTN, Section 6.1), after treelstm_forward(... |
+ * TREELSTM_SAVE_FOR_BACKWARD) on it; treelstm_set_classifier works on such a context as on any other.
+ *   An internal node n with x = [h_l ; h_r] and h_n = tanh(z_n):  dz = dh_n * (1 - h_n^2);
+ *   dW += x (x) dz;  db += dz;  RNTN: dV_j += dz_j * x (x) x;  the children's dh receive
+ *   W dz (+ RNTN: sum_j dz_j (V_j + V_j^T) x);  a leaf's state is its word vector, so its dh is
+ *   added to the gradient row of its token.  Wavefronts in reverse (Section 4.2.2).
+ *   labels, loss, dWc [H][C], dbc [C], touched_ids, n_touched: as for treelstm_backward.
+ *   dW [2H][H], db [H]  out;  dV [H][2H][2H] out (RNTN; may be NULL for TreeRNN);
+ *   dEmb_rows [n_leaves][H] out: one summed row per touched id.
+ * All device pointers; gradients are overwritten.  The level table is read back once (the call
+ * synchronises the stream of the forward if that was a TREELSTM_PERSISTENT one), then one launch per
+ * phase and wavefront; fp32.  Errors: as treelstm_backward; TREELSTM_ERR_STATE on a TreeLSTM context
+ * (and treelstm_backward returns it on a TreeRNN / RNTN context).
+ */
+TREELSTM_API int treelstm_backward_recursive(treelstm_t* ctx, const int32_t* labels, float* loss, float* dW,
+                                             float* db, float* dV, float* dWc, float* dbc, int32_t* touched_ids,
+                                             float* dEmb_rows, int32_t* n_touched, void* stream);
 
 /*
  * treelstm_forward_host - the same forward for callers whose data lives in HOST memory: copies

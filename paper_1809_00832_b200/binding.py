@@ -59,6 +59,7 @@ SIGNATURES = {
     "treelstm_status_sync": (_i, [_vp]),
     "treelstm_roots": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp]),
     "treelstm_backward": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "treelstm_backward_recursive": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "treelstm_forward_host": (_i, [_vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _vp,
                                    _vp, _vp, _i, _vp]),
     "treelstm_host_staging_bytes": (ctypes.c_size_t, [_vp, _i]),
@@ -319,6 +320,31 @@ class TreeLSTM:
         rc = self.lib.treelstm_status_sync(self.handle)
         if rc != OK:
             raise TreeLSTMError(rc, "treelstm_backward (device status)")
+        return out
+
+    def backward_recursive(self, labels: torch.Tensor, n_leaves: int) -> dict:
+        """treelstm_backward_recursive (TreeRNN / RNTN contexts) after forward(..., flags | SAVE_FOR_BACKWARD)."""
+        _dev(labels, torch.int32, "labels")
+        H, C = self.H, self.C
+        f32 = dict(dtype=torch.float32, device="cuda")
+        out = dict(
+            loss=torch.zeros(1, **f32), dW=torch.empty((2 * H, H), **f32), db=torch.empty(H, **f32),
+            dWc=torch.empty((H, C), **f32), dbc=torch.empty(C, **f32),
+            touched_ids=torch.empty(max(n_leaves, 1), dtype=torch.int32, device="cuda"),
+            dEmb_rows=torch.empty((max(n_leaves, 1), H), **f32),
+            n_touched=torch.zeros(1, dtype=torch.int32, device="cuda"),
+        )
+        if self.cell == CELL_RNTN:
+            out["dV"] = torch.empty((H, 2 * H, 2 * H), **f32)
+        rc = self.lib.treelstm_backward_recursive(
+            self.handle, _ptr(labels), _ptr(out["loss"]), _ptr(out["dW"]), _ptr(out["db"]), _ptr(out.get("dV")),
+            _ptr(out["dWc"]), _ptr(out["dbc"]), _ptr(out["touched_ids"]), _ptr(out["dEmb_rows"]),
+            _ptr(out["n_touched"]), _stream())
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_backward_recursive")
+        rc = self.lib.treelstm_status_sync(self.handle)
+        if rc != OK:
+            raise TreeLSTMError(rc, "treelstm_backward_recursive (device status)")
         return out
 
     # -- host-buffer forward ------------------------------------------------------------------

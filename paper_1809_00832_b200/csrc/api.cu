@@ -261,7 +261,7 @@ int treelstm_update_weights(treelstm_t* ctx, const float* emb, const float* W, c
 
 int treelstm_set_classifier(treelstm_t* ctx, int C, const float* Wc, const float* bc, void* stream) {
   if (!ctx || !Wc || !bc || C < 1) return TREELSTM_ERR_INVALID_ARG;
-  if (C > 32 || ctx->cell != 0) return TREELSTM_ERR_UNSUPPORTED;
+  if (C > 32) return TREELSTM_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaFree(ctx->Wc); cudaFree(ctx->bc);
   ctx->Wc = ctx->bc = nullptr; ctx->C = 0;
@@ -333,7 +333,6 @@ int treelstm_forward(treelstm_t* ctx, int n_nodes, const int32_t* left, const in
   if (n_nodes > 0 && (!left || !right || !token || !h || (!c && ctx->cell == 0) || !level || !order))
     return TREELSTM_ERR_INVALID_ARG;
   if (flags & ~(TREELSTM_PERSISTENT | TREELSTM_SAVE_FOR_BACKWARD | TREELSTM_SUBFORESTS)) return TREELSTM_ERR_INVALID_ARG;
-  if (ctx->cell != 0 && (flags & TREELSTM_SAVE_FOR_BACKWARD)) return TREELSTM_ERR_UNSUPPORTED;
   if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return TREELSTM_ERR_INVALID_ARG;
   const bool save = (flags & TREELSTM_SAVE_FOR_BACKWARD) != 0;
   const WsLayout lay = ws_layout(ctx, n_nodes, save);
@@ -431,10 +430,26 @@ int treelstm_backward(treelstm_t* ctx, const int32_t* labels, float* loss, float
     return TREELSTM_ERR_INVALID_ARG;
   if (!ctx->last.valid || !(ctx->last.flags & TREELSTM_SAVE_FOR_BACKWARD) || ctx->C < 1)
     return TREELSTM_ERR_STATE;
+  if (ctx->cell != 0) return TREELSTM_ERR_STATE;   // TreeRNN / RNTN contexts: treelstm_backward_recursive
   if (!on_own_device(ctx)) return TREELSTM_ERR_STATE;
   ctx->launches = 0;
   return launch_backward(ctx, labels, loss, dW, db, dWc, dbc, touched_ids, dEmb_rows, n_touched,
                          static_cast<cudaStream_t>(stream));
+}
+
+int treelstm_backward_recursive(treelstm_t* ctx, const int32_t* labels, float* loss, float* dW, float* db, float* dV,
+                                float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,
+                                int32_t* n_touched, void* stream) {
+  if (!ctx || !labels || !loss || !dW || !db || !dWc || !dbc || !touched_ids || !dEmb_rows || !n_touched)
+    return TREELSTM_ERR_INVALID_ARG;
+  if (ctx->cell == 0) return TREELSTM_ERR_STATE;
+  if (ctx->cell == TREELSTM_CELL_RNTN && !dV) return TREELSTM_ERR_INVALID_ARG;
+  if (!ctx->last.valid || !(ctx->last.flags & TREELSTM_SAVE_FOR_BACKWARD) || ctx->C < 1)
+    return TREELSTM_ERR_STATE;
+  if (!on_own_device(ctx)) return TREELSTM_ERR_STATE;
+  ctx->launches = 0;
+  return launch_backward_rec(ctx, labels, loss, dW, db, dV, dWc, dbc, touched_ids, dEmb_rows, n_touched,
+                             static_cast<cudaStream_t>(stream));
 }
 
 int treelstm_forward_host(treelstm_t* ctx, int n_nodes, const int32_t* left, const int32_t* right,

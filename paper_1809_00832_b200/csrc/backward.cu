@@ -606,4 +606,174 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
   return TREELSTM_OK;
 }
 
+
+// ---- TreeRNN / RNTN: backward through structure ------------------------------------------------ //
+// Section 4.2.2 for the two other evaluation models of Section 6.1, on the same schedule.  An
+// internal node n with x = [h_l ; h_r], p = h_n = tanh(z):
+//     dz   = dh_n * (1 - p^2)
+//     dW  += x (x) dz,  db += dz,  RNTN: dV_j += dz_j * x (x) x
+//     dx   = W dz  (+ RNTN: sum_j dz_j (V_j + V_j^T) x)      -> added to dh of the two children
+// a leaf's state is its word vector: dEmb[token] += dh.  Wavefronts in reverse, one launch per phase
+// and wavefront; plain fp32, one thread per output element - correct and measured, not tuned.
+namespace {
+
+struct RecBwd {
+  int n, H, n_leaves, tensor;
+  const int *left, *right, *token, *order;
+  const float *h, *W, *Vt;     // W [2H][H]; Vt [(a * 2H + b)][j] = V[j][a][b]
+  float *dh, *dz;
+  float *dW, *db, *dV, *dEmb_rows;
+  const int* tok_slot;
+  DevStatus* st;
+};
+
+__global__ void k_rec_bwd_dz(RecBwd p, int begin, int end) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)(end - begin) * p.H) return;
+  const int node = chk(p.st, p.order[begin + (int)(idx / p.H)], p.n), u = (int)(idx % p.H);
+  const float hv = p.h[(size_t)node * p.H + u];
+  p.dz[(size_t)node * p.H + u] = p.dh[(size_t)node * p.H + u] * (1.f - hv * hv);
+}
+
+// one thread per (node of the wavefront, input unit a in [0, 2H)); a child has one caller, so its dh
+// is updated without atomics
+__global__ void k_rec_bwd_dx(RecBwd p, int begin, int end) {
+  const int H = p.H, K = 2 * H;
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)(end - begin) * K) return;
+  const int node = chk(p.st, p.order[begin + (int)(idx / K)], p.n), a = (int)(idx % K);
+  const int l = chk(p.st, p.left[node], p.n), r = chk(p.st, p.right[node], p.n);
+  const float* dz = p.dz + (size_t)node * H;
+  float acc = 0.f;
+  for (int j = 0; j < H; ++j) acc = fmaf(p.W[(size_t)a * H + j], dz[j], acc);
+  if (p.tensor) {
+    const float* hl = p.h + (size_t)l * H;
+    const float* hr = p.h + (size_t)r * H;
+    for (int b = 0; b < K; ++b) {
+      const float xb = b < H ? hl[b] : hr[b - H];
+      const float* vab = p.Vt + ((size_t)a * K + b) * H;
+      const float* vba = p.Vt + ((size_t)b * K + a) * H;
+      float t = 0.f;
+      for (int j = 0; j < H; ++j) t = fmaf(dz[j], vab[j] + vba[j], t);
+      acc = fmaf(t, xb, acc);
+    }
+  }
+  const int child = a < H ? l : r;
+  p.dh[(size_t)child * H + (a < H ? a : a - H)] += acc;
+}
+
+__global__ void k_rec_bwd_leaves(RecBwd p) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)p.n_leaves * p.H) return;
+  const int node = chk(p.st, p.order[(int)(idx / p.H)], p.n), u = (int)(idx % p.H);
+  const int row = p.tok_slot[p.token[node]];
+  atomicAdd(&p.dEmb_rows[(size_t)row * p.H + u], p.dh[(size_t)node * p.H + u]);
+}
+
+// one thread per element of dW [2H][H] (+ db [H] in the threads of row 0): a fixed order of summation
+__global__ void k_rec_bwd_dw(RecBwd p) {
+  const int H = p.H, K = 2 * H;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= K * H) return;
+  const int a = idx / H, j = idx % H;
+  float acc = 0.f, accb = 0.f;
+  for (int pos = p.n_leaves; pos < p.n; ++pos) {
+    const int node = p.order[pos];
+    const int child = a < H ? p.left[node] : p.right[node];
+    const float dzj = p.dz[(size_t)node * H + j];
+    acc = fmaf(p.h[(size_t)child * H + (a < H ? a : a - H)], dzj, acc);
+    accb += dzj;
+  }
+  p.dW[idx] = acc;
+  if (a == 0) p.db[j] = accb;
+}
+
+// one thread per element of dV [H][2H][2H]
+__global__ void k_rec_bwd_dv(RecBwd p) {
+  const int H = p.H, K = 2 * H;
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)H * K * K) return;
+  const int j = (int)(idx / ((long long)K * K)), a = (int)((idx / K) % K), b = (int)(idx % K);
+  float acc = 0.f;
+  for (int pos = p.n_leaves; pos < p.n; ++pos) {
+    const int node = p.order[pos];
+    const int l = p.left[node], r = p.right[node];
+    const float xa = a < H ? p.h[(size_t)l * H + a] : p.h[(size_t)r * H + a - H];
+    const float xb = b < H ? p.h[(size_t)l * H + b] : p.h[(size_t)r * H + b - H];
+    acc = fmaf(p.dz[(size_t)node * H + j], xa * xb, acc);
+  }
+  p.dV[idx] = acc;
+}
+
+}  // namespace
+
+int launch_backward_rec(treelstm* ctx, const int32_t* labels, float* loss, float* dW, float* db, float* dV,
+                        float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows, int32_t* n_touched,
+                        cudaStream_t stream) {
+  auto& L = ctx->last;
+  L.stream = stream;
+  int rc = ensure_host_levels(ctx);      // one read of the level table (a persistent forward left it on the device)
+  if (rc != TREELSTM_OK) return rc;
+  const int n = L.n, H = ctx->H, C = ctx->C, n_levels = L.n_levels;
+  const bool tensor = ctx->cell == TREELSTM_CELL_RNTN;
+  const int32_t* off = ctx->host_level_offset;
+  const size_t K = 2 * (size_t)H;
+  TL_CUDA(ctx, cudaMemsetAsync(loss, 0, sizeof(float), stream));
+  TL_CUDA(ctx, cudaMemsetAsync(dW, 0, sizeof(float) * K * H, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(db, 0, sizeof(float) * H, stream));
+  if (tensor) TL_CUDA(ctx, cudaMemsetAsync(dV, 0, sizeof(float) * H * K * K, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(dWc, 0, sizeof(float) * H * C, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(dbc, 0, sizeof(float) * C, stream));
+  TL_CUDA(ctx, cudaMemsetAsync(n_touched, 0, sizeof(int), stream));
+  if (n == 0 || n_levels == 0) return TREELSTM_OK;
+  char* base = static_cast<char*>(L.ws);
+  const int n_leaves = off[1];
+  // the classifier, the loss and the touched-token bookkeeping are the TreeLSTM path's kernels
+  BwdParams p{};
+  p.n = n; p.H = H; p.E = H; p.C = C; p.vocab = ctx->vocab; p.n_leaves = n_leaves;
+  p.left = L.left; p.right = L.right; p.token = L.token; p.order = L.order; p.labels = labels;
+  p.Wc = ctx->Wc; p.bc = ctx->bc; p.h = L.h;
+  p.dh = reinterpret_cast<float*>(base + L.lay.dh);
+  p.dz = reinterpret_cast<float*>(base + L.lay.dz);
+  p.loss = loss; p.dWc = dWc; p.dbc = dbc; p.dEmb_rows = dEmb_rows;
+  p.tok_slot = reinterpret_cast<int*>(base + L.lay.tok_slot);
+  p.touched_ids = touched_ids; p.n_touched = n_touched;
+  p.st = reinterpret_cast<DevStatus*>(base + L.lay.status);
+  const size_t cls_smem = sizeof(float) * ((size_t)H * C + C);
+  if (cls_smem > 160 * 1024) return TREELSTM_ERR_UNSUPPORTED;
+  TL_CUDA(ctx, cudaMemsetAsync(p.tok_slot, 0, sizeof(int) * ((size_t)ctx->vocab + 1), stream));
+  TL_CUDA(ctx, cudaMemsetAsync(dEmb_rows, 0, sizeof(float) * (size_t)n_leaves * H, stream));
+  k_bwd_mark_tokens<<<(n_leaves + 255) / 256, 256, 0, stream>>>(p);
+  k_bwd_scan_tokens<<<1, 1024, 0, stream>>>(p);
+  if (cls_smem > 48 * 1024)
+    TL_CUDA(ctx, cudaFuncSetAttribute(k_bwd_classifier, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cls_smem));
+  k_bwd_classifier<<<(n + kClsNodesPerCta - 1) / kClsNodesPerCta, kClsWarps * 32, cls_smem, stream>>>(p);
+  ctx->launches += 3;
+
+  RecBwd q{};
+  q.n = n; q.H = H; q.n_leaves = n_leaves; q.tensor = tensor ? 1 : 0;
+  q.left = L.left; q.right = L.right; q.token = L.token; q.order = L.order;
+  q.h = L.h; q.Vt = ctx->Wcat; q.W = ctx->Wcat + (tensor ? K * K * H : 0);
+  q.dh = p.dh; q.dz = p.dz; q.dW = dW; q.db = db; q.dV = dV; q.dEmb_rows = dEmb_rows; q.tok_slot = p.tok_slot; q.st = p.st;
+  for (int lvl = n_levels - 1; lvl >= 1; --lvl) {
+    const int begin = off[lvl], end = off[lvl + 1];
+    const long long e1 = (long long)(end - begin) * H, e2 = (long long)(end - begin) * (long long)K;
+    k_rec_bwd_dz<<<(unsigned)((e1 + 255) / 256), 256, 0, stream>>>(q, begin, end);
+    k_rec_bwd_dx<<<(unsigned)((e2 + 127) / 128), 128, 0, stream>>>(q, begin, end);
+    ctx->launches += 2;
+  }
+  k_rec_bwd_leaves<<<(unsigned)(((long long)n_leaves * H + 255) / 256), 256, 0, stream>>>(q);
+  ctx->launches += 1;
+  if (n > n_leaves) {
+    k_rec_bwd_dw<<<(unsigned)((K * H + 127) / 128), 128, 0, stream>>>(q);
+    ctx->launches += 1;
+    if (tensor) {
+      k_rec_bwd_dv<<<(unsigned)((H * K * K + 127) / 128), 128, 0, stream>>>(q);
+      ctx->launches += 1;
+    }
+  }
+  TL_CUDA(ctx, cudaGetLastError());
+  return TREELSTM_OK;
+}
+
 }  // namespace tl

@@ -221,6 +221,10 @@ int launch_forward_bf16_tail(treelstm* ctx, int n, const int32_t* left, const in
 int launch_selftest_waits(treelstm* ctx, void* ws, int* result_dev, cudaStream_t stream);
 
 // backward.cu
+int launch_backward_rec(treelstm* ctx, const int32_t* labels, float* loss, float* dW, float* db, float* dV,
+                        float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows, int32_t* n_touched,
+                        cudaStream_t stream);
+int ensure_host_levels(treelstm* ctx);
 int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW, float* db,
                     float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,
                     int32_t* n_touched, cudaStream_t stream);
