@@ -113,7 +113,7 @@ typedef enum treelstm_status {
                                             /* forest had no tail worth handing over; the grid-wide kernel */
                                             /* keeps recording what the decision would have been, and the  */
                                             /* launch comes back with the first forest that has one        */
-#define TREELSTM_OPT_OVERLAP_LAUNCH 8       /* 1 (default): the persistent bf16 wavefront kernel is        */
+#define TREELSTM_OPT_OVERLAP_LAUNCH 8       /* 1 (default): the persistent wavefront kernel (bf16, fp32) is */
                                             /* launched as a programmatic dependent of the ready-set       */
                                             /* construction, so that its set-up (barriers, tensor memory,  */
                                             /* weights and biases asked into L2) runs while that kernel    */

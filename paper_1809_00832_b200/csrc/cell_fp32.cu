@@ -27,6 +27,7 @@ struct FwdParams {
   DevStatus* st;
   long long wait_limit;
   int w_stationary, a_row, w_row;   // persistent kernel: W_h slice resident in shared memory; row strides (floats)
+  int early_start = 0;              // persistent kernel: launched under the scheduler, waits for it on the device
 };
 
 __device__ __forceinline__ float sigmoidf_acc(float x) { return 1.0f / (1.0f + expf(-x)); }
@@ -328,11 +329,16 @@ k_fwd_fp32_persistent(FwdParams p) {
   int* s_node = reinterpret_cast<int*>(red + (p.w_stationary ? 4 * TMS * 5 * TU : 0));
   int* s_l = s_node + TM;
   int* s_r = s_l + TM;
-  if (ld_volatile(&p.st->status) != 0) return;
-  const int n_levels = p.st->n_levels;
   const int tiles_u = (p.H + TU - 1) / TU;
   const int H = p.H;
-  if (p.w_stationary && n_levels > 1) {
+  // Launched as a programmatic dependent of the ready-set construction (p.early_start), the kernel
+  // gets here while that one still runs: the weight slice needs nothing from it and is fetched first.
+  int n_levels = 0;
+  if (!p.early_start) {
+    if (ld_volatile(&p.st->status) != 0) return;
+    n_levels = p.st->n_levels;
+  }
+  if (p.w_stationary && (p.early_start || n_levels > 1)) {
     // The grid is a multiple of tiles_u, so tile t of any level, t = blockIdx.x + i * gridDim.x, has
     // the same hidden-unit slice: its rows of W_h are fetched once, transposed to [column][k].
     const int u0 = (blockIdx.x % tiles_u) * TU, K = 2 * H, w_row = p.w_row;
@@ -343,6 +349,11 @@ k_fwd_fp32_persistent(FwdParams p) {
       if (k < K && u0 + uu < H) v = __ldg(Wk + (size_t)k * 5 * H + g * H + u0 + uu);
       Ws[col * w_row + k] = v;
     }
+  }
+  if (p.early_start) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (ld_volatile(&p.st->status) != 0) return;
+    n_levels = p.st->n_levels;
   }
   // the first wavefront boundaries in shared memory: no dependent global load after every barrier
   constexpr int kOffCache = 256;
@@ -439,15 +450,27 @@ int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t
     int per_sm = 0;
     TL_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_fwd_fp32_persistent,
                                                                kThreads, smem));
-    int grid = per_sm * ctx->sm_count;
+    // Started under the single-CTA scheduler (see launch_forward_bf16 for the two ways to launch a
+    // kernel with a grid barrier): the scheduler keeps its SM.
+    const int single_max = ctx->opt.sched_single_cta_max < kSchedSingleMaxNodes ? ctx->opt.sched_single_cta_max : kSchedSingleMaxNodes;
+    const bool overlap = ctx->opt.overlap_launch && n <= single_max && per_sm >= 1 && ctx->sm_count > 1;
+    p.early_start = overlap ? 1 : 0;
+    int grid = per_sm * (overlap ? ctx->sm_count - 1 : ctx->sm_count);
     const int want = ((n + TMS - 1) / TMS + 1) * tiles_u;   // never more CTAs than the widest level has tiles
     if (grid > want) grid = want;
     if (grid > cap) grid = cap;
     if (p.w_stationary) grid = grid / tiles_u * tiles_u;    // every CTA keeps one hidden-unit slice
     if (grid < 1) grid = 1;
-    void* args[] = {&p};
-    TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_fwd_fp32_persistent, dim3(grid), dim3(kThreads),
-                                             args, smem, stream));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    if (overlap) {
+      attr.id = cudaLaunchAttributeProgrammaticStreamSerialization; attr.val.programmaticStreamSerializationAllowed = 1;
+    } else {
+      attr.id = cudaLaunchAttributeCooperative; attr.val.cooperative = 1;
+    }
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    TL_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_fwd_fp32_persistent, p));
     ctx->launches += 1;
     return TREELSTM_OK;
   }
