@@ -29,6 +29,7 @@ struct BwdParams {
   float *loss, *dW, *db, *dWc, *dbc, *dEmb_rows;
   int *tok_slot, *touched_ids, *n_touched;
   DevStatus* st;
+  long long* trace;   // cycle stamps of the one-launch backward (trace builds), else nullptr
 };
 
 // ---- touched embedding rows: flag, scan, compact ------------------------------------------- //
@@ -42,48 +43,40 @@ __global__ void k_bwd_mark_tokens(BwdParams p) {
 // ascending order and tok_slot[id] becomes the row index of id in dEmb_rows.
 __device__ void scan_tokens(const BwdParams& p) {   // one CTA of any size that is a multiple of 32
   __shared__ int warp_sum[32];
-  __shared__ int carry;
-  constexpr int kPer = 8;                            // consecutive ids per thread and trip: fewer CTA barriers
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nw = nt >> 5;
-  if (tid == 0) carry = 0;
-  __syncthreads();
-  for (int base = 0; base < p.vocab; base += nt * kPer) {
-    const int i0 = base + tid * kPer;
-    int v[kPer], sum = 0;
+  // Two passes over a contiguous range of ids per thread: count, one scan over the threads, then write.
+  // (A running scan over blocks of ids made every block wait for the loads of the one before: 3.6 k
+  // cycles per 2048 ids.)
+  const int per = (p.vocab + nt - 1) / nt;
+  const int lo = min(p.vocab, tid * per), hi = min(p.vocab, lo + per);
+  int sum = 0;
+  for (int i = lo; i < hi; ++i) sum += p.tok_slot[i];
+  int incl = sum;
 #pragma unroll
-    for (int j = 0; j < kPer; ++j) { v[j] = i0 + j < p.vocab ? p.tok_slot[i0 + j] : 0; sum += v[j]; }
-    int incl = sum;
+  for (int d = 1; d < 32; d <<= 1) {
+    int t = __shfl_up_sync(kFull, incl, d);
+    if (lane >= d) incl += t;
+  }
+  if (lane == 31) warp_sum[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = lane < nw ? warp_sum[lane] : 0, wi = w;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
-      int t = __shfl_up_sync(kFull, incl, d);
-      if (lane >= d) incl += t;
+      int t = __shfl_up_sync(kFull, wi, d);
+      if (lane >= d) wi += t;
     }
-    if (lane == 31) warp_sum[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-      int w = lane < nw ? warp_sum[lane] : 0, wi = w;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        int t = __shfl_up_sync(kFull, wi, d);
-        if (lane >= d) wi += t;
-      }
-      warp_sum[lane] = wi - w;
-    }
-    __syncthreads();
-    int excl = carry + warp_sum[warp] + incl - sum;
-#pragma unroll
-    for (int j = 0; j < kPer; ++j) {
-      if (i0 + j < p.vocab) {
-        p.tok_slot[i0 + j] = excl;
-        if (v[j]) p.touched_ids[excl] = i0 + j;
-      }
-      excl += v[j];
-    }
-    __syncthreads();
-    if (tid == nt - 1) carry = excl;
-    __syncthreads();
+    warp_sum[lane] = wi - w;
   }
-  if (tid == 0) { *p.n_touched = carry; p.st->n_touched = carry; }
+  __syncthreads();
+  int excl = warp_sum[warp] + incl - sum;
+  for (int i = lo; i < hi; ++i) {
+    const int v = p.tok_slot[i];
+    p.tok_slot[i] = excl;
+    if (v) p.touched_ids[excl] = i;
+    excl += v;
+  }
+  if (tid == nt - 1) { *p.n_touched = excl; p.st->n_touched = excl; }
 }
 __global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) { scan_tokens(p); }
 
@@ -91,7 +84,7 @@ __global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) { scan_to
 // One warp per node: the lanes share the contraction over h (lane j takes units j, j + 32, ...),
 // a butterfly sum gives every lane all logits, lane k keeps class k (C <= 32).
 constexpr int kClsWarps = 8;
-constexpr int kClsNodesPerCta = 16;
+constexpr int kClsNodesPerCta = 8;    // one node per warp and group: the chains of dependent loads of a node are long
 
 // The CTA takes the node groups vb_first, vb_first + vb_step, ...; s_dWc [H][C] + [C] collects its partial sums.
 __device__ void classifier_groups(const BwdParams& p, int vb_first, int vb_step, float* s_dWc) {
@@ -144,6 +137,7 @@ __device__ void classifier_groups(const BwdParams& p, int vb_first, int vb_step,
     }
   }
   __syncthreads();
+  if (vb_first >= n_groups) return;   // a CTA without a group has nothing to add (and 300 CTAs adding zeros to the same H x C words queue up)
   for (int i = tid; i < H * C; i += blockDim.x) atomicAdd(&p.dWc[i], s_dWc[i]);
   for (int i = tid; i < C; i += blockDim.x) atomicAdd(&p.dbc[i], s_dWc[H * C + i]);
 }
@@ -445,6 +439,12 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
   if (ld_volatile(&p.st->status) != 0) return;
   const int n_levels = p.st->n_levels;
   const int n = p.n, H = p.H, E = p.E, C = p.C, J = 5 * H;
+#ifdef TREELSTM_TRACE
+  // first CTA, first thread: row l of the stamp table = wavefront l (slot 0 start, 1 gate gradients done,
+  // 2 barrier, 3 input gradients done, 4 barrier); last row = phases of the kernel
+  long long* const trace = blockIdx.x == 0 && threadIdx.x == 0 ? p.trace : nullptr;
+#endif
+  TL_STAMP(trace, kTraceLevels - 1, 0);
   p.n_leaves = n_levels > 0 ? level_offset[1] : 0;
   const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, gthreads = (size_t)gridDim.x * blockDim.x;
   unsigned int arrivals = 0;
@@ -461,9 +461,11 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
   zero_range(p.tok_slot, (size_t)p.vocab + 1, gtid, gthreads);
   zero_range(p.dEmb_rows, (size_t)p.n_leaves * E, gtid, gthreads);
   if (!barrier()) return;
+  TL_STAMP(trace, kTraceLevels - 1, 1);   // outputs and scratch cleared
   for (size_t r = gtid; r < (size_t)p.n_leaves; r += gthreads)
     p.tok_slot[chk(p.st, p.token[chk(p.st, p.order[r], p.n)], p.vocab)] = 1;
   if (!barrier()) return;
+  TL_STAMP(trace, kTraceLevels - 1, 2);   // tokens marked
   if (gridDim.x == 1) {
     scan_tokens(p);
     classifier_groups(p, 0, 1, s_cls);
@@ -472,7 +474,9 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
   } else {
     classifier_groups(p, blockIdx.x - 1, gridDim.x - 1, s_cls);
   }
+  TL_STAMP(trace, kTraceLevels - 1, 3);   // this CTA's part (the first one: the token scan) done
   if (!barrier()) return;
+  TL_STAMP(trace, kTraceLevels - 1, 4);   // classifier, loss and token scan done everywhere
   // the first wavefront boundaries in shared memory: no dependent global load after every barrier
   // (filled here, ordered before its first use by the CTA barriers inside the grid barrier above)
   constexpr int kOffCache = 256;
@@ -483,13 +487,19 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
   for (int lvl = n_levels - 1; lvl >= 0; --lvl) {
     const int begin = level_begin(lvl), end = level_begin(lvl + 1), leaf = lvl == 0 ? 1 : 0;
     const long long elems = (long long)(end - begin) * H;
+    TL_STAMP(trace, lvl, 0);
     for (long long idx = (long long)gtid; idx < elems; idx += (long long)gthreads) gates_element(p, begin, idx, leaf);
+    TL_STAMP(trace, lvl, 1);
     if (!barrier()) return;
+    TL_STAMP(trace, lvl, 2);
     const int tiles = dinput_tiles(end - begin, leaf ? E : 2 * H), splits = dinput_splits(tiles, J);
     for (int vb = blockIdx.x; vb < tiles * splits; vb += gridDim.x)
       dinput_block(p, begin, end, leaf, vb % tiles, vb / tiles, splits, sm.di);
+    TL_STAMP(trace, lvl, 3);
     if (lvl > 0 && !barrier()) return;   // the leaves' dIn goes to the embedding rows only
+    TL_STAMP(trace, lvl, 4);
   }
+  TL_STAMP(trace, kTraceLevels - 1, 5);   // all wavefronts done
   const int tiles_j = (J + BT - 1) / BT, rows_per_split = kDwRows;
   for (int part = 0; part < 2; ++part) {
     const int begin = part == 0 ? 0 : p.n_leaves, end = part == 0 ? p.n_leaves : n;
@@ -498,10 +508,12 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
     const int nbx = ((K + BT - 1) / BT) * tiles_j, nby = (end - begin + rows_per_split - 1) / rows_per_split;
     for (int vb = blockIdx.x; vb < nbx * nby; vb += gridDim.x)
       dweight_block(p, part, begin, end, rows_per_split, vb % nbx, vb / nbx, sm.dw);
+    TL_STAMP(trace, kTraceLevels - 1, 6 + part);   // this CTA's blocks of dW from the leaves / the internal nodes done
   }
   const int nby = (n + 255) / 256;
   for (long long idx = (long long)gtid; idx < (long long)J * nby; idx += (long long)gthreads)
     dbias_piece(p, (int)(idx % J), (int)(idx / J));
+  TL_STAMP(trace, kTraceLevels - 1, 8);
 }
 
 }  // namespace
@@ -532,6 +544,11 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
   p.tok_slot = reinterpret_cast<int*>(base + L.lay.tok_slot);
   p.touched_ids = touched_ids; p.n_touched = n_touched;
   p.st = reinterpret_cast<DevStatus*>(base + L.lay.status);
+  p.trace = nullptr;
+#ifdef TREELSTM_TRACE
+  p.trace = reinterpret_cast<long long*>(base + L.lay.trace);   // the forward's table: an fp32 forward leaves it unused
+  TL_CUDA(ctx, cudaMemsetAsync(p.trace, 0, sizeof(long long) * kTraceSlots * kTraceLevels, stream));
+#endif
 
   const size_t J = 5 * (size_t)H;
   const size_t cls_smem = sizeof(float) * ((size_t)H * C + C);

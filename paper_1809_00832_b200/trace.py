@@ -24,6 +24,9 @@ Cluster kernel of the narrow tail (k_fwd_tc_tail), stamps of different warps of 
   s9  older child cell states are in      s5  cell updates done
   s10 new h complete in shared memory     s11 every peer's prefetch has landed (pushes may go)
   s6  pushes issued
+One-launch backward (--train: train25_fp32, fp32 forward + k_bwd_persistent), first CTA, per wavefront in
+reverse: s0 start, s1 gate gradients done, s2 barrier, s3 input gradients done, s4 barrier; and the
+phases of the kernel.
 The sub-forest kernel (--mode subforests) uses s0 start, s1 first operand request, s2 first box seen by
 the MMA issuer, s3 last MMAs committed, s4 epilogue starts waiting, s5 last tile stored, s6 arrival at
 the cluster barrier, s7 barrier left.  The stamps cost a few cycles each; the normal build is a little
@@ -53,6 +56,35 @@ def read_trace(model: binding.TreeLSTM, which: int) -> np.ndarray:
     return np.frombuffer(buf, dtype=np.int64).reshape(LEVELS, SLOTS).copy()
 
 
+def trace_training_step() -> int:
+    w = fg.make_workload("train25_fp32", 0)
+    f, p = w.forest, w.params
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    model = binding.TreeLSTM(p.H, p.E, p.vocab, dev(p.emb), dev(p.W), dev(p.b), binding.FP32, variant="trace")
+    model.set_classifier(dev(p.Wc), dev(p.bc))
+    left, right, token, labels = dev(f.left), dev(f.right), dev(f.token), dev(w.labels)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for i in range(4):
+        flush.fill_(i)
+        out = model.forward(left, right, token, flags=binding.PERSISTENT | binding.SAVE_FOR_BACKWARD)
+        model.backward(labels, f.n_leaves)
+    torch.cuda.synchronize()
+    widths = np.diff(out["level_offset"].cpu().numpy()[:int(out["n_levels"].item()) + 1])
+    t = read_trace(model, 0)
+    ph = t[LEVELS - 1]
+    names = ("outputs and scratch cleared", "tokens marked", "own part of token scan / classifier done",
+             "classifier, loss, token scan done everywhere", "all wavefronts done", "dW from the leaves (own blocks)",
+             "dW from the internal nodes (own blocks)", "db done")
+    print("# one-launch backward, first CTA, cycles since its start: " +
+          ", ".join(f"{nm} {int(ph[i + 1] - ph[0])}" for i, nm in enumerate(names) if ph[i + 1]))
+    print("level width gates_done barrier dinput_done barrier   (cycles since the wavefront's start; wavefronts run in reverse)")
+    for l in range(len(widths) - 1, -1, -1):
+        if t[l, 0] == 0:
+            continue
+        print(f"{l:<5d} {int(widths[l]):<5d} " + " ".join(f"{(t[l, k] - t[l, 0]) if t[l, k] else 0:<10d}" for k in range(1, 5)))
+    return 0
+
+
 def main() -> int:
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="batch256_bf16", choices=[w for w in fg.WORKLOADS if w.endswith("bf16")])
@@ -61,10 +93,13 @@ def main() -> int:
     ap.add_argument("--tail-min-levels", type=int, default=None)
     ap.add_argument("--trees", type=int, default=None)
     ap.add_argument("--levels", default=None, help="A:B - print only wavefronts A..B-1")
+    ap.add_argument("--train", action="store_true", help="trace the one-launch backward of a training step on train25_fp32")
     ap.add_argument("--plain-order", action="store_true",
                     help="launch the grid-wide kernel cooperatively behind the scheduler instead of under it")
     args = ap.parse_args()
     build.build(variant="trace")
+    if args.train:
+        return trace_training_step()
     w = fg.make_workload(args.workload, 0, args.trees)
     f, p = w.forest, w.params
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
