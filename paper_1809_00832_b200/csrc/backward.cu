@@ -28,6 +28,7 @@ struct BwdParams {
   float *dh, *dc, *dz;
   float *loss, *dW, *db, *dWc, *dbc, *dEmb_rows;
   int *tok_slot, *touched_ids, *n_touched;
+  int *pos_left, *pos_right;   // children of the node at every ready position (one-launch backward; scheduler scratch reused)
   DevStatus* st;
   long long* trace;   // cycle stamps of the one-launch backward (trace builds), else nullptr
 };
@@ -40,25 +41,49 @@ __global__ void k_bwd_mark_tokens(BwdParams p) {
 }
 
 // Exclusive scan of the flags over the vocabulary by one CTA; flagged ids are emitted in
-// ascending order and tok_slot[id] becomes the row index of id in dEmb_rows.
-__device__ void scan_tokens(const BwdParams& p) {   // one CTA of any size that is a multiple of 32
+// ascending order and tok_slot[id] becomes the row index of id in dEmb_rows.  A warp takes a
+// contiguous run of 128-id groups: lane l holds ids 4 l .. 4 l + 3 of a group (one 16-byte load,
+// eight groups in flight), four ballots per group (component c of every lane) kept in shared memory
+// (s_mask, mask_cap words; groups beyond that are read again), a scan over the warps' counts, then
+// a second pass that only stores.
+// flags of ids id .. id + 3 (id a multiple of 4), zeros beyond the vocabulary or where `take` is false.  No
+// branch: the compiler can then keep the loads of a batch in flight together.  The table has three
+// spare entries behind its vocab + 1, so the last quad may be read whole.
+__device__ __forceinline__ int4 load_flags4(const BwdParams& p, int id, bool take) {
+  const int last_quad = ((p.vocab - 1) >> 2) << 2;
+  int4 v = *reinterpret_cast<const int4*>(p.tok_slot + min(id, last_quad));
+  v.x = take && id < p.vocab ? v.x : 0;
+  v.y = take && id + 1 < p.vocab ? v.y : 0;
+  v.z = take && id + 2 < p.vocab ? v.z : 0;
+  v.w = take && id + 3 < p.vocab ? v.w : 0;
+  return v;
+}
+__device__ void scan_tokens(const BwdParams& p, unsigned int* s_mask, int mask_cap) {   // blockDim a multiple of 32
   __shared__ int warp_sum[32];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nw = nt >> 5;
-  // Two passes over a contiguous range of ids per thread: count, one scan over the threads, then write.
-  // (A running scan over blocks of ids made every block wait for the loads of the one before: 3.6 k
-  // cycles per 2048 ids.)
-  const int per = (p.vocab + nt - 1) / nt;
-  const int lo = min(p.vocab, tid * per), hi = min(p.vocab, lo + per);
-  int sum = 0;
-  for (int i = lo; i < hi; ++i) sum += p.tok_slot[i];
-  int incl = sum;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
+  const int n_groups = (p.vocab + 127) / 128, per = (n_groups + nw - 1) / nw;
+  const int g_lo = min(n_groups, warp * per), g_hi = min(n_groups, g_lo + per);
+  constexpr int kBatch = 8;
+  int count = 0;
+  for (int g0 = g_lo; g0 < g_hi; g0 += kBatch) {
+    int4 v[kBatch];
 #pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    int t = __shfl_up_sync(kFull, incl, d);
-    if (lane >= d) incl += t;
+    for (int b = 0; b < kBatch; ++b)
+      v[b] = load_flags4(p, (g0 + b) * 128 + 4 * lane, g0 + b < g_hi);
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      const unsigned int m0 = __ballot_sync(kFull, v[b].x != 0), m1 = __ballot_sync(kFull, v[b].y != 0);
+      const unsigned int m2 = __ballot_sync(kFull, v[b].z != 0), m3 = __ballot_sync(kFull, v[b].w != 0);
+      if (g0 + b < g_hi) {
+        if (4 * (g0 + b) + 3 < mask_cap && lane < 4) s_mask[4 * (g0 + b) + lane] = lane == 0 ? m0 : (lane == 1 ? m1 : (lane == 2 ? m2 : m3));
+        count += __popc(m0) + __popc(m1) + __popc(m2) + __popc(m3);
+      }
+    }
   }
-  if (lane == 31) warp_sum[warp] = incl;
+  if (lane == 0) warp_sum[warp] = count;
+  TL_STAMP(tid == 0 ? p.trace : nullptr, kTraceLevels - 1, 9);    // first warp: flags read
   __syncthreads();
+  TL_STAMP(tid == 0 ? p.trace : nullptr, kTraceLevels - 1, 10);   // all warps: flags read
   if (warp == 0) {
     int w = lane < nw ? warp_sum[lane] : 0, wi = w;
 #pragma unroll
@@ -69,16 +94,43 @@ __device__ void scan_tokens(const BwdParams& p) {   // one CTA of any size that 
     warp_sum[lane] = wi - w;
   }
   __syncthreads();
-  int excl = warp_sum[warp] + incl - sum;
-  for (int i = lo; i < hi; ++i) {
-    const int v = p.tok_slot[i];
-    p.tok_slot[i] = excl;
-    if (v) p.touched_ids[excl] = i;
-    excl += v;
+  int base = warp_sum[warp];
+  const unsigned int below = (1u << lane) - 1u;
+  for (int g = g_lo; g < g_hi; ++g) {
+    const int id = g * 128 + 4 * lane;
+    unsigned int m0, m1, m2, m3;
+    if (4 * g + 3 < mask_cap) {
+      const uint4 m = *reinterpret_cast<const uint4*>(s_mask + 4 * g);
+      m0 = m.x; m1 = m.y; m2 = m.z; m3 = m.w;
+    } else {
+      const int4 v = load_flags4(p, id, true);
+      m0 = __ballot_sync(kFull, v.x != 0); m1 = __ballot_sync(kFull, v.y != 0);
+      m2 = __ballot_sync(kFull, v.z != 0); m3 = __ballot_sync(kFull, v.w != 0);
+    }
+    // ids ascend lane by lane, component by component
+    const int f0 = (m0 >> lane) & 1u, f1 = (m1 >> lane) & 1u, f2 = (m2 >> lane) & 1u, f3 = (m3 >> lane) & 1u;
+    const int e0 = base + __popc(m0 & below) + __popc(m1 & below) + __popc(m2 & below) + __popc(m3 & below);
+    const int e1 = e0 + f0, e2 = e1 + f1, e3 = e2 + f2;
+    if (id + 3 < p.vocab) {
+      *reinterpret_cast<int4*>(p.tok_slot + id) = make_int4(e0, e1, e2, e3);
+    } else {
+      if (id < p.vocab) p.tok_slot[id] = e0;
+      if (id + 1 < p.vocab) p.tok_slot[id + 1] = e1;
+      if (id + 2 < p.vocab) p.tok_slot[id + 2] = e2;
+    }
+    if (f0) p.touched_ids[e0] = id;       // a set flag implies id < vocab: flags beyond it were read as 0
+    if (f1) p.touched_ids[e1] = id + 1;
+    if (f2) p.touched_ids[e2] = id + 2;
+    if (f3) p.touched_ids[e3] = id + 3;
+    base += __popc(m0) + __popc(m1) + __popc(m2) + __popc(m3);
   }
-  if (tid == nt - 1) { *p.n_touched = excl; p.st->n_touched = excl; }
+  if (warp == nw - 1 && lane == 0) { *p.n_touched = base; p.st->n_touched = base; }
 }
-__global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) { scan_tokens(p); }
+constexpr int kScanMaskWords = 8192;
+__global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) {
+  __shared__ __align__(16) unsigned int s_mask[kScanMaskWords];
+  scan_tokens(p, s_mask, kScanMaskWords);
+}
 
 // ---- classifier: logits, softmax, loss, dlogits, dh (classifier part), dWc, dbc -------------- //
 // One warp per node: the lanes share the contraction over h (lane j takes units j, j + 32, ...),
@@ -191,6 +243,7 @@ struct DinputSmem {
   __align__(16) float Bs[2][BT][kDiRow];
   int node[BT];
   int dst_a[BT], dst_b[BT];   // where a row's dIn goes: left / right child, or (leaves) its row of dEmb_rows
+  int fnode[2][BT], fleft[2][BT], fright[2][BT];   // the same for the blocks of dinput_fused: two sets used in turn
 };
 __device__ void dinput_block(const BwdParams& p, int row_begin, int row_end, int leaf, int bx, int by, int nby,
                              DinputSmem& sm) {
@@ -298,6 +351,178 @@ __global__ void __launch_bounds__(256)
 k_bwd_dinput(BwdParams p, int row_begin, int row_end, int leaf) {
   __shared__ DinputSmem sm;
   dinput_block(p, row_begin, row_end, leaf, blockIdx.x, blockIdx.y, gridDim.y, sm);
+}
+
+// ---- narrow internal wavefronts of the one-launch backward: gate gradients inside the contraction -- //
+// A block of dIn = dz W^T forms the dz values of its chunk itself instead of reading them back, so a
+// narrow wavefront needs neither a pass of its own for the gate gradients nor the grid barrier behind
+// it.  What does not depend on the wavefront above - the rows' index triples (node, left, right; kept
+// by position in pos_left / pos_right, filled once at the start) and the weight chunk - is asked for
+// with cp.async before the CTA enters the grid barrier and lands in shared memory while it waits;
+// after the barrier one round of loads brings dh, dc (just written by the wavefront above) together
+// with the forward's gate activations and cell states.  Same expressions as gates_element.  The
+// blocks of the first output tile (k0 == 0) also store dz for the dW contraction and hand dc to the
+// children; every (node, gate column) belongs to exactly one of them.
+struct FusedItem {
+  int row0, rows, k0, c_lo, chunks;   // first row (position in the ready order), valid rows, first output, chunk range
+};
+__device__ __forceinline__ FusedItem fused_item(const BwdParams& p, int row_begin, int row_end, int bx, int by, int nby) {
+  const int K = 2 * p.H, J = 5 * p.H;
+  const int tiles_k = (K + BT - 1) / BT;
+  const int chunks_all = (J + BK - 1) / BK, per_split = (chunks_all + nby - 1) / nby;
+  FusedItem it;
+  it.row0 = row_begin + (bx / tiles_k) * BT;
+  it.rows = min(BT, row_end - it.row0);
+  it.k0 = (bx % tiles_k) * BT;
+  it.c_lo = by * per_split;
+  it.chunks = min(chunks_all, it.c_lo + per_split);
+  return it;
+}
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* src, bool valid) {
+  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  const uint32_t bytes = valid ? 4u : 0u;   // 0: the word is filled with zeros, the source is not read
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+// index triples of the block's rows into set `ib` (asynchronous)
+__device__ __forceinline__ void fused_request_indices(const BwdParams& p, const FusedItem& it, DinputSmem& sm, int ib) {
+  const int t = threadIdx.x;
+  if (t < 3 * BT) {
+    const int which = t / BT, i = t % BT;
+    const bool valid = i < it.rows;
+    const int pos = valid ? it.row0 + i : 0;
+    const int* src = which == 0 ? p.order + pos : (which == 1 ? p.pos_left + pos : p.pos_right + pos);
+    int* dst = which == 0 ? &sm.fnode[ib][i] : (which == 1 ? &sm.fleft[ib][i] : &sm.fright[ib][i]);
+    cp_async4(dst, src, valid);
+  }
+}
+// weight chunk j0 of the block into operand buffer `buf` (asynchronous)
+__device__ __forceinline__ void fused_request_weights(const BwdParams& p, const FusedItem& it, DinputSmem& sm, int buf, int j0) {
+  const int J = 5 * p.H, K = 2 * p.H, tid = threadIdx.x;
+#pragma unroll
+  for (int q = 0; q < kLd; ++q) {
+    const int e = tid + q * 256, i = e / BK, j = j0 + e % BK;
+    const bool valid = it.k0 + i < K && j < J;
+    cp_async4(&sm.Bs[buf][i][e % BK], p.W + (valid ? (size_t)(p.E + it.k0 + i) * J + j : 0), valid);
+  }
+}
+__device__ __forceinline__ int gate_of_column(int j, int H) { return (j >= H) + (j >= 2 * H) + (j >= 3 * H) + (j >= 4 * H); }
+// dz values of chunk j0 for the block's rows -> operand buffer `buf`.  All loads first and without a
+// branch (rows and columns beyond the block are clamped onto valid ones and discarded afterwards), so that
+// they are in flight together: one round trip instead of one per element; then the arithmetic and the stores.
+__device__ __forceinline__ void fused_gate_gradients(const BwdParams& p, const FusedItem& it, DinputSmem& sm, int ib,
+                                                     int buf, int j0) {
+  const int H = p.H, J = 5 * H, tid = threadIdx.x;
+  float dhn[kLd], dci[kLd], go[kLd], cn[kLd], g1[kLd], g2[kLd];
+#pragma unroll
+  for (int q = 0; q < kLd; ++q) {
+    const int e = tid + q * 256, i = min(e / BK, it.rows - 1), j = min(j0 + e % BK, J - 1);
+    const int node = chk(p.st, sm.fnode[ib][i], p.n);
+    const int g = gate_of_column(j, H), u = j - g * H;
+    const bool forget = g == 1 || g == 2;
+    const int child = chk(p.st, g == 2 ? sm.fright[ib][i] : sm.fleft[ib][i], p.n);
+    const float* gt = p.gates + (size_t)node * J + u;
+    dhn[q] = p.dh[(size_t)node * H + u];
+    dci[q] = p.dc[(size_t)node * H + u];
+    go[q] = gt[3 * H];
+    cn[q] = p.c[(size_t)node * H + u];
+    g1[q] = gt[forget ? g * H : 0];                                   // f_l / f_r, else i
+    g2[q] = *(forget ? p.c + (size_t)child * H + u : gt + 4 * H);    // the child's cell state, else u
+  }
+  const bool keep = it.k0 == 0;
+#pragma unroll
+  for (int q = 0; q < kLd; ++q) {
+    const int e = tid + q * 256, i = e / BK, j = j0 + e % BK;
+    float dz = 0.f;
+    if (i < it.rows && j < J) {
+      const int node = chk(p.st, sm.fnode[ib][i], p.n);
+      const int g = gate_of_column(j, H), u = j - g * H;
+      const float tc = tanhf(cn[q]);
+      const float dcn = dci[q] + dhn[q] * go[q] * (1.f - tc * tc);
+      if (g == 3) {
+        dz = dhn[q] * tc * go[q] * (1.f - go[q]);
+      } else if (g == 1 || g == 2) {
+        const float gf = g1[q];
+        dz = dcn * g2[q] * gf * (1.f - gf);
+        if (keep) p.dc[(size_t)chk(p.st, g == 1 ? sm.fleft[ib][i] : sm.fright[ib][i], p.n) * H + u] = dcn * gf;
+      } else {
+        const float gi = g1[q], gu = g2[q];
+        dz = g == 0 ? dcn * gu * gi * (1.f - gi) : dcn * gi * (1.f - gu * gu);
+      }
+      if (keep) p.dz[(size_t)node * J + j] = dz;
+    }
+    sm.As[buf][i][e % BK] = dz;
+  }
+}
+// one chunk of the contraction for the first 16 NI rows of the tile (thread (tx, ty): rows ty + 16 i, outputs tx + 16 q)
+template <int NI>
+__device__ __forceinline__ void fused_chunk(const DinputSmem& sm, int buf, int tx, int ty, float (&acc)[4][4]) {
+#pragma unroll
+  for (int jj = 0; jj < BK; jj += 4) {
+    float4 a[NI], b[4];
+#pragma unroll
+    for (int i = 0; i < NI; ++i) a[i] = *reinterpret_cast<const float4*>(&sm.As[buf][ty + 16 * i][jj]);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) b[q] = *reinterpret_cast<const float4*>(&sm.Bs[buf][tx + 16 * q][jj]);
+#pragma unroll
+    for (int i = 0; i < NI; ++i)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        acc[i][q] = fmaf(a[i].x, b[q].x, acc[i][q]);
+        acc[i][q] = fmaf(a[i].y, b[q].y, acc[i][q]);
+        acc[i][q] = fmaf(a[i].z, b[q].z, acc[i][q]);
+        acc[i][q] = fmaf(a[i].w, b[q].w, acc[i][q]);
+      }
+  }
+}
+// One block.  prepared: this CTA's threads have requested index set `ib` and the block's first weight
+// chunk (operand buffer c_lo & 1) with cp.async, and no thread of the CTA still reads the operand buffers.
+__device__ void dinput_fused(const BwdParams& p, const FusedItem& it, DinputSmem& sm, int ib, bool prepared,
+                             long long* trace, int lvl) {
+  (void)trace; (void)lvl;
+  if (it.c_lo >= it.chunks) return;   // the same for every thread of the CTA
+  const int H = p.H, K = 2 * H;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  if (!prepared) {
+    __syncthreads();   // a previous block of this CTA may still be reading the shared arrays
+    fused_request_indices(p, it, sm, ib);
+    fused_request_weights(p, it, sm, it.c_lo & 1, it.c_lo * BK);
+  }
+  cp_async_wait();
+  __syncthreads();
+  TL_STAMP(trace, lvl, 8);   // index triples and first weight chunk in shared memory
+  float acc[4][4] = {};
+  fused_gate_gradients(p, it, sm, ib, it.c_lo & 1, it.c_lo * BK);
+  __syncthreads();
+  TL_STAMP(trace, lvl, 5);   // gate gradients of the first chunk formed by all warps
+  const int ni = (it.rows + 15) / 16;   // 16-row groups of the tile that hold nodes
+  for (int cidx = it.c_lo; cidx < it.chunks; ++cidx) {
+    const int buf = cidx & 1;
+    const bool more = cidx + 1 < it.chunks;
+    if (more) fused_request_weights(p, it, sm, buf ^ 1, (cidx + 1) * BK);
+    if (ni == 1) fused_chunk<1>(sm, buf, tx, ty, acc);
+    else if (ni == 2) fused_chunk<2>(sm, buf, tx, ty, acc);
+    else if (ni == 3) fused_chunk<3>(sm, buf, tx, ty, acc);
+    else fused_chunk<4>(sm, buf, tx, ty, acc);
+    if (more) {
+      fused_gate_gradients(p, it, sm, ib, buf ^ 1, (cidx + 1) * BK);
+      cp_async_wait();
+    }
+    __syncthreads();
+  }
+  TL_STAMP(trace, lvl, 6);   // contraction done
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = ty + 16 * i;
+    if (r >= it.rows) continue;
+    const int l = chk(p.st, sm.fleft[ib][r], p.n), rr = chk(p.st, sm.fright[ib][r], p.n);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int k = it.k0 + tx + 16 * q;
+      if (k >= K) continue;
+      atomicAdd(&p.dh[(size_t)(k < H ? l : rr) * H + (k < H ? k : k - H)], acc[i][q]);
+    }
+  }
 }
 
 // ---- dW = In^T dZ (contraction over nodes) and db ------------------------------------------- //
@@ -422,6 +647,12 @@ __global__ void k_bwd_dbias(BwdParams p) {
 // barrier: clear the outputs | mark leaf tokens | token scan (CTA 0) next to the classifier (all
 // other CTAs) | per wavefront from the top: gate gradients, then dIn = dz W^T into the children |
 // dW, db (they only need every dz).
+constexpr int kFusedMaxRows = 128;   // widest wavefront whose gate gradients are formed inside the contraction
+#ifdef TREELSTM_TRACE
+#define TL_TRACE_ARG trace
+#else
+#define TL_TRACE_ARG nullptr
+#endif
 union BwdSmem {
   DinputSmem di;
   DweightSmem dw;
@@ -430,7 +661,7 @@ template <class T>
 __device__ __forceinline__ void zero_range(T* ptr, size_t count, size_t gtid, size_t gthreads) {
   for (size_t i = gtid; i < count; i += gthreads) ptr[i] = T(0);
 }
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
   extern __shared__ float4 s_dyn4[];
   BwdSmem& sm = *reinterpret_cast<BwdSmem*>(s_dyn4);
@@ -464,13 +695,21 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
   TL_STAMP(trace, kTraceLevels - 1, 1);   // outputs and scratch cleared
   for (size_t r = gtid; r < (size_t)p.n_leaves; r += gthreads)
     p.tok_slot[chk(p.st, p.token[chk(p.st, p.order[r], p.n)], p.vocab)] = 1;
+  for (size_t r = (size_t)p.n_leaves + gtid; r < (size_t)n; r += gthreads) {   // children by ready position
+    const int node = chk(p.st, p.order[r], p.n);
+    p.pos_left[r] = p.left[node];
+    p.pos_right[r] = p.right[node];
+  }
   if (!barrier()) return;
   TL_STAMP(trace, kTraceLevels - 1, 2);   // tokens marked
+  // (the CTA's operand buffers are idle in this phase: they hold the scan's ballots)
+  unsigned int* const s_mask = reinterpret_cast<unsigned int*>(s_dyn4);
+  const int mask_cap = (int)(sizeof(BwdSmem) / sizeof(unsigned int));
   if (gridDim.x == 1) {
-    scan_tokens(p);
+    scan_tokens(p, s_mask, mask_cap);
     classifier_groups(p, 0, 1, s_cls);
   } else if (blockIdx.x == 0) {
-    scan_tokens(p);
+    scan_tokens(p, s_mask, mask_cap);
   } else {
     classifier_groups(p, blockIdx.x - 1, gridDim.x - 1, s_cls);
   }
@@ -484,17 +723,58 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
   for (int i = threadIdx.x; i < kOffCache && i <= n_levels; i += blockDim.x) s_off[i] = level_offset[i];
   __syncthreads();
   auto level_begin = [&](int l) { return l < kOffCache ? s_off[l] : level_offset[l]; };
+  auto is_fused = [&](int l) { return l > 0 && level_begin(l + 1) - level_begin(l) <= kFusedMaxRows; };
+  // this CTA's first block of every narrow wavefront, worked out once (thread l: wavefront l) - the
+  // divisions behind it would otherwise sit between a wavefront's last store and the grid barrier
+  auto first_block = [&](int l) {
+    FusedItem it{};   // c_lo == chunks == 0: no block
+    if (is_fused(l)) {
+      const int b = level_begin(l), e = level_begin(l + 1);
+      const int ntiles = dinput_tiles(e - b, 2 * H), nsplits = dinput_splits(ntiles, J);
+      if ((int)blockIdx.x < ntiles * nsplits) it = fused_item(p, b, e, blockIdx.x % ntiles, blockIdx.x / ntiles, nsplits);
+    }
+    return it;
+  };
+  __shared__ FusedItem s_first[kOffCache];
+  for (int l = threadIdx.x; l < kOffCache && l < n_levels; l += blockDim.x) s_first[l] = first_block(l);
+  __syncthreads();
+  bool prepared = false;
+  FusedItem pre_item{};
   for (int lvl = n_levels - 1; lvl >= 0; --lvl) {
     const int begin = level_begin(lvl), end = level_begin(lvl + 1), leaf = lvl == 0 ? 1 : 0;
     const long long elems = (long long)(end - begin) * H;
     TL_STAMP(trace, lvl, 0);
-    for (long long idx = (long long)gtid; idx < elems; idx += (long long)gthreads) gates_element(p, begin, idx, leaf);
-    TL_STAMP(trace, lvl, 1);
-    if (!barrier()) return;
+    // a narrow internal wavefront forms its gate gradients inside the contraction (dinput_fused)
+    const bool fused = is_fused(lvl);
+    if (!fused) {
+      for (long long idx = (long long)gtid; idx < elems; idx += (long long)gthreads) gates_element(p, begin, idx, leaf);
+      TL_STAMP(trace, lvl, 1);
+      if (!barrier()) return;
+    }
     TL_STAMP(trace, lvl, 2);
     const int tiles = dinput_tiles(end - begin, leaf ? E : 2 * H), splits = dinput_splits(tiles, J);
-    for (int vb = blockIdx.x; vb < tiles * splits; vb += gridDim.x)
-      dinput_block(p, begin, end, leaf, vb % tiles, vb / tiles, splits, sm.di);
+    if (fused) {
+      for (int vb = blockIdx.x; vb < tiles * splits; vb += gridDim.x) {
+        const bool ready = prepared && vb == (int)blockIdx.x;
+        if (!ready) pre_item = fused_item(p, begin, end, vb % tiles, vb / tiles, splits);
+        dinput_fused(p, pre_item, sm.di, lvl & 1, ready, TL_TRACE_ARG, lvl);
+      }
+      TL_STAMP(trace, lvl, 7);   // own blocks done
+    } else {
+      for (int vb = blockIdx.x; vb < tiles * splits; vb += gridDim.x)
+        dinput_block(p, begin, end, leaf, vb % tiles, vb / tiles, splits, sm.di);
+    }
+    // this CTA's first block of the next wavefront: its index triples and first weight chunk are
+    // requested now and land in shared memory during the grid barrier
+    prepared = false;
+    if (lvl > 1) {
+      pre_item = lvl - 1 < kOffCache ? s_first[lvl - 1] : first_block(lvl - 1);
+      if (pre_item.c_lo < pre_item.chunks) {
+        fused_request_indices(p, pre_item, sm.di, (lvl - 1) & 1);
+        fused_request_weights(p, pre_item, sm.di, pre_item.c_lo & 1, pre_item.c_lo * BK);
+        prepared = true;
+      }
+    }
     TL_STAMP(trace, lvl, 3);
     if (lvl > 0 && !barrier()) return;   // the leaves' dIn goes to the embedding rows only
     TL_STAMP(trace, lvl, 4);
@@ -543,6 +823,8 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
   p.loss = loss; p.dW = dW; p.db = db; p.dWc = dWc; p.dbc = dbc; p.dEmb_rows = dEmb_rows;
   p.tok_slot = reinterpret_cast<int*>(base + L.lay.tok_slot);
   p.touched_ids = touched_ids; p.n_touched = n_touched;
+  p.pos_left = reinterpret_cast<int*>(base + L.lay.parent);      // the scheduler's scratch is free once the forward has run
+  p.pos_right = reinterpret_cast<int*>(base + L.lay.order_tmp);
   p.st = reinterpret_cast<DevStatus*>(base + L.lay.status);
   p.trace = nullptr;
 #ifdef TREELSTM_TRACE
