@@ -129,6 +129,10 @@ typedef enum treelstm_status {
                                             /* this many nodes (default 4096); smaller forests keep the    */
                                             /* order of work of the cooperative launch: their scheduler    */
                                             /* is too short to hide the two extra grid barriers            */
+#define TREELSTM_OPT_DW_TENSOR_CORES 10     /* 1 (default): after a forward that kept its level table on   */
+                                            /* the device, treelstm_backward forms dW and db on the tensor */
+                                            /* cores, every fp32 operand split into three bf16 pieces (six */
+                                            /* products per term: fp32 accuracy); 0: fp32 multiply-adds    */
 
 /*
  * treelstm_create - build a context for one set of parameters.

@@ -42,6 +42,7 @@ OPT_TAIL_MIN_LEVELS = 6
 OPT_TAIL_MAX_NODES = 7
 OPT_OVERLAP_LAUNCH = 8
 OPT_LEAVES_FIRST_MIN_NODES = 9
+OPT_DW_TENSOR_CORES = 10
 
 _vp = ctypes.c_void_p
 _i = ctypes.c_int

@@ -24,7 +24,7 @@ def lib_path(variant: str = "") -> str:
     if variant not in VARIANT_FLAGS:
         raise ValueError(f"unknown library variant {variant!r}")
     return os.path.join(PKG_DIR, f"libtreelstm_b200_{variant}.so" if variant else "libtreelstm_b200.so")
-SOURCES = ("api.cu", "schedule.cu", "cell_fp32.cu", "cell_rec.cu", "gemm_tc.cu", "subforest_tc.cu", "tail_tc.cu", "backward.cu")
+SOURCES = ("api.cu", "schedule.cu", "cell_fp32.cu", "cell_rec.cu", "gemm_tc.cu", "subforest_tc.cu", "tail_tc.cu", "backward.cu", "dweight_tc.cu")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

@@ -205,6 +205,7 @@ int treelstm_create(treelstm_t** out, int H, int E, int vocab, const float* emb,
   }
   int rc = init_schedule_attributes(ctx);
   if (rc == TREELSTM_OK && precision == TREELSTM_BF16) rc = init_tc_attributes(ctx);
+  if (rc == TREELSTM_OK) rc = init_dweight_tc_attributes(ctx);
   if (rc != TREELSTM_OK) return fail(rc);
   rc = copy_params(ctx, emb, W, b, s);
   if (rc != TREELSTM_OK) return fail(rc);
@@ -300,6 +301,9 @@ int treelstm_set_option(treelstm_t* ctx, int key, long long value) {
       return TREELSTM_OK;
     case TREELSTM_OPT_OVERLAP_LAUNCH:
       ctx->opt.overlap_launch = value != 0;
+      return TREELSTM_OK;
+    case TREELSTM_OPT_DW_TENSOR_CORES:
+      ctx->opt.dw_tensor_cores = value != 0;
       return TREELSTM_OK;
     case TREELSTM_OPT_TAIL_MAX_NODES:
       ctx->opt.tail_max_nodes = value > (1 << 30) ? (1 << 30) : (int)value;

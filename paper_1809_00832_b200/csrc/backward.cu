@@ -662,7 +662,7 @@ __device__ __forceinline__ void zero_range(T* ptr, size_t count, size_t gtid, si
   for (size_t i = gtid; i < count; i += gthreads) ptr[i] = T(0);
 }
 __global__ void __launch_bounds__(256, 2)
-k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
+k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit, int with_dweight) {
   extern __shared__ float4 s_dyn4[];
   BwdSmem& sm = *reinterpret_cast<BwdSmem*>(s_dyn4);
   float* s_cls = reinterpret_cast<float*>(s_dyn4) + (sizeof(BwdSmem) + 3) / 4;
@@ -780,6 +780,7 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit) {
     TL_STAMP(trace, lvl, 4);
   }
   TL_STAMP(trace, kTraceLevels - 1, 5);   // all wavefronts done
+  if (!with_dweight) return;              // dW and db are left to the tensor-core kernel that follows on the stream
   const int tiles_j = (J + BT - 1) / BT, rows_per_split = kDwRows;
   for (int part = 0; part < 2; ++part) {
     const int begin = part == 0 ? 0 : p.n_leaves, end = part == 0 ? p.n_leaves : n;
@@ -856,9 +857,12 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
     TL_CUDA(ctx, cudaMemsetAsync(&st->barrier_bwd, 0, sizeof(unsigned int), stream));
     const int* lvl_off = L.level_offset;
     long long wait_limit = ctx->opt.wait_limit_kcycles * 1024;
-    void* args[] = {&p, &lvl_off, &wait_limit};
+    int with_dweight = ctx->opt.dw_tensor_cores ? 0 : 1;
+    void* args[] = {&p, &lvl_off, &wait_limit, &with_dweight};
     TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_bwd_persistent, dim3(grid), dim3(256), args, smem, stream));
     ctx->launches += 1;
+    if (!with_dweight)
+      return launch_dweight_tc(ctx, n, L.order, L.level_offset, L.token, L.left, L.right, L.h, p.dz, dW, db, p.st, stream);
     return TREELSTM_OK;
   }
   TL_CUDA(ctx, cudaMemsetAsync(loss, 0, sizeof(float), stream));

@@ -53,6 +53,7 @@ struct Options {
   int tail_min_levels = 0; // > 0: hand them over if at least this many remain; 0: the device decides by its cost model
   int tail_max_nodes = 4096;   // forests with more nodes never launch the cluster kernel
   int leaves_first_min_nodes = 4096;   // forests at least this large: leaf wavefront before the wait for the schedule
+  int dw_tensor_cores = 1;     // one-launch backward: dW and db by split-bf16 tensor-core contraction
   int overlap_launch = 1;      // persistent bf16 forward: the wavefront kernel starts under the scheduler (programmatic dependent launch)
 };
 
@@ -228,6 +229,12 @@ int ensure_host_levels(treelstm* ctx);
 int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW, float* db,
                     float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,
                     int32_t* n_touched, cudaStream_t stream);
+
+// dweight_tc.cu: dW += In^T dZ, db += sum dZ on the tensor cores (three bf16 pieces per fp32 value)
+int init_dweight_tc_attributes(treelstm* ctx);
+int launch_dweight_tc(treelstm* ctx, int n, const int32_t* order, const int32_t* level_offset, const int32_t* token,
+                      const int32_t* left, const int32_t* right, const float* h, const float* dz, float* dW, float* db,
+                      DevStatus* st, cudaStream_t stream);
 
 // Checked build: clears the per-row write counters before a forward / compares them after it
 // (schedule.cu); both do nothing in the normal build.  Counters: [h per node | Ain per position | Cin per position].
