@@ -144,6 +144,10 @@ __device__ void classifier_groups(const BwdParams& p, int vb_first, int vb_step,
   const int H = p.H, C = p.C;
   for (int i = tid; i < H * C + C; i += blockDim.x) s_dWc[i] = 0.f;
   __syncthreads();
+#ifdef TREELSTM_TRACE
+  long long* const ctrace = blockIdx.x == 1 && tid == 0 ? p.trace : nullptr;   // the first CTA with nodes to classify
+#endif
+  TL_STAMP(ctrace, kTraceLevels - 1, 11);
   const float inv_n = 1.0f / (float)p.n;
   const int n_groups = (p.n + kClsNodesPerCta - 1) / kClsNodesPerCta;
   for (int vb = vb_first; vb < n_groups; vb += vb_step)
@@ -187,11 +191,14 @@ __device__ void classifier_groups(const BwdParams& p, int vb_first, int vb_step,
       }
       if (j < H) p.dh[(size_t)node * H + j] = dhj;
     }
+    TL_STAMP(ctrace, kTraceLevels - 1, 12);   // first warp: a node done
   }
   __syncthreads();
+  TL_STAMP(ctrace, kTraceLevels - 1, 13);     // all warps: nodes done
   if (vb_first >= n_groups) return;   // a CTA without a group has nothing to add (and 300 CTAs adding zeros to the same H x C words queue up)
   for (int i = tid; i < H * C; i += blockDim.x) atomicAdd(&p.dWc[i], s_dWc[i]);
   for (int i = tid; i < C; i += blockDim.x) atomicAdd(&p.dbc[i], s_dWc[H * C + i]);
+  TL_STAMP(ctrace, kTraceLevels - 1, 14);     // partial sums sent
 }
 __global__ void __launch_bounds__(kClsWarps * 32) k_bwd_classifier(BwdParams p) {
   extern __shared__ float s_dyn[];
@@ -378,32 +385,53 @@ __device__ __forceinline__ FusedItem fused_item(const BwdParams& p, int row_begi
   it.chunks = min(chunks_all, it.c_lo + per_split);
   return it;
 }
-__device__ __forceinline__ void cp_async4(void* smem_dst, const void* src, bool valid) {
-  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
-  const uint32_t bytes = valid ? 4u : 0u;   // 0: the word is filled with zeros, the source is not read
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-// index triples of the block's rows into set `ib` (asynchronous)
-__device__ __forceinline__ void fused_request_indices(const BwdParams& p, const FusedItem& it, DinputSmem& sm, int ib) {
-  const int t = threadIdx.x;
+// What a block needs that does not depend on the wavefront above, fetched into registers (a 4-byte cp.async
+// per element measured ~130 cycles of issue each: slower than holding nine registers across the barrier) ...
+struct FusedFetch {
+  int idx;          // thread t < 192: order / pos_left / pos_right of row t % 64
+  float w[kLd];     // the thread's elements of the first weight chunk
+};
+__device__ __forceinline__ void fused_fetch(const BwdParams& p, const FusedItem& it, int j0, FusedFetch& f) {
+  const int J = 5 * p.H, K = 2 * p.H, t = threadIdx.x;
+  f.idx = 0;
   if (t < 3 * BT) {
     const int which = t / BT, i = t % BT;
-    const bool valid = i < it.rows;
-    const int pos = valid ? it.row0 + i : 0;
-    const int* src = which == 0 ? p.order + pos : (which == 1 ? p.pos_left + pos : p.pos_right + pos);
-    int* dst = which == 0 ? &sm.fnode[ib][i] : (which == 1 ? &sm.fleft[ib][i] : &sm.fright[ib][i]);
-    cp_async4(dst, src, valid);
+    const int pos = it.row0 + min(i, it.rows - 1);
+    f.idx = *(which == 0 ? p.order + pos : (which == 1 ? p.pos_left + pos : p.pos_right + pos));
   }
-}
-// weight chunk j0 of the block into operand buffer `buf` (asynchronous)
-__device__ __forceinline__ void fused_request_weights(const BwdParams& p, const FusedItem& it, DinputSmem& sm, int buf, int j0) {
-  const int J = 5 * p.H, K = 2 * p.H, tid = threadIdx.x;
 #pragma unroll
   for (int q = 0; q < kLd; ++q) {
-    const int e = tid + q * 256, i = e / BK, j = j0 + e % BK;
-    const bool valid = it.k0 + i < K && j < J;
-    cp_async4(&sm.Bs[buf][i][e % BK], p.W + (valid ? (size_t)(p.E + it.k0 + i) * J + j : 0), valid);
+    const int e = t + q * 256, i = min(it.k0 + e / BK, K - 1), j = min(j0 + e % BK, J - 1);
+    f.w[q] = __ldg(p.W + (size_t)(p.E + i) * J + j);
+  }
+}
+// ... and put into index set `ib` and operand buffer `buf` (a CTA barrier must follow)
+__device__ __forceinline__ void fused_deposit(const BwdParams& p, const FusedItem& it, DinputSmem& sm, int ib, int buf,
+                                              int j0, const FusedFetch& f) {
+  const int J = 5 * p.H, K = 2 * p.H, t = threadIdx.x;
+  if (t < 3 * BT) {
+    const int which = t / BT, i = t % BT;
+    *(which == 0 ? &sm.fnode[ib][i] : (which == 1 ? &sm.fleft[ib][i] : &sm.fright[ib][i])) = f.idx;
+  }
+#pragma unroll
+  for (int q = 0; q < kLd; ++q) {
+    const int e = t + q * 256;
+    sm.Bs[buf][e / BK][e % BK] = (it.k0 + e / BK < K && j0 + e % BK < J) ? f.w[q] : 0.f;
+  }
+}
+// weight chunk j0 of the block into operand buffer `buf` (later chunks of a block)
+__device__ __forceinline__ void fused_weights(const BwdParams& p, const FusedItem& it, DinputSmem& sm, int buf, int j0) {
+  const int J = 5 * p.H, K = 2 * p.H, t = threadIdx.x;
+  float w[kLd];
+#pragma unroll
+  for (int q = 0; q < kLd; ++q) {
+    const int e = t + q * 256, i = min(it.k0 + e / BK, K - 1), j = min(j0 + e % BK, J - 1);
+    w[q] = __ldg(p.W + (size_t)(p.E + i) * J + j);
+  }
+#pragma unroll
+  for (int q = 0; q < kLd; ++q) {
+    const int e = t + q * 256;
+    sm.Bs[buf][e / BK][e % BK] = (it.k0 + e / BK < K && j0 + e % BK < J) ? w[q] : 0.f;
   }
 }
 __device__ __forceinline__ int gate_of_column(int j, int H) { return (j >= H) + (j >= 2 * H) + (j >= 3 * H) + (j >= 4 * H); }
@@ -475,20 +503,21 @@ __device__ __forceinline__ void fused_chunk(const DinputSmem& sm, int buf, int t
       }
   }
 }
-// One block.  prepared: this CTA's threads have requested index set `ib` and the block's first weight
-// chunk (operand buffer c_lo & 1) with cp.async, and no thread of the CTA still reads the operand buffers.
-__device__ void dinput_fused(const BwdParams& p, const FusedItem& it, DinputSmem& sm, int ib, bool prepared,
-                             long long* trace, int lvl) {
+// One block.  fetched: `f` holds the block's index triples and first weight chunk (fused_fetch was called before
+// the grid barrier) and no thread of the CTA still reads the operand buffers.
+// buffers_free() runs once, when the block no longer needs the operand buffers and before its results go out.
+template <class FreeFn>
+__device__ __forceinline__ void dinput_fused(const BwdParams& p, const FusedItem& it, DinputSmem& sm, int ib, bool fetched,
+                                             FusedFetch& f, long long* trace, int lvl, FreeFn buffers_free) {
   (void)trace; (void)lvl;
-  if (it.c_lo >= it.chunks) return;   // the same for every thread of the CTA
+  if (it.c_lo >= it.chunks) { buffers_free(); return; }   // the same for every thread of the CTA
   const int H = p.H, K = 2 * H;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  if (!prepared) {
+  if (!fetched) {
     __syncthreads();   // a previous block of this CTA may still be reading the shared arrays
-    fused_request_indices(p, it, sm, ib);
-    fused_request_weights(p, it, sm, it.c_lo & 1, it.c_lo * BK);
+    fused_fetch(p, it, it.c_lo * BK, f);
   }
-  cp_async_wait();
+  fused_deposit(p, it, sm, ib, it.c_lo & 1, it.c_lo * BK, f);
   __syncthreads();
   TL_STAMP(trace, lvl, 8);   // index triples and first weight chunk in shared memory
   float acc[4][4] = {};
@@ -499,18 +528,18 @@ __device__ void dinput_fused(const BwdParams& p, const FusedItem& it, DinputSmem
   for (int cidx = it.c_lo; cidx < it.chunks; ++cidx) {
     const int buf = cidx & 1;
     const bool more = cidx + 1 < it.chunks;
-    if (more) fused_request_weights(p, it, sm, buf ^ 1, (cidx + 1) * BK);
+    if (more) fused_weights(p, it, sm, buf ^ 1, (cidx + 1) * BK);
     if (ni == 1) fused_chunk<1>(sm, buf, tx, ty, acc);
     else if (ni == 2) fused_chunk<2>(sm, buf, tx, ty, acc);
     else if (ni == 3) fused_chunk<3>(sm, buf, tx, ty, acc);
     else fused_chunk<4>(sm, buf, tx, ty, acc);
     if (more) {
       fused_gate_gradients(p, it, sm, ib, buf ^ 1, (cidx + 1) * BK);
-      cp_async_wait();
     }
     __syncthreads();
   }
   TL_STAMP(trace, lvl, 6);   // contraction done
+  buffers_free();
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int r = ty + 16 * i;
@@ -740,6 +769,7 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit, int
   __syncthreads();
   bool prepared = false;
   FusedItem pre_item{};
+  FusedFetch pre_fetch;
   for (int lvl = n_levels - 1; lvl >= 0; --lvl) {
     const int begin = level_begin(lvl), end = level_begin(lvl + 1), leaf = lvl == 0 ? 1 : 0;
     const long long elems = (long long)(end - begin) * H;
@@ -753,28 +783,37 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit, int
     }
     TL_STAMP(trace, lvl, 2);
     const int tiles = dinput_tiles(end - begin, leaf ? E : 2 * H), splits = dinput_splits(tiles, J);
+    // This CTA's first block of the next wavefront: its index triples and first weight chunk are requested
+    // as soon as the operand buffers are free - ahead of the atomic adds of this wavefront's results, which
+    // would otherwise hold the requests up - and land in shared memory during the grid barrier.
+    bool requested = false;
+    auto request_next = [&]() {
+      TL_STAMP(trace, lvl, 9);
+      requested = true;
+      prepared = false;
+      if (lvl > 1) {
+        pre_item = lvl - 1 < kOffCache ? s_first[lvl - 1] : first_block(lvl - 1);
+        if (pre_item.c_lo < pre_item.chunks) {
+          fused_fetch(p, pre_item, pre_item.c_lo * BK, pre_fetch);
+          prepared = true;
+        }
+      }
+      TL_STAMP(trace, lvl, 11);
+    };
     if (fused) {
       for (int vb = blockIdx.x; vb < tiles * splits; vb += gridDim.x) {
         const bool ready = prepared && vb == (int)blockIdx.x;
-        if (!ready) pre_item = fused_item(p, begin, end, vb % tiles, vb / tiles, splits);
-        dinput_fused(p, pre_item, sm.di, lvl & 1, ready, TL_TRACE_ARG, lvl);
+        const bool last = vb + (int)gridDim.x >= tiles * splits;
+        const FusedItem item = ready ? pre_item : fused_item(p, begin, end, vb % tiles, vb / tiles, splits);
+        if (last) dinput_fused(p, item, sm.di, lvl & 1, ready, pre_fetch, TL_TRACE_ARG, lvl, request_next);
+        else dinput_fused(p, item, sm.di, lvl & 1, ready, pre_fetch, TL_TRACE_ARG, lvl, []() {});
       }
       TL_STAMP(trace, lvl, 7);   // own blocks done
     } else {
       for (int vb = blockIdx.x; vb < tiles * splits; vb += gridDim.x)
         dinput_block(p, begin, end, leaf, vb % tiles, vb / tiles, splits, sm.di);
     }
-    // this CTA's first block of the next wavefront: its index triples and first weight chunk are
-    // requested now and land in shared memory during the grid barrier
-    prepared = false;
-    if (lvl > 1) {
-      pre_item = lvl - 1 < kOffCache ? s_first[lvl - 1] : first_block(lvl - 1);
-      if (pre_item.c_lo < pre_item.chunks) {
-        fused_request_indices(p, pre_item, sm.di, (lvl - 1) & 1);
-        fused_request_weights(p, pre_item, sm.di, pre_item.c_lo & 1, pre_item.c_lo * BK);
-        prepared = true;
-      }
-    }
+    if (!requested) request_next();
     TL_STAMP(trace, lvl, 3);
     if (lvl > 0 && !barrier()) return;   // the leaves' dIn goes to the embedding rows only
     TL_STAMP(trace, lvl, 4);

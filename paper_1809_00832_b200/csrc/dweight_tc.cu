@@ -46,14 +46,17 @@ struct DwParams {
   long long wait_limit;
 };
 
-// v -> three bf16 pieces (bit patterns)
-__device__ __forceinline__ void split3(float v, unsigned short& p0, unsigned short& p1, unsigned short& p2) {
-  const __nv_bfloat16 b0 = __float2bfloat16_rn(v);
-  const float r1 = v - __bfloat162float(b0);
-  const __nv_bfloat16 b1 = __float2bfloat16_rn(r1);
-  const float r2 = r1 - __bfloat162float(b1);
-  const __nv_bfloat16 b2 = __float2bfloat16_rn(r2);
-  p0 = __bfloat16_as_ushort(b0); p1 = __bfloat16_as_ushort(b1); p2 = __bfloat16_as_ushort(b2);
+// (x, y) -> three words of two bf16 pieces each (x in the low half): x = x0 + x1 + x2, y likewise
+__device__ __forceinline__ void split3_pair(float x, float y, uint32_t& w0, uint32_t& w1, uint32_t& w2) {
+  auto pack = [](float a, float b) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<const uint32_t*>(&v);
+  };
+  w0 = pack(x, y);
+  x -= __uint_as_float(w0 << 16);  y -= __uint_as_float(w0 & 0xFFFF0000u);
+  w1 = pack(x, y);
+  x -= __uint_as_float(w1 << 16);  y -= __uint_as_float(w1 & 0xFFFF0000u);
+  w2 = pack(x, y);
 }
 
 // byte offset of the 16-byte piece (row r, nodes 8 c .. 8 c + 7) inside a K-major tile with the 128-byte swizzle
@@ -61,23 +64,23 @@ __device__ __forceinline__ uint32_t swz_piece(int r, int c) {
   return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4));
 }
 
-// One operand tile (128 rows x 64 nodes, three pieces) of block `kb` of the work item into shared memory.
+// One operand tile (128 rows x 64 nodes, three pieces) of block `kb` of the work item, in two steps: the
+// fp32 values into registers (tile_load: nothing but loads, so all of a block's are in flight together),
+// then split, packed and stored into shared memory (tile_store).
 // kKind 0: input rows of the leaves (embedding units, then the row of ones), 1: input rows of the internal
 // nodes ([h_l | h_r], then the row of ones), 2: gate columns (dz).  row0: first row of the tile within its
 // operand.  s_node / s_ia / s_ib: per node of the item its id and where its input row comes from (token; left,
 // right child); entries behind the item's last node are 0 and their values are discarded.  Warp w takes the
-// nodes 8 w .. 8 w + 7 of the block for all four groups of 32 rows; all loads of a group are issued before
-// the first use.
+// nodes 8 w .. 8 w + 7 of the block, lane l the rows l, l + 32, l + 64, l + 96.
 template <int kKind>
-__device__ __forceinline__ void build_tile(const DwParams& p, unsigned char* tile, int row0, const int* s_node,
-                                           const int* s_ia, const int* s_ib, int kb, int valid_nodes) {
+__device__ __forceinline__ void tile_load(const DwParams& p, int row0, const int* s_node, const int* s_ia,
+                                          const int* s_ib, int kb, float (&v)[4][8]) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int H = p.H, E = p.E, J = 5 * H;
-  const int rows = kKind == 0 ? E : (kKind == 1 ? 2 * H : J);   // real rows of the operand; row `rows` of an input operand is the ones
+  const int rows = kKind == 0 ? E : (kKind == 1 ? 2 * H : J);
 #pragma unroll
-  for (int rg = 0; rg < kDwTile / 32; ++rg) {
-    const int r = rg * 32 + lane, f = row0 + r, fc = min(f, rows - 1);
-    float v[8];
+  for (int rg = 0; rg < 4; ++rg) {
+    const int fc = min(row0 + rg * 32 + lane, rows - 1);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int k = kb * kDwBlock + 8 * warp + i;
@@ -85,21 +88,29 @@ __device__ __forceinline__ void build_tile(const DwParams& p, unsigned char* til
       if (kKind == 0) src = p.emb + (size_t)s_ia[k] * E + fc;
       else if (kKind == 1) src = p.h + (size_t)(fc < H ? s_ia[k] : s_ib[k]) * H + (fc < H ? fc : fc - H);
       else src = p.dz + (size_t)s_node[k] * J + fc;
-      v[i] = kKind == 0 ? __ldg(src) : *src;
+      v[rg][i] = kKind == 0 ? __ldg(src) : *src;
     }
+  }
+}
+template <int kKind>
+__device__ __forceinline__ void tile_store(const DwParams& p, unsigned char* tile, int row0, int valid_nodes,
+                                           const float (&v)[4][8]) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rows = kKind == 0 ? p.E : (kKind == 1 ? 2 * p.H : 5 * p.H);   // row `rows` of an input operand is the ones
+#pragma unroll
+  for (int rg = 0; rg < 4; ++rg) {
+    const int r = rg * 32 + lane, f = row0 + r;
     uint32_t w0[4], w1[4], w2[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const bool node_ok = 8 * warp + i < valid_nodes;
-      float x = node_ok && f < rows ? v[i] : 0.f;
-      if (kKind != 2 && node_ok && f == rows) x = 1.f;
-      unsigned short a, b, c;
-      split3(x, a, b, c);
-      if (i & 1) {
-        w0[i >> 1] |= (uint32_t)a << 16; w1[i >> 1] |= (uint32_t)b << 16; w2[i >> 1] |= (uint32_t)c << 16;
-      } else {
-        w0[i >> 1] = a; w1[i >> 1] = b; w2[i >> 1] = c;
+    for (int i = 0; i < 8; i += 2) {
+      float x[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const bool node_ok = 8 * warp + i + e < valid_nodes;
+        x[e] = node_ok && f < rows ? v[rg][i + e] : 0.f;
+        if (kKind != 2 && node_ok && f == rows) x[e] = 1.f;
       }
+      split3_pair(x[0], x[1], w0[i >> 1], w1[i >> 1], w2[i >> 1]);
     }
     unsigned char* dst = tile + swz_piece(r, warp);
     *reinterpret_cast<uint4*>(dst) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
@@ -178,15 +189,19 @@ __global__ void __launch_bounds__(kDwThreads, 1) k_bwd_dweight_tc(DwParams p) {
     __syncthreads();
     for (int b = 0; b < nblk; ++b, ++built) {
       const uint32_t stage = built & 1u, use = built >> 1;
-      bool ok = true;
-      if (use >= 1)   // the MMAs that read this stage two blocks ago must have retired
-        ok = mbar_wait(stage_bar0 + 8 * stage, (use - 1) & 1u, &s_abort, p.wait_limit, p.st);
-      if (__syncthreads_or(!ok)) { failed = true; break; }
       unsigned char* st_tiles = tiles + stage * kDwStageBytes;
       const int valid_nodes = min(kDwBlock, pos_end - pos0 - b * kDwBlock);
-      if (part == 0) build_tile<0>(p, st_tiles, m0, s_node, s_ia, s_ib, b, valid_nodes);
-      else build_tile<1>(p, st_tiles, m0, s_node, s_ia, s_ib, b, valid_nodes);
-      build_tile<2>(p, st_tiles + kDwPieces * kDwTileBytes, j0, s_node, s_ia, s_ib, b, valid_nodes);
+      float va[4][8], vb[4][8];
+      if (part == 0) tile_load<0>(p, m0, s_node, s_ia, s_ib, b, va);
+      else tile_load<1>(p, m0, s_node, s_ia, s_ib, b, va);
+      tile_load<2>(p, j0, s_node, s_ia, s_ib, b, vb);
+      bool ok = true;
+      if (use >= 1)   // the MMAs that read this stage two blocks ago must have retired before it is overwritten
+        ok = mbar_wait(stage_bar0 + 8 * stage, (use - 1) & 1u, &s_abort, p.wait_limit, p.st);
+      if (__syncthreads_or(!ok)) { failed = true; break; }
+      if (part == 0) tile_store<0>(p, st_tiles, m0, valid_nodes, va);
+      else tile_store<1>(p, st_tiles, m0, valid_nodes, va);
+      tile_store<2>(p, st_tiles + kDwPieces * kDwTileBytes, j0, valid_nodes, vb);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the tensor core
       tc_fence_before();
       __syncthreads();

@@ -75,15 +75,16 @@ def trace_training_step() -> int:
     names = ("outputs and scratch cleared", "tokens marked", "own part of token scan / classifier done",
              "classifier, loss, token scan done everywhere", "all wavefronts done", "dW from the leaves (own blocks)",
              "dW from the internal nodes (own blocks)", "db done", "token scan: first warp has read its flags",
-             "token scan: all warps have")
+             "token scan: all warps have", "classifier (second CTA): starts", "classifier: first warp's node done",
+             "classifier: all warps' nodes done", "classifier: partial sums sent")
     print("# one-launch backward, first CTA, cycles since its start: " +
           ", ".join(f"{nm} {int(ph[i + 1] - ph[0])}" for i, nm in enumerate(names) if ph[i + 1]))
-    print("level width gates_done barrier dinput_done barrier first_dz contracted own_blocks operands_landed   (cycles since the wavefront's start; "
+    print("level width gates_done barrier dinput_done barrier first_dz contracted own_blocks operands_landed request_begin indices_requested weights_requested   (cycles since the wavefront's start; "
           "wavefronts run in reverse; the last three only where the gate gradients are formed inside the contraction)")
     for l in range(len(widths) - 1, -1, -1):
         if t[l, 0] == 0:
             continue
-        print(f"{l:<5d} {int(widths[l]):<5d} " + " ".join(f"{(t[l, k] - t[l, 0]) if t[l, k] else 0:<10d}" for k in range(1, 9)))
+        print(f"{l:<5d} {int(widths[l]):<5d} " + " ".join(f"{(t[l, k] - t[l, 0]) if t[l, k] else 0:<10d}" for k in range(1, 12)))
     return 0
 
 
