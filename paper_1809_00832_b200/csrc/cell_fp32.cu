@@ -240,6 +240,23 @@ __device__ void fp32_tile_stationary(const FwdParams& p, int row0, int row_end, 
   for (int i = 0; i < RPT; ++i)
 #pragma unroll
     for (int g = 0; g < 5; ++g) acc[i][g] = 0.f;
+  // what the cell update needs beside the contraction is asked for now and arrives while it runs: the bias
+  // and the children's cell states of the rows this thread will finish (row ty of a split tile, else its four)
+  const int u = u0 + tx;
+  float bias[5] = {};
+  constexpr int kFin = kSplit ? 1 : RPT;
+  float c_left[kFin], c_right[kFin];
+  if (u < H) {
+#pragma unroll
+    for (int g = 0; g < 5; ++g) bias[g] = __ldg(p.b + g * H + u);
+  }
+#pragma unroll
+  for (int i = 0; i < kFin; ++i) {
+    const int ii = kSplit ? ty : rg * RPT + i;
+    const bool valid = u < H && s_node[ii] >= 0;
+    c_left[i] = valid ? __ldcg(p.c + (size_t)s_l[ii] * H + u) : 0.f;
+    c_right[i] = valid ? __ldcg(p.c + (size_t)s_r[ii] * H + u) : 0.f;
+  }
   const int steps = K4 / 4, per = (steps + NQ - 1) / NQ;
   const int k_lo = kq * per * 4, k_hi = min(K4, k_lo + per * 4);
   for (int k = k_lo; k < k_hi; k += 4) {
@@ -258,13 +275,7 @@ __device__ void fp32_tile_stationary(const FwdParams& p, int row0, int row_end, 
         acc[i][g] = fmaf(a[i].w, w[g].w, acc[i][g]);
       }
   }
-  const int u = u0 + tx;
-  float bias[5] = {};
-  if (u < H) {
-#pragma unroll
-    for (int g = 0; g < 5; ++g) bias[g] = __ldg(p.b + g * H + u);
-  }
-  auto finish = [&](int ii, const float* z) {   // cell update of tile row ii, hidden unit u
+  auto finish = [&](int ii, const float* z, float cl, float cr) {   // cell update of tile row ii, hidden unit u
     const int node = s_node[ii];
     if (node < 0 || u >= H) return;
     const float gi = sigmoidf_acc(z[0] + bias[0]);
@@ -272,7 +283,7 @@ __device__ void fp32_tile_stationary(const FwdParams& p, int row0, int row_end, 
     const float gfr = sigmoidf_acc(z[2] + bias[2]);
     const float go = sigmoidf_acc(z[3] + bias[3]);
     const float gu = tanhf(z[4] + bias[4]);
-    const float cn = gi * gu + gfl * __ldcg(p.c + (size_t)s_l[ii] * H + u) + gfr * __ldcg(p.c + (size_t)s_r[ii] * H + u);
+    const float cn = gi * gu + gfl * cl + gfr * cr;
     p.c[(size_t)node * H + u] = cn;
     p.h[(size_t)node * H + u] = go * tanhf(cn);
     count_write(p.chk_counts, node, 1);
@@ -296,10 +307,10 @@ __device__ void fp32_tile_stationary(const FwdParams& p, int row0, int row_end, 
       for (int q = 0; q < NQ; ++q) sum += red[(q * TMS + ty) * (5 * TU) + g * TU + tx];
       z[g] = sum;
     }
-    finish(ty, z);
+    finish(ty, z, c_left[0], c_right[0]);
   } else {
 #pragma unroll
-    for (int i = 0; i < RPT; ++i) finish(rg * RPT + i, acc[i]);
+    for (int i = 0; i < RPT; ++i) finish(rg * RPT + i, acc[i], c_left[i], c_right[i]);
   }
 }
 

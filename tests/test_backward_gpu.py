@@ -105,3 +105,42 @@ def test_data_parallel_step_single_rank():
     res = {k: v.cpu().numpy() for k, v in out.items()}
     assert res["touched_ids"].shape[0] == len(ref["touched_ids"])
     _compare(res, ref, util.TOL["fp32"])
+
+
+@pytest.mark.parametrize("tensor_cores", [1, 0])
+def test_weight_gradient_on_tensor_cores_and_on_fp32_units(tensor_cores):
+    """dW and db of the one-launch backward, formed either by the split-bf16 tensor-core contraction
+    (three bf16 pieces per fp32 value, six products per term) or by fp32 multiply-adds: both must meet
+    the fp32 bounds against the oracle, on the full-size case with large gradients (several row tiles,
+    a ragged last gate-column tile, several node runs) and on sizes that fill no tile"""
+    rng = np.random.default_rng(151)
+    cases = [(150, 300, 2000, fg.random_forest(rng, 25, 2, 56, 2000), 5, 0.3),
+             (7, 5, 6, fg.forest_from_shapes([fg.random_split_shape(rng, 9), None, fg.left_chain_shape(70)], rng, 6), 3, 0.5)]
+    for H, E, vocab, forest, n_classes, w_scale in cases:
+        params = fg.draw_params(rng, H, E, vocab, emb_dist="normal", emb_scale=0.1, w_scale=w_scale, n_classes=n_classes)
+        forest, _ = fg.permute_node_ids(forest, rng)
+        labels = rng.integers(0, n_classes, size=forest.n_nodes).astype(np.int32)
+        ref = orc.loss_and_gradients(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
+                                     params.Wc, params.bc, labels)
+        model = util.make_model(params, "fp32")
+        model.set_option(binding.OPT_DW_TENSOR_CORES, tensor_cores)
+        res = _train_step(model, forest, labels, binding.PERSISTENT)
+        _compare(res, ref, util.TOL["fp32"])
+
+
+def test_training_step_on_forests_of_single_leaves_and_with_a_large_vocabulary():
+    """no internal node at all (the weight gradient's second part is empty, W_h gets zeros), and a
+    vocabulary beyond what the token scan keeps in shared memory (its ballots are then read again)"""
+    rng = np.random.default_rng(152)
+    vocab = 400_000
+    params = fg.draw_params(rng, 6, 4, vocab, emb_dist="uniform", emb_scale=0.5, w_scale=0.5, n_classes=3)
+    for shapes in ([None, None, None], [fg.random_split_shape(rng, 40), None, fg.left_chain_shape(5)]):
+        forest = fg.forest_from_shapes(shapes, rng, vocab)
+        forest.token[int(np.flatnonzero(forest.left < 0)[0])] = vocab - 1   # the last id of the table is in use
+        labels = rng.integers(0, 3, size=forest.n_nodes).astype(np.int32)
+        ref = orc.loss_and_gradients(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
+                                     params.Wc, params.bc, labels)
+        model = util.make_model(params, "fp32")
+        for flags in (binding.PERSISTENT, binding.PER_LEVEL):
+            res = _train_step(model, forest, labels, flags)
+            _compare(res, ref, util.TOL["fp32"])
