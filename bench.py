@@ -367,8 +367,10 @@ def train_step_time(peaks, flush, steps: int = 200, warmup: int = 5):
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gbs / peaks["hbm_gbs"], "algorithmic_bytes": bytes_, "algorithmic_flops": flops,
                          "fp32_tflops": flops / (mean * 1e-3) / 1e12,
-                         "note": "whole step (forward + backward launches together), fp32 FMA path"},
-            "note": "persistent forward + one-launch backward; the binding reads the status word back after each"}
+                         "note": "whole step (forward + backward launches together); fp32 FMA pipes except the "
+                                 "weight gradient, a split-bf16 tensor-core contraction"},
+            "note": "persistent forward + one-launch backward (wavefronts) + tensor-core dW/db kernel; the binding "
+                    "reads the status word back after each"}
 
 
 def run_sweeps(args):

@@ -130,9 +130,11 @@ typedef enum treelstm_status {
                                             /* order of work of the cooperative launch: their scheduler    */
                                             /* is too short to hide the two extra grid barriers            */
 #define TREELSTM_OPT_DW_TENSOR_CORES 10     /* 1 (default): after a forward that kept its level table on   */
-                                            /* the device, treelstm_backward forms dW and db on the tensor */
-                                            /* cores, every fp32 operand split into three bf16 pieces (six */
-                                            /* products per term: fp32 accuracy); 0: fp32 multiply-adds    */
+                                            /* the device, treelstm_backward forms dW, db and the input    */
+                                            /* gradients of the leaves (dEmb_rows) in a second kernel on   */
+                                            /* the tensor cores, every fp32 operand split into three bf16  */
+                                            /* pieces (six products per term: fp32 accuracy); 0: fp32      */
+                                            /* multiply-adds inside the one-launch backward                */
 
 /*
  * treelstm_create - build a context for one set of parameters.

@@ -779,6 +779,7 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit, int
     if (!fused) {
       for (long long idx = (long long)gtid; idx < elems; idx += (long long)gthreads) gates_element(p, begin, idx, leaf);
       TL_STAMP(trace, lvl, 1);
+      if (leaf && !with_dweight) break;   // the leaves' input gradients are left to the tensor-core kernel as well
       if (!barrier()) return;
     }
     TL_STAMP(trace, lvl, 2);
@@ -819,7 +820,7 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit, int
     TL_STAMP(trace, lvl, 4);
   }
   TL_STAMP(trace, kTraceLevels - 1, 5);   // all wavefronts done
-  if (!with_dweight) return;              // dW and db are left to the tensor-core kernel that follows on the stream
+  if (!with_dweight) return;              // dW, db and the leaves' dIn are left to the tensor-core kernel that follows on the stream
   const int tiles_j = (J + BT - 1) / BT, rows_per_split = kDwRows;
   for (int part = 0; part < 2; ++part) {
     const int begin = part == 0 ? 0 : p.n_leaves, end = part == 0 ? p.n_leaves : n;
@@ -901,7 +902,8 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
     TL_CUDA(ctx, cudaLaunchCooperativeKernel((void*)k_bwd_persistent, dim3(grid), dim3(256), args, smem, stream));
     ctx->launches += 1;
     if (!with_dweight)
-      return launch_dweight_tc(ctx, n, L.order, L.level_offset, L.token, L.left, L.right, L.h, p.dz, dW, db, p.st, stream);
+      return launch_dweight_tc(ctx, n, L.order, L.level_offset, L.token, L.left, L.right, L.h, p.dz, dW, db, p.tok_slot,
+                               dEmb_rows, p.st, stream);
     return TREELSTM_OK;
   }
   TL_CUDA(ctx, cudaMemsetAsync(loss, 0, sizeof(float), stream));

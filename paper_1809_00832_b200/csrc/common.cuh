@@ -230,11 +230,11 @@ int launch_backward(treelstm* ctx, const int32_t* labels, float* loss, float* dW
                     float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,
                     int32_t* n_touched, cudaStream_t stream);
 
-// dweight_tc.cu: dW += In^T dZ, db += sum dZ on the tensor cores (three bf16 pieces per fp32 value)
+// dweight_tc.cu: dW += In^T dZ, db += sum dZ, dEmb_rows += dz_leaves W_x^T on the tensor cores (three bf16 pieces per fp32 value)
 int init_dweight_tc_attributes(treelstm* ctx);
 int launch_dweight_tc(treelstm* ctx, int n, const int32_t* order, const int32_t* level_offset, const int32_t* token,
                       const int32_t* left, const int32_t* right, const float* h, const float* dz, float* dW, float* db,
-                      DevStatus* st, cudaStream_t stream);
+                      const int* tok_slot, float* dEmb_rows, DevStatus* st, cudaStream_t stream);
 
 // Checked build: clears the per-row write counters before a forward / compares them after it
 // (schedule.cu); both do nothing in the normal build.  Counters: [h per node | Ain per position | Cin per position].

@@ -40,8 +40,9 @@ struct DwParams {
   int run;                      // 64-node blocks per work item
   const int *order, *token, *left, *right;
   const int* level_offset;      // level_offset[1] = number of leaves (the host may not know it)
-  const float *emb, *h, *dz;
-  float *dW, *db;
+  const float *emb, *h, *dz, *W;
+  const int* tok_slot;          // row of every token in dEmb_rows (third kind of work item only)
+  float *dW, *db, *dEmb_rows;   // dEmb_rows == nullptr: the leaves' input gradients are not formed here
   DevStatus* st;
   long long wait_limit;
 };
@@ -119,10 +120,46 @@ __device__ __forceinline__ void tile_store(const DwParams& p, unsigned char* til
   }
 }
 
+// The third kind of work item, dEmb_rows += dz_leaves W_x^T, contracts over the gate columns, which are
+// contiguous in both operands (a leaf's dz row, a row of W): no transposition, a thread takes eight
+// consecutive columns of one row - one 16-byte piece - for four rows.  row_ptr(r): start of tile row r in
+// global memory or nullptr; j0: first column of the block; J: columns in a row.
+template <class RowFn>
+__device__ __forceinline__ void rows_load(RowFn row_ptr, int j0, int J, float (&v)[4][8]) {
+  const int c = threadIdx.x & 7;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float* row = row_ptr((threadIdx.x >> 3) + 32 * i);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[i][e] = row[min(j0 + 8 * c + e, J - 1)];
+  }
+}
+__device__ __forceinline__ void rows_store(unsigned char* tile, int rows_valid, int j0, int J, const float (&v)[4][8]) {
+  const int c = threadIdx.x & 7;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = (threadIdx.x >> 3) + 32 * i;
+    uint32_t w0[4], w1[4], w2[4];
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) {
+      const float x = r < rows_valid && j0 + 8 * c + e < J ? v[i][e] : 0.f;
+      const float y = r < rows_valid && j0 + 8 * c + e + 1 < J ? v[i][e + 1] : 0.f;
+      split3_pair(x, y, w0[e >> 1], w1[e >> 1], w2[e >> 1]);
+    }
+    unsigned char* dst = tile + swz_piece(r, c);
+    *reinterpret_cast<uint4*>(dst) = make_uint4(w0[0], w0[1], w0[2], w0[3]);
+    *reinterpret_cast<uint4*>(dst + kDwTileBytes) = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+    *reinterpret_cast<uint4*>(dst + 2 * kDwTileBytes) = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+  }
+}
+
 struct DwShape {
-  int rows[2], nodes[2], first_pos[2], m_tiles[2], runs[2], items[2], n_tiles;
+  int rows[2], nodes[2], first_pos[2], m_tiles[2], runs[2], items[3], n_tiles;
+  // third kind (input gradients of the leaves): tiles of 128 leaves x 128 embedding units, contraction over
+  // the 64-column blocks of the gate columns that are not all forget gates (those are zero for a leaf)
+  int leaf_tiles, e_tiles, kblocks, skip_first, skip_count, runs2;
 };
-__host__ __device__ inline DwShape dw_shape(int n, int n_leaves, int H, int E, int run) {
+__host__ __device__ inline DwShape dw_shape(int n, int n_leaves, int H, int E, int run, bool leaf_dinput) {
   DwShape s;
   s.rows[0] = E; s.rows[1] = 2 * H;
   s.nodes[0] = n_leaves; s.nodes[1] = n - n_leaves;
@@ -134,7 +171,25 @@ __host__ __device__ inline DwShape dw_shape(int n, int n_leaves, int H, int E, i
     s.runs[q] = (blocks + run - 1) / run;
     s.items[q] = s.m_tiles[q] * s.n_tiles * s.runs[q];
   }
+  const int all = (5 * H + kDwBlock - 1) / kDwBlock;
+  s.skip_first = (H + kDwBlock - 1) / kDwBlock;              // first block that starts inside [H, 3H)
+  const int skip_end = 3 * H / kDwBlock;                     // first block that ends outside it
+  s.skip_count = skip_end > s.skip_first ? skip_end - s.skip_first : 0;
+  s.kblocks = all - s.skip_count;
+  s.leaf_tiles = (n_leaves + kDwTile - 1) / kDwTile;
+  s.e_tiles = (E + kDwTile - 1) / kDwTile;
+  s.runs2 = (s.kblocks + run - 1) / run;
+  s.items[2] = leaf_dinput ? s.leaf_tiles * s.e_tiles * s.runs2 : 0;
   return s;
+}
+// The number of 64-wide blocks per work item: as few as give every CTA of the grid at most one item.
+__host__ __device__ inline int dw_run(int n, int n_leaves, int H, int E, bool leaf_dinput, int ctas) {
+  int run = 1;
+  for (; run < kDwMaxRun; ++run) {
+    const DwShape s = dw_shape(n, n_leaves, H, E, run, leaf_dinput);
+    if (s.items[0] + s.items[1] + s.items[2] <= ctas) break;
+  }
+  return run;
 }
 
 __global__ void __launch_bounds__(kDwThreads, 1) k_bwd_dweight_tc(DwParams p) {
@@ -163,45 +218,76 @@ __global__ void __launch_bounds__(kDwThreads, 1) k_bwd_dweight_tc(DwParams p) {
   const uint32_t tmem_base = s_tmem;
   const int H = p.H, E = p.E, J = 5 * H;
   const int n_leaves = p.st->n_levels > 0 ? min(p.n, max(0, p.level_offset[1])) : 0;
-  const DwShape sh = dw_shape(p.n, n_leaves, H, E, p.run);
+  const bool leaf_dinput = p.dEmb_rows != nullptr;
+  const int run = dw_run(p.n, n_leaves, H, E, leaf_dinput, (int)gridDim.x);   // the host does not know the number of leaves
+  const DwShape sh = dw_shape(p.n, n_leaves, H, E, run, leaf_dinput);
   const uint32_t idesc = umma_idesc(kDwTile);
   uint32_t built = 0, items_done = 0;   // blocks built / items finished by this CTA so far (barrier phases)
   bool failed = false;
-  for (int item = blockIdx.x; item < sh.items[0] + sh.items[1] && !failed; item += gridDim.x) {
-    const int part = item < sh.items[0] ? 0 : 1;
-    int it = item - (part ? sh.items[0] : 0);
-    const int nt = it % sh.n_tiles; it /= sh.n_tiles;
-    const int mt = it % sh.m_tiles[part], ri = it / sh.m_tiles[part];
-    const int m0 = mt * kDwTile, j0 = nt * kDwTile;
-    const int pos0 = sh.first_pos[part] + ri * p.run * kDwBlock;
-    const int pos_end = min(sh.first_pos[part] + sh.nodes[part], pos0 + p.run * kDwBlock);
-    const int nblk = (pos_end - pos0 + kDwBlock - 1) / kDwBlock;
-    // the item's nodes and where their input rows come from
-    for (int t = tid; t < nblk * kDwBlock; t += kDwThreads) {
-      int node = 0, ia = 0, ib = 0;
-      if (pos0 + t < pos_end) {
-        node = chk(p.st, p.order[pos0 + t], p.n);
-        if (part == 0) ia = chk(p.st, p.token[node], p.vocab);
-        else { ia = chk(p.st, p.left[node], p.n); ib = chk(p.st, p.right[node], p.n); }
+  for (int item = blockIdx.x; item < sh.items[0] + sh.items[1] + sh.items[2] && !failed; item += gridDim.x) {
+    const int part = item < sh.items[0] ? 0 : (item < sh.items[0] + sh.items[1] ? 1 : 2);
+    int it = item - (part > 0 ? sh.items[0] : 0) - (part > 1 ? sh.items[1] : 0);
+    int m0, j0, pos0 = 0, pos_end = 0, nblk, kb0 = 0, rows_here = 0;
+    if (part < 2) {
+      const int nt = it % sh.n_tiles; it /= sh.n_tiles;
+      const int mt = it % sh.m_tiles[part], ri = it / sh.m_tiles[part];
+      m0 = mt * kDwTile; j0 = nt * kDwTile;
+      pos0 = sh.first_pos[part] + ri * run * kDwBlock;
+      pos_end = min(sh.first_pos[part] + sh.nodes[part], pos0 + run * kDwBlock);
+      nblk = (pos_end - pos0 + kDwBlock - 1) / kDwBlock;
+      // the item's nodes and where their input rows come from
+      for (int t = tid; t < nblk * kDwBlock; t += kDwThreads) {
+        int node = 0, ia = 0, ib = 0;
+        if (pos0 + t < pos_end) {
+          node = chk(p.st, p.order[pos0 + t], p.n);
+          if (part == 0) ia = chk(p.st, p.token[node], p.vocab);
+          else { ia = chk(p.st, p.left[node], p.n); ib = chk(p.st, p.right[node], p.n); }
+        }
+        s_node[t] = node; s_ia[t] = ia; s_ib[t] = ib;
       }
-      s_node[t] = node; s_ia[t] = ia; s_ib[t] = ib;
+    } else {
+      const int et = it % sh.e_tiles; it /= sh.e_tiles;
+      const int lt = it % sh.leaf_tiles, ri = it / sh.leaf_tiles;
+      m0 = lt * kDwTile;                 // first leaf (position in the ready order: the leaves are wavefront 0)
+      j0 = et * kDwTile;                 // first embedding unit
+      rows_here = min(kDwTile, n_leaves - m0);
+      kb0 = ri * run;                    // first of the item's blocks among those that are not skipped
+      nblk = min(run, sh.kblocks - kb0);
+      // the tile's leaves and their rows of dEmb_rows
+      for (int t = tid; t < kDwTile; t += kDwThreads) {
+        int node = 0, slot = 0;
+        if (t < rows_here) {
+          node = chk(p.st, p.order[m0 + t], p.n);
+          slot = chk(p.st, p.tok_slot[chk(p.st, p.token[node], p.vocab)], n_leaves);
+        }
+        s_node[t] = node; s_ia[t] = slot;
+      }
     }
     __syncthreads();
     for (int b = 0; b < nblk; ++b, ++built) {
       const uint32_t stage = built & 1u, use = built >> 1;
       unsigned char* st_tiles = tiles + stage * kDwStageBytes;
       const int valid_nodes = min(kDwBlock, pos_end - pos0 - b * kDwBlock);
+      int kcol = 0;                      // part 2: first gate column of the block
+      if (part == 2) {
+        const int kb = kb0 + b;
+        kcol = (kb < sh.skip_first ? kb : kb + sh.skip_count) * kDwBlock;
+      }
       float va[4][8], vb[4][8];
       if (part == 0) tile_load<0>(p, m0, s_node, s_ia, s_ib, b, va);
-      else tile_load<1>(p, m0, s_node, s_ia, s_ib, b, va);
-      tile_load<2>(p, j0, s_node, s_ia, s_ib, b, vb);
+      else if (part == 1) tile_load<1>(p, m0, s_node, s_ia, s_ib, b, va);
+      else rows_load([&](int r) { return p.dz + (size_t)s_node[r] * J; }, kcol, J, va);
+      if (part < 2) tile_load<2>(p, j0, s_node, s_ia, s_ib, b, vb);
+      else rows_load([&](int r) { return p.W + (size_t)min(j0 + r, E - 1) * J; }, kcol, J, vb);
       bool ok = true;
       if (use >= 1)   // the MMAs that read this stage two blocks ago must have retired before it is overwritten
         ok = mbar_wait(stage_bar0 + 8 * stage, (use - 1) & 1u, &s_abort, p.wait_limit, p.st);
       if (__syncthreads_or(!ok)) { failed = true; break; }
       if (part == 0) tile_store<0>(p, st_tiles, m0, valid_nodes, va);
-      else tile_store<1>(p, st_tiles, m0, valid_nodes, va);
-      tile_store<2>(p, st_tiles + kDwPieces * kDwTileBytes, j0, valid_nodes, vb);
+      else if (part == 1) tile_store<1>(p, st_tiles, m0, valid_nodes, va);
+      else rows_store(st_tiles, rows_here, kcol, J, va);
+      if (part < 2) tile_store<2>(p, st_tiles + kDwPieces * kDwTileBytes, j0, valid_nodes, vb);
+      else rows_store(st_tiles + kDwPieces * kDwTileBytes, min(kDwTile, E - j0), kcol, J, vb);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the tensor core
       tc_fence_before();
       __syncthreads();
@@ -245,10 +331,16 @@ __global__ void __launch_bounds__(kDwThreads, 1) k_bwd_dweight_tc(DwParams p) {
                                                               __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
     }
     __syncthreads();
-    const int rows_valid = min(kDwTile, sh.rows[part] + 1 - m0), cols_valid = min(kDwTile, J - j0);
+    const int rows_valid = part < 2 ? min(kDwTile, sh.rows[part] + 1 - m0) : rows_here;
+    const int cols_valid = part < 2 ? min(kDwTile, J - j0) : min(kDwTile, E - j0);
     for (int r = warp; r < rows_valid; r += kDwThreads / 32) {
-      const int f = m0 + r;
-      float* out = f == sh.rows[part] ? p.db + j0 : p.dW + (size_t)((part ? E : 0) + f) * J + j0;
+      float* out;
+      if (part < 2) {
+        const int f = m0 + r;
+        out = f == sh.rows[part] ? p.db + j0 : p.dW + (size_t)((part ? E : 0) + f) * J + j0;
+      } else {
+        out = p.dEmb_rows + (size_t)s_ia[r] * E + j0;   // leaves with the same token share a row
+      }
 #pragma unroll
       for (int i = 0; i < kDwTile / 32; ++i) {
         const int c = lane + 32 * i;
@@ -278,28 +370,27 @@ int init_dweight_tc_attributes(treelstm* ctx) {
   return TREELSTM_OK;
 }
 
-// dW and db must have been cleared on the stream before; dz holds the gate gradients of every node.
+// dW, db (and dEmb_rows, if given: then tok_slot holds every token's row) must have been cleared on the
+// stream before; dz holds the gate gradients of every node.
 int launch_dweight_tc(treelstm* ctx, int n, const int32_t* order, const int32_t* level_offset, const int32_t* token,
                       const int32_t* left, const int32_t* right, const float* h, const float* dz, float* dW, float* db,
-                      DevStatus* st, cudaStream_t stream) {
+                      const int* tok_slot, float* dEmb_rows, DevStatus* st, cudaStream_t stream) {
   DwParams p;
-  p.n = n; p.n_leaves = 0; p.H = ctx->H; p.E = ctx->E; p.vocab = ctx->vocab;
+  p.n = n; p.n_leaves = 0; p.H = ctx->H; p.E = ctx->E; p.vocab = ctx->vocab; p.run = 0;
   p.order = order; p.level_offset = level_offset; p.token = token; p.left = left; p.right = right;
-  p.emb = ctx->emb; p.h = h; p.dz = dz; p.dW = dW; p.db = db; p.st = st;
+  p.emb = ctx->emb; p.h = h; p.dz = dz; p.W = ctx->W; p.dW = dW; p.db = db; p.st = st;
+  p.tok_slot = tok_slot; p.dEmb_rows = dEmb_rows;
   p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
-  // Blocks per work item: as few as give every SM at most one item.  The host does not know how the nodes
-  // divide into leaves and internal nodes (the level table stayed on the device): it counts one run more than
-  // the nodes need and the larger number of row tiles; CTAs without an item leave at once.
-  const int n_tiles = (5 * p.H + kDwTile - 1) / kDwTile;
-  const int m_tiles = ((p.E > 2 * p.H ? p.E : 2 * p.H) + 1 + kDwTile - 1) / kDwTile;
-  const int blocks = (n + kDwBlock - 1) / kDwBlock;
-  int run = 1, items = 0;
-  for (;; ++run) {
-    items = n_tiles * m_tiles * ((blocks + run - 1) / run + 1);
-    if (items <= ctx->sm_count || run == kDwMaxRun) break;
-  }
-  p.run = run;
   if (n == 0) return TREELSTM_OK;
+  // The host does not know how the nodes divide into leaves and internal nodes (the level table stayed on the
+  // device), so the kernel sizes its work items itself from the grid it finds: one CTA per SM unless even
+  // single-block items are fewer (counted for the division that gives the most).
+  int items = 0;
+  for (int nl = 0; nl <= n; nl += (n > 8 ? n / 8 : 1)) {
+    const DwShape s = dw_shape(n, nl, p.H, p.E, 1, dEmb_rows != nullptr);
+    const int c = s.items[0] + s.items[1] + s.items[2];
+    if (c > items) items = c;
+  }
   const int grid = items < ctx->sm_count ? items : ctx->sm_count;
   k_bwd_dweight_tc<<<grid, kDwThreads, kDwSmemBytes, stream>>>(p);
   TL_CUDA(ctx, cudaGetLastError());
