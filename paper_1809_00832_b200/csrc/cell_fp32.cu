@@ -28,13 +28,16 @@ struct FwdParams {
   long long wait_limit;
   int w_stationary, a_row, w_row;   // persistent kernel: W_h slice resident in shared memory; row strides (floats)
   int early_start = 0;              // persistent kernel: launched under the scheduler, waits for it on the device
+  long long* trace = nullptr;       // cycle stamps of the persistent kernel (trace builds), else nullptr
 };
 
 __device__ __forceinline__ float sigmoidf_acc(float x) { return 1.0f / (1.0f + expf(-x)); }
 
+constexpr int kChunkRow = KC + 4;   // floats per shared-memory row of a chunk: 16-byte reads along the contraction,
+                                    // consecutive rows 4 banks apart (eight rows cover all banks)
 struct TileSmem {
-  float A[2][TM][KC + 1];
-  float W[2][KC][5 * TU];
+  __align__(16) float A[2][TM][kChunkRow];
+  __align__(16) float W[2][5 * TU][kChunkRow];   // transposed: one row per gate column
   int node[TM], l[TM], r[TM];
 };
 
@@ -51,7 +54,8 @@ __host__ __device__ inline int rows_per_tile(int rows, int tiles_u, int n_sms) {
 // memory (two buffers, one CTA barrier per chunk).
 template <int TM>
 __device__ void fp32_tile(const FwdParams& p, int row0, int row_end, int u0, bool leaf,
-                          TileSmem& s) {
+                          TileSmem& s, long long* trace = nullptr, int lvl = 0) {
+  (void)trace; (void)lvl;
   constexpr int RPT = TM / (kThreads / TU);          // rows per thread: 4 or 1
   constexpr int kALoads = TM * KC / kThreads;        // operand elements per thread and chunk: 8 or 2
   const int tid = threadIdx.x, tx = tid % TU, ty = tid / TU;
@@ -76,66 +80,79 @@ __device__ void fp32_tile(const FwdParams& p, int row0, int row_end, int u0, boo
     for (int g = 0; g < 5; ++g) acc[i][g] = 0.f;
 
   float ra[kALoads], rw[kWLoads];
+  // All loads of a chunk without a branch (indices clamped onto valid elements, values discarded afterwards),
+  // so that they are in flight together: a load behind a branch waits for the one before it.
   auto fetch = [&](int k0) {
+    if (leaf) {
+#pragma unroll
+      for (int j = 0; j < kALoads; ++j) {
+        const int e = tid + j * kThreads, i = e / KC, k = min(k0 + e % KC, K - 1);
+        ra[j] = __ldg(p.emb + (size_t)s.l[i] * E + k);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < kALoads; ++j) {
+        const int e = tid + j * kThreads, i = e / KC, k = min(k0 + e % KC, K - 1);
+        ra[j] = __ldcg(p.h + (size_t)(k < H ? s.l[i] : s.r[i]) * H + (k < H ? k : k - H));
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kWLoads; ++j) {
+      const int e = tid + j * kThreads, kk = e / (5 * TU), g = (e % (5 * TU)) / TU, uu = e % TU;
+      rw[j] = __ldg(Wk + (size_t)min(k0 + kk, K - 1) * 5 * H + g * H + min(u0 + uu, H - 1));
+    }
+  };
+  // (what the clamped loads brought for elements outside the tile is replaced by zeros here, not in fetch: a
+  // use of the loaded values right behind the loads would make the multiply-adds of the current chunk wait)
+  auto stash = [&](int buf, int k0) {
 #pragma unroll
     for (int j = 0; j < kALoads; ++j) {
       const int e = tid + j * kThreads, i = e / KC, k = k0 + e % KC;
-      float v = 0.f;
-      if (s.node[i] >= 0 && k < K) {
-        if (leaf) v = __ldg(p.emb + (size_t)s.l[i] * E + k);
-        else v = k < H ? __ldcg(p.h + (size_t)s.l[i] * H + k) : __ldcg(p.h + (size_t)s.r[i] * H + (k - H));
-      }
-      ra[j] = v;
+      s.A[buf][i][e % KC] = (s.node[i] < 0 || k >= K) ? 0.f : ra[j];
     }
 #pragma unroll
     for (int j = 0; j < kWLoads; ++j) {
-      const int e = tid + j * kThreads, kk = e / (5 * TU), g = (e % (5 * TU)) / TU, uu = e % TU, k = k0 + kk;
-      float v = 0.f;
-      if (k < K && u0 + uu < H && !(leaf && (g == 1 || g == 2)))
-        v = __ldg(Wk + (size_t)k * 5 * H + g * H + u0 + uu);
-      rw[j] = v;
+      const int e = tid + j * kThreads, kk = e / (5 * TU), g = (e % (5 * TU)) / TU, uu = e % TU;
+      s.W[buf][e % (5 * TU)][kk] = (k0 + kk >= K || u0 + uu >= H || (leaf && (g == 1 || g == 2))) ? 0.f : rw[j];
     }
   };
-  auto stash = [&](int buf) {
+  // the bias is asked for now and arrives while the contraction runs
+  const int u = u0 + tx;
+  float bias[5];
 #pragma unroll
-    for (int j = 0; j < kALoads; ++j) {
-      const int e = tid + j * kThreads;
-      s.A[buf][e / KC][e % KC] = ra[j];
-    }
-#pragma unroll
-    for (int j = 0; j < kWLoads; ++j) {
-      const int e = tid + j * kThreads;
-      s.W[buf][e / (5 * TU)][e % (5 * TU)] = rw[j];
-    }
-  };
+  for (int g = 0; g < 5; ++g) bias[g] = __ldg(p.b + g * H + min(u, H - 1));
+  TL_STAMP(trace, lvl, 3);   // row ids resolved
   fetch(0);
-  stash(0);
+  stash(0, 0);
   __syncthreads();
+  TL_STAMP(trace, lvl, 4);   // first chunk in shared memory
   const int chunks = (K + KC - 1) / KC;
   for (int cidx = 0; cidx < chunks; ++cidx) {
     const int buf = cidx & 1;
     if (cidx + 1 < chunks) fetch((cidx + 1) * KC);
 #pragma unroll
-    for (int kk = 0; kk < KC; ++kk) {
-      float a[RPT], w[5];
+    for (int kk = 0; kk < KC; kk += 4) {
+      float4 a[RPT], w[5];
 #pragma unroll
-      for (int i = 0; i < RPT; ++i) a[i] = s.A[buf][ty * RPT + i][kk];
+      for (int i = 0; i < RPT; ++i) a[i] = *reinterpret_cast<const float4*>(&s.A[buf][ty * RPT + i][kk]);
 #pragma unroll
-      for (int g = 0; g < 5; ++g) w[g] = s.W[buf][kk][g * TU + tx];
+      for (int g = 0; g < 5; ++g) w[g] = *reinterpret_cast<const float4*>(&s.W[buf][g * TU + tx][kk]);
 #pragma unroll
       for (int i = 0; i < RPT; ++i)
 #pragma unroll
-        for (int g = 0; g < 5; ++g) acc[i][g] = fmaf(a[i], w[g], acc[i][g]);
+        for (int g = 0; g < 5; ++g) {
+          acc[i][g] = fmaf(a[i].x, w[g].x, acc[i][g]);
+          acc[i][g] = fmaf(a[i].y, w[g].y, acc[i][g]);
+          acc[i][g] = fmaf(a[i].z, w[g].z, acc[i][g]);
+          acc[i][g] = fmaf(a[i].w, w[g].w, acc[i][g]);
+        }
     }
-    if (cidx + 1 < chunks) stash(buf ^ 1);
+    if (cidx + 1 < chunks) stash(buf ^ 1, (cidx + 1) * KC);
     __syncthreads();
   }
 
-  const int u = u0 + tx;
+  TL_STAMP(trace, lvl, 5);   // contraction done
   if (u >= H) return;
-  float bias[5];
-#pragma unroll
-  for (int g = 0; g < 5; ++g) bias[g] = __ldg(p.b + g * H + u);
 #pragma unroll
   for (int i = 0; i < RPT; ++i) {
     const int ii = ty * RPT + i;
@@ -342,6 +359,11 @@ k_fwd_fp32_persistent(FwdParams p) {
   int* s_r = s_l + TM;
   const int tiles_u = (p.H + TU - 1) / TU;
   const int H = p.H;
+#ifdef TREELSTM_TRACE
+  // first CTA, first thread: row l = wavefront l (slot 0 start, 1 own tiles done, 2 barrier passed); last row: phases
+  long long* const trace = blockIdx.x == 0 && threadIdx.x == 0 ? p.trace : nullptr;
+#endif
+  TL_STAMP(trace, kTraceLevels - 1, 0);
   // Launched as a programmatic dependent of the ready-set construction (p.early_start), the kernel
   // gets here while that one still runs: the weight slice needs nothing from it and is fetched first.
   int n_levels = 0;
@@ -361,11 +383,35 @@ k_fwd_fp32_persistent(FwdParams p) {
       Ws[col * w_row + k] = v;
     }
   }
+  {
+    // The leaf wavefront streams W_x and the leaves' embedding rows chunk by chunk, one dependent fetch per
+    // chunk: asked into L2 now (which nodes are leaves and their tokens are the caller's arrays, readable
+    // before the schedule exists; tokens are clamped, nothing has been validated yet), those fetches find
+    // them there instead of in DRAM.
+    const size_t gthread = (size_t)blockIdx.x * kThreads + threadIdx.x, gthreads = (size_t)gridDim.x * kThreads;
+    const char* wx = reinterpret_cast<const char*>(p.W);
+    const size_t wx_bytes = sizeof(float) * (size_t)p.E * 5 * H;
+    for (size_t off = gthread * 128; off < wx_bytes; off += gthreads * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(wx + off));
+    const int lane = threadIdx.x & 31;
+    const int row_lines = (int)((sizeof(float) * (size_t)p.E + 127) / 128) + 1;   // + 1: rows do not start on a line
+    for (int node = (int)(gthread >> 5); node < p.n; node += (int)(gthreads >> 5)) {
+      if (p.left[node] >= 0) continue;
+      const int tok = min(max(p.token[node], 0), p.vocab - 1);
+      const char* row = reinterpret_cast<const char*>(p.emb + (size_t)tok * p.E);
+      for (int l = lane; l < row_lines; l += 32) {
+        const char* q = row + (size_t)l * 128;
+        if (q < row + sizeof(float) * (size_t)p.E) asm volatile("prefetch.global.L2 [%0];" ::"l"(q));
+      }
+    }
+  }
+  TL_STAMP(trace, kTraceLevels - 1, 1);   // weight slice requested (own part stored)
   if (p.early_start) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (ld_volatile(&p.st->status) != 0) return;
     n_levels = p.st->n_levels;
   }
+  TL_STAMP(trace, kTraceLevels - 1, 2);   // schedule there
   // the first wavefront boundaries in shared memory: no dependent global load after every barrier
   constexpr int kOffCache = 256;
   __shared__ int s_off[kOffCache];
@@ -377,6 +423,7 @@ k_fwd_fp32_persistent(FwdParams p) {
     const int begin = level_begin(lvl), end = level_begin(lvl + 1);
     const int tmr = rows_per_tile(end - begin, tiles_u, p.n_sms);
     const int tiles = ((end - begin + tmr - 1) / tmr) * tiles_u;
+    TL_STAMP(trace, lvl, 0);
     for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
       const int tm = t / tiles_u, u0 = (t - tm * tiles_u) * TU;
       if (lvl > 0 && p.w_stationary) {
@@ -384,10 +431,16 @@ k_fwd_fp32_persistent(FwdParams p) {
         if (tmr == TM) fp32_tile_stationary<TM>(p, begin + tm * TM, end, u0, As, Ws, red, s_node, s_l, s_r, ready);
         else fp32_tile_stationary<TMS>(p, begin + tm * TMS, end, u0, As, Ws, red, s_node, s_l, s_r, ready);
       } else {
+#ifdef TREELSTM_TRACE
+        if (tmr == TM) fp32_tile<TM>(p, begin + tm * TM, end, u0, lvl == 0, s, trace, lvl);
+        else fp32_tile<TMS>(p, begin + tm * TMS, end, u0, lvl == 0, s, trace, lvl);
+#else
         if (tmr == TM) fp32_tile<TM>(p, begin + tm * TM, end, u0, lvl == 0, s);
         else fp32_tile<TMS>(p, begin + tm * TMS, end, u0, lvl == 0, s);
+#endif
       }
     }
+    TL_STAMP(trace, lvl, 1);
     if (lvl + 1 < n_levels) {
       // Which rows the next wavefront holds and who their children are is the scheduler's output and
       // does not depend on the wavefront just finished: threads outside the polling warp fetch the
@@ -412,6 +465,7 @@ k_fwd_fp32_persistent(FwdParams p) {
             s_node[i] = node; s_l[i] = l; s_r[i] = r;
           });
       if (!passed) return;
+      TL_STAMP(trace, lvl, 2);
       ids_ahead = p.w_stationary != 0;
     }
   }
@@ -436,6 +490,11 @@ int launch_forward_fp32(treelstm* ctx, int n, const int32_t* left, const int32_t
   p.st = reinterpret_cast<DevStatus*>(base + lay.status);
   p.wait_limit = ctx->opt.wait_limit_kcycles * 1024;
   p.w_stationary = 0; p.a_row = 0; p.w_row = 0;
+#ifdef TREELSTM_TRACE
+  p.trace = reinterpret_cast<long long*>(base + lay.trace) + kTraceSlots * kTraceLevels;   // second table: the backward clears the first
+  if (flags & TREELSTM_PERSISTENT)
+    TL_CUDA(ctx, cudaMemsetAsync(p.trace, 0, sizeof(long long) * kTraceSlots * kTraceLevels, stream));
+#endif
   const int tiles_u = (ctx->H + TU - 1) / TU;
   if (flags & TREELSTM_PERSISTENT) {
     // Resident W_h slice: 80 rows of w_row floats (w_row = 4 mod 32, so that the float4 reads of the

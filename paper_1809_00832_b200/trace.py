@@ -70,6 +70,14 @@ def trace_training_step() -> int:
         model.backward(labels, f.n_leaves)
     torch.cuda.synchronize()
     widths = np.diff(out["level_offset"].cpu().numpy()[:int(out["n_levels"].item()) + 1])
+    tf = read_trace(model, 1)
+    phf = tf[LEVELS - 1]
+    print(f"# fp32 persistent forward, first CTA, cycles since its start: weight slice fetched {int(phf[1] - phf[0])}, "
+          f"schedule there {int(phf[2] - phf[0])}, last stamp {int(tf[:LEVELS - 1].max() - phf[0])}")
+    print("level width tiles_done barrier_passed ids_resolved first_chunk contracted   (cycles since the wavefront's start; the last three: streaming tiles only)")
+    for l in range(len(widths)):
+        if tf[l, 0]:
+            print(f"{l:<5d} {int(widths[l]):<5d} " + " ".join(f"{(tf[l, k] - tf[l, 0]) if tf[l, k] else 0:<10d}" for k in (1, 2, 3, 4, 5)))
     t = read_trace(model, 0)
     ph = t[LEVELS - 1]
     names = ("outputs and scratch cleared", "tokens marked", "own part of token scan / classifier done",
