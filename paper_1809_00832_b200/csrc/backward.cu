@@ -276,20 +276,23 @@ __device__ void dinput_block(const BwdParams& p, int row_begin, int row_end, int
   __syncthreads();
   float acc[4][4] = {};
   float ra[kLd], rb[kLd];
+  // Loads without a branch (rows and columns outside the block clamped onto valid ones); what they brought for
+  // elements outside is replaced by zeros at the store - a use right behind the loads would make the
+  // multiply-adds of the current chunk wait for them.
   auto fetch = [&](int j0) {
 #pragma unroll
     for (int q = 0; q < kLd; ++q) {
-      const int e = tid + q * 256, i = e / BK, j = j0 + e % BK;
-      ra[q] = (s_node[i] >= 0 && j < J) ? p.dz[(size_t)s_node[i] * J + j] : 0.f;
-      rb[q] = (k0 + i < K && j < J) ? __ldg(p.W + (size_t)(koff + k0 + i) * J + j) : 0.f;
+      const int e = tid + q * 256, i = e / BK, j = min(j0 + e % BK, J - 1);
+      ra[q] = p.dz[(size_t)max(s_node[i], 0) * J + j];
+      rb[q] = __ldg(p.W + (size_t)(koff + min(k0 + i, K - 1)) * J + j);
     }
   };
-  auto stash = [&](int buf) {
+  auto stash = [&](int buf, int j0) {
 #pragma unroll
     for (int q = 0; q < kLd; ++q) {
-      const int e = tid + q * 256;
-      As[buf][e / BK][e % BK] = ra[q];
-      Bs[buf][e / BK][e % BK] = rb[q];
+      const int e = tid + q * 256, i = e / BK, j = j0 + e % BK;
+      As[buf][i][e % BK] = (s_node[i] >= 0 && j < J) ? ra[q] : 0.f;
+      Bs[buf][i][e % BK] = (k0 + i < K && j < J) ? rb[q] : 0.f;
     }
   };
   // gridDim.y CTAs share the contraction: each takes a contiguous run of chunks and adds its
@@ -300,7 +303,7 @@ __device__ void dinput_block(const BwdParams& p, int row_begin, int row_end, int
   const int c_lo = by * per_split, chunks = min(chunks_all, c_lo + per_split);
   if (c_lo >= chunks) return;
   fetch(c_lo * BK);
-  stash(c_lo & 1);
+  stash(c_lo & 1, c_lo * BK);
   __syncthreads();
   for (int cidx = c_lo; cidx < chunks; ++cidx) {
     const int buf = cidx & 1;
@@ -323,7 +326,7 @@ __device__ void dinput_block(const BwdParams& p, int row_begin, int row_end, int
           acc[i][q] = fmaf(a[i].w, b[q].w, acc[i][q]);
         }
     }
-    if (cidx + 1 < chunks) stash(buf ^ 1);
+    if (cidx + 1 < chunks) stash(buf ^ 1, (cidx + 1) * BK);
     __syncthreads();
   }
 #pragma unroll
