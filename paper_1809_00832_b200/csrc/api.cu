@@ -36,7 +36,8 @@ WsLayout ws_layout(const treelstm* ctx, int n, bool with_backward) {
     L.dh = take(4 * nn * H);
     L.dc = take(4 * nn * H);
     L.dz = take(4 * nn * 5 * H);
-    L.tok_slot = take(4 * ((size_t)ctx->vocab + 4));   // vocab + 1 entries in use; the scan reads whole quads
+    L.tok_slot = take(4 * ((size_t)ctx->vocab + 4 + ((size_t)ctx->vocab + 127) / 128));   // vocab + 1 entries in use, the scan
+                                                                   // reads whole quads; then one count per 128 ids
   }
   L.trace = off;
 #ifdef TREELSTM_TRACE

@@ -126,6 +126,54 @@ __device__ void scan_tokens(const BwdParams& p, unsigned int* s_mask, int mask_c
   }
   if (warp == nw - 1 && lane == 0) { *p.n_touched = base; p.st->n_touched = base; }
 }
+// The same scan spread over the CTAs of the one-launch backward, in two steps with a grid barrier between
+// them: scan_count_groups writes the number of flagged ids of every 128-id group to group_count[], then
+// scan_place_groups sums the counts before a group and places its ids.  Group g belongs to warp 0 of CTA
+// gridDim.x - 1 - g % gridDim.x: the high-numbered CTAs, which have no block in a narrow wavefront, so that
+// the second step runs beside the first wavefronts instead of ahead of them.
+__device__ __forceinline__ void scan_count_groups(const BwdParams& p, int* group_count) {
+  if (threadIdx.x >= 32) return;
+  const int lane = threadIdx.x, n_groups = (p.vocab + 127) / 128;
+  for (int g = (int)(gridDim.x - 1 - blockIdx.x); g < n_groups; g += (int)gridDim.x) {
+    const int4 v = load_flags4(p, g * 128 + 4 * lane, true);
+    const int c = __popc(__ballot_sync(kFull, v.x != 0)) + __popc(__ballot_sync(kFull, v.y != 0)) +
+                  __popc(__ballot_sync(kFull, v.z != 0)) + __popc(__ballot_sync(kFull, v.w != 0));
+    if (lane == 0) group_count[g] = c;
+  }
+}
+__device__ __forceinline__ void scan_place_groups(const BwdParams& p, const int* group_count) {
+  if (threadIdx.x >= 32) return;
+  const int lane = threadIdx.x, n_groups = (p.vocab + 127) / 128;
+  const unsigned int below = (1u << lane) - 1u;
+  for (int g = (int)(gridDim.x - 1 - blockIdx.x); g < n_groups; g += (int)gridDim.x) {
+    const int id = g * 128 + 4 * lane;
+    const int4 v = load_flags4(p, id, true);          // the group's flags: nobody else touches them
+    int base = 0;
+    for (int q = lane; q < g; q += 32) base += group_count[q];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) base += __shfl_xor_sync(kFull, base, d);
+    const unsigned int m0 = __ballot_sync(kFull, v.x != 0), m1 = __ballot_sync(kFull, v.y != 0);
+    const unsigned int m2 = __ballot_sync(kFull, v.z != 0), m3 = __ballot_sync(kFull, v.w != 0);
+    const int f0 = (m0 >> lane) & 1u, f1 = (m1 >> lane) & 1u, f2 = (m2 >> lane) & 1u, f3 = (m3 >> lane) & 1u;
+    const int e0 = base + __popc(m0 & below) + __popc(m1 & below) + __popc(m2 & below) + __popc(m3 & below);
+    const int e1 = e0 + f0, e2 = e1 + f1, e3 = e2 + f2;
+    if (id + 3 < p.vocab) {
+      *reinterpret_cast<int4*>(p.tok_slot + id) = make_int4(e0, e1, e2, e3);
+    } else {
+      if (id < p.vocab) p.tok_slot[id] = e0;
+      if (id + 1 < p.vocab) p.tok_slot[id + 1] = e1;
+      if (id + 2 < p.vocab) p.tok_slot[id + 2] = e2;
+    }
+    if (f0) p.touched_ids[e0] = id;
+    if (f1) p.touched_ids[e1] = id + 1;
+    if (f2) p.touched_ids[e2] = id + 2;
+    if (f3) p.touched_ids[e3] = id + 3;
+    if (g == n_groups - 1 && lane == 0) {
+      const int total = base + __popc(m0) + __popc(m1) + __popc(m2) + __popc(m3);
+      *p.n_touched = total; p.st->n_touched = total;
+    }
+  }
+}
 constexpr int kScanMaskWords = 8192;
 __global__ void __launch_bounds__(1024) k_bwd_scan_tokens(BwdParams p) {
   __shared__ __align__(16) unsigned int s_mask[kScanMaskWords];
@@ -156,13 +204,15 @@ __device__ void classifier_groups(const BwdParams& p, int vb_first, int vb_step,
     const int node = node0 + q;
     if (node >= p.n) break;
     const float* hn = p.h + (size_t)node * H;
+    const int y = p.labels[node];                       // asked for now: they arrive with the first h values
+    const float my_bias = lane < C ? __ldg(p.bc + lane) : 0.f;
     float logit = -INFINITY;
     for (int k = 0; k < C; ++k) {
       float part = 0.f;
       for (int j = lane; j < H; j += 32) part = fmaf(hn[j], __ldg(p.Wc + j * C + k), part);
 #pragma unroll
       for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(kFull, part, d);
-      if (lane == k) logit = part + p.bc[k];
+      if (lane == k) logit = part + my_bias;
     }
     float m = logit;
 #pragma unroll
@@ -170,7 +220,6 @@ __device__ void classifier_groups(const BwdParams& p, int vb_first, int vb_step,
     float e = lane < C ? expf(logit - m) : 0.f, sum = e;
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(kFull, sum, d);
-    const int y = p.labels[node];
     const bool y_ok = y >= 0 && y < C;
     if (!y_ok && lane == 0) report(p.st, TREELSTM_ERR_LABEL_OUT_OF_RANGE);
     const float lse = m + logf(sum);
@@ -737,17 +786,18 @@ k_bwd_persistent(BwdParams p, const int* level_offset, long long wait_limit, int
   // (the CTA's operand buffers are idle in this phase: they hold the scan's ballots)
   unsigned int* const s_mask = reinterpret_cast<unsigned int*>(s_dyn4);
   const int mask_cap = (int)(sizeof(BwdSmem) / sizeof(unsigned int));
+  int* const group_count = p.tok_slot + p.vocab + 4;   // behind the table and its spare entries
   if (gridDim.x == 1) {
     scan_tokens(p, s_mask, mask_cap);
     classifier_groups(p, 0, 1, s_cls);
-  } else if (blockIdx.x == 0) {
-    scan_tokens(p, s_mask, mask_cap);
   } else {
-    classifier_groups(p, blockIdx.x - 1, gridDim.x - 1, s_cls);
+    scan_count_groups(p, group_count);
+    classifier_groups(p, blockIdx.x, gridDim.x, s_cls);
   }
   TL_STAMP(trace, kTraceLevels - 1, 3);   // this CTA's part (the first one: the token scan) done
   if (!barrier()) return;
   TL_STAMP(trace, kTraceLevels - 1, 4);   // classifier, loss and token scan done everywhere
+  if (gridDim.x > 1) scan_place_groups(p, group_count);   // needs nothing but the counts; its results are read after the kernel
   // the first wavefront boundaries in shared memory: no dependent global load after every barrier
   // (filled here, ordered before its first use by the CTA barriers inside the grid barrier above)
   constexpr int kOffCache = 256;
