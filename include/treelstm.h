@@ -253,11 +253,13 @@ TREELSTM_API int treelstm_roots(treelstm_t* ctx, int max_roots, int32_t* root_id
  *                summed gradient row per touched id (duplicates accumulate); n_touched [1] out.
  *                Rows past n_touched are unspecified.
  * The forest arrays, h, c, order, level and the workspace of the forward call must still be
- * valid and unchanged.  After a TREELSTM_PERSISTENT or TREELSTM_SUBFORESTS forward the whole pass
- * is one cooperative launch that reads the level table on the device (asynchronous, no host round
- * trip; a label out of range is reported by treelstm_status_sync); after a TREELSTM_PER_LEVEL
- * forward it is one launch pair per wavefront, driven by the level table the forward already read
- * back.  Computes in fp32 from the fp32 parameters whatever the forward precision.
+ * valid and unchanged.  After a TREELSTM_PERSISTENT or TREELSTM_SUBFORESTS forward the loss and all
+ * wavefronts are one cooperative launch that reads the level table on the device (asynchronous, no
+ * host round trip; a label out of range is reported by treelstm_status_sync), followed - unless
+ * TREELSTM_OPT_DW_TENSOR_CORES is 0 - by one tensor-core launch for dW, db and dEmb_rows (their sums
+ * run over all nodes and depend on no wavefront order); after a TREELSTM_PER_LEVEL forward it is one
+ * launch pair per wavefront, driven by the level table the forward already read back.  Computes at
+ * fp32 accuracy from the fp32 parameters whatever the forward precision.
  */
 TREELSTM_API int treelstm_backward(treelstm_t* ctx, const int32_t* labels, float* loss, float* dW, float* db,
                       float* dWc, float* dbc, int32_t* touched_ids, float* dEmb_rows,
