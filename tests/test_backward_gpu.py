@@ -144,3 +144,21 @@ def test_training_step_on_forests_of_single_leaves_and_with_a_large_vocabulary()
         for flags in (binding.PERSISTENT, binding.PER_LEVEL):
             res = _train_step(model, forest, labels, flags)
             _compare(res, ref, util.TOL["fp32"])
+
+
+@pytest.mark.parametrize("ctas", [1, 3, 40])
+def test_training_step_on_small_grids(ctas):
+    """the one-launch backward on a grid of one CTA (token scan and classifier in the same CTA), of a few
+    CTAs (every CTA takes several blocks of a narrow wavefront, only the first of them fetched ahead of
+    the grid barrier) and of fewer CTAs than a narrow wavefront has blocks"""
+    rng = np.random.default_rng(160 + ctas)
+    params = fg.draw_params(rng, 20, 12, 300, emb_dist="normal", emb_scale=0.3, w_scale=0.3, n_classes=4)
+    forest = fg.random_forest(rng, 9, 2, 40, 300)
+    forest, _ = fg.permute_node_ids(forest, rng)
+    labels = rng.integers(0, 4, size=forest.n_nodes).astype(np.int32)
+    ref = orc.loss_and_gradients(forest.left, forest.right, forest.token, params.emb, params.W, params.b,
+                                 params.Wc, params.bc, labels)
+    model = util.make_model(params, "fp32")
+    model.set_option(binding.OPT_MAX_CTAS, ctas)
+    res = _train_step(model, forest, labels, binding.PERSISTENT)
+    _compare(res, ref, util.TOL["fp32"])
